@@ -1,0 +1,283 @@
+"""Pins for the oracle's acceptance rules (O3, O3'): the greedy operator against a literal
+set-comprehension over every input of a tiny case, fixed cases, the Fig. 1 example, exact
+integration of the speculative-sampling rule (losslessness for one branch), and the reuse
+probability of Proposition 1."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+
+from oracle import oracle as O
+from paper_2510_13161_b200.inputs import comb_parent
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def literal_accept_len(draft, target):
+    """Eq. 3 as printed: the largest r in {0..gamma} with draft_j == target_j for all j <= r."""
+    gamma = len(draft)
+    return max(r for r in range(gamma + 1) if all(draft[j] == target[j] for j in range(r)))
+
+
+def test_greedy_rule_exhaustively_on_a_tiny_case():
+    V, kappa, gamma = 3, 2, 2
+    parent = comb_parent(kappa, gamma)           # nodes: 0 | 1,2 | 3,4
+    n = len(parent)
+    toks, ams = [], []
+    for tok in itertools.product(range(V), repeat=n - 1):
+        for am in itertools.product(range(V), repeat=n):
+            toks.append((0,) + tok); ams.append(am)
+    toks = np.array(toks, np.int32); ams = np.array(ams, np.int32)
+    o = O.accept_greedy(toks, ams, parent, gamma)
+    for k in range(len(toks)):
+        tok, am = toks[k], ams[k]
+        lens = []
+        for i in range(kappa):
+            nodes = [1 + i * gamma + j for j in range(gamma)]
+            draft = [tok[c] for c in nodes]
+            target = [am[parent[c]] for c in nodes]      # row of the parent checks the child
+            lens.append(literal_accept_len(draft, target))
+        A = max(lens)
+        best = min(i for i in range(kappa) if lens[i] == A)
+        R = 0 if A == 0 else 1 + best * gamma + A - 1
+        assert o["n_accepted"][k] == A
+        assert o["best_branch"][k] == best
+        assert o["decide_row"][k] == R
+        assert o["n_emitted"][k] == A + 1
+        exp = [tok[1 + best * gamma + j] for j in range(A)] + [am[R]]
+        assert o["emitted"][k, :A + 1].tolist() == exp
+        assert (o["emitted"][k, A + 1:] == -1).all()
+        assert o["accepted_nodes"][k, :A].tolist() == [1 + best * gamma + j for j in range(A)]
+
+
+def test_greedy_fixed_cases():
+    kappa, gamma = 2, 3
+    parent = comb_parent(kappa, gamma)
+    n = len(parent)
+    am = np.array([[5, 6, 7, 8, 1, 1, 1]], np.int32)
+    # all-accept on branch 0: bonus token from the last node's row
+    tok = np.array([[0, 5, 6, 7, 9, 9, 9]], np.int32)
+    o = O.accept_greedy(tok, am, parent, gamma)
+    assert (o["n_accepted"][0], o["best_branch"][0], o["decide_row"][0], o["n_emitted"][0]) == (3, 0, 3, 4)
+    assert o["emitted"][0].tolist() == [5, 6, 7, 8]
+    o = O.accept_greedy(tok, am, parent, gamma, emit_bonus=False)
+    assert o["n_emitted"][0] == 3 and o["emitted"][0].tolist() == [5, 6, 7, -1]
+    # first-token reject everywhere: A = 0, branch 0, correction = argmax of the root row
+    tok = np.array([[0, 4, 6, 7, 4, 1, 1]], np.int32)
+    o = O.accept_greedy(tok, am, parent, gamma)
+    assert (o["n_accepted"][0], o["best_branch"][0], o["decide_row"][0]) == (0, 0, 0)
+    assert o["emitted"][0].tolist() == [5, -1, -1, -1]
+    # two identical branches: the lower index wins
+    am2 = np.array([[5, 6, 0, 0, 6, 0, 0]], np.int32)
+    tok = np.array([[0, 5, 6, 2, 5, 6, 2]], np.int32)
+    o = O.accept_greedy(tok, am2, parent, gamma)
+    assert (o["n_accepted"][0], o["best_branch"][0], o["decide_row"][0]) == (2, 0, 2)
+    # the longer agreement wins even on the higher branch index
+    tok = np.array([[0, 5, 9, 2, 5, 6, 2]], np.int32)
+    o = O.accept_greedy(tok, am2, parent, gamma)
+    assert (o["n_accepted"][0], o["best_branch"][0], o["decide_row"][0]) == (2, 1, 5)
+    assert o["accepted_nodes"][0].tolist() == [4, 5, -1]
+    # a mismatch hides later matches (prefix semantics, not a count of matches)
+    tok = np.array([[0, 4, 6, 7, 4, 1, 1]], np.int32)
+    assert O.accept_greedy(tok, am, parent, gamma)["n_accepted"][0] == 0
+
+
+def read_golden(name):
+    d = {}
+    for line in open(os.path.join(GOLDEN, name)):
+        if line.startswith("#") or ":" not in line:
+            continue
+        k, v = line.split(":", 1)
+        d[k.strip()] = [int(t) for t in v.split()]
+    return d
+
+
+def test_fig1_worked_example():
+    g = read_golden("fig1_example.txt")
+    gamma, kappa = g["gamma"][0], g["kappa"][0]
+    parent = comb_parent(kappa, gamma)
+    tok = np.array([[0] + g["draft_window"]], np.int32)
+    # row r holds the target's token for the position after node r (root row checks the first draft token)
+    am = np.array([g["target_tokens"]], np.int32)
+    for cands, want in ((g["candidates_with_reuse"], g["expected_reuse_slot_with"][0]),
+                        (g["candidates_without_reuse"], g["expected_reuse_slot_without"][0])):
+        cand = np.tile(np.array(cands, np.int32), (1, len(parent), 1))
+        o = O.accept_greedy(tok, am, parent, gamma, cand_ids=cand)
+        assert o["n_accepted"][0] == g["expected_accepted"][0]
+        A = o["n_accepted"][0]
+        assert o["emitted"][0, :A + 1].tolist() == g["expected_emitted"]
+        assert o["emitted"][0, A] == g["expected_correction"][0]
+        assert o["decide_row"][0] == 2          # the correction sits at 0-based depth tau = 2
+        assert o["reuse_slot"][0] == want
+
+
+# ---------------------------------------------------------------------------------------------
+# speculative sampling
+# ---------------------------------------------------------------------------------------------
+def spec_inputs_chain(p_rows, q_rows, xs, u_acc, u_res):
+    """One request: a chain root -> node1 -> ... ; p_rows[r] is row r's target distribution,
+    q_rows[c-1] node c's draft distribution, xs the drafted tokens."""
+    n = len(xs) + 1
+    logits = np.log(np.maximum(np.array(p_rows, np.float64), 1e-300)).astype(np.float32)
+    lse = np.zeros(n, np.float32)
+    return (np.array([0] + list(xs), np.int32), logits, lse, np.array(q_rows, np.float32),
+            np.array(u_acc, np.float32), np.array(u_res, np.float32))
+
+
+def batch_spec(items, parent, gamma, **kw):
+    tok = np.stack([i[0] for i in items]); logits = np.stack([i[1] for i in items]).reshape(-1, items[0][1].shape[-1])
+    lse = np.concatenate([i[2] for i in items]); q = np.stack([i[3] for i in items])
+    ua = np.stack([i[4] for i in items]); ur = np.stack([i[5] for i in items])
+    return O.accept_spec(tok, logits, lse, q, ua, ur, parent, gamma, **kw)
+
+
+def test_spec_rule_is_lossless_for_one_branch_exact_integration():
+    # gamma = 1, kappa = 1, |V| = 4.  p, q are sixteenths; every boundary of the rule (accept
+    # thresholds p/q in {1/4, 1/3}, residual CDF steps in sevenths) lies on a grid edge, so the
+    # midpoint rule integrates the emitted-token law exactly: it must equal p (the speculative
+    # sampling theorem of the works the paper cites for its lossless claim, Sec. 4.1).
+    p = np.array([1, 5, 2, 8]) / 16.0
+    q = np.array([4, 4, 6, 2]) / 16.0
+    Na, Nr = 12, 7
+    parent = comb_parent(1, 1)
+    items, weights = [], []
+    for x in range(4):
+        for a in range(Na):
+            for r in range(Nr):
+                ua, ur = (a + 0.5) / Na, (r + 0.5) / Nr
+                items.append(spec_inputs_chain([p, p], [q], [x], [0.0, ua], [ur, ur]))
+                weights.append(q[x] / (Na * Nr))
+    o = batch_spec(items, parent, 1)
+    w = np.array(weights)
+    law = np.zeros(4)
+    for k in range(len(items)):
+        law[o["emitted"][k, 0]] += w[k]
+    np.testing.assert_allclose(law, p, atol=1e-12)
+    # P[accept] = sum_v min(p_v, q_v)
+    np.testing.assert_allclose((w * (o["n_accepted"] == 1)).sum(), np.minimum(p, q).sum(), atol=1e-12)
+    assert (o["n_emitted"] == o["n_accepted"] + 1).all()
+
+
+def test_spec_rule_two_step_chain_law():
+    # gamma = 2: the first emitted token follows p0; given that the draft's first token v was
+    # accepted, the second emitted token follows the row of that node, p1.
+    V = 4
+    p0 = np.array([1, 5, 2, 8]) / 16.0; q1 = np.array([4, 4, 6, 2]) / 16.0
+    p1 = np.array([6, 2, 7, 1]) / 16.0; q2 = np.array([2, 8, 3, 3]) / 16.0
+    p2 = np.array([3, 3, 5, 5]) / 16.0
+    parent = comb_parent(1, 2)
+    items, weights = [], []
+    # accept thresholds: p0/q1 in {1/4, 1/3}, p1/q2 in {1/4, 1/3}: a 12-cell grid holds them all.
+    # CDF steps: residual of row 0 in 7ths, of row 1 in 8ths, bonus row p2 in 16ths: 112 = lcm(7, 8, 16).
+    sub = [(a + 0.5) / 12 for a in range(12)]
+    res_grid = [(r + 0.5) / 112 for r in range(112)]
+    for x1 in range(V):
+        for x2 in range(V):
+            for ua1 in sub:
+                for ua2 in sub:
+                    for ur in res_grid:
+                        items.append(spec_inputs_chain([p0, p1, p2], [q1, q2], [x1, x2], [0.0, ua1, ua2], [ur, ur, ur]))
+                        weights.append(q1[x1] * q2[x2] / (12 * 12 * 112))
+    o = batch_spec(items, parent, 2)
+    w = np.array(weights)
+    law1 = np.zeros(V); joint = np.zeros((V, V)); law3 = np.zeros(V)
+    for k in range(len(items)):
+        e = o["emitted"][k]
+        law1[e[0]] += w[k]
+        if o["n_accepted"][k] >= 1:
+            joint[e[0], e[1]] += w[k]
+        if o["n_accepted"][k] == 2:
+            law3[e[2]] += w[k]
+    np.testing.assert_allclose(law1, p0, atol=1e-12)
+    acc1 = np.minimum(p0, q1)
+    np.testing.assert_allclose(joint, acc1[:, None] * p1[None, :], atol=1e-12)
+    # all accepted: the bonus token follows the last node's row
+    np.testing.assert_allclose(law3, acc1.sum() * np.minimum(p1, q2).sum() * p2, atol=1e-12)
+
+
+def test_spec_rule_special_cases():
+    parent = comb_parent(1, 1)
+    p = np.array([0.1, 0.2, 0.3, 0.4])
+    # p == q: always accept, whatever u
+    for u in (0.0, 0.5, 0.999999):
+        for x in range(4):
+            o = batch_spec([spec_inputs_chain([p, p], [p], [x], [0, u], [0.3, 0.3])], parent, 1)
+            assert o["n_accepted"][0] == 1 and o["emitted"][0, 0] == x
+    # q one-hot on a token the target gives zero mass: always reject, correction ~ p (residual == p)
+    pz = np.array([0.0, 0.5, 0.25, 0.25]); q = np.array([1.0, 0, 0, 0])
+    cdf = np.cumsum(pz)
+    for ur in (0.01, 0.49, 0.51, 0.74, 0.76, 0.99):
+        o = batch_spec([spec_inputs_chain([pz, pz], [q], [0], [0, 0.5], [ur, ur])], parent, 1)
+        assert o["n_accepted"][0] == 0
+        assert o["emitted"][0, 0] == int(np.searchsorted(cdf, ur, side="right"))
+    # u = 0 accepts anything the target gives positive mass
+    o = batch_spec([spec_inputs_chain([p, p], [np.array([0.97, 0.01, 0.01, 0.01])], [0], [0, 0.0], [0.3, 0.3])], parent, 1)
+    assert o["n_accepted"][0] == 1
+
+
+def test_spec_rule_generic_grid_is_close_to_p():
+    # the same law on values that are not grid-aligned: midpoint integration, tolerance ~ 1/N
+    rng = np.random.default_rng(3)
+    p = rng.dirichlet(np.ones(5)); q = rng.dirichlet(np.ones(5))
+    parent = comb_parent(1, 1)
+    N = 200
+    items, weights = [], []
+    for x in range(5):
+        for a in range(N):
+            for r in range(N):
+                items.append(spec_inputs_chain([p, p], [q], [x], [0, (a + 0.5) / N], [(r + 0.5) / N] * 2))
+                weights.append(q[x] / N / N)
+    o = batch_spec(items, parent, 1)
+    law = np.bincount(o["emitted"][:, 0], weights=np.array(weights), minlength=5)
+    np.testing.assert_allclose(law, p, atol=2.0 / N)
+
+
+def test_spec_temperature_uses_scaled_logits():
+    # with lse given for logits/T, the accept test compares against Softmax(logits/T)
+    parent = comb_parent(1, 1)
+    logits = np.array([[1.0, 2.0, 0.5, -1.0]] * 2, np.float32)
+    T = 2.0
+    pT = np.exp(logits[0] / T); pT /= pT.sum()
+    lse = np.full(2, np.log(np.exp(logits[0].astype(np.float64) / T).sum()), np.float32)
+    q = np.array([[[0.25, 0.25, 0.25, 0.25]]], np.float32)
+    x = 3                                         # p/q = pT[3]/0.25 < 1
+    thr = pT[x] / 0.25
+    for u, want in ((thr * 0.99, 1), (thr * 1.01, 0)):
+        o = O.accept_spec(np.array([[0, x]], np.int32), logits, lse, q, np.array([[0, u]], np.float32),
+                          np.array([[0.5, 0.5]], np.float32), parent, 1, temperature=T)
+        assert o["n_accepted"][0] == want
+
+
+def test_reuse_probability_equals_overlap_mass():
+    # Proposition 1: with A = 0 reuse succeeds iff the target's token is in the early-exit Top-kappa
+    # set, so P[reuse] = Omega_kappa.  A root-only tree draws the token from the root row.
+    rng = np.random.default_rng(5)
+    V = 8
+    final = np.array([3, 1, 4, 1, 5, 9, 2, 7]) / 32.0
+    early_logits = np.log(final)[None] + rng.normal(size=(1, V))
+    N = 32                                       # CDF steps of `final` are 32nds
+    prev = -1.0
+    for kappa in (1, 2, 4, 8):
+        ids = O.row_reduce(early_logits, topk=kappa)["topk_id"][0]
+        omega = O.overlap_mass(final, ids)
+        B = N
+        tok = np.zeros((B, 1), np.int32)
+        logits = np.tile(np.log(final).astype(np.float32), (B, 1))
+        o = O.accept_spec(tok, logits, np.zeros(B, np.float32), np.zeros((B, 0, V), np.float32),
+                          np.zeros((B, 1), np.float32), ((np.arange(B) + 0.5) / N).astype(np.float32)[:, None],
+                          [-1], 1, cand_ids=np.tile(ids, (B, 1, 1)))
+        p_reuse = (o["reuse_slot"] >= 0).mean()
+        assert abs(p_reuse - omega) < 1e-12
+        assert p_reuse >= prev                    # monotone in kappa; reaches 1 at kappa = |V|
+        prev = p_reuse
+    assert prev == 1.0
+
+
+def test_branches_of_general_tree():
+    parent = [-1, 0, 1, 1, 0, 4]
+    paths, plen = O.branches(parent, 3)
+    assert paths.tolist() == [[1, 2, -1], [1, 3, -1], [4, 5, -1]]
+    assert plen.tolist() == [2, 2, 2]
+    with pytest.raises(ValueError):
+        O.tree([-1, 1])
