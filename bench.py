@@ -1,0 +1,351 @@
+#!/usr/bin/env python
+"""Benchmark of the Mirror-SD target-side verify step on B200.
+
+One "step" is one whole pass of the hot path over one batch of synthetic input: branch-tree attention
+for all layers -> LM head with fused reductions -> acceptance / branch selection, through the C-ABI
+call mirror_verify_step.  The workload is the 14B-shaped configuration (48 layers, prefix 2048 in
+16-token pages, kappa 4 x gamma 4, vocab 152064, greedy), which fits one GPU.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload NAME]
+
+Prints ONE JSON line.  With --impl reference the CPU oracle is timed instead (a deliberately plain
+program: the ratio to it says nothing about kernel quality; parity and the roofline fraction do).
+N > 1 runs independent replicas (the path does not shard): launch under torch.distributed.run.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import re
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "verify_steps_per_sec"
+UNIT = "steps/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="mirror", choices=["mirror", "reference"])
+    ap.add_argument("--workload", default="qwen14b")
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+# ---------------------------------------------------------------------------------------------------
+# algorithmic work of one step (what the method must move / compute), used for the roofline
+# ---------------------------------------------------------------------------------------------------
+def algorithmic_work(cfg, prefix_lens):
+    d, Hq, Hkv, n, L, B = cfg.head_dim, cfg.n_q_heads, cfg.n_kv_heads, cfg.n_nodes, cfg.layers, cfg.batch
+    kv_tokens = sum(int(l) for l in prefix_lens)
+    attn_bytes = L * (2 * kv_tokens * Hkv * d * 2          # prefix K and V, read once
+                      + 2 * B * n * Hkv * d * 2            # the tree's K and V
+                      + 2 * B * n * Hq * d * 2)            # Q read, O written
+    attn_flops = L * sum(4 * d * Hq * n * (int(l) + n) for l in prefix_lens)
+    lm_bytes = cfg.vocab * cfg.hidden * 2 + cfg.rows * cfg.hidden * 2
+    lm_flops = 2 * cfg.rows * cfg.vocab * cfg.hidden
+    return dict(attn_bytes=attn_bytes, attn_flops=attn_flops, lm_bytes=lm_bytes, lm_flops=lm_flops)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1400.0, source="fallback")
+
+
+def profiled_traffic(kernel_md: str):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary (None if absent)."""
+    path = os.path.join(ROOT, "profiles", kernel_md)
+    if not os.path.exists(path):
+        return None
+    m = re.search(r"dram_bytes_per_launch:\s*([0-9.eE+]+)", open(path).read())
+    return float(m.group(1)) if m else None
+
+
+# ---------------------------------------------------------------------------------------------------
+# clocks during the timed region (read-only NVML)
+# ---------------------------------------------------------------------------------------------------
+class ClockSampler:
+    def __init__(self, index: int):
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20,
+                 "hw_power_brake": 0x80}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(0.005)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        s = sorted(self.samples)
+        return dict(sm_mhz=(s[len(s) // 2] if s else None), sm_max_mhz=self.max_mhz, reasons=sorted(self.reasons),
+                    samples=len(s))
+
+
+# ---------------------------------------------------------------------------------------------------
+# CPU oracle timing (cpu_baseline leg and --impl reference)
+# ---------------------------------------------------------------------------------------------------
+def oracle_sample_seconds(x, cfg, vocab_slices: int = 8):
+    """Times the oracle, as it stands, on a bounded sample of one step: ONE of the attention layers (all
+    requests and rows) and the LM head on all rows over the first 1/vocab_slices of the vocabulary plus
+    the acceptance rule.  Returns (sample seconds, extrapolated seconds for a whole step, description)."""
+    import numpy as np
+    from oracle import oracle as O
+    from paper_2510_13161_b200 import inputs as I
+    anc, _ = O.tree(x.parent)
+    scale = 1.0 / np.sqrt(cfg.head_dim)
+    pt, pl = x.page_table.cpu().numpy(), x.prefix_len.cpu().numpy()
+    args = (I.bf16_bits(x.q[0]), I.bf16_bits(x.k_pool[0]), I.bf16_bits(x.v_pool[0]), pt, pl,
+            I.bf16_bits(x.k_new[0]), I.bf16_bits(x.v_new[0]), anc, scale)
+    vs = cfg.vocab // vocab_slices
+    Wb = I.bf16_bits(x.W[:vs])
+    t0 = time.perf_counter()
+    out, _, _ = O.attention_layer(*args)
+    t1 = time.perf_counter()
+    hid = out.reshape(cfg.rows, -1) if x.hidden is None else I.bf16_bits(x.hidden)
+    if hid.shape[1] != cfg.hidden:
+        hid = I.bf16_bits(x.hidden)
+    logits = O.lmhead_logits(hid, Wb)
+    red = O.row_reduce(logits)
+    tok = x.tokens.cpu().numpy()
+    O.accept_greedy(tok, red["argmax"].reshape(tok.shape), x.parent, cfg.gamma)
+    t2 = time.perf_counter()
+    sample = t2 - t0
+    full = (t1 - t0) * cfg.layers + (t2 - t1) * vocab_slices
+    desc = (f"1 of {cfg.layers} attention layers (all rows) + LM head / reductions / acceptance over the first "
+            f"1/{vocab_slices} of the vocabulary; whole-step time extrapolated linearly")
+    return sample, full, desc
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import torch
+    from oracle import oracle as O
+    from paper_2510_13161_b200 import inputs as I
+    cfg = I.CONFIGS[args.workload]
+    x = I.gen_verify_inputs(cfg, args.seed, "cpu", layers=1, force_hidden=cfg.explicit_hidden)
+    steps, warm = max(1, min(args.steps, 3)), max(0, min(args.warmup, 1))
+    for _ in range(warm):
+        oracle_sample_seconds(x, cfg)
+    fulls, samples, desc = [], [], ""
+    for _ in range(steps):
+        s, f, desc = oracle_sample_seconds(x, cfg)
+        samples.append(s); fulls.append(f)
+    full = sum(fulls) / len(fulls)
+    value = 1.0 / full
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+            "warmup": warm, "ms_per_step": full * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic", "draft_tokens_per_sec": value * cfg.draft_tokens,
+            "config": {"workload": cfg.name, "kappa": cfg.kappa, "gamma": cfg.gamma, "batch": cfg.batch,
+                       "layers": cfg.layers, "prefix": [cfg.prefix_lo, cfg.prefix_hi], "vocab": cfg.vocab},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle", "sample": desc,
+                             "sample_seconds": sum(samples) / len(samples)},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------------
+# the CUDA arm
+# ---------------------------------------------------------------------------------------------------
+def run_mirror(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2510_13161_b200 import binding, inputs as I
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the verify path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+
+    cfg = I.CONFIGS[args.workload]
+    x = I.gen_verify_inputs(cfg, args.seed + rank, dev)          # replicas: each rank draws its own problem
+    m = binding.Mirror(cfg.hidden, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.vocab, temperature=cfg.temperature,
+                       device=local)
+    kv = m.kv(x.k_pool, x.v_pool, x.page_table, x.prefix_len)
+    tree = m.tree(x.tokens, cfg.kappa, cfg.gamma)
+    mode = binding.ACCEPT_SPEC_SAMPLING if cfg.mode == "spec_sampling" else binding.ACCEPT_GREEDY
+    acc = m.accept_in(mode, True, q_probs=x.q_probs, u_accept=x.u_accept, u_resample=x.u_resample)
+    attn_out = torch.empty_like(x.q)
+    res = binding.AcceptResult(cfg.batch, cfg.gamma, dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        m.mirror_verify_step(kv, tree, x.q, x.k_new, x.v_new, x.hidden, x.W, acc, attn_out, out=res, stream=stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    code, detail = m.device_status()
+    if code != 0:
+        raise SystemExit(f"device status {code} (detail {detail}) during warm-up")
+
+    # ---- timed region: K steps, resident inputs, CUDA events on the launching stream; per-stage events ride along
+    K = args.steps
+    stage_ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local)
+    launches0 = m.launch_count()
+    barrier()
+    sampler.start()
+    ev0.record(stream)
+    for k in range(K):
+        m.set_stage_events(stage_ev[k])
+        step()
+    ev1.record(stream)
+    m.set_stage_events(None)
+    barrier()
+    clocks = sampler.stop()
+    launches = m.launch_count() - launches0
+    ms_total = ev0.elapsed_time(ev1)
+    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    ms_step = ms_total / K
+    value = world * 1e3 / ms_step
+    attn_ms = sum(e[0].elapsed_time(e[1]) for e in stage_ev) / K
+    lm_ms = sum(e[1].elapsed_time(e[2]) for e in stage_ev) / K
+    tail_ms = sum(e[2].elapsed_time(e[3]) for e in stage_ev) / K
+    code, detail = m.device_status()
+    if code != 0:
+        raise SystemExit(f"device status {code} (detail {detail}) during the timed region")
+
+    # ---- end to end: per step, this step's inputs come from pinned host memory and the decision goes back
+    h_in = {k: getattr(x, k).cpu().pin_memory() for k in ("q", "k_new", "v_new", "tokens")}
+    d_in = {k: torch.empty_like(getattr(x, k)) for k in h_in}
+    tree_e = m.tree(d_in["tokens"], cfg.kappa, cfg.gamma)
+    h_out = {k: torch.empty_like(getattr(res, k), device="cpu").pin_memory() for k in ("n_accepted", "n_emitted", "emitted", "best_branch")}
+    h2d = sum(v.numel() * v.element_size() for v in h_in.values())
+    d2h = sum(v.numel() * v.element_size() for v in h_out.values())
+
+    def e2e_step():
+        for k, v in h_in.items():
+            d_in[k].copy_(v, non_blocking=True)
+        m.mirror_verify_step(kv, tree_e, d_in["q"], d_in["k_new"], d_in["v_new"], x.hidden, x.W, acc, attn_out, out=res,
+                             stream=stream)
+        for k, v in h_out.items():
+            v.copy_(getattr(res, k), non_blocking=True)
+        stream.synchronize()      # the caller needs the decision before it can build the next step
+
+    for _ in range(3):
+        e2e_step()
+    Ke = max(10, min(K, 200))
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(Ke):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    te = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(te, op=dist.ReduceOp.MAX)
+    e2e_value = world * 1e3 / (float(te.item()) / Ke)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    work = algorithmic_work(cfg, x.prefix_len.cpu().tolist())
+    peaks = measured_peaks()
+    lm_gbs = work["lm_bytes"] / (lm_ms * 1e-3) / 1e9
+    attn_gbs = work["attn_bytes"] / (attn_ms * 1e-3) / 1e9
+    roofline = {"kernel": "lmhead_kernel", "bound": "hbm", "achieved": lm_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": lm_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                "traffic": profiled_traffic("lmhead_kernel_qwen14b.md"),
+                "algorithmic_bytes_per_launch": work["lm_bytes"], "ms_per_launch": lm_ms}
+    stages = {"attn_ms": attn_ms, "lmhead_ms": lm_ms, "merge_accept_ms": tail_ms,
+              "attn_gbs": attn_gbs, "attn_frac_hbm": attn_gbs / peaks["hbm_gbs"],
+              "attn_tflops": work["attn_flops"] / (attn_ms * 1e-3) / 1e12,
+              "lmhead_tflops": work["lm_flops"] / (lm_ms * 1e-3) / 1e12,
+              "step_hbm_frac": (work["attn_bytes"] + work["lm_bytes"]) / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+
+    cpu = None
+    if not args.no_cpu_baseline and world == 1:
+        from oracle import oracle as O
+        xs = I.gen_verify_inputs(cfg, args.seed, "cpu", layers=1, force_hidden=cfg.explicit_hidden)
+        s, full, desc = oracle_sample_seconds(xs, cfg)
+        cpu = {"value": 1.0 / full, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle", "sample": desc,
+               "sample_seconds": s}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic", "draft_tokens_per_sec": value * cfg.draft_tokens,
+            "config": {"workload": cfg.name, "kappa": cfg.kappa, "gamma": cfg.gamma, "batch": cfg.batch, "layers": cfg.layers,
+                       "prefix": [cfg.prefix_lo, cfg.prefix_hi], "vocab": cfg.vocab, "hidden": cfg.hidden,
+                       "l2": "inputs (KV cache + LM-head weights, about 2 GB) are larger than L2; no flush",
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "resident": "KV cache and LM-head weights stay on the device; Q, tree K/V and tokens are copied every step"},
+            "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "stages": stages, "cpu_baseline": cpu}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_mirror(args)
+
+
+if __name__ == "__main__":
+    main()

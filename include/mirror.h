@@ -1,0 +1,211 @@
+/*
+ * mirror.h -- C ABI of the B200 (sm_100a) library for the target-side verify step of
+ * Mirror Speculative Decoding.
+ *
+ * One verify step scores a token tree of draft proposals hanging off the last committed token
+ * (the hypothesis tree T_t of Sec. 3.1: kappa branches x gamma lookahead tokens) with the target
+ * model and decides what to commit:
+ *
+ *   mirror_attn_verify    branch-tree attention of every tree node against the paged KV cache of
+ *                         the verified prefix plus the tree's own K/V under the branch-causal mask
+ *                         (each branch is scored as if decoded alone: "verifies left-to-right", Eq. 3)
+ *   mirror_lmhead_reduce  logits = W h (the output head of Eq. 1; applied to an intermediate state it
+ *                         is the early-exit proxy of Eq. 5) fused with per-row argmax / log-sum-exp /
+ *                         Top-kappa (ids + log-probabilities: the token-channel message of Eq. 6)
+ *   mirror_accept_select  acceptance operator of Eq. 3 / Eq. 10 per branch (greedy), or the standard
+ *                         speculative-sampling rule (Sec. 3.1) with residual resampling; the longest
+ *                         accepted branch, the correction / bonus token, and the reuse lookup of
+ *                         Sec. 3.1 ("Verification vs. reuse criterion")
+ *   mirror_verify_step    the three chained on one stream
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless its comment says "host".  The caller owns every buffer;
+ *     inputs are never written.  bf16 tensors are passed as `const void*`.
+ *   - All compute calls only enqueue work on `stream` (a cudaStream_t passed as void*) and return without
+ *     synchronising.  Host-side argument errors are returned immediately; device-side problems (a bounded
+ *     wait that ran out, an index outside its table) set a status word read by mirror_device_status().
+ *   - The library allocates device memory only inside mirror_create() (one status word).  Scratch memory
+ *     is a caller-provided workspace, sized by mirror_workspace_bytes() and attached with
+ *     mirror_set_workspace(); its contents need not survive between calls but two calls that use the
+ *     same ctx must not overlap on the GPU.
+ *   - Token tree: node 0 is the root (the last committed token, whose row verifies every branch's first
+ *     token); parent[i] < i.  A "branch" is a root-to-leaf path, leaves taken in increasing node order.
+ *     Row r of any [batch*n_nodes, ...] tensor is (request r / n_nodes, node r % n_nodes): the target's
+ *     distribution for the token that follows that node.
+ *   - Ties: argmax and Top-kappa prefer the lowest token id; branch selection the lowest branch index.
+ */
+#ifndef MIRROR_H_
+#define MIRROR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mirror_ctx mirror_ctx;
+
+typedef enum {
+    MIRROR_OK = 0,
+    MIRROR_ERR_ARG = 1,          /* null pointer / negative size */
+    MIRROR_ERR_SHAPE = 2,        /* inconsistent or out-of-range dimensions */
+    MIRROR_ERR_UNSUPPORTED = 3,  /* head_dim not in {64,128}, page_size != 16, device is not sm_100, ... */
+    MIRROR_ERR_WORKSPACE = 4,    /* workspace missing or too small */
+    MIRROR_ERR_CUDA = 5,         /* a CUDA runtime / driver call failed */
+    MIRROR_ERR_DEVICE_CHECK = 6, /* device-side bounds check tripped (reported by mirror_device_status) */
+    MIRROR_ERR_TIMEOUT = 7       /* a bounded device-side wait expired (reported by mirror_device_status) */
+} mirror_status;
+
+#define MIRROR_MAX_NODES 128     /* tree nodes per request, root included */
+#define MIRROR_MAX_BRANCHES 64   /* root-to-leaf paths */
+#define MIRROR_MAX_DEPTH 32      /* nodes on a path below the root (gamma) */
+#define MIRROR_MAX_TOPK 32
+
+typedef struct {
+    int hidden;            /* H: width of the rows fed to the LM head */
+    int n_q_heads;         /* Hq */
+    int n_kv_heads;        /* Hkv, divides Hq */
+    int head_dim;          /* d: 64 or 128 */
+    int vocab;             /* |V| */
+    int page_size;         /* tokens per KV page: 16 */
+    float softmax_scale;   /* attention score scale; 0 selects 1/sqrt(head_dim) */
+    float temperature;     /* T > 0: probabilities are Softmax(logits / T); 0 selects 1.  Greedy ignores it. */
+} mirror_model_desc;
+
+typedef struct {
+    int batch;             /* B independent requests, all with the same tree shape */
+    int n_nodes;           /* n <= MIRROR_MAX_NODES, root included */
+    int kappa;             /* branches of the canonical tree (used when parent == NULL) */
+    int gamma;             /* maximum branch length; width of the per-request outputs */
+    const int32_t* tokens; /* device [B, n]: token id of each node (node 0: last committed token) */
+    const int32_t* parent; /* HOST [n], parent[0] = -1, parent[i] < i; NULL selects the canonical comb:
+                              branch i = chain of nodes 1+i*gamma .. 1+i*gamma+gamma-1 (n = 1+kappa*gamma) */
+} mirror_tree;
+
+typedef struct {
+    const void* k_pool;        /* device bf16 [num_layers][num_pages, Hkv, page_size, d] */
+    const void* v_pool;        /* same layout */
+    int64_t layer_stride;      /* elements between consecutive layers' pools; a multiple of Hkv*page_size*d */
+    int num_layers;
+    int num_pages;             /* pages in one layer's pool */
+    int max_pages_per_req;
+    const int32_t* page_table; /* device [B, max_pages_per_req]: physical page of each logical page (shared by layers) */
+    const int32_t* prefix_len; /* device [B]: verified-prefix length in tokens, <= max_pages_per_req*page_size */
+} mirror_kv;
+
+typedef enum { MIRROR_ACCEPT_GREEDY = 0, MIRROR_ACCEPT_SPEC_SAMPLING = 1 } mirror_accept_mode;
+
+typedef struct {
+    mirror_accept_mode mode;
+    int emit_bonus;               /* 1: when a whole branch is accepted also emit the token of its last row */
+    const int32_t* target_argmax; /* [B*n]  greedy: the target's token for each row */
+    const float* logits;          /* [B*n, V] fp32   spec sampling */
+    const float* lse;             /* [B*n] fp32      spec sampling: log sum exp(logits / T) per row */
+    const float* q_probs;         /* [B, n-1, V] fp32 spec sampling: draft distribution that proposed node i+1 */
+    const float* u_accept;        /* [B, n] fp32 in [0,1): uniform of node c's accept test */
+    const float* u_resample;      /* [B, n] fp32 in [0,1): uniform of the correction / bonus draw at row R */
+    const int32_t* cand_ids;      /* nullable [B*n, n_cand]: ids the draft already expanded below each row
+                                     (e.g. the early-exit Top-kappa of that row) for the reuse lookup */
+    int n_cand;
+} mirror_accept_in;
+
+typedef struct {
+    int32_t* n_accepted;     /* [B]   A: accepted draft tokens */
+    int32_t* best_branch;    /* [B]   lowest branch index attaining A */
+    int32_t* n_emitted;      /* [B]   A + 1 (A when a whole branch is accepted and emit_bonus == 0) */
+    int32_t* emitted;        /* [B, gamma+1] accepted tokens then the correction / bonus token, -1 padded */
+    int32_t* accepted_nodes; /* [B, gamma] node ids of the accepted tokens, -1 padded (for the caller's KV commit) */
+    int32_t* decide_row;     /* [B]   node whose row produced the correction / bonus token */
+    int32_t* reuse_slot;     /* [B]   index of that token in cand_ids[row], or -1 (fallback: fresh rollout) */
+} mirror_accept_out;
+
+/* What mirror_workspace_bytes should size for. */
+#define MIRROR_WS_ATTN 1u           /* mirror_attn_verify */
+#define MIRROR_WS_LMHEAD 2u         /* mirror_lmhead_reduce (M = batch * n_nodes rows) */
+#define MIRROR_WS_LMHEAD_LOGITS 10u /* mirror_lmhead_reduce with topk > 0 and logits_out == NULL */
+#define MIRROR_WS_STEP_GREEDY 7u    /* mirror_verify_step, greedy */
+#define MIRROR_WS_STEP_SPEC 15u     /* mirror_verify_step, speculative sampling (holds the fp32 logits) */
+
+/* Create a context for one model shape on CUDA device `device` (made current for the call).
+ * Allocates one device status word.  Fails with MIRROR_ERR_UNSUPPORTED on a device that is not sm_100. */
+mirror_status mirror_create(mirror_ctx** out, const mirror_model_desc* desc, int device);
+mirror_status mirror_destroy(mirror_ctx* ctx);
+
+/* Bytes of workspace needed for the calls selected by `what` (OR of MIRROR_WS_*) on this tree / cache
+ * shape.  `tree` and `kv` are read for their sizes only (pointers inside may be NULL). */
+mirror_status mirror_workspace_bytes(const mirror_ctx* ctx, const mirror_tree* tree, const mirror_kv* kv,
+                                     unsigned what, size_t* bytes);
+/* Attach a device workspace (256-byte aligned).  The ctx keeps the pointer, not the memory. */
+mirror_status mirror_set_workspace(mirror_ctx* ctx, void* dev_ptr, size_t bytes);
+
+/* Branch-tree attention for all layers of `kv` (a1 + a2 of the verify step).
+ *   q      bf16 [L, B, n, Hq, d]   queries of the tree nodes (already position-encoded)
+ *   k_new  bf16 [L, B, n, Hkv, d]  this step's keys of the tree nodes;  v_new likewise
+ *   out    bf16 [L, B, n, Hq, d]   softmax(scale * q k^T over Vis(node)) v, with
+ *                                  Vis(node) = verified prefix  U  {node and its ancestors}
+ *   lse_out fp32 [L, B, Hq, n], nullable: natural-log softmax denominator of each row
+ * Needs a workspace sized for MIRROR_WS_ATTN. */
+mirror_status mirror_attn_verify(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree,
+                                 const void* q, const void* k_new, const void* v_new,
+                                 void* out, float* lse_out, void* stream);
+
+/* LM head with fused row reductions: logits[r][v] = sum_k hidden[r][k] * W[v][k]  (Eq. 1, Eq. 5).
+ *   hidden bf16 [M, H] (row stride H);  W bf16 [V, H]
+ *   argmax   int32 [M]  lowest id attaining the maximum          (nullable)
+ *   maxlogit fp32 [M]   that maximum                              (nullable)
+ *   lse      fp32 [M]   log sum_v exp(logits/T)                   (nullable)
+ *   topk > 0: topk_id int32 [M, topk], topk_logprob fp32 [M, topk] = logits/T - lse, ordered by
+ *             (logit descending, id ascending): the Top-kappa message of Eq. 6.  topk <= MIRROR_MAX_TOPK.
+ *   gather_row/gather_tok int32 [n_gather] -> gather_logit fp32 [n_gather] = logits[row][tok]  (nullable)
+ *   logits_out fp32 [M, V], nullable: the full logits (needed by speculative sampling; Top-kappa uses the
+ *             workspace when this is NULL)
+ * Needs a workspace sized for MIRROR_WS_LMHEAD. */
+mirror_status mirror_lmhead_reduce(mirror_ctx* ctx, const void* hidden, int M, const void* W, int topk,
+                                   const int32_t* gather_row, const int32_t* gather_tok, int n_gather,
+                                   int32_t* argmax, float* maxlogit, float* lse,
+                                   int32_t* topk_id, float* topk_logprob, float* gather_logit,
+                                   float* logits_out, void* stream);
+
+/* Acceptance, branch selection, emitted tokens and reuse lookup (a5 + a6).
+ * Greedy (Eq. 3 / Eq. 10): branch length a = number of leading nodes c with tokens[c] == target_argmax[parent(c)].
+ * Speculative sampling: node c (token x, parent row r) passes iff u_accept[c] * q_c[x] <= p_r[x] with
+ * p_r[v] = exp(logits[r][v]/T - lse[r]), evaluated in fp64; the extra token is drawn by inverse CDF with
+ * u_resample[R] from the normalised residual max(0, p_R - q_c') of the first rejected node c' of the chosen
+ * branch, or from p_R when the whole branch was accepted (or the residual has no mass).
+ * Selecting the longest of several independently tested branches is distribution-preserving only for a
+ * single branch. */
+mirror_status mirror_accept_select(mirror_ctx* ctx, const mirror_tree* tree, const mirror_accept_in* in,
+                                   const mirror_accept_out* out, void* stream);
+
+/* One whole verify step on one stream: attention over all layers -> LM head rows -> reductions -> acceptance.
+ *   hidden   bf16 [B*n, H], or NULL to feed the last layer's attention output (requires Hq*d == H)
+ *   attn_out bf16 [L, B, n, Hq, d]  (required: it is also the chained LM-head input)
+ *   acc      mode, emit_bonus, q_probs, u_accept, u_resample, cand_ids are read; target_argmax / logits / lse
+ *            are produced internally (in the workspace)
+ *   argmax_out int32 [B*n], nullable: the target's greedy token per row, for inspection
+ * Needs a workspace sized for MIRROR_WS_STEP_GREEDY or MIRROR_WS_STEP_SPEC. */
+mirror_status mirror_verify_step(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree,
+                                 const void* q, const void* k_new, const void* v_new,
+                                 const void* hidden, const void* W, const mirror_accept_in* acc,
+                                 const mirror_accept_out* out, void* attn_out, int32_t* argmax_out,
+                                 void* stream);
+
+/* Optional timing hooks for mirror_verify_step: four cudaEvent_t (passed as void*) that every later
+ * mirror_verify_step on this ctx records on its stream -- before attention, after attention, after the
+ * LM-head GEMM kernel, after acceptance -- until cleared with NULL.  The caller owns the events. */
+mirror_status mirror_set_stage_events(mirror_ctx* ctx, void* const* events4);
+
+/* Synchronises the device and returns the sticky device-side status (MIRROR_OK, MIRROR_ERR_TIMEOUT or
+ * MIRROR_ERR_DEVICE_CHECK) in *code, with a detail word in *detail (nullable); then clears it. */
+mirror_status mirror_device_status(mirror_ctx* ctx, int* code, int* detail);
+
+/* Number of kernels the library has launched through this ctx since creation (for accounting). */
+mirror_status mirror_launch_count(const mirror_ctx* ctx, long long* count);
+
+const char* mirror_status_str(mirror_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MIRROR_H_ */

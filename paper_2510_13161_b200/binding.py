@@ -1,0 +1,274 @@
+"""Thin ctypes binding of libmirror.so (see include/mirror.h).
+
+Argument marshalling only: every step of the verify path runs in the CUDA kernels
+of the library.  torch is used for device memory and streams.  There is no CPU
+fallback: if the library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmirror.so")
+
+ACCEPT_GREEDY = 0
+ACCEPT_SPEC_SAMPLING = 1
+WS_ATTN, WS_LMHEAD, WS_LMHEAD_LOGITS, WS_STEP_GREEDY, WS_STEP_SPEC = 1, 2, 10, 7, 15
+
+EXPORTS = [
+    "mirror_create", "mirror_destroy", "mirror_workspace_bytes", "mirror_set_workspace",
+    "mirror_attn_verify", "mirror_lmhead_reduce", "mirror_accept_select", "mirror_verify_step",
+    "mirror_device_status", "mirror_launch_count", "mirror_status_str", "mirror_set_stage_events",
+]
+
+
+class MirrorError(RuntimeError):
+    def __init__(self, code: int, where: str, text: str):
+        super().__init__(f"{where}: mirror_status {code} ({text})")
+        self.code = code
+
+
+class ModelDesc(C.Structure):
+    _fields_ = [("hidden", C.c_int), ("n_q_heads", C.c_int), ("n_kv_heads", C.c_int), ("head_dim", C.c_int),
+                ("vocab", C.c_int), ("page_size", C.c_int), ("softmax_scale", C.c_float), ("temperature", C.c_float)]
+
+
+class Tree(C.Structure):
+    _fields_ = [("batch", C.c_int), ("n_nodes", C.c_int), ("kappa", C.c_int), ("gamma", C.c_int),
+                ("tokens", C.c_void_p), ("parent", C.POINTER(C.c_int32))]
+
+
+class KV(C.Structure):
+    _fields_ = [("k_pool", C.c_void_p), ("v_pool", C.c_void_p), ("layer_stride", C.c_int64),
+                ("num_layers", C.c_int), ("num_pages", C.c_int), ("max_pages_per_req", C.c_int),
+                ("page_table", C.c_void_p), ("prefix_len", C.c_void_p)]
+
+
+class AcceptIn(C.Structure):
+    _fields_ = [("mode", C.c_int), ("emit_bonus", C.c_int), ("target_argmax", C.c_void_p), ("logits", C.c_void_p),
+                ("lse", C.c_void_p), ("q_probs", C.c_void_p), ("u_accept", C.c_void_p), ("u_resample", C.c_void_p),
+                ("cand_ids", C.c_void_p), ("n_cand", C.c_int)]
+
+
+class AcceptOut(C.Structure):
+    _fields_ = [("n_accepted", C.c_void_p), ("best_branch", C.c_void_p), ("n_emitted", C.c_void_p),
+                ("emitted", C.c_void_p), ("accepted_nodes", C.c_void_p), ("decide_row", C.c_void_p),
+                ("reuse_slot", C.c_void_p)]
+
+
+_lib = None
+
+
+def load_library():
+    """Load libmirror.so; raises if it has not been built (python -m paper_2510_13161_b200._build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(f"{LIB_PATH} is missing: build it with `python -m paper_2510_13161_b200._build`; "
+                                    "there is no fallback path")
+        lib = C.CDLL(LIB_PATH)
+        lib.mirror_status_str.restype = C.c_char_p
+        lib.mirror_status_str.argtypes = [C.c_int]
+        for name in EXPORTS:
+            if name != "mirror_status_str":
+                getattr(lib, name).restype = C.c_int
+        _lib = lib
+    return _lib
+
+
+def _check(code: int, where: str):
+    if code != 0:
+        raise MirrorError(code, where, load_library().mirror_status_str(code).decode())
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None, name: str = "tensor"):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"{name} must be {dtype}, got {t.dtype}")
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> C.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+class AcceptResult:
+    """Device tensors written by mirror_accept_select / mirror_verify_step."""
+
+    def __init__(self, batch: int, gamma: int, device):
+        i32 = dict(dtype=torch.int32, device=device)
+        self.n_accepted = torch.empty(batch, **i32)
+        self.best_branch = torch.empty(batch, **i32)
+        self.n_emitted = torch.empty(batch, **i32)
+        self.emitted = torch.empty((batch, gamma + 1), **i32)
+        self.accepted_nodes = torch.empty((batch, max(gamma, 1)), **i32)
+        self.decide_row = torch.empty(batch, **i32)
+        self.reuse_slot = torch.empty(batch, **i32)
+
+    def struct(self) -> AcceptOut:
+        return AcceptOut(*[C.c_void_p(getattr(self, f).data_ptr()) for f, _ in AcceptOut._fields_])
+
+    def cpu(self) -> dict:
+        return {f: getattr(self, f).cpu().numpy() for f, _ in AcceptOut._fields_}
+
+
+class Mirror:
+    """One library context: a model shape on one device, plus its workspace."""
+
+    def __init__(self, hidden: int, n_q_heads: int, n_kv_heads: int, head_dim: int, vocab: int,
+                 page_size: int = 16, softmax_scale: float = 0.0, temperature: float = 1.0, device: int = 0):
+        self.lib = load_library()
+        self.desc = ModelDesc(hidden, n_q_heads, n_kv_heads, head_dim, vocab, page_size, softmax_scale, temperature)
+        self.device = torch.device("cuda", device)
+        self._ctx = C.c_void_p()
+        _check(self.lib.mirror_create(C.byref(self._ctx), C.byref(self.desc), device), "mirror_create")
+        self._ws = None
+        self._keep = []
+
+    def close(self):
+        if self._ctx:
+            self.lib.mirror_destroy(self._ctx)
+            self._ctx = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- argument structs -------------------------------------------------------------------
+    def tree(self, tokens: torch.Tensor, kappa: int, gamma: int, parent: Optional[Sequence[int]] = None) -> Tree:
+        B, n = tokens.shape
+        par = None
+        if parent is not None:
+            arr = (C.c_int32 * len(parent))(*parent)
+            self._keep.append(arr)
+            par = C.cast(arr, C.POINTER(C.c_int32))
+        t = Tree(B, n, kappa, gamma, _ptr(tokens, torch.int32, "tokens"), par)
+        t._refs = (tokens,)          # the struct holds raw pointers: keep the tensors alive with it
+        return t
+
+    def kv(self, k_pool: torch.Tensor, v_pool: torch.Tensor, page_table: torch.Tensor, prefix_len: torch.Tensor) -> KV:
+        """k_pool / v_pool: bf16 [L, num_pages, Hkv, page, d] (one allocation, layers consecutive)."""
+        L, num_pages = k_pool.shape[0], k_pool.shape[1]
+        stride = k_pool.stride(0) if L > 1 else k_pool[0].numel()
+        kv = KV(_ptr(k_pool, torch.bfloat16, "k_pool"), _ptr(v_pool, torch.bfloat16, "v_pool"), stride, L, num_pages,
+                page_table.shape[1], _ptr(page_table, torch.int32, "page_table"), _ptr(prefix_len, torch.int32, "prefix_len"))
+        kv._refs = (k_pool, v_pool, page_table, prefix_len)
+        return kv
+
+    # ---- workspace --------------------------------------------------------------------------
+    def workspace_bytes(self, tree: Tree, kv: Optional[KV], what: int) -> int:
+        out = C.c_size_t()
+        _check(self.lib.mirror_workspace_bytes(self._ctx, C.byref(tree), C.byref(kv) if kv is not None else None,
+                                               C.c_uint(what), C.byref(out)), "mirror_workspace_bytes")
+        return out.value
+
+    def ensure_workspace(self, tree: Tree, kv: Optional[KV], what: int):
+        need = self.workspace_bytes(tree, kv, what)
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device=self.device)
+            _check(self.lib.mirror_set_workspace(self._ctx, C.c_void_p(self._ws.data_ptr()), C.c_size_t(need)),
+                   "mirror_set_workspace")
+
+    # ---- entry points -----------------------------------------------------------------------
+    def mirror_attn_verify(self, kv: KV, tree: Tree, q, k_new, v_new, out=None, lse_out=None, stream=None):
+        if out is None:
+            out = torch.empty_like(q)
+        self.ensure_workspace(tree, kv, WS_ATTN)
+        _check(self.lib.mirror_attn_verify(self._ctx, C.byref(kv), C.byref(tree), _ptr(q, torch.bfloat16, "q"),
+                                           _ptr(k_new, torch.bfloat16, "k_new"), _ptr(v_new, torch.bfloat16, "v_new"),
+                                           _ptr(out, torch.bfloat16, "out"), _ptr(lse_out, torch.float32, "lse_out"),
+                                           _stream(stream)), "mirror_attn_verify")
+        return out
+
+    def mirror_lmhead_reduce(self, hidden, W, topk: int = 0, gather_row=None, gather_tok=None, want_lse: bool = True,
+                             want_logits: bool = False, stream=None) -> dict:
+        M = hidden.shape[0]
+        dev = hidden.device
+        res = dict(argmax=torch.empty(M, dtype=torch.int32, device=dev),
+                   maxlogit=torch.empty(M, dtype=torch.float32, device=dev),
+                   lse=torch.empty(M, dtype=torch.float32, device=dev) if want_lse else None,
+                   topk_id=torch.empty((M, topk), dtype=torch.int32, device=dev) if topk else None,
+                   topk_logprob=torch.empty((M, topk), dtype=torch.float32, device=dev) if topk else None,
+                   gather_logit=None, logits=None)
+        n_gather = 0
+        if gather_row is not None:
+            n_gather = gather_row.numel()
+            res["gather_logit"] = torch.empty(n_gather, dtype=torch.float32, device=dev)
+        if want_logits:
+            res["logits"] = torch.empty((M, self.desc.vocab), dtype=torch.float32, device=dev)
+        t = Tree(1, M if M <= 128 else 128, 0, 0, None, None)
+        t.batch, t.n_nodes = (M + 127) // 128, min(M, 128)      # sizes only: batch * n_nodes >= M
+        self.ensure_workspace(t, None, WS_LMHEAD_LOGITS if (topk and not want_logits) else WS_LMHEAD)
+        _check(self.lib.mirror_lmhead_reduce(self._ctx, _ptr(hidden, torch.bfloat16, "hidden"), M,
+                                             _ptr(W, torch.bfloat16, "W"), topk,
+                                             _ptr(gather_row, torch.int32, "gather_row"),
+                                             _ptr(gather_tok, torch.int32, "gather_tok"), n_gather,
+                                             _ptr(res["argmax"]), _ptr(res["maxlogit"]), _ptr(res["lse"]),
+                                             _ptr(res["topk_id"]), _ptr(res["topk_logprob"]), _ptr(res["gather_logit"]),
+                                             _ptr(res["logits"]), _stream(stream)), "mirror_lmhead_reduce")
+        return res
+
+    def accept_in(self, mode: int, emit_bonus: bool = True, target_argmax=None, logits=None, lse=None, q_probs=None,
+                  u_accept=None, u_resample=None, cand_ids=None) -> AcceptIn:
+        n_cand = 0 if cand_ids is None else cand_ids.shape[-1]
+        a = AcceptIn(mode, int(emit_bonus), _ptr(target_argmax, torch.int32, "target_argmax"),
+                     _ptr(logits, torch.float32, "logits"), _ptr(lse, torch.float32, "lse"),
+                     _ptr(q_probs, torch.float32, "q_probs"), _ptr(u_accept, torch.float32, "u_accept"),
+                     _ptr(u_resample, torch.float32, "u_resample"), _ptr(cand_ids, torch.int32, "cand_ids"), n_cand)
+        a._refs = (target_argmax, logits, lse, q_probs, u_accept, u_resample, cand_ids)
+        return a
+
+    def mirror_accept_select(self, tree: Tree, acc: AcceptIn, out: Optional[AcceptResult] = None, stream=None) -> AcceptResult:
+        if out is None:
+            out = AcceptResult(tree.batch, tree.gamma, self.device)
+        o = out.struct()
+        _check(self.lib.mirror_accept_select(self._ctx, C.byref(tree), C.byref(acc), C.byref(o), _stream(stream)),
+               "mirror_accept_select")
+        return out
+
+    def mirror_verify_step(self, kv: KV, tree: Tree, q, k_new, v_new, hidden, W, acc: AcceptIn, attn_out,
+                           out: Optional[AcceptResult] = None, argmax_out=None, stream=None) -> AcceptResult:
+        if out is None:
+            out = AcceptResult(tree.batch, tree.gamma, self.device)
+        self.ensure_workspace(tree, kv, WS_STEP_SPEC if acc.mode == ACCEPT_SPEC_SAMPLING else WS_STEP_GREEDY)
+        o = out.struct()
+        _check(self.lib.mirror_verify_step(self._ctx, C.byref(kv), C.byref(tree), _ptr(q, torch.bfloat16, "q"),
+                                           _ptr(k_new, torch.bfloat16, "k_new"), _ptr(v_new, torch.bfloat16, "v_new"),
+                                           _ptr(hidden, torch.bfloat16, "hidden"), _ptr(W, torch.bfloat16, "W"),
+                                           C.byref(acc), C.byref(o), _ptr(attn_out, torch.bfloat16, "attn_out"),
+                                           _ptr(argmax_out, torch.int32, "argmax_out"), _stream(stream)),
+               "mirror_verify_step")
+        return out
+
+    def set_stage_events(self, events):
+        """events: four torch.cuda.Event(enable_timing=True) recorded by later mirror_verify_step calls, or None."""
+        if events is None:
+            _check(self.lib.mirror_set_stage_events(self._ctx, None), "mirror_set_stage_events")
+            return
+        for e in events:
+            if e.cuda_event == 0:       # torch creates the CUDA event lazily, on first record
+                e.record()
+        arr = (C.c_void_p * 4)(*[C.c_void_p(e.cuda_event) for e in events])
+        _check(self.lib.mirror_set_stage_events(self._ctx, arr), "mirror_set_stage_events")
+
+    def device_status(self):
+        code, detail = C.c_int(), C.c_int()
+        _check(self.lib.mirror_device_status(self._ctx, C.byref(code), C.byref(detail)), "mirror_device_status")
+        return code.value, detail.value
+
+    def launch_count(self) -> int:
+        n = C.c_longlong()
+        _check(self.lib.mirror_launch_count(self._ctx, C.byref(n)), "mirror_launch_count")
+        return n.value

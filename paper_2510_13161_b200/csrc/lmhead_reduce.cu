@@ -1,0 +1,481 @@
+// LM head logits = W h (Eq. 1; early-exit proxy Eq. 5) as a tcgen05 / TMEM GEMM with the per-row
+// argmax / max / log-sum-exp reduction fused into the epilogue, so that the [M, V] logits never
+// travel through HBM unless the caller asks for them (speculative sampling, Top-kappa of Eq. 6).
+//
+// Orientation ("swap-AB"): the vocabulary is the UMMA M axis (128 weight rows per tile, one TMEM
+// lane per vocabulary id), the hidden rows are the UMMA N axis (<= 256 per chunk, one TMEM column
+// per hidden row).  The verify step has few rows (B * (1 + kappa*gamma)), so the kernel is a weight
+// stream: W leaves HBM exactly once per row chunk and the per-SM TMA pipeline is what has to keep
+// HBM busy.
+//
+// Persistent CTAs, one per SM, 6 warps:
+//   warp 0      TMA producer: W tile [128 x 64] + hidden tile [N x 64] per stage, 128-byte swizzle
+//   warp 1      TMEM owner and UMMA issuer (one elected lane): 4 x (128 x N x 16) per stage
+//   warps 2..5  epilogue: tcgen05.ld the accumulator (lane = vocabulary id), per-column warp
+//               reductions, running (max, argmax, sum-exp) per hidden row, optional fp32 spill
+// The vocabulary is split over CTAs in 8-row groups (the swizzle atom), so every CTA streams the same
+// number of weight bytes (+-8 rows); the ragged last tile of a CTA is fetched as 8-row TMA boxes.
+// Each (CTA, epilogue warp) leaves one partial per hidden row; a second tiny kernel merges them in a
+// fixed order with the comparator (logit descending, id ascending).
+//
+// Every mbarrier wait is bounded; on expiry the kernel records MIRROR_DEV_TIMEOUT and unwinds.
+#include <math.h>
+
+#include "mirror_internal.h"
+
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kBK = 64;                 // K elements per pipeline stage (one 128-byte swizzle row)
+constexpr int kTileV = 128;             // vocabulary rows per UMMA tile
+constexpr int kATileBytes = kTileV * kBK * 2;
+constexpr int kMaxStages = 10;
+constexpr int kMaxAcc = 4;
+constexpr int kMaxChunkRows = 256;
+constexpr int kSmemBudget = 232448;     // 227 KB
+constexpr int kCtrlBytes = 1024 + 4 * kMaxChunkRows * 12;   // barriers + per-warp running state
+
+struct LmParams {
+    int M, V, H;
+    int n_chunks, chunk_rows;           // hidden rows are processed in chunks of chunk_rows (multiple of 16)
+    int acc_stride, n_acc, tmem_cols;   // TMEM columns per accumulator buffer, number of buffers, allocation
+    int stages, stage_bytes;
+    int groups_total;                   // ceil(V / 8)
+    float inv_T, inv_T_log2e;
+    float* logits_out;                  // nullable [M, V]
+    float* part_max;                    // [grid*4][M]
+    int* part_idx;
+    float* part_sum;
+    int* status;
+};
+
+struct Ctrl {
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
+    uint64_t acc_full[kMaxAcc];
+    uint64_t acc_empty[kMaxAcc];
+    uint32_t tmem_base;
+    volatile int abort;
+};
+
+__device__ __forceinline__ void fail(const LmParams& p, Ctrl* c, int where) {
+    c->abort = 1;
+    if (atomicCAS(p.status, 0, MIRROR_DEV_TIMEOUT) == 0) atomicExch(p.status + 1, where);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+lmhead_kernel(const __grid_constant__ CUtensorMap tm_w_full, const __grid_constant__ CUtensorMap tm_w_grp,
+              const __grid_constant__ CUtensorMap tm_h, const LmParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t* stage_base = smem;
+    Ctrl* ctrl = (Ctrl*)(smem + (size_t)p.stages * p.stage_bytes);
+    float* st_max = (float*)((uint8_t*)ctrl + 1024);          // [4][kMaxChunkRows]
+    int* st_idx = (int*)(st_max + 4 * kMaxChunkRows);
+    float* st_sum = (float*)(st_idx + 4 * kMaxChunkRows);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    // this CTA's slice of the vocabulary, in 8-row groups
+    const int g0 = (int)(((long long)p.groups_total * blockIdx.x) / gridDim.x);
+    const int g1 = (int)(((long long)p.groups_total * (blockIdx.x + 1)) / gridDim.x);
+    const int row_begin = g0 * 8;
+    const int row_end = min(g1 * 8, p.V);
+    const int n_tiles = (g1 - g0 + 15) / 16;
+    const int n_kb = p.H / kBK;
+
+    if (tid == 0) {
+        for (int s = 0; s < p.stages; ++s) { ptx::mbar_init(&ctrl->full[s], 1); ptx::mbar_init(&ctrl->empty[s], 1); }
+        for (int a = 0; a < p.n_acc; ++a) { ptx::mbar_init(&ctrl->acc_full[a], 1); ptx::mbar_init(&ctrl->acc_empty[a], 4); }
+        ctrl->abort = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tmap(&tm_w_full);
+        ptx::prefetch_tmap(&tm_w_grp);
+        ptx::prefetch_tmap(&tm_h);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(&ctrl->tmem_base, (uint32_t)p.tmem_cols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = ctrl->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            const uint64_t pol_w = ptx::policy_evict_first();
+            const uint64_t pol_h = ptx::policy_evict_last();
+            const uint32_t b_bytes = (uint32_t)p.chunk_rows * kBK * 2;
+            long long it = 0;
+            bool ok = true;
+            for (int chunk = 0; chunk < p.n_chunks && ok; ++chunk)
+                for (int t = 0; t < n_tiles && ok; ++t) {
+                    const int row0 = row_begin + t * kTileV;
+                    const int ng = min(16, g1 - (g0 + t * 16));
+                    for (int kb = 0; kb < n_kb; ++kb, ++it) {
+                        const int s = (int)(it % p.stages);
+                        const uint32_t ph = (uint32_t)((it / p.stages) & 1);
+                        if (ctrl->abort || !ptx::mbar_wait(&ctrl->empty[s], ph ^ 1)) { fail(p, ctrl, 1); ok = false; break; }
+                        uint8_t* sa = stage_base + (size_t)s * p.stage_bytes;
+                        uint8_t* sb = sa + kATileBytes;
+                        if (ng == 16) {
+                            ptx::mbar_arrive_expect_tx(&ctrl->full[s], kATileBytes + b_bytes);
+                            ptx::tma_load_2d_hint(sa, &tm_w_full, &ctrl->full[s], kb * kBK, row0, pol_w);
+                        } else {
+                            ptx::mbar_arrive_expect_tx(&ctrl->full[s], (uint32_t)ng * 1024u + b_bytes);
+                            for (int g = 0; g < ng; ++g)
+                                ptx::tma_load_2d_hint(sa + g * 1024, &tm_w_grp, &ctrl->full[s], kb * kBK, row0 + g * 8, pol_w);
+                        }
+                        ptx::tma_load_2d_hint(sb, &tm_h, &ctrl->full[s], kb * kBK, chunk * p.chunk_rows, pol_h);
+                    }
+                }
+            if (!ok) {
+                // let copies already in flight land before the CTA's shared memory goes away
+                const long long first = it > p.stages ? it - p.stages : 0;
+                for (long long j = first; j < it; ++j)
+                    ptx::mbar_wait(&ctrl->full[j % p.stages], (uint32_t)((j / p.stages) & 1), 100000000ull);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ UMMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = ptx::umma_idesc_bf16(kTileV, p.chunk_rows);
+            long long it = 0, acc_it = 0;
+            bool ok = true;
+            for (int chunk = 0; chunk < p.n_chunks && ok; ++chunk)
+                for (int t = 0; t < n_tiles && ok; ++t, ++acc_it) {
+                    const int ab = (int)(acc_it % p.n_acc);
+                    const uint32_t aph = (uint32_t)((acc_it / p.n_acc) & 1);
+                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->acc_empty[ab], aph ^ 1)) { fail(p, ctrl, 2); ok = false; break; }
+                    ptx::tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + (uint32_t)(ab * p.acc_stride);
+                    for (int kb = 0; kb < n_kb; ++kb, ++it) {
+                        const int s = (int)(it % p.stages);
+                        const uint32_t ph = (uint32_t)((it / p.stages) & 1);
+                        if (ctrl->abort || !ptx::mbar_wait(&ctrl->full[s], ph)) { fail(p, ctrl, 3); ok = false; break; }
+                        ptx::tc_fence_after();
+                        const uint32_t sa = ptx::smem_u32(stage_base + (size_t)s * p.stage_bytes);
+                        const uint32_t sb = sa + kATileBytes;
+#pragma unroll
+                        for (int k4 = 0; k4 < kBK / 16; ++k4)
+                            ptx::umma_f16(d_tmem, ptx::umma_desc_k_sw128(sa + k4 * 32), ptx::umma_desc_k_sw128(sb + k4 * 32),
+                                          idesc, (kb | k4) != 0);
+                        ptx::umma_commit(&ctrl->empty[s]);
+                    }
+                    if (ok) ptx::umma_commit(&ctrl->acc_full[ab]);
+                }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue
+        const int q = warp & 3;                       // TMEM lane quarter this warp may read
+        float* my_max = st_max + q * kMaxChunkRows;
+        int* my_idx = st_idx + q * kMaxChunkRows;
+        float* my_sum = st_sum + q * kMaxChunkRows;
+        const int n_cg = (p.chunk_rows + 31) / 32;
+        long long acc_it = 0;
+        bool ok = true;
+        for (int chunk = 0; chunk < p.n_chunks && ok; ++chunk) {
+            const int rbase = chunk * p.chunk_rows;
+            for (int c = lane; c < kMaxChunkRows; c += 32) { my_max[c] = -INFINITY; my_idx[c] = 0x7fffffff; my_sum[c] = 0.f; }
+            __syncwarp();
+            for (int t = 0; t < n_tiles && ok; ++t, ++acc_it) {
+                const int ab = (int)(acc_it % p.n_acc);
+                const uint32_t aph = (uint32_t)((acc_it / p.n_acc) & 1);
+                if (ctrl->abort || !ptx::mbar_wait(&ctrl->acc_full[ab], aph)) { fail(p, ctrl, 4); ok = false; break; }
+                ptx::tc_fence_after();
+                const int vid = row_begin + t * kTileV + q * 32 + lane;      // this thread's vocabulary id
+                const bool valid = vid < row_end;
+                for (int cg = 0; cg < n_cg; ++cg) {
+                    uint32_t r[32];
+                    ptx::tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * p.acc_stride + cg * 32), r);
+                    ptx::tmem_ld_wait();
+                    float upd_m = -INFINITY, upd_s = 0.f;
+                    int upd_i = 0x7fffffff;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int row = rbase + cg * 32 + j;
+                        if (cg * 32 + j >= p.chunk_rows || row >= p.M) break;      // warp-uniform
+                        const float v = valid ? __uint_as_float(r[j]) : -INFINITY;
+                        if (p.logits_out && valid) p.logits_out[(size_t)row * p.V + vid] = v;
+                        float m = v;
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+                        if (m == -INFINITY) continue;                               // warp-uniform
+                        const unsigned eq = __ballot_sync(0xffffffffu, v == m);
+                        float e = exp2f((v - m) * p.inv_T_log2e);
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
+                        if (lane == j) { upd_m = m; upd_s = e; upd_i = vid - lane + (__ffs(eq) - 1); }
+                    }
+                    // lane j folds column cg*32+j of this tile into the running state
+                    const int c = cg * 32 + lane;
+                    if (upd_m != -INFINITY) {
+                        const float om = my_max[c], os = my_sum[c];
+                        if (upd_m > om) {           // ids only grow along a CTA's tiles: equality keeps the older, lower id
+                            my_sum[c] = upd_s + (om == -INFINITY ? 0.f : os * exp2f((om - upd_m) * p.inv_T_log2e));
+                            my_max[c] = upd_m;
+                            my_idx[c] = upd_i;
+                        } else {
+                            my_sum[c] = os + upd_s * exp2f((upd_m - om) * p.inv_T_log2e);
+                        }
+                    }
+                }
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&ctrl->acc_empty[ab]);
+            }
+            __syncwarp();
+            if (ok) {
+                const size_t pbase = ((size_t)blockIdx.x * 4 + q) * p.M;
+                for (int c = lane; c < p.chunk_rows; c += 32) {
+                    const int row = rbase + c;
+                    if (row < p.M) {
+                        p.part_max[pbase + row] = my_max[c];
+                        p.part_idx[pbase + row] = my_idx[c];
+                        p.part_sum[pbase + row] = my_sum[c];
+                    }
+                }
+            }
+            __syncwarp();
+        }
+    }
+
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+    }
+}
+
+// Merge the per-(CTA, warp) partials of each hidden row: one warp per row, fixed order.
+__global__ void lmhead_merge_kernel(int M, int P, float inv_T, float inv_T_log2e, const float* part_max,
+                                    const int* part_idx, const float* part_sum, int32_t* argmax, float* maxlogit,
+                                    float* lse) {
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= M) return;
+    float m = -INFINITY, s = 0.f;
+    int idx = 0x7fffffff;
+    for (int k = lane; k < P; k += 32) {
+        const float pm = part_max[(size_t)k * M + row], ps = part_sum[(size_t)k * M + row];
+        const int pi = part_idx[(size_t)k * M + row];
+        if (pm == -INFINITY) continue;
+        if (pm > m || (pm == m && pi < idx)) {
+            s = ps + (m == -INFINITY ? 0.f : s * exp2f((m - pm) * inv_T_log2e));
+            m = pm; idx = pi;
+        } else {
+            s += ps * exp2f((pm - m) * inv_T_log2e);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, m, o), os = __shfl_xor_sync(0xffffffffu, s, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+        if (om == -INFINITY) continue;
+        if (om > m || (om == m && oi < idx)) {
+            s = os + (m == -INFINITY ? 0.f : s * exp2f((m - om) * inv_T_log2e));
+            m = om; idx = oi;
+        } else {
+            s += os * exp2f((om - m) * inv_T_log2e);
+        }
+    }
+    if (lane == 0) {
+        if (argmax) argmax[row] = idx;
+        if (maxlogit) maxlogit[row] = m;
+        if (lse) lse[row] = m * inv_T + logf(s);
+    }
+}
+
+// Top-kappa of each row from the fp32 logits (Eq. 6): k rounds of "best element strictly after the
+// previous pick" in the order (logit descending, id ascending).  One block per row.
+__global__ void __launch_bounds__(1024, 1)
+lmhead_topk_kernel(int V, int topk, float inv_T, const float* logits, const float* lse, int32_t* topk_id,
+                   float* topk_logprob) {
+    __shared__ float s_v[32];
+    __shared__ int s_i[32];
+    __shared__ float s_prev_v;
+    __shared__ int s_prev_i;
+    const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float* l = logits + (size_t)row * V;
+    if (tid == 0) { s_prev_v = INFINITY; s_prev_i = -1; }
+    __syncthreads();
+    for (int k = 0; k < topk; ++k) {
+        const float pv = s_prev_v;
+        const int pi = s_prev_i;
+        float bv = -INFINITY;
+        int bi = 0x7fffffff;
+        for (int v = tid; v < V; v += blockDim.x) {
+            const float x = l[v];
+            const bool after = (x < pv) || (x == pv && v > pi);
+            if (after && (x > bv || (x == bv && v < bi))) { bv = x; bi = v; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+        }
+        if (lane == 0) { s_v[warp] = bv; s_i[warp] = bi; }
+        __syncthreads();
+        if (warp == 0) {
+            bv = s_v[lane]; bi = s_i[lane];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+                if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+            }
+            if (lane == 0) {
+                s_prev_v = bv; s_prev_i = bi;
+                topk_id[(size_t)row * topk + k] = bi;
+                topk_logprob[(size_t)row * topk + k] = bv * inv_T - lse[row];
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// logits[row][tok] for a short list of (row, token) pairs: one warp per pair, fp32 dot product.
+__global__ void lmhead_gather_kernel(int n_gather, int M, int V, int H, const __nv_bfloat16* hidden,
+                                     const __nv_bfloat16* W, const int32_t* gather_row, const int32_t* gather_tok,
+                                     float* gather_logit, int* status) {
+    const int g = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (g >= n_gather) return;
+    const int row = gather_row[g], tok = gather_tok[g];
+    if (row < 0 || row >= M || tok < 0 || tok >= V) {
+        if (lane == 0) {
+            gather_logit[g] = __int_as_float(0x7fc00000);
+            if (atomicCAS(status, 0, MIRROR_DEV_CHECK) == 0) atomicExch(status + 1, 200);
+        }
+        return;
+    }
+    const __nv_bfloat162* h2 = (const __nv_bfloat162*)(hidden + (size_t)row * H);
+    const __nv_bfloat162* w2 = (const __nv_bfloat162*)(W + (size_t)tok * H);
+    float acc = 0.f;
+    for (int k = lane; k < H / 2; k += 32) {
+        const float2 a = __bfloat1622float2(h2[k]), b = __bfloat1622float2(w2[k]);
+        acc = fmaf(a.x, b.x, acc);
+        acc = fmaf(a.y, b.y, acc);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) gather_logit[g] = acc;
+}
+
+int next_pow2(int x) {
+    int p = 1;
+    while (p < x) p <<= 1;
+    return p;
+}
+
+}  // namespace
+
+mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, const void* W, int topk,
+                                   const int32_t* gather_row, const int32_t* gather_tok, int n_gather,
+                                   int32_t* argmax, float* maxlogit, float* lse, int32_t* topk_id,
+                                   float* topk_logprob, float* gather_logit, float* logits_out,
+                                   void* partial_ws, size_t partial_bytes, float* lse_scratch, cudaStream_t stream,
+                                   cudaEvent_t after_gemm) {
+    const int V = ctx->desc.vocab, H = ctx->desc.hidden;
+    LmParams p;
+    p.M = M; p.V = V; p.H = H;
+    p.n_chunks = (M + kMaxChunkRows - 1) / kMaxChunkRows;
+    p.chunk_rows = (int)align_up((size_t)((M + p.n_chunks - 1) / p.n_chunks), 16);
+    p.acc_stride = next_pow2(p.chunk_rows < 32 ? 32 : p.chunk_rows);
+    p.n_acc = 512 / p.acc_stride < kMaxAcc ? 512 / p.acc_stride : kMaxAcc;
+    p.tmem_cols = p.n_acc * p.acc_stride;
+    p.stage_bytes = kATileBytes + p.chunk_rows * kBK * 2;
+    p.stages = (kSmemBudget - kCtrlBytes - 1024) / p.stage_bytes;
+    if (p.stages > kMaxStages) p.stages = kMaxStages;
+    if (p.stages < 2) return MIRROR_ERR_SHAPE;
+    p.groups_total = (V + 7) / 8;
+    p.inv_T = 1.0f / ctx->temperature;
+    p.inv_T_log2e = p.inv_T * 1.4426950408889634f;
+    p.logits_out = logits_out;
+    p.status = ctx->d_status;
+
+    int grid = ctx->num_sms;
+    if (grid > p.groups_total) grid = p.groups_total;
+    const size_t P = (size_t)grid * 4;
+    if (partial_bytes < P * M * 12) return MIRROR_ERR_WORKSPACE;
+    p.part_max = (float*)partial_ws;
+    p.part_idx = (int*)(p.part_max + P * M);
+    p.part_sum = (float*)(p.part_idx + P * M);
+
+    CUtensorMap tm_w_full, tm_w_grp, tm_h;
+    {
+        const uint64_t dims[2] = {(uint64_t)H, (uint64_t)V};
+        const uint64_t strides[1] = {(uint64_t)H * 2};
+        const uint32_t box_full[2] = {kBK, kTileV}, box_grp[2] = {kBK, 8};
+        mirror_status st = mirror_make_tmap(ctx, &tm_w_full, W, 2, dims, strides, box_full);
+        if (st != MIRROR_OK) return st;
+        st = mirror_make_tmap(ctx, &tm_w_grp, W, 2, dims, strides, box_grp);
+        if (st != MIRROR_OK) return st;
+        const uint64_t hdims[2] = {(uint64_t)H, (uint64_t)M};
+        const uint32_t box_h[2] = {kBK, (uint32_t)p.chunk_rows};
+        st = mirror_make_tmap(ctx, &tm_h, hidden, 2, hdims, strides, box_h);
+        if (st != MIRROR_OK) return st;
+    }
+    const size_t smem = (size_t)p.stages * p.stage_bytes + kCtrlBytes + 1024;
+    if (!ctx->lm_attr_set) {
+        MIRROR_CUDA_OK(cudaFuncSetAttribute(lmhead_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+        ctx->lm_attr_set = true;
+    }
+    lmhead_kernel<<<grid, kThreads, smem, stream>>>(tm_w_full, tm_w_grp, tm_h, p);
+    ctx->launches += 1;
+    MIRROR_CUDA_OK(cudaGetLastError());
+    if (after_gemm) MIRROR_CUDA_OK(cudaEventRecord(after_gemm, stream));
+
+    float* lse_dst = lse ? lse : (topk > 0 ? lse_scratch : nullptr);
+    if (argmax || maxlogit || lse_dst) {
+        const int warps = 8;
+        lmhead_merge_kernel<<<(M + warps - 1) / warps, warps * 32, 0, stream>>>(M, (int)P, p.inv_T, p.inv_T_log2e, p.part_max,
+                                                                               p.part_idx, p.part_sum, argmax, maxlogit, lse_dst);
+        ctx->launches += 1;
+        MIRROR_CUDA_OK(cudaGetLastError());
+    }
+    if (topk > 0) {
+        lmhead_topk_kernel<<<M, 1024, 0, stream>>>(V, topk, p.inv_T, logits_out, lse_dst, topk_id, topk_logprob);
+        ctx->launches += 1;
+        MIRROR_CUDA_OK(cudaGetLastError());
+    }
+    if (n_gather > 0) {
+        const int warps = 8;
+        lmhead_gather_kernel<<<(n_gather + warps - 1) / warps, warps * 32, 0, stream>>>(
+            n_gather, M, V, H, (const __nv_bfloat16*)hidden, (const __nv_bfloat16*)W, gather_row, gather_tok, gather_logit,
+            ctx->d_status);
+        ctx->launches += 1;
+        MIRROR_CUDA_OK(cudaGetLastError());
+    }
+    return MIRROR_OK;
+}
+
+extern "C" mirror_status mirror_lmhead_reduce(mirror_ctx* ctx, const void* hidden, int M, const void* W, int topk,
+                                              const int32_t* gather_row, const int32_t* gather_tok, int n_gather,
+                                              int32_t* argmax, float* maxlogit, float* lse, int32_t* topk_id,
+                                              float* topk_logprob, float* gather_logit, float* logits_out,
+                                              void* stream) {
+    if (!ctx || !hidden || !W || M <= 0 || topk < 0 || n_gather < 0) return MIRROR_ERR_ARG;
+    if (topk > MIRROR_MAX_TOPK || topk > ctx->desc.vocab) return MIRROR_ERR_SHAPE;
+    if (topk > 0 && (!topk_id || !topk_logprob)) return MIRROR_ERR_ARG;
+    if (n_gather > 0 && (!gather_row || !gather_tok || !gather_logit)) return MIRROR_ERR_ARG;
+    if (((uintptr_t)hidden & 15) || ((uintptr_t)W & 15)) return MIRROR_ERR_ARG;
+    if (!ctx->ws) return MIRROR_ERR_WORKSPACE;
+    MIRROR_CUDA_OK(cudaSetDevice(ctx->device));
+    MirrorWsLayout L;
+    mirror_ws_layout(ctx, (size_t)M, &L);
+    size_t need = L.end_lmhead;
+    float* lse_scratch = (float*)((uint8_t*)ctx->ws + L.lse);
+    if (topk > 0 && !logits_out) {
+        logits_out = (float*)((uint8_t*)ctx->ws + L.logits);
+        need = L.end_logits;
+    }
+    if (ctx->ws_bytes < need) return MIRROR_ERR_WORKSPACE;
+    return mirror_lmhead_launch(ctx, hidden, M, W, topk, gather_row, gather_tok, n_gather, argmax, maxlogit, lse, topk_id,
+                                topk_logprob, gather_logit, logits_out, (uint8_t*)ctx->ws + L.lm_partial, L.lm_partial_bytes, lse_scratch,
+                                (cudaStream_t)stream);
+}

@@ -1,0 +1,145 @@
+"""GPU parity: mirror_accept_select against the oracle's acceptance rules (bit-exact outputs)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2510_13161_b200 import inputs as I
+from tests.helpers import make_mirror
+
+pytestmark = pytest.mark.gpu
+FIELDS = ["n_accepted", "best_branch", "decide_row", "n_emitted", "emitted", "accepted_nodes", "reuse_slot"]
+
+
+def cfg_for(V, kappa, gamma, B):
+    return I.VerifyConfig("t", 256, 4, 2, 64, 1, B, 16, 16, kappa, gamma, V, "greedy")
+
+
+def planted_greedy_case(B, kappa, gamma, V, seed, parent=None):
+    """Random tokens / target argmax with agreement planted to random depths on random branches."""
+    rng = np.random.default_rng(seed)
+    par = I.comb_parent(kappa, gamma) if parent is None else parent
+    n = len(par)
+    tok = rng.integers(0, V, size=(B, n)).astype(np.int32)
+    am = rng.integers(0, V, size=(B, n)).astype(np.int32)
+    paths, plen = O.branches(par, gamma)
+    for b in range(B):
+        for i in range(len(paths)):
+            depth = rng.integers(0, plen[i] + 1)
+            for j in range(depth):
+                c = paths[i, j]
+                am[b, par[c]] = tok[b, c]
+    return par, tok, am
+
+
+@pytest.mark.parametrize("kappa,gamma,B", [(2, 4, 1), (4, 4, 3), (8, 6, 8), (8, 8, 16), (1, 7, 2), (8, 7, 1), (1, 1, 1)])
+@pytest.mark.parametrize("emit_bonus", [True, False])
+def test_greedy_matches_oracle_bit_exact(kappa, gamma, B, emit_bonus):
+    V = 97
+    m = make_mirror(cfg_for(V, kappa, gamma, B))
+    for seed in range(3):
+        par, tok, am = planted_greedy_case(B, kappa, gamma, V, seed)
+        cand = np.random.default_rng(seed).integers(0, V, size=(B, len(par), 5)).astype(np.int32)
+        # make some reuse hits likely
+        cand[:, :, 2] = am
+        if seed == 1:
+            cand[:, :, 2] = -7
+        ref = O.accept_greedy(tok, am, par, gamma, emit_bonus, cand)
+        tok_d = torch.from_numpy(tok).cuda(); am_d = torch.from_numpy(am).cuda(); cand_d = torch.from_numpy(cand).cuda()
+        tree = m.tree(tok_d, kappa, gamma)
+        acc = m.accept_in(0, emit_bonus, target_argmax=am_d, cand_ids=cand_d)
+        got = m.mirror_accept_select(tree, acc).cpu()
+        for f in FIELDS:
+            np.testing.assert_array_equal(got[f], ref[f], err_msg=f)
+        assert m.device_status() == (0, 0)
+
+
+def test_greedy_general_tree_and_all_accept():
+    V, gamma = 50, 5
+    par = [-1, 0, 1, 1, 0, 4, 5, 5, 2, 8, 3]
+    m = make_mirror(cfg_for(V, 1, gamma, 4))
+    for seed in range(4):
+        par_, tok, am = planted_greedy_case(4, 0, gamma, V, seed, parent=par)
+        if seed == 3:                       # everything agrees: every branch fully accepted, lowest index wins
+            for b in range(4):
+                for c in range(1, len(par)):
+                    am[b, par[c]] = tok[b, c] = 7
+        ref = O.accept_greedy(tok, am, par, gamma)
+        tok_d = torch.from_numpy(tok).cuda(); am_d = torch.from_numpy(am).cuda()
+        tree = m.tree(tok_d, 0, gamma, parent=par)
+        got = m.mirror_accept_select(tree, m.accept_in(0, True, target_argmax=am_d)).cpu()
+        for f in FIELDS:
+            np.testing.assert_array_equal(got[f], ref[f], err_msg=f)
+
+
+def spec_case(B, kappa, gamma, V, seed, peaked=False):
+    g = torch.Generator().manual_seed(seed)
+    n = 1 + kappa * gamma
+    logits = torch.randn((B * n, V), generator=g) * (3.0 if peaked else 1.0)
+    qp = torch.softmax(torch.randn((B, n - 1, V), generator=g) * (3.0 if peaked else 1.0), -1)
+    tok = torch.randint(0, V, (B, n), generator=g, dtype=torch.int32)
+    # draw the drafted tokens from q so that acceptance actually happens
+    for b in range(B):
+        for c in range(1, n):
+            tok[b, c] = int(torch.multinomial(qp[b, c - 1], 1, generator=g))
+    ua = torch.rand((B, n), generator=g); ur = torch.rand((B, n), generator=g)
+    return logits.float(), qp.float(), tok, ua.float(), ur.float()
+
+
+@pytest.mark.parametrize("kappa,gamma,B,V,T", [(1, 4, 4, 1000, 1.0), (2, 4, 3, 1024, 1.0), (8, 6, 8, 5003, 0.7),
+                                               (4, 4, 2, 152064, 1.0), (8, 8, 2, 128256, 1.3)])
+def test_spec_sampling_matches_oracle(kappa, gamma, B, V, T):
+    m = make_mirror(cfg_for(V, kappa, gamma, B), temperature=T)
+    par = I.comb_parent(kappa, gamma)
+    accepted_total = 0
+    for seed in range(3):
+        logits, qp, tok, ua, ur = spec_case(B, kappa, gamma, V, seed, peaked=(seed == 2))
+        if seed == 1:
+            qp[:, 0] = torch.softmax(logits.view(B, -1, V)[:, 0] / T, -1)     # p == q at the first node: residual has no mass
+        lse = torch.logsumexp(logits.double() / T, -1).float()
+        cand = torch.topk(logits, 4, dim=-1).indices.to(torch.int32)
+        ref = O.accept_spec(tok.numpy(), logits.numpy(), lse.numpy(), qp.numpy(), ua.numpy(), ur.numpy(), par, gamma,
+                            True, T, cand.numpy())
+        tree = m.tree(tok.cuda(), kappa, gamma)
+        acc = m.accept_in(1, True, logits=logits.cuda(), lse=lse.cuda(), q_probs=qp.cuda(), u_accept=ua.cuda(),
+                          u_resample=ur.cuda(), cand_ids=cand.cuda())
+        got = m.mirror_accept_select(tree, acc).cpu()
+        assert m.device_status() == (0, 0)
+        for b in range(B):
+            same = all(np.array_equal(got[f][b], ref[f][b]) for f in FIELDS)
+            # a disagreement is tolerated only on a knife edge of the fp64 decision (exp implementations differ in the last ulp)
+            assert same or ref["margin"][b] < 1e-9, (b, ref["margin"][b], {f: (got[f][b], ref[f][b]) for f in FIELDS})
+        accepted_total += int(ref["n_accepted"].sum())
+    assert accepted_total > 0
+
+
+def test_spec_root_only_tree_draws_from_the_root_row():
+    V, B = 777, 5
+    m = make_mirror(cfg_for(V, 0, 0, B))
+    g = torch.Generator().manual_seed(0)
+    logits = torch.randn((B, V), generator=g)
+    lse = torch.logsumexp(logits.double(), -1).float()
+    tok = torch.zeros((B, 1), dtype=torch.int32)
+    ua = torch.rand((B, 1), generator=g); ur = torch.rand((B, 1), generator=g)
+    ref = O.accept_spec(tok.numpy(), logits.numpy(), lse.numpy(), np.zeros((B, 0, V), np.float32), ua.numpy(), ur.numpy(), [-1], 0)
+    tree = m.tree(tok.cuda(), 0, 0)
+    acc = m.accept_in(1, True, logits=logits.cuda(), lse=lse.cuda(), u_accept=ua.cuda(), u_resample=ur.cuda())
+    got = m.mirror_accept_select(tree, acc).cpu()
+    for f in ("n_accepted", "n_emitted", "decide_row", "reuse_slot"):
+        np.testing.assert_array_equal(got[f], ref[f])
+    np.testing.assert_array_equal(got["emitted"][:, 0], ref["emitted"][:, 0])
+
+
+def test_bad_arguments_are_rejected_on_the_host():
+    from paper_2510_13161_b200.binding import MirrorError
+    m = make_mirror(cfg_for(100, 2, 2, 1))
+    tok = torch.zeros((1, 5), dtype=torch.int32).cuda()
+    with pytest.raises(MirrorError) as e:
+        m.mirror_accept_select(m.tree(tok, 2, 2), m.accept_in(0, True))        # no target_argmax
+    assert e.value.code == 1
+    with pytest.raises(MirrorError) as e:
+        m.mirror_accept_select(m.tree(tok, 3, 2), m.accept_in(0, True, target_argmax=tok))   # n != 1 + kappa*gamma
+    assert e.value.code == 2
+    with pytest.raises(MirrorError) as e:
+        m.mirror_accept_select(m.tree(tok, 0, 2, parent=[-1, 0, 2, 1, 0]), m.accept_in(0, True, target_argmax=tok))
+    assert e.value.code == 2

@@ -1,0 +1,131 @@
+"""GPU parity: mirror_attn_verify (branch-tree attention over a paged KV cache) against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2510_13161_b200 import inputs as I
+from tests.helpers import make_mirror, oracle_attention
+
+pytestmark = pytest.mark.gpu
+
+ATTN_TOL = 2e-2            # stated bound: max-abs of bf16 output against the fp64 oracle
+
+
+def run_gpu(m, x, want_lse=True):
+    kv = m.kv(x.k_pool, x.v_pool, x.page_table, x.prefix_len)
+    tree = m.tree(x.tokens, x.cfg.kappa, x.cfg.gamma, parent=x.parent)
+    L, B, n, Hq, d = x.q.shape
+    lse = torch.empty((L, B, Hq, n), dtype=torch.float32, device="cuda") if want_lse else None
+    out = m.mirror_attn_verify(kv, tree, x.q, x.k_new, x.v_new, lse_out=lse)
+    torch.cuda.synchronize()
+    assert m.device_status() == (0, 0)
+    return out, lse
+
+
+def compare(out, lse, ref, layers, rel=1e-2):
+    worst = 0.0
+    for l in layers:
+        o_ref, lse_ref = ref[l]
+        got = out[l].float().cpu().numpy().astype(np.float64)
+        err = np.abs(got - o_ref).max()
+        scale = np.abs(o_ref).max()
+        assert err < ATTN_TOL, (l, err)
+        assert err <= rel * scale + 1e-5, (l, err, scale)      # tighter, magnitude-aware gate (bf16 output rounding)
+        if lse is not None:
+            np.testing.assert_allclose(lse[l].cpu().numpy(), lse_ref, atol=2e-3)
+        worst = max(worst, err / max(scale, 1e-30))
+    return worst
+
+
+def small(**kw):
+    base = dict(hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=64, layers=2, batch=2, prefix_lo=1, prefix_hi=300,
+                kappa=2, gamma=4, vocab=64, mode="greedy", kv_std=1.0)
+    base.update(kw)
+    return I.VerifyConfig("t", **base)
+
+
+def test_tiny_config():
+    cfg = I.CONFIGS["tiny"]
+    x = I.gen_verify_inputs(cfg, 0, "cuda", with_lm_head=False)
+    m = make_mirror(cfg)
+    out, lse = run_gpu(m, x)
+    compare(out, lse, oracle_attention(x), range(cfg.layers))
+
+
+@pytest.mark.parametrize("kw", [
+    dict(),                                                          # d = 64, ragged prefixes, 2 layers
+    dict(head_dim=128, n_q_heads=8, n_kv_heads=2, hidden=1024),      # d = 128
+    dict(head_dim=128, n_q_heads=10, n_kv_heads=2, hidden=1280, kappa=4, gamma=4, batch=3, layers=3),   # G = 5 (85 rows)
+    dict(prefix_lo=0, prefix_hi=0),                                  # empty prefix: tree tokens only
+    dict(prefix_lo=16, prefix_hi=16, batch=1),                       # exactly one full page
+    dict(prefix_lo=15, prefix_hi=17, batch=4),                       # around a page boundary
+    dict(head_dim=128, n_q_heads=16, n_kv_heads=2, hidden=2048, kappa=4, gamma=4, batch=2, prefix_hi=700),   # 136 rows: two row blocks
+    dict(head_dim=128, n_q_heads=16, n_kv_heads=2, hidden=2048, kappa=8, gamma=8, batch=2, prefix_hi=500),   # 520 rows: five row blocks, n = 65
+    dict(kappa=8, gamma=15, batch=1, prefix_hi=100),                 # n = 121 tree tokens: two tree tiles
+    dict(prefix_lo=3000, prefix_hi=5000, batch=2, layers=1),         # long prefixes: units cut across many CTAs
+])
+def test_shapes_and_ragged_cases(kw):
+    cfg = small(**kw)
+    x = I.gen_verify_inputs(cfg, 1, "cuda", with_lm_head=False)
+    m = make_mirror(cfg)
+    out, lse = run_gpu(m, x)
+    compare(out, lse, oracle_attention(x), range(cfg.layers))
+
+
+def test_general_tree_mask():
+    cfg = small(head_dim=128, n_q_heads=8, n_kv_heads=2, hidden=1024, kappa=1, gamma=6, batch=2)
+    par = I.random_tree_parent(24, 5, max_depth=6)
+    x = I.gen_verify_inputs(cfg, 2, "cuda", parent=par, with_lm_head=False)
+    m = make_mirror(cfg)
+    out, lse = run_gpu(m, x)
+    compare(out, lse, oracle_attention(x), range(cfg.layers))
+
+
+def test_peaked_scores_exercise_rescaling_and_split_merge():
+    """Scores with a wide spread and a few dominant keys placed late in the prefix and right at the cuts between
+    CTAs, so that the running maximum moves and partials with very different maxima are merged."""
+    cfg = small(head_dim=128, n_q_heads=8, n_kv_heads=2, hidden=1024, prefix_lo=4096, prefix_hi=4096, batch=1, layers=1)
+    x = I.gen_verify_inputs(cfg, 3, "cuda", with_lm_head=False, q_std=3.0)
+    # plant keys aligned with the root's query of head 0 at assorted positions
+    qv = x.q[0, 0, 0, 0].float()
+    for t, gain in ((5, 0.5), (1023, 0.8), (1024, 1.0), (2047, 1.2), (3000, 1.5), (4095, 2.0)):
+        page = int(x.page_table[0, t // 16])
+        x.k_pool[0, page, 0, t % 16] = (qv * gain / qv.norm() * 4.0).to(torch.bfloat16)
+    m = make_mirror(cfg)
+    out, lse = run_gpu(m, x)
+    ref = oracle_attention(x)
+    compare(out, lse, ref, [0], rel=1.5e-2)
+
+
+def test_run_to_run_determinism_and_workspace_reuse():
+    cfg = small(head_dim=128, n_q_heads=8, n_kv_heads=2, hidden=1024, prefix_lo=500, prefix_hi=2000, batch=3, layers=2)
+    x = I.gen_verify_inputs(cfg, 4, "cuda", with_lm_head=False)
+    m = make_mirror(cfg)
+    a, _ = run_gpu(m, x)
+    b, _ = run_gpu(m, x)
+    assert torch.equal(a, b)
+
+
+def test_full_size_14b_sampled_layers():
+    """The bench launch configuration (48 layers, prefix 2048, 17 nodes): all rows of sampled layers."""
+    cfg = I.CONFIGS["qwen14b"]
+    x = I.gen_verify_inputs(cfg, 0, "cuda", with_lm_head=False)
+    m = make_mirror(cfg)
+    out, lse = run_gpu(m, x)
+    layers = [0, 24, 47, 13, 38]
+    worst = compare(out, lse, oracle_attention(x, layers), layers)
+    print("worst relative error", worst)
+
+
+def test_out_of_range_page_is_reported_not_faulted():
+    cfg = small(batch=1, prefix_lo=64, prefix_hi=64, layers=1)
+    x = I.gen_verify_inputs(cfg, 6, "cuda", with_lm_head=False)
+    x.page_table[0, 1] = 10 ** 6
+    m = make_mirror(cfg)
+    kv = m.kv(x.k_pool, x.v_pool, x.page_table, x.prefix_len)
+    tree = m.tree(x.tokens, cfg.kappa, cfg.gamma)
+    m.mirror_attn_verify(kv, tree, x.q, x.k_new, x.v_new)
+    code, detail = m.device_status()
+    assert code == 6 and detail in (400, 401)
+    assert m.device_status() == (0, 0)        # sticky status is cleared once read

@@ -1,0 +1,107 @@
+"""GPU parity of the fused verify step (attention -> LM head -> acceptance) against the oracle chain."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2510_13161_b200 import inputs as I
+from tests.helpers import make_mirror, oracle_attention
+
+pytestmark = pytest.mark.gpu
+FIELDS = ["n_accepted", "best_branch", "decide_row", "n_emitted", "emitted", "accepted_nodes", "reuse_slot"]
+
+
+def oracle_step_greedy(x, logits=None):
+    """Oracle chain: last-layer attention (fp64, unrounded) -> LM head -> argmax -> greedy acceptance."""
+    cfg = x.cfg
+    L = x.q.shape[0]
+    if logits is None:
+        if x.hidden is not None:
+            logits = O.lmhead_logits(I.bf16_bits(x.hidden), I.bf16_bits(x.W))
+        else:
+            out, _ = oracle_attention(x, [L - 1])[L - 1]
+            logits = O.lmhead_logits(out.reshape(-1, cfg.hidden), I.bf16_bits(x.W))
+    red = O.row_reduce(logits)
+    return logits, red
+
+
+def gpu_step(m, x, mode=0, **acc_kw):
+    kv = m.kv(x.k_pool, x.v_pool, x.page_table, x.prefix_len)
+    tree = m.tree(x.tokens, x.cfg.kappa, x.cfg.gamma, parent=x.parent)
+    attn_out = torch.empty_like(x.q)
+    argmax = torch.empty(x.tokens.numel(), dtype=torch.int32, device="cuda")
+    acc = m.accept_in(mode, True, **acc_kw)
+    res = m.mirror_verify_step(kv, tree, x.q, x.k_new, x.v_new, x.hidden, x.W, acc, attn_out, argmax_out=argmax)
+    torch.cuda.synchronize()
+    assert m.device_status() == (0, 0)
+    return res.cpu(), argmax.cpu().numpy(), attn_out
+
+
+def count_flips(argmax_gpu, logits, tol=2e-3):
+    red = O.row_reduce(logits)
+    flips = np.nonzero(argmax_gpu != red["argmax"])[0]
+    for r in flips:      # a flip is legitimate only when the oracle's gap is inside the logit error bound
+        assert logits[r, red["argmax"][r]] - logits[r, argmax_gpu[r]] < tol, r
+    return len(flips)
+
+
+def test_tiny_config_uniform_and_planted():
+    cfg = I.CONFIGS["tiny"]
+    x = I.gen_verify_inputs(cfg, 0, "cuda")
+    m = make_mirror(cfg)
+    logits, red = oracle_step_greedy(x)
+    got, am, _ = gpu_step(m, x)
+    flips = count_flips(am, logits)
+    tok = x.tokens.cpu().numpy()
+    ref = O.accept_greedy(tok, am.reshape(tok.shape), x.parent, cfg.gamma)      # identical argmax in: outputs bit-exact
+    for f in FIELDS:
+        np.testing.assert_array_equal(got[f], ref[f], err_msg=f)
+    # planted variant: branch 1 copies the oracle's target argmax for its first 3 positions
+    g = cfg.gamma
+    tok2 = tok.copy()
+    rows = [0, 1 + g, 2 + g]
+    for j, r in enumerate(rows):
+        tok2[0, 1 + g + j] = red["argmax"][r]
+    x.tokens = torch.from_numpy(tok2).cuda()
+    got, am, _ = gpu_step(m, x)
+    ref = O.accept_greedy(tok2, red["argmax"].reshape(tok.shape), x.parent, cfg.gamma)
+    if flips == 0 and count_flips(am, logits) == 0:
+        for f in FIELDS:
+            np.testing.assert_array_equal(got[f], ref[f], err_msg=f)
+        assert got["n_accepted"][0] >= 3 and got["best_branch"][0] == 1
+
+
+def test_spec_sampling_step_small():
+    cfg = I.VerifyConfig("s", 512, 8, 2, 64, 2, 3, 40, 200, 3, 3, 2000, "spec_sampling")
+    x = I.gen_verify_inputs(cfg, 1, "cuda")
+    # draft tokens drawn from q so that some are accepted
+    g = torch.Generator().manual_seed(0)
+    tok = x.tokens.cpu()
+    for b in range(cfg.batch):
+        for c in range(1, cfg.n_nodes):
+            tok[b, c] = int(torch.multinomial(x.q_probs[b, c - 1].cpu(), 1, generator=g))
+    x.tokens = tok.cuda()
+    m = make_mirror(cfg)
+    got, am, attn_out = gpu_step(m, x, 1, q_probs=x.q_probs, u_accept=x.u_accept, u_resample=x.u_resample)
+    # feed the oracle the identical logits the GPU used: recompute them with the same kernel and the spill on
+    rows = attn_out[-1].reshape(cfg.rows, cfg.hidden)
+    lm = m.mirror_lmhead_reduce(rows, x.W, want_logits=True)
+    ref = O.accept_spec(tok.numpy(), lm["logits"].cpu().numpy(), lm["lse"].cpu().numpy(), x.q_probs.cpu().numpy(),
+                        x.u_accept.cpu().numpy(), x.u_resample.cpu().numpy(), x.parent, cfg.gamma)
+    for b in range(cfg.batch):
+        same = all(np.array_equal(got[f][b], ref[f][b]) for f in FIELDS)
+        assert same or ref["margin"][b] < 1e-9, (b, ref["margin"][b])
+
+
+def test_full_size_14b_step_flip_count():
+    cfg = I.CONFIGS["qwen14b"]
+    x = I.gen_verify_inputs(cfg, 0, "cuda")
+    m = make_mirror(cfg)
+    got, am, attn_out = gpu_step(m, x)
+    logits, red = oracle_step_greedy(x)
+    flips = count_flips(am, logits)
+    print("end-to-end argmax flips:", flips, "of", len(am))
+    tok = x.tokens.cpu().numpy()
+    ref = O.accept_greedy(tok, am.reshape(tok.shape), x.parent, cfg.gamma)
+    for f in FIELDS:
+        np.testing.assert_array_equal(got[f], ref[f], err_msg=f)
