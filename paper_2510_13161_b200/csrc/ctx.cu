@@ -150,7 +150,7 @@ void mirror_ws_layout(const mirror_ctx* ctx, size_t M, MirrorWsLayout* out) {
     at += L.attn_partial_bytes;
     L.end_attn = at;
     L.lm_partial = at;
-    L.lm_partial_bytes = align_up((size_t)ctx->num_sms * 4 * M * 12, 256);
+    L.lm_partial_bytes = align_up((size_t)ctx->num_sms * M * 12, 256);
     at += L.lm_partial_bytes;
     L.lse = at;
     at += align_up(M * sizeof(float), 256);

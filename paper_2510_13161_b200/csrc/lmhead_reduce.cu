@@ -20,6 +20,7 @@
 //
 // Every mbarrier wait is bounded; on expiry the kernel records MIRROR_DEV_TIMEOUT and unwinds.
 #include <math.h>
+#include <stdlib.h>
 
 #include "mirror_internal.h"
 
@@ -40,10 +41,11 @@ struct LmParams {
     int n_chunks, chunk_rows;           // hidden rows are processed in chunks of chunk_rows (multiple of 16)
     int acc_stride, n_acc, tmem_cols;   // TMEM columns per accumulator buffer, number of buffers, allocation
     int stages, stage_bytes;
+    int k_group;                        // producer batching: K blocks requested together
     int groups_total;                   // ceil(V / 8)
     float inv_T, inv_T_log2e;
     float* logits_out;                  // nullable [M, V]
-    float* part_max;                    // [grid*4][M]
+    float* part_max;                    // [grid][M]
     int* part_idx;
     float* part_sum;
     int* status;
@@ -108,63 +110,97 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tm_w_full, const __grid_consta
             const uint64_t pol_w = ptx::policy_evict_first();
             const uint64_t pol_h = ptx::policy_evict_last();
             const uint32_t b_bytes = (uint32_t)p.chunk_rows * kBK * 2;
-            long long it = 0;
+            // pipeline position kept as (stage, phase) counters: this single thread is on the critical path
+            // and 64-bit divisions by a run-time stage count would cost more than the copies it issues
+            int s0 = 0;                 // stage of the next K block to issue
+            uint32_t ph0 = 0;           // its phase bit
+            int issued = 0;
             bool ok = true;
             for (int chunk = 0; chunk < p.n_chunks && ok; ++chunk)
                 for (int t = 0; t < n_tiles && ok; ++t) {
                     const int row0 = row_begin + t * kTileV;
                     const int ng = min(16, g1 - (g0 + t * 16));
-                    for (int kb = 0; kb < n_kb; ++kb, ++it) {
-                        const int s = (int)(it % p.stages);
-                        const uint32_t ph = (uint32_t)((it / p.stages) & 1);
-                        if (ctrl->abort || !ptx::mbar_wait(&ctrl->empty[s], ph ^ 1)) { fail(p, ctrl, 1); ok = false; break; }
-                        uint8_t* sa = stage_base + (size_t)s * p.stage_bytes;
-                        uint8_t* sb = sa + kATileBytes;
-                        if (ng == 16) {
-                            ptx::mbar_arrive_expect_tx(&ctrl->full[s], kATileBytes + b_bytes);
-                            ptx::tma_load_2d_hint(sa, &tm_w_full, &ctrl->full[s], kb * kBK, row0, pol_w);
-                        } else {
-                            ptx::mbar_arrive_expect_tx(&ctrl->full[s], (uint32_t)ng * 1024u + b_bytes);
-                            for (int g = 0; g < ng; ++g)
-                                ptx::tma_load_2d_hint(sa + g * 1024, &tm_w_grp, &ctrl->full[s], kb * kBK, row0 + g * 8, pol_w);
+                    const uint32_t tx_bytes = (uint32_t)ng * 1024u + b_bytes;
+                    // K blocks are issued in batches of k_group so that the copies that touch one DRAM page
+                    // (consecutive 128-byte pieces of one weight row) are requested together instead of one
+                    // pipeline stage apart.
+                    for (int kb0 = 0; kb0 < n_kb && ok; kb0 += p.k_group) {
+                        const int nk = min(p.k_group, n_kb - kb0);
+                        {
+                            int s = s0;
+                            uint32_t ph = ph0;
+                            for (int j = 0; j < nk; ++j) {
+                                if (ctrl->abort || !ptx::mbar_wait(&ctrl->empty[s], ph ^ 1)) { fail(p, ctrl, 1); ok = false; break; }
+                                ptx::mbar_arrive_expect_tx(&ctrl->full[s], tx_bytes);
+                                if (++s == p.stages) { s = 0; ph ^= 1; }
+                            }
                         }
-                        ptx::tma_load_2d_hint(sb, &tm_h, &ctrl->full[s], kb * kBK, chunk * p.chunk_rows, pol_h);
+                        if (!ok) break;
+                        // (the tensor maps are named directly: a pointer chosen at run time would make the compiler
+                        // copy the kernel parameters to local memory)
+                        if (ng == 16) {
+                            int s = s0;
+                            for (int j = 0; j < nk; ++j) {
+                                ptx::tma_load_2d_hint(stage_base + s * p.stage_bytes, &tm_w_full, &ctrl->full[s],
+                                                      (kb0 + j) * kBK, row0, pol_w);
+                                if (++s == p.stages) s = 0;
+                            }
+                        } else {
+                            for (int g = 0; g < ng; ++g) {
+                                int s = s0;
+                                for (int j = 0; j < nk; ++j) {
+                                    ptx::tma_load_2d_hint(stage_base + s * p.stage_bytes + g * 1024, &tm_w_grp, &ctrl->full[s],
+                                                          (kb0 + j) * kBK, row0 + g * 8, pol_w);
+                                    if (++s == p.stages) s = 0;
+                                }
+                            }
+                        }
+                        for (int j = 0; j < nk; ++j) {
+                            ptx::tma_load_2d_hint(stage_base + s0 * p.stage_bytes + kATileBytes, &tm_h, &ctrl->full[s0],
+                                                  (kb0 + j) * kBK, chunk * p.chunk_rows, pol_h);
+                            if (++s0 == p.stages) { s0 = 0; ph0 ^= 1; }
+                        }
+                        issued += nk;
                     }
                 }
             if (!ok) {
                 // let copies already in flight land before the CTA's shared memory goes away
-                const long long first = it > p.stages ? it - p.stages : 0;
-                for (long long j = first; j < it; ++j)
-                    ptx::mbar_wait(&ctrl->full[j % p.stages], (uint32_t)((j / p.stages) & 1), 100000000ull);
+                const int back = issued < p.stages ? issued : p.stages;
+                int s = s0;
+                uint32_t ph = ph0;
+                for (int j = 0; j < back; ++j) {
+                    if (--s < 0) { s = p.stages - 1; ph ^= 1; }
+                    ptx::mbar_wait(&ctrl->full[s], ph, 100000000ull);
+                }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ UMMA issuer
         if (lane == 0) {
             const uint32_t idesc = ptx::umma_idesc_bf16(kTileV, p.chunk_rows);
-            long long it = 0, acc_it = 0;
+            const uint32_t stage_u32 = ptx::smem_u32(stage_base);
+            int s = 0, ab = 0;
+            uint32_t ph = 0, aph = 0;
             bool ok = true;
             for (int chunk = 0; chunk < p.n_chunks && ok; ++chunk)
-                for (int t = 0; t < n_tiles && ok; ++t, ++acc_it) {
-                    const int ab = (int)(acc_it % p.n_acc);
-                    const uint32_t aph = (uint32_t)((acc_it / p.n_acc) & 1);
+                for (int t = 0; t < n_tiles && ok; ++t) {
                     if (ctrl->abort || !ptx::mbar_wait(&ctrl->acc_empty[ab], aph ^ 1)) { fail(p, ctrl, 2); ok = false; break; }
                     ptx::tc_fence_after();
                     const uint32_t d_tmem = tmem_base + (uint32_t)(ab * p.acc_stride);
-                    for (int kb = 0; kb < n_kb; ++kb, ++it) {
-                        const int s = (int)(it % p.stages);
-                        const uint32_t ph = (uint32_t)((it / p.stages) & 1);
+                    for (int kb = 0; kb < n_kb; ++kb) {
                         if (ctrl->abort || !ptx::mbar_wait(&ctrl->full[s], ph)) { fail(p, ctrl, 3); ok = false; break; }
                         ptx::tc_fence_after();
-                        const uint32_t sa = ptx::smem_u32(stage_base + (size_t)s * p.stage_bytes);
+                        const uint32_t sa = stage_u32 + (uint32_t)(s * p.stage_bytes);
                         const uint32_t sb = sa + kATileBytes;
 #pragma unroll
                         for (int k4 = 0; k4 < kBK / 16; ++k4)
                             ptx::umma_f16(d_tmem, ptx::umma_desc_k_sw128(sa + k4 * 32), ptx::umma_desc_k_sw128(sb + k4 * 32),
                                           idesc, (kb | k4) != 0);
                         ptx::umma_commit(&ctrl->empty[s]);
+                        if (++s == p.stages) { s = 0; ph ^= 1; }
                     }
                     if (ok) ptx::umma_commit(&ctrl->acc_full[ab]);
+                    if (++ab == p.n_acc) { ab = 0; aph ^= 1; }
                 }
         }
     } else {
@@ -174,15 +210,14 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tm_w_full, const __grid_consta
         int* my_idx = st_idx + q * kMaxChunkRows;
         float* my_sum = st_sum + q * kMaxChunkRows;
         const int n_cg = (p.chunk_rows + 31) / 32;
-        long long acc_it = 0;
+        int ab = 0;
+        uint32_t aph = 0;
         bool ok = true;
-        for (int chunk = 0; chunk < p.n_chunks && ok; ++chunk) {
+        for (int chunk = 0; chunk < p.n_chunks; ++chunk) {
             const int rbase = chunk * p.chunk_rows;
             for (int c = lane; c < kMaxChunkRows; c += 32) { my_max[c] = -INFINITY; my_idx[c] = 0x7fffffff; my_sum[c] = 0.f; }
             __syncwarp();
-            for (int t = 0; t < n_tiles && ok; ++t, ++acc_it) {
-                const int ab = (int)(acc_it % p.n_acc);
-                const uint32_t aph = (uint32_t)((acc_it / p.n_acc) & 1);
+            for (int t = 0; t < n_tiles && ok; ++t) {
                 if (ctrl->abort || !ptx::mbar_wait(&ctrl->acc_full[ab], aph)) { fail(p, ctrl, 4); ok = false; break; }
                 ptx::tc_fence_after();
                 const int vid = row_begin + t * kTileV + q * 32 + lane;      // this thread's vocabulary id
@@ -225,20 +260,35 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tm_w_full, const __grid_consta
                 ptx::tc_fence_before();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&ctrl->acc_empty[ab]);
+                if (++ab == p.n_acc) { ab = 0; aph ^= 1; }
             }
-            __syncwarp();
-            if (ok) {
-                const size_t pbase = ((size_t)blockIdx.x * 4 + q) * p.M;
-                for (int c = lane; c < p.chunk_rows; c += 32) {
+            // fold the four warps' states (disjoint vocabulary rows) into one partial per hidden row
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (ok && !ctrl->abort) {
+                const size_t pbase = (size_t)blockIdx.x * p.M;
+                for (int c = (warp - 2) * 32 + lane; c < p.chunk_rows; c += 128) {
                     const int row = rbase + c;
-                    if (row < p.M) {
-                        p.part_max[pbase + row] = my_max[c];
-                        p.part_idx[pbase + row] = my_idx[c];
-                        p.part_sum[pbase + row] = my_sum[c];
+                    if (row >= p.M) continue;
+                    float m = -INFINITY, s = 0.f;
+                    int idx = 0x7fffffff;
+#pragma unroll
+                    for (int w = 0; w < 4; ++w) {
+                        const float pm = st_max[w * kMaxChunkRows + c], ps = st_sum[w * kMaxChunkRows + c];
+                        const int pi = st_idx[w * kMaxChunkRows + c];
+                        if (pm == -INFINITY) continue;
+                        if (pm > m || (pm == m && pi < idx)) {
+                            s = ps + (m == -INFINITY ? 0.f : s * exp2f((m - pm) * p.inv_T_log2e));
+                            m = pm; idx = pi;
+                        } else {
+                            s += ps * exp2f((pm - m) * p.inv_T_log2e);
+                        }
                     }
+                    p.part_max[pbase + row] = m;
+                    p.part_idx[pbase + row] = idx;
+                    p.part_sum[pbase + row] = s;
                 }
             }
-            __syncwarp();
+            asm volatile("bar.sync 1, 128;" ::: "memory");
         }
     }
 
@@ -250,39 +300,38 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tm_w_full, const __grid_consta
     }
 }
 
-// Merge the per-(CTA, warp) partials of each hidden row: one warp per row, fixed order.
-__global__ void lmhead_merge_kernel(int M, int P, float inv_T, float inv_T_log2e, const float* part_max,
-                                    const int* part_idx, const float* part_sum, int32_t* argmax, float* maxlogit,
-                                    float* lse) {
-    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (row >= M) return;
+// Merge the per-CTA partials of each hidden row: one block per row, one partial per thread, fixed
+// reduction tree; the comparator (logit descending, id ascending) makes the result order-independent.
+__global__ void __launch_bounds__(256)
+lmhead_merge_kernel(int M, int P, float inv_T, float inv_T_log2e, const float* part_max, const int* part_idx,
+                    const float* part_sum, int32_t* argmax, float* maxlogit, float* lse) {
+    __shared__ float s_m[8], s_s[8];
+    __shared__ int s_i[8];
+    const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     float m = -INFINITY, s = 0.f;
     int idx = 0x7fffffff;
-    for (int k = lane; k < P; k += 32) {
-        const float pm = part_max[(size_t)k * M + row], ps = part_sum[(size_t)k * M + row];
-        const int pi = part_idx[(size_t)k * M + row];
-        if (pm == -INFINITY) continue;
-        if (pm > m || (pm == m && pi < idx)) {
-            s = ps + (m == -INFINITY ? 0.f : s * exp2f((m - pm) * inv_T_log2e));
-            m = pm; idx = pi;
-        } else {
-            s += ps * exp2f((pm - m) * inv_T_log2e);
-        }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        const float om = __shfl_xor_sync(0xffffffffu, m, o), os = __shfl_xor_sync(0xffffffffu, s, o);
-        const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
-        if (om == -INFINITY) continue;
+    auto fold = [&](float om, int oi, float os) {
+        if (om == -INFINITY) return;
         if (om > m || (om == m && oi < idx)) {
             s = os + (m == -INFINITY ? 0.f : s * exp2f((m - om) * inv_T_log2e));
             m = om; idx = oi;
         } else {
             s += os * exp2f((om - m) * inv_T_log2e);
         }
+    };
+    for (int k = tid; k < P; k += blockDim.x)
+        fold(part_max[(size_t)k * M + row], part_idx[(size_t)k * M + row], part_sum[(size_t)k * M + row]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, m, o), os = __shfl_xor_sync(0xffffffffu, s, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+        fold(om, oi, os);
     }
-    if (lane == 0) {
+    if (lane == 0) { s_m[warp] = m; s_i[warp] = idx; s_s[warp] = s; }
+    __syncthreads();
+    if (tid == 0) {
+        m = -INFINITY; s = 0.f; idx = 0x7fffffff;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) fold(s_m[w], s_i[w], s_s[w]);
         if (argmax) argmax[row] = idx;
         if (maxlogit) maxlogit[row] = m;
         if (lse) lse[row] = m * inv_T + logf(s);
@@ -392,6 +441,12 @@ mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, c
     p.stages = (kSmemBudget - kCtrlBytes - 1024) / p.stage_bytes;
     if (p.stages > kMaxStages) p.stages = kMaxStages;
     if (p.stages < 2) return MIRROR_ERR_SHAPE;
+    // producer batching (tuning knobs; the defaults were picked by measurement on B200)
+    p.k_group = p.stages / 2 < 5 ? (p.stages / 2 > 0 ? p.stages / 2 : 1) : 5;
+    if (const char* e = getenv("MIRROR_LM_KGROUP")) p.k_group = atoi(e);
+    if (const char* e = getenv("MIRROR_LM_STAGES")) { const int s = atoi(e); if (s >= 2 && s < p.stages) p.stages = s; }
+    if (p.k_group < 1) p.k_group = 1;
+    if (p.k_group > p.stages) p.k_group = p.stages;
     p.groups_total = (V + 7) / 8;
     p.inv_T = 1.0f / ctx->temperature;
     p.inv_T_log2e = p.inv_T * 1.4426950408889634f;
@@ -400,7 +455,7 @@ mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, c
 
     int grid = ctx->num_sms;
     if (grid > p.groups_total) grid = p.groups_total;
-    const size_t P = (size_t)grid * 4;
+    const size_t P = (size_t)grid;
     if (partial_bytes < P * M * 12) return MIRROR_ERR_WORKSPACE;
     p.part_max = (float*)partial_ws;
     p.part_idx = (int*)(p.part_max + P * M);
@@ -432,9 +487,8 @@ mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, c
 
     float* lse_dst = lse ? lse : (topk > 0 ? lse_scratch : nullptr);
     if (argmax || maxlogit || lse_dst) {
-        const int warps = 8;
-        lmhead_merge_kernel<<<(M + warps - 1) / warps, warps * 32, 0, stream>>>(M, (int)P, p.inv_T, p.inv_T_log2e, p.part_max,
-                                                                               p.part_idx, p.part_sum, argmax, maxlogit, lse_dst);
+        lmhead_merge_kernel<<<M, 256, 0, stream>>>(M, (int)P, p.inv_T, p.inv_T_log2e, p.part_max, p.part_idx, p.part_sum,
+                                                   argmax, maxlogit, lse_dst);
         ctx->launches += 1;
         MIRROR_CUDA_OK(cudaGetLastError());
     }
