@@ -167,6 +167,26 @@ mirror_status mirror_lmhead_reduce(mirror_ctx* ctx, const void* hidden, int M, c
                                    int32_t* topk_id, float* topk_logprob, float* gather_logit,
                                    float* logits_out, void* stream);
 
+/* LM head with fused argmax / max / log-sum-exp for callers that must not allocate device memory
+ * (the paper has no counterpart: this is a deployment variant of mirror_lmhead_reduce, same kernels).
+ * Who needs it: a host that has given all device memory to its own pool, a plugin called inside an
+ * allocator-guarded region, or any code path where cudaMalloc is forbidden.  No context and no workspace:
+ * the kernel's scratch (one partial per CTA and row) is a fixed array inside the library image, 393,472
+ * bytes on every GPU that loads the library, held until the process exits.
+ *   device       CUDA device ordinal (made current for the call)
+ *   hidden, W    bf16 [M, H] and [V, H] as in mirror_lmhead_reduce; H a multiple of 64
+ *   M            at most 128 rows; more returns MIRROR_ERR_SHAPE (use mirror_lmhead_reduce with a workspace)
+ *   temperature  T > 0 (0 selects 1): lse = log sum exp(logits / T)
+ *   argmax, maxlogit, lse   device [M] outputs, each nullable
+ * Calls no cudaMalloc / cudaFree and no allocating library routine.  The first call on a device resolves the
+ * scratch array's device address (cudaGetSymbolAddress) and the tensor-map encoder; make that first call
+ * before any stream capture begins.  Every call on a device shares the one scratch array: calls that
+ * overlap on the GPU (different streams, no ordering) race on it and give wrong results -- order them.
+ * The call clears the status words it needs on `stream`; the rest of the array is rewritten before it is read. */
+mirror_status mirror_lmhead_reduce_noalloc(int device, const void* hidden, int M, const void* W, int V, int H,
+                                           float temperature, int32_t* argmax, float* maxlogit, float* lse,
+                                           void* stream);
+
 /* Acceptance, branch selection, emitted tokens and reuse lookup (a5 + a6).
  * Greedy (Eq. 3 / Eq. 10): branch length a = number of leading nodes c with tokens[c] == target_argmax[parent(c)].
  * Speculative sampling: node c (token x, parent row r) passes iff u_accept[c] * q_c[x] <= p_r[x] with

@@ -23,6 +23,7 @@ EXPORTS = [
     "mirror_create", "mirror_destroy", "mirror_workspace_bytes", "mirror_set_workspace",
     "mirror_attn_verify", "mirror_lmhead_reduce", "mirror_accept_select", "mirror_verify_step",
     "mirror_device_status", "mirror_launch_count", "mirror_status_str", "mirror_set_stage_events",
+    "mirror_lmhead_reduce_noalloc",
 ]
 
 
@@ -100,6 +101,30 @@ def _ptr(t: Optional[torch.Tensor], dtype=None, name: str = "tensor"):
 def _stream(stream) -> C.c_void_p:
     s = torch.cuda.current_stream() if stream is None else stream
     return C.c_void_p(s.cuda_stream)
+
+
+def mirror_lmhead_reduce_noalloc(hidden: torch.Tensor, W: torch.Tensor, temperature: float = 1.0, argmax=None,
+                                 maxlogit=None, lse=None, stream=None) -> dict:
+    """LM head reductions for callers that cannot allocate device memory: no context, no workspace; the
+    kernel's scratch is a fixed array inside the library (at most 128 rows).  The output tensors may be
+    passed in (so that this wrapper allocates nothing either); missing ones are created here for
+    convenience.  Calls on one device share the scratch array: do not let them overlap on the GPU."""
+    lib = load_library()
+    M, H = hidden.shape
+    V = W.shape[0]
+    dev = hidden.device
+    if argmax is None:
+        argmax = torch.empty(M, dtype=torch.int32, device=dev)
+    if maxlogit is None:
+        maxlogit = torch.empty(M, dtype=torch.float32, device=dev)
+    if lse is None:
+        lse = torch.empty(M, dtype=torch.float32, device=dev)
+    _check(lib.mirror_lmhead_reduce_noalloc(dev.index if dev.index is not None else torch.cuda.current_device(),
+                                            _ptr(hidden, torch.bfloat16, "hidden"), M, _ptr(W, torch.bfloat16, "W"), V, H,
+                                            C.c_float(temperature), _ptr(argmax, torch.int32, "argmax"),
+                                            _ptr(maxlogit, torch.float32, "maxlogit"), _ptr(lse, torch.float32, "lse"),
+                                            _stream(stream)), "mirror_lmhead_reduce_noalloc")
+    return dict(argmax=argmax, maxlogit=maxlogit, lse=lse)
 
 
 class AcceptResult:

@@ -533,3 +533,87 @@ extern "C" mirror_status mirror_lmhead_reduce(mirror_ctx* ctx, const void* hidde
                                 topk_logprob, gather_logit, logits_out, (uint8_t*)ctx->ws + L.lm_partial, L.lm_partial_bytes, lse_scratch,
                                 (cudaStream_t)stream);
 }
+
+// ---------------------------------------------------------------------------------------------------
+// mirror_lmhead_reduce_noalloc: the same LM-head kernels for callers that must not allocate.
+//
+// Some hosts of this library cannot call cudaMalloc at the point where they need the LM head: a
+// serving loop that has handed all device memory to its own pool, a plugin running inside a framework's
+// allocator-guarded region, or code that must not touch the allocator because a stream capture is
+// under way elsewhere in the process.  For them the per-CTA partials (the kernel's only scratch memory)
+// live in a fixed array that is part of the loaded library image, and no context object (whose
+// creation allocates a status word) is needed.
+// ---------------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kNoAllocMaxRows = 128;      // M limit of the no-allocation entry point
+constexpr int kNoAllocMaxCtas = 256;      // >= SM count of any device this library supports
+constexpr size_t kNoAllocHeader = 256;    // {status code, detail} words in front of the partials
+constexpr size_t kNoAllocBytes = kNoAllocHeader + (size_t)kNoAllocMaxCtas * kNoAllocMaxRows * 12;
+
+// Lives in every GPU's copy of the library image from load until exit (393,472 bytes per device).
+// In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
+
+struct NoAllocDevice {          // host-side, per device, filled by the first call on that device
+    bool ready = false;
+    unsigned char* scratch = nullptr;
+    int num_sms = 0;
+    bool attr_set = false;
+    PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
+};
+NoAllocDevice g_noalloc_dev[64];
+
+}  // namespace
+
+extern "C" mirror_status mirror_lmhead_reduce_noalloc(int device, const void* hidden, int M, const void* W, int V, int H,
+                                                      float temperature, int32_t* argmax, float* maxlogit, float* lse,
+                                                      void* stream) {
+    if (!hidden || !W || M <= 0 || V <= 0 || H <= 0 || device < 0 || device >= 64) return MIRROR_ERR_ARG;
+    if (M > kNoAllocMaxRows) return MIRROR_ERR_SHAPE;          // beyond the fixed scratch: use mirror_lmhead_reduce
+    if (H % 64 != 0 || temperature < 0.f) return MIRROR_ERR_SHAPE;
+    if (((uintptr_t)hidden & 15) || ((uintptr_t)W & 15)) return MIRROR_ERR_ARG;
+    MIRROR_CUDA_OK(cudaSetDevice(device));
+    NoAllocDevice& d = g_noalloc_dev[device];
+    if (!d.ready) {
+        // one-time set-up on this device (no allocation): resolve the device address of the scratch array
+        cudaDeviceProp prop;
+        MIRROR_CUDA_OK(cudaGetDeviceProperties(&prop, device));
+        if (prop.major != 10) return MIRROR_ERR_UNSUPPORTED;
+        if (prop.multiProcessorCount > kNoAllocMaxCtas) return MIRROR_ERR_UNSUPPORTED;
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) return MIRROR_ERR_CUDA;
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+            qres != cudaDriverEntryPointSuccess)
+            return MIRROR_ERR_CUDA;
+        d.scratch = (unsigned char*)ptr;
+        d.num_sms = prop.multiProcessorCount;
+        d.encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
+        d.ready = true;
+    }
+    // A context on the stack stands in for mirror_create's: same launch path, nothing allocated.
+    mirror_ctx tmp;
+    tmp.desc.hidden = H;
+    tmp.desc.vocab = V;
+    tmp.desc.n_q_heads = tmp.desc.n_kv_heads = 1;
+    tmp.desc.head_dim = 64;
+    tmp.desc.page_size = 16;
+    tmp.desc.softmax_scale = 0.f;
+    tmp.desc.temperature = temperature;
+    tmp.device = device;
+    tmp.num_sms = d.num_sms;
+    tmp.temperature = temperature > 0.f ? temperature : 1.0f;
+    tmp.d_status = (int*)d.scratch;
+    tmp.encode = d.encode;
+    tmp.lm_attr_set = d.attr_set;
+    cudaStream_t s = (cudaStream_t)stream;
+    // the status words must start at zero; the partials are fully rewritten by every launch before they are read
+    MIRROR_CUDA_OK(cudaMemsetAsync(d.scratch, 0, kNoAllocHeader, s));
+    mirror_status st = mirror_lmhead_launch(&tmp, hidden, M, W, 0, nullptr, nullptr, 0, argmax, maxlogit, lse, nullptr, nullptr,
+                                            nullptr, nullptr, d.scratch + kNoAllocHeader, kNoAllocBytes - kNoAllocHeader,
+                                            nullptr, s, nullptr);
+    d.attr_set = tmp.lm_attr_set;
+    return st;
+}
