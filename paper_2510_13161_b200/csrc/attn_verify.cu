@@ -5,22 +5,24 @@
 // Work decomposition.  A "unit" is (layer, request, KV head): all G = Hq/Hkv query heads of all n tree
 // nodes (G*n rows) share that head's K/V stream, so one CTA owning the unit's rows reads each K/V byte
 // once from HBM and reuses it from shared memory for every row (the GQA / tree sharing).  A unit's keys
-// are cut into 16-token slots (one KV page, or 16 tree tokens) and 128-token tiles.  The tiles of all
+// are cut into 16-token slots (one KV page, or 16 tree tokens) and 64-token tiles.  The tiles of all
 // units form one sequence that is split evenly over persistent CTAs (one per SM), so a unit may be cut
 // across CTAs; each CTA then leaves a partial (max, sum, accumulator) and the last one to arrive at the
 // unit's counter merges them in a fixed order.  No CTA ever waits for another.
 // More than 128 rows per unit are handled by row blocks: a group of CTAs walks the same tiles at the
 // same time, each with its own rows, so the second read of a tile is served by L2.
 //
-// Per CTA (6 warps):
-//   warp 0      stages K and V tiles: one TMA box per (page, 64-column half) issued by separate lanes,
+// Per CTA (7 warps):
+//   warp 0      stages K and V tiles into two 4-deep rings: one TMA box per (page, 64-column half),
 //               128-byte swizzle; ragged page and tree tokens by plain loads with zero fill
-//   warp 1      owns TMEM and issues tcgen05.mma: S = Q K^T (M=128 rows, N=tokens of the tile) into one of
-//               two S buffers, then O += P V with P read from shared memory and V as an MN-major operand
+//   warp 1      owns TMEM and issues S = Q K^T (tcgen05.mma, M=128 rows, N=tokens of the tile) into one of
+//               four S buffers, as far ahead as the K ring and the S buffers allow
 //   warps 2..5  one thread per row (TMEM lane): tcgen05.ld of the row's scores, mask in registers, online
-//               softmax without any shuffle, P written as bf16 into the swizzled A-operand layout; the
-//               accumulator O stays in TMEM and is rescaled only when a row's maximum grew by more than
-//               2^8 (the stale offset is carried exactly through the running sum and the final division)
+//               softmax without any shuffle, P written as bf16 into one of two swizzled A-operand buffers;
+//               the accumulator O stays in TMEM and is rescaled only when a row's maximum grew by more
+//               than 2^8 (the stale offset is carried exactly through the running sum and the division)
+//   warp 6      issues O += P V (P from shared memory, V as an MN-major operand)
+// Every ring index and mbarrier parity is a function of one per-CTA tile counter, identical in all roles.
 // Every mbarrier wait is bounded; on expiry the kernel records MIRROR_DEV_TIMEOUT and unwinds.
 #include <math.h>
 #include <string.h>
@@ -29,15 +31,18 @@
 
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;
 constexpr int kSlotTok = 16;
-constexpr int kTileSlots = 8;
-constexpr int kTileTok = kSlotTok * kTileSlots;     // 128
+constexpr int kTileSlots = 4;
+constexpr int kTileTok = kSlotTok * kTileSlots;     // 64
 constexpr int kRows = 128;                          // UMMA M: rows per row block
 constexpr int kMaxBatch = 1024;
-constexpr int kKVStages = 2;
+constexpr int kKVStages = 4;                        // power of two: stage = tile counter & 3
+constexpr int kSBufs = 4;                           // S buffers in TMEM (power of two)
 constexpr int kMergeWarps = 4;
 constexpr float kRescaleLog2 = 8.0f;
+constexpr int kTmemCols = 512;                      // S0..S3 (64 columns each) | O (up to 128 columns)
+constexpr int kTmemO = kSBufs * kTileTok;
 
 struct AttnTree {
     unsigned long long anc[MIRROR_MAX_NODES][2];
@@ -59,7 +64,7 @@ struct AttnParams {
     const __nv_bfloat16* v_new;
     __nv_bfloat16* out;
     float* lse_out;
-    float* partial;                       // [grid][2][128][D+2]
+    float* partial;                       // [grid][2][D+2][128]
     int* ticket;                          // [units][n_rb][kMergeWarps]
     int* status;
 };
@@ -72,8 +77,9 @@ struct UnitPos {                          // where a global tile index falls
 
 struct Ctrl {
     uint64_t k_full[kKVStages], k_empty[kKVStages], v_full[kKVStages], v_empty[kKVStages];
-    uint64_t s_full[2], s_free[2];
-    uint64_t q_full, p_full, pv_done;
+    uint64_t s_full[kSBufs], s_free[kSBufs];
+    uint64_t p_full[2], pv_done[2];
+    uint64_t q_full;
     uint32_t tmem_base;
     volatile int abort;
 };
@@ -108,22 +114,11 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 // Shared-memory operand tiles are [64-column half][row][128 B] with the 128-byte swizzle: the 16-byte chunk
-// index is XORed with (row % 8).  A half holds 128 rows = 16 KB.
-constexpr int kHalfBytes = 128 * 128;
-__device__ __forceinline__ uint32_t tile_off(int row, int chunk) {      // chunk: 16-byte column chunk, 0 .. D/8-1
-    return (uint32_t)((chunk >> 3) * kHalfBytes + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
-}
-
-// MN-major B operand (V: rows = tokens along K, 64 d-columns contiguous): 8-token groups 1024 B apart,
-// 64-column halves kHalfBytes apart.
-__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr & 0x3FFFF) >> 4);
-    d |= (uint64_t)(kHalfBytes >> 4) << 16;          // leading byte offset: next 64-column atom
-    d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset: next 8-token group
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
-    return d;
+// index is XORed with (row % 8).  A half of Q or P holds 128 rows (16 KB), a half of a K/V stage 64 tokens (8 KB).
+constexpr int kHalfBytes = kRows * 128;
+constexpr int kKVHalfBytes = kTileTok * 128;
+__device__ __forceinline__ uint32_t tile_off(int row, int chunk, int half_bytes) {   // chunk: 16-byte column chunk
+    return (uint32_t)((chunk >> 3) * half_bytes + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
 }
 
 __device__ __forceinline__ void tmem_st_32x32b_x32(uint32_t taddr, const uint32_t (&r)[32]) {
@@ -142,12 +137,32 @@ __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.
 template <int D>
 struct Cfg {
     static constexpr int kHalves = D / 64;
-    static constexpr int kOperandBytes = kHalves * kHalfBytes;     // a 128-row operand tile (Q, one K stage, one V stage)
-    static constexpr int kPBytes = 2 * kHalfBytes;                 // P: 128 rows x 128 tokens
+    static constexpr int kQBytes = kHalves * kHalfBytes;           // Q: 128 rows x D
+    static constexpr int kStageBytes = kHalves * kKVHalfBytes;     // one K (or V) stage: 64 tokens x D
+    static constexpr int kPBytes = kRows * 128;                    // one P buffer: 128 rows x 64 tokens
     static constexpr int kSlotBoxBytes = kSlotTok * 128;           // one TMA box: 16 tokens x 64 columns
-    static constexpr size_t kSmemData = (size_t)kOperandBytes * (1 + 2 * kKVStages) + kPBytes;
+    static constexpr size_t kSmemData = (size_t)kQBytes + 2 * kPBytes + 2 * (size_t)kKVStages * kStageBytes;
     static constexpr size_t kSmemBytes = kSmemData + 1024 /*ctrl*/ + (2 * kMaxBatch + 2) * 4 + 1024 /*align*/;
 };
+
+// A segment: the part of one unit that this CTA processes.
+struct Segment {
+    UnitPos u;
+    int t_first, t_last;                  // tiles [t_first, t_last) of the unit
+    int len, pages_full, pages_all, slots_all;
+};
+__device__ __forceinline__ Segment make_segment(long long x, long long x_end, const AttnParams& p, const int* cumT,
+                                                const int* s_len, long long tiles_per_layer) {
+    Segment s;
+    s.u = locate(x, p, cumT, tiles_per_layer);
+    s.t_first = s.u.tile_in_unit;
+    s.t_last = (int)min((long long)s.u.tiles_in_unit, (long long)s.t_first + (x_end - x));
+    s.len = s_len[s.u.b];
+    s.pages_full = s.len / kSlotTok;
+    s.pages_all = (s.len + kSlotTok - 1) / kSlotTok;
+    s.slots_all = s.pages_all + p.tree_slots;
+    return s;
+}
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -157,10 +172,10 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* sQ = smem;
-    uint8_t* sP = sQ + C::kOperandBytes;
-    uint8_t* sK = sP + C::kPBytes;                                  // [kKVStages]
-    uint8_t* sV = sK + kKVStages * C::kOperandBytes;                // [kKVStages]
-    Ctrl* ctrl = (Ctrl*)(sV + kKVStages * C::kOperandBytes);
+    uint8_t* sP = sQ + C::kQBytes;                                  // [2]
+    uint8_t* sK = sP + 2 * C::kPBytes;                              // [kKVStages]
+    uint8_t* sV = sK + kKVStages * C::kStageBytes;                  // [kKVStages]
+    Ctrl* ctrl = (Ctrl*)(sV + kKVStages * C::kStageBytes);
     int* cumT = (int*)((uint8_t*)ctrl + 1024);                      // [B+1] tiles per request, prefix-summed
     int* s_len = cumT + (kMaxBatch + 1);                            // [B] clamped prefix lengths
 
@@ -178,17 +193,16 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             ptx::mbar_init(&ctrl->k_full[s], 2); ptx::mbar_init(&ctrl->k_empty[s], 1);
             ptx::mbar_init(&ctrl->v_full[s], 2); ptx::mbar_init(&ctrl->v_empty[s], 1);
         }
-        for (int s = 0; s < 2; ++s) { ptx::mbar_init(&ctrl->s_full[s], 1); ptx::mbar_init(&ctrl->s_free[s], 4); }
+        for (int s = 0; s < kSBufs; ++s) { ptx::mbar_init(&ctrl->s_full[s], 1); ptx::mbar_init(&ctrl->s_free[s], 4); }
+        for (int s = 0; s < 2; ++s) { ptx::mbar_init(&ctrl->p_full[s], 4); ptx::mbar_init(&ctrl->pv_done[s], 1); }
         ptx::mbar_init(&ctrl->q_full, 4);
-        ptx::mbar_init(&ctrl->p_full, 4);
-        ptx::mbar_init(&ctrl->pv_done, 1);
         ctrl->abort = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tmap(&tm_k);
         ptx::prefetch_tmap(&tm_v);
     }
     if (warp == 1) {
-        ptx::tmem_alloc(&ctrl->tmem_base, 512);
+        ptx::tmem_alloc(&ctrl->tmem_base, kTmemCols);
         ptx::tmem_relinquish();
     }
     ptx::tc_fence_before();
@@ -214,152 +228,169 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 
     if (warp == 0) {
         // =========================================================================== producer
-        int ks = 0, vs = 0;
-        uint32_t kph = 0, vph = 0;
-        int issued = 0;
+        uint32_t it = 0;                   // tiles issued by this CTA so far (ring index and parity source)
         bool ok = true;
         long long x = x_begin;
+        constexpr int kBoxLanes = kTileSlots * C::kHalves * 2;       // one TMA box per lane: (slot, half, K|V)
+        const int my_slot = lane / (C::kHalves * 2), my_half = (lane >> 1) % C::kHalves, my_is_v = lane & 1;
         while (x < x_end && ok) {
-            const UnitPos u = locate(x, p, cumT, tiles_per_layer);
-            const int len = s_len[u.b];
-            const int pages_full = len / kSlotTok, pages_all = (len + kSlotTok - 1) / kSlotTok;
-            const int slots_all = pages_all + p.tree_slots;
-            const int t_last = (int)min((long long)u.tiles_in_unit, (long long)u.tile_in_unit + (x_end - x));
+            const Segment sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
+            const UnitPos& u = sg.u;
             const int32_t* pt = p.page_table + (size_t)u.b * p.max_pages;
-            for (int t = u.tile_in_unit; t < t_last && ok; ++t, ++x) {
+            // the page id a lane needs is fetched one tile ahead, so its latency hides behind the ring wait
+            auto fetch_page = [&](int tt) -> int {
+                const int sl = tt * kTileSlots + my_slot;
+                return (lane < kBoxLanes && sl < sg.pages_full) ? pt[sl] : 0;
+            };
+            int my_page = fetch_page(sg.t_first);
+            for (int t = sg.t_first; t < sg.t_last && ok; ++t, ++x, ++it) {
+                const int st = it & (kKVStages - 1);
+                const uint32_t ph = (it / kKVStages) & 1;
+                const int next_page = (t + 1 < sg.t_last) ? fetch_page(t + 1) : 0;
                 bool w = true;
                 if (lane == 0)
-                    w = !ctrl->abort && ptx::mbar_wait(&ctrl->k_empty[ks], kph ^ 1) && ptx::mbar_wait(&ctrl->v_empty[vs], vph ^ 1);
+                    w = !ctrl->abort && ptx::mbar_wait(&ctrl->k_empty[st], ph ^ 1) && ptx::mbar_wait(&ctrl->v_empty[st], ph ^ 1);
                 w = __shfl_sync(0xffffffffu, w, 0);
                 if (!w) { if (lane == 0) timeout(p, ctrl, 10); ok = false; break; }
-                uint8_t* dk = sK + (size_t)ks * C::kOperandBytes;
-                uint8_t* dv = sV + (size_t)vs * C::kOperandBytes;
+                uint8_t* dk = sK + (size_t)st * C::kStageBytes;
+                uint8_t* dv = sV + (size_t)st * C::kStageBytes;
                 const int sl0 = t * kTileSlots;
-                const int n_slots = min(kTileSlots, slots_all - sl0);               // slots that exist in this tile
-                const int n_tma = max(0, min(kTileSlots, pages_full - sl0));        // leading slots that are whole pages
+                const int n_slots = min(kTileSlots, sg.slots_all - sl0);               // slots that exist in this tile
+                const int n_tma = max(0, min(kTileSlots, sg.pages_full - sl0));        // leading slots that are whole pages
                 if (lane == 0) {
-                    ptx::fence_proxy_async();          // earlier plain stores to these stages precede the bulk copies
-                    ptx::mbar_arrive_expect_tx(&ctrl->k_full[ks], (uint32_t)(n_tma * C::kHalves * C::kSlotBoxBytes));
-                    ptx::mbar_arrive_expect_tx(&ctrl->v_full[vs], (uint32_t)(n_tma * C::kHalves * C::kSlotBoxBytes));
+                    ptx::mbar_arrive_expect_tx(&ctrl->k_full[st], (uint32_t)(n_tma * C::kHalves * C::kSlotBoxBytes));
+                    ptx::mbar_arrive_expect_tx(&ctrl->v_full[st], (uint32_t)(n_tma * C::kHalves * C::kSlotBoxBytes));
                 }
                 __syncwarp();
-                // one box per (slot, 64-column half, tensor), spread over the lanes
-                for (int i = lane; i < n_tma * C::kHalves * 2; i += 32) {
-                    const int j = i / (C::kHalves * 2), half = (i / 2) % C::kHalves, is_v = i & 1;
-                    int page = pt[sl0 + j];
+                if (lane < n_tma * C::kHalves * 2) {
+                    int page = my_page;
                     if (page < 0 || page >= p.num_pages) { dev_check(p, 400); page = 0; }
                     const int pg = u.layer * p.layer_pages + page;
-                    if (is_v)
-                        ptx::tma_load_5d(dv + half * kHalfBytes + j * C::kSlotBoxBytes, &tm_v, &ctrl->v_full[vs], 0, 0, half, u.g, pg);
+                    if (my_is_v)
+                        ptx::tma_load_5d(dv + my_half * kKVHalfBytes + my_slot * C::kSlotBoxBytes, &tm_v, &ctrl->v_full[st], 0, 0, my_half, u.g, pg);
                     else
-                        ptx::tma_load_5d(dk + half * kHalfBytes + j * C::kSlotBoxBytes, &tm_k, &ctrl->k_full[ks], 0, 0, half, u.g, pg);
+                        ptx::tma_load_5d(dk + my_half * kKVHalfBytes + my_slot * C::kSlotBoxBytes, &tm_k, &ctrl->k_full[st], 0, 0, my_half, u.g, pg);
                 }
-                // ragged page and tree tokens by plain loads (rows beyond the valid count are zero)
-                for (int j = n_tma; j < n_slots; ++j) {
-                    const int sl = sl0 + j;
-                    const __nv_bfloat16 *ksrc, *vsrc;
-                    size_t row_stride;
-                    int valid;
-                    if (sl < pages_all) {
-                        int page = pt[sl];
-                        if (page < 0 || page >= p.num_pages) { if (lane == 0) dev_check(p, 401); page = 0; }
-                        const size_t off = (((size_t)u.layer * p.layer_pages + page) * p.Hkv + u.g) * (size_t)(kSlotTok * D);
-                        ksrc = p.k_pool + off; vsrc = p.v_pool + off;
-                        row_stride = D;
-                        valid = len - pages_full * kSlotTok;
-                    } else {
-                        const int j0 = (sl - pages_all) * kSlotTok;
-                        const size_t off = ((((size_t)u.layer * p.B + u.b) * p.n + j0) * p.Hkv + u.g) * (size_t)D;
-                        ksrc = p.k_new + off; vsrc = p.v_new + off;
-                        row_stride = (size_t)p.Hkv * D;
-                        valid = min(kSlotTok, p.n - j0);
-                    }
-                    constexpr int kChunks = kSlotTok * D / 8;          // 16-byte chunks per tensor slot
-                    for (int c = lane; c < kChunks; c += 32) {
-                        const int tr = c / (D / 8), cc = c % (D / 8);
-                        uint4 kvv = make_uint4(0, 0, 0, 0), vvv = make_uint4(0, 0, 0, 0);
-                        if (tr < valid) {
-                            kvv = *reinterpret_cast<const uint4*>(ksrc + tr * row_stride + cc * 8);
-                            vvv = *reinterpret_cast<const uint4*>(vsrc + tr * row_stride + cc * 8);
+                if (n_tma < n_slots) {
+                    // ragged page and tree tokens by plain loads (rows beyond the valid count are zero)
+                    for (int j = n_tma; j < n_slots; ++j) {
+                        const int sl = sl0 + j;
+                        const __nv_bfloat16 *ksrc, *vsrc;
+                        size_t row_stride;
+                        int valid;
+                        if (sl < sg.pages_all) {
+                            int page = pt[sl];
+                            if (page < 0 || page >= p.num_pages) { if (lane == 0) dev_check(p, 401); page = 0; }
+                            const size_t off = (((size_t)u.layer * p.layer_pages + page) * p.Hkv + u.g) * (size_t)(kSlotTok * D);
+                            ksrc = p.k_pool + off; vsrc = p.v_pool + off;
+                            row_stride = D;
+                            valid = sg.len - sg.pages_full * kSlotTok;
+                        } else {
+                            const int j0 = (sl - sg.pages_all) * kSlotTok;
+                            const size_t off = ((((size_t)u.layer * p.B + u.b) * p.n + j0) * p.Hkv + u.g) * (size_t)D;
+                            ksrc = p.k_new + off; vsrc = p.v_new + off;
+                            row_stride = (size_t)p.Hkv * D;
+                            valid = min(kSlotTok, p.n - j0);
                         }
-                        *reinterpret_cast<uint4*>(dk + tile_off(j * kSlotTok + tr, cc)) = kvv;
-                        *reinterpret_cast<uint4*>(dv + tile_off(j * kSlotTok + tr, cc)) = vvv;
+                        constexpr int kChunks = kSlotTok * D / 8;          // 16-byte chunks per tensor slot
+                        constexpr int kPer = kChunks / 32;
+                        uint4 kvv[kPer], vvv[kPer];
+#pragma unroll
+                        for (int i = 0; i < kPer; ++i) {
+                            const int c = lane + i * 32, tr = c / (D / 8), cc = c % (D / 8);
+                            kvv[i] = vvv[i] = make_uint4(0, 0, 0, 0);
+                            if (tr < valid) {
+                                kvv[i] = *reinterpret_cast<const uint4*>(ksrc + tr * row_stride + cc * 8);
+                                vvv[i] = *reinterpret_cast<const uint4*>(vsrc + tr * row_stride + cc * 8);
+                            }
+                        }
+#pragma unroll
+                        for (int i = 0; i < kPer; ++i) {
+                            const int c = lane + i * 32, tr = c / (D / 8), cc = c % (D / 8);
+                            *reinterpret_cast<uint4*>(dk + tile_off(j * kSlotTok + tr, cc, kKVHalfBytes)) = kvv[i];
+                            *reinterpret_cast<uint4*>(dv + tile_off(j * kSlotTok + tr, cc, kKVHalfBytes)) = vvv[i];
+                        }
                     }
+                    // the plain stores are read by the tensor core, and later overwritten by bulk copies (async proxy)
+                    ptx::fence_proxy_async();
                 }
-                ptx::fence_proxy_async();              // plain stores above are read by the tensor core (async proxy)
                 __syncwarp();
-                if (lane == 0) { ptx::mbar_arrive(&ctrl->k_full[ks]); ptx::mbar_arrive(&ctrl->v_full[vs]); }
-                if (++ks == kKVStages) { ks = 0; kph ^= 1; }
-                if (++vs == kKVStages) { vs = 0; vph ^= 1; }
-                ++issued;
+                if (lane == 0) { ptx::mbar_arrive(&ctrl->k_full[st]); ptx::mbar_arrive(&ctrl->v_full[st]); }
+                my_page = next_page;
             }
         }
         if (!ok && lane == 0) {
             // let copies already in flight land before the CTA's shared memory goes away
-            const int back = issued < kKVStages ? issued : kKVStages;
-            for (int j = 0; j < back; ++j) {
-                if (--ks < 0) { ks = kKVStages - 1; kph ^= 1; }
-                if (--vs < 0) { vs = kKVStages - 1; vph ^= 1; }
-                ptx::mbar_wait(&ctrl->k_full[ks], kph, 100000000ull);
-                ptx::mbar_wait(&ctrl->v_full[vs], vph, 100000000ull);
+            const uint32_t back = it < (uint32_t)kKVStages ? it : (uint32_t)kKVStages;
+            for (uint32_t j = it - back; j < it; ++j) {
+                ptx::mbar_wait(&ctrl->k_full[j & (kKVStages - 1)], (j / kKVStages) & 1, 200000000ll);
+                ptx::mbar_wait(&ctrl->v_full[j & (kKVStages - 1)], (j / kKVStages) & 1, 200000000ll);
             }
         }
     } else if (warp == 1) {
-        // =========================================================================== UMMA issuer
+        // =========================================================================== Q K^T issuer
         if (lane == 0) {
-            const uint32_t q_addr = ptx::smem_u32(sQ), p_addr = ptx::smem_u32(sP);
-            const uint32_t k_addr = ptx::smem_u32(sK), v_addr = ptx::smem_u32(sV);
-            const uint32_t idesc_pv = ptx::umma_idesc_bf16(kRows, D) | (1u << 16);      // B operand MN-major
-            int ks = 0, vs = 0, sb = 0;
-            uint32_t kph = 0, vph = 0, sph = 0, qph = 0, pph = 0;
+            // descriptor words: the high words and the Q base are constants; per tile only low words move
+            const uint32_t hi = ptx::umma_desc_hi_sw128(1024);
+            const uint32_t q_lo = ptx::umma_desc_lo(ptx::smem_u32(sQ), 16);
+            const uint32_t k_lo = ptx::umma_desc_lo(ptx::smem_u32(sK), 16);
+            const uint32_t idesc_full = ptx::umma_idesc_bf16(kRows, kTileTok);
+            uint32_t it = 0, seg = 0;
             bool ok = true;
             long long x = x_begin;
-
-            auto issue_qk = [&](int n_slots) -> bool {
-                if (ctrl->abort || !ptx::mbar_wait(&ctrl->k_full[ks], kph) || !ptx::mbar_wait(&ctrl->s_free[sb], sph ^ 1)) return false;
-                ptx::tc_fence_after();
-                const uint32_t idesc = ptx::umma_idesc_bf16(kRows, n_slots * kSlotTok);
-                const uint32_t kb = k_addr + (uint32_t)(ks * C::kOperandBytes);
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (uint32_t)((kk >> 2) * kHalfBytes + (kk & 3) * 32);
-                    ptx::umma_f16(tmem_base + (uint32_t)(sb * kTileTok), ptx::umma_desc_k_sw128(q_addr + off),
-                                  ptx::umma_desc_k_sw128(kb + off), idesc, kk != 0);
-                }
-                ptx::umma_commit(&ctrl->k_empty[ks]);
-                ptx::umma_commit(&ctrl->s_full[sb]);
-                if (++ks == kKVStages) { ks = 0; kph ^= 1; }
-                if (++sb == 2) { sb = 0; sph ^= 1; }
-                return true;
-            };
-
             while (x < x_end && ok) {
-                const UnitPos u = locate(x, p, cumT, tiles_per_layer);
-                const int len = s_len[u.b];
-                const int slots_all = (len + kSlotTok - 1) / kSlotTok + p.tree_slots;
-                const int t_last = (int)min((long long)u.tiles_in_unit, (long long)u.tile_in_unit + (x_end - x));
-                const int t_first = u.tile_in_unit;
-                if (ctrl->abort || !ptx::mbar_wait(&ctrl->q_full, qph)) { timeout(p, ctrl, 20); ok = false; break; }
-                qph ^= 1;
-                if (!issue_qk(min(kTileSlots, slots_all - t_first * kTileSlots))) { timeout(p, ctrl, 21); ok = false; break; }
-                for (int t = t_first; t < t_last; ++t, ++x) {
-                    if (t + 1 < t_last)
-                        if (!issue_qk(min(kTileSlots, slots_all - (t + 1) * kTileSlots))) { timeout(p, ctrl, 22); ok = false; break; }
-                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->p_full, pph) || !ptx::mbar_wait(&ctrl->v_full[vs], vph)) {
+                const Segment sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
+                if (ctrl->abort || !ptx::mbar_wait(&ctrl->q_full, seg & 1)) { timeout(p, ctrl, 20); ok = false; break; }
+                ++seg;
+                for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
+                    const int st = it & (kKVStages - 1), sb = it & (kSBufs - 1);
+                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->k_full[st], (it / kKVStages) & 1) ||
+                        !ptx::mbar_wait(&ctrl->s_free[sb], ((it / kSBufs) & 1) ^ 1)) {
+                        timeout(p, ctrl, 21); ok = false; break;
+                    }
+                    ptx::tc_fence_after();
+                    const int n_slots = min(kTileSlots, sg.slots_all - t * kTileSlots);
+                    const uint32_t idesc = n_slots == kTileSlots ? idesc_full : ptx::umma_idesc_bf16(kRows, n_slots * kSlotTok);
+                    const uint32_t kb = k_lo + (uint32_t)((st * C::kStageBytes) >> 4);
+                    const uint32_t d = tmem_base + (uint32_t)(sb * kTileTok);
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk)
+                        ptx::umma_f16_lohi(d, q_lo + (uint32_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4), hi,
+                                           kb + (uint32_t)(((kk >> 2) * kKVHalfBytes + (kk & 3) * 32) >> 4), hi, idesc, kk != 0);
+                    ptx::umma_commit(&ctrl->k_empty[st]);
+                    ptx::umma_commit(&ctrl->s_full[sb]);
+                }
+            }
+        }
+    } else if (warp == 6) {
+        // =========================================================================== P V issuer
+        if (lane == 0) {
+            const uint32_t hi = ptx::umma_desc_hi_sw128(1024);
+            const uint32_t p_lo = ptx::umma_desc_lo(ptx::smem_u32(sP), 16);
+            const uint32_t v_lo = ptx::umma_desc_lo(ptx::smem_u32(sV), kKVHalfBytes);     // MN-major: LBO = next 64-column atom
+            const uint32_t idesc_pv = ptx::umma_idesc_bf16(kRows, D) | (1u << 16);          // B operand MN-major
+            uint32_t it = 0;
+            bool ok = true;
+            long long x = x_begin;
+            while (x < x_end && ok) {
+                const Segment sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
+                for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
+                    const int st = it & (kKVStages - 1), pb = it & 1;
+                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->p_full[pb], (it >> 1) & 1) ||
+                        !ptx::mbar_wait(&ctrl->v_full[st], (it / kKVStages) & 1)) {
                         timeout(p, ctrl, 23); ok = false; break;
                     }
-                    pph ^= 1;
                     ptx::tc_fence_after();
-                    const int n_slots = min(kTileSlots, slots_all - t * kTileSlots);
-                    const uint32_t vb = v_addr + (uint32_t)(vs * C::kOperandBytes);
-                    for (int k = 0; k < n_slots; ++k) {
-                        const uint32_t a_off = (uint32_t)((k >> 2) * kHalfBytes + (k & 3) * 32);
-                        ptx::umma_f16(tmem_base + 2 * kTileTok, ptx::umma_desc_k_sw128(p_addr + a_off),
-                                      umma_desc_mn_sw128(vb + (uint32_t)(k * kSlotTok * 128)), idesc_pv, (t != t_first) || (k != 0));
-                    }
-                    ptx::umma_commit(&ctrl->v_empty[vs]);
-                    ptx::umma_commit(&ctrl->pv_done);
-                    if (++vs == kKVStages) { vs = 0; vph ^= 1; }
+                    const int n_slots = min(kTileSlots, sg.slots_all - t * kTileSlots);
+                    const uint32_t vb = v_lo + (uint32_t)((st * C::kStageBytes) >> 4);
+                    const uint32_t pa = p_lo + (uint32_t)((pb * C::kPBytes) >> 4);
+#pragma unroll
+                    for (int k = 0; k < kTileSlots; ++k)
+                        if (k < n_slots)
+                            ptx::umma_f16_lohi(tmem_base + kTmemO, pa + (uint32_t)(k * 2), hi, vb + (uint32_t)(k * (kSlotTok * 128 / 16)), hi,
+                                               idesc_pv, (t != sg.t_first) || (k != 0));
+                    ptx::umma_commit(&ctrl->v_empty[st]);
+                    ptx::umma_commit(&ctrl->pv_done[pb]);
                 }
             }
         }
@@ -375,39 +406,42 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         const int node = row_ok ? r_abs / p.G : 0, hl = row_ok ? r_abs % p.G : 0;
         const unsigned long long anc0 = tree.anc[node][0], anc1 = tree.anc[node][1];
         const uint32_t lane_base = tmem_base + ((uint32_t)(w4 * 32) << 16);
-        const uint32_t o_taddr = lane_base + 2 * kTileTok;
-        int sb = 0;
-        uint32_t sph = 0, dph = 0;
+        const uint32_t o_taddr = lane_base + kTmemO;
+        constexpr int kRowW = D + 2;                               // partial: D accumulator columns, then max and sum
+
+        // Q rows of a unit into the swizzled A-operand tile (rows that do not exist are zero); signals q_full
+        auto stage_q = [&](const UnitPos& u) {
+            const __nv_bfloat16* qrow = p.q + ((((size_t)u.layer * p.B + u.b) * p.n + node) * (size_t)p.Hq + u.g * p.G + hl) * D;
+            uint4 qv[D / 8];
+#pragma unroll
+            for (int cc = 0; cc < D / 8; ++cc) qv[cc] = row_ok ? *reinterpret_cast<const uint4*>(qrow + cc * 8) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+            for (int cc = 0; cc < D / 8; ++cc) *reinterpret_cast<uint4*>(sQ + tile_off(row_in_blk, cc, kHalfBytes)) = qv[cc];
+            ptx::fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&ctrl->q_full);
+        };
+
+        uint32_t it = 0;
         bool ok = true;
         long long x = x_begin;
+        Segment sg;
+        if (x < x_end) {
+            sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
+            stage_q(sg.u);
+        }
         while (x < x_end && ok) {
-            const UnitPos u = locate(x, p, cumT, tiles_per_layer);
-            const int len = s_len[u.b];
-            const int pages_full = len / kSlotTok, pages_all = (len + kSlotTok - 1) / kSlotTok;
-            const int slots_all = pages_all + p.tree_slots;
-            const int t_first = u.tile_in_unit;
-            const int t_last = (int)min((long long)u.tiles_in_unit, (long long)t_first + (x_end - x));
-            const bool whole_unit = (t_first == 0 && t_last == u.tiles_in_unit);
-
-            // ---- Q rows of this unit into the swizzled A-operand tile (rows that do not exist are zero)
-            {
-                const __nv_bfloat16* qrow = p.q + ((((size_t)u.layer * p.B + u.b) * p.n + node) * (size_t)p.Hq + u.g * p.G + hl) * D;
-#pragma unroll
-                for (int cc = 0; cc < D / 8; ++cc) {
-                    uint4 v = make_uint4(0, 0, 0, 0);
-                    if (row_ok) v = *reinterpret_cast<const uint4*>(qrow + cc * 8);
-                    *reinterpret_cast<uint4*>(sQ + tile_off(row_in_blk, cc)) = v;
-                }
-                ptx::fence_proxy_async();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&ctrl->q_full);
-            }
+            const UnitPos u = sg.u;
+            const bool whole_unit = (sg.t_first == 0 && sg.t_last == u.tiles_in_unit);
             float m_used = -INFINITY, l_run = 0.f;
 
-            for (int t = t_first; t < t_last; ++t, ++x) {
-                if (ctrl->abort || !ptx::mbar_wait(&ctrl->s_full[sb], sph)) { timeout(p, ctrl, 30); ok = false; break; }
+            for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
+                const int sb = it & (kSBufs - 1), pb = it & 1;
+                const bool first = (t == sg.t_first);
+                if (ctrl->abort || !ptx::mbar_wait(&ctrl->s_full[sb], (it / kSBufs) & 1)) { timeout(p, ctrl, 30); ok = false; break; }
                 ptx::tc_fence_after();
                 float s[kTileTok];
+                float mx = -INFINITY;
                 if (warp_has_rows) {
 #pragma unroll
                     for (int c4 = 0; c4 < kTileTok / 32; ++c4) {
@@ -418,181 +452,193 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     }
                     ptx::tmem_ld_wait();
                 }
+                // the scores are in registers: the S buffer can be refilled
                 ptx::tc_fence_before();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&ctrl->s_free[sb]);
-                if (++sb == 2) { sb = 0; sph ^= 1; }
-
-                float mx = -INFINITY;
                 if (warp_has_rows) {
-                    // mask: only tiles that hold a ragged page, tree tokens or missing slots need it
                     const int sl0 = t * kTileSlots;
-                    if (sl0 + kTileSlots > pages_full) {
+                    if (sl0 + kTileSlots > sg.pages_full) {     // a ragged page, tree tokens or missing slots in this tile
 #pragma unroll
                         for (int j = 0; j < kTileSlots; ++j) {
                             const int sl = sl0 + j;
-                            if (sl < pages_full) continue;
+                            if (sl < sg.pages_full) continue;
 #pragma unroll
                             for (int tr = 0; tr < kSlotTok; ++tr) {
                                 bool vis;
-                                if (sl < pages_all) vis = (sl * kSlotTok + tr) < len;
-                                else if (sl < slots_all) {
-                                    const int jt = (sl - pages_all) * kSlotTok + tr;
+                                if (sl < sg.pages_all) vis = (sl * kSlotTok + tr) < sg.len;
+                                else if (sl < sg.slots_all) {
+                                    const int jt = (sl - sg.pages_all) * kSlotTok + tr;
                                     vis = jt < p.n && (((jt < 64) ? (anc0 >> jt) : (anc1 >> (jt - 64))) & 1ull);
                                 } else vis = false;
                                 if (!vis) s[j * kSlotTok + tr] = -INFINITY;
                             }
                         }
                     }
+                    float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                    for (int j = 0; j < kTileTok; ++j) mx = fmaxf(mx, s[j]);
+                    for (int j = 0; j < kTileTok; ++j) m4[j & 3] = fmaxf(m4[j & 3], s[j]);
+                    mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
                 }
-                // the previous tile's P V must be complete before P is overwritten or O is touched
-                if (t != t_first) {
-                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->pv_done, dph)) { timeout(p, ctrl, 31); ok = false; break; }
-                    dph ^= 1;
+                // offset in use: set at the first tile, moved only when the row maximum outgrew it by more than 2^8
+                const bool move = warp_has_rows && (first || ((mx - m_used) * p.scale_log2e > kRescaleLog2) ||
+                                                    (m_used == -INFINITY && mx > -INFINITY));
+                const float m_next = move ? fmaxf(mx, m_used) : m_used;
+                if (!first && __any_sync(0xffffffffu, move)) {
+                    // rare: O is touched, so the previous tile's P V must be complete
+                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->pv_done[(it - 1) & 1], ((it - 1) >> 1) & 1)) { timeout(p, ctrl, 31); ok = false; break; }
                     ptx::tc_fence_after();
+                    const float alpha = (m_used == -INFINITY) ? ((m_next == -INFINITY) ? 1.f : 0.f)
+                                                              : exp2f((m_used - m_next) * p.scale_log2e);
+#pragma unroll
+                    for (int c4 = 0; c4 < D / 32; ++c4) {
+                        uint32_t r[32];
+                        ptx::tmem_ld_32x32b_x32(o_taddr + (uint32_t)(c4 * 32), r);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * alpha);
+                        tmem_st_32x32b_x32(o_taddr + (uint32_t)(c4 * 32), r);
+                    }
+                    tmem_st_wait();
+                    l_run *= alpha;
+                }
+                m_used = m_next;
+                // this tile's P buffer was last read by the P V of two tiles ago
+                if (it >= 2) {
+                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->pv_done[pb], ((it - 2) >> 1) & 1)) { timeout(p, ctrl, 33); ok = false; break; }
                 }
                 if (warp_has_rows) {
-                    // offset in use: moved only at the first tile or when the row maximum outgrew it by 2^8
-                    const bool move = (t == t_first) || ((mx - m_used) * p.scale_log2e > kRescaleLog2) ||
-                                      (m_used == -INFINITY && mx > -INFINITY);
-                    const float m_next = move ? fmaxf(mx, m_used) : m_used;
-                    if (t != t_first && __any_sync(0xffffffffu, move)) {
-                        const float alpha = (m_used == -INFINITY) ? ((m_next == -INFINITY) ? 1.f : 0.f)
-                                                                  : exp2f((m_used - m_next) * p.scale_log2e);
-#pragma unroll
-                        for (int c4 = 0; c4 < D / 32; ++c4) {
-                            uint32_t r[32];
-                            ptx::tmem_ld_32x32b_x32(o_taddr + (uint32_t)(c4 * 32), r);
-                            ptx::tmem_ld_wait();
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * alpha);
-                            tmem_st_32x32b_x32(o_taddr + (uint32_t)(c4 * 32), r);
-                        }
-                        tmem_st_wait();
-                        l_run *= alpha;
-                    }
-                    m_used = m_next;
                     const float off = (m_used == -INFINITY) ? 0.f : m_used * p.scale_log2e;
-                    float sum = 0.f;
+                    uint8_t* prow = sP + pb * C::kPBytes;
+                    float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                     for (int c8 = 0; c8 < kTileTok / 8; ++c8) {
                         float e[8];
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) { e[j] = exp2f(fmaf(s[c8 * 8 + j], p.scale_log2e, -off)); sum += e[j]; }
-                        uint4 v;
-                        v.x = pack_bf16(e[0], e[1]); v.y = pack_bf16(e[2], e[3]); v.z = pack_bf16(e[4], e[5]); v.w = pack_bf16(e[6], e[7]);
-                        *reinterpret_cast<uint4*>(sP + tile_off(row_in_blk, c8)) = v;
+                        for (int j = 0; j < 8; ++j) {
+                            e[j] = ptx::ex2_approx(fmaf(s[c8 * 8 + j], p.scale_log2e, -off));
+                            sum4[j & 3] += e[j];
+                        }
+                        uint4 pk;
+                        pk.x = pack_bf16(e[0], e[1]); pk.y = pack_bf16(e[2], e[3]); pk.z = pack_bf16(e[4], e[5]); pk.w = pack_bf16(e[6], e[7]);
+                        *reinterpret_cast<uint4*>(prow + tile_off(row_in_blk, c8, kHalfBytes)) = pk;
                     }
-                    l_run += sum;
+                    l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
                 }
-                ptx::fence_proxy_async();
-                ptx::tc_fence_before();
+                ptx::fence_proxy_async();       // P (plain stores) is read by the tensor core
+                ptx::tc_fence_before();         // orders a possible O rescale before the next P V
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&ctrl->p_full);
+                if (lane == 0) ptx::mbar_arrive(&ctrl->p_full[pb]);
             }
             if (!ok) break;
+
+            // ---- the next unit's Q can be staged now (every Q K^T of this one has completed), so that its first
+            //      tiles are scored while this unit's epilogue runs
+            Segment sg_next;
+            const bool has_next = x < x_end;
+            if (has_next) {
+                sg_next = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
+                stage_q(sg_next.u);
+            }
+
             // ---- end of this CTA's part of the unit: read O once the last P V is complete
-            if (ctrl->abort || !ptx::mbar_wait(&ctrl->pv_done, dph)) { timeout(p, ctrl, 32); ok = false; break; }
-            dph ^= 1;
+            if (ctrl->abort || !ptx::mbar_wait(&ctrl->pv_done[(it - 1) & 1], ((it - 1) >> 1) & 1)) { timeout(p, ctrl, 32); ok = false; break; }
             ptx::tc_fence_after();
-            if (!warp_has_rows) continue;
 
-            __nv_bfloat16* orow = p.out + ((((size_t)u.layer * p.B + u.b) * p.n + node) * (size_t)p.Hq + u.g * p.G + hl) * D;
-            float* lse_ptr = p.lse_out ? p.lse_out + (((size_t)u.layer * p.B + u.b) * p.Hq + u.g * p.G + hl) * p.n + node : nullptr;
-
-            if (whole_unit) {
-                const float inv = 1.f / l_run;
+            if (warp_has_rows) {
+                __nv_bfloat16* orow = p.out + ((((size_t)u.layer * p.B + u.b) * p.n + node) * (size_t)p.Hq + u.g * p.G + hl) * D;
+                float* lse_ptr = p.lse_out ? p.lse_out + (((size_t)u.layer * p.B + u.b) * p.Hq + u.g * p.G + hl) * p.n + node : nullptr;
+                if (whole_unit) {
+                    const float inv = 1.f / l_run;
 #pragma unroll
-                for (int c4 = 0; c4 < D / 32; ++c4) {
-                    uint32_t r[32];
-                    ptx::tmem_ld_32x32b_x32(o_taddr + (uint32_t)(c4 * 32), r);
-                    ptx::tmem_ld_wait();
-                    if (row_ok) {
+                    for (int c4 = 0; c4 < D / 32; ++c4) {
+                        uint32_t r[32];
+                        ptx::tmem_ld_32x32b_x32(o_taddr + (uint32_t)(c4 * 32), r);
+                        ptx::tmem_ld_wait();
+                        if (row_ok) {
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            uint4 v;
-                            v.x = pack_bf16(__uint_as_float(r[j * 8 + 0]) * inv, __uint_as_float(r[j * 8 + 1]) * inv);
-                            v.y = pack_bf16(__uint_as_float(r[j * 8 + 2]) * inv, __uint_as_float(r[j * 8 + 3]) * inv);
-                            v.z = pack_bf16(__uint_as_float(r[j * 8 + 4]) * inv, __uint_as_float(r[j * 8 + 5]) * inv);
-                            v.w = pack_bf16(__uint_as_float(r[j * 8 + 6]) * inv, __uint_as_float(r[j * 8 + 7]) * inv);
-                            *reinterpret_cast<uint4*>(orow + c4 * 32 + j * 8) = v;
+                            for (int j = 0; j < 4; ++j) {
+                                uint4 v;
+                                v.x = pack_bf16(__uint_as_float(r[j * 8 + 0]) * inv, __uint_as_float(r[j * 8 + 1]) * inv);
+                                v.y = pack_bf16(__uint_as_float(r[j * 8 + 2]) * inv, __uint_as_float(r[j * 8 + 3]) * inv);
+                                v.z = pack_bf16(__uint_as_float(r[j * 8 + 4]) * inv, __uint_as_float(r[j * 8 + 5]) * inv);
+                                v.w = pack_bf16(__uint_as_float(r[j * 8 + 6]) * inv, __uint_as_float(r[j * 8 + 7]) * inv);
+                                *reinterpret_cast<uint4*>(orow + c4 * 32 + j * 8) = v;
+                            }
+                        }
+                    }
+                    if (lse_ptr && row_ok) *lse_ptr = m_used * p.scale + logf(l_run);
+                    ptx::tc_fence_before();
+                } else {
+                    // ---- the unit is cut across CTA groups: leave a partial, last arrival merges ------------
+                    // groups ga..gb cover this unit (group g owns tiles [total*g/n_groups, total*(g+1)/n_groups))
+                    const long long per = total_tiles;
+                    int ga = group, gb = group;
+                    while (ga > 0 && per * ga / n_groups > u.unit_first_tile) --ga;
+                    const long long unit_last = u.unit_first_tile + u.tiles_in_unit - 1;
+                    while (gb + 1 < n_groups && per * (gb + 1) / n_groups <= unit_last) ++gb;
+                    const int parts = gb - ga + 1;
+                    const int slot = (sg.t_first > 0) ? 0 : 1;   // a unit that began before this CTA's range uses slot 0
+                    // partial layout [column][row]: a warp's store of one column is one contiguous 128-byte line
+                    float* my = p.partial + ((size_t)blockIdx.x * 2 + slot) * kRowW * kRows + row_in_blk;
+#pragma unroll
+                    for (int c4 = 0; c4 < D / 32; ++c4) {
+                        uint32_t r[32];
+                        ptx::tmem_ld_32x32b_x32(o_taddr + (uint32_t)(c4 * 32), r);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) my[(size_t)(c4 * 32 + j) * kRows] = __uint_as_float(r[j]);
+                    }
+                    my[(size_t)D * kRows] = m_used;
+                    my[(size_t)(D + 1) * kRows] = l_run;
+                    ptx::tc_fence_before();
+                    __threadfence();
+                    __syncwarp();
+                    const size_t unit_idx = ((size_t)u.layer * p.B + u.b) * p.Hkv + u.g;
+                    int* tk = p.ticket + (unit_idx * p.n_rb + rb) * kMergeWarps + w4;
+                    int arrived = 0;
+                    if (lane == 0) arrived = atomicAdd(tk, 1);
+                    arrived = __shfl_sync(0xffffffffu, arrived, 0);
+                    if (arrived == parts - 1) {
+                        __threadfence();
+                        if (lane == 0) *tk = 0;                          // ready for the next launch
+                        // merge in group order
+                        float M = -INFINITY;
+                        for (int gsrc = ga; gsrc <= gb; ++gsrc) {
+                            const int sslot = (per * gsrc / n_groups > u.unit_first_tile) ? 0 : 1;
+                            const float* src = p.partial + ((size_t)(gsrc * p.n_rb + rb) * 2 + sslot) * kRowW * kRows + row_in_blk;
+                            M = fmaxf(M, __ldcg(src + (size_t)D * kRows));
+                        }
+                        float Lsum = 0.f;
+                        float acc[D];
+#pragma unroll
+                        for (int j = 0; j < D; ++j) acc[j] = 0.f;
+                        for (int gsrc = ga; gsrc <= gb; ++gsrc) {
+                            const int sslot = (per * gsrc / n_groups > u.unit_first_tile) ? 0 : 1;
+                            const float* src = p.partial + ((size_t)(gsrc * p.n_rb + rb) * 2 + sslot) * kRowW * kRows + row_in_blk;
+                            const float pm = __ldcg(src + (size_t)D * kRows);
+                            const float wgt = (pm == -INFINITY) ? 0.f : exp2f((pm - M) * p.scale_log2e);
+                            Lsum += wgt * __ldcg(src + (size_t)(D + 1) * kRows);
+#pragma unroll
+                            for (int j = 0; j < D; ++j) acc[j] += wgt * __ldcg(src + (size_t)j * kRows);
+                        }
+                        if (row_ok) {
+                            const float inv = 1.f / Lsum;
+#pragma unroll
+                            for (int j = 0; j < D / 8; ++j) {
+                                uint4 v;
+                                v.x = pack_bf16(acc[j * 8 + 0] * inv, acc[j * 8 + 1] * inv);
+                                v.y = pack_bf16(acc[j * 8 + 2] * inv, acc[j * 8 + 3] * inv);
+                                v.z = pack_bf16(acc[j * 8 + 4] * inv, acc[j * 8 + 5] * inv);
+                                v.w = pack_bf16(acc[j * 8 + 6] * inv, acc[j * 8 + 7] * inv);
+                                *reinterpret_cast<uint4*>(orow + j * 8) = v;
+                            }
+                            if (lse_ptr) *lse_ptr = M * p.scale + logf(Lsum);
                         }
                     }
                 }
-                if (lse_ptr && row_ok) *lse_ptr = m_used * p.scale + logf(l_run);
-                ptx::tc_fence_before();
-                continue;
             }
-
-            // ---- the unit is cut across CTA groups: leave a partial, last arrival merges ----------------
-            // groups ga..gb cover this unit (group g owns tiles [total*g/n_groups, total*(g+1)/n_groups))
-            const long long per = total_tiles;
-            int ga = group, gb = group;
-            while (ga > 0 && per * ga / n_groups > u.unit_first_tile) --ga;
-            const long long unit_last = u.unit_first_tile + u.tiles_in_unit - 1;
-            while (gb + 1 < n_groups && per * (gb + 1) / n_groups <= unit_last) ++gb;
-            const int parts = gb - ga + 1;
-            const int slot = (t_first > 0) ? 0 : 1;      // a unit that began before this CTA's range uses slot 0
-            constexpr int kRowW = D + 2;
-            float* my = p.partial + (((size_t)blockIdx.x * 2 + slot) * kRows + row_in_blk) * kRowW;
-#pragma unroll
-            for (int c4 = 0; c4 < D / 32; ++c4) {
-                uint32_t r[32];
-                ptx::tmem_ld_32x32b_x32(o_taddr + (uint32_t)(c4 * 32), r);
-                ptx::tmem_ld_wait();
-#pragma unroll
-                for (int j = 0; j < 16; ++j)
-                    *reinterpret_cast<float2*>(my + c4 * 32 + j * 2) = make_float2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
-            }
-            *reinterpret_cast<float2*>(my + D) = make_float2(m_used, l_run);
-            ptx::tc_fence_before();
-            __threadfence();
-            __syncwarp();
-            const size_t unit_idx = ((size_t)u.layer * p.B + u.b) * p.Hkv + u.g;
-            int* tk = p.ticket + (unit_idx * p.n_rb + rb) * kMergeWarps + w4;
-            int arrived = 0;
-            if (lane == 0) arrived = atomicAdd(tk, 1);
-            arrived = __shfl_sync(0xffffffffu, arrived, 0);
-            if (arrived != parts - 1) continue;
-            __threadfence();
-            if (lane == 0) *tk = 0;                              // ready for the next launch
-            if (!row_ok) continue;
-            // merge in group order
-            float M = -INFINITY;
-            for (int gsrc = ga; gsrc <= gb; ++gsrc) {
-                const int sslot = (per * gsrc / n_groups > u.unit_first_tile) ? 0 : 1;
-                const float* src = p.partial + (((size_t)(gsrc * p.n_rb + rb) * 2 + sslot) * kRows + row_in_blk) * kRowW;
-                M = fmaxf(M, __ldcg(src + D));
-            }
-            float Lsum = 0.f;
-            float acc[D];
-#pragma unroll
-            for (int j = 0; j < D; ++j) acc[j] = 0.f;
-            for (int gsrc = ga; gsrc <= gb; ++gsrc) {
-                const int sslot = (per * gsrc / n_groups > u.unit_first_tile) ? 0 : 1;
-                const float* src = p.partial + (((size_t)(gsrc * p.n_rb + rb) * 2 + sslot) * kRows + row_in_blk) * kRowW;
-                const float2 ml = __ldcg(reinterpret_cast<const float2*>(src + D));
-                const float wgt = (ml.x == -INFINITY) ? 0.f : exp2f((ml.x - M) * p.scale_log2e);
-                Lsum += wgt * ml.y;
-#pragma unroll
-                for (int j = 0; j < D / 2; ++j) {
-                    const float2 v = __ldcg(reinterpret_cast<const float2*>(src + 2 * j));
-                    acc[2 * j] += wgt * v.x; acc[2 * j + 1] += wgt * v.y;
-                }
-            }
-            const float inv = 1.f / Lsum;
-#pragma unroll
-            for (int j = 0; j < D / 8; ++j) {
-                uint4 v;
-                v.x = pack_bf16(acc[j * 8 + 0] * inv, acc[j * 8 + 1] * inv);
-                v.y = pack_bf16(acc[j * 8 + 2] * inv, acc[j * 8 + 3] * inv);
-                v.z = pack_bf16(acc[j * 8 + 4] * inv, acc[j * 8 + 5] * inv);
-                v.w = pack_bf16(acc[j * 8 + 6] * inv, acc[j * 8 + 7] * inv);
-                *reinterpret_cast<uint4*>(orow + j * 8) = v;
-            }
-            if (lse_ptr) *lse_ptr = M * p.scale + logf(Lsum);
+            if (has_next) sg = sg_next;
         }
     }
 
@@ -600,7 +646,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     __syncthreads();
     if (warp == 1) {
         ptx::tc_fence_after();
-        ptx::tmem_dealloc(tmem_base, 512);
+        ptx::tmem_dealloc(tmem_base, kTmemCols);
     }
 }
 

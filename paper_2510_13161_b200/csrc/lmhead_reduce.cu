@@ -170,7 +170,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tm_w_full, const __grid_consta
                 uint32_t ph = ph0;
                 for (int j = 0; j < back; ++j) {
                     if (--s < 0) { s = p.stages - 1; ph ^= 1; }
-                    ptx::mbar_wait(&ctrl->full[s], ph, 100000000ull);
+                    ptx::mbar_wait(&ctrl->full[s], ph, 200000000ll);
                 }
             }
         }
