@@ -12,26 +12,30 @@
 // More than 128 rows per unit are handled by row blocks: a group of CTAs walks the same tiles at the
 // same time, each with its own rows, so the second read of a tile is served by L2.
 //
-// Per CTA (7 warps):
-//   warp 0      stages K and V tiles into two 4-deep rings: one TMA box per (page, 64-column half),
-//               128-byte swizzle; ragged page and tree tokens by plain loads with zero fill
+// Per CTA (12 warps):
+//   warp 0, 11  stage K and V tiles into two 4-deep rings: TMA boxes per page with 128-byte swizzle (K: one per
+//               64-column half, V: one per page); ragged page and tree tokens by plain loads with zero fill
 //   warp 1      owns TMEM and issues S = Q K^T (tcgen05.mma, M=128 rows, N=tokens of the tile) into one of
 //               four S buffers, as far ahead as the K ring and the S buffers allow
-//   warps 2..5  one thread per row (TMEM lane): tcgen05.ld of the row's scores, mask in registers, online
-//               softmax without any shuffle, P written as bf16 into one of two swizzled A-operand buffers;
-//               the accumulator O stays in TMEM and is rescaled only when a row's maximum grew by more
-//               than 2^8 (the stale offset is carried exactly through the running sum and the division)
-//   warp 6      issues O += P V (P from shared memory, V as an MN-major operand)
+//   warp 2      issues O += P V (P from shared memory, V as an MN-major operand)
+//   warps 3..10 softmax, two groups of four warps on alternate tiles, one thread per row (TMEM lane):
+//               tcgen05.ld of the row's scores, mask in registers, online softmax without any shuffle, P written
+//               as bf16 into the group's swizzled A-operand buffer; each group keeps its own accumulator O in
+//               TMEM (rescaled only when a row's maximum grew by more than 2^8: the stale offset is carried
+//               exactly through the sum and the division) and the two are merged like split-KV partials
 // Every ring index and mbarrier parity is a function of one per-CTA tile counter, identical in all roles.
 // Every mbarrier wait is bounded; on expiry the kernel records MIRROR_DEV_TIMEOUT and unwinds.
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include "mirror_internal.h"
 
 namespace {
 
-constexpr int kThreads = 224;
+constexpr int kSoftmaxWarps = 8;
+constexpr int kThreads = 32 * (4 + kSoftmaxWarps);   // K producer, Q K^T issuer, P V issuer, softmax pairs, V producer
+constexpr int kVProducerWarp = 3 + kSoftmaxWarps;
 constexpr int kSlotTok = 16;
 constexpr int kTileSlots = 4;
 constexpr int kTileTok = kSlotTok * kTileSlots;     // 64
@@ -39,9 +43,9 @@ constexpr int kRows = 128;                          // UMMA M: rows per row bloc
 constexpr int kMaxBatch = 1024;
 constexpr int kKVStages = 4;                        // power of two: stage = tile counter & 3
 constexpr int kSBufs = 4;                           // S buffers in TMEM (power of two)
-constexpr int kMergeWarps = 4;
+constexpr int kMergeWarps = 8;
 constexpr float kRescaleLog2 = 8.0f;
-constexpr int kTmemCols = 512;                      // S0..S3 (64 columns each) | O (up to 128 columns)
+constexpr int kTmemCols = 512;                      // S0..S3 (64 columns each) | O of group 0 | O of group 1 (D columns each)
 constexpr int kTmemO = kSBufs * kTileTok;
 
 struct AttnTree {
@@ -64,9 +68,10 @@ struct AttnParams {
     const __nv_bfloat16* v_new;
     __nv_bfloat16* out;
     float* lse_out;
-    float* partial;                       // [grid][2][D+2][128]
+    float* partial;                       // [grid][2][D+4][128]
     int* ticket;                          // [units][n_rb][kMergeWarps]
     int* status;
+    long long* timing;                    // developer aid (MIRROR_ATTN_TIMING builds): per-role cycle counters of one CTA
 };
 
 struct UnitPos {                          // where a global tile index falls
@@ -76,10 +81,12 @@ struct UnitPos {                          // where a global tile index falls
 };
 
 struct Ctrl {
-    uint64_t k_full[kKVStages], k_empty[kKVStages], v_full[kKVStages], v_empty[kKVStages];
+    uint64_t kv_full[kKVStages], kv_empty[kKVStages];   // one stage = a K tile and a V tile
     uint64_t s_full[kSBufs], s_free[kSBufs];
     uint64_t p_full[2], pv_done[2];
     uint64_t q_full;
+    uint64_t pair[4];                                   // softmax warp pairs' exchange
+    uint64_t o_free;                                    // accumulators read out at the end of a unit's part
     uint32_t tmem_base;
     volatile int abort;
 };
@@ -134,15 +141,32 @@ __device__ __forceinline__ void tmem_st_32x32b_x32(uint32_t taddr, const uint32_
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// Developer timing aid: with -DMIRROR_ATTN_TIMING each role of CTA 5 accumulates the cycles it spends in its waits
+// and writes them to p.timing; otherwise these macros vanish.
+#ifdef MIRROR_ATTN_TIMING
+#define T_DECL(...) long long __VA_ARGS__
+#define T_WAIT(acc, expr) ({ long long t__ = clock64(); bool r__ = (expr); acc += clock64() - t__; r__; })
+#define T_NOW() clock64()
+#define T_MARK(acc) do { long long n__ = clock64(); acc += n__ - tm__; tm__ = n__; } while (0)
+#define T_STORE(base, ...) do { if (p.timing && blockIdx.x == 5) { long long v__[] = {__VA_ARGS__}; for (int i__ = 0; i__ < (int)(sizeof v__ / sizeof v__[0]); ++i__) p.timing[(base) + i__] = v__[i__]; } } while (0)
+#else
+#define T_DECL(...)
+#define T_WAIT(acc, expr) (expr)
+#define T_NOW() 0ll
+#define T_MARK(acc) do { } while (0)
+#define T_STORE(base, ...) do { } while (0)
+#endif
+
 template <int D>
 struct Cfg {
     static constexpr int kHalves = D / 64;
     static constexpr int kQBytes = kHalves * kHalfBytes;           // Q: 128 rows x D
     static constexpr int kStageBytes = kHalves * kKVHalfBytes;     // one K (or V) stage: 64 tokens x D
     static constexpr int kPBytes = kRows * 128;                    // one P buffer: 128 rows x 64 tokens
-    static constexpr int kSlotBoxBytes = kSlotTok * 128;           // one TMA box: 16 tokens x 64 columns
+    static constexpr int kSlotBoxBytes = kSlotTok * 128;           // one K box: 16 tokens x 64 columns
+    static constexpr int kVSlotBytes = kHalves * kSlotTok * 128;   // one V box: 16 tokens x D columns, [half][token][128 B]
     static constexpr size_t kSmemData = (size_t)kQBytes + 2 * kPBytes + 2 * (size_t)kKVStages * kStageBytes;
-    static constexpr size_t kSmemBytes = kSmemData + 1024 /*ctrl*/ + (2 * kMaxBatch + 2) * 4 + 1024 /*align*/;
+    static constexpr size_t kSmemBytes = kSmemData + 512 /*ctrl*/ + 2 * 2 * kRows * 4 /*pair exchange*/ + (2 * kMaxBatch + 2) * 4 + 1024 /*align*/;
 };
 
 // A segment: the part of one unit that this CTA processes.
@@ -173,10 +197,11 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* sQ = smem;
     uint8_t* sP = sQ + C::kQBytes;                                  // [2]
-    uint8_t* sK = sP + 2 * C::kPBytes;                              // [kKVStages]
-    uint8_t* sV = sK + kKVStages * C::kStageBytes;                  // [kKVStages]
+    uint8_t* sK = sP + 2 * C::kPBytes;                              // [kKVStages]  [half][64 tokens][128 B]
+    uint8_t* sV = sK + kKVStages * C::kStageBytes;                  // [kKVStages]  [slot][half][16 tokens][128 B]
     Ctrl* ctrl = (Ctrl*)(sV + kKVStages * C::kStageBytes);
-    int* cumT = (int*)((uint8_t*)ctrl + 1024);                      // [B+1] tiles per request, prefix-summed
+    float* xch = (float*)((uint8_t*)ctrl + 512);                    // [2 tiles][2 halves][128 rows] pair exchange
+    int* cumT = (int*)((uint8_t*)ctrl + 512 + 2 * 2 * kRows * 4);   // [B+1] tiles per request, prefix-summed
     int* s_len = cumT + (kMaxBatch + 1);                            // [B] clamped prefix lengths
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -189,13 +214,12 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         s_len[b] = len;
     }
     if (tid == 0) {
-        for (int s = 0; s < kKVStages; ++s) {
-            ptx::mbar_init(&ctrl->k_full[s], 2); ptx::mbar_init(&ctrl->k_empty[s], 1);
-            ptx::mbar_init(&ctrl->v_full[s], 2); ptx::mbar_init(&ctrl->v_empty[s], 1);
-        }
-        for (int s = 0; s < kSBufs; ++s) { ptx::mbar_init(&ctrl->s_full[s], 1); ptx::mbar_init(&ctrl->s_free[s], 4); }
-        for (int s = 0; s < 2; ++s) { ptx::mbar_init(&ctrl->p_full[s], 4); ptx::mbar_init(&ctrl->pv_done[s], 1); }
-        ptx::mbar_init(&ctrl->q_full, 4);
+        for (int s = 0; s < kKVStages; ++s) { ptx::mbar_init(&ctrl->kv_full[s], 2); ptx::mbar_init(&ctrl->kv_empty[s], 2); }
+        for (int s = 0; s < kSBufs; ++s) { ptx::mbar_init(&ctrl->s_full[s], 1); ptx::mbar_init(&ctrl->s_free[s], kSoftmaxWarps / 2); }
+        for (int s = 0; s < 2; ++s) { ptx::mbar_init(&ctrl->p_full[s], kSoftmaxWarps / 2); ptx::mbar_init(&ctrl->pv_done[s], 1); }
+        ptx::mbar_init(&ctrl->q_full, kSoftmaxWarps);
+        for (int s = 0; s < 4; ++s) ptx::mbar_init(&ctrl->pair[s], 2);
+        ptx::mbar_init(&ctrl->o_free, kSoftmaxWarps);
         ctrl->abort = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tmap(&tm_k);
@@ -226,13 +250,19 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     const long long x_begin = group < n_groups ? total_tiles * group / n_groups : 0;
     const long long x_end = group < n_groups ? total_tiles * (group + 1) / n_groups : 0;
 
-    if (warp == 0) {
-        // =========================================================================== producer
+    if (warp == 0 || warp == kVProducerWarp) {
+        // =========================================================================== producers
+        // warp 0 stages K, the last warp stages V: a warp issues its TMA boxes one after the other, so two
+        // warps halve the time a stage takes to request
+        const bool vrole = (warp == kVProducerWarp);
         uint32_t it = 0;                   // tiles issued by this CTA so far (ring index and parity source)
         bool ok = true;
         long long x = x_begin;
-        constexpr int kBoxLanes = kTileSlots * C::kHalves * 2;       // one TMA box per lane: (slot, half, K|V)
-        const int my_slot = lane / (C::kHalves * 2), my_half = (lane >> 1) % C::kHalves, my_is_v = lane & 1;
+        T_DECL(w_empty = 0, t0 = T_NOW());
+        // one TMA box per lane: K wants (slot, half) boxes, V one box per slot (both halves)
+        const int n_boxes = vrole ? kTileSlots : kTileSlots * C::kHalves;
+        const bool has_box = lane < n_boxes;
+        const int my_slot = vrole ? lane : lane / C::kHalves, my_half = lane % C::kHalves;
         while (x < x_end && ok) {
             const Segment sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
             const UnitPos& u = sg.u;
@@ -240,7 +270,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             // the page id a lane needs is fetched one tile ahead, so its latency hides behind the ring wait
             auto fetch_page = [&](int tt) -> int {
                 const int sl = tt * kTileSlots + my_slot;
-                return (lane < kBoxLanes && sl < sg.pages_full) ? pt[sl] : 0;
+                return (has_box && sl < sg.pages_full) ? pt[sl] : 0;
             };
             int my_page = fetch_page(sg.t_first);
             for (int t = sg.t_first; t < sg.t_last && ok; ++t, ++x, ++it) {
@@ -248,84 +278,71 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 const uint32_t ph = (it / kKVStages) & 1;
                 const int next_page = (t + 1 < sg.t_last) ? fetch_page(t + 1) : 0;
                 bool w = true;
-                if (lane == 0)
-                    w = !ctrl->abort && ptx::mbar_wait(&ctrl->k_empty[st], ph ^ 1) && ptx::mbar_wait(&ctrl->v_empty[st], ph ^ 1);
+                if (lane == 0) w = !ctrl->abort && T_WAIT(w_empty, ptx::mbar_wait(&ctrl->kv_empty[st], ph ^ 1));
                 w = __shfl_sync(0xffffffffu, w, 0);
                 if (!w) { if (lane == 0) timeout(p, ctrl, 10); ok = false; break; }
-                uint8_t* dk = sK + (size_t)st * C::kStageBytes;
-                uint8_t* dv = sV + (size_t)st * C::kStageBytes;
+                uint8_t* dst = (vrole ? sV : sK) + (size_t)st * C::kStageBytes;
                 const int sl0 = t * kTileSlots;
                 const int n_slots = min(kTileSlots, sg.slots_all - sl0);               // slots that exist in this tile
                 const int n_tma = max(0, min(kTileSlots, sg.pages_full - sl0));        // leading slots that are whole pages
-                if (lane == 0) {
-                    ptx::mbar_arrive_expect_tx(&ctrl->k_full[st], (uint32_t)(n_tma * C::kHalves * C::kSlotBoxBytes));
-                    ptx::mbar_arrive_expect_tx(&ctrl->v_full[st], (uint32_t)(n_tma * C::kHalves * C::kSlotBoxBytes));
-                }
-                __syncwarp();
-                if (lane < n_tma * C::kHalves * 2) {
-                    int page = my_page;
-                    if (page < 0 || page >= p.num_pages) { dev_check(p, 400); page = 0; }
-                    const int pg = u.layer * p.layer_pages + page;
-                    if (my_is_v)
-                        ptx::tma_load_5d(dv + my_half * kKVHalfBytes + my_slot * C::kSlotBoxBytes, &tm_v, &ctrl->v_full[st], 0, 0, my_half, u.g, pg);
-                    else
-                        ptx::tma_load_5d(dk + my_half * kKVHalfBytes + my_slot * C::kSlotBoxBytes, &tm_k, &ctrl->k_full[st], 0, 0, my_half, u.g, pg);
-                }
                 if (n_tma < n_slots) {
                     // ragged page and tree tokens by plain loads (rows beyond the valid count are zero)
                     for (int j = n_tma; j < n_slots; ++j) {
                         const int sl = sl0 + j;
-                        const __nv_bfloat16 *ksrc, *vsrc;
+                        const __nv_bfloat16* src;
                         size_t row_stride;
                         int valid;
                         if (sl < sg.pages_all) {
                             int page = pt[sl];
                             if (page < 0 || page >= p.num_pages) { if (lane == 0) dev_check(p, 401); page = 0; }
-                            const size_t off = (((size_t)u.layer * p.layer_pages + page) * p.Hkv + u.g) * (size_t)(kSlotTok * D);
-                            ksrc = p.k_pool + off; vsrc = p.v_pool + off;
+                            src = (vrole ? p.v_pool : p.k_pool) + (((size_t)u.layer * p.layer_pages + page) * p.Hkv + u.g) * (size_t)(kSlotTok * D);
                             row_stride = D;
                             valid = sg.len - sg.pages_full * kSlotTok;
                         } else {
                             const int j0 = (sl - sg.pages_all) * kSlotTok;
-                            const size_t off = ((((size_t)u.layer * p.B + u.b) * p.n + j0) * p.Hkv + u.g) * (size_t)D;
-                            ksrc = p.k_new + off; vsrc = p.v_new + off;
+                            src = (vrole ? p.v_new : p.k_new) + ((((size_t)u.layer * p.B + u.b) * p.n + j0) * p.Hkv + u.g) * (size_t)D;
                             row_stride = (size_t)p.Hkv * D;
                             valid = min(kSlotTok, p.n - j0);
                         }
-                        constexpr int kChunks = kSlotTok * D / 8;          // 16-byte chunks per tensor slot
+                        constexpr int kChunks = kSlotTok * D / 8;          // 16-byte chunks per slot
                         constexpr int kPer = kChunks / 32;
-                        uint4 kvv[kPer], vvv[kPer];
+                        uint4 vv[kPer];
 #pragma unroll
                         for (int i = 0; i < kPer; ++i) {
                             const int c = lane + i * 32, tr = c / (D / 8), cc = c % (D / 8);
-                            kvv[i] = vvv[i] = make_uint4(0, 0, 0, 0);
-                            if (tr < valid) {
-                                kvv[i] = *reinterpret_cast<const uint4*>(ksrc + tr * row_stride + cc * 8);
-                                vvv[i] = *reinterpret_cast<const uint4*>(vsrc + tr * row_stride + cc * 8);
-                            }
+                            vv[i] = (tr < valid) ? *reinterpret_cast<const uint4*>(src + tr * row_stride + cc * 8) : make_uint4(0, 0, 0, 0);
                         }
 #pragma unroll
                         for (int i = 0; i < kPer; ++i) {
                             const int c = lane + i * 32, tr = c / (D / 8), cc = c % (D / 8);
-                            *reinterpret_cast<uint4*>(dk + tile_off(j * kSlotTok + tr, cc, kKVHalfBytes)) = kvv[i];
-                            *reinterpret_cast<uint4*>(dv + tile_off(j * kSlotTok + tr, cc, kKVHalfBytes)) = vvv[i];
+                            if (vrole) *reinterpret_cast<uint4*>(dst + j * C::kVSlotBytes + tile_off(tr, cc, kSlotTok * 128)) = vv[i];
+                            else *reinterpret_cast<uint4*>(dst + tile_off(j * kSlotTok + tr, cc, kKVHalfBytes)) = vv[i];
                         }
                     }
                     // the plain stores are read by the tensor core, and later overwritten by bulk copies (async proxy)
                     ptx::fence_proxy_async();
+                    __syncwarp();
                 }
+                if (lane == 0) ptx::mbar_arrive_expect_tx(&ctrl->kv_full[st], (uint32_t)(n_tma * C::kVSlotBytes));
                 __syncwarp();
-                if (lane == 0) { ptx::mbar_arrive(&ctrl->k_full[st]); ptx::mbar_arrive(&ctrl->v_full[st]); }
+                if (has_box && my_slot < n_tma) {
+                    int page = my_page;
+                    if (page < 0 || page >= p.num_pages) { dev_check(p, 400); page = 0; }
+                    const int pg = u.layer * p.layer_pages + page;
+                    if (vrole)
+                        ptx::tma_load_5d(dst + my_slot * C::kVSlotBytes, &tm_v, &ctrl->kv_full[st], 0, 0, 0, u.g, pg);
+                    else
+                        ptx::tma_load_5d(dst + my_half * kKVHalfBytes + my_slot * C::kSlotBoxBytes, &tm_k, &ctrl->kv_full[st], 0, 0, my_half, u.g, pg);
+                }
                 my_page = next_page;
             }
         }
+        if (lane == 0) T_STORE(vrole ? 32 : 16, T_NOW() - t0, w_empty, (long long)it);
         if (!ok && lane == 0) {
             // let copies already in flight land before the CTA's shared memory goes away
             const uint32_t back = it < (uint32_t)kKVStages ? it : (uint32_t)kKVStages;
-            for (uint32_t j = it - back; j < it; ++j) {
-                ptx::mbar_wait(&ctrl->k_full[j & (kKVStages - 1)], (j / kKVStages) & 1, 200000000ll);
-                ptx::mbar_wait(&ctrl->v_full[j & (kKVStages - 1)], (j / kKVStages) & 1, 200000000ll);
-            }
+            for (uint32_t j = it - back; j < it; ++j)
+                ptx::mbar_wait(&ctrl->kv_full[j & (kKVStages - 1)], (j / kKVStages) & 1, 200000000ll);
         }
     } else if (warp == 1) {
         // =========================================================================== Q K^T issuer
@@ -338,14 +355,15 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             uint32_t it = 0, seg = 0;
             bool ok = true;
             long long x = x_begin;
+            T_DECL(w_q = 0, w_k = 0, w_s = 0, t0 = T_NOW());
             while (x < x_end && ok) {
                 const Segment sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
-                if (ctrl->abort || !ptx::mbar_wait(&ctrl->q_full, seg & 1)) { timeout(p, ctrl, 20); ok = false; break; }
+                if (ctrl->abort || !T_WAIT(w_q, ptx::mbar_wait(&ctrl->q_full, seg & 1))) { timeout(p, ctrl, 20); ok = false; break; }
                 ++seg;
                 for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
                     const int st = it & (kKVStages - 1), sb = it & (kSBufs - 1);
-                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->k_full[st], (it / kKVStages) & 1) ||
-                        !ptx::mbar_wait(&ctrl->s_free[sb], ((it / kSBufs) & 1) ^ 1)) {
+                    if (ctrl->abort || !T_WAIT(w_k, ptx::mbar_wait(&ctrl->kv_full[st], (it / kKVStages) & 1)) ||
+                        !T_WAIT(w_s, ptx::mbar_wait(&ctrl->s_free[sb], ((it / kSBufs) & 1) ^ 1))) {
                         timeout(p, ctrl, 21); ok = false; break;
                     }
                     ptx::tc_fence_after();
@@ -357,27 +375,33 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     for (int kk = 0; kk < D / 16; ++kk)
                         ptx::umma_f16_lohi(d, q_lo + (uint32_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4), hi,
                                            kb + (uint32_t)(((kk >> 2) * kKVHalfBytes + (kk & 3) * 32) >> 4), hi, idesc, kk != 0);
-                    ptx::umma_commit(&ctrl->k_empty[st]);
+                    ptx::umma_commit(&ctrl->kv_empty[st]);
                     ptx::umma_commit(&ctrl->s_full[sb]);
                 }
             }
+            T_STORE(0, T_NOW() - t0, w_q, w_k, w_s, (long long)it);
         }
-    } else if (warp == 6) {
+    } else if (warp == 2) {
         // =========================================================================== P V issuer
         if (lane == 0) {
             const uint32_t hi = ptx::umma_desc_hi_sw128(1024);
             const uint32_t p_lo = ptx::umma_desc_lo(ptx::smem_u32(sP), 16);
-            const uint32_t v_lo = ptx::umma_desc_lo(ptx::smem_u32(sV), kKVHalfBytes);     // MN-major: LBO = next 64-column atom
+            const uint32_t v_lo = ptx::umma_desc_lo(ptx::smem_u32(sV), kSlotTok * 128);   // MN-major: LBO = next 64-column atom
             const uint32_t idesc_pv = ptx::umma_idesc_bf16(kRows, D) | (1u << 16);          // B operand MN-major
             uint32_t it = 0;
             bool ok = true;
             long long x = x_begin;
+            T_DECL(w_p = 0, w_v = 0, t0 = T_NOW());
+            uint32_t seg = 0;
             while (x < x_end && ok) {
                 const Segment sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
+                // the accumulators of the previous part must have been read out by every softmax warp
+                if (seg > 0 && (ctrl->abort || !ptx::mbar_wait(&ctrl->o_free, (seg - 1) & 1))) { timeout(p, ctrl, 24); ok = false; break; }
+                ++seg;
                 for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
                     const int st = it & (kKVStages - 1), pb = it & 1;
-                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->p_full[pb], (it >> 1) & 1) ||
-                        !ptx::mbar_wait(&ctrl->v_full[st], (it / kKVStages) & 1)) {
+                    if (ctrl->abort || !T_WAIT(w_p, ptx::mbar_wait(&ctrl->p_full[pb], (it >> 1) & 1)) ||
+                        !T_WAIT(w_v, ptx::mbar_wait(&ctrl->kv_full[st], (it / kKVStages) & 1))) {
                         timeout(p, ctrl, 23); ok = false; break;
                     }
                     ptx::tc_fence_after();
@@ -387,16 +411,22 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 #pragma unroll
                     for (int k = 0; k < kTileSlots; ++k)
                         if (k < n_slots)
-                            ptx::umma_f16_lohi(tmem_base + kTmemO, pa + (uint32_t)(k * 2), hi, vb + (uint32_t)(k * (kSlotTok * 128 / 16)), hi,
-                                               idesc_pv, (t != sg.t_first) || (k != 0));
-                    ptx::umma_commit(&ctrl->v_empty[st]);
+                            ptx::umma_f16_lohi(tmem_base + kTmemO + (uint32_t)(pb * D), pa + (uint32_t)(k * 2), hi,
+                                               vb + (uint32_t)(k * (C::kVSlotBytes / 16)), hi, idesc_pv, (t >= sg.t_first + 2) || (k != 0));
+                    ptx::umma_commit(&ctrl->kv_empty[st]);
                     ptx::umma_commit(&ctrl->pv_done[pb]);
                 }
             }
+            T_STORE(24, T_NOW() - t0, w_p, w_v);
         }
     } else {
         // =========================================================================== softmax / epilogue
+        // Two groups of four warps (one thread per row each) take alternate tiles: group g owns the tiles whose
+        // counter is g mod 2, with its own offset, running sum, P buffer and accumulator O_g in TMEM, exactly like
+        // two split-KV partitions that are merged when the unit's part ends.  Nothing couples the groups per tile.
         const int w4 = warp & 3;                                   // TMEM lane quarter of this warp
+        const int grp = (warp - 3) >> 2;                           // 0: warps 3..6, 1: warps 7..10
+        uint32_t xph = 0;                                          // parity of the pair's exchange barrier
         const int row_in_blk = w4 * 32 + lane;
         const int rb_row0 = rb * p.rows_per_rb;
         const int rb_rows = min(p.rows_per_rb, p.rows - rb_row0);
@@ -406,17 +436,26 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         const int node = row_ok ? r_abs / p.G : 0, hl = row_ok ? r_abs % p.G : 0;
         const unsigned long long anc0 = tree.anc[node][0], anc1 = tree.anc[node][1];
         const uint32_t lane_base = tmem_base + ((uint32_t)(w4 * 32) << 16);
-        const uint32_t o_taddr = lane_base + kTmemO;
-        constexpr int kRowW = D + 2;                               // partial: D accumulator columns, then max and sum
+        const uint32_t o_mine = lane_base + kTmemO + (uint32_t)(grp * D);       // this group's accumulator
+        constexpr int kDH = D / 2;                                 // output columns this warp finalises
+        constexpr int kRowW = D + 4;                               // partial: D accumulator columns, then (max, sum) twice
+        // both warps that share a TMEM quarter arrive (bounded wait, like every other wait in this kernel)
+        auto pair_sync = [&]() -> bool {
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&ctrl->pair[w4]);
+            const bool r = !ctrl->abort && ptx::mbar_wait(&ctrl->pair[w4], xph);
+            xph ^= 1;
+            return r;
+        };
 
-        // Q rows of a unit into the swizzled A-operand tile (rows that do not exist are zero); signals q_full
+        // this thread's half of its Q row into the swizzled A-operand tile (rows that do not exist are zero)
         auto stage_q = [&](const UnitPos& u) {
             const __nv_bfloat16* qrow = p.q + ((((size_t)u.layer * p.B + u.b) * p.n + node) * (size_t)p.Hq + u.g * p.G + hl) * D;
-            uint4 qv[D / 8];
+            uint4 qv[D / 16];
 #pragma unroll
-            for (int cc = 0; cc < D / 8; ++cc) qv[cc] = row_ok ? *reinterpret_cast<const uint4*>(qrow + cc * 8) : make_uint4(0, 0, 0, 0);
+            for (int i = 0; i < D / 16; ++i) qv[i] = row_ok ? *reinterpret_cast<const uint4*>(qrow + (grp * (D / 16) + i) * 8) : make_uint4(0, 0, 0, 0);
 #pragma unroll
-            for (int cc = 0; cc < D / 8; ++cc) *reinterpret_cast<uint4*>(sQ + tile_off(row_in_blk, cc, kHalfBytes)) = qv[cc];
+            for (int i = 0; i < D / 16; ++i) *reinterpret_cast<uint4*>(sQ + tile_off(row_in_blk, grp * (D / 16) + i, kHalfBytes)) = qv[i];
             ptx::fence_proxy_async();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&ctrl->q_full);
@@ -425,7 +464,61 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         uint32_t it = 0;
         bool ok = true;
         long long x = x_begin;
+        T_DECL(w_sf = 0, w_pv = 0, w_end = 0, t_epi = 0, t_q = 0, t0 = T_NOW(), te = 0, tm__ = 0, s_ld = 0, s_free = 0, s_max = 0, s_xch = 0, s_exp = 0, s_fin = 0);
         Segment sg;
+        // one 32-column chunk of this row's scores: tcgen05.ld, then the visibility mask where the tile needs one
+        auto load_scores = [&](int sb, int c4, int t, float (&v)[32]) {
+            uint32_t r[32];
+            ptx::tmem_ld_32x32b_x32(lane_base + (uint32_t)(sb * kTileTok + c4 * 32), r);
+            ptx::tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+            const int sl0 = t * kTileSlots + c4 * 2;
+            if (sl0 + 2 > sg.pages_full) {             // a ragged page, tree tokens or missing slots
+#pragma unroll
+                for (int jj = 0; jj < 2; ++jj) {
+                    const int sl = sl0 + jj;
+                    if (sl < sg.pages_full) continue;
+#pragma unroll
+                    for (int tr = 0; tr < kSlotTok; ++tr) {
+                        bool vis;
+                        if (sl < sg.pages_all) vis = (sl * kSlotTok + tr) < sg.len;
+                        else if (sl < sg.slots_all) {
+                            const int jt = (sl - sg.pages_all) * kSlotTok + tr;
+                            vis = jt < p.n && (((jt < 64) ? (anc0 >> jt) : (anc1 >> (jt - 64))) & 1ull);
+                        } else vis = false;
+                        if (!vis) v[jj * kSlotTok + tr] = -INFINITY;
+                    }
+                }
+            }
+        };
+        // P = exp2(s*c - offset) for the whole tile into the group's P buffer; returns the row sum and watches the maximum
+        auto softmax_tile = [&](int sb, int t, uint8_t* prow, float m_off, float& mx_out) -> float {
+            const float off = (m_off == -INFINITY) ? 0.f : m_off * p.scale_log2e;
+            float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+            float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int c4 = 0; c4 < kTileTok / 32; ++c4) {
+                float v[32];
+                load_scores(sb, c4, t, v);
+#pragma unroll
+                for (int c8 = 0; c8 < 4; ++c8) {
+                    float e[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        m4[j & 3] = fmaxf(m4[j & 3], v[c8 * 8 + j]);
+                        e[j] = ptx::ex2_approx(fmaf(v[c8 * 8 + j], p.scale_log2e, -off));
+                        sum4[j & 3] += e[j];
+                    }
+                    uint4 pk;
+                    pk.x = pack_bf16(e[0], e[1]); pk.y = pack_bf16(e[2], e[3]); pk.z = pack_bf16(e[4], e[5]); pk.w = pack_bf16(e[6], e[7]);
+                    *reinterpret_cast<uint4*>(prow + tile_off(row_in_blk, c4 * 4 + c8, kHalfBytes)) = pk;
+                }
+            }
+            mx_out = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+            return (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+        };
+
         if (x < x_end) {
             sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
             stage_q(sg.u);
@@ -433,169 +526,176 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         while (x < x_end && ok) {
             const UnitPos u = sg.u;
             const bool whole_unit = (sg.t_first == 0 && sg.t_last == u.tiles_in_unit);
-            float m_used = -INFINITY, l_run = 0.f;
+            float m_used = -INFINITY, l_run = 0.f;                 // this group's offset and running sum
+            bool first = true;                                     // no tile of this unit's part seen by this group yet
 
             for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
-                const int sb = it & (kSBufs - 1), pb = it & 1;
-                const bool first = (t == sg.t_first);
-                if (ctrl->abort || !ptx::mbar_wait(&ctrl->s_full[sb], (it / kSBufs) & 1)) { timeout(p, ctrl, 30); ok = false; break; }
+                if ((int)(it & 1) != grp) continue;
+                const int sb = it & (kSBufs - 1), pb = grp;
+                if (ctrl->abort || !T_WAIT(w_sf, ptx::mbar_wait(&ctrl->s_full[sb], (it / kSBufs) & 1))) { timeout(p, ctrl, 30); ok = false; break; }
                 ptx::tc_fence_after();
-                float s[kTileTok];
-                float mx = -INFINITY;
-                if (warp_has_rows) {
-#pragma unroll
-                    for (int c4 = 0; c4 < kTileTok / 32; ++c4) {
-                        uint32_t r[32];
-                        ptx::tmem_ld_32x32b_x32(lane_base + (uint32_t)(sb * kTileTok + c4 * 32), r);
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) s[c4 * 32 + j] = __uint_as_float(r[j]);
-                    }
-                    ptx::tmem_ld_wait();
-                }
-                // the scores are in registers: the S buffer can be refilled
-                ptx::tc_fence_before();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&ctrl->s_free[sb]);
-                if (warp_has_rows) {
-                    const int sl0 = t * kTileSlots;
-                    if (sl0 + kTileSlots > sg.pages_full) {     // a ragged page, tree tokens or missing slots in this tile
-#pragma unroll
-                        for (int j = 0; j < kTileSlots; ++j) {
-                            const int sl = sl0 + j;
-                            if (sl < sg.pages_full) continue;
-#pragma unroll
-                            for (int tr = 0; tr < kSlotTok; ++tr) {
-                                bool vis;
-                                if (sl < sg.pages_all) vis = (sl * kSlotTok + tr) < sg.len;
-                                else if (sl < sg.slots_all) {
-                                    const int jt = (sl - sg.pages_all) * kSlotTok + tr;
-                                    vis = jt < p.n && (((jt < 64) ? (anc0 >> jt) : (anc1 >> (jt - 64))) & 1ull);
-                                } else vis = false;
-                                if (!vis) s[j * kSlotTok + tr] = -INFINITY;
-                            }
-                        }
-                    }
-                    float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-                    for (int j = 0; j < kTileTok; ++j) m4[j & 3] = fmaxf(m4[j & 3], s[j]);
-                    mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
-                }
-                // offset in use: set at the first tile, moved only when the row maximum outgrew it by more than 2^8
-                const bool move = warp_has_rows && (first || ((mx - m_used) * p.scale_log2e > kRescaleLog2) ||
-                                                    (m_used == -INFINITY && mx > -INFINITY));
-                const float m_next = move ? fmaxf(mx, m_used) : m_used;
-                if (!first && __any_sync(0xffffffffu, move)) {
-                    // rare: O is touched, so the previous tile's P V must be complete
-                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->pv_done[(it - 1) & 1], ((it - 1) >> 1) & 1)) { timeout(p, ctrl, 31); ok = false; break; }
+#ifdef MIRROR_ATTN_TIMING
+                tm__ = T_NOW();
+#endif
+                // this group's P buffer and accumulator were last used by the P V of two tiles ago
+                if (it >= 2) {
+                    if (ctrl->abort || !T_WAIT(w_pv, ptx::mbar_wait(&ctrl->pv_done[pb], ((it - 2) >> 1) & 1))) { timeout(p, ctrl, 33); ok = false; break; }
                     ptx::tc_fence_after();
+                }
+                uint8_t* prow = sP + pb * C::kPBytes;
+                float mx = -INFINITY, sum = 0.f;
+                if (warp_has_rows) {
+                    if (first) {
+                        // no offset yet: one pass for the row maximum
+                        float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                        for (int c4 = 0; c4 < kTileTok / 32; ++c4) {
+                            float v[32];
+                            load_scores(sb, c4, t, v);
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) m4[j & 3] = fmaxf(m4[j & 3], v[j]);
+                        }
+                        m_used = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+                    }
+                    sum = softmax_tile(sb, t, prow, m_used, mx);
+                }
+                T_MARK(s_exp);
+                // offset in use: moved only when the row maximum outgrew it by more than 2^8
+                const bool move = warp_has_rows && !first &&
+                                  (((mx - m_used) * p.scale_log2e > kRescaleLog2) || (m_used == -INFINITY && mx > -INFINITY));
+                if (__any_sync(0xffffffffu, move)) {
+                    // rare: rescale this group's accumulator (its last P V is complete, see the wait above) and the
+                    // running sum, then redo this tile's P with the new offset
+                    const float m_next = move ? fmaxf(mx, m_used) : m_used;
                     const float alpha = (m_used == -INFINITY) ? ((m_next == -INFINITY) ? 1.f : 0.f)
                                                               : exp2f((m_used - m_next) * p.scale_log2e);
 #pragma unroll
                     for (int c4 = 0; c4 < D / 32; ++c4) {
                         uint32_t r[32];
-                        ptx::tmem_ld_32x32b_x32(o_taddr + (uint32_t)(c4 * 32), r);
+                        ptx::tmem_ld_32x32b_x32(o_mine + (uint32_t)(c4 * 32), r);
                         ptx::tmem_ld_wait();
 #pragma unroll
                         for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * alpha);
-                        tmem_st_32x32b_x32(o_taddr + (uint32_t)(c4 * 32), r);
+                        tmem_st_32x32b_x32(o_mine + (uint32_t)(c4 * 32), r);
                     }
                     tmem_st_wait();
                     l_run *= alpha;
+                    m_used = m_next;
+                    sum = softmax_tile(sb, t, prow, m_used, mx);
                 }
-                m_used = m_next;
-                // this tile's P buffer was last read by the P V of two tiles ago
-                if (it >= 2) {
-                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->pv_done[pb], ((it - 2) >> 1) & 1)) { timeout(p, ctrl, 33); ok = false; break; }
-                }
-                if (warp_has_rows) {
-                    const float off = (m_used == -INFINITY) ? 0.f : m_used * p.scale_log2e;
-                    uint8_t* prow = sP + pb * C::kPBytes;
-                    float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                    for (int c8 = 0; c8 < kTileTok / 8; ++c8) {
-                        float e[8];
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            e[j] = ptx::ex2_approx(fmaf(s[c8 * 8 + j], p.scale_log2e, -off));
-                            sum4[j & 3] += e[j];
-                        }
-                        uint4 pk;
-                        pk.x = pack_bf16(e[0], e[1]); pk.y = pack_bf16(e[2], e[3]); pk.z = pack_bf16(e[4], e[5]); pk.w = pack_bf16(e[6], e[7]);
-                        *reinterpret_cast<uint4*>(prow + tile_off(row_in_blk, c8, kHalfBytes)) = pk;
-                    }
-                    l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-                }
+                l_run += sum;
+                first = false;
+                // all reads of this S buffer are done; P is in shared memory (and any O rescale in TMEM)
                 ptx::fence_proxy_async();       // P (plain stores) is read by the tensor core
-                ptx::tc_fence_before();         // orders a possible O rescale before the next P V
+                ptx::tc_fence_before();
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&ctrl->p_full[pb]);
+                if (lane == 0) { ptx::mbar_arrive(&ctrl->s_free[sb]); ptx::mbar_arrive(&ctrl->p_full[pb]); }
+                T_MARK(s_fin);
             }
             if (!ok) break;
 
             // ---- the next unit's Q can be staged now (every Q K^T of this one has completed), so that its first
             //      tiles are scored while this unit's epilogue runs
+            // (a group that did not take the part's last tile has not yet seen that tile's scores complete)
+            if (ctrl->abort || !ptx::mbar_wait(&ctrl->s_full[(it - 1) & (kSBufs - 1)], ((it - 1) / kSBufs) & 1)) { timeout(p, ctrl, 37); ok = false; break; }
             Segment sg_next;
             const bool has_next = x < x_end;
             if (has_next) {
+#ifdef MIRROR_ATTN_TIMING
+                te = T_NOW();
+#endif
                 sg_next = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
                 stage_q(sg_next.u);
+#ifdef MIRROR_ATTN_TIMING
+                t_q += T_NOW() - te;
+#endif
             }
 
-            // ---- end of this CTA's part of the unit: read O once the last P V is complete
-            if (ctrl->abort || !ptx::mbar_wait(&ctrl->pv_done[(it - 1) & 1], ((it - 1) >> 1) & 1)) { timeout(p, ctrl, 32); ok = false; break; }
+            // ---- end of this CTA's part of the unit: the two groups exchange (offset, sum), then each warp
+            //      combines its half of the columns of both accumulators once the last P V is complete
+            float* xc = xch + (size_t)row_in_blk * 4;              // [row][group][max, sum]
+            xc[grp * 2] = m_used;
+            xc[grp * 2 + 1] = l_run;
+            if (!pair_sync()) { timeout(p, ctrl, 35); ok = false; break; }
+            const float m_a = xc[0], l_a = xc[1], m_b = xc[2], l_b = xc[3];
+            if (ctrl->abort || !T_WAIT(w_end, ptx::mbar_wait(&ctrl->pv_done[(it - 1) & 1], ((it - 1) >> 1) & 1))) { timeout(p, ctrl, 32); ok = false; break; }
             ptx::tc_fence_after();
+#ifdef MIRROR_ATTN_TIMING
+            te = T_NOW();
+#endif
+            const bool has_b = (sg.t_last - sg.t_first) >= 2;      // did the later-starting group see any tile?
+            // group of the first tile of this part: the tile counter's parity when the part began
+            const int g_first = (int)((it - (uint32_t)(sg.t_last - sg.t_first)) & 1);
+            const bool has0 = has_b || g_first == 0, has1 = has_b || g_first == 1;
+            const float M = fmaxf(has0 ? m_a : -INFINITY, has1 ? m_b : -INFINITY);
+            const float w0 = (has0 && m_a != -INFINITY) ? exp2f((m_a - M) * p.scale_log2e) : 0.f;
+            const float w1 = (has1 && m_b != -INFINITY) ? exp2f((m_b - M) * p.scale_log2e) : 0.f;
+            const float Lsum = w0 * (has0 ? l_a : 0.f) + w1 * (has1 ? l_b : 0.f);
 
             if (warp_has_rows) {
-                __nv_bfloat16* orow = p.out + ((((size_t)u.layer * p.B + u.b) * p.n + node) * (size_t)p.Hq + u.g * p.G + hl) * D;
-                float* lse_ptr = p.lse_out ? p.lse_out + (((size_t)u.layer * p.B + u.b) * p.Hq + u.g * p.G + hl) * p.n + node : nullptr;
-                if (whole_unit) {
-                    const float inv = 1.f / l_run;
+                __nv_bfloat16* orow = p.out + ((((size_t)u.layer * p.B + u.b) * p.n + node) * (size_t)p.Hq + u.g * p.G + hl) * D + grp * kDH;
+                float* lse_ptr = (p.lse_out && grp == 0) ? p.lse_out + (((size_t)u.layer * p.B + u.b) * p.Hq + u.g * p.G + hl) * p.n + node : nullptr;
+                // groups ga..gb cover this unit (group g owns tiles [total*g/n_groups, total*(g+1)/n_groups))
+                const long long per = total_tiles;
+                int ga = group, gb = group;
+                if (!whole_unit) {
+                    while (ga > 0 && per * ga / n_groups > u.unit_first_tile) --ga;
+                    const long long unit_last = u.unit_first_tile + u.tiles_in_unit - 1;
+                    while (gb + 1 < n_groups && per * (gb + 1) / n_groups <= unit_last) ++gb;
+                }
+                const int slot = (sg.t_first > 0) ? 0 : 1;       // a unit that began before this CTA's range uses slot 0
+                // partial layout [column][row]: a warp's store of one column is one contiguous 128-byte line;
+                // each warp of a pair leaves its own copy of (max, sum) so that its columns stand alone
+                float* my = p.partial + ((size_t)blockIdx.x * 2 + slot) * kRowW * kRows + row_in_blk;
+                const float inv = 1.f / Lsum;
+                // combined accumulator columns [grp*kDH, (grp+1)*kDH) of both groups' O, 32 at a time
 #pragma unroll
-                    for (int c4 = 0; c4 < D / 32; ++c4) {
-                        uint32_t r[32];
-                        ptx::tmem_ld_32x32b_x32(o_taddr + (uint32_t)(c4 * 32), r);
-                        ptx::tmem_ld_wait();
+                for (int c4 = 0; c4 < kDH / 32; ++c4) {
+                    float acc[32];
+                    {
+                        uint32_t ra[32];
+                        if (has0) {
+                            ptx::tmem_ld_32x32b_x32(lane_base + kTmemO + (uint32_t)(grp * kDH + c4 * 32), ra);
+                            ptx::tmem_ld_wait();
+                        }
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) acc[j] = has0 ? w0 * __uint_as_float(ra[j]) : 0.f;
+                        if (has1) {
+                            ptx::tmem_ld_32x32b_x32(lane_base + kTmemO + (uint32_t)(D + grp * kDH + c4 * 32), ra);
+                            ptx::tmem_ld_wait();
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) acc[j] = fmaf(w1, __uint_as_float(ra[j]), acc[j]);
+                        }
+                    }
+                    if (whole_unit) {
                         if (row_ok) {
 #pragma unroll
                             for (int j = 0; j < 4; ++j) {
                                 uint4 v;
-                                v.x = pack_bf16(__uint_as_float(r[j * 8 + 0]) * inv, __uint_as_float(r[j * 8 + 1]) * inv);
-                                v.y = pack_bf16(__uint_as_float(r[j * 8 + 2]) * inv, __uint_as_float(r[j * 8 + 3]) * inv);
-                                v.z = pack_bf16(__uint_as_float(r[j * 8 + 4]) * inv, __uint_as_float(r[j * 8 + 5]) * inv);
-                                v.w = pack_bf16(__uint_as_float(r[j * 8 + 6]) * inv, __uint_as_float(r[j * 8 + 7]) * inv);
+                                v.x = pack_bf16(acc[j * 8 + 0] * inv, acc[j * 8 + 1] * inv);
+                                v.y = pack_bf16(acc[j * 8 + 2] * inv, acc[j * 8 + 3] * inv);
+                                v.z = pack_bf16(acc[j * 8 + 4] * inv, acc[j * 8 + 5] * inv);
+                                v.w = pack_bf16(acc[j * 8 + 6] * inv, acc[j * 8 + 7] * inv);
                                 *reinterpret_cast<uint4*>(orow + c4 * 32 + j * 8) = v;
                             }
                         }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) my[(size_t)(grp * kDH + c4 * 32 + j) * kRows] = acc[j];
                     }
-                    if (lse_ptr && row_ok) *lse_ptr = m_used * p.scale + logf(l_run);
-                    ptx::tc_fence_before();
+                }
+                ptx::tc_fence_before();
+                if (whole_unit) {
+                    if (lse_ptr && row_ok) *lse_ptr = M * p.scale + logf(Lsum);
                 } else {
-                    // ---- the unit is cut across CTA groups: leave a partial, last arrival merges ------------
-                    // groups ga..gb cover this unit (group g owns tiles [total*g/n_groups, total*(g+1)/n_groups))
-                    const long long per = total_tiles;
-                    int ga = group, gb = group;
-                    while (ga > 0 && per * ga / n_groups > u.unit_first_tile) --ga;
-                    const long long unit_last = u.unit_first_tile + u.tiles_in_unit - 1;
-                    while (gb + 1 < n_groups && per * (gb + 1) / n_groups <= unit_last) ++gb;
+                    // ---- the unit is cut across CTA groups: the partial is left, the last arrival merges ------
                     const int parts = gb - ga + 1;
-                    const int slot = (sg.t_first > 0) ? 0 : 1;   // a unit that began before this CTA's range uses slot 0
-                    // partial layout [column][row]: a warp's store of one column is one contiguous 128-byte line
-                    float* my = p.partial + ((size_t)blockIdx.x * 2 + slot) * kRowW * kRows + row_in_blk;
-#pragma unroll
-                    for (int c4 = 0; c4 < D / 32; ++c4) {
-                        uint32_t r[32];
-                        ptx::tmem_ld_32x32b_x32(o_taddr + (uint32_t)(c4 * 32), r);
-                        ptx::tmem_ld_wait();
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) my[(size_t)(c4 * 32 + j) * kRows] = __uint_as_float(r[j]);
-                    }
-                    my[(size_t)D * kRows] = m_used;
-                    my[(size_t)(D + 1) * kRows] = l_run;
-                    ptx::tc_fence_before();
+                    my[(size_t)(D + 2 * grp) * kRows] = M;
+                    my[(size_t)(D + 2 * grp + 1) * kRows] = Lsum;
                     __threadfence();
                     __syncwarp();
                     const size_t unit_idx = ((size_t)u.layer * p.B + u.b) * p.Hkv + u.g;
-                    int* tk = p.ticket + (unit_idx * p.n_rb + rb) * kMergeWarps + w4;
+                    int* tk = p.ticket + (unit_idx * p.n_rb + rb) * kMergeWarps + (grp * 4 + w4);
                     int arrived = 0;
                     if (lane == 0) arrived = atomicAdd(tk, 1);
                     arrived = __shfl_sync(0xffffffffu, arrived, 0);
@@ -603,43 +703,62 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                         __threadfence();
                         if (lane == 0) *tk = 0;                          // ready for the next launch
                         // merge in group order
-                        float M = -INFINITY;
+                        float Mm = -INFINITY;
                         for (int gsrc = ga; gsrc <= gb; ++gsrc) {
                             const int sslot = (per * gsrc / n_groups > u.unit_first_tile) ? 0 : 1;
                             const float* src = p.partial + ((size_t)(gsrc * p.n_rb + rb) * 2 + sslot) * kRowW * kRows + row_in_blk;
-                            M = fmaxf(M, __ldcg(src + (size_t)D * kRows));
+                            Mm = fmaxf(Mm, __ldcg(src + (size_t)(D + 2 * grp) * kRows));
                         }
-                        float Lsum = 0.f;
-                        float acc[D];
-#pragma unroll
-                        for (int j = 0; j < D; ++j) acc[j] = 0.f;
+                        float Lm = 0.f;
                         for (int gsrc = ga; gsrc <= gb; ++gsrc) {
                             const int sslot = (per * gsrc / n_groups > u.unit_first_tile) ? 0 : 1;
                             const float* src = p.partial + ((size_t)(gsrc * p.n_rb + rb) * 2 + sslot) * kRowW * kRows + row_in_blk;
-                            const float pm = __ldcg(src + (size_t)D * kRows);
-                            const float wgt = (pm == -INFINITY) ? 0.f : exp2f((pm - M) * p.scale_log2e);
-                            Lsum += wgt * __ldcg(src + (size_t)(D + 1) * kRows);
-#pragma unroll
-                            for (int j = 0; j < D; ++j) acc[j] += wgt * __ldcg(src + (size_t)j * kRows);
+                            const float pm = __ldcg(src + (size_t)(D + 2 * grp) * kRows);
+                            Lm += ((pm == -INFINITY) ? 0.f : exp2f((pm - Mm) * p.scale_log2e)) * __ldcg(src + (size_t)(D + 2 * grp + 1) * kRows);
                         }
-                        if (row_ok) {
-                            const float inv = 1.f / Lsum;
+                        const float invm = 1.f / Lm;
+#pragma unroll 1
+                        for (int c4 = 0; c4 < kDH / 32; ++c4) {
+                            float acc[32];
 #pragma unroll
-                            for (int j = 0; j < D / 8; ++j) {
-                                uint4 v;
-                                v.x = pack_bf16(acc[j * 8 + 0] * inv, acc[j * 8 + 1] * inv);
-                                v.y = pack_bf16(acc[j * 8 + 2] * inv, acc[j * 8 + 3] * inv);
-                                v.z = pack_bf16(acc[j * 8 + 4] * inv, acc[j * 8 + 5] * inv);
-                                v.w = pack_bf16(acc[j * 8 + 6] * inv, acc[j * 8 + 7] * inv);
-                                *reinterpret_cast<uint4*>(orow + j * 8) = v;
+                            for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+                            for (int gsrc = ga; gsrc <= gb; ++gsrc) {
+                                const int sslot = (per * gsrc / n_groups > u.unit_first_tile) ? 0 : 1;
+                                const float* src = p.partial + ((size_t)(gsrc * p.n_rb + rb) * 2 + sslot) * kRowW * kRows + row_in_blk;
+                                const float pm = __ldcg(src + (size_t)(D + 2 * grp) * kRows);
+                                const float wgt = (pm == -INFINITY) ? 0.f : exp2f((pm - Mm) * p.scale_log2e);
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) acc[j] = fmaf(wgt, __ldcg(src + (size_t)(grp * kDH + c4 * 32 + j) * kRows), acc[j]);
                             }
-                            if (lse_ptr) *lse_ptr = M * p.scale + logf(Lsum);
+                            if (row_ok) {
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) {
+                                    uint4 v;
+                                    v.x = pack_bf16(acc[j * 8 + 0] * invm, acc[j * 8 + 1] * invm);
+                                    v.y = pack_bf16(acc[j * 8 + 2] * invm, acc[j * 8 + 3] * invm);
+                                    v.z = pack_bf16(acc[j * 8 + 4] * invm, acc[j * 8 + 5] * invm);
+                                    v.w = pack_bf16(acc[j * 8 + 6] * invm, acc[j * 8 + 7] * invm);
+                                    *reinterpret_cast<uint4*>(orow + c4 * 32 + j * 8) = v;
+                                }
+                            }
                         }
+                        if (lse_ptr && row_ok) *lse_ptr = Mm * p.scale + logf(Lm);
                     }
                 }
+            } else {
+                ptx::tc_fence_before();
             }
+            // both accumulators have been read by this warp: the next unit's P V may overwrite them once all have
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&ctrl->o_free);
+#ifdef MIRROR_ATTN_TIMING
+            t_epi += T_NOW() - te;
+#endif
+            // the exchange words are rewritten at the end of the next part: the partner must have read them
+            if (!pair_sync()) { timeout(p, ctrl, 36); ok = false; break; }
             if (has_next) sg = sg_next;
         }
+        if (warp == 4 && lane == 0) { T_STORE(8, T_NOW() - t0, w_sf, w_pv, w_end, t_epi, t_q, (long long)it); T_STORE(40, s_ld, s_free, s_max, s_xch, s_exp, s_fin); }
     }
 
     ptx::tc_fence_before();
@@ -676,6 +795,10 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
     p.k_new = (const __nv_bfloat16*)k_new; p.v_new = (const __nv_bfloat16*)v_new;
     p.out = (__nv_bfloat16*)out; p.lse_out = lse_out;
     p.partial = partial_ws; p.ticket = ticket_ws; p.status = ctx->d_status;
+    p.timing = nullptr;
+#ifdef MIRROR_ATTN_TIMING
+    if (const char* e = getenv("MIRROR_ATTN_TIMING_PTR")) p.timing = (long long*)strtoull(e, nullptr, 0);
+#endif
     if ((size_t)p.L * p.B * Hkv * p.n_rb * kMergeWarps > ticket_ints) return MIRROR_ERR_WORKSPACE;
     if (p.B > kMaxBatch) return MIRROR_ERR_SHAPE;
 
@@ -688,10 +811,13 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
         const uint64_t total_pages = (uint64_t)(p.L - 1) * p.layer_pages + p.num_pages;
         const uint64_t dims[5] = {64, (uint64_t)kSlotTok, (uint64_t)(D / 64), (uint64_t)Hkv, total_pages};
         const uint64_t strides[4] = {(uint64_t)D * 2, 128, (uint64_t)kSlotTok * D * 2, (uint64_t)page_elems * 2};
-        const uint32_t box[5] = {64, (uint32_t)kSlotTok, 1, 1, 1};
-        mirror_status st = mirror_make_tmap(ctx, &tm_k, kv->k_pool, 5, dims, strides, box);
+        // K: one box per 64-column half (the K-major operand wants all tokens of a half contiguous);
+        // V: one box per page (both halves), which is already the MN-major operand layout of one 16-token step
+        const uint32_t box_k[5] = {64, (uint32_t)kSlotTok, 1, 1, 1};
+        const uint32_t box_v[5] = {64, (uint32_t)kSlotTok, (uint32_t)(D / 64), 1, 1};
+        mirror_status st = mirror_make_tmap(ctx, &tm_k, kv->k_pool, 5, dims, strides, box_k);
         if (st != MIRROR_OK) return st;
-        st = mirror_make_tmap(ctx, &tm_v, kv->v_pool, 5, dims, strides, box);
+        st = mirror_make_tmap(ctx, &tm_v, kv->v_pool, 5, dims, strides, box_v);
         if (st != MIRROR_OK) return st;
     }
     const int grid = p.n_groups * p.n_rb;

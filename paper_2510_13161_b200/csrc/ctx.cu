@@ -146,7 +146,7 @@ void mirror_ws_layout(const mirror_ctx* ctx, size_t M, MirrorWsLayout* out) {
     at += kWsTicketBytes;
     L.attn_partial = at;
     // two partial slots per CTA (a CTA's range of KV tiles cuts at most two units), 128 rows each
-    L.attn_partial_bytes = align_up((size_t)ctx->num_sms * 2 * 128 * (size_t)(ctx->desc.head_dim + 2) * sizeof(float), 256);
+    L.attn_partial_bytes = align_up((size_t)ctx->num_sms * 2 * 128 * (size_t)(ctx->desc.head_dim + 4) * sizeof(float), 256);
     at += L.attn_partial_bytes;
     L.end_attn = at;
     L.lm_partial = at;
