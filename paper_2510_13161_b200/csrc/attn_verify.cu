@@ -81,7 +81,8 @@ struct UnitPos {                          // where a global tile index falls
 };
 
 struct Ctrl {
-    uint64_t kv_full[kKVStages], kv_empty[kKVStages];   // one stage = a K tile and a V tile
+    uint64_t k_full[kKVStages], k_empty[kKVStages];     // K ring: refilled as soon as Q K^T has read a stage
+    uint64_t v_full[kKVStages], v_empty[kKVStages];     // V ring: refilled once P V has read a stage
     uint64_t s_full[kSBufs], s_free[kSBufs];
     uint64_t p_full[2], pv_done[2];
     uint64_t q_full;
@@ -214,7 +215,10 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         s_len[b] = len;
     }
     if (tid == 0) {
-        for (int s = 0; s < kKVStages; ++s) { ptx::mbar_init(&ctrl->kv_full[s], 2); ptx::mbar_init(&ctrl->kv_empty[s], 2); }
+        for (int s = 0; s < kKVStages; ++s) {
+            ptx::mbar_init(&ctrl->k_full[s], 1); ptx::mbar_init(&ctrl->k_empty[s], 1);
+            ptx::mbar_init(&ctrl->v_full[s], 1); ptx::mbar_init(&ctrl->v_empty[s], 1);
+        }
         for (int s = 0; s < kSBufs; ++s) { ptx::mbar_init(&ctrl->s_full[s], 1); ptx::mbar_init(&ctrl->s_free[s], kSoftmaxWarps / 2); }
         for (int s = 0; s < 2; ++s) { ptx::mbar_init(&ctrl->p_full[s], kSoftmaxWarps / 2); ptx::mbar_init(&ctrl->pv_done[s], 1); }
         ptx::mbar_init(&ctrl->q_full, kSoftmaxWarps);
@@ -255,6 +259,8 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         // warp 0 stages K, the last warp stages V: a warp issues its TMA boxes one after the other, so two
         // warps halve the time a stage takes to request
         const bool vrole = (warp == kVProducerWarp);
+        uint64_t* const full = vrole ? ctrl->v_full : ctrl->k_full;
+        uint64_t* const empty = vrole ? ctrl->v_empty : ctrl->k_empty;
         uint32_t it = 0;                   // tiles issued by this CTA so far (ring index and parity source)
         bool ok = true;
         long long x = x_begin;
@@ -278,7 +284,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 const uint32_t ph = (it / kKVStages) & 1;
                 const int next_page = (t + 1 < sg.t_last) ? fetch_page(t + 1) : 0;
                 bool w = true;
-                if (lane == 0) w = !ctrl->abort && T_WAIT(w_empty, ptx::mbar_wait(&ctrl->kv_empty[st], ph ^ 1));
+                if (lane == 0) w = !ctrl->abort && T_WAIT(w_empty, ptx::mbar_wait(&empty[st], ph ^ 1));
                 w = __shfl_sync(0xffffffffu, w, 0);
                 if (!w) { if (lane == 0) timeout(p, ctrl, 10); ok = false; break; }
                 uint8_t* dst = (vrole ? sV : sK) + (size_t)st * C::kStageBytes;
@@ -323,16 +329,16 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     ptx::fence_proxy_async();
                     __syncwarp();
                 }
-                if (lane == 0) ptx::mbar_arrive_expect_tx(&ctrl->kv_full[st], (uint32_t)(n_tma * C::kVSlotBytes));
+                if (lane == 0) ptx::mbar_arrive_expect_tx(&full[st], (uint32_t)(n_tma * C::kVSlotBytes));
                 __syncwarp();
                 if (has_box && my_slot < n_tma) {
                     int page = my_page;
                     if (page < 0 || page >= p.num_pages) { dev_check(p, 400); page = 0; }
                     const int pg = u.layer * p.layer_pages + page;
                     if (vrole)
-                        ptx::tma_load_5d(dst + my_slot * C::kVSlotBytes, &tm_v, &ctrl->kv_full[st], 0, 0, 0, u.g, pg);
+                        ptx::tma_load_5d(dst + my_slot * C::kVSlotBytes, &tm_v, &full[st], 0, 0, 0, u.g, pg);
                     else
-                        ptx::tma_load_5d(dst + my_half * kKVHalfBytes + my_slot * C::kSlotBoxBytes, &tm_k, &ctrl->kv_full[st], 0, 0, my_half, u.g, pg);
+                        ptx::tma_load_5d(dst + my_half * kKVHalfBytes + my_slot * C::kSlotBoxBytes, &tm_k, &full[st], 0, 0, my_half, u.g, pg);
                 }
                 my_page = next_page;
             }
@@ -342,7 +348,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             // let copies already in flight land before the CTA's shared memory goes away
             const uint32_t back = it < (uint32_t)kKVStages ? it : (uint32_t)kKVStages;
             for (uint32_t j = it - back; j < it; ++j)
-                ptx::mbar_wait(&ctrl->kv_full[j & (kKVStages - 1)], (j / kKVStages) & 1, 200000000ll);
+                ptx::mbar_wait(&full[j & (kKVStages - 1)], (j / kKVStages) & 1, 200000000ll);
         }
     } else if (warp == 1) {
         // =========================================================================== Q K^T issuer
@@ -362,7 +368,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 ++seg;
                 for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
                     const int st = it & (kKVStages - 1), sb = it & (kSBufs - 1);
-                    if (ctrl->abort || !T_WAIT(w_k, ptx::mbar_wait(&ctrl->kv_full[st], (it / kKVStages) & 1)) ||
+                    if (ctrl->abort || !T_WAIT(w_k, ptx::mbar_wait(&ctrl->k_full[st], (it / kKVStages) & 1)) ||
                         !T_WAIT(w_s, ptx::mbar_wait(&ctrl->s_free[sb], ((it / kSBufs) & 1) ^ 1))) {
                         timeout(p, ctrl, 21); ok = false; break;
                     }
@@ -375,7 +381,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     for (int kk = 0; kk < D / 16; ++kk)
                         ptx::umma_f16_lohi(d, q_lo + (uint32_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4), hi,
                                            kb + (uint32_t)(((kk >> 2) * kKVHalfBytes + (kk & 3) * 32) >> 4), hi, idesc, kk != 0);
-                    ptx::umma_commit(&ctrl->kv_empty[st]);
+                    ptx::umma_commit(&ctrl->k_empty[st]);
                     ptx::umma_commit(&ctrl->s_full[sb]);
                 }
             }
@@ -401,7 +407,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
                     const int st = it & (kKVStages - 1), pb = it & 1;
                     if (ctrl->abort || !T_WAIT(w_p, ptx::mbar_wait(&ctrl->p_full[pb], (it >> 1) & 1)) ||
-                        !T_WAIT(w_v, ptx::mbar_wait(&ctrl->kv_full[st], (it / kKVStages) & 1))) {
+                        !T_WAIT(w_v, ptx::mbar_wait(&ctrl->v_full[st], (it / kKVStages) & 1))) {
                         timeout(p, ctrl, 23); ok = false; break;
                     }
                     ptx::tc_fence_after();
@@ -413,7 +419,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                         if (k < n_slots)
                             ptx::umma_f16_lohi(tmem_base + kTmemO + (uint32_t)(pb * D), pa + (uint32_t)(k * 2), hi,
                                                vb + (uint32_t)(k * (C::kVSlotBytes / 16)), hi, idesc_pv, (t >= sg.t_first + 2) || (k != 0));
-                    ptx::umma_commit(&ctrl->kv_empty[st]);
+                    ptx::umma_commit(&ctrl->v_empty[st]);
                     ptx::umma_commit(&ctrl->pv_done[pb]);
                 }
             }
