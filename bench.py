@@ -127,10 +127,12 @@ class ClockSampler:
 # ---------------------------------------------------------------------------------------------------
 # CPU oracle timing (cpu_baseline leg and --impl reference)
 # ---------------------------------------------------------------------------------------------------
-def oracle_sample_seconds(x, cfg, vocab_slices: int = 8):
-    """Times the oracle, as it stands, on a bounded sample of one step: ONE of the attention layers (all
-    requests and rows) and the LM head on all rows over the first 1/vocab_slices of the vocabulary plus
-    the acceptance rule.  Returns (sample seconds, extrapolated seconds for a whole step, description)."""
+def oracle_sample_seconds(x, cfg, target_seconds: float = 15.0):
+    """Times the oracle, as it stands, on a bounded sample of one step.  A short calibration (one attention
+    layer, 1/16 of the vocabulary) sizes the sample to about `target_seconds` of CPU work: `n_layers` of the
+    attention layers (all requests and rows; layers cost the same, so one layer's tensors are reused) and the
+    LM head + reductions + acceptance on all rows over the first `vocab_frac` of the vocabulary.  Returns
+    (sample seconds, extrapolated seconds for a whole step, description)."""
     import numpy as np
     from oracle import oracle as O
     from paper_2510_13161_b200 import inputs as I
@@ -139,23 +141,36 @@ def oracle_sample_seconds(x, cfg, vocab_slices: int = 8):
     pt, pl = x.page_table.cpu().numpy(), x.prefix_len.cpu().numpy()
     args = (I.bf16_bits(x.q[0]), I.bf16_bits(x.k_pool[0]), I.bf16_bits(x.v_pool[0]), pt, pl,
             I.bf16_bits(x.k_new[0]), I.bf16_bits(x.v_new[0]), anc, scale)
-    vs = cfg.vocab // vocab_slices
-    Wb = I.bf16_bits(x.W[:vs])
-    t0 = time.perf_counter()
-    out, _, _ = O.attention_layer(*args)
-    t1 = time.perf_counter()
-    hid = out.reshape(cfg.rows, -1) if x.hidden is None else I.bf16_bits(x.hidden)
-    if hid.shape[1] != cfg.hidden:
-        hid = I.bf16_bits(x.hidden)
-    logits = O.lmhead_logits(hid, Wb)
-    red = O.row_reduce(logits)
     tok = x.tokens.cpu().numpy()
-    O.accept_greedy(tok, red["argmax"].reshape(tok.shape), x.parent, cfg.gamma)
-    t2 = time.perf_counter()
-    sample = t2 - t0
-    full = (t1 - t0) * cfg.layers + (t2 - t1) * vocab_slices
-    desc = (f"1 of {cfg.layers} attention layers (all rows) + LM head / reductions / acceptance over the first "
-            f"1/{vocab_slices} of the vocabulary; whole-step time extrapolated linearly")
+
+    def attn_layers(n):
+        t = time.perf_counter()
+        out = None
+        for _ in range(n):
+            out, _, _ = O.attention_layer(*args)
+        return time.perf_counter() - t, out
+
+    def lm_slice(out, rows_v):
+        t = time.perf_counter()
+        hid = I.bf16_bits(x.hidden) if x.hidden is not None else out.reshape(cfg.rows, -1)
+        logits = O.lmhead_logits(hid, I.bf16_bits(x.W[:rows_v]))
+        red = O.row_reduce(logits)
+        O.accept_greedy(tok, red["argmax"].reshape(tok.shape), x.parent, cfg.gamma)
+        return time.perf_counter() - t
+
+    # calibration (not part of the timed sample)
+    t_layer, out = attn_layers(1)
+    v_cal = max(1024, cfg.vocab // 16)
+    t_lm_cal = lm_slice(out, v_cal)
+    n_layers = int(max(1, min(cfg.layers, round(0.5 * target_seconds / max(t_layer, 1e-6)))))
+    rows_v = int(max(v_cal, min(cfg.vocab, round(v_cal * 0.5 * target_seconds / max(t_lm_cal, 1e-6)))))
+    # timed sample
+    t_attn, out = attn_layers(n_layers)
+    t_lm = lm_slice(out, rows_v)
+    sample = t_attn + t_lm
+    full = t_attn * cfg.layers / n_layers + t_lm * cfg.vocab / rows_v
+    desc = (f"{n_layers} of {cfg.layers} attention layers (all rows) + LM head / reductions / acceptance over the first "
+            f"{rows_v} of {cfg.vocab} vocabulary rows; whole-step time extrapolated linearly")
     return sample, full, desc
 
 
@@ -168,9 +183,9 @@ def run_reference(args):
     from paper_2510_13161_b200 import inputs as I
     cfg = I.CONFIGS[args.workload]
     x = I.gen_verify_inputs(cfg, args.seed, "cpu", layers=1, force_hidden=cfg.explicit_hidden)
-    steps, warm = max(1, min(args.steps, 3)), max(0, min(args.warmup, 1))
+    steps, warm = max(1, min(args.steps, 4)), max(0, min(args.warmup, 1))
     for _ in range(warm):
-        oracle_sample_seconds(x, cfg)
+        oracle_sample_seconds(x, cfg, 5.0)
     fulls, samples, desc = [], [], ""
     for _ in range(steps):
         s, f, desc = oracle_sample_seconds(x, cfg)
@@ -187,6 +202,23 @@ def run_reference(args):
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
+
+
+def max_over_ranks(value: float, device=None) -> float:
+    """Max of a per-rank scalar over the process group (the slowest rank sets the job's time); identity
+    without a process group.  Works on any backend: the multi-process CPU test drives it under gloo."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(steps_per_rank: int, world: int, ms_max: float) -> float:
+    """Whole-job steps/s of `world` independent replicas that each ran `steps_per_rank` steps in `ms_max` ms."""
+    return world * steps_per_rank * 1e3 / ms_max
 
 
 # ---------------------------------------------------------------------------------------------------
@@ -251,13 +283,9 @@ def run_mirror(args):
     barrier()
     clocks = sampler.stop()
     launches = m.launch_count() - launches0
-    ms_total = ev0.elapsed_time(ev1)
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
+    ms_total = max_over_ranks(ev0.elapsed_time(ev1), dev)
     ms_step = ms_total / K
-    value = world * 1e3 / ms_step
+    value = job_throughput(K, world, ms_total)
     attn_ms = sum(e[0].elapsed_time(e[1]) for e in stage_ev) / K
     lm_ms = sum(e[1].elapsed_time(e[2]) for e in stage_ev) / K
     tail_ms = sum(e[2].elapsed_time(e[3]) for e in stage_ev) / K
@@ -292,10 +320,7 @@ def run_mirror(args):
         e2e_step()
     e1.record(stream)
     barrier()
-    te = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(te, op=dist.ReduceOp.MAX)
-    e2e_value = world * 1e3 / (float(te.item()) / Ke)
+    e2e_value = job_throughput(Ke, world, max_over_ranks(e0.elapsed_time(e1), dev))
 
     if rank != 0:
         if world > 1:
