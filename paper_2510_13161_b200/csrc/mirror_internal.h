@@ -119,19 +119,30 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Bounded wait: spins on try_wait, and once the fast path has failed keeps an eye on the SM cycle counter;
-// gives up after `limit_cycles` (about 2 s at 2 GHz by default).  Returns false on expiry; the caller then
-// records the failure and unwinds (no trap, no endless spin).  The cycle counter is read only on the slow
-// path: a wait that is satisfied quickly costs nothing but the try_wait itself.
+// try_wait that lets the hardware park the thread (up to `ns` nanoseconds) until the phase completes, instead of
+// returning at once: a hot spin on try_wait issues a shared-memory operation every few cycles and starves the
+// warps that share the SM's shared-memory pipeline.
+__device__ __forceinline__ bool mbar_try_wait_park(uint64_t* bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait.  One plain try_wait first (the common case: the phase is already complete); after that the
+// thread parks in the barrier unit for up to 20 us at a time and keeps an eye on the SM cycle counter: it gives
+// up after `limit_cycles` (about 2 s at 2 GHz by default).  Returns false on expiry; the caller then records
+// the failure and unwinds (no trap, no endless spin).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, long long limit_cycles = 4000000000ll) {
-#pragma unroll 1
-    for (int i = 0; i < 256; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
-#pragma unroll 1
-        for (int i = 0; i < 64; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait_park(bar, parity, 20000u)) return true;
         if (clock64() - t0 > limit_cycles) return false;
     }
 }
