@@ -125,6 +125,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // index is XORed with (row % 8).  A half of Q or P holds 128 rows (16 KB), a half of a K/V stage 64 tokens (8 KB).
 constexpr int kHalfBytes = kRows * 128;
 constexpr int kKVHalfBytes = kTileTok * 128;
+constexpr int kKRingHalfBytes = kKVStages * kKVHalfBytes;   // K ring: [half][stage][64 tokens][128 B], so that two
+                                                            // consecutive stages form one 128-token K-major operand
 __device__ __forceinline__ uint32_t tile_off(int row, int chunk, int half_bytes) {   // chunk: 16-byte column chunk
     return (uint32_t)((chunk >> 3) * half_bytes + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
 }
@@ -287,7 +289,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 if (lane == 0) w = !ctrl->abort && T_WAIT(w_empty, ptx::mbar_wait(&empty[st], ph ^ 1));
                 w = __shfl_sync(0xffffffffu, w, 0);
                 if (!w) { if (lane == 0) timeout(p, ctrl, 10); ok = false; break; }
-                uint8_t* dst = (vrole ? sV : sK) + (size_t)st * C::kStageBytes;
+                uint8_t* dst = vrole ? sV + (size_t)st * C::kStageBytes : sK + (size_t)st * kKVHalfBytes;
                 const int sl0 = t * kTileSlots;
                 const int n_slots = min(kTileSlots, sg.slots_all - sl0);               // slots that exist in this tile
                 const int n_tma = max(0, min(kTileSlots, sg.pages_full - sl0));        // leading slots that are whole pages
@@ -322,15 +324,15 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                         for (int i = 0; i < kPer; ++i) {
                             const int c = lane + i * 32, tr = c / (D / 8), cc = c % (D / 8);
                             if (vrole) *reinterpret_cast<uint4*>(dst + j * C::kVSlotBytes + tile_off(tr, cc, kSlotTok * 128)) = vv[i];
-                            else *reinterpret_cast<uint4*>(dst + tile_off(j * kSlotTok + tr, cc, kKVHalfBytes)) = vv[i];
+                            else *reinterpret_cast<uint4*>(dst + tile_off(j * kSlotTok + tr, cc, kKRingHalfBytes)) = vv[i];
                         }
                     }
                     // the plain stores are read by the tensor core, and later overwritten by bulk copies (async proxy)
                     ptx::fence_proxy_async();
                     __syncwarp();
                 }
+                // (the barrier's one arrival is this arming, so copies that land before it cannot complete the phase)
                 if (lane == 0) ptx::mbar_arrive_expect_tx(&full[st], (uint32_t)(n_tma * C::kVSlotBytes));
-                __syncwarp();
                 if (has_box && my_slot < n_tma) {
                     int page = my_page;
                     if (page < 0 || page >= p.num_pages) { dev_check(p, 400); page = 0; }
@@ -338,7 +340,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     if (vrole)
                         ptx::tma_load_5d(dst + my_slot * C::kVSlotBytes, &tm_v, &full[st], 0, 0, 0, u.g, pg);
                     else
-                        ptx::tma_load_5d(dst + my_half * kKVHalfBytes + my_slot * C::kSlotBoxBytes, &tm_k, &full[st], 0, 0, my_half, u.g, pg);
+                        ptx::tma_load_5d(dst + my_half * kKRingHalfBytes + my_slot * C::kSlotBoxBytes, &tm_k, &full[st], 0, 0, my_half, u.g, pg);
                 }
                 my_page = next_page;
             }
@@ -357,7 +359,6 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             const uint32_t hi = ptx::umma_desc_hi_sw128(1024);
             const uint32_t q_lo = ptx::umma_desc_lo(ptx::smem_u32(sQ), 16);
             const uint32_t k_lo = ptx::umma_desc_lo(ptx::smem_u32(sK), 16);
-            const uint32_t idesc_full = ptx::umma_idesc_bf16(kRows, kTileTok);
             uint32_t it = 0, seg = 0;
             bool ok = true;
             long long x = x_begin;
@@ -366,24 +367,33 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 const Segment sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
                 if (ctrl->abort || !T_WAIT(w_q, ptx::mbar_wait(&ctrl->q_full, seg & 1))) { timeout(p, ctrl, 20); ok = false; break; }
                 ++seg;
-                for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
-                    const int st = it & (kKVStages - 1), sb = it & (kSBufs - 1);
-                    if (ctrl->abort || !T_WAIT(w_k, ptx::mbar_wait(&ctrl->k_full[st], (it / kKVStages) & 1)) ||
-                        !T_WAIT(w_s, ptx::mbar_wait(&ctrl->s_free[sb], ((it / kSBufs) & 1) ^ 1))) {
-                        timeout(p, ctrl, 21); ok = false; break;
+                int t = sg.t_first;
+                while (t < sg.t_last) {
+                    // two consecutive tiles whose stages are an aligned pair of the K ring are scored by one N=128 UMMA set
+                    const bool pair = ((it & 1) == 0) && (t + 1 < sg.t_last);
+                    const int nt = pair ? 2 : 1;
+                    bool ready = !ctrl->abort;
+                    for (int j = 0; j < nt && ready; ++j) {
+                        const uint32_t i2 = it + j;
+                        ready = T_WAIT(w_k, ptx::mbar_wait(&ctrl->k_full[i2 & (kKVStages - 1)], (i2 / kKVStages) & 1)) &&
+                                T_WAIT(w_s, ptx::mbar_wait(&ctrl->s_free[i2 & (kSBufs - 1)], ((i2 / kSBufs) & 1) ^ 1));
                     }
+                    if (!ready) { timeout(p, ctrl, 21); ok = false; break; }
                     ptx::tc_fence_after();
-                    const int n_slots = min(kTileSlots, sg.slots_all - t * kTileSlots);
-                    const uint32_t idesc = n_slots == kTileSlots ? idesc_full : ptx::umma_idesc_bf16(kRows, n_slots * kSlotTok);
-                    const uint32_t kb = k_lo + (uint32_t)((st * C::kStageBytes) >> 4);
+                    const int st = it & (kKVStages - 1), sb = it & (kSBufs - 1);
+                    const int n_tok = min(nt * kTileTok, (sg.slots_all - t * kTileSlots) * kSlotTok);
+                    const uint32_t idesc = ptx::umma_idesc_bf16(kRows, n_tok);
+                    const uint32_t kb = k_lo + (uint32_t)((st * kKVHalfBytes) >> 4);
                     const uint32_t d = tmem_base + (uint32_t)(sb * kTileTok);
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk)
                         ptx::umma_f16_lohi(d, q_lo + (uint32_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4), hi,
-                                           kb + (uint32_t)(((kk >> 2) * kKVHalfBytes + (kk & 3) * 32) >> 4), hi, idesc, kk != 0);
-                    ptx::umma_commit(&ctrl->k_empty[st]);
-                    ptx::umma_commit(&ctrl->s_full[sb]);
+                                           kb + (uint32_t)(((kk >> 2) * kKRingHalfBytes + (kk & 3) * 32) >> 4), hi, idesc, kk != 0);
+                    for (int j = 0; j < nt; ++j) ptx::umma_commit(&ctrl->k_empty[(it + j) & (kKVStages - 1)]);
+                    for (int j = 0; j < nt; ++j) ptx::umma_commit(&ctrl->s_full[(it + j) & (kSBufs - 1)]);
+                    t += nt; x += nt; it += nt;
                 }
+                if (!ok) break;
             }
             T_STORE(0, T_NOW() - t0, w_q, w_k, w_s, (long long)it);
         }
