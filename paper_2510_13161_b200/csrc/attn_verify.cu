@@ -266,7 +266,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         uint32_t it = 0;                   // tiles issued by this CTA so far (ring index and parity source)
         bool ok = true;
         long long x = x_begin;
-        T_DECL(w_empty = 0, t0 = T_NOW());
+        T_DECL(w_empty = 0, t0 = T_NOW(), tm__ = 0, p_pre = 0, p_issue = 0, p_fill = 0);
         // one TMA box per lane: K wants (slot, half) boxes, V one box per slot (both halves)
         const int n_boxes = vrole ? kTileSlots : kTileSlots * C::kHalves;
         const bool has_box = lane < n_boxes;
@@ -282,6 +282,9 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             };
             int my_page = fetch_page(sg.t_first);
             for (int t = sg.t_first; t < sg.t_last && ok; ++t, ++x, ++it) {
+#ifdef MIRROR_ATTN_TIMING
+                tm__ = T_NOW();
+#endif
                 const int st = it & (kKVStages - 1);
                 const uint32_t ph = (it / kKVStages) & 1;
                 const int next_page = (t + 1 < sg.t_last) ? fetch_page(t + 1) : 0;
@@ -293,6 +296,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 const int sl0 = t * kTileSlots;
                 const int n_slots = min(kTileSlots, sg.slots_all - sl0);               // slots that exist in this tile
                 const int n_tma = max(0, min(kTileSlots, sg.pages_full - sl0));        // leading slots that are whole pages
+                T_MARK(p_pre);
                 if (n_tma < n_slots) {
                     // ragged page and tree tokens by plain loads (rows beyond the valid count are zero)
                     for (int j = n_tma; j < n_slots; ++j) {
@@ -331,6 +335,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     ptx::fence_proxy_async();
                     __syncwarp();
                 }
+                T_MARK(p_fill);
                 // (the barrier's one arrival is this arming, so copies that land before it cannot complete the phase)
                 if (lane == 0) ptx::mbar_arrive_expect_tx(&full[st], (uint32_t)(n_tma * C::kVSlotBytes));
                 if (has_box && my_slot < n_tma) {
@@ -343,9 +348,10 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                         ptx::tma_load_5d(dst + my_half * kKRingHalfBytes + my_slot * C::kSlotBoxBytes, &tm_k, &full[st], 0, 0, my_half, u.g, pg);
                 }
                 my_page = next_page;
+                T_MARK(p_issue);
             }
         }
-        if (lane == 0) T_STORE(vrole ? 32 : 16, T_NOW() - t0, w_empty, (long long)it);
+        if (lane == 0) T_STORE(vrole ? 32 : 16, T_NOW() - t0, w_empty, (long long)it, p_pre, p_fill, p_issue);
         if (!ok && lane == 0) {
             // let copies already in flight land before the CTA's shared memory goes away
             const uint32_t back = it < (uint32_t)kKVStages ? it : (uint32_t)kKVStages;
