@@ -5,7 +5,9 @@
 // Work decomposition.  A "unit" is (layer, request, KV head): all G = Hq/Hkv query heads of all n tree
 // nodes (G*n rows) share that head's K/V stream, so one CTA owning the unit's rows reads each K/V byte
 // once from HBM and reuses it from shared memory for every row (the GQA / tree sharing).  A unit's keys
-// are cut into 16-token slots (one KV page, or 16 tree tokens) and 64-token tiles.  The tiles of all
+// are cut into 16-token slots (one KV page, or 16 tree tokens); eight slots form a pair of 64-token tiles: tile 0
+// of the pair holds the first eight tokens of each of the eight slots, tile 1 the second eight (so that a whole
+// page is one TMA box and still a legal UMMA operand: the 8-row groups of one tile are a slot apart).  The tiles of all
 // units form one sequence that is split evenly over persistent CTAs (one per SM), so a unit may be cut
 // across CTAs; each CTA then leaves a partial (max, sum, accumulator) and the last one to arrive at the
 // unit's counter merges them in a fixed order.  No CTA ever waits for another.
@@ -13,10 +15,10 @@
 // same time, each with its own rows, so the second read of a tile is served by L2.
 //
 // Per CTA (12 warps):
-//   warp 0, 11  stage K and V tiles into two 4-deep rings: TMA boxes per page with 128-byte swizzle (K: one per
-//               64-column half, V: one per page); ragged page and tree tokens by plain loads with zero fill
-//   warp 1      owns TMEM and issues S = Q K^T (tcgen05.mma, M=128 rows, N=tokens of the tile) into one of
-//               four S buffers, as far ahead as the K ring and the S buffers allow
+//   warp 0, 11  stage K and V into two 4-deep rings of 4-slot stages: one TMA box per page and tensor, 128-byte
+//               swizzle; ragged page and tree tokens by plain loads with zero fill
+//   warp 1      owns TMEM and issues S = Q K^T for a pair of tiles at a time (tcgen05.mma, M=128 rows, N=64 per
+//               tile, 8-row groups 4096 B apart) into two of four S buffers, as far ahead as the rings allow
 //   warp 2      issues O += P V (P from shared memory, V as an MN-major operand)
 //   warps 3..10 softmax, two groups of four warps on alternate tiles, one thread per row (TMEM lane):
 //               tcgen05.ld of the row's scores, mask in registers, online softmax without any shuffle, P written
@@ -124,9 +126,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // Shared-memory operand tiles are [64-column half][row][128 B] with the 128-byte swizzle: the 16-byte chunk
 // index is XORed with (row % 8).  A half of Q or P holds 128 rows (16 KB), a half of a K/V stage 64 tokens (8 KB).
 constexpr int kHalfBytes = kRows * 128;
-constexpr int kKVHalfBytes = kTileTok * 128;
-constexpr int kKRingHalfBytes = kKVStages * kKVHalfBytes;   // K ring: [half][stage][64 tokens][128 B], so that two
-                                                            // consecutive stages form one 128-token K-major operand
+constexpr int kStageSlots = 4;                      // slots per ring stage
 __device__ __forceinline__ uint32_t tile_off(int row, int chunk, int half_bytes) {   // chunk: 16-byte column chunk
     return (uint32_t)((chunk >> 3) * half_bytes + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
 }
@@ -164,10 +164,9 @@ template <int D>
 struct Cfg {
     static constexpr int kHalves = D / 64;
     static constexpr int kQBytes = kHalves * kHalfBytes;           // Q: 128 rows x D
-    static constexpr int kStageBytes = kHalves * kKVHalfBytes;     // one K (or V) stage: 64 tokens x D
+    static constexpr int kSlotBytes = kHalves * kSlotTok * 128;    // one slot of K or V: [half][16 tokens][128 B] = one TMA box
+    static constexpr int kStageBytes = kStageSlots * kSlotBytes;   // one K (or V) stage: 4 slots; stages are contiguous
     static constexpr int kPBytes = kRows * 128;                    // one P buffer: 128 rows x 64 tokens
-    static constexpr int kSlotBoxBytes = kSlotTok * 128;           // one K box: 16 tokens x 64 columns
-    static constexpr int kVSlotBytes = kHalves * kSlotTok * 128;   // one V box: 16 tokens x D columns, [half][token][128 B]
     static constexpr size_t kSmemData = (size_t)kQBytes + 2 * kPBytes + 2 * (size_t)kKVStages * kStageBytes;
     static constexpr size_t kSmemBytes = kSmemData + 512 /*ctrl*/ + 2 * 2 * kRows * 4 /*pair exchange*/ + (2 * kMaxBatch + 2) * 4 + 1024 /*align*/;
 };
@@ -200,7 +199,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* sQ = smem;
     uint8_t* sP = sQ + C::kQBytes;                                  // [2]
-    uint8_t* sK = sP + 2 * C::kPBytes;                              // [kKVStages]  [half][64 tokens][128 B]
+    uint8_t* sK = sP + 2 * C::kPBytes;                              // [kKVStages]  [slot][half][16 tokens][128 B]
     uint8_t* sV = sK + kKVStages * C::kStageBytes;                  // [kKVStages]  [slot][half][16 tokens][128 B]
     Ctrl* ctrl = (Ctrl*)(sV + kKVStages * C::kStageBytes);
     float* xch = (float*)((uint8_t*)ctrl + 512);                    // [2 tiles][2 halves][128 rows] pair exchange
@@ -219,7 +218,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     if (tid == 0) {
         for (int s = 0; s < kKVStages; ++s) {
             ptx::mbar_init(&ctrl->k_full[s], 1); ptx::mbar_init(&ctrl->k_empty[s], 1);
-            ptx::mbar_init(&ctrl->v_full[s], 1); ptx::mbar_init(&ctrl->v_empty[s], 1);
+            ptx::mbar_init(&ctrl->v_full[s], 1); ptx::mbar_init(&ctrl->v_empty[s], 2);   // both tiles of a pair read a V stage
         }
         for (int s = 0; s < kSBufs; ++s) { ptx::mbar_init(&ctrl->s_full[s], 1); ptx::mbar_init(&ctrl->s_free[s], kSoftmaxWarps / 2); }
         for (int s = 0; s < 2; ++s) { ptx::mbar_init(&ctrl->p_full[s], kSoftmaxWarps / 2); ptx::mbar_init(&ctrl->pv_done[s], 1); }
@@ -243,7 +242,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         cumT[0] = 0;
         for (int b = 0; b < p.B; ++b) {
             const int slots = (s_len[b] + kSlotTok - 1) / kSlotTok + p.tree_slots;
-            acc += (slots + kTileSlots - 1) / kTileSlots;
+            acc += 2 * ((slots + 2 * kStageSlots - 1) / (2 * kStageSlots));      // whole pairs of tiles
             cumT[b + 1] = acc;
         }
     }
@@ -251,10 +250,13 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     const uint32_t tmem_base = ctrl->tmem_base;
     const long long tiles_per_layer = (long long)p.Hkv * cumT[p.B];
     const long long total_tiles = tiles_per_layer * p.L;
-    // never more groups than tiles, so that every group's range is non-empty and boundaries are distinct
-    const int n_groups = (int)min((long long)p.n_groups, total_tiles);
-    const long long x_begin = group < n_groups ? total_tiles * group / n_groups : 0;
-    const long long x_end = group < n_groups ? total_tiles * (group + 1) / n_groups : 0;
+    // CTA groups own whole pairs of tiles; never more groups than pairs, so that every group's range is non-empty
+    // and boundaries are distinct
+    const long long total_pairs = total_tiles / 2;
+    const int n_groups = (int)min((long long)p.n_groups, total_pairs);
+    auto group_begin = [&](int g) -> long long { return 2 * (total_pairs * g / n_groups); };
+    const long long x_begin = group < n_groups ? group_begin(group) : 0;
+    const long long x_end = group < n_groups ? group_begin(group + 1) : 0;
 
     if (warp == 0 || warp == kVProducerWarp) {
         // =========================================================================== producers
@@ -267,17 +269,16 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         bool ok = true;
         long long x = x_begin;
         T_DECL(w_empty = 0, t0 = T_NOW(), tm__ = 0, p_pre = 0, p_issue = 0, p_fill = 0);
-        // one TMA box per lane: K wants (slot, half) boxes, V one box per slot (both halves)
-        const int n_boxes = vrole ? kTileSlots : kTileSlots * C::kHalves;
-        const bool has_box = lane < n_boxes;
-        const int my_slot = vrole ? lane : lane / C::kHalves, my_half = lane % C::kHalves;
+        // one TMA box (a whole page of this tensor) per lane
+        const bool has_box = lane < kStageSlots;
+        const int my_slot = lane;
         while (x < x_end && ok) {
             const Segment sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
             const UnitPos& u = sg.u;
             const int32_t* pt = p.page_table + (size_t)u.b * p.max_pages;
             // the page id a lane needs is fetched one tile ahead, so its latency hides behind the ring wait
             auto fetch_page = [&](int tt) -> int {
-                const int sl = tt * kTileSlots + my_slot;
+                const int sl = tt * kStageSlots + my_slot;
                 return (has_box && sl < sg.pages_full) ? pt[sl] : 0;
             };
             int my_page = fetch_page(sg.t_first);
@@ -292,19 +293,24 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 if (lane == 0) w = !ctrl->abort && T_WAIT(w_empty, ptx::mbar_wait(&empty[st], ph ^ 1));
                 w = __shfl_sync(0xffffffffu, w, 0);
                 if (!w) { if (lane == 0) timeout(p, ctrl, 10); ok = false; break; }
-                uint8_t* dst = vrole ? sV + (size_t)st * C::kStageBytes : sK + (size_t)st * kKVHalfBytes;
-                const int sl0 = t * kTileSlots;
-                const int n_slots = min(kTileSlots, sg.slots_all - sl0);               // slots that exist in this tile
-                const int n_tma = max(0, min(kTileSlots, sg.pages_full - sl0));        // leading slots that are whole pages
+                uint8_t* dst = (vrole ? sV : sK) + (size_t)st * C::kStageBytes;
+                const int sl0 = t * kStageSlots;
+                const int n_slots = max(0, min(kStageSlots, sg.slots_all - sl0));      // slots that exist in this stage
+                const int n_tma = max(0, min(kStageSlots, sg.pages_full - sl0));       // leading slots that are whole pages
+                // a pair of tiles is scored on an even number of slots: an odd last slot gets a zero V partner
+                const int n_fill = (vrole && (sg.slots_all & 1) && sl0 <= sg.slots_all && sg.slots_all < sl0 + kStageSlots)
+                                       ? n_slots + 1 : n_slots;
                 T_MARK(p_pre);
-                if (n_tma < n_slots) {
+                if (n_tma < n_fill) {
                     // ragged page and tree tokens by plain loads (rows beyond the valid count are zero)
-                    for (int j = n_tma; j < n_slots; ++j) {
+                    for (int j = n_tma; j < n_fill; ++j) {
                         const int sl = sl0 + j;
-                        const __nv_bfloat16* src;
-                        size_t row_stride;
-                        int valid;
-                        if (sl < sg.pages_all) {
+                        const __nv_bfloat16* src = p.k_pool;
+                        size_t row_stride = 0;
+                        int valid = 0;
+                        if (sl >= sg.slots_all) {
+                            // the zero partner slot
+                        } else if (sl < sg.pages_all) {
                             int page = pt[sl];
                             if (page < 0 || page >= p.num_pages) { if (lane == 0) dev_check(p, 401); page = 0; }
                             src = (vrole ? p.v_pool : p.k_pool) + (((size_t)u.layer * p.layer_pages + page) * p.Hkv + u.g) * (size_t)(kSlotTok * D);
@@ -327,8 +333,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 #pragma unroll
                         for (int i = 0; i < kPer; ++i) {
                             const int c = lane + i * 32, tr = c / (D / 8), cc = c % (D / 8);
-                            if (vrole) *reinterpret_cast<uint4*>(dst + j * C::kVSlotBytes + tile_off(tr, cc, kSlotTok * 128)) = vv[i];
-                            else *reinterpret_cast<uint4*>(dst + tile_off(j * kSlotTok + tr, cc, kKRingHalfBytes)) = vv[i];
+                            *reinterpret_cast<uint4*>(dst + j * C::kSlotBytes + tile_off(tr, cc, kSlotTok * 128)) = vv[i];
                         }
                     }
                     // the plain stores are read by the tensor core, and later overwritten by bulk copies (async proxy)
@@ -337,15 +342,15 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 }
                 T_MARK(p_fill);
                 // (the barrier's one arrival is this arming, so copies that land before it cannot complete the phase)
-                if (lane == 0) ptx::mbar_arrive_expect_tx(&full[st], (uint32_t)(n_tma * C::kVSlotBytes));
+                if (lane == 0) ptx::mbar_arrive_expect_tx(&full[st], (uint32_t)(n_tma * C::kSlotBytes));
                 if (has_box && my_slot < n_tma) {
                     int page = my_page;
                     if (page < 0 || page >= p.num_pages) { dev_check(p, 400); page = 0; }
                     const int pg = u.layer * p.layer_pages + page;
                     if (vrole)
-                        ptx::tma_load_5d(dst + my_slot * C::kVSlotBytes, &tm_v, &full[st], 0, 0, 0, u.g, pg);
+                        ptx::tma_load_5d(dst + my_slot * C::kSlotBytes, &tm_v, &full[st], 0, 0, 0, u.g, pg);
                     else
-                        ptx::tma_load_5d(dst + my_half * kKRingHalfBytes + my_slot * C::kSlotBoxBytes, &tm_k, &full[st], 0, 0, my_half, u.g, pg);
+                        ptx::tma_load_5d(dst + my_slot * C::kSlotBytes, &tm_k, &full[st], 0, 0, 0, u.g, pg);
                 }
                 my_page = next_page;
                 T_MARK(p_issue);
@@ -361,8 +366,9 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     } else if (warp == 1) {
         // =========================================================================== Q K^T issuer
         if (lane == 0) {
-            // descriptor words: the high words and the Q base are constants; per tile only low words move
-            const uint32_t hi = ptx::umma_desc_hi_sw128(1024);
+            // descriptor words: the high words and the Q base are constants; per pair only low words move
+            const uint32_t hi_q = ptx::umma_desc_hi_sw128(1024);
+            const uint32_t hi_k = ptx::umma_desc_hi_sw128(C::kSlotBytes);     // 8-token groups of one tile are a slot apart
             const uint32_t q_lo = ptx::umma_desc_lo(ptx::smem_u32(sQ), 16);
             const uint32_t k_lo = ptx::umma_desc_lo(ptx::smem_u32(sK), 16);
             uint32_t it = 0, seg = 0;
@@ -373,13 +379,10 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 const Segment sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
                 if (ctrl->abort || !T_WAIT(w_q, ptx::mbar_wait(&ctrl->q_full, seg & 1))) { timeout(p, ctrl, 20); ok = false; break; }
                 ++seg;
-                int t = sg.t_first;
-                while (t < sg.t_last) {
-                    // two consecutive tiles whose stages are an aligned pair of the K ring are scored by one N=128 UMMA set
-                    const bool pair = ((it & 1) == 0) && (t + 1 < sg.t_last);
-                    const int nt = pair ? 2 : 1;
+                // parts begin and end on pairs of tiles: a pair is the eight slots of two consecutive ring stages
+                for (int t = sg.t_first; t < sg.t_last; t += 2, x += 2, it += 2) {
                     bool ready = !ctrl->abort;
-                    for (int j = 0; j < nt && ready; ++j) {
+                    for (int j = 0; j < 2 && ready; ++j) {
                         const uint32_t i2 = it + j;
                         ready = T_WAIT(w_k, ptx::mbar_wait(&ctrl->k_full[i2 & (kKVStages - 1)], (i2 / kKVStages) & 1)) &&
                                 T_WAIT(w_s, ptx::mbar_wait(&ctrl->s_free[i2 & (kSBufs - 1)], ((i2 / kSBufs) & 1) ^ 1));
@@ -387,17 +390,23 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     if (!ready) { timeout(p, ctrl, 21); ok = false; break; }
                     ptx::tc_fence_after();
                     const int st = it & (kKVStages - 1), sb = it & (kSBufs - 1);
-                    const int n_tok = min(nt * kTileTok, (sg.slots_all - t * kTileSlots) * kSlotTok);
-                    const uint32_t idesc = ptx::umma_idesc_bf16(kRows, n_tok);
-                    const uint32_t kb = k_lo + (uint32_t)((st * kKVHalfBytes) >> 4);
-                    const uint32_t d = tmem_base + (uint32_t)(sb * kTileTok);
+                    // slots scored: those that exist, rounded up to even (N must be a multiple of 16)
+                    const int ne = min(2 * kStageSlots, (sg.slots_all - t * kStageSlots + 1) & ~1);
+                    const uint32_t idesc = ptx::umma_idesc_bf16(kRows, ne * 8);
+                    const uint32_t kb = k_lo + (uint32_t)((st * C::kStageBytes) >> 4);
 #pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk)
-                        ptx::umma_f16_lohi(d, q_lo + (uint32_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4), hi,
-                                           kb + (uint32_t)(((kk >> 2) * kKRingHalfBytes + (kk & 3) * 32) >> 4), hi, idesc, kk != 0);
-                    for (int j = 0; j < nt; ++j) ptx::umma_commit(&ctrl->k_empty[(it + j) & (kKVStages - 1)]);
-                    for (int j = 0; j < nt; ++j) ptx::umma_commit(&ctrl->s_full[(it + j) & (kSBufs - 1)]);
-                    t += nt; x += nt; it += nt;
+                    for (int h = 0; h < 2; ++h) {
+                        // tile h of the pair: tokens 8h..8h+7 of every slot
+                        const uint32_t d = tmem_base + (uint32_t)((sb + h) * kTileTok);
+#pragma unroll
+                        for (int kk = 0; kk < D / 16; ++kk)
+                            ptx::umma_f16_lohi(d, q_lo + (uint32_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4), hi_q,
+                                               kb + (uint32_t)(((kk >> 2) * (kSlotTok * 128) + h * 1024 + (kk & 3) * 32) >> 4), hi_k,
+                                               idesc, kk != 0);
+                        ptx::umma_commit(&ctrl->s_full[sb + h]);
+                    }
+                    ptx::umma_commit(&ctrl->k_empty[st]);
+                    ptx::umma_commit(&ctrl->k_empty[st + 1]);
                 }
                 if (!ok) break;
             }
@@ -406,7 +415,8 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     } else if (warp == 2) {
         // =========================================================================== P V issuer
         if (lane == 0) {
-            const uint32_t hi = ptx::umma_desc_hi_sw128(1024);
+            const uint32_t hi_p = ptx::umma_desc_hi_sw128(1024);
+            const uint32_t hi_v = ptx::umma_desc_hi_sw128(C::kSlotBytes);                  // the two 8-token groups of a step: two slots
             const uint32_t p_lo = ptx::umma_desc_lo(ptx::smem_u32(sP), 16);
             const uint32_t v_lo = ptx::umma_desc_lo(ptx::smem_u32(sV), kSlotTok * 128);   // MN-major: LBO = next 64-column atom
             const uint32_t idesc_pv = ptx::umma_idesc_bf16(kRows, D) | (1u << 16);          // B operand MN-major
@@ -421,21 +431,25 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 if (seg > 0 && (ctrl->abort || !ptx::mbar_wait(&ctrl->o_free, (seg - 1) & 1))) { timeout(p, ctrl, 24); ok = false; break; }
                 ++seg;
                 for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
-                    const int st = it & (kKVStages - 1), pb = it & 1;
+                    // tile h of a pair reads tokens 8h..8h+7 of the pair's eight slots (both stages)
+                    const uint32_t it0 = it & ~1u;
+                    const int st0 = it0 & (kKVStages - 1), pb = it & 1;
                     if (ctrl->abort || !T_WAIT(w_p, ptx::mbar_wait(&ctrl->p_full[pb], (it >> 1) & 1)) ||
-                        !T_WAIT(w_v, ptx::mbar_wait(&ctrl->v_full[st], (it / kKVStages) & 1))) {
+                        !T_WAIT(w_v, ptx::mbar_wait(&ctrl->v_full[st0], (it0 / kKVStages) & 1)) ||
+                        !T_WAIT(w_v, ptx::mbar_wait(&ctrl->v_full[st0 + 1], (it0 / kKVStages) & 1))) {
                         timeout(p, ctrl, 23); ok = false; break;
                     }
                     ptx::tc_fence_after();
-                    const int n_slots = min(kTileSlots, sg.slots_all - t * kTileSlots);
-                    const uint32_t vb = v_lo + (uint32_t)((st * C::kStageBytes) >> 4);
+                    const int ne = min(2 * kStageSlots, (sg.slots_all - (t & ~1) * kStageSlots + 1) & ~1);
+                    const uint32_t vb = v_lo + (uint32_t)((st0 * C::kStageBytes + pb * 1024) >> 4);
                     const uint32_t pa = p_lo + (uint32_t)((pb * C::kPBytes) >> 4);
 #pragma unroll
-                    for (int k = 0; k < kTileSlots; ++k)
-                        if (k < n_slots)
-                            ptx::umma_f16_lohi(tmem_base + kTmemO + (uint32_t)(pb * D), pa + (uint32_t)(k * 2), hi,
-                                               vb + (uint32_t)(k * (C::kVSlotBytes / 16)), hi, idesc_pv, (t >= sg.t_first + 2) || (k != 0));
-                    ptx::umma_commit(&ctrl->v_empty[st]);
+                    for (int k = 0; k < kStageSlots; ++k)
+                        if (2 * k < ne)
+                            ptx::umma_f16_lohi(tmem_base + kTmemO + (uint32_t)(pb * D), pa + (uint32_t)(k * 2), hi_p,
+                                               vb + (uint32_t)(k * (2 * C::kSlotBytes / 16)), hi_v, idesc_pv, (t >= sg.t_first + 2) || (k != 0));
+                    ptx::umma_commit(&ctrl->v_empty[st0]);
+                    ptx::umma_commit(&ctrl->v_empty[st0 + 1]);
                     ptx::umma_commit(&ctrl->pv_done[pb]);
                 }
             }
@@ -495,21 +509,24 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             ptx::tmem_ld_wait();
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-            const int sl0 = t * kTileSlots + c4 * 2;
-            if (sl0 + 2 > sg.pages_full) {             // a ragged page, tree tokens or missing slots
+            // column c of tile h of a pair is token 8h + c%8 of the pair's slot c/8
+            const int sl0 = (t & ~1) * kStageSlots + c4 * 4;
+            const int tr0 = (t & 1) * 8;
+            if (sl0 + 4 > sg.pages_full) {             // a ragged page, tree tokens or missing slots
 #pragma unroll
-                for (int jj = 0; jj < 2; ++jj) {
+                for (int jj = 0; jj < 4; ++jj) {
                     const int sl = sl0 + jj;
                     if (sl < sg.pages_full) continue;
 #pragma unroll
-                    for (int tr = 0; tr < kSlotTok; ++tr) {
+                    for (int tr = 0; tr < 8; ++tr) {
+                        const int tok = tr0 + tr;
                         bool vis;
-                        if (sl < sg.pages_all) vis = (sl * kSlotTok + tr) < sg.len;
+                        if (sl < sg.pages_all) vis = (sl * kSlotTok + tok) < sg.len;
                         else if (sl < sg.slots_all) {
-                            const int jt = (sl - sg.pages_all) * kSlotTok + tr;
+                            const int jt = (sl - sg.pages_all) * kSlotTok + tok;
                             vis = jt < p.n && (((jt < 64) ? (anc0 >> jt) : (anc1 >> (jt - 64))) & 1ull);
                         } else vis = false;
-                        if (!vis) v[jj * kSlotTok + tr] = -INFINITY;
+                        if (!vis) v[jj * 8 + tr] = -INFINITY;
                     }
                 }
             }
@@ -658,12 +675,11 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 __nv_bfloat16* orow = p.out + ((((size_t)u.layer * p.B + u.b) * p.n + node) * (size_t)p.Hq + u.g * p.G + hl) * D + grp * kDH;
                 float* lse_ptr = (p.lse_out && grp == 0) ? p.lse_out + (((size_t)u.layer * p.B + u.b) * p.Hq + u.g * p.G + hl) * p.n + node : nullptr;
                 // groups ga..gb cover this unit (group g owns tiles [total*g/n_groups, total*(g+1)/n_groups))
-                const long long per = total_tiles;
                 int ga = group, gb = group;
                 if (!whole_unit) {
-                    while (ga > 0 && per * ga / n_groups > u.unit_first_tile) --ga;
+                    while (ga > 0 && group_begin(ga) > u.unit_first_tile) --ga;
                     const long long unit_last = u.unit_first_tile + u.tiles_in_unit - 1;
-                    while (gb + 1 < n_groups && per * (gb + 1) / n_groups <= unit_last) ++gb;
+                    while (gb + 1 < n_groups && group_begin(gb + 1) <= unit_last) ++gb;
                 }
                 const int slot = (sg.t_first > 0) ? 0 : 1;       // a unit that began before this CTA's range uses slot 0
                 // partial layout [column][row]: a warp's store of one column is one contiguous 128-byte line;
@@ -727,13 +743,13 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                         // merge in group order
                         float Mm = -INFINITY;
                         for (int gsrc = ga; gsrc <= gb; ++gsrc) {
-                            const int sslot = (per * gsrc / n_groups > u.unit_first_tile) ? 0 : 1;
+                            const int sslot = (group_begin(gsrc) > u.unit_first_tile) ? 0 : 1;
                             const float* src = p.partial + ((size_t)(gsrc * p.n_rb + rb) * 2 + sslot) * kRowW * kRows + row_in_blk;
                             Mm = fmaxf(Mm, __ldcg(src + (size_t)(D + 2 * grp) * kRows));
                         }
                         float Lm = 0.f;
                         for (int gsrc = ga; gsrc <= gb; ++gsrc) {
-                            const int sslot = (per * gsrc / n_groups > u.unit_first_tile) ? 0 : 1;
+                            const int sslot = (group_begin(gsrc) > u.unit_first_tile) ? 0 : 1;
                             const float* src = p.partial + ((size_t)(gsrc * p.n_rb + rb) * 2 + sslot) * kRowW * kRows + row_in_blk;
                             const float pm = __ldcg(src + (size_t)(D + 2 * grp) * kRows);
                             Lm += ((pm == -INFINITY) ? 0.f : exp2f((pm - Mm) * p.scale_log2e)) * __ldcg(src + (size_t)(D + 2 * grp + 1) * kRows);
@@ -745,7 +761,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 #pragma unroll
                             for (int j = 0; j < 32; ++j) acc[j] = 0.f;
                             for (int gsrc = ga; gsrc <= gb; ++gsrc) {
-                                const int sslot = (per * gsrc / n_groups > u.unit_first_tile) ? 0 : 1;
+                                const int sslot = (group_begin(gsrc) > u.unit_first_tile) ? 0 : 1;
                                 const float* src = p.partial + ((size_t)(gsrc * p.n_rb + rb) * 2 + sslot) * kRowW * kRows + row_in_blk;
                                 const float pm = __ldcg(src + (size_t)(D + 2 * grp) * kRows);
                                 const float wgt = (pm == -INFINITY) ? 0.f : exp2f((pm - Mm) * p.scale_log2e);
@@ -829,17 +845,15 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
 
     CUtensorMap tm_k, tm_v;
     {
-        // pool viewed as (64 columns, 16 tokens, D/64 halves, Hkv heads, layers*pages); one box = one half of one page
+        // pool viewed as (64 columns, 16 tokens, D/64 halves, Hkv heads, layers*pages)
         const uint64_t total_pages = (uint64_t)(p.L - 1) * p.layer_pages + p.num_pages;
         const uint64_t dims[5] = {64, (uint64_t)kSlotTok, (uint64_t)(D / 64), (uint64_t)Hkv, total_pages};
         const uint64_t strides[4] = {(uint64_t)D * 2, 128, (uint64_t)kSlotTok * D * 2, (uint64_t)page_elems * 2};
-        // K: one box per 64-column half (the K-major operand wants all tokens of a half contiguous);
-        // V: one box per page (both halves), which is already the MN-major operand layout of one 16-token step
-        const uint32_t box_k[5] = {64, (uint32_t)kSlotTok, 1, 1, 1};
-        const uint32_t box_v[5] = {64, (uint32_t)kSlotTok, (uint32_t)(D / 64), 1, 1};
-        mirror_status st = mirror_make_tmap(ctx, &tm_k, kv->k_pool, 5, dims, strides, box_k);
+        // one box per page and tensor (all halves): [half][16 tokens][128 B] in shared memory
+        const uint32_t box[5] = {64, (uint32_t)kSlotTok, (uint32_t)(D / 64), 1, 1};
+        mirror_status st = mirror_make_tmap(ctx, &tm_k, kv->k_pool, 5, dims, strides, box);
         if (st != MIRROR_OK) return st;
-        st = mirror_make_tmap(ctx, &tm_v, kv->v_pool, 5, dims, strides, box_v);
+        st = mirror_make_tmap(ctx, &tm_v, kv->v_pool, 5, dims, strides, box);
         if (st != MIRROR_OK) return st;
     }
     const int grid = p.n_groups * p.n_rb;
