@@ -58,6 +58,7 @@ struct AttnParams {
     int L, B, n, Hq, Hkv, G;
     int rows, n_rb, rows_per_rb;          // rows per unit, row blocks, rows per block
     int n_groups;                         // CTA groups (grid = n_groups * n_rb)
+    int snap_cap;                         // boundaries move to a unit boundary that is at most this many tiles away
     int max_pages, num_pages, layer_pages;
     int tree_slots;
     float scale_log2e, scale;
@@ -208,6 +209,12 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int group = blockIdx.x / p.n_rb, rb = blockIdx.x % p.n_rb;
+#ifdef MIRROR_ATTN_TIMING
+#define T_STAMP(i) do { if (p.timing && tid == 0) { unsigned long long g__; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g__)); p.timing[64 + blockIdx.x * 4 + (i)] = (long long)g__; } } while (0)
+#else
+#define T_STAMP(i) do { } while (0)
+#endif
+    T_STAMP(0);
 
     // ---- prologue ---------------------------------------------------------------------------------
     for (int b = tid; b < p.B; b += kThreads) {
@@ -254,10 +261,25 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     // and boundaries are distinct
     const long long total_pairs = total_tiles / 2;
     const int n_groups = (int)min((long long)p.n_groups, total_pairs);
-    auto group_begin = [&](int g) -> long long { return 2 * (total_pairs * g / n_groups); };
+    // A boundary that falls within snap_tol tiles (a cut costs about as much as a dozen tiles) of a unit boundary moves there: both neighbours then hold whole
+    // units and no partial has to be left and merged.  snap_tol is less than a quarter of the smallest even share,
+    // so boundaries stay strictly increasing and every group's range is non-empty.
+    const long long snap_tol = min((long long)p.snap_cap, (2 * (total_pairs / n_groups)) / 4);
+    auto group_begin = [&](int g) -> long long {
+        if (g <= 0) return 0;
+        if (g >= n_groups) return total_tiles;
+        const long long e = 2 * (total_pairs * g / n_groups);
+        if (snap_tol == 0) return e;
+        const UnitPos u = locate(e, p, cumT, tiles_per_layer);
+        const long long lo = u.unit_first_tile, hi = lo + u.tiles_in_unit;
+        const long long best = (e - lo <= hi - e) ? lo : hi;
+        const long long dist = best > e ? best - e : e - best;
+        return dist <= snap_tol ? best : e;
+    };
     const long long x_begin = group < n_groups ? group_begin(group) : 0;
     const long long x_end = group < n_groups ? group_begin(group + 1) : 0;
 
+    T_STAMP(1);
     if (warp == 0 || warp == kVProducerWarp) {
         // =========================================================================== producers
         // warp 0 stages K, the last warp stages V: a warp issues its TMA boxes one after the other, so two
@@ -375,6 +397,9 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             bool ok = true;
             long long x = x_begin;
             T_DECL(w_q = 0, w_k = 0, w_s = 0, t0 = T_NOW());
+#ifdef MIRROR_ATTN_TIMING
+            unsigned long long g0; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g0));
+#endif
             while (x < x_end && ok) {
                 const Segment sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
                 if (ctrl->abort || !T_WAIT(w_q, ptx::mbar_wait(&ctrl->q_full, seg & 1))) { timeout(p, ctrl, 20); ok = false; break; }
@@ -411,6 +436,9 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 if (!ok) break;
             }
             T_STORE(0, T_NOW() - t0, w_q, w_k, w_s, (long long)it);
+#ifdef MIRROR_ATTN_TIMING
+            { unsigned long long g1; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g1)); T_STORE(48, (long long)(g1 - g0)); }
+#endif
         }
     } else if (warp == 2) {
         // =========================================================================== P V issuer
@@ -500,7 +528,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         uint32_t it = 0;
         bool ok = true;
         long long x = x_begin;
-        T_DECL(w_sf = 0, w_pv = 0, w_end = 0, t_epi = 0, t_q = 0, t0 = T_NOW(), te = 0, tm__ = 0, s_ld = 0, s_free = 0, s_max = 0, s_xch = 0, s_exp = 0, s_fin = 0);
+        T_DECL(w_sf = 0, w_pv = 0, w_end = 0, t_epi = 0, t_q = 0, t0 = T_NOW(), te = 0, tm__ = 0, s_ld = 0, s_free = 0, s_max = 0, s_xch = 0, s_exp = 0, s_fin = 0, t_init = 0, t_loop = 0, tl = 0);
         Segment sg;
         // one 32-column chunk of this row's scores: tcgen05.ld, then the visibility mask where the tile needs one
         auto load_scores = [&](int sb, int c4, int t, float (&v)[32]) {
@@ -562,12 +590,33 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
             stage_q(sg.u);
         }
+#ifdef MIRROR_ATTN_TIMING
+        t_init = T_NOW() - t0;
+#endif
         while (x < x_end && ok) {
             const UnitPos u = sg.u;
             const bool whole_unit = (sg.t_first == 0 && sg.t_last == u.tiles_in_unit);
             float m_used = -INFINITY, l_run = 0.f;                 // this group's offset and running sum
             bool first = true;                                     // no tile of this unit's part seen by this group yet
+            // the part after this one: its Q row is pulled into L2 now and staged when this part's scores are complete
+            Segment sg_next;
+            const long long x_next = x + (sg.t_last - sg.t_first);
+            const bool has_next = x_next < x_end;
+#ifdef MIRROR_ATTN_TIMING
+            te = T_NOW();
+#endif
+            if (has_next) {
+                sg_next = make_segment(x_next, x_end, p, cumT, s_len, tiles_per_layer);
+                if (row_ok)
+                    ptx::prefetch_l2(p.q + ((((size_t)sg_next.u.layer * p.B + sg_next.u.b) * p.n + node) * (size_t)p.Hq + sg_next.u.g * p.G + hl) * D + grp * (D / 2));
+            }
+#ifdef MIRROR_ATTN_TIMING
+            s_xch += T_NOW() - te;
+#endif
 
+#ifdef MIRROR_ATTN_TIMING
+            tl = T_NOW();
+#endif
             for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
                 if ((int)(it & 1) != grp) continue;
                 const int sb = it & (kSBufs - 1), pb = grp;
@@ -632,18 +681,18 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 T_MARK(s_fin);
             }
             if (!ok) break;
+#ifdef MIRROR_ATTN_TIMING
+            t_loop += T_NOW() - tl;
+#endif
 
             // ---- the next unit's Q can be staged now (every Q K^T of this one has completed), so that its first
             //      tiles are scored while this unit's epilogue runs
             // (a group that did not take the part's last tile has not yet seen that tile's scores complete)
-            if (ctrl->abort || !ptx::mbar_wait(&ctrl->s_full[(it - 1) & (kSBufs - 1)], ((it - 1) / kSBufs) & 1)) { timeout(p, ctrl, 37); ok = false; break; }
-            Segment sg_next;
-            const bool has_next = x < x_end;
+            if (ctrl->abort || !T_WAIT(s_max, ptx::mbar_wait(&ctrl->s_full[(it - 1) & (kSBufs - 1)], ((it - 1) / kSBufs) & 1))) { timeout(p, ctrl, 37); ok = false; break; }
             if (has_next) {
 #ifdef MIRROR_ATTN_TIMING
                 te = T_NOW();
 #endif
-                sg_next = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
                 stage_q(sg_next.u);
 #ifdef MIRROR_ATTN_TIMING
                 t_q += T_NOW() - te;
@@ -655,7 +704,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             float* xc = xch + (size_t)row_in_blk * 4;              // [row][group][max, sum]
             xc[grp * 2] = m_used;
             xc[grp * 2 + 1] = l_run;
-            if (!pair_sync()) { timeout(p, ctrl, 35); ok = false; break; }
+            if (!T_WAIT(s_ld, pair_sync())) { timeout(p, ctrl, 35); ok = false; break; }
             const float m_a = xc[0], l_a = xc[1], m_b = xc[2], l_b = xc[3];
             if (ctrl->abort || !T_WAIT(w_end, ptx::mbar_wait(&ctrl->pv_done[(it - 1) & 1], ((it - 1) >> 1) & 1))) { timeout(p, ctrl, 32); ok = false; break; }
             ptx::tc_fence_after();
@@ -722,7 +771,10 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                         for (int j = 0; j < 32; ++j) my[(size_t)(grp * kDH + c4 * 32 + j) * kRows] = acc[j];
                     }
                 }
+                // both accumulators have been read by this warp: the next unit's P V may overwrite them once all have
                 ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&ctrl->o_free);
                 if (whole_unit) {
                     if (lse_ptr && row_ok) *lse_ptr = M * p.scale + logf(Lsum);
                 } else {
@@ -785,22 +837,22 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 }
             } else {
                 ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&ctrl->o_free);
             }
-            // both accumulators have been read by this warp: the next unit's P V may overwrite them once all have
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&ctrl->o_free);
 #ifdef MIRROR_ATTN_TIMING
             t_epi += T_NOW() - te;
 #endif
             // the exchange words are rewritten at the end of the next part: the partner must have read them
-            if (!pair_sync()) { timeout(p, ctrl, 36); ok = false; break; }
+            if (!T_WAIT(s_free, pair_sync())) { timeout(p, ctrl, 36); ok = false; break; }
             if (has_next) sg = sg_next;
         }
-        if (warp == 4 && lane == 0) { T_STORE(8, T_NOW() - t0, w_sf, w_pv, w_end, t_epi, t_q, (long long)it); T_STORE(40, s_ld, s_free, s_max, s_xch, s_exp, s_fin); }
+        if (warp == 4 && lane == 0) { T_STORE(8, T_NOW() - t0, w_sf, w_pv, w_end, t_epi, t_q, (long long)it); T_STORE(40, s_ld, s_free, s_max, s_xch, s_exp, s_fin); T_STORE(52, t_init, t_loop); }
     }
 
     ptx::tc_fence_before();
     __syncthreads();
+    T_STAMP(2);
     if (warp == 1) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem_base, kTmemCols);
@@ -820,6 +872,8 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
     p.rows_per_rb = (p.rows + p.n_rb - 1) / p.n_rb;
     p.n_groups = ctx->num_sms / p.n_rb;
     if (p.n_groups < 1) return MIRROR_ERR_SHAPE;
+    p.snap_cap = 12;
+    if (const char* e = getenv("MIRROR_ATTN_SNAP")) { p.snap_cap = atoi(e); if (p.snap_cap < 0) p.snap_cap = 0; }
     p.max_pages = kv->max_pages_per_req; p.num_pages = kv->num_pages;
     const int64_t page_elems = (int64_t)Hkv * kSlotTok * D;
     if (kv->layer_stride % page_elems != 0) return MIRROR_ERR_UNSUPPORTED;
