@@ -47,7 +47,7 @@ constexpr int kKVStages = 4;                        // power of two: stage = til
 constexpr int kSBufs = 4;                           // S buffers in TMEM (power of two)
 constexpr int kMergeWarps = 8;
 constexpr float kRescaleLog2 = 8.0f;
-constexpr int kTmemCols = 512;                      // S0..S3 (64 columns each) | O of group 0 | O of group 1 (D columns each)
+constexpr int kTmemCols = 512;                      // S0..S3 (64 columns each; P overwrites the first 32 of its S) | O of group 0 | O of group 1
 constexpr int kTmemO = kSBufs * kTileTok;
 
 struct AttnTree {
@@ -87,8 +87,8 @@ struct Ctrl {
     uint64_t k_full[kKVStages], k_empty[kKVStages];     // K ring: refilled as soon as Q K^T has read a stage
     uint64_t v_full[kKVStages], v_empty[kKVStages];     // V ring: refilled once P V has read a stage
     uint64_t s_full[kSBufs], s_free[kSBufs];
-    uint64_t p_full[2], pv_done[2];
-    uint64_t q_full;
+    uint64_t p_full[kSBufs], pv_done[2];
+    uint64_t q_full[2];
     uint64_t pair[4];                                   // softmax warp pairs' exchange
     uint64_t o_free;                                    // accumulators read out at the end of a unit's part
     uint32_t tmem_base;
@@ -143,6 +143,13 @@ __device__ __forceinline__ void tmem_st_32x32b_x32(uint32_t taddr, const uint32_
           "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
         : "memory");
 }
+__device__ __forceinline__ void tmem_st_32x32b_x16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // Developer timing aid: with -DMIRROR_ATTN_TIMING each role of CTA 5 accumulates the cycles it spends in its waits
@@ -167,8 +174,7 @@ struct Cfg {
     static constexpr int kQBytes = kHalves * kHalfBytes;           // Q: 128 rows x D
     static constexpr int kSlotBytes = kHalves * kSlotTok * 128;    // one slot of K or V: [half][16 tokens][128 B] = one TMA box
     static constexpr int kStageBytes = kStageSlots * kSlotBytes;   // one K (or V) stage: 4 slots; stages are contiguous
-    static constexpr int kPBytes = kRows * 128;                    // one P buffer: 128 rows x 64 tokens
-    static constexpr size_t kSmemData = (size_t)kQBytes + 2 * kPBytes + 2 * (size_t)kKVStages * kStageBytes;
+    static constexpr size_t kSmemData = 2 * (size_t)kQBytes + 2 * (size_t)kKVStages * kStageBytes;
     static constexpr size_t kSmemBytes = kSmemData + 512 /*ctrl*/ + 2 * 2 * kRows * 4 /*pair exchange*/ + (2 * kMaxBatch + 2) * 4 + 1024 /*align*/;
 };
 
@@ -198,9 +204,8 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     using C = Cfg<D>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint8_t* sQ = smem;
-    uint8_t* sP = sQ + C::kQBytes;                                  // [2]
-    uint8_t* sK = sP + 2 * C::kPBytes;                              // [kKVStages]  [slot][half][16 tokens][128 B]
+    uint8_t* sQ = smem;                                             // [2]: the units a CTA walks alternate
+    uint8_t* sK = sQ + 2 * C::kQBytes;                              // [kKVStages]  [slot][half][16 tokens][128 B]
     uint8_t* sV = sK + kKVStages * C::kStageBytes;                  // [kKVStages]  [slot][half][16 tokens][128 B]
     Ctrl* ctrl = (Ctrl*)(sV + kKVStages * C::kStageBytes);
     float* xch = (float*)((uint8_t*)ctrl + 512);                    // [2 tiles][2 halves][128 rows] pair exchange
@@ -227,9 +232,11 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             ptx::mbar_init(&ctrl->k_full[s], 1); ptx::mbar_init(&ctrl->k_empty[s], 1);
             ptx::mbar_init(&ctrl->v_full[s], 1); ptx::mbar_init(&ctrl->v_empty[s], 2);   // both tiles of a pair read a V stage
         }
-        for (int s = 0; s < kSBufs; ++s) { ptx::mbar_init(&ctrl->s_full[s], 1); ptx::mbar_init(&ctrl->s_free[s], kSoftmaxWarps / 2); }
-        for (int s = 0; s < 2; ++s) { ptx::mbar_init(&ctrl->p_full[s], kSoftmaxWarps / 2); ptx::mbar_init(&ctrl->pv_done[s], 1); }
-        ptx::mbar_init(&ctrl->q_full, kSoftmaxWarps);
+        for (int s = 0; s < kSBufs; ++s) {
+            ptx::mbar_init(&ctrl->s_full[s], 1); ptx::mbar_init(&ctrl->s_free[s], 1);     // freed by the P V that read P from it
+            ptx::mbar_init(&ctrl->p_full[s], kSoftmaxWarps / 2);
+        }
+        for (int s = 0; s < 2; ++s) { ptx::mbar_init(&ctrl->pv_done[s], 1); ptx::mbar_init(&ctrl->q_full[s], kSoftmaxWarps); }
         for (int s = 0; s < 4; ++s) ptx::mbar_init(&ctrl->pair[s], 2);
         ptx::mbar_init(&ctrl->o_free, kSoftmaxWarps);
         ctrl->abort = 0;
@@ -402,7 +409,8 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 #endif
             while (x < x_end && ok) {
                 const Segment sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
-                if (ctrl->abort || !T_WAIT(w_q, ptx::mbar_wait(&ctrl->q_full, seg & 1))) { timeout(p, ctrl, 20); ok = false; break; }
+                if (ctrl->abort || !T_WAIT(w_q, ptx::mbar_wait(&ctrl->q_full[seg & 1], (seg >> 1) & 1))) { timeout(p, ctrl, 20); ok = false; break; }
+                const uint32_t q_seg = q_lo + (uint32_t)(((seg & 1) * C::kQBytes) >> 4);
                 ++seg;
                 // parts begin and end on pairs of tiles: a pair is the eight slots of two consecutive ring stages
                 for (int t = sg.t_first; t < sg.t_last; t += 2, x += 2, it += 2) {
@@ -425,7 +433,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                         const uint32_t d = tmem_base + (uint32_t)((sb + h) * kTileTok);
 #pragma unroll
                         for (int kk = 0; kk < D / 16; ++kk)
-                            ptx::umma_f16_lohi(d, q_lo + (uint32_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4), hi_q,
+                            ptx::umma_f16_lohi(d, q_seg + (uint32_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4), hi_q,
                                                kb + (uint32_t)(((kk >> 2) * (kSlotTok * 128) + h * 1024 + (kk & 3) * 32) >> 4), hi_k,
                                                idesc, kk != 0);
                         ptx::umma_commit(&ctrl->s_full[sb + h]);
@@ -443,9 +451,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     } else if (warp == 2) {
         // =========================================================================== P V issuer
         if (lane == 0) {
-            const uint32_t hi_p = ptx::umma_desc_hi_sw128(1024);
             const uint32_t hi_v = ptx::umma_desc_hi_sw128(C::kSlotBytes);                  // the two 8-token groups of a step: two slots
-            const uint32_t p_lo = ptx::umma_desc_lo(ptx::smem_u32(sP), 16);
             const uint32_t v_lo = ptx::umma_desc_lo(ptx::smem_u32(sV), kSlotTok * 128);   // MN-major: LBO = next 64-column atom
             const uint32_t idesc_pv = ptx::umma_idesc_bf16(kRows, D) | (1u << 16);          // B operand MN-major
             uint32_t it = 0;
@@ -461,8 +467,8 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
                     // tile h of a pair reads tokens 8h..8h+7 of the pair's eight slots (both stages)
                     const uint32_t it0 = it & ~1u;
-                    const int st0 = it0 & (kKVStages - 1), pb = it & 1;
-                    if (ctrl->abort || !T_WAIT(w_p, ptx::mbar_wait(&ctrl->p_full[pb], (it >> 1) & 1)) ||
+                    const int st0 = it0 & (kKVStages - 1), pb = it & 1, sb = it & (kSBufs - 1);
+                    if (ctrl->abort || !T_WAIT(w_p, ptx::mbar_wait(&ctrl->p_full[sb], (it / kSBufs) & 1)) ||
                         !T_WAIT(w_v, ptx::mbar_wait(&ctrl->v_full[st0], (it0 / kKVStages) & 1)) ||
                         !T_WAIT(w_v, ptx::mbar_wait(&ctrl->v_full[st0 + 1], (it0 / kKVStages) & 1))) {
                         timeout(p, ctrl, 23); ok = false; break;
@@ -470,14 +476,15 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     ptx::tc_fence_after();
                     const int ne = min(2 * kStageSlots, (sg.slots_all - (t & ~1) * kStageSlots + 1) & ~1);
                     const uint32_t vb = v_lo + (uint32_t)((st0 * C::kStageBytes + pb * 1024) >> 4);
-                    const uint32_t pa = p_lo + (uint32_t)((pb * C::kPBytes) >> 4);
+                    const uint32_t pa = tmem_base + (uint32_t)(sb * kTileTok);       // P: 8 columns per 16-token step
 #pragma unroll
                     for (int k = 0; k < kStageSlots; ++k)
                         if (2 * k < ne)
-                            ptx::umma_f16_lohi(tmem_base + kTmemO + (uint32_t)(pb * D), pa + (uint32_t)(k * 2), hi_p,
-                                               vb + (uint32_t)(k * (2 * C::kSlotBytes / 16)), hi_v, idesc_pv, (t >= sg.t_first + 2) || (k != 0));
+                            ptx::umma_f16_tmem_a(tmem_base + kTmemO + (uint32_t)(pb * D), pa + (uint32_t)(k * 8),
+                                                 vb + (uint32_t)(k * (2 * C::kSlotBytes / 16)), hi_v, idesc_pv, (t >= sg.t_first + 2) || (k != 0));
                     ptx::umma_commit(&ctrl->v_empty[st0]);
                     ptx::umma_commit(&ctrl->v_empty[st0 + 1]);
+                    ptx::umma_commit(&ctrl->s_free[sb]);
                     ptx::umma_commit(&ctrl->pv_done[pb]);
                 }
             }
@@ -512,23 +519,30 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             return r;
         };
 
-        // this thread's half of its Q row into the swizzled A-operand tile (rows that do not exist are zero)
-        auto stage_q = [&](const UnitPos& u) {
+        // this thread's half of its Q row goes into the swizzled A-operand tile `buf` by asynchronous 16-byte copies
+        // (rows that do not exist are zero-filled); q_ready() later makes them visible to the tensor core
+        auto stage_q = [&](const UnitPos& u, int buf) {
             const __nv_bfloat16* qrow = p.q + ((((size_t)u.layer * p.B + u.b) * p.n + node) * (size_t)p.Hq + u.g * p.G + hl) * D;
-            uint4 qv[D / 16];
+            uint8_t* q = sQ + buf * C::kQBytes;
+            const uint32_t src_bytes = row_ok ? 16u : 0u;
 #pragma unroll
-            for (int i = 0; i < D / 16; ++i) qv[i] = row_ok ? *reinterpret_cast<const uint4*>(qrow + (grp * (D / 16) + i) * 8) : make_uint4(0, 0, 0, 0);
-#pragma unroll
-            for (int i = 0; i < D / 16; ++i) *reinterpret_cast<uint4*>(sQ + tile_off(row_in_blk, grp * (D / 16) + i, kHalfBytes)) = qv[i];
+            for (int i = 0; i < D / 16; ++i) {
+                const int chunk = grp * (D / 16) + i;
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
+                             ::"r"(ptx::smem_u32(q + tile_off(row_in_blk, chunk, kHalfBytes))), "l"(qrow + chunk * 8), "r"(src_bytes) : "memory");
+            }
+        };
+        auto q_ready = [&](int buf) {
+            asm volatile("cp.async.wait_all;" ::: "memory");
             ptx::fence_proxy_async();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&ctrl->q_full);
+            if (lane == 0) ptx::mbar_arrive(&ctrl->q_full[buf]);
         };
 
         uint32_t it = 0;
         bool ok = true;
         long long x = x_begin;
-        T_DECL(w_sf = 0, w_pv = 0, w_end = 0, t_epi = 0, t_q = 0, t0 = T_NOW(), te = 0, tm__ = 0, s_ld = 0, s_free = 0, s_max = 0, s_xch = 0, s_exp = 0, s_fin = 0, t_init = 0, t_loop = 0, tl = 0);
+        T_DECL(w_sf = 0, w_pv = 0, w_end = 0, t_epi = 0, t_q = 0, t0 = T_NOW(), te = 0, tm__ = 0, s_ld = 0, s_free = 0, s_max = 0, s_xch = 0, s_exp = 0, s_fin = 0, t_init = 0, t_loop = 0, tl = 0, t_max = 0, t_ld1 = 0);
         Segment sg;
         // one 32-column chunk of this row's scores: tcgen05.ld, then the visibility mask where the tile needs one
         auto load_scores = [&](int sb, int c4, int t, float (&v)[32]) {
@@ -545,50 +559,63 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 for (int jj = 0; jj < 4; ++jj) {
                     const int sl = sl0 + jj;
                     if (sl < sg.pages_full) continue;
-#pragma unroll
-                    for (int tr = 0; tr < 8; ++tr) {
-                        const int tok = tr0 + tr;
-                        bool vis;
-                        if (sl < sg.pages_all) vis = (sl * kSlotTok + tok) < sg.len;
-                        else if (sl < sg.slots_all) {
-                            const int jt = (sl - sg.pages_all) * kSlotTok + tok;
-                            vis = jt < p.n && (((jt < 64) ? (anc0 >> jt) : (anc1 >> (jt - 64))) & 1ull);
-                        } else vis = false;
-                        if (!vis) v[jj * 8 + tr] = -INFINITY;
+                    // visibility of the slot's 16 tokens as a bit mask
+                    uint32_t bits = 0;
+                    if (sl < sg.pages_all) {
+                        bits = (1u << (sg.len - sl * kSlotTok)) - 1u;                       // ragged page: 1..15 valid tokens
+                    } else if (sl < sg.slots_all) {
+                        const int ts = sl - sg.pages_all;                                   // tree tokens 16*ts .. 16*ts+15
+                        bits = (uint32_t)(((ts < 4) ? anc0 : anc1) >> ((ts & 3) * 16)) & 0xffffu;   // ancestors-or-self (all < n)
                     }
+                    bits >>= tr0;
+#pragma unroll
+                    for (int tr = 0; tr < 8; ++tr)
+                        if (!((bits >> tr) & 1u)) v[jj * 8 + tr] = -INFINITY;
                 }
             }
         };
-        // P = exp2(s*c - offset) for the whole tile into the group's P buffer; returns the row sum and watches the maximum
-        auto softmax_tile = [&](int sb, int t, uint8_t* prow, float m_off, float& mx_out) -> float {
-            const float off = (m_off == -INFINITY) ? 0.f : m_off * p.scale_log2e;
-            float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+        // pass 1: the row maximum of a tile
+        auto tile_max = [&](int sb, int t) -> float {
             float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
             for (int c4 = 0; c4 < kTileTok / 32; ++c4) {
                 float v[32];
                 load_scores(sb, c4, t, v);
+                if (c4 == 0) T_MARK(t_ld1);
 #pragma unroll
-                for (int c8 = 0; c8 < 4; ++c8) {
-                    float e[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        m4[j & 3] = fmaxf(m4[j & 3], v[c8 * 8 + j]);
-                        e[j] = ptx::ex2_approx(fmaf(v[c8 * 8 + j], p.scale_log2e, -off));
-                        sum4[j & 3] += e[j];
-                    }
-                    uint4 pk;
-                    pk.x = pack_bf16(e[0], e[1]); pk.y = pack_bf16(e[2], e[3]); pk.z = pack_bf16(e[4], e[5]); pk.w = pack_bf16(e[6], e[7]);
-                    *reinterpret_cast<uint4*>(prow + tile_off(row_in_blk, c4 * 4 + c8, kHalfBytes)) = pk;
-                }
+                for (int j = 0; j < 32; ++j) m4[j & 3] = fmaxf(m4[j & 3], v[j]);
             }
-            mx_out = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+            return fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+        };
+        // pass 2: P = exp2(s*c - offset) as bf16 pairs over the first 32 columns of the same S buffer (a thread
+        // only ever touches its own lane, and a 32-column chunk of S is in registers before its P is written
+        // over columns that were read earlier); returns the row sum
+        auto tile_p = [&](int sb, int t, float m_off) -> float {
+            const float off = (m_off == -INFINITY) ? 0.f : m_off * p.scale_log2e;
+            float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int c4 = 0; c4 < kTileTok / 32; ++c4) {
+                float v[32];
+                load_scores(sb, c4, t, v);
+                uint32_t pk[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const float e0 = ptx::ex2_approx(fmaf(v[2 * j], p.scale_log2e, -off));
+                    const float e1 = ptx::ex2_approx(fmaf(v[2 * j + 1], p.scale_log2e, -off));
+                    sum4[j & 3] += e0 + e1;
+                    pk[j] = pack_bf16(e0, e1);
+                }
+                tmem_st_32x32b_x16(lane_base + (uint32_t)(sb * kTileTok + c4 * 16), pk);
+            }
+            tmem_st_wait();
             return (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
         };
 
+        uint32_t seg = 0;                                          // parts walked so far: Q buffer = seg & 1
         if (x < x_end) {
             sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
-            stage_q(sg.u);
+            stage_q(sg.u, 0);
+            q_ready(0);
         }
 #ifdef MIRROR_ATTN_TIMING
         t_init = T_NOW() - t0;
@@ -598,7 +625,8 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             const bool whole_unit = (sg.t_first == 0 && sg.t_last == u.tiles_in_unit);
             float m_used = -INFINITY, l_run = 0.f;                 // this group's offset and running sum
             bool first = true;                                     // no tile of this unit's part seen by this group yet
-            // the part after this one: its Q row is pulled into L2 now and staged when this part's scores are complete
+            // the part after this one: its Q goes into the other Q buffer now (every Q K^T that read that buffer
+            // belongs to the part before this one and has completed), so the issuer can run on into the next unit
             Segment sg_next;
             const long long x_next = x + (sg.t_last - sg.t_first);
             const bool has_next = x_next < x_end;
@@ -607,9 +635,9 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 #endif
             if (has_next) {
                 sg_next = make_segment(x_next, x_end, p, cumT, s_len, tiles_per_layer);
-                if (row_ok)
-                    ptx::prefetch_l2(p.q + ((((size_t)sg_next.u.layer * p.B + sg_next.u.b) * p.n + node) * (size_t)p.Hq + sg_next.u.g * p.G + hl) * D + grp * (D / 2));
+                stage_q(sg_next.u, (seg + 1) & 1);
             }
+            bool q_pending = has_next;
 #ifdef MIRROR_ATTN_TIMING
             s_xch += T_NOW() - te;
 #endif
@@ -619,41 +647,23 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 #endif
             for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
                 if ((int)(it & 1) != grp) continue;
-                const int sb = it & (kSBufs - 1), pb = grp;
+                const int sb = it & (kSBufs - 1);
                 if (ctrl->abort || !T_WAIT(w_sf, ptx::mbar_wait(&ctrl->s_full[sb], (it / kSBufs) & 1))) { timeout(p, ctrl, 30); ok = false; break; }
                 ptx::tc_fence_after();
 #ifdef MIRROR_ATTN_TIMING
                 tm__ = T_NOW();
 #endif
-                // this group's P buffer and accumulator were last used by the P V of two tiles ago
-                if (it >= 2) {
-                    if (ctrl->abort || !T_WAIT(w_pv, ptx::mbar_wait(&ctrl->pv_done[pb], ((it - 2) >> 1) & 1))) { timeout(p, ctrl, 33); ok = false; break; }
-                    ptx::tc_fence_after();
-                }
-                uint8_t* prow = sP + pb * C::kPBytes;
                 float mx = -INFINITY, sum = 0.f;
-                if (warp_has_rows) {
-                    if (first) {
-                        // no offset yet: one pass for the row maximum
-                        float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-                        for (int c4 = 0; c4 < kTileTok / 32; ++c4) {
-                            float v[32];
-                            load_scores(sb, c4, t, v);
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) m4[j & 3] = fmaxf(m4[j & 3], v[j]);
-                        }
-                        m_used = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
-                    }
-                    sum = softmax_tile(sb, t, prow, m_used, mx);
-                }
-                T_MARK(s_exp);
-                // offset in use: moved only when the row maximum outgrew it by more than 2^8
+                if (warp_has_rows) mx = tile_max(sb, t);
+                T_MARK(t_max);
+                if (first) m_used = mx;
+                // offset in use: set by the group's first tile, moved only when the row maximum outgrew it by more than 2^8
                 const bool move = warp_has_rows && !first &&
                                   (((mx - m_used) * p.scale_log2e > kRescaleLog2) || (m_used == -INFINITY && mx > -INFINITY));
                 if (__any_sync(0xffffffffu, move)) {
-                    // rare: rescale this group's accumulator (its last P V is complete, see the wait above) and the
-                    // running sum, then redo this tile's P with the new offset
+                    // rare: rescale this group's accumulator and running sum once its last P V (two tiles ago) is complete
+                    if (ctrl->abort || !T_WAIT(w_pv, ptx::mbar_wait(&ctrl->pv_done[grp], ((it - 2) >> 1) & 1))) { timeout(p, ctrl, 33); ok = false; break; }
+                    ptx::tc_fence_after();
                     const float m_next = move ? fmaxf(mx, m_used) : m_used;
                     const float alpha = (m_used == -INFINITY) ? ((m_next == -INFINITY) ? 1.f : 0.f)
                                                               : exp2f((m_used - m_next) * p.scale_log2e);
@@ -669,15 +679,16 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     tmem_st_wait();
                     l_run *= alpha;
                     m_used = m_next;
-                    sum = softmax_tile(sb, t, prow, m_used, mx);
                 }
+                if (warp_has_rows) sum = tile_p(sb, t, m_used);
+                T_MARK(s_exp);
                 l_run += sum;
                 first = false;
-                // all reads of this S buffer are done; P is in shared memory (and any O rescale in TMEM)
-                ptx::fence_proxy_async();       // P (plain stores) is read by the tensor core
+                // P is in tensor memory (and any O rescale too): the P V of this tile may go
                 ptx::tc_fence_before();
                 __syncwarp();
-                if (lane == 0) { ptx::mbar_arrive(&ctrl->s_free[sb]); ptx::mbar_arrive(&ctrl->p_full[pb]); }
+                if (lane == 0) ptx::mbar_arrive(&ctrl->p_full[sb]);
+                if (q_pending) { q_ready((seg + 1) & 1); q_pending = false; }
                 T_MARK(s_fin);
             }
             if (!ok) break;
@@ -685,19 +696,11 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             t_loop += T_NOW() - tl;
 #endif
 
-            // ---- the next unit's Q can be staged now (every Q K^T of this one has completed), so that its first
-            //      tiles are scored while this unit's epilogue runs
-            // (a group that did not take the part's last tile has not yet seen that tile's scores complete)
+            // every Q K^T of this part must have completed before this part's Q buffer is overwritten at the start of
+            // the next part (a group that did not take the last tile has not yet seen that tile's scores complete)
             if (ctrl->abort || !T_WAIT(s_max, ptx::mbar_wait(&ctrl->s_full[(it - 1) & (kSBufs - 1)], ((it - 1) / kSBufs) & 1))) { timeout(p, ctrl, 37); ok = false; break; }
-            if (has_next) {
-#ifdef MIRROR_ATTN_TIMING
-                te = T_NOW();
-#endif
-                stage_q(sg_next.u);
-#ifdef MIRROR_ATTN_TIMING
-                t_q += T_NOW() - te;
-#endif
-            }
+            if (q_pending) { q_ready((seg + 1) & 1); q_pending = false; }
+            ++seg;
 
             // ---- end of this CTA's part of the unit: the two groups exchange (offset, sum), then each warp
             //      combines its half of the columns of both accumulators once the last P V is complete
@@ -847,7 +850,8 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             if (!T_WAIT(s_free, pair_sync())) { timeout(p, ctrl, 36); ok = false; break; }
             if (has_next) sg = sg_next;
         }
-        if (warp == 4 && lane == 0) { T_STORE(8, T_NOW() - t0, w_sf, w_pv, w_end, t_epi, t_q, (long long)it); T_STORE(40, s_ld, s_free, s_max, s_xch, s_exp, s_fin); T_STORE(52, t_init, t_loop); }
+        asm volatile("cp.async.wait_all;" ::: "memory");      // (only an aborted run can still have copies in flight here)
+        if (warp == 4 && lane == 0) { T_STORE(8, T_NOW() - t0, w_sf, w_pv, w_end, t_epi, t_q, (long long)it); T_STORE(40, s_ld, s_free, s_max, s_xch, s_exp, s_fin); T_STORE(52, t_init, t_loop, t_max, t_ld1); }
     }
 
     ptx::tc_fence_before();
