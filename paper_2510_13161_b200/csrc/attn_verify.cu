@@ -31,6 +31,8 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <type_traits>
+
 #include "mirror_internal.h"
 
 namespace {
@@ -43,7 +45,7 @@ constexpr int kTileSlots = 4;
 constexpr int kTileTok = kSlotTok * kTileSlots;     // 64
 constexpr int kRows = 128;                          // UMMA M: rows per row block
 constexpr int kMaxBatch = 1024;
-constexpr int kKVStages = 4;                        // power of two: stage = tile counter & 3
+constexpr int kMaxStages = 8;                       // ring depths are template parameters (even: tiles are staged in pairs)
 constexpr int kSBufs = 4;                           // S buffers in TMEM (power of two)
 constexpr int kMergeWarps = 8;
 constexpr float kRescaleLog2 = 8.0f;
@@ -60,6 +62,7 @@ struct AttnParams {
     int n_groups;                         // CTA groups (grid = n_groups * n_rb)
     int snap_cap;                         // boundaries move to a unit boundary that is at most this many tiles away
     int max_pages, num_pages, layer_pages;
+    int q_half_bytes;                     // one 64-column half of a Q buffer: rows rounded up to 8, 128 B each
     int tree_slots;
     float scale_log2e, scale;
     const int32_t* page_table;
@@ -84,8 +87,8 @@ struct UnitPos {                          // where a global tile index falls
 };
 
 struct Ctrl {
-    uint64_t k_full[kKVStages], k_empty[kKVStages];     // K ring: refilled as soon as Q K^T has read a stage
-    uint64_t v_full[kKVStages], v_empty[kKVStages];     // V ring: refilled once P V has read a stage
+    uint64_t k_full[kMaxStages], k_empty[kMaxStages];   // K ring: refilled as soon as Q K^T has read a stage
+    uint64_t v_full[kMaxStages], v_empty[kMaxStages];   // V ring: refilled once P V has read a stage
     uint64_t s_full[kSBufs], s_free[kSBufs];
     uint64_t p_full[kSBufs], pv_done[2];
     uint64_t q_full[2];
@@ -103,16 +106,17 @@ __device__ __forceinline__ void timeout(const AttnParams& p, Ctrl* c, int where)
     if (atomicCAS(p.status, 0, MIRROR_DEV_TIMEOUT) == 0) atomicExch(p.status + 1, where);
 }
 
-__device__ __forceinline__ UnitPos locate(long long x, const AttnParams& p, const int* cumT, long long tiles_per_layer) {
+__device__ __noinline__ UnitPos locate(long long x, const AttnParams& p, const int* cumT, long long tiles_per_layer) {
     UnitPos u;
-    u.layer = (int)(x / tiles_per_layer);
+    // (the tile count fits 31 bits: checked in the prologue; 32-bit divisions are several times cheaper)
+    u.layer = (int)((uint32_t)x / (uint32_t)tiles_per_layer);
     const long long rem = x - (long long)u.layer * tiles_per_layer;
     int b = 0;
     while (b + 1 < p.B && (long long)p.Hkv * cumT[b + 1] <= rem) ++b;
     const int Tb = cumT[b + 1] - cumT[b];
     const long long r2 = rem - (long long)p.Hkv * cumT[b];
     u.b = b;
-    u.g = (int)(r2 / Tb);
+    u.g = (int)((uint32_t)r2 / (uint32_t)Tb);
     u.tile_in_unit = (int)(r2 - (long long)u.g * Tb);
     u.tiles_in_unit = Tb;
     u.unit_first_tile = x - u.tile_in_unit;
@@ -126,7 +130,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 // Shared-memory operand tiles are [64-column half][row][128 B] with the 128-byte swizzle: the 16-byte chunk
 // index is XORed with (row % 8).  A half of Q or P holds 128 rows (16 KB), a half of a K/V stage 64 tokens (8 KB).
-constexpr int kHalfBytes = kRows * 128;
 constexpr int kStageSlots = 4;                      // slots per ring stage
 __device__ __forceinline__ uint32_t tile_off(int row, int chunk, int half_bytes) {   // chunk: 16-byte column chunk
     return (uint32_t)((chunk >> 3) * half_bytes + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
@@ -171,12 +174,45 @@ __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.
 template <int D>
 struct Cfg {
     static constexpr int kHalves = D / 64;
-    static constexpr int kQBytes = kHalves * kHalfBytes;           // Q: 128 rows x D
     static constexpr int kSlotBytes = kHalves * kSlotTok * 128;    // one slot of K or V: [half][16 tokens][128 B] = one TMA box
     static constexpr int kStageBytes = kStageSlots * kSlotBytes;   // one K (or V) stage: 4 slots; stages are contiguous
-    static constexpr size_t kSmemData = 2 * (size_t)kQBytes + 2 * (size_t)kKVStages * kStageBytes;
-    static constexpr size_t kSmemBytes = kSmemData + 512 /*ctrl*/ + 2 * 2 * kRows * 4 /*pair exchange*/ + (2 * kMaxBatch + 2) * 4 + 1024 /*align*/;
+    static constexpr size_t kSmemFixed = 512 /*ctrl*/ + 2 * 2 * kRows * 4 /*pair exchange*/ + (2 * kMaxBatch + 2) * 4 + 1024 /*align*/;
+    // Shared memory: two Q buffers sized by the rows a CTA really has (the UMMA reads 128 rows per half and
+    // runs on into whatever follows; those rows only reach TMEM lanes nobody reads), then the K and V rings.
+    // What the rings can hold in flight bounds the bandwidth one SM can pull at HBM latency, so they get
+    // every byte the Q buffers leave.
+    static size_t smem_bytes(int q_half_bytes, int ks, int vs) {
+        return 2 * (size_t)kHalves * q_half_bytes + (size_t)(ks + vs) * kStageBytes + kSmemFixed;
+    }
 };
+
+struct PendingUnit {                      // a unit whose partial this CTA has left; arrival and merge come at the CTA's end
+    int layer, b, g, ga, gb;
+    long long unit_first_tile;
+};
+
+// Visibility of 32 score columns (four slots from sl0, eight tokens from tr0 of each: column c is token tr0 + c%8 of
+// slot sl0 + c/8) for a row whose visible tree tokens are the bits of (anc0, anc1).  Kept out of line and rolled:
+// it runs for a unit's last tiles only.
+__device__ __noinline__ uint32_t chunk_mask(int sl0, int tr0, int pages_full, int pages_all, int slots_all, int len,
+                                            unsigned long long anc0, unsigned long long anc1) {
+    uint32_t cm = 0;
+#pragma unroll 1
+    for (int jj = 0; jj < 4; ++jj) {
+        const int sl = sl0 + jj;
+        uint32_t bits = 0;
+        if (sl < pages_full) {
+            bits = 0xffffu;
+        } else if (sl < pages_all) {
+            bits = (1u << (len - sl * kSlotTok)) - 1u;                              // ragged page: 1..15 valid tokens
+        } else if (sl < slots_all) {
+            const int ts = sl - pages_all;                                          // tree tokens 16*ts .. 16*ts+15
+            bits = (uint32_t)(((ts < 4) ? anc0 : anc1) >> ((ts & 3) * 16)) & 0xffffu;   // ancestors-or-self (all < n)
+        }
+        cm |= ((bits >> tr0) & 0xffu) << (jj * 8);
+    }
+    return cm;
+}
 
 // A segment: the part of one unit that this CTA processes.
 struct Segment {
@@ -184,7 +220,7 @@ struct Segment {
     int t_first, t_last;                  // tiles [t_first, t_last) of the unit
     int len, pages_full, pages_all, slots_all;
 };
-__device__ __forceinline__ Segment make_segment(long long x, long long x_end, const AttnParams& p, const int* cumT,
+__device__ __noinline__ Segment make_segment(long long x, long long x_end, const AttnParams& p, const int* cumT,
                                                 const int* s_len, long long tiles_per_layer) {
     Segment s;
     s.u = locate(x, p, cumT, tiles_per_layer);
@@ -197,7 +233,7 @@ __device__ __forceinline__ Segment make_segment(long long x, long long x_end, co
     return s;
 }
 
-template <int D>
+template <int D, int KS, int VS>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                    const __grid_constant__ AttnTree tree, const AttnParams p) {
@@ -205,9 +241,10 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* sQ = smem;                                             // [2]: the units a CTA walks alternate
-    uint8_t* sK = sQ + 2 * C::kQBytes;                              // [kKVStages]  [slot][half][16 tokens][128 B]
-    uint8_t* sV = sK + kKVStages * C::kStageBytes;                  // [kKVStages]  [slot][half][16 tokens][128 B]
-    Ctrl* ctrl = (Ctrl*)(sV + kKVStages * C::kStageBytes);
+    const int q_buf_bytes = C::kHalves * p.q_half_bytes;
+    uint8_t* sK = sQ + 2 * q_buf_bytes;                             // [KS]  [slot][half][16 tokens][128 B]
+    uint8_t* sV = sK + KS * C::kStageBytes;                         // [VS]  [slot][half][16 tokens][128 B]
+    Ctrl* ctrl = (Ctrl*)(sV + VS * C::kStageBytes);
     float* xch = (float*)((uint8_t*)ctrl + 512);                    // [2 tiles][2 halves][128 rows] pair exchange
     int* cumT = (int*)((uint8_t*)ctrl + 512 + 2 * 2 * kRows * 4);   // [B+1] tiles per request, prefix-summed
     int* s_len = cumT + (kMaxBatch + 1);                            // [B] clamped prefix lengths
@@ -228,7 +265,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         s_len[b] = len;
     }
     if (tid == 0) {
-        for (int s = 0; s < kKVStages; ++s) {
+        for (int s = 0; s < kMaxStages; ++s) {
             ptx::mbar_init(&ctrl->k_full[s], 1); ptx::mbar_init(&ctrl->k_empty[s], 1);
             ptx::mbar_init(&ctrl->v_full[s], 1); ptx::mbar_init(&ctrl->v_empty[s], 2);   // both tiles of a pair read a V stage
         }
@@ -283,8 +320,10 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         const long long dist = best > e ? best - e : e - best;
         return dist <= snap_tol ? best : e;
     };
-    const long long x_begin = group < n_groups ? group_begin(group) : 0;
-    const long long x_end = group < n_groups ? group_begin(group + 1) : 0;
+    const bool fits = total_tiles < (1ll << 31);
+    if (!fits && tid == 0) dev_check(p, 600);
+    const long long x_begin = (fits && group < n_groups) ? group_begin(group) : 0;
+    const long long x_end = (fits && group < n_groups) ? group_begin(group + 1) : 0;
 
     T_STAMP(1);
     if (warp == 0 || warp == kVProducerWarp) {
@@ -311,12 +350,26 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 return (has_box && sl < sg.pages_full) ? pt[sl] : 0;
             };
             int my_page = fetch_page(sg.t_first);
+            if (sg.t_last == u.tiles_in_unit) {
+                // the unit's last slots (a ragged page, the tree's own tokens) are staged by plain loads many tiles
+                // from now: pull them into L2 so that those loads do not hold up the ring for an HBM round trip
+                for (int j = lane; j < p.n; j += 32) {
+                    const __nv_bfloat16* row = (vrole ? p.v_new : p.k_new) + ((((size_t)u.layer * p.B + u.b) * p.n + j) * p.Hkv + u.g) * (size_t)D;
+                    ptx::prefetch_l2(row);
+                    if (D == 128) ptx::prefetch_l2(row + 64);
+                }
+                if (sg.pages_all > sg.pages_full) {
+                    const int page = pt[sg.pages_full];
+                    if (page >= 0 && page < p.num_pages && lane < kSlotTok * D * 2 / 128)
+                        ptx::prefetch_l2((vrole ? p.v_pool : p.k_pool) + (((size_t)u.layer * p.layer_pages + page) * p.Hkv + u.g) * (size_t)(kSlotTok * D) + lane * 64);
+                }
+            }
             for (int t = sg.t_first; t < sg.t_last && ok; ++t, ++x, ++it) {
 #ifdef MIRROR_ATTN_TIMING
                 tm__ = T_NOW();
 #endif
-                const int st = it & (kKVStages - 1);
-                const uint32_t ph = (it / kKVStages) & 1;
+                const int st = vrole ? (int)(it % VS) : (int)(it % KS);
+                const uint32_t ph = (vrole ? it / VS : it / KS) & 1;
                 const int next_page = (t + 1 < sg.t_last) ? fetch_page(t + 1) : 0;
                 bool w = true;
                 if (lane == 0) w = !ctrl->abort && T_WAIT(w_empty, ptx::mbar_wait(&empty[st], ph ^ 1));
@@ -331,7 +384,12 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                                        ? n_slots + 1 : n_slots;
                 T_MARK(p_pre);
                 if (n_tma < n_fill) {
-                    // ragged page and tree tokens by plain loads (rows beyond the valid count are zero)
+                    // ragged page and tree tokens by asynchronous 16-byte copies (rows beyond the valid count are
+                    // zero-filled), all in flight together; the loops are kept rolled: this path runs once per unit, and
+                    // what it costs is mostly the instruction fetch
+                    constexpr int kChunks = kSlotTok * D / 8;          // 16-byte chunks per slot
+                    constexpr int kPer = kChunks / 32;
+#pragma unroll 1
                     for (int j = n_tma; j < n_fill; ++j) {
                         const int sl = sl0 + j;
                         const __nv_bfloat16* src = p.k_pool;
@@ -351,21 +409,17 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                             row_stride = (size_t)p.Hkv * D;
                             valid = min(kSlotTok, p.n - j0);
                         }
-                        constexpr int kChunks = kSlotTok * D / 8;          // 16-byte chunks per slot
-                        constexpr int kPer = kChunks / 32;
-                        uint4 vv[kPer];
-#pragma unroll
+#pragma unroll 1
                         for (int i = 0; i < kPer; ++i) {
                             const int c = lane + i * 32, tr = c / (D / 8), cc = c % (D / 8);
-                            vv[i] = (tr < valid) ? *reinterpret_cast<const uint4*>(src + tr * row_stride + cc * 8) : make_uint4(0, 0, 0, 0);
-                        }
-#pragma unroll
-                        for (int i = 0; i < kPer; ++i) {
-                            const int c = lane + i * 32, tr = c / (D / 8), cc = c % (D / 8);
-                            *reinterpret_cast<uint4*>(dst + j * C::kSlotBytes + tile_off(tr, cc, kSlotTok * 128)) = vv[i];
+                            const bool in = tr < valid;
+                            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
+                                         ::"r"(ptx::smem_u32(dst + j * C::kSlotBytes + tile_off(tr, cc, kSlotTok * 128))),
+                                           "l"(in ? src + tr * row_stride + cc * 8 : p.k_pool), "r"(in ? 16u : 0u) : "memory");
                         }
                     }
-                    // the plain stores are read by the tensor core, and later overwritten by bulk copies (async proxy)
+                    asm volatile("cp.async.wait_all;" ::: "memory");
+                    // these copies are read by the tensor core, and later overwritten by bulk copies (async proxy)
                     ptx::fence_proxy_async();
                     __syncwarp();
                 }
@@ -388,9 +442,10 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         if (lane == 0) T_STORE(vrole ? 32 : 16, T_NOW() - t0, w_empty, (long long)it, p_pre, p_fill, p_issue);
         if (!ok && lane == 0) {
             // let copies already in flight land before the CTA's shared memory goes away
-            const uint32_t back = it < (uint32_t)kKVStages ? it : (uint32_t)kKVStages;
+            const uint32_t ns = vrole ? VS : KS;
+            const uint32_t back = it < ns ? it : ns;
             for (uint32_t j = it - back; j < it; ++j)
-                ptx::mbar_wait(&full[j & (kKVStages - 1)], (j / kKVStages) & 1, 200000000ll);
+                ptx::mbar_wait(&full[j % ns], (j / ns) & 1, 200000000ll);
         }
     } else if (warp == 1) {
         // =========================================================================== Q K^T issuer
@@ -410,19 +465,19 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             while (x < x_end && ok) {
                 const Segment sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
                 if (ctrl->abort || !T_WAIT(w_q, ptx::mbar_wait(&ctrl->q_full[seg & 1], (seg >> 1) & 1))) { timeout(p, ctrl, 20); ok = false; break; }
-                const uint32_t q_seg = q_lo + (uint32_t)(((seg & 1) * C::kQBytes) >> 4);
+                const uint32_t q_seg = q_lo + (uint32_t)(((seg & 1) * q_buf_bytes) >> 4);
                 ++seg;
                 // parts begin and end on pairs of tiles: a pair is the eight slots of two consecutive ring stages
                 for (int t = sg.t_first; t < sg.t_last; t += 2, x += 2, it += 2) {
                     bool ready = !ctrl->abort;
                     for (int j = 0; j < 2 && ready; ++j) {
                         const uint32_t i2 = it + j;
-                        ready = T_WAIT(w_k, ptx::mbar_wait(&ctrl->k_full[i2 & (kKVStages - 1)], (i2 / kKVStages) & 1)) &&
+                        ready = T_WAIT(w_k, ptx::mbar_wait(&ctrl->k_full[i2 % KS], (i2 / KS) & 1)) &&
                                 T_WAIT(w_s, ptx::mbar_wait(&ctrl->s_free[i2 & (kSBufs - 1)], ((i2 / kSBufs) & 1) ^ 1));
                     }
                     if (!ready) { timeout(p, ctrl, 21); ok = false; break; }
                     ptx::tc_fence_after();
-                    const int st = it & (kKVStages - 1), sb = it & (kSBufs - 1);
+                    const int st = it % KS, sb = it & (kSBufs - 1);
                     // slots scored: those that exist, rounded up to even (N must be a multiple of 16)
                     const int ne = min(2 * kStageSlots, (sg.slots_all - t * kStageSlots + 1) & ~1);
                     const uint32_t idesc = ptx::umma_idesc_bf16(kRows, ne * 8);
@@ -433,7 +488,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                         const uint32_t d = tmem_base + (uint32_t)((sb + h) * kTileTok);
 #pragma unroll
                         for (int kk = 0; kk < D / 16; ++kk)
-                            ptx::umma_f16_lohi(d, q_seg + (uint32_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4), hi_q,
+                            ptx::umma_f16_lohi(d, q_seg + (uint32_t)(((kk >> 2) * p.q_half_bytes + (kk & 3) * 32) >> 4), hi_q,
                                                kb + (uint32_t)(((kk >> 2) * (kSlotTok * 128) + h * 1024 + (kk & 3) * 32) >> 4), hi_k,
                                                idesc, kk != 0);
                         ptx::umma_commit(&ctrl->s_full[sb + h]);
@@ -467,10 +522,10 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
                     // tile h of a pair reads tokens 8h..8h+7 of the pair's eight slots (both stages)
                     const uint32_t it0 = it & ~1u;
-                    const int st0 = it0 & (kKVStages - 1), pb = it & 1, sb = it & (kSBufs - 1);
+                    const int st0 = it0 % VS, pb = it & 1, sb = it & (kSBufs - 1);
                     if (ctrl->abort || !T_WAIT(w_p, ptx::mbar_wait(&ctrl->p_full[sb], (it / kSBufs) & 1)) ||
-                        !T_WAIT(w_v, ptx::mbar_wait(&ctrl->v_full[st0], (it0 / kKVStages) & 1)) ||
-                        !T_WAIT(w_v, ptx::mbar_wait(&ctrl->v_full[st0 + 1], (it0 / kKVStages) & 1))) {
+                        !T_WAIT(w_v, ptx::mbar_wait(&ctrl->v_full[st0], (it0 / VS) & 1)) ||
+                        !T_WAIT(w_v, ptx::mbar_wait(&ctrl->v_full[st0 + 1], (it0 / VS) & 1))) {
                         timeout(p, ctrl, 23); ok = false; break;
                     }
                     ptx::tc_fence_after();
@@ -523,13 +578,14 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         // (rows that do not exist are zero-filled); q_ready() later makes them visible to the tensor core
         auto stage_q = [&](const UnitPos& u, int buf) {
             const __nv_bfloat16* qrow = p.q + ((((size_t)u.layer * p.B + u.b) * p.n + node) * (size_t)p.Hq + u.g * p.G + hl) * D;
-            uint8_t* q = sQ + buf * C::kQBytes;
+            uint8_t* q = sQ + buf * q_buf_bytes;
             const uint32_t src_bytes = row_ok ? 16u : 0u;
+            if (row_in_blk * 128 >= p.q_half_bytes) return;        // the buffer holds no such row
 #pragma unroll
             for (int i = 0; i < D / 16; ++i) {
                 const int chunk = grp * (D / 16) + i;
                 asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
-                             ::"r"(ptx::smem_u32(q + tile_off(row_in_blk, chunk, kHalfBytes))), "l"(qrow + chunk * 8), "r"(src_bytes) : "memory");
+                             ::"r"(ptx::smem_u32(q + tile_off(row_in_blk, chunk, p.q_half_bytes))), "l"(qrow + chunk * 8), "r"(src_bytes) : "memory");
             }
         };
         auto q_ready = [&](int buf) {
@@ -544,43 +600,27 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         long long x = x_begin;
         T_DECL(w_sf = 0, w_pv = 0, w_end = 0, t_epi = 0, t_q = 0, t0 = T_NOW(), te = 0, tm__ = 0, s_ld = 0, s_free = 0, s_max = 0, s_xch = 0, s_exp = 0, s_fin = 0, t_init = 0, t_loop = 0, tl = 0, t_max = 0, t_ld1 = 0);
         Segment sg;
-        // one 32-column chunk of this row's scores: tcgen05.ld, then the visibility mask where the tile needs one
-        auto load_scores = [&](int sb, int c4, int t, float (&v)[32]) {
+        // one 32-column chunk of this row's scores: tcgen05.ld, then the visibility mask (bit j: column j) where the
+        // tile needs one
+        auto load_scores = [&](int sb, int c4, uint32_t cm, float (&v)[32]) {
             uint32_t r[32];
             ptx::tmem_ld_32x32b_x32(lane_base + (uint32_t)(sb * kTileTok + c4 * 32), r);
             ptx::tmem_ld_wait();
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-            // column c of tile h of a pair is token 8h + c%8 of the pair's slot c/8
-            const int sl0 = (t & ~1) * kStageSlots + c4 * 4;
-            const int tr0 = (t & 1) * 8;
-            if (sl0 + 4 > sg.pages_full) {             // a ragged page, tree tokens or missing slots
+            if (cm != 0xffffffffu) {
 #pragma unroll
-                for (int jj = 0; jj < 4; ++jj) {
-                    const int sl = sl0 + jj;
-                    if (sl < sg.pages_full) continue;
-                    // visibility of the slot's 16 tokens as a bit mask
-                    uint32_t bits = 0;
-                    if (sl < sg.pages_all) {
-                        bits = (1u << (sg.len - sl * kSlotTok)) - 1u;                       // ragged page: 1..15 valid tokens
-                    } else if (sl < sg.slots_all) {
-                        const int ts = sl - sg.pages_all;                                   // tree tokens 16*ts .. 16*ts+15
-                        bits = (uint32_t)(((ts < 4) ? anc0 : anc1) >> ((ts & 3) * 16)) & 0xffffu;   // ancestors-or-self (all < n)
-                    }
-                    bits >>= tr0;
-#pragma unroll
-                    for (int tr = 0; tr < 8; ++tr)
-                        if (!((bits >> tr) & 1u)) v[jj * 8 + tr] = -INFINITY;
-                }
+                for (int j = 0; j < 32; ++j)
+                    if (!((cm >> j) & 1u)) v[j] = -INFINITY;
             }
         };
         // pass 1: the row maximum of a tile
-        auto tile_max = [&](int sb, int t) -> float {
+        auto tile_max = [&](int sb, uint32_t cm0, uint32_t cm1) -> float {
             float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
             for (int c4 = 0; c4 < kTileTok / 32; ++c4) {
                 float v[32];
-                load_scores(sb, c4, t, v);
+                load_scores(sb, c4, c4 == 0 ? cm0 : cm1, v);
                 if (c4 == 0) T_MARK(t_ld1);
 #pragma unroll
                 for (int j = 0; j < 32; ++j) m4[j & 3] = fmaxf(m4[j & 3], v[j]);
@@ -590,13 +630,13 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         // pass 2: P = exp2(s*c - offset) as bf16 pairs over the first 32 columns of the same S buffer (a thread
         // only ever touches its own lane, and a 32-column chunk of S is in registers before its P is written
         // over columns that were read earlier); returns the row sum
-        auto tile_p = [&](int sb, int t, float m_off) -> float {
+        auto tile_p = [&](int sb, uint32_t cm0, uint32_t cm1, float m_off) -> float {
             const float off = (m_off == -INFINITY) ? 0.f : m_off * p.scale_log2e;
             float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int c4 = 0; c4 < kTileTok / 32; ++c4) {
                 float v[32];
-                load_scores(sb, c4, t, v);
+                load_scores(sb, c4, c4 == 0 ? cm0 : cm1, v);
                 uint32_t pk[16];
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
@@ -612,6 +652,8 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         };
 
         uint32_t seg = 0;                                          // parts walked so far: Q buffer = seg & 1
+        PendingUnit pend0, pend1;                                  // units cut across CTAs: at most the first and the last part
+        int n_pend = 0;
         if (x < x_end) {
             sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
             stage_q(sg.u, 0);
@@ -654,7 +696,13 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 tm__ = T_NOW();
 #endif
                 float mx = -INFINITY, sum = 0.f;
-                if (warp_has_rows) mx = tile_max(sb, t);
+                // visibility of this tile's columns for this row: all ones except in a unit's last pairs
+                uint32_t cm0 = 0xffffffffu, cm1 = 0xffffffffu;
+                if ((t & ~1) * kStageSlots + 2 * kStageSlots > sg.pages_full) {
+                    cm0 = chunk_mask((t & ~1) * kStageSlots, (t & 1) * 8, sg.pages_full, sg.pages_all, sg.slots_all, sg.len, anc0, anc1);
+                    cm1 = chunk_mask((t & ~1) * kStageSlots + 4, (t & 1) * 8, sg.pages_full, sg.pages_all, sg.slots_all, sg.len, anc0, anc1);
+                }
+                if (warp_has_rows) mx = tile_max(sb, cm0, cm1);
                 T_MARK(t_max);
                 if (first) m_used = mx;
                 // offset in use: set by the group's first tile, moved only when the row maximum outgrew it by more than 2^8
@@ -667,7 +715,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     const float m_next = move ? fmaxf(mx, m_used) : m_used;
                     const float alpha = (m_used == -INFINITY) ? ((m_next == -INFINITY) ? 1.f : 0.f)
                                                               : exp2f((m_used - m_next) * p.scale_log2e);
-#pragma unroll
+#pragma unroll 1
                     for (int c4 = 0; c4 < D / 32; ++c4) {
                         uint32_t r[32];
                         ptx::tmem_ld_32x32b_x32(o_mine + (uint32_t)(c4 * 32), r);
@@ -680,7 +728,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     l_run *= alpha;
                     m_used = m_next;
                 }
-                if (warp_has_rows) sum = tile_p(sb, t, m_used);
+                if (warp_has_rows) sum = tile_p(sb, cm0, cm1, m_used);
                 T_MARK(s_exp);
                 l_run += sum;
                 first = false;
@@ -696,9 +744,11 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             t_loop += T_NOW() - tl;
 #endif
 
-            // every Q K^T of this part must have completed before this part's Q buffer is overwritten at the start of
-            // the next part (a group that did not take the last tile has not yet seen that tile's scores complete)
-            if (ctrl->abort || !T_WAIT(s_max, ptx::mbar_wait(&ctrl->s_full[(it - 1) & (kSBufs - 1)], ((it - 1) / kSBufs) & 1))) { timeout(p, ctrl, 37); ok = false; break; }
+            // (This part's Q buffer is overwritten at the start of the next part.  Every Q K^T that reads it has
+            // completed by then: both groups wait below for the P V of the part's last tile, which follows that
+            // tile's P, its S and so its Q K^T.  Waiting here on the last tile's s_full instead would be wrong: the
+            // issuer can run on into the next unit, and a second completion of that barrier would make a late
+            // waiter's parity match the wrong phase.)
             if (q_pending) { q_ready((seg + 1) & 1); q_pending = false; }
             ++seg;
 
@@ -739,7 +789,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 float* my = p.partial + ((size_t)blockIdx.x * 2 + slot) * kRowW * kRows + row_in_blk;
                 const float inv = 1.f / Lsum;
                 // combined accumulator columns [grp*kDH, (grp+1)*kDH) of both groups' O, 32 at a time
-#pragma unroll
+#pragma unroll 1
                 for (int c4 = 0; c4 < kDH / 32; ++c4) {
                     float acc[32];
                     {
@@ -781,61 +831,17 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 if (whole_unit) {
                     if (lse_ptr && row_ok) *lse_ptr = M * p.scale + logf(Lsum);
                 } else {
-                    // ---- the unit is cut across CTA groups: the partial is left, the last arrival merges ------
-                    const int parts = gb - ga + 1;
+                    // ---- the unit is cut across CTA groups: the partial is left now; the arrival at the unit's
+                    //      counter (and the merge, for the last one to arrive) waits until this CTA has walked all its
+                    //      tiles, so that neither the fence nor the merge stalls the tiles that follow
                     my[(size_t)(D + 2 * grp) * kRows] = M;
                     my[(size_t)(D + 2 * grp + 1) * kRows] = Lsum;
-                    __threadfence();
-                    __syncwarp();
-                    const size_t unit_idx = ((size_t)u.layer * p.B + u.b) * p.Hkv + u.g;
-                    int* tk = p.ticket + (unit_idx * p.n_rb + rb) * kMergeWarps + (grp * 4 + w4);
-                    int arrived = 0;
-                    if (lane == 0) arrived = atomicAdd(tk, 1);
-                    arrived = __shfl_sync(0xffffffffu, arrived, 0);
-                    if (arrived == parts - 1) {
-                        __threadfence();
-                        if (lane == 0) *tk = 0;                          // ready for the next launch
-                        // merge in group order
-                        float Mm = -INFINITY;
-                        for (int gsrc = ga; gsrc <= gb; ++gsrc) {
-                            const int sslot = (group_begin(gsrc) > u.unit_first_tile) ? 0 : 1;
-                            const float* src = p.partial + ((size_t)(gsrc * p.n_rb + rb) * 2 + sslot) * kRowW * kRows + row_in_blk;
-                            Mm = fmaxf(Mm, __ldcg(src + (size_t)(D + 2 * grp) * kRows));
-                        }
-                        float Lm = 0.f;
-                        for (int gsrc = ga; gsrc <= gb; ++gsrc) {
-                            const int sslot = (group_begin(gsrc) > u.unit_first_tile) ? 0 : 1;
-                            const float* src = p.partial + ((size_t)(gsrc * p.n_rb + rb) * 2 + sslot) * kRowW * kRows + row_in_blk;
-                            const float pm = __ldcg(src + (size_t)(D + 2 * grp) * kRows);
-                            Lm += ((pm == -INFINITY) ? 0.f : exp2f((pm - Mm) * p.scale_log2e)) * __ldcg(src + (size_t)(D + 2 * grp + 1) * kRows);
-                        }
-                        const float invm = 1.f / Lm;
-#pragma unroll 1
-                        for (int c4 = 0; c4 < kDH / 32; ++c4) {
-                            float acc[32];
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) acc[j] = 0.f;
-                            for (int gsrc = ga; gsrc <= gb; ++gsrc) {
-                                const int sslot = (group_begin(gsrc) > u.unit_first_tile) ? 0 : 1;
-                                const float* src = p.partial + ((size_t)(gsrc * p.n_rb + rb) * 2 + sslot) * kRowW * kRows + row_in_blk;
-                                const float pm = __ldcg(src + (size_t)(D + 2 * grp) * kRows);
-                                const float wgt = (pm == -INFINITY) ? 0.f : exp2f((pm - Mm) * p.scale_log2e);
-#pragma unroll
-                                for (int j = 0; j < 32; ++j) acc[j] = fmaf(wgt, __ldcg(src + (size_t)(grp * kDH + c4 * 32 + j) * kRows), acc[j]);
-                            }
-                            if (row_ok) {
-#pragma unroll
-                                for (int j = 0; j < 4; ++j) {
-                                    uint4 v;
-                                    v.x = pack_bf16(acc[j * 8 + 0] * invm, acc[j * 8 + 1] * invm);
-                                    v.y = pack_bf16(acc[j * 8 + 2] * invm, acc[j * 8 + 3] * invm);
-                                    v.z = pack_bf16(acc[j * 8 + 4] * invm, acc[j * 8 + 5] * invm);
-                                    v.w = pack_bf16(acc[j * 8 + 6] * invm, acc[j * 8 + 7] * invm);
-                                    *reinterpret_cast<uint4*>(orow + c4 * 32 + j * 8) = v;
-                                }
-                            }
-                        }
-                        if (lse_ptr && row_ok) *lse_ptr = Mm * p.scale + logf(Lm);
+                    if (n_pend >= 2) {
+                        dev_check(p, 500);                       // a CTA's range cuts at most two units
+                    } else {
+                        PendingUnit& q = (n_pend == 0) ? pend0 : pend1;
+                        q.layer = u.layer; q.b = u.b; q.g = u.g; q.ga = ga; q.gb = gb; q.unit_first_tile = u.unit_first_tile;
+                        ++n_pend;
                     }
                 }
             } else {
@@ -849,6 +855,78 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             // the exchange words are rewritten at the end of the next part: the partner must have read them
             if (!T_WAIT(s_free, pair_sync())) { timeout(p, ctrl, 36); ok = false; break; }
             if (has_next) sg = sg_next;
+        }
+        // ---- units that this CTA shares with others: arrive, and merge where this is the last arrival -----------
+        if (ok && warp_has_rows && n_pend > 0) {
+            __threadfence();
+            __syncwarp();
+            for (int i = 0; i < n_pend; ++i) {
+                const PendingUnit q = (i == 0) ? pend0 : pend1;
+                const int parts = q.gb - q.ga + 1;
+                const size_t unit_idx = ((size_t)q.layer * p.B + q.b) * p.Hkv + q.g;
+                int* tk = p.ticket + (unit_idx * p.n_rb + rb) * kMergeWarps + (grp * 4 + w4);
+                int arrived = 0;
+                if (lane == 0) arrived = atomicAdd(tk, 1);
+                arrived = __shfl_sync(0xffffffffu, arrived, 0);
+                if (arrived != parts - 1) continue;
+                __threadfence();
+                if (lane == 0) *tk = 0;                          // ready for the next launch
+                __nv_bfloat16* orow = p.out + ((((size_t)q.layer * p.B + q.b) * p.n + node) * (size_t)p.Hq + q.g * p.G + hl) * D + grp * kDH;
+                float* lse_ptr = (p.lse_out && grp == 0) ? p.lse_out + (((size_t)q.layer * p.B + q.b) * p.Hq + q.g * p.G + hl) * p.n + node : nullptr;
+                auto part_of = [&](int gsrc) -> const float* {
+                    const int sslot = (group_begin(gsrc) > q.unit_first_tile) ? 0 : 1;
+                    return p.partial + ((size_t)(gsrc * p.n_rb + rb) * 2 + sslot) * kRowW * kRows + row_in_blk;
+                };
+                // merge in group order; (max, sum) of the first parts stay in registers
+                constexpr int kKeep = 4;
+                float pmv[kKeep], plv[kKeep];
+                float Mm = -INFINITY;
+#pragma unroll
+                for (int k = 0; k < kKeep; ++k) {
+                    pmv[k] = -INFINITY; plv[k] = 0.f;
+                    if (k < parts) {
+                        const float* src = part_of(q.ga + k);
+                        pmv[k] = __ldcg(src + (size_t)(D + 2 * grp) * kRows);
+                        plv[k] = __ldcg(src + (size_t)(D + 2 * grp + 1) * kRows);
+                    }
+                }
+#pragma unroll
+                for (int k = 0; k < kKeep; ++k) Mm = fmaxf(Mm, pmv[k]);
+                for (int k = kKeep; k < parts; ++k) Mm = fmaxf(Mm, __ldcg(part_of(q.ga + k) + (size_t)(D + 2 * grp) * kRows));
+                auto weight = [&](float pm) -> float { return (pm == -INFINITY) ? 0.f : exp2f((pm - Mm) * p.scale_log2e); };
+                float Lm = 0.f;
+#pragma unroll
+                for (int k = 0; k < kKeep; ++k) Lm += weight(pmv[k]) * plv[k];
+                for (int k = kKeep; k < parts; ++k) {
+                    const float* src = part_of(q.ga + k);
+                    Lm += weight(__ldcg(src + (size_t)(D + 2 * grp) * kRows)) * __ldcg(src + (size_t)(D + 2 * grp + 1) * kRows);
+                }
+                const float invm = 1.f / Lm;
+#pragma unroll 1
+                for (int c4 = 0; c4 < kDH / 32; ++c4) {
+                    float acc[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+                    for (int k = 0; k < parts; ++k) {
+                        const float* src = part_of(q.ga + k);
+                        const float wgt = weight(__ldcg(src + (size_t)(D + 2 * grp) * kRows));
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) acc[j] = fmaf(wgt, __ldcg(src + (size_t)(grp * kDH + c4 * 32 + j) * kRows), acc[j]);
+                    }
+                    if (row_ok) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            uint4 v;
+                            v.x = pack_bf16(acc[j * 8 + 0] * invm, acc[j * 8 + 1] * invm);
+                            v.y = pack_bf16(acc[j * 8 + 2] * invm, acc[j * 8 + 3] * invm);
+                            v.z = pack_bf16(acc[j * 8 + 4] * invm, acc[j * 8 + 5] * invm);
+                            v.w = pack_bf16(acc[j * 8 + 6] * invm, acc[j * 8 + 7] * invm);
+                            *reinterpret_cast<uint4*>(orow + c4 * 32 + j * 8) = v;
+                        }
+                    }
+                }
+                if (lse_ptr && row_ok) *lse_ptr = Mm * p.scale + logf(Lm);
+            }
         }
         asm volatile("cp.async.wait_all;" ::: "memory");      // (only an aborted run can still have copies in flight here)
         if (warp == 4 && lane == 0) { T_STORE(8, T_NOW() - t0, w_sf, w_pv, w_end, t_epi, t_q, (long long)it); T_STORE(40, s_ld, s_free, s_max, s_xch, s_exp, s_fin); T_STORE(52, t_init, t_loop, t_max, t_ld1); }
@@ -883,6 +961,7 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
     if (kv->layer_stride % page_elems != 0) return MIRROR_ERR_UNSUPPORTED;
     p.layer_pages = (int)(kv->layer_stride / page_elems);
     p.tree_slots = (p.n + kSlotTok - 1) / kSlotTok;
+    p.q_half_bytes = ((p.rows_per_rb + 7) / 8) * 8 * 128;
     p.scale = ctx->scale;
     p.scale_log2e = ctx->scale * 1.4426950408889634f;
     p.page_table = kv->page_table; p.prefix_len = kv->prefix_len;
@@ -915,13 +994,29 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
         if (st != MIRROR_OK) return st;
     }
     const int grid = p.n_groups * p.n_rb;
-    if (D == 128) {
-        MIRROR_CUDA_OK(cudaFuncSetAttribute(attn_verify_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<128>::kSmemBytes));
-        attn_verify_kernel<128><<<grid, kThreads, Cfg<128>::kSmemBytes, stream>>>(tm_k, tm_v, at, p);
-    } else {
-        MIRROR_CUDA_OK(cudaFuncSetAttribute(attn_verify_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<64>::kSmemBytes));
-        attn_verify_kernel<64><<<grid, kThreads, Cfg<64>::kSmemBytes, stream>>>(tm_k, tm_v, at, p);
-    }
+    // ring depths: the deepest pair (K, V) that fits beside the Q buffers
+    constexpr size_t kSmemLimit = 232448;       // 227 KB
+    auto launch = [&](auto d_tag) -> mirror_status {
+        constexpr int DD = decltype(d_tag)::value;
+        using C = Cfg<DD>;
+        int ks = 4, vs = 4;
+        if (C::smem_bytes(p.q_half_bytes, 6, 4) <= kSmemLimit) ks = 6;
+        if (C::smem_bytes(p.q_half_bytes, 6, 6) <= kSmemLimit) vs = 6;
+        if (const char* e = getenv("MIRROR_ATTN_RING")) { const int r = atoi(e); ks = r / 10; vs = r % 10; }
+        if (!((ks == 4 || ks == 6) && (vs == 4 || (vs == 6 && ks == 6)))) return MIRROR_ERR_ARG;
+        const size_t smem = C::smem_bytes(p.q_half_bytes, ks, vs);
+        if (smem > kSmemLimit) return MIRROR_ERR_UNSUPPORTED;
+        auto go = [&](auto kern) -> mirror_status {
+            MIRROR_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit));
+            kern<<<grid, kThreads, smem, stream>>>(tm_k, tm_v, at, p);
+            return MIRROR_OK;
+        };
+        if (ks == 6 && vs == 6) return go(attn_verify_kernel<DD, 6, 6>);
+        if (ks == 6) return go(attn_verify_kernel<DD, 6, 4>);
+        return go(attn_verify_kernel<DD, 4, 4>);
+    };
+    mirror_status lst = (D == 128) ? launch(std::integral_constant<int, 128>{}) : launch(std::integral_constant<int, 64>{});
+    if (lst != MIRROR_OK) return lst;
     ctx->launches += 1;
     MIRROR_CUDA_OK(cudaGetLastError());
     return MIRROR_OK;
