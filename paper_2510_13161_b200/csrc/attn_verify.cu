@@ -9,22 +9,25 @@
 // of the pair holds the first eight tokens of each of the eight slots, tile 1 the second eight (so that a whole
 // page is one TMA box and still a legal UMMA operand: the 8-row groups of one tile are a slot apart).  The tiles of all
 // units form one sequence that is split evenly over persistent CTAs (one per SM), so a unit may be cut
-// across CTAs; each CTA then leaves a partial (max, sum, accumulator) and the last one to arrive at the
-// unit's counter merges them in a fixed order.  No CTA ever waits for another.
+// across CTAs; each CTA then leaves a partial (max, sum, accumulator) and a small second kernel merges the parts
+// of every cut unit in a fixed order (no counters, fences or atomics: no CTA ever waits for, or signals, another).
 // More than 128 rows per unit are handled by row blocks: a group of CTAs walks the same tiles at the
 // same time, each with its own rows, so the second read of a tile is served by L2.
 //
 // Per CTA (12 warps):
-//   warp 0, 11  stage K and V into two 4-deep rings of 4-slot stages: one TMA box per page and tensor, 128-byte
-//               swizzle; ragged page and tree tokens by plain loads with zero fill
+//   warp 0, 11  stage K and V into two rings of 4-slot stages (4 or 6 deep: whatever the Q buffers leave): one TMA box
+//               per page and tensor, 128-byte swizzle; ragged page and tree tokens by 16-byte asynchronous copies
+//               with zero fill
 //   warp 1      owns TMEM and issues S = Q K^T for a pair of tiles at a time (tcgen05.mma, M=128 rows, N=64 per
-//               tile, 8-row groups 4096 B apart) into two of four S buffers, as far ahead as the rings allow
-//   warp 2      issues O += P V (P from shared memory, V as an MN-major operand)
-//   warps 3..10 softmax, two groups of four warps on alternate tiles, one thread per row (TMEM lane):
-//               tcgen05.ld of the row's scores, mask in registers, online softmax without any shuffle, P written
-//               as bf16 into the group's swizzled A-operand buffer; each group keeps its own accumulator O in
-//               TMEM (rescaled only when a row's maximum grew by more than 2^8: the stale offset is carried
-//               exactly through the sum and the division) and the two are merged like split-KV partials
+//               tile, 8-row groups one slot apart) into two of four S buffers, as far ahead as rings and buffers allow;
+//               Q is double-buffered, so it runs on into the next unit while the softmax warps finish this one
+//   warp 2      issues O += P V (P as the A operand from tensor memory, V as an MN-major operand from shared memory)
+//   warps 3..10 softmax, two groups of four warps on alternate tiles, one thread per row (TMEM lane): a first pass
+//               over the row's scores for the maximum, a second for P = exp2(s*c - offset), written as bf16 over the
+//               first half of the same S buffer (the buffer is released by the P V that reads it); no shuffles, no
+//               shared memory; each group keeps its own accumulator O in TMEM (rescaled only when a row's maximum
+//               grew by more than 2^8: the stale offset is carried exactly through the sum and the division) and the
+//               two are merged like split-KV partials; they also stage the next unit's Q a unit ahead
 // Every ring index and mbarrier parity is a function of one per-CTA tile counter, identical in all roles.
 // Every mbarrier wait is bounded; on expiry the kernel records MIRROR_DEV_TIMEOUT and unwinds.
 #include <math.h>
@@ -47,7 +50,6 @@ constexpr int kRows = 128;                          // UMMA M: rows per row bloc
 constexpr int kMaxBatch = 1024;
 constexpr int kMaxStages = 8;                       // ring depths are template parameters (even: tiles are staged in pairs)
 constexpr int kSBufs = 4;                           // S buffers in TMEM (power of two)
-constexpr int kMergeWarps = 8;
 constexpr float kRescaleLog2 = 8.0f;
 constexpr int kTmemCols = 512;                      // S0..S3 (64 columns each; P overwrites the first 32 of its S) | O of group 0 | O of group 1
 constexpr int kTmemO = kSBufs * kTileTok;
@@ -75,8 +77,8 @@ struct AttnParams {
     __nv_bfloat16* out;
     float* lse_out;
     float* partial;                       // [grid][2][D+4][128]
-    int* ticket;                          // [units][n_rb][kMergeWarps]
     int* status;
+    int timing_exit;                      // developer aid: leave the kernel early (1: at entry, 2: after the prologue)
     long long* timing;                    // developer aid (MIRROR_ATTN_TIMING builds): per-role cycle counters of one CTA
 };
 
@@ -186,11 +188,6 @@ struct Cfg {
     }
 };
 
-struct PendingUnit {                      // a unit whose partial this CTA has left; arrival and merge come at the CTA's end
-    int layer, b, g, ga, gb;
-    long long unit_first_tile;
-};
-
 // Visibility of 32 score columns (four slots from sl0, eight tokens from tr0 of each: column c is token tr0 + c%8 of
 // slot sl0 + c/8) for a row whose visible tree tokens are the bits of (anc0, anc1).  Kept out of line and rolled:
 // it runs for a unit's last tiles only.
@@ -233,11 +230,42 @@ __device__ __noinline__ Segment make_segment(long long x, long long x_end, const
     return s;
 }
 
+// How the tile sequence is cut into one range per CTA group.
+struct Partition {
+    long long tiles_per_layer, total_tiles, total_pairs, snap_tol;
+    int n_groups;
+};
+__device__ __forceinline__ Partition make_partition(const AttnParams& p, const int* cumT) {
+    Partition q;
+    q.tiles_per_layer = (long long)p.Hkv * cumT[p.B];
+    q.total_tiles = q.tiles_per_layer * p.L;
+    // CTA groups own whole pairs of tiles; never more groups than pairs, so that every group's range is non-empty
+    q.total_pairs = q.total_tiles / 2;
+    q.n_groups = (int)min((long long)p.n_groups, q.total_pairs);
+    // A boundary that falls within snap_tol tiles (a cut costs about as much as a few tiles) of a unit boundary
+    // moves there: both neighbours then hold whole units and no partial has to be left and merged.  snap_tol is
+    // at most a quarter of the smallest even share, so boundaries stay strictly increasing.
+    q.snap_tol = q.n_groups > 0 ? min((long long)p.snap_cap, (2 * (q.total_pairs / q.n_groups)) / 4) : 0;
+    return q;
+}
+__device__ __noinline__ long long group_begin(const Partition& q, int g, const AttnParams& p, const int* cumT) {
+    if (g <= 0) return 0;
+    if (g >= q.n_groups) return q.total_tiles;
+    const long long e = 2 * (q.total_pairs * g / q.n_groups);
+    if (q.snap_tol == 0) return e;
+    const UnitPos u = locate(e, p, cumT, q.tiles_per_layer);
+    const long long lo = u.unit_first_tile, hi = lo + u.tiles_in_unit;
+    const long long best = (e - lo <= hi - e) ? lo : hi;
+    const long long dist = best > e ? best - e : e - best;
+    return dist <= q.snap_tol ? best : e;
+}
+
 template <int D, int KS, int VS>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                    const __grid_constant__ AttnTree tree, const AttnParams p) {
     using C = Cfg<D>;
+    constexpr int KR = KS;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* sQ = smem;                                             // [2]: the units a CTA walks alternate
@@ -252,11 +280,14 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int group = blockIdx.x / p.n_rb, rb = blockIdx.x % p.n_rb;
 #ifdef MIRROR_ATTN_TIMING
-#define T_STAMP(i) do { if (p.timing && tid == 0) { unsigned long long g__; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g__)); p.timing[64 + blockIdx.x * 4 + (i)] = (long long)g__; } } while (0)
+#define T_STAMP(i) do { if (p.timing && tid == 0) { unsigned long long g__; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g__) :: "memory"); p.timing[64 + blockIdx.x * 4 + (i)] = (long long)g__; } } while (0)
 #else
 #define T_STAMP(i) do { } while (0)
 #endif
     T_STAMP(0);
+#ifdef MIRROR_ATTN_TIMING
+    if (p.timing_exit == 1) return;
+#endif
 
     // ---- prologue ---------------------------------------------------------------------------------
     for (int b = tid; b < p.B; b += kThreads) {
@@ -299,33 +330,22 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     }
     __syncthreads();
     const uint32_t tmem_base = ctrl->tmem_base;
-    const long long tiles_per_layer = (long long)p.Hkv * cumT[p.B];
-    const long long total_tiles = tiles_per_layer * p.L;
-    // CTA groups own whole pairs of tiles; never more groups than pairs, so that every group's range is non-empty
-    // and boundaries are distinct
-    const long long total_pairs = total_tiles / 2;
-    const int n_groups = (int)min((long long)p.n_groups, total_pairs);
-    // A boundary that falls within snap_tol tiles (a cut costs about as much as a dozen tiles) of a unit boundary moves there: both neighbours then hold whole
-    // units and no partial has to be left and merged.  snap_tol is less than a quarter of the smallest even share,
-    // so boundaries stay strictly increasing and every group's range is non-empty.
-    const long long snap_tol = min((long long)p.snap_cap, (2 * (total_pairs / n_groups)) / 4);
-    auto group_begin = [&](int g) -> long long {
-        if (g <= 0) return 0;
-        if (g >= n_groups) return total_tiles;
-        const long long e = 2 * (total_pairs * g / n_groups);
-        if (snap_tol == 0) return e;
-        const UnitPos u = locate(e, p, cumT, tiles_per_layer);
-        const long long lo = u.unit_first_tile, hi = lo + u.tiles_in_unit;
-        const long long best = (e - lo <= hi - e) ? lo : hi;
-        const long long dist = best > e ? best - e : e - best;
-        return dist <= snap_tol ? best : e;
-    };
+    const Partition part = make_partition(p, cumT);
+    const long long tiles_per_layer = part.tiles_per_layer, total_tiles = part.total_tiles;
+    const int n_groups = part.n_groups;
     const bool fits = total_tiles < (1ll << 31);
     if (!fits && tid == 0) dev_check(p, 600);
-    const long long x_begin = (fits && group < n_groups) ? group_begin(group) : 0;
-    const long long x_end = (fits && group < n_groups) ? group_begin(group + 1) : 0;
+    const long long x_begin = (fits && group < n_groups) ? group_begin(part, group, p, cumT) : 0;
+    const long long x_end = (fits && group < n_groups) ? group_begin(part, group + 1, p, cumT) : 0;
 
     T_STAMP(1);
+#ifdef MIRROR_ATTN_TIMING
+    if (p.timing_exit == 2) {
+        __syncthreads();
+        if (warp == 1) ptx::tmem_dealloc(tmem_base, kTmemCols);
+        return;
+    }
+#endif
     if (warp == 0 || warp == kVProducerWarp) {
         // =========================================================================== producers
         // warp 0 stages K, the last warp stages V: a warp issues its TMA boxes one after the other, so two
@@ -368,8 +388,8 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 #ifdef MIRROR_ATTN_TIMING
                 tm__ = T_NOW();
 #endif
-                const int st = vrole ? (int)(it % VS) : (int)(it % KS);
-                const uint32_t ph = (vrole ? it / VS : it / KS) & 1;
+                const int st = vrole ? (int)(it % VS) : (int)(it % KR);
+                const uint32_t ph = (vrole ? it / VS : it / KR) & 1;
                 const int next_page = (t + 1 < sg.t_last) ? fetch_page(t + 1) : 0;
                 bool w = true;
                 if (lane == 0) w = !ctrl->abort && T_WAIT(w_empty, ptx::mbar_wait(&empty[st], ph ^ 1));
@@ -442,7 +462,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         if (lane == 0) T_STORE(vrole ? 32 : 16, T_NOW() - t0, w_empty, (long long)it, p_pre, p_fill, p_issue);
         if (!ok && lane == 0) {
             // let copies already in flight land before the CTA's shared memory goes away
-            const uint32_t ns = vrole ? VS : KS;
+            const uint32_t ns = vrole ? VS : KR;
             const uint32_t back = it < ns ? it : ns;
             for (uint32_t j = it - back; j < it; ++j)
                 ptx::mbar_wait(&full[j % ns], (j / ns) & 1, 200000000ll);
@@ -460,7 +480,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             long long x = x_begin;
             T_DECL(w_q = 0, w_k = 0, w_s = 0, t0 = T_NOW());
 #ifdef MIRROR_ATTN_TIMING
-            unsigned long long g0; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g0));
+            unsigned long long g0; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g0) :: "memory");
 #endif
             while (x < x_end && ok) {
                 const Segment sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
@@ -472,12 +492,12 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     bool ready = !ctrl->abort;
                     for (int j = 0; j < 2 && ready; ++j) {
                         const uint32_t i2 = it + j;
-                        ready = T_WAIT(w_k, ptx::mbar_wait(&ctrl->k_full[i2 % KS], (i2 / KS) & 1)) &&
+                        ready = T_WAIT(w_k, ptx::mbar_wait(&ctrl->k_full[i2 % KR], (i2 / KR) & 1)) &&
                                 T_WAIT(w_s, ptx::mbar_wait(&ctrl->s_free[i2 & (kSBufs - 1)], ((i2 / kSBufs) & 1) ^ 1));
                     }
                     if (!ready) { timeout(p, ctrl, 21); ok = false; break; }
                     ptx::tc_fence_after();
-                    const int st = it % KS, sb = it & (kSBufs - 1);
+                    const int st = it % KR, sb = it & (kSBufs - 1);
                     // slots scored: those that exist, rounded up to even (N must be a multiple of 16)
                     const int ne = min(2 * kStageSlots, (sg.slots_all - t * kStageSlots + 1) & ~1);
                     const uint32_t idesc = ptx::umma_idesc_bf16(kRows, ne * 8);
@@ -500,7 +520,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             }
             T_STORE(0, T_NOW() - t0, w_q, w_k, w_s, (long long)it);
 #ifdef MIRROR_ATTN_TIMING
-            { unsigned long long g1; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g1)); T_STORE(48, (long long)(g1 - g0)); }
+            { unsigned long long g1; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g1) :: "memory"); T_STORE(48, (long long)(g1 - g0)); }
 #endif
         }
     } else if (warp == 2) {
@@ -652,8 +672,6 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         };
 
         uint32_t seg = 0;                                          // parts walked so far: Q buffer = seg & 1
-        PendingUnit pend0, pend1;                                  // units cut across CTAs: at most the first and the last part
-        int n_pend = 0;
         if (x < x_end) {
             sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
             stage_q(sg.u, 0);
@@ -732,6 +750,10 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 T_MARK(s_exp);
                 l_run += sum;
                 first = false;
+                // Keep in step with this group's P V barrier: a parity wait can only tell apart two consecutive
+                // phases, so a warp must never fall two completions behind it.  The P V of two tiles ago has
+                // normally long completed here.
+                if (it >= 2 && (ctrl->abort || !T_WAIT(w_pv, ptx::mbar_wait(&ctrl->pv_done[grp], ((it - 2) >> 1) & 1)))) { timeout(p, ctrl, 34); ok = false; break; }
                 // P is in tensor memory (and any O rescale too): the P V of this tile may go
                 ptx::tc_fence_before();
                 __syncwarp();
@@ -745,8 +767,9 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 #endif
 
             // (This part's Q buffer is overwritten at the start of the next part.  Every Q K^T that reads it has
-            // completed by then: both groups wait below for the P V of the part's last tile, which follows that
-            // tile's P, its S and so its Q K^T.  Waiting here on the last tile's s_full instead would be wrong: the
+            // completed by then: below, each group waits for the P V of its own last tile and then meets the other;
+            // the P V of the part's last tile follows that tile's P, its S and so its Q K^T.  Waiting here on the
+            // last tile's s_full instead would be wrong: the
             // issuer can run on into the next unit, and a second completion of that barrier would make a late
             // waiter's parity match the wrong phase.)
             if (q_pending) { q_ready((seg + 1) & 1); q_pending = false; }
@@ -757,10 +780,16 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             float* xc = xch + (size_t)row_in_blk * 4;              // [row][group][max, sum]
             xc[grp * 2] = m_used;
             xc[grp * 2 + 1] = l_run;
+            // each group waits for the P V of its own last tile (the barrier it has kept in step with), then the
+            // groups meet: past the meeting both accumulators are complete
+            {
+                const uint32_t j_last = (((it - 1) & 1) == (uint32_t)grp) ? it - 1 : it - 2;
+                if (ctrl->abort || !T_WAIT(w_end, ptx::mbar_wait(&ctrl->pv_done[grp], (j_last >> 1) & 1))) { timeout(p, ctrl, 32); ok = false; break; }
+            }
+            ptx::tc_fence_before();
             if (!T_WAIT(s_ld, pair_sync())) { timeout(p, ctrl, 35); ok = false; break; }
-            const float m_a = xc[0], l_a = xc[1], m_b = xc[2], l_b = xc[3];
-            if (ctrl->abort || !T_WAIT(w_end, ptx::mbar_wait(&ctrl->pv_done[(it - 1) & 1], ((it - 1) >> 1) & 1))) { timeout(p, ctrl, 32); ok = false; break; }
             ptx::tc_fence_after();
+            const float m_a = xc[0], l_a = xc[1], m_b = xc[2], l_b = xc[3];
 #ifdef MIRROR_ATTN_TIMING
             te = T_NOW();
 #endif
@@ -776,13 +805,6 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             if (warp_has_rows) {
                 __nv_bfloat16* orow = p.out + ((((size_t)u.layer * p.B + u.b) * p.n + node) * (size_t)p.Hq + u.g * p.G + hl) * D + grp * kDH;
                 float* lse_ptr = (p.lse_out && grp == 0) ? p.lse_out + (((size_t)u.layer * p.B + u.b) * p.Hq + u.g * p.G + hl) * p.n + node : nullptr;
-                // groups ga..gb cover this unit (group g owns tiles [total*g/n_groups, total*(g+1)/n_groups))
-                int ga = group, gb = group;
-                if (!whole_unit) {
-                    while (ga > 0 && group_begin(ga) > u.unit_first_tile) --ga;
-                    const long long unit_last = u.unit_first_tile + u.tiles_in_unit - 1;
-                    while (gb + 1 < n_groups && group_begin(gb + 1) <= unit_last) ++gb;
-                }
                 const int slot = (sg.t_first > 0) ? 0 : 1;       // a unit that began before this CTA's range uses slot 0
                 // partial layout [column][row]: a warp's store of one column is one contiguous 128-byte line;
                 // each warp of a pair leaves its own copy of (max, sum) so that its columns stand alone
@@ -831,18 +853,10 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 if (whole_unit) {
                     if (lse_ptr && row_ok) *lse_ptr = M * p.scale + logf(Lsum);
                 } else {
-                    // ---- the unit is cut across CTA groups: the partial is left now; the arrival at the unit's
-                    //      counter (and the merge, for the last one to arrive) waits until this CTA has walked all its
-                    //      tiles, so that neither the fence nor the merge stalls the tiles that follow
+                    // ---- the unit is cut across CTA groups: this part's (max, sum, accumulator) is left for the merge
+                    //      kernel that follows; nothing here waits for another CTA
                     my[(size_t)(D + 2 * grp) * kRows] = M;
                     my[(size_t)(D + 2 * grp + 1) * kRows] = Lsum;
-                    if (n_pend >= 2) {
-                        dev_check(p, 500);                       // a CTA's range cuts at most two units
-                    } else {
-                        PendingUnit& q = (n_pend == 0) ? pend0 : pend1;
-                        q.layer = u.layer; q.b = u.b; q.g = u.g; q.ga = ga; q.gb = gb; q.unit_first_tile = u.unit_first_tile;
-                        ++n_pend;
-                    }
                 }
             } else {
                 ptx::tc_fence_before();
@@ -856,89 +870,111 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             if (!T_WAIT(s_free, pair_sync())) { timeout(p, ctrl, 36); ok = false; break; }
             if (has_next) sg = sg_next;
         }
-        // ---- units that this CTA shares with others: arrive, and merge where this is the last arrival -----------
-        if (ok && warp_has_rows && n_pend > 0) {
-            __threadfence();
-            __syncwarp();
-            for (int i = 0; i < n_pend; ++i) {
-                const PendingUnit q = (i == 0) ? pend0 : pend1;
-                const int parts = q.gb - q.ga + 1;
-                const size_t unit_idx = ((size_t)q.layer * p.B + q.b) * p.Hkv + q.g;
-                int* tk = p.ticket + (unit_idx * p.n_rb + rb) * kMergeWarps + (grp * 4 + w4);
-                int arrived = 0;
-                if (lane == 0) arrived = atomicAdd(tk, 1);
-                arrived = __shfl_sync(0xffffffffu, arrived, 0);
-                if (arrived != parts - 1) continue;
-                __threadfence();
-                if (lane == 0) *tk = 0;                          // ready for the next launch
-                __nv_bfloat16* orow = p.out + ((((size_t)q.layer * p.B + q.b) * p.n + node) * (size_t)p.Hq + q.g * p.G + hl) * D + grp * kDH;
-                float* lse_ptr = (p.lse_out && grp == 0) ? p.lse_out + (((size_t)q.layer * p.B + q.b) * p.Hq + q.g * p.G + hl) * p.n + node : nullptr;
-                auto part_of = [&](int gsrc) -> const float* {
-                    const int sslot = (group_begin(gsrc) > q.unit_first_tile) ? 0 : 1;
-                    return p.partial + ((size_t)(gsrc * p.n_rb + rb) * 2 + sslot) * kRowW * kRows + row_in_blk;
-                };
-                // merge in group order; (max, sum) of the first parts stay in registers
-                constexpr int kKeep = 4;
-                float pmv[kKeep], plv[kKeep];
-                float Mm = -INFINITY;
-#pragma unroll
-                for (int k = 0; k < kKeep; ++k) {
-                    pmv[k] = -INFINITY; plv[k] = 0.f;
-                    if (k < parts) {
-                        const float* src = part_of(q.ga + k);
-                        pmv[k] = __ldcg(src + (size_t)(D + 2 * grp) * kRows);
-                        plv[k] = __ldcg(src + (size_t)(D + 2 * grp + 1) * kRows);
-                    }
-                }
-#pragma unroll
-                for (int k = 0; k < kKeep; ++k) Mm = fmaxf(Mm, pmv[k]);
-                for (int k = kKeep; k < parts; ++k) Mm = fmaxf(Mm, __ldcg(part_of(q.ga + k) + (size_t)(D + 2 * grp) * kRows));
-                auto weight = [&](float pm) -> float { return (pm == -INFINITY) ? 0.f : exp2f((pm - Mm) * p.scale_log2e); };
-                float Lm = 0.f;
-#pragma unroll
-                for (int k = 0; k < kKeep; ++k) Lm += weight(pmv[k]) * plv[k];
-                for (int k = kKeep; k < parts; ++k) {
-                    const float* src = part_of(q.ga + k);
-                    Lm += weight(__ldcg(src + (size_t)(D + 2 * grp) * kRows)) * __ldcg(src + (size_t)(D + 2 * grp + 1) * kRows);
-                }
-                const float invm = 1.f / Lm;
-#pragma unroll 1
-                for (int c4 = 0; c4 < kDH / 32; ++c4) {
-                    float acc[32];
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) acc[j] = 0.f;
-                    for (int k = 0; k < parts; ++k) {
-                        const float* src = part_of(q.ga + k);
-                        const float wgt = weight(__ldcg(src + (size_t)(D + 2 * grp) * kRows));
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) acc[j] = fmaf(wgt, __ldcg(src + (size_t)(grp * kDH + c4 * 32 + j) * kRows), acc[j]);
-                    }
-                    if (row_ok) {
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            uint4 v;
-                            v.x = pack_bf16(acc[j * 8 + 0] * invm, acc[j * 8 + 1] * invm);
-                            v.y = pack_bf16(acc[j * 8 + 2] * invm, acc[j * 8 + 3] * invm);
-                            v.z = pack_bf16(acc[j * 8 + 4] * invm, acc[j * 8 + 5] * invm);
-                            v.w = pack_bf16(acc[j * 8 + 6] * invm, acc[j * 8 + 7] * invm);
-                            *reinterpret_cast<uint4*>(orow + c4 * 32 + j * 8) = v;
-                        }
-                    }
-                }
-                if (lse_ptr && row_ok) *lse_ptr = Mm * p.scale + logf(Lm);
-            }
-        }
         asm volatile("cp.async.wait_all;" ::: "memory");      // (only an aborted run can still have copies in flight here)
         if (warp == 4 && lane == 0) { T_STORE(8, T_NOW() - t0, w_sf, w_pv, w_end, t_epi, t_q, (long long)it); T_STORE(40, s_ld, s_free, s_max, s_xch, s_exp, s_fin); T_STORE(52, t_init, t_loop, t_max, t_ld1); }
     }
 
+#ifdef MIRROR_ATTN_TIMING
+#define T_G(i) do { if (p.timing && blockIdx.x == 5) { unsigned long long g__; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g__) :: "memory"); p.timing[680 + (i)] = (long long)g__; } } while (0)
+#else
+#define T_G(i) do { } while (0)
+#endif
+    if (lane == 0) T_G(warp);
+    if (warp == 1 && lane == 1) T_G(12);
     ptx::tc_fence_before();
     __syncthreads();
     T_STAMP(2);
+    if (lane == 0) T_G(16 + warp);
+    if (lane == 0 && warp == 1) T_G(13);
     if (warp == 1) {
         ptx::tc_fence_after();
+        if (lane == 0) T_G(14);
         ptx::tmem_dealloc(tmem_base, kTmemCols);
+        if (lane == 0) T_G(15);
+#ifdef MIRROR_ATTN_TIMING
+        if (p.timing && lane == 0) { unsigned long long g__; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g__) :: "memory"); p.timing[64 + blockIdx.x * 4 + 3] = (long long)g__; }
+#endif
     }
+}
+
+// Merge of the units that the partition cut across CTA groups.  One block per (inner boundary, row block): the
+// block whose boundary is the first one inside a unit combines all of that unit's parts, in group order, from the
+// (max, sum, accumulator) records the attention kernel left, exactly like split-KV partials.  Blocks whose boundary
+// coincides with a unit boundary, or is not the first inside its unit, have nothing to do.
+constexpr int kMergeThreads = 512;        // 128 rows x 4 column quarters
+template <int D>
+__global__ void __launch_bounds__(kMergeThreads) attn_merge_kernel(const AttnParams p) {
+    __shared__ int cumT[kMaxBatch + 1];
+    __shared__ int s_len[kMaxBatch];
+    const int tid = threadIdx.x;
+    for (int b = tid; b < p.B; b += kMergeThreads) {
+        const int len = p.prefix_len[b];
+        s_len[b] = len < 0 ? 0 : (len > p.max_pages * kSlotTok ? p.max_pages * kSlotTok : len);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int acc = 0;
+        cumT[0] = 0;
+        for (int b = 0; b < p.B; ++b) {
+            const int slots = (s_len[b] + kSlotTok - 1) / kSlotTok + p.tree_slots;
+            acc += 2 * ((slots + 2 * kStageSlots - 1) / (2 * kStageSlots));
+            cumT[b + 1] = acc;
+        }
+    }
+    __syncthreads();
+    const Partition part = make_partition(p, cumT);
+    const int g = blockIdx.x + 1, rb = blockIdx.y;
+    if (g >= part.n_groups || part.total_tiles >= (1ll << 31)) return;
+    const long long x = group_begin(part, g, p, cumT);
+    const UnitPos u = locate(x, p, cumT, part.tiles_per_layer);
+    if (u.tile_in_unit == 0) return;                                            // the boundary is a unit boundary
+    if (group_begin(part, g - 1, p, cumT) > u.unit_first_tile) return;          // an earlier boundary cuts this unit too
+    const int ga = g - 1;
+    int gb = g;
+    const long long unit_last = u.unit_first_tile + u.tiles_in_unit - 1;
+    while (gb + 1 < part.n_groups && group_begin(part, gb + 1, p, cumT) <= unit_last) ++gb;
+    const int parts = gb - ga + 1;
+
+    constexpr int kRowW = D + 4;
+    constexpr int kQ = D / 4;                                                   // columns per thread
+    const int row = tid & (kRows - 1), cq = tid >> 7;
+    const int rb_row0 = rb * p.rows_per_rb;
+    const int rb_rows = min(p.rows_per_rb, p.rows - rb_row0);
+    if (row >= rb_rows) return;
+    const int r_abs = rb_row0 + row, node = r_abs / p.G, hl = r_abs % p.G;
+    // group ga holds the unit's first tile (its record is in slot 1), the later groups began inside the unit (slot 0)
+    auto part_of = [&](int k) -> const float* {
+        return p.partial + ((size_t)((ga + k) * p.n_rb + rb) * 2 + (k == 0 ? 1 : 0)) * kRowW * kRows + row;
+    };
+    float Mm = -INFINITY;
+#pragma unroll 4
+    for (int k = 0; k < parts; ++k) Mm = fmaxf(Mm, __ldcg(part_of(k) + (size_t)D * kRows));
+    float Lm = 0.f;
+    float acc[kQ];
+#pragma unroll
+    for (int j = 0; j < kQ; ++j) acc[j] = 0.f;
+#pragma unroll 2
+    for (int k = 0; k < parts; ++k) {
+        const float* src = part_of(k);
+        const float pm = __ldcg(src + (size_t)D * kRows);
+        const float wgt = (pm == -INFINITY) ? 0.f : exp2f((pm - Mm) * p.scale_log2e);
+        Lm = fmaf(wgt, __ldcg(src + (size_t)(D + 1) * kRows), Lm);
+#pragma unroll
+        for (int j = 0; j < kQ; ++j) acc[j] = fmaf(wgt, __ldcg(src + (size_t)(cq * kQ + j) * kRows), acc[j]);
+    }
+    const float inv = 1.f / Lm;
+    __nv_bfloat16* orow = p.out + ((((size_t)u.layer * p.B + u.b) * p.n + node) * (size_t)p.Hq + u.g * p.G + hl) * D + cq * kQ;
+#pragma unroll
+    for (int j = 0; j < kQ / 8; ++j) {
+        uint4 v;
+        v.x = pack_bf16(acc[j * 8 + 0] * inv, acc[j * 8 + 1] * inv);
+        v.y = pack_bf16(acc[j * 8 + 2] * inv, acc[j * 8 + 3] * inv);
+        v.z = pack_bf16(acc[j * 8 + 4] * inv, acc[j * 8 + 5] * inv);
+        v.w = pack_bf16(acc[j * 8 + 6] * inv, acc[j * 8 + 7] * inv);
+        *reinterpret_cast<uint4*>(orow + j * 8) = v;
+    }
+    if (p.lse_out && cq == 0)
+        p.lse_out[(((size_t)u.layer * p.B + u.b) * p.Hq + u.g * p.G + hl) * p.n + node] = Mm * p.scale + logf(Lm);
 }
 
 }  // namespace
@@ -954,7 +990,7 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
     p.rows_per_rb = (p.rows + p.n_rb - 1) / p.n_rb;
     p.n_groups = ctx->num_sms / p.n_rb;
     if (p.n_groups < 1) return MIRROR_ERR_SHAPE;
-    p.snap_cap = 12;
+    p.snap_cap = 4;
     if (const char* e = getenv("MIRROR_ATTN_SNAP")) { p.snap_cap = atoi(e); if (p.snap_cap < 0) p.snap_cap = 0; }
     p.max_pages = kv->max_pages_per_req; p.num_pages = kv->num_pages;
     const int64_t page_elems = (int64_t)Hkv * kSlotTok * D;
@@ -962,6 +998,7 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
     p.layer_pages = (int)(kv->layer_stride / page_elems);
     p.tree_slots = (p.n + kSlotTok - 1) / kSlotTok;
     p.q_half_bytes = ((p.rows_per_rb + 7) / 8) * 8 * 128;
+    if (getenv("MIRROR_ATTN_QFULL")) p.q_half_bytes = kRows * 128;
     p.scale = ctx->scale;
     p.scale_log2e = ctx->scale * 1.4426950408889634f;
     p.page_table = kv->page_table; p.prefix_len = kv->prefix_len;
@@ -969,12 +1006,14 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
     p.k_pool = (const __nv_bfloat16*)kv->k_pool; p.v_pool = (const __nv_bfloat16*)kv->v_pool;
     p.k_new = (const __nv_bfloat16*)k_new; p.v_new = (const __nv_bfloat16*)v_new;
     p.out = (__nv_bfloat16*)out; p.lse_out = lse_out;
-    p.partial = partial_ws; p.ticket = ticket_ws; p.status = ctx->d_status;
+    p.partial = partial_ws; (void)ticket_ws; p.status = ctx->d_status;
     p.timing = nullptr;
+    p.timing_exit = 0;
 #ifdef MIRROR_ATTN_TIMING
     if (const char* e = getenv("MIRROR_ATTN_TIMING_PTR")) p.timing = (long long*)strtoull(e, nullptr, 0);
+    if (const char* e = getenv("MIRROR_ATTN_EXIT")) p.timing_exit = atoi(e);
 #endif
-    if ((size_t)p.L * p.B * Hkv * p.n_rb * kMergeWarps > ticket_ints) return MIRROR_ERR_WORKSPACE;
+    (void)ticket_ints;
     if (p.B > kMaxBatch) return MIRROR_ERR_SHAPE;
 
     AttnTree at;
@@ -1019,5 +1058,13 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
     if (lst != MIRROR_OK) return lst;
     ctx->launches += 1;
     MIRROR_CUDA_OK(cudaGetLastError());
+    if (p.n_groups > 1) {
+        // which units the partition cut is only known on the device (it depends on the prefix lengths)
+        const dim3 mgrid((unsigned)(p.n_groups - 1), (unsigned)p.n_rb);
+        if (D == 128) attn_merge_kernel<128><<<mgrid, kMergeThreads, 0, stream>>>(p);
+        else attn_merge_kernel<64><<<mgrid, kMergeThreads, 0, stream>>>(p);
+        ctx->launches += 1;
+        MIRROR_CUDA_OK(cudaGetLastError());
+    }
     return MIRROR_OK;
 }

@@ -119,6 +119,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
+#ifndef MIRROR_PARK_NS
+#define MIRROR_PARK_NS 20000u
+#endif
 // try_wait that lets the hardware park the thread (up to `ns` nanoseconds) until the phase completes, instead of
 // returning at once: a hot spin on try_wait issues a shared-memory operation every few cycles and starves the
 // warps that share the SM's shared-memory pipeline.
@@ -142,7 +145,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, long l
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
-        if (mbar_try_wait_park(bar, parity, 20000u)) return true;
+        if (mbar_try_wait_park(bar, parity, MIRROR_PARK_NS)) return true;
         if (clock64() - t0 > limit_cycles) return false;
     }
 }
