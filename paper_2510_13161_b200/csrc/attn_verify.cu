@@ -5,9 +5,10 @@
 // Work decomposition.  A "unit" is (layer, request, KV head): all G = Hq/Hkv query heads of all n tree
 // nodes (G*n rows) share that head's K/V stream, so one CTA owning the unit's rows reads each K/V byte
 // once from HBM and reuses it from shared memory for every row (the GQA / tree sharing).  A unit's keys
-// are cut into 16-token slots (one KV page, or 16 tree tokens); eight slots form a pair of 64-token tiles: tile 0
-// of the pair holds the first eight tokens of each of the eight slots, tile 1 the second eight (so that a whole
-// page is one TMA box and still a legal UMMA operand: the 8-row groups of one tile are a slot apart).  The tiles of all
+// are cut into 16-token slots (one KV page, or 16 tree tokens); four slots form a 64-token tile and a ring stage.  A
+// slot lands in shared memory as [token / 8][64-column half][token % 8][128 B] (one 5-D TMA box per page), so that the
+// 8-token groups of a half are evenly spaced across slots and stages: two consecutive stages are one K-major UMMA
+// operand of up to 128 tokens in token order, and each slot is one MN-major 16-token P V step.  The tiles of all
 // units form one sequence that is split evenly over persistent CTAs (one per SM), so a unit may be cut
 // across CTAs; each CTA then leaves a partial (max, sum, accumulator) and a small second kernel merges the parts
 // of every cut unit in a fixed order (no counters, fences or atomics: no CTA ever waits for, or signals, another).
@@ -18,8 +19,8 @@
 //   warp 0, 11  stage K and V into two rings of 4-slot stages (4 or 6 deep: whatever the Q buffers leave): one TMA box
 //               per page and tensor, 128-byte swizzle; ragged page and tree tokens by 16-byte asynchronous copies
 //               with zero fill
-//   warp 1      owns TMEM and issues S = Q K^T for a pair of tiles at a time (tcgen05.mma, M=128 rows, N=64 per
-//               tile, 8-row groups one slot apart) into two of four S buffers, as far ahead as rings and buffers allow;
+//   warp 1      owns TMEM and issues S = Q K^T for a pair of tiles at a time (tcgen05.mma, M=128 rows, N up to 128
+//               tokens, d/16 instructions) into two adjacent of four S buffers, as far ahead as rings and buffers allow;
 //               Q is double-buffered, so it runs on into the next unit while the softmax warps finish this one
 //   warp 2      issues O += P V (P as the A operand from tensor memory, V as an MN-major operand from shared memory)
 //   warps 3..10 softmax, two groups of four warps on alternate tiles, one thread per row (TMEM lane): a first pass
@@ -133,6 +134,13 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // Shared-memory operand tiles are [64-column half][row][128 B] with the 128-byte swizzle: the 16-byte chunk
 // index is XORed with (row % 8).  A half of Q or P holds 128 rows (16 KB), a half of a K/V stage 64 tokens (8 KB).
 constexpr int kStageSlots = 4;                      // slots per ring stage
+// A K/V slot (16 tokens of one head) is [token / 8][64-column half][token % 8][128 B]: the 8-token groups of one half
+// are 1024 * (d / 64) bytes apart, uniformly across the slots of a ring, which is the 8-row-group stride (SBO) of the
+// K-major Q K^T operand over up to 128 tokens and, with the halves 1024 B apart (LBO), the MN-major P V operand.
+template <int D>
+__device__ __forceinline__ uint32_t kv_slot_off(int tok, int chunk) {                 // chunk: 16-byte column chunk
+    return (uint32_t)((tok >> 3) * (D / 64) * 1024 + (chunk >> 3) * 1024 + (tok & 7) * 128 + (((chunk & 7) ^ (tok & 7)) << 4));
+}
 __device__ __forceinline__ uint32_t tile_off(int row, int chunk, int half_bytes) {   // chunk: 16-byte column chunk
     return (uint32_t)((chunk >> 3) * half_bytes + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
 }
@@ -176,7 +184,8 @@ __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.
 template <int D>
 struct Cfg {
     static constexpr int kHalves = D / 64;
-    static constexpr int kSlotBytes = kHalves * kSlotTok * 128;    // one slot of K or V: [half][16 tokens][128 B] = one TMA box
+    static constexpr int kSlotBytes = kHalves * kSlotTok * 128;    // one slot of K or V (see kv_slot_off) = one TMA box
+    static constexpr int kGroupStride = kHalves * 1024;            // between the 8-token groups of one half
     static constexpr int kStageBytes = kStageSlots * kSlotBytes;   // one K (or V) stage: 4 slots; stages are contiguous
     static constexpr size_t kSmemFixed = 512 /*ctrl*/ + 2 * 2 * kRows * 4 /*pair exchange*/ + (2 * kMaxBatch + 2) * 4 + 1024 /*align*/;
     // Shared memory: two Q buffers sized by the rows a CTA really has (the UMMA reads 128 rows per half and
@@ -188,14 +197,13 @@ struct Cfg {
     }
 };
 
-// Visibility of 32 score columns (four slots from sl0, eight tokens from tr0 of each: column c is token tr0 + c%8 of
-// slot sl0 + c/8) for a row whose visible tree tokens are the bits of (anc0, anc1).  Kept out of line and rolled:
-// it runs for a unit's last tiles only.
-__device__ __noinline__ uint32_t chunk_mask(int sl0, int tr0, int pages_full, int pages_all, int slots_all, int len,
+// Visibility of 32 score columns (the 16 tokens of slots sl0 and sl0 + 1) for a row whose visible tree tokens are the
+// bits of (anc0, anc1).  Kept out of line and rolled: it runs for a unit's last tiles only.
+__device__ __noinline__ uint32_t chunk_mask(int sl0, int pages_full, int pages_all, int slots_all, int len,
                                             unsigned long long anc0, unsigned long long anc1) {
     uint32_t cm = 0;
 #pragma unroll 1
-    for (int jj = 0; jj < 4; ++jj) {
+    for (int jj = 0; jj < 2; ++jj) {
         const int sl = sl0 + jj;
         uint32_t bits = 0;
         if (sl < pages_full) {
@@ -206,7 +214,7 @@ __device__ __noinline__ uint32_t chunk_mask(int sl0, int tr0, int pages_full, in
             const int ts = sl - pages_all;                                          // tree tokens 16*ts .. 16*ts+15
             bits = (uint32_t)(((ts < 4) ? anc0 : anc1) >> ((ts & 3) * 16)) & 0xffffu;   // ancestors-or-self (all < n)
         }
-        cm |= ((bits >> tr0) & 0xffu) << (jj * 8);
+        cm |= bits << (jj * 16);
     }
     return cm;
 }
@@ -298,7 +306,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     if (tid == 0) {
         for (int s = 0; s < kMaxStages; ++s) {
             ptx::mbar_init(&ctrl->k_full[s], 1); ptx::mbar_init(&ctrl->k_empty[s], 1);
-            ptx::mbar_init(&ctrl->v_full[s], 1); ptx::mbar_init(&ctrl->v_empty[s], 2);   // both tiles of a pair read a V stage
+            ptx::mbar_init(&ctrl->v_full[s], 1); ptx::mbar_init(&ctrl->v_empty[s], 1);
         }
         for (int s = 0; s < kSBufs; ++s) {
             ptx::mbar_init(&ctrl->s_full[s], 1); ptx::mbar_init(&ctrl->s_free[s], 1);     // freed by the P V that read P from it
@@ -399,9 +407,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 const int sl0 = t * kStageSlots;
                 const int n_slots = max(0, min(kStageSlots, sg.slots_all - sl0));      // slots that exist in this stage
                 const int n_tma = max(0, min(kStageSlots, sg.pages_full - sl0));       // leading slots that are whole pages
-                // a pair of tiles is scored on an even number of slots: an odd last slot gets a zero V partner
-                const int n_fill = (vrole && (sg.slots_all & 1) && sl0 <= sg.slots_all && sg.slots_all < sl0 + kStageSlots)
-                                       ? n_slots + 1 : n_slots;
+                const int n_fill = n_slots;
                 T_MARK(p_pre);
                 if (n_tma < n_fill) {
                     // ragged page and tree tokens by asynchronous 16-byte copies (rows beyond the valid count are
@@ -415,9 +421,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                         const __nv_bfloat16* src = p.k_pool;
                         size_t row_stride = 0;
                         int valid = 0;
-                        if (sl >= sg.slots_all) {
-                            // the zero partner slot
-                        } else if (sl < sg.pages_all) {
+                        if (sl < sg.pages_all) {
                             int page = pt[sl];
                             if (page < 0 || page >= p.num_pages) { if (lane == 0) dev_check(p, 401); page = 0; }
                             src = (vrole ? p.v_pool : p.k_pool) + (((size_t)u.layer * p.layer_pages + page) * p.Hkv + u.g) * (size_t)(kSlotTok * D);
@@ -434,7 +438,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                             const int c = lane + i * 32, tr = c / (D / 8), cc = c % (D / 8);
                             const bool in = tr < valid;
                             asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
-                                         ::"r"(ptx::smem_u32(dst + j * C::kSlotBytes + tile_off(tr, cc, kSlotTok * 128))),
+                                         ::"r"(ptx::smem_u32(dst + j * C::kSlotBytes + kv_slot_off<D>(tr, cc))),
                                            "l"(in ? src + tr * row_stride + cc * 8 : p.k_pool), "r"(in ? 16u : 0u) : "memory");
                         }
                     }
@@ -451,9 +455,9 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     if (page < 0 || page >= p.num_pages) { dev_check(p, 400); page = 0; }
                     const int pg = u.layer * p.layer_pages + page;
                     if (vrole)
-                        ptx::tma_load_5d(dst + my_slot * C::kSlotBytes, &tm_v, &full[st], 0, 0, 0, u.g, pg);
+                        ptx::tma_load_5d(dst + my_slot * C::kSlotBytes, &tm_v, &full[st], 0, 0, 0, 0, pg * p.Hkv + u.g);
                     else
-                        ptx::tma_load_5d(dst + my_slot * C::kSlotBytes, &tm_k, &full[st], 0, 0, 0, u.g, pg);
+                        ptx::tma_load_5d(dst + my_slot * C::kSlotBytes, &tm_k, &full[st], 0, 0, 0, 0, pg * p.Hkv + u.g);
                 }
                 my_page = next_page;
                 T_MARK(p_issue);
@@ -472,7 +476,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         if (lane == 0) {
             // descriptor words: the high words and the Q base are constants; per pair only low words move
             const uint32_t hi_q = ptx::umma_desc_hi_sw128(1024);
-            const uint32_t hi_k = ptx::umma_desc_hi_sw128(C::kSlotBytes);     // 8-token groups of one tile are a slot apart
+            const uint32_t hi_k = ptx::umma_desc_hi_sw128(C::kGroupStride);   // 8-token groups of a half: uniform over the pair's slots
             const uint32_t q_lo = ptx::umma_desc_lo(ptx::smem_u32(sQ), 16);
             const uint32_t k_lo = ptx::umma_desc_lo(ptx::smem_u32(sK), 16);
             uint32_t it = 0, seg = 0;
@@ -498,21 +502,17 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     if (!ready) { timeout(p, ctrl, 21); ok = false; break; }
                     ptx::tc_fence_after();
                     const int st = it % KR, sb = it & (kSBufs - 1);
-                    // slots scored: those that exist, rounded up to even (N must be a multiple of 16)
-                    const int ne = min(2 * kStageSlots, (sg.slots_all - t * kStageSlots + 1) & ~1);
-                    const uint32_t idesc = ptx::umma_idesc_bf16(kRows, ne * 8);
+                    // one instruction per 16 columns of d scores both tiles: up to 128 tokens in token order
+                    const int n_sl = min(2 * kStageSlots, sg.slots_all - t * kStageSlots);
+                    const uint32_t idesc = ptx::umma_idesc_bf16(kRows, n_sl * kSlotTok);
                     const uint32_t kb = k_lo + (uint32_t)((st * C::kStageBytes) >> 4);
+                    const uint32_t d = tmem_base + (uint32_t)(sb * kTileTok);
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        // tile h of the pair: tokens 8h..8h+7 of every slot
-                        const uint32_t d = tmem_base + (uint32_t)((sb + h) * kTileTok);
-#pragma unroll
-                        for (int kk = 0; kk < D / 16; ++kk)
-                            ptx::umma_f16_lohi(d, q_seg + (uint32_t)(((kk >> 2) * p.q_half_bytes + (kk & 3) * 32) >> 4), hi_q,
-                                               kb + (uint32_t)(((kk >> 2) * (kSlotTok * 128) + h * 1024 + (kk & 3) * 32) >> 4), hi_k,
-                                               idesc, kk != 0);
-                        ptx::umma_commit(&ctrl->s_full[sb + h]);
-                    }
+                    for (int kk = 0; kk < D / 16; ++kk)
+                        ptx::umma_f16_lohi(d, q_seg + (uint32_t)(((kk >> 2) * p.q_half_bytes + (kk & 3) * 32) >> 4), hi_q,
+                                           kb + (uint32_t)(((kk >> 2) * 1024 + (kk & 3) * 32) >> 4), hi_k, idesc, kk != 0);
+                    ptx::umma_commit(&ctrl->s_full[sb]);
+                    ptx::umma_commit(&ctrl->s_full[sb + 1]);
                     ptx::umma_commit(&ctrl->k_empty[st]);
                     ptx::umma_commit(&ctrl->k_empty[st + 1]);
                 }
@@ -526,8 +526,8 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     } else if (warp == 2) {
         // =========================================================================== P V issuer
         if (lane == 0) {
-            const uint32_t hi_v = ptx::umma_desc_hi_sw128(C::kSlotBytes);                  // the two 8-token groups of a step: two slots
-            const uint32_t v_lo = ptx::umma_desc_lo(ptx::smem_u32(sV), kSlotTok * 128);   // MN-major: LBO = next 64-column atom
+            const uint32_t hi_v = ptx::umma_desc_hi_sw128(C::kGroupStride);                // the two 8-token groups of a slot
+            const uint32_t v_lo = ptx::umma_desc_lo(ptx::smem_u32(sV), 1024);             // MN-major: LBO = next 64-column atom
             const uint32_t idesc_pv = ptx::umma_idesc_bf16(kRows, D) | (1u << 16);          // B operand MN-major
             uint32_t it = 0;
             bool ok = true;
@@ -540,25 +540,21 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 if (seg > 0 && (ctrl->abort || !ptx::mbar_wait(&ctrl->o_free, (seg - 1) & 1))) { timeout(p, ctrl, 24); ok = false; break; }
                 ++seg;
                 for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
-                    // tile h of a pair reads tokens 8h..8h+7 of the pair's eight slots (both stages)
-                    const uint32_t it0 = it & ~1u;
-                    const int st0 = it0 % VS, pb = it & 1, sb = it & (kSBufs - 1);
+                    const int st = it % VS, pb = it & 1, sb = it & (kSBufs - 1);
                     if (ctrl->abort || !T_WAIT(w_p, ptx::mbar_wait(&ctrl->p_full[sb], (it / kSBufs) & 1)) ||
-                        !T_WAIT(w_v, ptx::mbar_wait(&ctrl->v_full[st0], (it0 / VS) & 1)) ||
-                        !T_WAIT(w_v, ptx::mbar_wait(&ctrl->v_full[st0 + 1], (it0 / VS) & 1))) {
+                        !T_WAIT(w_v, ptx::mbar_wait(&ctrl->v_full[st], (it / VS) & 1))) {
                         timeout(p, ctrl, 23); ok = false; break;
                     }
                     ptx::tc_fence_after();
-                    const int ne = min(2 * kStageSlots, (sg.slots_all - (t & ~1) * kStageSlots + 1) & ~1);
-                    const uint32_t vb = v_lo + (uint32_t)((st0 * C::kStageBytes + pb * 1024) >> 4);
+                    const int n_sl = max(0, min(kStageSlots, sg.slots_all - t * kStageSlots));    // one 16-token step per slot
+                    const uint32_t vb = v_lo + (uint32_t)((st * C::kStageBytes) >> 4);
                     const uint32_t pa = tmem_base + (uint32_t)(sb * kTileTok);       // P: 8 columns per 16-token step
 #pragma unroll
                     for (int k = 0; k < kStageSlots; ++k)
-                        if (2 * k < ne)
+                        if (k < n_sl)
                             ptx::umma_f16_tmem_a(tmem_base + kTmemO + (uint32_t)(pb * D), pa + (uint32_t)(k * 8),
-                                                 vb + (uint32_t)(k * (2 * C::kSlotBytes / 16)), hi_v, idesc_pv, (t >= sg.t_first + 2) || (k != 0));
-                    ptx::umma_commit(&ctrl->v_empty[st0]);
-                    ptx::umma_commit(&ctrl->v_empty[st0 + 1]);
+                                                 vb + (uint32_t)(k * (C::kSlotBytes / 16)), hi_v, idesc_pv, (t >= sg.t_first + 2) || (k != 0));
+                    ptx::umma_commit(&ctrl->v_empty[st]);
                     ptx::umma_commit(&ctrl->s_free[sb]);
                     ptx::umma_commit(&ctrl->pv_done[pb]);
                 }
@@ -716,9 +712,9 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 float mx = -INFINITY, sum = 0.f;
                 // visibility of this tile's columns for this row: all ones except in a unit's last pairs
                 uint32_t cm0 = 0xffffffffu, cm1 = 0xffffffffu;
-                if ((t & ~1) * kStageSlots + 2 * kStageSlots > sg.pages_full) {
-                    cm0 = chunk_mask((t & ~1) * kStageSlots, (t & 1) * 8, sg.pages_full, sg.pages_all, sg.slots_all, sg.len, anc0, anc1);
-                    cm1 = chunk_mask((t & ~1) * kStageSlots + 4, (t & 1) * 8, sg.pages_full, sg.pages_all, sg.slots_all, sg.len, anc0, anc1);
+                if (t * kStageSlots + kStageSlots > sg.pages_full) {
+                    cm0 = chunk_mask(t * kStageSlots, sg.pages_full, sg.pages_all, sg.slots_all, sg.len, anc0, anc1);
+                    cm1 = chunk_mask(t * kStageSlots + 2, sg.pages_full, sg.pages_all, sg.slots_all, sg.len, anc0, anc1);
                 }
                 if (warp_has_rows) mx = tile_max(sb, cm0, cm1);
                 T_MARK(t_max);
@@ -821,12 +817,12 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                             ptx::tmem_ld_wait();
                         }
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) acc[j] = has0 ? w0 * __uint_as_float(ra[j]) : 0.f;
+                        for (int j = 0; j < 32; ++j) acc[j] = (has0 && m_a != -INFINITY) ? w0 * __uint_as_float(ra[j]) : 0.f;   // (an accumulator no P V wrote may hold anything)
                         if (has1) {
                             ptx::tmem_ld_32x32b_x32(lane_base + kTmemO + (uint32_t)(D + grp * kDH + c4 * 32), ra);
                             ptx::tmem_ld_wait();
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) acc[j] = fmaf(w1, __uint_as_float(ra[j]), acc[j]);
+                            for (int j = 0; j < 32; ++j) acc[j] = (m_b != -INFINITY) ? fmaf(w1, __uint_as_float(ra[j]), acc[j]) : acc[j];
                         }
                     }
                     if (whole_unit) {
@@ -1021,12 +1017,12 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
 
     CUtensorMap tm_k, tm_v;
     {
-        // pool viewed as (64 columns, 16 tokens, D/64 halves, Hkv heads, layers*pages)
+        // pool viewed as (64 columns, 8 tokens, D/64 halves, 2 token groups, (layer*page)*head): one box is one page of
+        // one head, landing as [token / 8][half][token % 8][128 B] (see kv_slot_off)
         const uint64_t total_pages = (uint64_t)(p.L - 1) * p.layer_pages + p.num_pages;
-        const uint64_t dims[5] = {64, (uint64_t)kSlotTok, (uint64_t)(D / 64), (uint64_t)Hkv, total_pages};
-        const uint64_t strides[4] = {(uint64_t)D * 2, 128, (uint64_t)kSlotTok * D * 2, (uint64_t)page_elems * 2};
-        // one box per page and tensor (all halves): [half][16 tokens][128 B] in shared memory
-        const uint32_t box[5] = {64, (uint32_t)kSlotTok, (uint32_t)(D / 64), 1, 1};
+        const uint64_t dims[5] = {64, 8, (uint64_t)(D / 64), 2, total_pages * (uint64_t)Hkv};
+        const uint64_t strides[4] = {(uint64_t)D * 2, 128, (uint64_t)8 * D * 2, (uint64_t)kSlotTok * D * 2};
+        const uint32_t box[5] = {64, 8, (uint32_t)(D / 64), 2, 1};
         mirror_status st = mirror_make_tmap(ctx, &tm_k, kv->k_pool, 5, dims, strides, box);
         if (st != MIRROR_OK) return st;
         st = mirror_make_tmap(ctx, &tm_v, kv->v_pool, 5, dims, strides, box);
