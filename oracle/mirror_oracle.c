@@ -19,8 +19,12 @@
  * forms for the LM head, exhaustive enumeration of the greedy rule, exact
  * integration of the speculative-sampling rule for one branch (losslessness),
  * the worked example of Fig. 1, and the reuse probability of Proposition 1.
- * The speculative-sampling rule over kappa > 1 branches is this build's own
- * reading (the paper verifies one path per step): parity unpinned for kappa > 1.
+ * The independent per-branch speculative-sampling rule over kappa > 1 branches
+ * (oracle_accept_spec) is this build's own reading (the paper verifies one path
+ * per step): parity unpinned for kappa > 1.  The lossless rule over sibling sets
+ * (oracle_accept_tree) is pinned by exact integration for two and three independent
+ * siblings (the emitted token follows the target distribution), by its chain special
+ * case (equal to the single-branch rule) and by fixed walk-order cases.
  */
 #include <math.h>
 #include <stdint.h>
@@ -391,6 +395,93 @@ int oracle_accept_spec(const int32_t* tokens, const float* logits, const float* 
         if (margin) margin[b] = mg;
     }
     free(mass); free(paths); free(plen);
+    return 0;
+}
+
+/* ----------------------------------------------------------------------------------------
+ * O3'': lossless acceptance over a token tree (Sec. 3.1's speculative-sampling rule applied to the
+ * sibling sets of a tree draft: sequential multi-round rejection).
+ * Walk down from the root.  At row r the target distribution is p_r; its children c_1 < c_2 < ...
+ * (node order) are tested one after the other against the CURRENT distribution m (m = p_r at first):
+ * child c with token x and draft distribution q_c passes iff u_accept[c] * q_c[x] <= m[x]; the walk
+ * then moves to row c.  A child that fails turns m into the normalised residual max(0, m - q_c)
+ * (left unchanged when that residual has no mass).  When every child of r has failed, or r is a
+ * leaf and emit_bonus is set, the extra token is drawn from m by inverse CDF with u_resample[r].
+ * If the siblings of a node are independent draws from one q, the emitted tokens are distributed
+ * exactly as the target's own samples, for any number of siblings.
+ * best_branch is the lowest-index root-to-leaf branch that contains the accepted path.
+ * margin[b]: smallest relative distance of any decision of request b from its knife edge.
+ * ---------------------------------------------------------------------------------------- */
+int oracle_accept_tree(const int32_t* tokens, const float* logits, const float* lse, const float* q_probs,
+                       const float* u_accept, const float* u_resample, const int32_t* parent,
+                       int B, int n, int V, int max_len, int emit_bonus, double temperature,
+                       const int32_t* cand_ids, int n_cand,
+                       int32_t* n_accepted, int32_t* best_branch, int32_t* decide_row,
+                       int32_t* n_emitted, int32_t* emitted, int32_t* accepted_nodes,
+                       int32_t* reuse_slot, double* margin) {
+    int32_t* paths = (int32_t*)malloc(sizeof(int32_t) * (size_t)n * max_len);
+    int32_t* plen = (int32_t*)malloc(sizeof(int32_t) * (size_t)n);
+    int nb = oracle_branches(parent, n, max_len, paths, plen);
+    if (nb < 0) { free(paths); free(plen); return -1; }
+    double* m = (double*)malloc(sizeof(double) * (size_t)V);
+    for (int b = 0; b < B; ++b) {
+        const int32_t* tok = tokens + (size_t)b * n;
+        double mg = INFINITY;
+        for (int k = 0; k < max_len + 1; ++k) emitted[(size_t)b * (max_len + 1) + k] = -1;
+        for (int k = 0; k < max_len; ++k) accepted_nodes[(size_t)b * max_len + k] = -1;
+        int r = 0, A = 0, ne = 0, extra = -1, have_extra = 0;
+        for (;;) {
+            size_t row = (size_t)b * n + r;
+            for (int v = 0; v < V; ++v) m[v] = exp((double)logits[row * V + v] / temperature - (double)lse[row]);
+            int n_children = 0, next = -1;
+            for (int c = r + 1; c < n && next < 0; ++c) {
+                if (parent[c] != r) continue;
+                ++n_children;
+                int x = tok[c];
+                const float* qc = q_probs + ((size_t)b * (n - 1) + (c - 1)) * V;
+                double lhs = (double)u_accept[(size_t)b * n + c] * (double)qc[x];
+                double rel = fabs(lhs - m[x]) / (m[x] > 0 ? m[x] : 1.0);
+                if (rel < mg) mg = rel;
+                if (lhs <= m[x]) { next = c; break; }
+                double Z = 0.0;
+                for (int v = 0; v < V; ++v) {
+                    double res = m[v] - (double)qc[v];
+                    Z += (res > 0.0) ? res : 0.0;
+                }
+                if (Z > 0.0)
+                    for (int v = 0; v < V; ++v) {
+                        double res = m[v] - (double)qc[v];
+                        m[v] = ((res > 0.0) ? res : 0.0) / Z;
+                    }
+            }
+            if (next >= 0) {
+                accepted_nodes[(size_t)b * max_len + A] = next;
+                emitted[(size_t)b * (max_len + 1) + A] = tok[next];
+                ++A;
+                r = next;
+                continue;
+            }
+            have_extra = (n_children > 0) || emit_bonus != 0;
+            if (have_extra) extra = inverse_cdf(m, V, (double)u_resample[(size_t)b * n + r], &mg);
+            break;
+        }
+        ne = A;
+        if (have_extra) emitted[(size_t)b * (max_len + 1) + ne++] = extra;
+        int best = 0;
+        for (int i = 0; i < nb; ++i) {
+            int ok = plen[i] >= A;
+            for (int k = 0; k < A && ok; ++k) ok = paths[(size_t)i * max_len + k] == accepted_nodes[(size_t)b * max_len + k];
+            if (ok) { best = i; break; }
+        }
+        n_accepted[b] = A; best_branch[b] = best; decide_row[b] = r; n_emitted[b] = ne;
+        int slot = -1;
+        if (have_extra && cand_ids)
+            for (int k = 0; k < n_cand; ++k)
+                if (cand_ids[((size_t)b * n + r) * n_cand + k] == extra) { slot = k; break; }
+        reuse_slot[b] = slot;
+        if (margin) margin[b] = mg;
+    }
+    free(m); free(paths); free(plen);
     return 0;
 }
 

@@ -156,6 +156,28 @@ def accept_spec(tokens, logits, lse, q_probs, u_accept, u_resample, parent, max_
     return o
 
 
+def accept_tree(tokens, logits, lse, q_probs, u_accept, u_resample, parent, max_len: int,
+                emit_bonus: bool = True, temperature: float = 1.0, cand_ids=None):
+    """O3'': lossless acceptance over a token tree (sequential multi-round rejection over siblings)."""
+    tokens = _c(tokens, np.int32); par = _c(parent, np.int32)
+    logits = _c(logits, np.float32); lse = _c(lse, np.float32); q_probs = _c(q_probs, np.float32)
+    u_accept = _c(u_accept, np.float32); u_resample = _c(u_resample, np.float32)
+    B, n = tokens.shape
+    V = logits.shape[-1]
+    cand = None if cand_ids is None else _c(cand_ids, np.int32)
+    n_cand = 0 if cand is None else cand.shape[-1]
+    o = _accept_out(B, max_len)
+    o["margin"] = np.zeros(B, np.float64)
+    rc = lib().oracle_accept_tree(_p(tokens), _p(logits), _p(lse), _p(q_probs), _p(u_accept), _p(u_resample),
+                                  _p(par), B, n, V, max_len, int(emit_bonus), C.c_double(temperature),
+                                  _p(cand), n_cand, _p(o["n_accepted"]), _p(o["best_branch"]),
+                                  _p(o["decide_row"]), _p(o["n_emitted"]), _p(o["emitted"]),
+                                  _p(o["accepted_nodes"]), _p(o["reuse_slot"]), _p(o["margin"]))
+    if rc != 0:
+        raise ValueError("bad tree")
+    return o
+
+
 def overlap_mass(q_final, ids) -> float:
     """Eq. 7: Omega_kappa, the final distribution's mass on the early-exit Top-kappa ids."""
     q_final = _c(q_final, np.float64); ids = _c(ids, np.int32)

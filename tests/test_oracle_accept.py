@@ -1,7 +1,8 @@
 """Pins for the oracle's acceptance rules (O3, O3'): the greedy operator against a literal
 set-comprehension over every input of a tiny case, fixed cases, the Fig. 1 example, exact
-integration of the speculative-sampling rule (losslessness for one branch), and the reuse
-probability of Proposition 1."""
+integration of the speculative-sampling rule (losslessness for one branch), the reuse
+probability of Proposition 1, and the lossless rule over sibling sets of a tree (exact integration
+for two and three independent siblings, the chain special case, fixed walk-order cases)."""
 import itertools
 import os
 
@@ -281,3 +282,105 @@ def test_branches_of_general_tree():
     assert plen.tolist() == [2, 2, 2]
     with pytest.raises(ValueError):
         O.tree([-1, 1])
+
+
+# ---------------------------------------------------------------------------------------------
+# O3'': lossless acceptance over a tree (sequential multi-round rejection over siblings)
+# ---------------------------------------------------------------------------------------------
+def tree_inputs(p_rows, q_rows, xs, u_acc, u_res):
+    """One request on an arbitrary tree: p_rows[r] row r's target distribution, q_rows[c-1] node c's draft
+    distribution, xs[c-1] node c's token."""
+    n = len(xs) + 1
+    logits = np.log(np.maximum(np.array(p_rows, np.float64), 1e-300)).astype(np.float32)
+    return (np.array([0] + list(xs), np.int32), logits, np.zeros(n, np.float32), np.array(q_rows, np.float32),
+            np.array(u_acc, np.float32), np.array(u_res, np.float32))
+
+
+def batch_tree(items, parent, max_len, **kw):
+    tok = np.stack([i[0] for i in items]); logits = np.stack([i[1] for i in items]).reshape(-1, items[0][1].shape[-1])
+    lse = np.concatenate([i[2] for i in items]); q = np.stack([i[3] for i in items])
+    ua = np.stack([i[4] for i in items]); ur = np.stack([i[5] for i in items])
+    return O.accept_tree(tok, logits, lse, q, ua, ur, parent, max_len, **kw)
+
+
+@pytest.mark.parametrize("p16,q16,m,grids", [
+    # thresholds of sibling 1: p/q in {1/4, 1/3} (12 cells); of sibling 2: residual/q = 4/7 (7 cells); the last
+    # residual is a point mass
+    ([1, 5, 2, 8], [4, 4, 6, 2], 2, (12, 7, 3)),
+    ([1, 5, 2, 8], [4, 4, 6, 2], 3, (12, 7, 3)),
+    # thresholds 1/3 and 3/5 (15 cells); after two rejections the residual is (7, 26)/33 on ids 2, 3 (33 cells)
+    ([2, 3, 5, 6], [6, 5, 3, 2], 2, (15, 2, 33)),
+])
+def test_tree_rule_is_lossless_for_iid_siblings_exact_integration(p16, q16, m, grids):
+    """m sibling drafts drawn independently from q under the root: whatever m is, the first emitted token must
+    follow the target distribution p exactly (the property that makes multi-branch verification lossless).  Every
+    decision boundary lies on a grid edge, so the midpoint rule integrates the law exactly."""
+    V = 4
+    p = np.array(p16) / 16.0
+    q = np.array(q16) / 16.0
+    parent = np.array([-1] + [0] * m, np.int32)
+    Na1, Na2, Nr = grids
+    items, weights = [], []
+    for xs in itertools.product(range(V), repeat=m):
+        for a1 in range(Na1):
+            for a2 in range(Na2):
+                for r in range(Nr):
+                    ua = [0.0, (a1 + 0.5) / Na1] + [(a2 + 0.5) / Na2] * (m - 1)
+                    ur = [(r + 0.5) / Nr] * (m + 1)
+                    items.append(tree_inputs([p] * (m + 1), [q] * m, xs, ua, ur))
+                    weights.append(np.prod([q[x] for x in xs]) / (Na1 * Na2 * Nr))
+    # (with three siblings the third one's threshold is 0 or above 1 for these numbers, so sharing sibling 2's
+    # uniform integrates it exactly too)
+    o = batch_tree(items, parent, 1)
+    w = np.array(weights)
+    law = np.zeros(V)
+    for k in range(len(items)):
+        law[o["emitted"][k, 0]] += w[k]
+    np.testing.assert_allclose(law, p, atol=1e-12)
+    # more siblings can only help: the acceptance probability is at least that of one draft
+    assert (w * (o["n_accepted"] == 1)).sum() >= np.minimum(p, q).sum() - 1e-12
+
+
+def test_tree_rule_on_a_chain_is_the_single_branch_rule():
+    rng = np.random.default_rng(5)
+    V, gamma, B = 23, 4, 200
+    parent = comb_parent(1, gamma)
+    n = gamma + 1
+    logits = rng.normal(0, 2, (B * n, V)).astype(np.float32)
+    lse = np.log(np.exp(logits.astype(np.float64)).sum(1)).astype(np.float32)
+    q = rng.dirichlet(np.ones(V), (B, n - 1)).astype(np.float32)
+    tok = rng.integers(0, V, (B, n)).astype(np.int32)
+    ua = rng.random((B, n)).astype(np.float32); ur = rng.random((B, n)).astype(np.float32)
+    a = O.accept_spec(tok, logits, lse, q, ua, ur, parent, gamma)
+    b = O.accept_tree(tok, logits, lse, q, ua, ur, parent, gamma)
+    for key in ("n_accepted", "best_branch", "decide_row", "n_emitted", "emitted", "accepted_nodes", "reuse_slot"):
+        assert (a[key] == b[key]).all(), key
+    assert (a["n_accepted"] > 0).any() and (a["n_accepted"] < gamma).any()
+
+
+def test_tree_rule_walk_order_on_a_two_level_tree():
+    # nodes: 1, 2 under the root; 3, 4 under node 1; 5 under node 2.  Branches (leaves in order): [1,3], [1,4], [2,5].
+    parent = np.array([-1, 0, 0, 1, 1, 2], np.int32)
+    V = 3
+    flat = np.full(V, 1.0 / V)
+    peaked = np.array([0.98, 0.01, 0.01])
+    # node 1 proposes token 1 from a draft that is sure of it, the target gives it 1%: rejected for u = 0.9;
+    # node 2 (u = 0) and node 5 (u = 0) pass whatever their numbers are; node 5 is a leaf: bonus from its row
+    p_rows = [peaked, flat, flat, flat, flat, np.array([0.0, 0.0, 1.0])]
+    q_rows = [np.array([0.01, 0.98, 0.01]), flat, flat, flat, flat]
+    item = tree_inputs(p_rows, q_rows, [1, 0, 2, 2, 1], [0.0, 0.9, 0.0, 0.5, 0.5, 0.0], [0.5] * 6)
+    o = batch_tree([item], parent, 2)
+    assert o["n_accepted"][0] == 2 and o["accepted_nodes"][0].tolist() == [2, 5]
+    assert o["best_branch"][0] == 2 and o["decide_row"][0] == 5
+    assert o["emitted"][0].tolist() == [0, 1, 2] and o["n_emitted"][0] == 3
+    # both children of the root rejected (u close to 1 against drafts that overrate their tokens): the extra token
+    # comes from the twice-reduced distribution at the root, which has lost ids 1 and 2 entirely -> id 0
+    q_over = [np.array([0.0, 1.0, 0.0]), np.array([0.0, 0.0, 1.0]), flat, flat, flat]
+    item = tree_inputs([np.array([0.5, 0.25, 0.25])] + [flat] * 5, q_over, [1, 2, 0, 0, 0], [0.0, 0.99, 0.99, 0.5, 0.5, 0.5], [0.7] * 6)
+    o = batch_tree([item], parent, 2)
+    assert o["n_accepted"][0] == 0 and o["decide_row"][0] == 0 and o["n_emitted"][0] == 1
+    assert o["emitted"][0].tolist() == [0, -1, -1]
+    # without a bonus a fully accepted path emits only its own tokens
+    item = tree_inputs(p_rows, q_rows, [1, 0, 2, 2, 1], [0.0, 0.9, 0.0, 0.5, 0.5, 0.0], [0.5] * 6)
+    o = batch_tree([item], parent, 2, emit_bonus=False)
+    assert o["n_emitted"][0] == 2 and o["emitted"][0].tolist() == [0, 1, -1]
