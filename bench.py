@@ -38,6 +38,8 @@ def parse_args():
     ap.add_argument("--workload", default="qwen14b")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--accept-mode", default=None, choices=["greedy", "spec_sampling", "spec_tree"],
+                    help="override the workload's acceptance rule")
     return ap.parse_args()
 
 
@@ -182,6 +184,8 @@ def run_reference(args):
     from oracle import oracle as O
     from paper_2510_13161_b200 import inputs as I
     cfg = I.CONFIGS[args.workload]
+    if args.accept_mode:
+        cfg = I.shrink(cfg, mode=args.accept_mode)
     x = I.gen_verify_inputs(cfg, args.seed, "cpu", layers=1, force_hidden=cfg.explicit_hidden)
     steps, warm = max(1, min(args.steps, 4)), max(0, min(args.warmup, 1))
     for _ in range(warm):
@@ -240,12 +244,14 @@ def run_mirror(args):
     dev = torch.device("cuda", local)
 
     cfg = I.CONFIGS[args.workload]
+    if args.accept_mode:
+        cfg = I.shrink(cfg, mode=args.accept_mode)
     x = I.gen_verify_inputs(cfg, args.seed + rank, dev)          # replicas: each rank draws its own problem
     m = binding.Mirror(cfg.hidden, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.vocab, temperature=cfg.temperature,
                        device=local)
     kv = m.kv(x.k_pool, x.v_pool, x.page_table, x.prefix_len)
     tree = m.tree(x.tokens, cfg.kappa, cfg.gamma)
-    mode = binding.ACCEPT_SPEC_SAMPLING if cfg.mode == "spec_sampling" else binding.ACCEPT_GREEDY
+    mode = {"spec_sampling": binding.ACCEPT_SPEC_SAMPLING, "spec_tree": binding.ACCEPT_SPEC_TREE}.get(cfg.mode, binding.ACCEPT_GREEDY)
     acc = m.accept_in(mode, True, q_probs=x.q_probs, u_accept=x.u_accept, u_resample=x.u_resample)
     attn_out = torch.empty_like(x.q)
     res = binding.AcceptResult(cfg.batch, cfg.gamma, dev)
@@ -353,7 +359,7 @@ def run_mirror(args):
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic", "draft_tokens_per_sec": value * cfg.draft_tokens,
             "config": {"workload": cfg.name, "kappa": cfg.kappa, "gamma": cfg.gamma, "batch": cfg.batch, "layers": cfg.layers,
-                       "prefix": [cfg.prefix_lo, cfg.prefix_hi], "vocab": cfg.vocab, "hidden": cfg.hidden,
+                       "prefix": [cfg.prefix_lo, cfg.prefix_hi], "vocab": cfg.vocab, "hidden": cfg.hidden, "accept": cfg.mode,
                        "l2": "inputs (KV cache + LM-head weights, about 2 GB) are larger than L2; no flush",
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

@@ -94,7 +94,11 @@ typedef struct {
     const int32_t* prefix_len; /* device [B]: verified-prefix length in tokens, <= max_pages_per_req*page_size */
 } mirror_kv;
 
-typedef enum { MIRROR_ACCEPT_GREEDY = 0, MIRROR_ACCEPT_SPEC_SAMPLING = 1 } mirror_accept_mode;
+typedef enum {
+    MIRROR_ACCEPT_GREEDY = 0,        /* Eq. 3 / Eq. 10 on every branch, longest branch wins */
+    MIRROR_ACCEPT_SPEC_SAMPLING = 1, /* speculative-sampling rule on every branch independently, longest wins */
+    MIRROR_ACCEPT_SPEC_TREE = 2      /* lossless rule over the tree: sequential rejection over siblings (below) */
+} mirror_accept_mode;
 
 typedef struct {
     mirror_accept_mode mode;
@@ -126,6 +130,9 @@ typedef struct {
 #define MIRROR_WS_LMHEAD_LOGITS 10u /* mirror_lmhead_reduce with topk > 0 and logits_out == NULL */
 #define MIRROR_WS_STEP_GREEDY 7u    /* mirror_verify_step, greedy */
 #define MIRROR_WS_STEP_SPEC 15u     /* mirror_verify_step, speculative sampling (holds the fp32 logits) */
+#define MIRROR_WS_ACCEPT_TREE 16u   /* adds the fp64 scratch of MIRROR_ACCEPT_SPEC_TREE (optional: without it the rule
+                                       re-evaluates the running distribution instead of storing it, which is slower) */
+#define MIRROR_WS_STEP_TREE 31u     /* mirror_verify_step, MIRROR_ACCEPT_SPEC_TREE */
 
 /* Create a context for one model shape on CUDA device `device` (made current for the call).
  * Allocates one device status word.  Fails with MIRROR_ERR_UNSUPPORTED on a device that is not sm_100. */
@@ -194,7 +201,15 @@ mirror_status mirror_lmhead_reduce_noalloc(int device, const void* hidden, int M
  * u_resample[R] from the normalised residual max(0, p_R - q_c') of the first rejected node c' of the chosen
  * branch, or from p_R when the whole branch was accepted (or the residual has no mass).
  * Selecting the longest of several independently tested branches is distribution-preserving only for a
- * single branch. */
+ * single branch.
+ * MIRROR_ACCEPT_SPEC_TREE (same inputs; tree drafts, Sec. 3.1's rule applied to sibling sets): walk down from the
+ * root; at row r the current distribution m starts as p_r, the children of r are tested in node order, child c
+ * (token x) passes iff u_accept[c] * q_c[x] <= m[x] and the walk moves to c; a child that fails turns m into the
+ * normalised residual max(0, m - q_c) (left as it is when that residual has no mass).  When every child of r has
+ * failed -- or r is a leaf and emit_bonus is set -- the extra token is drawn from m by inverse CDF with
+ * u_resample[r].  If the siblings of each node are independent draws from one q, the emitted tokens are distributed
+ * exactly as the target's own samples for any tree.  best_branch is the lowest-index branch that contains the
+ * accepted path.  All decision arithmetic is fp64. */
 mirror_status mirror_accept_select(mirror_ctx* ctx, const mirror_tree* tree, const mirror_accept_in* in,
                                    const mirror_accept_out* out, void* stream);
 

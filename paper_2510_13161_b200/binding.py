@@ -17,7 +17,8 @@ LIB_PATH = os.path.join(_HERE, "libmirror.so")
 
 ACCEPT_GREEDY = 0
 ACCEPT_SPEC_SAMPLING = 1
-WS_ATTN, WS_LMHEAD, WS_LMHEAD_LOGITS, WS_STEP_GREEDY, WS_STEP_SPEC = 1, 2, 10, 7, 15
+ACCEPT_SPEC_TREE = 2
+WS_ATTN, WS_LMHEAD, WS_LMHEAD_LOGITS, WS_STEP_GREEDY, WS_STEP_SPEC, WS_ACCEPT_TREE, WS_STEP_TREE = 1, 2, 10, 7, 15, 16, 31
 
 EXPORTS = [
     "mirror_create", "mirror_destroy", "mirror_workspace_bytes", "mirror_set_workspace",
@@ -255,9 +256,13 @@ class Mirror:
         a._refs = (target_argmax, logits, lse, q_probs, u_accept, u_resample, cand_ids)
         return a
 
-    def mirror_accept_select(self, tree: Tree, acc: AcceptIn, out: Optional[AcceptResult] = None, stream=None) -> AcceptResult:
+    def mirror_accept_select(self, tree: Tree, acc: AcceptIn, out: Optional[AcceptResult] = None, stream=None,
+                             tree_scratch: bool = False) -> AcceptResult:
+        """tree_scratch: size the workspace so that the tree rule can keep its running distribution in memory."""
         if out is None:
             out = AcceptResult(tree.batch, tree.gamma, self.device)
+        if tree_scratch:
+            self.ensure_workspace(tree, None, WS_STEP_TREE)
         o = out.struct()
         _check(self.lib.mirror_accept_select(self._ctx, C.byref(tree), C.byref(acc), C.byref(o), _stream(stream)),
                "mirror_accept_select")
@@ -267,7 +272,7 @@ class Mirror:
                            out: Optional[AcceptResult] = None, argmax_out=None, stream=None) -> AcceptResult:
         if out is None:
             out = AcceptResult(tree.batch, tree.gamma, self.device)
-        self.ensure_workspace(tree, kv, WS_STEP_SPEC if acc.mode == ACCEPT_SPEC_SAMPLING else WS_STEP_GREEDY)
+        self.ensure_workspace(tree, kv, {ACCEPT_GREEDY: WS_STEP_GREEDY, ACCEPT_SPEC_TREE: WS_STEP_TREE}.get(acc.mode, WS_STEP_SPEC))
         o = out.struct()
         _check(self.lib.mirror_verify_step(self._ctx, C.byref(kv), C.byref(tree), _ptr(q, torch.bfloat16, "q"),
                                            _ptr(k_new, torch.bfloat16, "k_new"), _ptr(v_new, torch.bfloat16, "v_new"),

@@ -30,6 +30,7 @@ struct AcceptArgs {
     const float* u_resample;
     const int32_t* cand_ids;
     mirror_accept_out out;
+    double* tree_scratch;          // nullable fp64 [B, 2, V]: running distribution of the tree rule
     int* status;
 };
 
@@ -197,10 +198,217 @@ accept_select_kernel(const __grid_constant__ AcceptTreeParams tp, const AcceptAr
     }
 }
 
+// ---------------------------------------------------------------------------------------------------
+// Lossless acceptance over a token tree: sequential multi-round rejection over the siblings of each accepted
+// row (the speculative-sampling rule of Sec. 3.1 applied to sibling sets, for tree drafts).  One block per
+// request walks down from the root.  At row r the current distribution m starts as the target's p_r; the
+// children of r are tested in node order against m: child c (token x, draft distribution q_c) passes iff
+// u_accept[c] * q_c[x] <= m[x] and the walk moves to c; a child that fails turns m into the normalised residual
+// max(0, m - q_c).  m is never stored: m[v] is re-evaluated from the logits, the rejected siblings' q rows and
+// their normalisers Z_i (fp64, same operation order per element as the definition), so a rejection costs one
+// pass over the vocabulary for Z and the final draw one more.
+// ---------------------------------------------------------------------------------------------------
+constexpr int kMaxRejected = MIRROR_MAX_BRANCHES;     // siblings rejected at one row
+
+__global__ void __launch_bounds__(kThreads, 1)
+accept_tree_kernel(const __grid_constant__ AcceptTreeParams tp, const AcceptArgs a) {
+    __shared__ double s_seg[kThreads];
+    __shared__ double s_Z[kMaxRejected];
+    __shared__ int s_rej[kMaxRejected];
+    __shared__ int s_path[MIRROR_MAX_DEPTH];
+    __shared__ double s_tot, s_thr, s_excl;
+    __shared__ int s_pass, s_found, s_extra, s_last_pos;
+
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n = tp.n, V = a.V;
+    const int32_t* tok = a.tokens + (size_t)b * n;
+    const int S = (V + kThreads - 1) / kThreads;
+    const int v0 = min(tid * S, V), v1 = min(v0 + S, V);
+
+    int r = 0, A = 0, n_rej = 0, n_children = 0;
+    // With scratch memory the unnormalised residual of the last effective rejection is stored (two buffers, so that a
+    // residual without mass can be dropped) and m[v] = stored[v] / Z_last: the same operations as the definition.
+    double* const buf0 = a.tree_scratch ? a.tree_scratch + (size_t)b * 2 * V : nullptr;
+    double* const buf1 = buf0 ? buf0 + V : nullptr;
+    int cur = 0;                                   // buffer that holds the current residual (when n_rej > 0)
+    double inv_Z = 1.0;                            // 1 / Z of the last effective rejection
+    // m[v] at row r after the rejections recorded so far
+    auto mass = [&](const float* lr, double lse_r, int v) -> double {
+        if (buf0 && n_rej > 0) return (cur ? buf1 : buf0)[v] * inv_Z;       // (times 1/Z: one rounding away from the quotient)
+        double m = exp((double)lr[v] * a.inv_T - lse_r);
+        for (int i = 0; i < n_rej; ++i) {
+            const double res = m - (double)a.q_probs[((size_t)b * (n - 1) + (s_rej[i] - 1)) * V + v];
+            m = ((res > 0.0) ? res : 0.0) / s_Z[i];
+        }
+        return m;
+    };
+    // block-wide sum of f over the vocabulary in a fixed order: per-thread contiguous segments, then warp 0
+    // adds the segments in order
+    // (contiguous = true: per-thread contiguous segments, whose sums the inverse-CDF search then reuses; false: ids
+    // interleaved over the threads, which keeps the loads of a warp in one line -- any fixed order will do for a sum)
+    auto block_total = [&](auto f, bool contiguous) -> double {
+        double part = 0.0;
+        if (contiguous) {
+            for (int v = v0; v < v1; ++v) part += f(v);
+        } else {
+            double p0 = 0.0, p1 = 0.0, p2 = 0.0, p3 = 0.0;
+            int v = tid;
+            for (; v + 3 * kThreads < V; v += 4 * kThreads) {
+                p0 += f(v); p1 += f(v + kThreads); p2 += f(v + 2 * kThreads); p3 += f(v + 3 * kThreads);
+            }
+            for (; v < V; v += kThreads) p0 += f(v);
+            part = (p0 + p1) + (p2 + p3);
+        }
+        s_seg[tid] = part;
+        __syncthreads();
+        if (warp == 0) {
+            double lp = 0.0;
+            for (int k = 0; k < 32; ++k) lp += s_seg[lane * 32 + k];
+            double tot;
+            warp_excl_scan(lp, lane, &tot);
+            if (lane == 0) s_tot = tot;
+        }
+        __syncthreads();
+        return s_tot;
+    };
+
+    for (;;) {
+        const size_t row = (size_t)b * n + r;
+        const float* lr = a.logits + row * V;
+        const double lse_r = (double)a.lse[row];
+        n_rej = 0;
+        n_children = 0;
+        int next = -1;
+        for (int c = r + 1; c < n; ++c) {
+            if (tp.parent[c] != r) continue;
+            ++n_children;
+            const float* qc = a.q_probs + ((size_t)b * (n - 1) + (c - 1)) * V;
+            if (tid == 0) {
+                const int x = tok[c];
+                int pass = 0;
+                if (x < 0 || x >= V) {
+                    atomicExch(a.status, MIRROR_DEV_CHECK);
+                    atomicExch(a.status + 1, 100 + c);
+                } else {
+                    const double lhs = (double)a.u_accept[(size_t)b * n + c] * (double)qc[x];
+                    pass = (lhs <= mass(lr, lse_r, x)) ? 1 : 0;
+                }
+                s_pass = pass;
+            }
+            __syncthreads();
+            if (s_pass) { next = c; break; }
+            // rejected: normaliser of the residual (a residual without mass leaves m as it is)
+            double* const nxt = !buf0 ? nullptr : ((n_rej > 0 && cur == 0) ? buf1 : buf0);      // the buffer not in use
+            const double Z = block_total([&](int v) {
+                double res = mass(lr, lse_r, v) - (double)qc[v];
+                res = (res > 0.0) ? res : 0.0;
+                if (nxt) nxt[v] = res;
+                return res;
+            }, false);
+            if (Z > 0.0 && n_rej < kMaxRejected) {
+                if (tid == 0) { s_rej[n_rej] = c; s_Z[n_rej] = Z; }
+                if (nxt) cur = (nxt == buf1) ? 1 : 0;
+                inv_Z = 1.0 / Z;
+                ++n_rej;
+            }
+            __syncthreads();
+        }
+        if (next >= 0) {
+            if (tid == 0 && A < MIRROR_MAX_DEPTH) s_path[A] = next;
+            ++A;
+            r = next;
+            __syncthreads();
+            if (A >= MIRROR_MAX_DEPTH) { n_children = 0; n_rej = 0; break; }      // (cannot happen: depth <= gamma <= 32)
+            continue;
+        }
+        break;
+    }
+    const bool have_extra = (n_children > 0) || a.emit_bonus != 0;
+    if (tid == 0) { s_extra = -1; s_last_pos = -1; s_found = -1; }
+    __syncthreads();
+    if (have_extra) {
+        // inverse-CDF draw from m at row r
+        const size_t row = (size_t)b * n + r;
+        const float* lr = a.logits + row * V;
+        const double lse_r = (double)a.lse[row];
+        const double tot = block_total([&](int v) { return mass(lr, lse_r, v); }, true);
+        if (warp == 0) {
+            const double thr = (double)a.u_resample[row] * tot;
+            double lp = 0.0;
+            for (int k = 0; k < 32; ++k) lp += s_seg[lane * 32 + k];
+            double dummy;
+            double run = warp_excl_scan(lp, lane, &dummy);
+            int found = -1;
+            double found_excl = 0.0;
+            for (int k = 0; k < 32; ++k) {
+                const double seg = s_seg[lane * 32 + k];
+                if (found < 0 && run + seg > thr) { found = lane * 32 + k; found_excl = run; }
+                run += seg;
+            }
+            const unsigned mk = __ballot_sync(0xffffffffu, found >= 0);
+            if (mk) {
+                const int src = __ffs(mk) - 1;
+                if (lane == src) { s_found = found; s_excl = found_excl; }
+            }
+            if (lane == 0) s_thr = thr;
+        }
+        __syncthreads();
+        if (s_found >= 0) {
+            if (tid == s_found) {
+                const double thr = s_thr, excl = s_excl;
+                double loc = 0.0;
+                int pick = v1 - 1;
+                for (int v = v0; v < v1; ++v) {
+                    loc += mass(lr, lse_r, v);
+                    if (excl + loc > thr) { pick = v; break; }
+                }
+                s_extra = pick;
+            }
+        } else {
+            // rounding left no crossing: take the last id with positive mass
+            int last = -1;
+            for (int v = v0; v < v1; ++v)
+                if (mass(lr, lse_r, v) > 0.0) last = v;
+            if (last >= 0) atomicMax(&s_last_pos, last);
+            __syncthreads();
+            if (tid == 0) s_extra = s_last_pos;
+        }
+    }
+    __syncthreads();
+
+    const int gamma = tp.gamma;
+    if (tid <= gamma) {
+        int e = -1;
+        if (tid < A) e = tok[s_path[tid]];
+        else if (tid == A && have_extra) e = s_extra;
+        a.out.emitted[(size_t)b * (gamma + 1) + tid] = e;
+        if (tid < gamma) a.out.accepted_nodes[(size_t)b * gamma + tid] = (tid < A) ? s_path[tid] : -1;
+    }
+    if (tid == 0) {
+        // the lowest-index branch that contains the accepted path
+        int best = 0;
+        for (int i = 0; i < tp.n_branches; ++i) {
+            bool ok = tp.path_len[i] >= A;
+            for (int k = 0; k < A && ok; ++k) ok = (tp.path[i][k] == s_path[k]);
+            if (ok) { best = i; break; }
+        }
+        a.out.n_accepted[b] = A;
+        a.out.best_branch[b] = best;
+        a.out.decide_row[b] = r;
+        a.out.n_emitted[b] = A + (have_extra ? 1 : 0);
+        int slot = -1;
+        if (have_extra && a.cand_ids)
+            for (int k = 0; k < a.n_cand; ++k)
+                if (a.cand_ids[((size_t)b * n + r) * a.n_cand + k] == s_extra) { slot = k; break; }
+        a.out.reuse_slot[b] = slot;
+    }
+}
+
 }  // namespace
 
 mirror_status mirror_accept_launch(mirror_ctx* ctx, const mirror_tree* tree, const MirrorTreeInfo& ti,
-                                   const mirror_accept_in* in, const mirror_accept_out* out, cudaStream_t stream) {
+                                   const mirror_accept_in* in, const mirror_accept_out* out, cudaStream_t stream,
+                                   double* tree_scratch) {
     AcceptTreeParams tp;
     tp.n = ti.n;
     tp.n_branches = ti.n_branches;
@@ -223,8 +431,10 @@ mirror_status mirror_accept_launch(mirror_ctx* ctx, const mirror_tree* tree, con
     a.u_resample = in->u_resample;
     a.cand_ids = in->cand_ids;
     a.out = *out;
+    a.tree_scratch = tree_scratch;
     a.status = ctx->d_status;
-    accept_select_kernel<<<tree->batch, kThreads, 0, stream>>>(tp, a);
+    if (in->mode == MIRROR_ACCEPT_SPEC_TREE) accept_tree_kernel<<<tree->batch, kThreads, 0, stream>>>(tp, a);
+    else accept_select_kernel<<<tree->batch, kThreads, 0, stream>>>(tp, a);
     ctx->launches += 1;
     MIRROR_CUDA_OK(cudaGetLastError());
     return MIRROR_OK;
@@ -238,7 +448,7 @@ extern "C" mirror_status mirror_accept_select(mirror_ctx* ctx, const mirror_tree
         return MIRROR_ERR_ARG;
     if (in->mode == MIRROR_ACCEPT_GREEDY) {
         if (!in->target_argmax) return MIRROR_ERR_ARG;
-    } else if (in->mode == MIRROR_ACCEPT_SPEC_SAMPLING) {
+    } else if (in->mode == MIRROR_ACCEPT_SPEC_SAMPLING || in->mode == MIRROR_ACCEPT_SPEC_TREE) {
         if (!in->logits || !in->lse || !in->u_accept || !in->u_resample) return MIRROR_ERR_ARG;
         if (tree->n_nodes > 1 && !in->q_probs) return MIRROR_ERR_ARG;
     } else {
@@ -249,5 +459,11 @@ extern "C" mirror_status mirror_accept_select(mirror_ctx* ctx, const mirror_tree
     mirror_status st = mirror_build_tree(tree, &ti);
     if (st != MIRROR_OK) return st;
     MIRROR_CUDA_OK(cudaSetDevice(ctx->device));
-    return mirror_accept_launch(ctx, tree, ti, in, out, (cudaStream_t)stream);
+    double* tree_scratch = nullptr;
+    if (in->mode == MIRROR_ACCEPT_SPEC_TREE && ctx->ws) {
+        MirrorWsLayout L;
+        mirror_ws_layout(ctx, (size_t)tree->batch * tree->n_nodes, &L, (size_t)tree->batch);
+        if (ctx->ws_bytes >= L.end_accept) tree_scratch = (double*)((uint8_t*)ctx->ws + L.accept_scratch);
+    }
+    return mirror_accept_launch(ctx, tree, ti, in, out, (cudaStream_t)stream, tree_scratch);
 }

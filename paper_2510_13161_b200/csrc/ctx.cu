@@ -139,7 +139,7 @@ mirror_status mirror_build_tree(const mirror_tree* tree, MirrorTreeInfo* info) {
 // ---------------------------------------------------------------------------------------------
 // workspace
 // ---------------------------------------------------------------------------------------------
-void mirror_ws_layout(const mirror_ctx* ctx, size_t M, MirrorWsLayout* out) {
+void mirror_ws_layout(const mirror_ctx* ctx, size_t M, MirrorWsLayout* out, size_t B) {
     MirrorWsLayout L;
     size_t at = 0;
     L.attn_ticket = at;
@@ -161,6 +161,9 @@ void mirror_ws_layout(const mirror_ctx* ctx, size_t M, MirrorWsLayout* out) {
     L.logits_bytes = align_up(M * (size_t)ctx->desc.vocab * sizeof(float), 256);
     at += L.logits_bytes;
     L.end_logits = at;
+    L.accept_scratch = at;
+    at += align_up(B * 2 * (size_t)ctx->desc.vocab * sizeof(double), 256);
+    L.end_accept = at;
     *out = L;
 }
 
@@ -170,10 +173,11 @@ extern "C" mirror_status mirror_workspace_bytes(const mirror_ctx* ctx, const mir
     if (!ctx || !tree || !bytes) return MIRROR_ERR_ARG;
     if (tree->batch <= 0 || tree->n_nodes <= 0 || tree->n_nodes > MIRROR_MAX_NODES) return MIRROR_ERR_SHAPE;
     MirrorWsLayout L;
-    mirror_ws_layout(ctx, (size_t)tree->batch * tree->n_nodes, &L);
+    mirror_ws_layout(ctx, (size_t)tree->batch * tree->n_nodes, &L, (size_t)tree->batch);
     size_t need = L.end_attn;
     if (what & (MIRROR_WS_LMHEAD | 4u)) need = L.end_lmhead;
     if (what & 8u) need = L.end_logits;
+    if (what & 16u) need = L.end_accept;
     *bytes = need;
     return MIRROR_OK;
 }

@@ -40,7 +40,7 @@ mirror_status mirror_build_tree(const mirror_tree* tree, MirrorTreeInfo* info);
 
 // Workspace carving.  The layout depends only on the model shape and the row count M, so every entry
 // point finds the same regions: [arrival counters | attention partials | LM-head partials | lse, argmax
-// scratch | fp32 logits].  Offsets are 256-byte aligned; the counters are zeroed when the workspace is attached.
+// scratch | fp32 logits | fp64 acceptance scratch].  Offsets are 256-byte aligned; the counters are zeroed when the workspace is attached.
 constexpr size_t kWsTicketBytes = 4u << 20;
 struct MirrorWsLayout {
     size_t attn_ticket = 0;                              // arrival counters (kWsTicketBytes)
@@ -48,12 +48,14 @@ struct MirrorWsLayout {
     size_t lm_partial = 0, lm_partial_bytes = 0;         // per-(CTA, warp) row partials
     size_t lse = 0, argmax = 0;                          // [M] scratch each
     size_t logits = 0, logits_bytes = 0;                 // fp32 [M, V]
-    size_t end_attn = 0, end_lmhead = 0, end_logits = 0; // bytes needed up to each region
+    size_t accept_scratch = 0;                           // fp64 [B, 2, V]: running distribution of the tree acceptance
+    size_t end_attn = 0, end_lmhead = 0, end_logits = 0, end_accept = 0;   // bytes needed up to each region
 };
-void mirror_ws_layout(const mirror_ctx* ctx, size_t M, MirrorWsLayout* out);
+void mirror_ws_layout(const mirror_ctx* ctx, size_t M, MirrorWsLayout* out, size_t B = 0);
 
 mirror_status mirror_accept_launch(mirror_ctx* ctx, const mirror_tree* tree, const MirrorTreeInfo& ti,
-                                   const mirror_accept_in* in, const mirror_accept_out* out, cudaStream_t stream);
+                                   const mirror_accept_in* in, const mirror_accept_out* out, cudaStream_t stream,
+                                   double* tree_scratch = nullptr);
 mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, const void* W, int topk,
                                    const int32_t* gather_row, const int32_t* gather_tok, int n_gather,
                                    int32_t* argmax, float* maxlogit, float* lse, int32_t* topk_id,

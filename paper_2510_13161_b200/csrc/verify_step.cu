@@ -46,7 +46,7 @@ extern "C" mirror_status mirror_verify_step(mirror_ctx* ctx, const mirror_kv* kv
         return MIRROR_ERR_ARG;
     mirror_status st = check_kv(ctx, kv, tree);
     if (st != MIRROR_OK) return st;
-    const bool spec = acc->mode == MIRROR_ACCEPT_SPEC_SAMPLING;
+    const bool spec = acc->mode == MIRROR_ACCEPT_SPEC_SAMPLING || acc->mode == MIRROR_ACCEPT_SPEC_TREE;
     if (!spec && acc->mode != MIRROR_ACCEPT_GREEDY) return MIRROR_ERR_ARG;
     if (spec && (!acc->u_accept || !acc->u_resample || (tree->n_nodes > 1 && !acc->q_probs))) return MIRROR_ERR_ARG;
     if (!hidden && ctx->desc.n_q_heads * ctx->desc.head_dim != ctx->desc.hidden) return MIRROR_ERR_SHAPE;
@@ -55,7 +55,7 @@ extern "C" mirror_status mirror_verify_step(mirror_ctx* ctx, const mirror_kv* kv
     if (st != MIRROR_OK) return st;
     const size_t M = (size_t)tree->batch * tree->n_nodes;
     MirrorWsLayout L;
-    mirror_ws_layout(ctx, M, &L);
+    mirror_ws_layout(ctx, M, &L, (size_t)tree->batch);
     if (!ctx->ws || ctx->ws_bytes < (spec ? L.end_logits : L.end_lmhead)) return MIRROR_ERR_WORKSPACE;
     MIRROR_CUDA_OK(cudaSetDevice(ctx->device));
     uint8_t* ws = (uint8_t*)ctx->ws;
@@ -86,7 +86,9 @@ extern "C" mirror_status mirror_verify_step(mirror_ctx* ctx, const mirror_kv* kv
     in.target_argmax = d_argmax;
     in.logits = d_logits;
     in.lse = d_lse;
-    st = mirror_accept_launch(ctx, tree, ti, &in, out, s);
+    // the tree rule keeps its running distribution in the workspace when the caller sized it for that
+    double* tree_scratch = (acc->mode == MIRROR_ACCEPT_SPEC_TREE && ctx->ws_bytes >= L.end_accept) ? (double*)(ws + L.accept_scratch) : nullptr;
+    st = mirror_accept_launch(ctx, tree, ti, &in, out, s, tree_scratch);
     if (st != MIRROR_OK) return st;
     if (ev) MIRROR_CUDA_OK(cudaEventRecord(ctx->stage_ev[3], s));
     return MIRROR_OK;

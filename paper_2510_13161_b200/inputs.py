@@ -39,7 +39,7 @@ class VerifyConfig:
     kappa: int              # branches
     gamma: int              # lookahead tokens per branch
     vocab: int
-    mode: str               # "greedy" | "spec_sampling"
+    mode: str               # "greedy" | "spec_sampling" (independent per-branch rule) | "spec_tree" (lossless rule over the tree)
     w_std: float = 0.02
     kv_std: float = 1.0
     explicit_hidden: bool = False   # LM-head rows given as an input instead of the last layer's attention output
@@ -204,7 +204,7 @@ def gen_verify_inputs(cfg: VerifyConfig, seed: int = 0, device: str = "cpu", *,
 
     out = VerifyInputs(cfg, seed, par, prefix_len.to(device), page_table.to(device), num_pages,
                        q, k_pool, v_pool, k_new, v_new, W, hidden, tokens.to(device))
-    if cfg.mode == "spec_sampling":
+    if cfg.mode in ("spec_sampling", "spec_tree"):
         out.u_accept = torch.rand((B, n), generator=_gen("cpu", seed, "u_accept"), dtype=torch.float32).to(device)
         out.u_resample = torch.rand((B, n), generator=_gen("cpu", seed, "u_resample"), dtype=torch.float32).to(device)
         if with_lm_head:

@@ -4,7 +4,7 @@ import pytest
 import torch
 
 from oracle import oracle as O
-from paper_2510_13161_b200 import inputs as I
+from paper_2510_13161_b200 import binding, inputs as I
 from tests.helpers import make_mirror
 
 pytestmark = pytest.mark.gpu
@@ -111,6 +111,64 @@ def test_spec_sampling_matches_oracle(kappa, gamma, B, V, T):
             assert same or ref["margin"][b] < 1e-9, (b, ref["margin"][b], {f: (got[f][b], ref[f][b]) for f in FIELDS})
         accepted_total += int(ref["n_accepted"].sum())
     assert accepted_total > 0
+
+
+def tree_case(B, parent, V, seed, peaked=False, iid_siblings=True):
+    """Drafts on an arbitrary tree: the children of a node are independent draws from one q (the lossless setting)
+    or each from its own q."""
+    g = torch.Generator().manual_seed(seed)
+    n = len(parent)
+    scale = 3.0 if peaked else 1.0
+    logits = torch.randn((B * n, V), generator=g) * scale
+    qp = torch.softmax(torch.randn((B, n - 1, V), generator=g) * scale, -1)
+    if iid_siblings:
+        first_child = {}
+        for c in range(1, n):
+            first_child.setdefault(parent[c], c)
+            qp[:, c - 1] = qp[:, first_child[parent[c]] - 1]
+    tok = torch.zeros((B, n), dtype=torch.int32)
+    for b in range(B):
+        for c in range(1, n):
+            tok[b, c] = int(torch.multinomial(qp[b, c - 1], 1, generator=g))
+    ua = torch.rand((B, n), generator=g); ur = torch.rand((B, n), generator=g)
+    return logits.float(), qp.float(), tok, ua.float(), ur.float()
+
+
+@pytest.mark.parametrize("shape,B,V,T", [(("comb", 1, 4), 4, 1000, 1.0), (("comb", 4, 4), 6, 1024, 1.0),
+                                         (("comb", 8, 6), 8, 5003, 0.7), (("random", 24, 5), 6, 3001, 1.0),
+                                         (("wide", 12, 1), 6, 2000, 1.0), (("comb", 8, 8), 2, 128256, 1.3)])
+def test_lossless_tree_acceptance_matches_oracle(shape, B, V, T):
+    kind, a, b_ = shape
+    if kind == "comb":
+        par, gamma, kappa = I.comb_parent(a, b_), b_, a
+    elif kind == "random":
+        par, gamma, kappa = I.random_tree_parent(a, 3, max_depth=b_), b_, 0
+    else:                                   # one level of many siblings
+        par, gamma, kappa = [-1] + [0] * a, 1, 0
+    n = len(par)
+    m = make_mirror(cfg_for(V, 1, n - 1, B), temperature=T)
+    accepted_total = rejected_siblings = 0
+    for seed in range(4):
+        logits, qp, tok, ua, ur = tree_case(B, par, V, seed, peaked=(seed == 2), iid_siblings=(seed != 3))
+        if seed == 1:
+            qp[:, 0] = torch.softmax(logits.view(B, -1, V)[:, 0] / T, -1)     # p == q at the first node: residual has no mass
+        lse = torch.logsumexp(logits.double() / T, -1).float()
+        cand = torch.topk(logits, 4, dim=-1).indices.to(torch.int32)
+        ref = O.accept_tree(tok.numpy(), logits.numpy(), lse.numpy(), qp.numpy(), ua.numpy(), ur.numpy(), par, gamma,
+                            True, T, cand.numpy())
+        tree = m.tree(tok.cuda(), kappa, gamma, parent=par)
+        acc = m.accept_in(binding.ACCEPT_SPEC_TREE, True, logits=logits.cuda(), lse=lse.cuda(), q_probs=qp.cuda(),
+                          u_accept=ua.cuda(), u_resample=ur.cuda(), cand_ids=cand.cuda())
+        got = m.mirror_accept_select(tree, acc, tree_scratch=(seed % 2 == 0)).cpu()      # with and without the fp64 scratch
+        assert m.device_status() == (0, 0)
+        for b in range(B):
+            same = all(np.array_equal(got[f][b], ref[f][b]) for f in FIELDS)
+            # a disagreement is tolerated only on a knife edge of the fp64 decision (the normalisers are summed in a
+            # different order, exp implementations differ in the last ulp)
+            assert same or ref["margin"][b] < 1e-9, (b, ref["margin"][b], {f: (got[f][b], ref[f][b]) for f in FIELDS})
+        accepted_total += int(ref["n_accepted"].sum())
+        rejected_siblings += int((ref["n_accepted"] == 0).sum())
+    assert accepted_total > 0 and rejected_siblings > 0
 
 
 def test_spec_root_only_tree_draws_from_the_root_row():

@@ -71,7 +71,8 @@ def test_tiny_config_uniform_and_planted():
         assert got["n_accepted"][0] >= 3 and got["best_branch"][0] == 1
 
 
-def test_spec_sampling_step_small():
+@pytest.mark.parametrize("mode", [1, 2])            # independent per-branch rule; lossless rule over the tree
+def test_spec_sampling_step_small(mode):
     cfg = I.VerifyConfig("s", 512, 8, 2, 64, 2, 3, 40, 200, 3, 3, 2000, "spec_sampling")
     x = I.gen_verify_inputs(cfg, 1, "cuda")
     # draft tokens drawn from q so that some are accepted
@@ -82,12 +83,13 @@ def test_spec_sampling_step_small():
             tok[b, c] = int(torch.multinomial(x.q_probs[b, c - 1].cpu(), 1, generator=g))
     x.tokens = tok.cuda()
     m = make_mirror(cfg)
-    got, am, attn_out = gpu_step(m, x, 1, q_probs=x.q_probs, u_accept=x.u_accept, u_resample=x.u_resample)
+    got, am, attn_out = gpu_step(m, x, mode, q_probs=x.q_probs, u_accept=x.u_accept, u_resample=x.u_resample)
     # feed the oracle the identical logits the GPU used: recompute them with the same kernel and the spill on
     rows = attn_out[-1].reshape(cfg.rows, cfg.hidden)
     lm = m.mirror_lmhead_reduce(rows, x.W, want_logits=True)
-    ref = O.accept_spec(tok.numpy(), lm["logits"].cpu().numpy(), lm["lse"].cpu().numpy(), x.q_probs.cpu().numpy(),
-                        x.u_accept.cpu().numpy(), x.u_resample.cpu().numpy(), x.parent, cfg.gamma)
+    rule = O.accept_spec if mode == 1 else O.accept_tree
+    ref = rule(tok.numpy(), lm["logits"].cpu().numpy(), lm["lse"].cpu().numpy(), x.q_probs.cpu().numpy(),
+               x.u_accept.cpu().numpy(), x.u_resample.cpu().numpy(), x.parent, cfg.gamma)
     for b in range(cfg.batch):
         same = all(np.array_equal(got[f][b], ref[f][b]) for f in FIELDS)
         assert same or ref["margin"][b] < 1e-9, (b, ref["margin"][b])
