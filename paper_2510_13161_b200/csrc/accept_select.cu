@@ -56,6 +56,8 @@ accept_select_kernel(const __grid_constant__ AcceptTreeParams tp, const AcceptAr
     const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n = tp.n, V = a.V;
     const int32_t* tok = a.tokens + (size_t)b * n;
+    ptx::grid_dep_wait();
+    ptx::grid_dep_launch();
 
     for (int br = warp; br < tp.n_branches; br += kThreads / 32) {
         const int len = tp.path_len[br];
@@ -222,6 +224,8 @@ accept_tree_kernel(const __grid_constant__ AcceptTreeParams tp, const AcceptArgs
     const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n = tp.n, V = a.V;
     const int32_t* tok = a.tokens + (size_t)b * n;
+    ptx::grid_dep_wait();
+    ptx::grid_dep_launch();
     const int S = (V + kThreads - 1) / kThreads;
     const int v0 = min(tid * S, V), v1 = min(v0 + S, V);
 
@@ -433,8 +437,8 @@ mirror_status mirror_accept_launch(mirror_ctx* ctx, const mirror_tree* tree, con
     a.out = *out;
     a.tree_scratch = tree_scratch;
     a.status = ctx->d_status;
-    if (in->mode == MIRROR_ACCEPT_SPEC_TREE) accept_tree_kernel<<<tree->batch, kThreads, 0, stream>>>(tp, a);
-    else accept_select_kernel<<<tree->batch, kThreads, 0, stream>>>(tp, a);
+    if (in->mode == MIRROR_ACCEPT_SPEC_TREE) MIRROR_CUDA_OK(mirror_launch_pdl(accept_tree_kernel, dim3(tree->batch), dim3(kThreads), 0, stream, tp, a));
+    else MIRROR_CUDA_OK(mirror_launch_pdl(accept_select_kernel, dim3(tree->batch), dim3(kThreads), 0, stream, tp, a));
     ctx->launches += 1;
     MIRROR_CUDA_OK(cudaGetLastError());
     return MIRROR_OK;

@@ -297,6 +297,10 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     if (p.timing_exit == 1) return;
 #endif
 
+    // (programmatic dependent launch: nothing of global memory is touched before the kernel ahead in the stream has
+    // completed; the merge kernel behind may be scheduled as soon as SMs free up)
+    ptx::grid_dep_wait();
+    ptx::grid_dep_launch();
     // ---- prologue ---------------------------------------------------------------------------------
     for (int b = tid; b < p.B; b += kThreads) {
         int len = p.prefix_len[b];
@@ -930,6 +934,10 @@ __global__ void __launch_bounds__(kMergeThreads) attn_merge_kernel(const AttnPar
     const long long unit_last = u.unit_first_tile + u.tiles_in_unit - 1;
     while (gb + 1 < part.n_groups && group_begin(part, gb + 1, p, cumT) <= unit_last) ++gb;
     const int parts = gb - ga + 1;
+    // launched with programmatic stream serialization: everything above overlaps the attention kernel's tail;
+    // its records (and the outputs this block overwrites) are only touched after it has completed
+    ptx::grid_dep_wait();
+    ptx::grid_dep_launch();
 
     constexpr int kRowW = D + 4;
     constexpr int kQ = D / 4;                                                   // columns per thread
@@ -1043,7 +1051,7 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
         if (smem > kSmemLimit) return MIRROR_ERR_UNSUPPORTED;
         auto go = [&](auto kern) -> mirror_status {
             MIRROR_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit));
-            kern<<<grid, kThreads, smem, stream>>>(tm_k, tm_v, at, p);
+            MIRROR_CUDA_OK(mirror_launch_pdl(kern, dim3(grid), dim3(kThreads), smem, stream, tm_k, tm_v, at, p));
             return MIRROR_OK;
         };
         if (ks == 6 && vs == 6) return go(attn_verify_kernel<DD, 6, 6>);
@@ -1057,8 +1065,8 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
     if (p.n_groups > 1) {
         // which units the partition cut is only known on the device (it depends on the prefix lengths)
         const dim3 mgrid((unsigned)(p.n_groups - 1), (unsigned)p.n_rb);
-        if (D == 128) attn_merge_kernel<128><<<mgrid, kMergeThreads, 0, stream>>>(p);
-        else attn_merge_kernel<64><<<mgrid, kMergeThreads, 0, stream>>>(p);
+        if (D == 128) MIRROR_CUDA_OK(mirror_launch_pdl(attn_merge_kernel<128>, mgrid, dim3(kMergeThreads), 0, stream, p));
+        else MIRROR_CUDA_OK(mirror_launch_pdl(attn_merge_kernel<64>, mgrid, dim3(kMergeThreads), 0, stream, p));
         ctx->launches += 1;
         MIRROR_CUDA_OK(cudaGetLastError());
     }

@@ -103,6 +103,10 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tm_w_full, const __grid_consta
     __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem_base = ctrl->tmem_base;
+    // (programmatic dependent launch: the set-up above overlaps the kernel ahead in the stream; nothing of global
+    // memory is touched before it has completed)
+    ptx::grid_dep_wait();
+    ptx::grid_dep_launch();
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -308,6 +312,8 @@ lmhead_merge_kernel(int M, int P, float inv_T, float inv_T_log2e, const float* p
     __shared__ float s_m[8], s_s[8];
     __shared__ int s_i[8];
     const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    ptx::grid_dep_wait();
+    ptx::grid_dep_launch();
     float m = -INFINITY, s = 0.f;
     int idx = 0x7fffffff;
     auto fold = [&](float om, int oi, float os) {
@@ -343,6 +349,8 @@ lmhead_merge_kernel(int M, int P, float inv_T, float inv_T_log2e, const float* p
 __global__ void __launch_bounds__(1024, 1)
 lmhead_topk_kernel(int V, int topk, float inv_T, const float* logits, const float* lse, int32_t* topk_id,
                    float* topk_logprob) {
+    ptx::grid_dep_wait();
+    ptx::grid_dep_launch();
     __shared__ float s_v[32];
     __shared__ int s_i[32];
     __shared__ float s_prev_v;
@@ -391,6 +399,8 @@ lmhead_topk_kernel(int V, int topk, float inv_T, const float* logits, const floa
 __global__ void lmhead_gather_kernel(int n_gather, int M, int V, int H, const __nv_bfloat16* hidden,
                                      const __nv_bfloat16* W, const int32_t* gather_row, const int32_t* gather_tok,
                                      float* gather_logit, int* status) {
+    ptx::grid_dep_wait();
+    ptx::grid_dep_launch();
     const int g = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (g >= n_gather) return;
@@ -480,20 +490,21 @@ mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, c
         MIRROR_CUDA_OK(cudaFuncSetAttribute(lmhead_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
         ctx->lm_attr_set = true;
     }
-    lmhead_kernel<<<grid, kThreads, smem, stream>>>(tm_w_full, tm_w_grp, tm_h, p);
+    MIRROR_CUDA_OK(mirror_launch_pdl(lmhead_kernel, dim3(grid), dim3(kThreads), smem, stream, tm_w_full, tm_w_grp, tm_h, p));
     ctx->launches += 1;
     MIRROR_CUDA_OK(cudaGetLastError());
     if (after_gemm) MIRROR_CUDA_OK(cudaEventRecord(after_gemm, stream));
 
     float* lse_dst = lse ? lse : (topk > 0 ? lse_scratch : nullptr);
     if (argmax || maxlogit || lse_dst) {
-        lmhead_merge_kernel<<<M, 256, 0, stream>>>(M, (int)P, p.inv_T, p.inv_T_log2e, p.part_max, p.part_idx, p.part_sum,
-                                                   argmax, maxlogit, lse_dst);
+        MIRROR_CUDA_OK(mirror_launch_pdl(lmhead_merge_kernel, dim3(M), dim3(256), 0, stream, M, (int)P, p.inv_T, p.inv_T_log2e,
+                                         p.part_max, p.part_idx, p.part_sum, argmax, maxlogit, lse_dst));
         ctx->launches += 1;
         MIRROR_CUDA_OK(cudaGetLastError());
     }
     if (topk > 0) {
-        lmhead_topk_kernel<<<M, 1024, 0, stream>>>(V, topk, p.inv_T, logits_out, lse_dst, topk_id, topk_logprob);
+        MIRROR_CUDA_OK(mirror_launch_pdl(lmhead_topk_kernel, dim3(M), dim3(1024), 0, stream, V, topk, p.inv_T, logits_out, lse_dst,
+                                         topk_id, topk_logprob));
         ctx->launches += 1;
         MIRROR_CUDA_OK(cudaGetLastError());
     }
