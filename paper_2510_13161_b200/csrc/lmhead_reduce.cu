@@ -49,6 +49,7 @@ struct LmParams {
     int* part_idx;
     float* part_sum;
     int* status;
+    long long* timing;                  // developer aid (timing builds): per-CTA start / end stamps
 };
 
 struct Ctrl {
@@ -77,6 +78,9 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tm_w_full, const __grid_consta
     float* st_sum = (float*)(st_idx + 4 * kMaxChunkRows);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef MIRROR_ATTN_TIMING
+    if (p.timing && tid == 0) { unsigned long long g__; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g__) :: "memory"); p.timing[blockIdx.x * 2] = (long long)g__; }
+#endif
 
     // this CTA's slice of the vocabulary, in 8-row groups
     const int g0 = (int)(((long long)p.groups_total * blockIdx.x) / gridDim.x);
@@ -296,6 +300,9 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tm_w_full, const __grid_consta
         }
     }
 
+#ifdef MIRROR_ATTN_TIMING
+    if (p.timing && tid == 64) { unsigned long long g__; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g__) :: "memory"); p.timing[blockIdx.x * 2 + 1] = (long long)g__; }
+#endif
     ptx::tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -462,6 +469,10 @@ mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, c
     p.inv_T_log2e = p.inv_T * 1.4426950408889634f;
     p.logits_out = logits_out;
     p.status = ctx->d_status;
+    p.timing = nullptr;
+#ifdef MIRROR_ATTN_TIMING
+    if (const char* e = getenv("MIRROR_LM_TIMING_PTR")) p.timing = (long long*)strtoull(e, nullptr, 0);
+#endif
 
     int grid = ctx->num_sms;
     if (grid > p.groups_total) grid = p.groups_total;
