@@ -5,6 +5,8 @@
 // Eq. 3 applied to that branch).  Thread 0 then picks the longest branch (lowest index on ties) and the
 // deciding row R.  Greedy mode emits argmax[R]; speculative-sampling mode draws the extra token by an
 // inverse-CDF search over the vocabulary that the whole block cooperates on, all in fp64.
+#include <cooperative_groups.h>
+
 #include "mirror_internal.h"
 
 namespace {
@@ -202,36 +204,47 @@ accept_select_kernel(const __grid_constant__ AcceptTreeParams tp, const AcceptAr
 
 // ---------------------------------------------------------------------------------------------------
 // Lossless acceptance over a token tree: sequential multi-round rejection over the siblings of each accepted
-// row (the speculative-sampling rule of Sec. 3.1 applied to sibling sets, for tree drafts).  One block per
-// request walks down from the root.  At row r the current distribution m starts as the target's p_r; the
-// children of r are tested in node order against m: child c (token x, draft distribution q_c) passes iff
-// u_accept[c] * q_c[x] <= m[x] and the walk moves to c; a child that fails turns m into the normalised residual
-// max(0, m - q_c).  m is never stored: m[v] is re-evaluated from the logits, the rejected siblings' q rows and
-// their normalisers Z_i (fp64, same operation order per element as the definition), so a rejection costs one
-// pass over the vocabulary for Z and the final draw one more.
+// row (the speculative-sampling rule of Sec. 3.1 applied to sibling sets, for tree drafts).  A cluster of
+// kTreeCluster CTAs per request walks down from the root, every CTA holding one contiguous slice of the vocabulary.
+// At row r the current distribution m starts as the target's p_r; the children of r are tested in node order
+// against m: child c (token x, draft distribution q_c) passes iff u_accept[c] * q_c[x] <= m[x] and the walk moves to
+// c; a child that fails turns m into the normalised residual max(0, m - q_c).  m[v] is either re-evaluated from the
+// logits, the rejected siblings' q rows and their normalisers Z_i, or -- when the caller's workspace has room --
+// kept in fp64 scratch memory (two buffers, so that a residual without mass can be dropped); both follow the
+// definition's operation order per element.  A rejection costs one pass over the vocabulary for Z, the final draw
+// one more; the CTAs exchange their slice sums through distributed shared memory and add them in rank order, so
+// all of them see identical numbers, take identical decisions and stay in step (one hardware cluster barrier per
+// pass, nothing spins).
 // ---------------------------------------------------------------------------------------------------
 constexpr int kMaxRejected = MIRROR_MAX_BRANCHES;     // siblings rejected at one row
+constexpr int kTreeCluster = 8;                       // CTAs per request
 
 __global__ void __launch_bounds__(kThreads, 1)
 accept_tree_kernel(const __grid_constant__ AcceptTreeParams tp, const AcceptArgs a) {
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
     __shared__ double s_seg[kThreads];
     __shared__ double s_Z[kMaxRejected];
     __shared__ int s_rej[kMaxRejected];
     __shared__ int s_path[MIRROR_MAX_DEPTH];
-    __shared__ double s_tot, s_thr, s_excl;
-    __shared__ int s_pass, s_found, s_extra, s_last_pos;
+    __shared__ double s_slice[2];                     // this CTA's slice sum of the current pass (by pass parity): read by peers
+    __shared__ double s_excl;
+    __shared__ int s_pass, s_found, s_extra, s_last;
 
-    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int rank = (int)cluster.block_rank();
+    const int b = blockIdx.x / kTreeCluster, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n = tp.n, V = a.V;
     const int32_t* tok = a.tokens + (size_t)b * n;
     ptx::grid_dep_wait();
     ptx::grid_dep_launch();
-    const int S = (V + kThreads - 1) / kThreads;
-    const int v0 = min(tid * S, V), v1 = min(v0 + S, V);
+    // this CTA's slice of the vocabulary and this thread's contiguous segment of it
+    const int Vs = (V + kTreeCluster - 1) / kTreeCluster;
+    const int s0 = min(rank * Vs, V), s1 = min(s0 + Vs, V);
+    const int S = (Vs + kThreads - 1) / kThreads;
+    const int v0 = min(s0 + tid * S, s1), v1 = min(v0 + S, s1);
 
     int r = 0, A = 0, n_rej = 0, n_children = 0;
-    // With scratch memory the unnormalised residual of the last effective rejection is stored (two buffers, so that a
-    // residual without mass can be dropped) and m[v] = stored[v] / Z_last: the same operations as the definition.
+    uint32_t pass_no = 0;                          // vocabulary passes so far (identical in every CTA)
     double* const buf0 = a.tree_scratch ? a.tree_scratch + (size_t)b * 2 * V : nullptr;
     double* const buf1 = buf0 ? buf0 + V : nullptr;
     int cur = 0;                                   // buffer that holds the current residual (when n_rej > 0)
@@ -246,34 +259,45 @@ accept_tree_kernel(const __grid_constant__ AcceptTreeParams tp, const AcceptArgs
         }
         return m;
     };
-    // block-wide sum of f over the vocabulary in a fixed order: per-thread contiguous segments, then warp 0
-    // adds the segments in order
-    // (contiguous = true: per-thread contiguous segments, whose sums the inverse-CDF search then reuses; false: ids
-    // interleaved over the threads, which keeps the loads of a warp in one line -- any fixed order will do for a sum)
-    auto block_total = [&](auto f, bool contiguous) -> double {
+    // Sum of f over the whole vocabulary in a fixed order: per-thread partial sums over this CTA's slice (contiguous
+    // segments, whose sums the inverse-CDF search reuses, or ids interleaved over the threads, which keeps a warp's
+    // loads in one line), warp 0 adds them in order, then every CTA adds the eight slice sums in rank order.
+    // excl_out: sum of the slices before this CTA's.
+    auto cluster_total = [&](auto f, bool contiguous, double* excl_out) -> double {
         double part = 0.0;
         if (contiguous) {
             for (int v = v0; v < v1; ++v) part += f(v);
         } else {
             double p0 = 0.0, p1 = 0.0, p2 = 0.0, p3 = 0.0;
-            int v = tid;
-            for (; v + 3 * kThreads < V; v += 4 * kThreads) {
+            int v = s0 + tid;
+            for (; v + 3 * kThreads < s1; v += 4 * kThreads) {
                 p0 += f(v); p1 += f(v + kThreads); p2 += f(v + 2 * kThreads); p3 += f(v + 3 * kThreads);
             }
-            for (; v < V; v += kThreads) p0 += f(v);
+            for (; v < s1; v += kThreads) p0 += f(v);
             part = (p0 + p1) + (p2 + p3);
         }
         s_seg[tid] = part;
         __syncthreads();
+        const int par = pass_no & 1;
         if (warp == 0) {
             double lp = 0.0;
             for (int k = 0; k < 32; ++k) lp += s_seg[lane * 32 + k];
             double tot;
             warp_excl_scan(lp, lane, &tot);
-            if (lane == 0) s_tot = tot;
+            if (lane == 0) s_slice[par] = tot;
         }
-        __syncthreads();
-        return s_tot;
+        // (release / acquire at cluster scope: the slice sums and, with scratch memory, the residuals the peers wrote
+        // to global memory in this pass are visible after the barrier.  A buffer of this parity is written again two
+        // passes later, after every peer has passed the barrier in between and so finished reading it.)
+        cluster.sync();
+        double tot = 0.0, excl = 0.0;
+        for (int c = 0; c < kTreeCluster; ++c) {
+            if (c == rank) excl = tot;
+            tot += *cluster.map_shared_rank(&s_slice[par], c);
+        }
+        ++pass_no;
+        if (excl_out) *excl_out = excl;
+        return tot;
     };
 
     for (;;) {
@@ -288,6 +312,7 @@ accept_tree_kernel(const __grid_constant__ AcceptTreeParams tp, const AcceptArgs
             ++n_children;
             const float* qc = a.q_probs + ((size_t)b * (n - 1) + (c - 1)) * V;
             if (tid == 0) {
+                // (every CTA evaluates the test itself, from numbers that are identical in all of them)
                 const int x = tok[c];
                 int pass = 0;
                 if (x < 0 || x >= V) {
@@ -303,12 +328,12 @@ accept_tree_kernel(const __grid_constant__ AcceptTreeParams tp, const AcceptArgs
             if (s_pass) { next = c; break; }
             // rejected: normaliser of the residual (a residual without mass leaves m as it is)
             double* const nxt = !buf0 ? nullptr : ((n_rej > 0 && cur == 0) ? buf1 : buf0);      // the buffer not in use
-            const double Z = block_total([&](int v) {
+            const double Z = cluster_total([&](int v) {
                 double res = mass(lr, lse_r, v) - (double)qc[v];
                 res = (res > 0.0) ? res : 0.0;
                 if (nxt) nxt[v] = res;
                 return res;
-            }, false);
+            }, false, nullptr);
             if (Z > 0.0 && n_rej < kMaxRejected) {
                 if (tid == 0) { s_rej[n_rej] = c; s_Z[n_rej] = Z; }
                 if (nxt) cur = (nxt == buf1) ? 1 : 0;
@@ -328,20 +353,21 @@ accept_tree_kernel(const __grid_constant__ AcceptTreeParams tp, const AcceptArgs
         break;
     }
     const bool have_extra = (n_children > 0) || a.emit_bonus != 0;
-    if (tid == 0) { s_extra = -1; s_last_pos = -1; s_found = -1; }
+    if (tid == 0) { s_extra = -1; s_last = -1; s_found = -1; }
     __syncthreads();
     if (have_extra) {
-        // inverse-CDF draw from m at row r
+        // inverse-CDF draw from m at row r: the CTA whose slice holds the crossing searches it
         const size_t row = (size_t)b * n + r;
         const float* lr = a.logits + row * V;
         const double lse_r = (double)a.lse[row];
-        const double tot = block_total([&](int v) { return mass(lr, lse_r, v); }, true);
+        double excl_cta = 0.0;
+        const double tot = cluster_total([&](int v) { return mass(lr, lse_r, v); }, true, &excl_cta);
+        const double thr = (double)a.u_resample[row] * tot;
         if (warp == 0) {
-            const double thr = (double)a.u_resample[row] * tot;
             double lp = 0.0;
             for (int k = 0; k < 32; ++k) lp += s_seg[lane * 32 + k];
             double dummy;
-            double run = warp_excl_scan(lp, lane, &dummy);
+            double run = excl_cta + warp_excl_scan(lp, lane, &dummy);
             int found = -1;
             double found_excl = 0.0;
             for (int k = 0; k < 32; ++k) {
@@ -349,63 +375,72 @@ accept_tree_kernel(const __grid_constant__ AcceptTreeParams tp, const AcceptArgs
                 if (found < 0 && run + seg > thr) { found = lane * 32 + k; found_excl = run; }
                 run += seg;
             }
+            // only the first CTA whose cumulative sum passes the threshold holds the crossing
+            if (!(excl_cta <= thr)) found = -1;
             const unsigned mk = __ballot_sync(0xffffffffu, found >= 0);
             if (mk) {
                 const int src = __ffs(mk) - 1;
                 if (lane == src) { s_found = found; s_excl = found_excl; }
             }
-            if (lane == 0) s_thr = thr;
         }
         __syncthreads();
-        if (s_found >= 0) {
-            if (tid == s_found) {
-                const double thr = s_thr, excl = s_excl;
-                double loc = 0.0;
-                int pick = v1 - 1;
-                for (int v = v0; v < v1; ++v) {
-                    loc += mass(lr, lse_r, v);
-                    if (excl + loc > thr) { pick = v; break; }
-                }
-                s_extra = pick;
+        if (s_found >= 0 && tid == s_found) {
+            const double excl = s_excl;
+            double loc = 0.0;
+            int pick = v1 - 1;
+            for (int v = v0; v < v1; ++v) {
+                loc += mass(lr, lse_r, v);
+                if (excl + loc > thr) { pick = v; break; }
             }
-        } else {
-            // rounding left no crossing: take the last id with positive mass
+            *cluster.map_shared_rank(&s_extra, 0) = pick;              // hand the token to the CTA that writes the outputs
+        }
+        cluster.sync();
+        if (*cluster.map_shared_rank(&s_extra, 0) < 0) {
+            // rounding left the threshold above every cumulative sum (the same in every CTA): the last id with positive mass
             int last = -1;
             for (int v = v0; v < v1; ++v)
                 if (mass(lr, lse_r, v) > 0.0) last = v;
-            if (last >= 0) atomicMax(&s_last_pos, last);
-            __syncthreads();
-            if (tid == 0) s_extra = s_last_pos;
+            if (last >= 0) atomicMax(&s_last, last);
+            cluster.sync();
+            if (rank == 0 && tid == 0) {
+                int best_last = -1;
+                for (int c = 0; c < kTreeCluster; ++c) best_last = max(best_last, *cluster.map_shared_rank(&s_last, c));
+                s_extra = best_last;
+            }
         }
     }
     __syncthreads();
 
     const int gamma = tp.gamma;
-    if (tid <= gamma) {
-        int e = -1;
-        if (tid < A) e = tok[s_path[tid]];
-        else if (tid == A && have_extra) e = s_extra;
-        a.out.emitted[(size_t)b * (gamma + 1) + tid] = e;
-        if (tid < gamma) a.out.accepted_nodes[(size_t)b * gamma + tid] = (tid < A) ? s_path[tid] : -1;
-    }
-    if (tid == 0) {
-        // the lowest-index branch that contains the accepted path
-        int best = 0;
-        for (int i = 0; i < tp.n_branches; ++i) {
-            bool ok = tp.path_len[i] >= A;
-            for (int k = 0; k < A && ok; ++k) ok = (tp.path[i][k] == s_path[k]);
-            if (ok) { best = i; break; }
+    if (rank == 0) {
+        if (tid <= gamma) {
+            int e = -1;
+            if (tid < A) e = tok[s_path[tid]];
+            else if (tid == A && have_extra) e = s_extra;
+            a.out.emitted[(size_t)b * (gamma + 1) + tid] = e;
+            if (tid < gamma) a.out.accepted_nodes[(size_t)b * gamma + tid] = (tid < A) ? s_path[tid] : -1;
         }
-        a.out.n_accepted[b] = A;
-        a.out.best_branch[b] = best;
-        a.out.decide_row[b] = r;
-        a.out.n_emitted[b] = A + (have_extra ? 1 : 0);
-        int slot = -1;
-        if (have_extra && a.cand_ids)
-            for (int k = 0; k < a.n_cand; ++k)
-                if (a.cand_ids[((size_t)b * n + r) * a.n_cand + k] == s_extra) { slot = k; break; }
-        a.out.reuse_slot[b] = slot;
+        if (tid == 0) {
+            // the lowest-index branch that contains the accepted path
+            int best = 0;
+            for (int i = 0; i < tp.n_branches; ++i) {
+                bool ok = tp.path_len[i] >= A;
+                for (int k = 0; k < A && ok; ++k) ok = (tp.path[i][k] == s_path[k]);
+                if (ok) { best = i; break; }
+            }
+            a.out.n_accepted[b] = A;
+            a.out.best_branch[b] = best;
+            a.out.decide_row[b] = r;
+            a.out.n_emitted[b] = A + (have_extra ? 1 : 0);
+            int slot = -1;
+            if (have_extra && a.cand_ids)
+                for (int k = 0; k < a.n_cand; ++k)
+                    if (a.cand_ids[((size_t)b * n + r) * a.n_cand + k] == s_extra) { slot = k; break; }
+            a.out.reuse_slot[b] = slot;
+        }
     }
+    // no CTA may leave while a peer can still read its shared memory
+    cluster.sync();
 }
 
 }  // namespace
@@ -437,8 +472,23 @@ mirror_status mirror_accept_launch(mirror_ctx* ctx, const mirror_tree* tree, con
     a.out = *out;
     a.tree_scratch = tree_scratch;
     a.status = ctx->d_status;
-    if (in->mode == MIRROR_ACCEPT_SPEC_TREE) MIRROR_CUDA_OK(mirror_launch_pdl(accept_tree_kernel, dim3(tree->batch), dim3(kThreads), 0, stream, tp, a));
-    else MIRROR_CUDA_OK(mirror_launch_pdl(accept_select_kernel, dim3(tree->batch), dim3(kThreads), 0, stream, tp, a));
+    if (in->mode == MIRROR_ACCEPT_SPEC_TREE) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)tree->batch * kTreeCluster);
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = 0;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = kTreeCluster;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 2;
+        MIRROR_CUDA_OK(cudaLaunchKernelEx(&cfg, accept_tree_kernel, tp, a));
+    } else MIRROR_CUDA_OK(mirror_launch_pdl(accept_select_kernel, dim3(tree->batch), dim3(kThreads), 0, stream, tp, a));
     ctx->launches += 1;
     MIRROR_CUDA_OK(cudaGetLastError());
     return MIRROR_OK;
