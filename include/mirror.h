@@ -213,6 +213,26 @@ mirror_status mirror_lmhead_reduce_noalloc(int device, const void* hidden, int M
 mirror_status mirror_accept_select(mirror_ctx* ctx, const mirror_tree* tree, const mirror_accept_in* in,
                                    const mirror_accept_out* out, void* stream);
 
+/* Early-exit tap (Sec. 3.1, Eq. 5 and Eq. 6): the LM head applied to the hidden states of an intermediate layer,
+ * reduced per row to the Top-kappa message M_t that the token channel carries to the draft.
+ *   hidden_le        bf16 [M, H]: early-exit hidden rows (one per window position / tree node)
+ *   msg_ids          int32 [M, kappa]: candidate ids ordered by (logit descending, id ascending)
+ *   msg_logprob_bf16 bf16 [M, kappa]: their log-probabilities logit/T - lse under the early-exit proxy (the token
+ *                    channel's payload type)
+ * kappa <= MIRROR_MAX_TOPK.  Needs a workspace sized for MIRROR_WS_LMHEAD_LOGITS with M rows (the selection runs over
+ * the spilled fp32 logits).  msg_ids is what mirror_accept_select / mirror_verify_step take as cand_ids (n_cand =
+ * kappa) for the reuse decision of the same rows. */
+mirror_status mirror_early_exit_tap(mirror_ctx* ctx, const void* hidden_le, int M, const void* W, int kappa,
+                                    int32_t* msg_ids, void* msg_logprob_bf16, void* stream);
+
+/* Overlap mass (Eq. 7): omega[row] = sum over the row's kappa message ids y of q(y), with
+ * q(y) = exp(logits_final[row][y]/T - lse_final[row]) the target's final distribution of that row; by Proposition 1,
+ * 1 - omega is the probability that a rejection at the row falls back to a fresh rollout.
+ *   logits_final fp32 [M, V], lse_final fp32 [M] (e.g. from mirror_lmhead_reduce with logits_out), msg_ids int32
+ *   [M, kappa], omega fp32 [M] (device).  Ids outside [0, V) are skipped and reported as a device-side check. */
+mirror_status mirror_overlap_mass(mirror_ctx* ctx, const float* logits_final, const float* lse_final,
+                                  const int32_t* msg_ids, int M, int kappa, float* omega, void* stream);
+
 /* One whole verify step on one stream: attention over all layers -> LM head rows -> reductions -> acceptance.
  *   hidden   bf16 [B*n, H], or NULL to feed the last layer's attention output (requires Hq*d == H)
  *   attn_out bf16 [L, B, n, Hq, d]  (required: it is also the chained LM-head input)

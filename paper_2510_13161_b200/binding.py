@@ -24,7 +24,7 @@ EXPORTS = [
     "mirror_create", "mirror_destroy", "mirror_workspace_bytes", "mirror_set_workspace",
     "mirror_attn_verify", "mirror_lmhead_reduce", "mirror_accept_select", "mirror_verify_step",
     "mirror_device_status", "mirror_launch_count", "mirror_status_str", "mirror_set_stage_events",
-    "mirror_lmhead_reduce_noalloc",
+    "mirror_lmhead_reduce_noalloc", "mirror_early_exit_tap", "mirror_overlap_mass",
 ]
 
 
@@ -255,6 +255,28 @@ class Mirror:
                      _ptr(u_resample, torch.float32, "u_resample"), _ptr(cand_ids, torch.int32, "cand_ids"), n_cand)
         a._refs = (target_argmax, logits, lse, q_probs, u_accept, u_resample, cand_ids)
         return a
+
+    def mirror_early_exit_tap(self, hidden_le: torch.Tensor, W: torch.Tensor, kappa: int, stream=None):
+        """Top-kappa message of the early-exit proxy: (ids int32 [M, kappa], log-probs bf16 [M, kappa])."""
+        M = hidden_le.shape[0]
+        ids = torch.empty((M, kappa), dtype=torch.int32, device=hidden_le.device)
+        lp = torch.empty((M, kappa), dtype=torch.bfloat16, device=hidden_le.device)
+        t = Tree(1, M if M <= 128 else 128, 0, 0, None, None)
+        t.batch, t.n_nodes = (M + 127) // 128, min(M, 128)      # sizes only: batch * n_nodes >= M
+        self.ensure_workspace(t, None, WS_LMHEAD_LOGITS)
+        _check(self.lib.mirror_early_exit_tap(self._ctx, _ptr(hidden_le, torch.bfloat16, "hidden_le"), M,
+                                              _ptr(W, torch.bfloat16, "W"), kappa, _ptr(ids, torch.int32, "msg_ids"),
+                                              _ptr(lp, torch.bfloat16, "msg_logprob"), _stream(stream)), "mirror_early_exit_tap")
+        return ids, lp
+
+    def mirror_overlap_mass(self, logits_final: torch.Tensor, lse_final: torch.Tensor, msg_ids: torch.Tensor, stream=None):
+        """Eq. 7 per row: mass of the final distribution on the message's ids (fp32 [M])."""
+        M, kappa = msg_ids.shape
+        omega = torch.empty(M, dtype=torch.float32, device=msg_ids.device)
+        _check(self.lib.mirror_overlap_mass(self._ctx, _ptr(logits_final, torch.float32, "logits_final"),
+                                            _ptr(lse_final, torch.float32, "lse_final"), _ptr(msg_ids, torch.int32, "msg_ids"),
+                                            M, kappa, _ptr(omega, torch.float32, "omega"), _stream(stream)), "mirror_overlap_mass")
+        return omega
 
     def mirror_accept_select(self, tree: Tree, acc: AcceptIn, out: Optional[AcceptResult] = None, stream=None,
                              tree_scratch: bool = False) -> AcceptResult:

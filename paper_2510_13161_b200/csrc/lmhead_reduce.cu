@@ -355,7 +355,7 @@ lmhead_merge_kernel(int M, int P, float inv_T, float inv_T_log2e, const float* p
 // previous pick" in the order (logit descending, id ascending).  One block per row.
 __global__ void __launch_bounds__(1024, 1)
 lmhead_topk_kernel(int V, int topk, float inv_T, const float* logits, const float* lse, int32_t* topk_id,
-                   float* topk_logprob) {
+                   float* topk_logprob, __nv_bfloat16* topk_logprob_bf16) {
     ptx::grid_dep_wait();
     ptx::grid_dep_launch();
     __shared__ float s_v[32];
@@ -395,7 +395,9 @@ lmhead_topk_kernel(int V, int topk, float inv_T, const float* logits, const floa
             if (lane == 0) {
                 s_prev_v = bv; s_prev_i = bi;
                 topk_id[(size_t)row * topk + k] = bi;
-                topk_logprob[(size_t)row * topk + k] = bv * inv_T - lse[row];
+                const float lp = bv * inv_T - lse[row];
+                if (topk_logprob) topk_logprob[(size_t)row * topk + k] = lp;
+                if (topk_logprob_bf16) topk_logprob_bf16[(size_t)row * topk + k] = __float2bfloat16_rn(lp);      // token-channel payload
             }
         }
         __syncthreads();
@@ -445,7 +447,7 @@ mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, c
                                    int32_t* argmax, float* maxlogit, float* lse, int32_t* topk_id,
                                    float* topk_logprob, float* gather_logit, float* logits_out,
                                    void* partial_ws, size_t partial_bytes, float* lse_scratch, cudaStream_t stream,
-                                   cudaEvent_t after_gemm) {
+                                   cudaEvent_t after_gemm, void* topk_logprob_bf16) {
     const int V = ctx->desc.vocab, H = ctx->desc.hidden;
     LmParams p;
     p.M = M; p.V = V; p.H = H;
@@ -515,7 +517,7 @@ mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, c
     }
     if (topk > 0) {
         MIRROR_CUDA_OK(mirror_launch_pdl(lmhead_topk_kernel, dim3(M), dim3(1024), 0, stream, V, topk, p.inv_T, logits_out, lse_dst,
-                                         topk_id, topk_logprob));
+                                         topk_id, topk_logprob, (__nv_bfloat16*)topk_logprob_bf16));
         ctx->launches += 1;
         MIRROR_CUDA_OK(cudaGetLastError());
     }

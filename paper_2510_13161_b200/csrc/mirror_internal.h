@@ -61,7 +61,7 @@ mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, c
                                    int32_t* argmax, float* maxlogit, float* lse, int32_t* topk_id,
                                    float* topk_logprob, float* gather_logit, float* logits_out,
                                    void* partial_ws, size_t partial_bytes, float* lse_scratch, cudaStream_t stream,
-                                   cudaEvent_t after_gemm = nullptr);
+                                   cudaEvent_t after_gemm = nullptr, void* topk_logprob_bf16 = nullptr);
 mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const MirrorTreeInfo& ti,
                                  const void* q, const void* k_new, const void* v_new, void* out, float* lse_out,
                                  float* partial_ws, int* ticket_ws, size_t ticket_ints, cudaStream_t stream);
