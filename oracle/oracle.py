@@ -178,6 +178,26 @@ def accept_tree(tokens, logits, lse, q_probs, u_accept, u_resample, parent, max_
     return o
 
 
+def kv_commit(k_pool, v_pool, page_table, prefix_len, k_new, v_new, accepted_nodes, n_accepted, page_size: int = 16):
+    """Roll-forward of the paged cache after a verify step (Sec. 3.1): for every request the K/V rows of the root and
+    of its accepted nodes, in path order, become tokens prefix_len .. prefix_len + A of every layer and head; the
+    prefix grows by A + 1.  Pools are [L, num_pages, Hkv, page, d] arrays of bf16 bit patterns (uint16), k_new / v_new
+    [L, B, n, Hkv, d].  Returns new (k_pool, v_pool, prefix_len); the inputs are not modified."""
+    k_pool = np.array(k_pool, copy=True); v_pool = np.array(v_pool, copy=True)
+    page_table = np.asarray(page_table); prefix_len = np.array(prefix_len, copy=True)
+    accepted_nodes = np.asarray(accepted_nodes); n_accepted = np.asarray(n_accepted)
+    B = prefix_len.shape[0]
+    for b in range(B):
+        nodes = [0] + [int(c) for c in accepted_nodes[b, :int(n_accepted[b])]]
+        for j, node in enumerate(nodes):
+            pos = int(prefix_len[b]) + j
+            page, slot = int(page_table[b, pos // page_size]), pos % page_size
+            k_pool[:, page, :, slot, :] = k_new[:, b, node]
+            v_pool[:, page, :, slot, :] = v_new[:, b, node]
+        prefix_len[b] += len(nodes)
+    return k_pool, v_pool, prefix_len
+
+
 def overlap_mass(q_final, ids) -> float:
     """Eq. 7: Omega_kappa, the final distribution's mass on the early-exit Top-kappa ids."""
     q_final = _c(q_final, np.float64); ids = _c(ids, np.int32)

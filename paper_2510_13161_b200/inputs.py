@@ -122,10 +122,11 @@ def draw_prefix_lens(cfg: VerifyConfig, seed: int) -> torch.Tensor:
     return torch.randint(cfg.prefix_lo, cfg.prefix_hi + 1, (cfg.batch,), generator=g, dtype=torch.int32)
 
 
-def gen_page_table(prefix_len: torch.Tensor, seed: int, spare_pages: int = 3, shuffle: bool = True):
+def gen_page_table(prefix_len: torch.Tensor, seed: int, spare_pages: int = 3, shuffle: bool = True, headroom: int = 0):
     """Physical pages handed out by a seeded random permutation of the pool (a fragmented
-    cache); unused table slots hold -1.  Returns (page_table [B,max_pages] int32, num_pages)."""
-    pages = [(int(l) + PAGE_SIZE - 1) // PAGE_SIZE for l in prefix_len]
+    cache); unused table slots hold -1.  `headroom` tokens beyond each prefix get pages too (room to commit
+    accepted tokens).  Returns (page_table [B,max_pages] int32, num_pages)."""
+    pages = [(int(l) + headroom + PAGE_SIZE - 1) // PAGE_SIZE for l in prefix_len]
     total = sum(pages)
     num_pages = total + spare_pages
     max_pages = max(1, max(pages) if pages else 1)
@@ -170,7 +171,7 @@ class VerifyInputs:
 def gen_verify_inputs(cfg: VerifyConfig, seed: int = 0, device: str = "cpu", *,
                       parent: Optional[Sequence[int]] = None, with_lm_head: bool = True,
                       layers: Optional[int] = None, shuffle_pages: bool = True,
-                      q_std: float = 1.0, force_hidden: bool = False) -> VerifyInputs:
+                      q_std: float = 1.0, force_hidden: bool = False, headroom: int = 0) -> VerifyInputs:
     """Draw one verify-step problem.  `layers` overrides cfg.layers (parity tests on big
     configs generate a few layers only; each layer's tensors depend on (seed, layer) alone,
     so layer l is the same tensor whatever `layers` is)."""
@@ -180,7 +181,7 @@ def gen_verify_inputs(cfg: VerifyConfig, seed: int = 0, device: str = "cpu", *,
     n = len(par)
     bf = torch.bfloat16
     prefix_len = draw_prefix_lens(cfg, seed)
-    page_table, num_pages = gen_page_table(prefix_len, seed, shuffle=shuffle_pages)
+    page_table, num_pages = gen_page_table(prefix_len, seed, shuffle=shuffle_pages, headroom=headroom)
 
     q = torch.empty((L, B, n, Hq, d), dtype=bf, device=device)
     k_pool = torch.empty((L, num_pages, Hkv, PAGE_SIZE, d), dtype=bf, device=device)

@@ -209,3 +209,38 @@ def test_single_branch_reduces_to_plain_causal_decode():
         ref = causal_attention(qf[:, h], np.concatenate([kp, knf[:, h // G]]), np.concatenate([vp, vnf[:, h // G]]), 33,
                                1 / np.sqrt(cfg.head_dim))
         np.testing.assert_allclose(out[0, :, h], ref, atol=1e-12)
+
+
+def test_kv_commit_then_root_only_attention_equals_attention_over_the_accepted_path():
+    """Roll-forward pin: after committing the root and an accepted path into the paged cache, a fresh query that sees
+    only the (longer) prefix must get exactly what it would get from the old prefix plus those tree tokens as visible
+    tree nodes -- the commit puts the right rows at the right positions of the right pages, for every layer and head."""
+    from paper_2510_13161_b200 import inputs as I
+    cfg = I.VerifyConfig("c", 256, 4, 2, 64, 2, 3, 20, 70, 2, 3, 512, "greedy")
+    x = I.gen_verify_inputs(cfg, 3, "cpu", with_lm_head=False, headroom=cfg.gamma + 1)
+    n = cfg.n_nodes
+    kp, vp = I.bf16_bits(x.k_pool), I.bf16_bits(x.v_pool)
+    kn, vn = I.bf16_bits(x.k_new), I.bf16_bits(x.v_new)
+    pt, pl = x.page_table.numpy(), x.prefix_len.numpy()
+    accepted = np.array([[1, 2, 3], [4, 5, -1], [-1, -1, -1]], np.int32)      # paths of length 3, 2, 0
+    n_acc = np.array([3, 2, 0], np.int32)
+    kp2, vp2, pl2 = O.kv_commit(kp, vp, pt, pl, kn, vn, accepted, n_acc)
+    assert (pl2 == pl + n_acc + 1).all() and (kp == I.bf16_bits(x.k_pool)).all()       # inputs untouched
+    parent = x.parent
+    anc, _ = O.tree(parent)
+    scale = 1.0 / np.sqrt(cfg.head_dim)
+    q = I.bf16_bits(x.q)
+    for layer in range(cfg.layers):
+        # (a) new cache, every node a root-like query that sees no tree token but itself; node 0's row is the probe
+        eye = np.eye(n, dtype=np.uint8)
+        out_new, _, _ = O.attention_layer(q[layer], kp2[layer], vp2[layer], pt, pl2, kn[layer], vn[layer], eye, scale)
+        for b in range(cfg.batch):
+            path = [0] + [int(c) for c in accepted[b, :n_acc[b]]]
+            # (b) old cache, the probe row sees exactly the committed tree tokens plus itself
+            vis = np.eye(n, dtype=np.uint8)
+            probe = n - 1                                  # a node outside every committed path
+            assert probe not in path
+            vis[probe, path] = 1
+            out_old, _, _ = O.attention_layer(q[layer], kp[layer], vp[layer], pt, pl, kn[layer], vn[layer], vis, scale)
+            # the same query vector must be used on both sides: compare row `probe` of (b) with row `probe` of (a)
+            np.testing.assert_allclose(out_new[b, probe], out_old[b, probe], rtol=1e-9, atol=1e-12)
