@@ -233,6 +233,21 @@ mirror_status mirror_early_exit_tap(mirror_ctx* ctx, const void* hidden_le, int 
 mirror_status mirror_overlap_mass(mirror_ctx* ctx, const float* logits_final, const float* lse_final,
                                   const int32_t* msg_ids, int M, int kappa, float* omega, void* stream);
 
+/* Roll-forward of the paged cache after a verify step (Sec. 3.1): for every request b the K/V rows of the root
+ * (node 0, the last committed token) and of its accepted nodes, in path order, are written as tokens
+ * prefix_len[b] .. prefix_len[b] + n_accepted[b] of every layer and KV head, then prefix_len[b] += n_accepted[b] + 1.
+ *   kv              the cache: k_pool / v_pool are WRITTEN here (the struct's const is not honoured by this call);
+ *                   page_table must already hold pages for the new positions (it is not modified);
+ *                   kv->prefix_len is ignored in favour of the prefix_len argument
+ *   k_new, v_new    bf16 [L, B, n, Hkv, d]: the tree's own K/V of the step just verified
+ *   accepted_nodes  int32 [B, gamma], n_accepted int32 [B]: as written by mirror_accept_select / mirror_verify_step
+ *   prefix_len      int32 [B], device, read and updated in place
+ * A position beyond max_pages_per_req*16, a page outside the pool or a node id outside the tree is skipped and
+ * reported through mirror_device_status.  Enqueues two small kernels; runs after the step on the same stream. */
+mirror_status mirror_kv_commit(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const void* k_new,
+                               const void* v_new, const int32_t* accepted_nodes, const int32_t* n_accepted,
+                               int32_t* prefix_len, void* stream);
+
 /* One whole verify step on one stream: attention over all layers -> LM head rows -> reductions -> acceptance.
  *   hidden   bf16 [B*n, H], or NULL to feed the last layer's attention output (requires Hq*d == H)
  *   attn_out bf16 [L, B, n, Hq, d]  (required: it is also the chained LM-head input)

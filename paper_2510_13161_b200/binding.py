@@ -24,7 +24,7 @@ EXPORTS = [
     "mirror_create", "mirror_destroy", "mirror_workspace_bytes", "mirror_set_workspace",
     "mirror_attn_verify", "mirror_lmhead_reduce", "mirror_accept_select", "mirror_verify_step",
     "mirror_device_status", "mirror_launch_count", "mirror_status_str", "mirror_set_stage_events",
-    "mirror_lmhead_reduce_noalloc", "mirror_early_exit_tap", "mirror_overlap_mass",
+    "mirror_lmhead_reduce_noalloc", "mirror_early_exit_tap", "mirror_overlap_mass", "mirror_kv_commit",
 ]
 
 
@@ -277,6 +277,13 @@ class Mirror:
                                             _ptr(lse_final, torch.float32, "lse_final"), _ptr(msg_ids, torch.int32, "msg_ids"),
                                             M, kappa, _ptr(omega, torch.float32, "omega"), _stream(stream)), "mirror_overlap_mass")
         return omega
+
+    def mirror_kv_commit(self, kv: KV, tree: Tree, k_new, v_new, res: "AcceptResult", prefix_len: torch.Tensor, stream=None):
+        """Append the root and the accepted path of `res` to the paged cache and advance prefix_len in place."""
+        _check(self.lib.mirror_kv_commit(self._ctx, C.byref(kv), C.byref(tree), _ptr(k_new, torch.bfloat16, "k_new"),
+                                         _ptr(v_new, torch.bfloat16, "v_new"), _ptr(res.accepted_nodes, torch.int32, "accepted_nodes"),
+                                         _ptr(res.n_accepted, torch.int32, "n_accepted"), _ptr(prefix_len, torch.int32, "prefix_len"),
+                                         _stream(stream)), "mirror_kv_commit")
 
     def mirror_accept_select(self, tree: Tree, acc: AcceptIn, out: Optional[AcceptResult] = None, stream=None,
                              tree_scratch: bool = False) -> AcceptResult:
