@@ -985,7 +985,7 @@ __global__ void __launch_bounds__(kMergeThreads) attn_merge_kernel(const AttnPar
 
 mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const MirrorTreeInfo& ti,
                                  const void* q, const void* k_new, const void* v_new, void* out, float* lse_out,
-                                 float* partial_ws, int* ticket_ws, size_t ticket_ints, cudaStream_t stream) {
+                                 float* partial_ws, cudaStream_t stream) {
     const int D = ctx->desc.head_dim, Hkv = ctx->desc.n_kv_heads, Hq = ctx->desc.n_q_heads;
     AttnParams p;
     p.L = kv->num_layers; p.B = tree->batch; p.n = ti.n; p.Hq = Hq; p.Hkv = Hkv; p.G = Hq / Hkv;
@@ -1010,14 +1010,13 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
     p.k_pool = (const __nv_bfloat16*)kv->k_pool; p.v_pool = (const __nv_bfloat16*)kv->v_pool;
     p.k_new = (const __nv_bfloat16*)k_new; p.v_new = (const __nv_bfloat16*)v_new;
     p.out = (__nv_bfloat16*)out; p.lse_out = lse_out;
-    p.partial = partial_ws; (void)ticket_ws; p.status = ctx->d_status;
+    p.partial = partial_ws; p.status = ctx->d_status;
     p.timing = nullptr;
     p.timing_exit = 0;
 #ifdef MIRROR_ATTN_TIMING
     if (const char* e = getenv("MIRROR_ATTN_TIMING_PTR")) p.timing = (long long*)strtoull(e, nullptr, 0);
     if (const char* e = getenv("MIRROR_ATTN_EXIT")) p.timing_exit = atoi(e);
 #endif
-    (void)ticket_ints;
     if (p.B > kMaxBatch) return MIRROR_ERR_SHAPE;
 
     AttnTree at;

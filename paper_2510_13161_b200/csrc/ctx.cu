@@ -75,8 +75,7 @@ extern "C" mirror_status mirror_device_status(mirror_ctx* ctx, int* code, int* d
     if (detail) *detail = h[1];
     if (h[0] != 0) {
         MIRROR_CUDA_OK(cudaMemset(ctx->d_status, 0, sizeof h));
-        // arrival counters may be stale after an aborted launch
-        if (ctx->ws) MIRROR_CUDA_OK(cudaMemset(ctx->ws, 0, ctx->ws_bytes < kWsTicketBytes ? ctx->ws_bytes : kWsTicketBytes));
+        if (ctx->ws) MIRROR_CUDA_OK(cudaMemset(ctx->ws, 0, ctx->ws_bytes < kWsZeroedBytes ? ctx->ws_bytes : kWsZeroedBytes));
     }
     return MIRROR_OK;
 }
@@ -142,8 +141,8 @@ mirror_status mirror_build_tree(const mirror_tree* tree, MirrorTreeInfo* info) {
 void mirror_ws_layout(const mirror_ctx* ctx, size_t M, MirrorWsLayout* out, size_t B) {
     MirrorWsLayout L;
     size_t at = 0;
-    L.attn_ticket = at;
-    at += kWsTicketBytes;
+    L.zeroed = at;
+    at += kWsZeroedBytes;
     L.attn_partial = at;
     // two partial slots per CTA (a CTA's range of KV tiles cuts at most two units), 128 rows each
     L.attn_partial_bytes = align_up((size_t)ctx->num_sms * 2 * 128 * (size_t)(ctx->desc.head_dim + 4) * sizeof(float), 256);
@@ -188,9 +187,8 @@ extern "C" mirror_status mirror_set_workspace(mirror_ctx* ctx, void* dev_ptr, si
     ctx->ws = dev_ptr;
     ctx->ws_bytes = dev_ptr ? bytes : 0;
     if (dev_ptr) {
-        // arrival counters live at the front of the workspace and must start at zero
         MIRROR_CUDA_OK(cudaSetDevice(ctx->device));
-        MIRROR_CUDA_OK(cudaMemset(dev_ptr, 0, bytes < kWsTicketBytes ? bytes : kWsTicketBytes));
+        MIRROR_CUDA_OK(cudaMemset(dev_ptr, 0, bytes < kWsZeroedBytes ? bytes : kWsZeroedBytes));
     }
     return MIRROR_OK;
 }

@@ -39,11 +39,11 @@ struct mirror_ctx {
 mirror_status mirror_build_tree(const mirror_tree* tree, MirrorTreeInfo* info);
 
 // Workspace carving.  The layout depends only on the model shape and the row count M, so every entry
-// point finds the same regions: [arrival counters | attention partials | LM-head partials | lse, argmax
-// scratch | fp32 logits | fp64 acceptance scratch].  Offsets are 256-byte aligned; the counters are zeroed when the workspace is attached.
-constexpr size_t kWsTicketBytes = 4u << 20;
+// point finds the same regions: [zeroed words | attention split records | LM-head partials | lse, argmax
+// scratch | fp32 logits | fp64 acceptance scratch].  Offsets are 256-byte aligned; the first region is zeroed when the workspace is attached.
+constexpr size_t kWsZeroedBytes = 4096;     // words at the front of the workspace that are zero between launches (none in use now)
 struct MirrorWsLayout {
-    size_t attn_ticket = 0;                              // arrival counters (kWsTicketBytes)
+    size_t zeroed = 0;                                   // kWsZeroedBytes of zeroed words
     size_t attn_partial = 0, attn_partial_bytes = 0;     // split-KV partial accumulators
     size_t lm_partial = 0, lm_partial_bytes = 0;         // per-(CTA, warp) row partials
     size_t lse = 0, argmax = 0;                          // [M] scratch each
@@ -64,7 +64,7 @@ mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, c
                                    cudaEvent_t after_gemm = nullptr, void* topk_logprob_bf16 = nullptr);
 mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const MirrorTreeInfo& ti,
                                  const void* q, const void* k_new, const void* v_new, void* out, float* lse_out,
-                                 float* partial_ws, int* ticket_ws, size_t ticket_ints, cudaStream_t stream);
+                                 float* partial_ws, cudaStream_t stream);
 
 // bf16 tensor map with 128-byte swizzle.  dims/box are innermost-first; strides_bytes[i] is the byte
 // stride of dimension i+1 (rank-1 entries).

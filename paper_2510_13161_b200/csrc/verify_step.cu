@@ -32,8 +32,7 @@ extern "C" mirror_status mirror_attn_verify(mirror_ctx* ctx, const mirror_kv* kv
     if (!ctx->ws || ctx->ws_bytes < L.end_attn) return MIRROR_ERR_WORKSPACE;
     MIRROR_CUDA_OK(cudaSetDevice(ctx->device));
     uint8_t* ws = (uint8_t*)ctx->ws;
-    return mirror_attn_launch(ctx, kv, tree, ti, q, k_new, v_new, out, lse_out, (float*)(ws + L.attn_partial),
-                              (int*)(ws + L.attn_ticket), kWsTicketBytes / sizeof(int), (cudaStream_t)stream);
+    return mirror_attn_launch(ctx, kv, tree, ti, q, k_new, v_new, out, lse_out, (float*)(ws + L.attn_partial), (cudaStream_t)stream);
 }
 
 extern "C" mirror_status mirror_verify_step(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree,
@@ -63,8 +62,7 @@ extern "C" mirror_status mirror_verify_step(mirror_ctx* ctx, const mirror_kv* kv
 
     const bool ev = ctx->stage_ev_on;
     if (ev) MIRROR_CUDA_OK(cudaEventRecord(ctx->stage_ev[0], s));
-    st = mirror_attn_launch(ctx, kv, tree, ti, q, k_new, v_new, attn_out, nullptr, (float*)(ws + L.attn_partial),
-                            (int*)(ws + L.attn_ticket), kWsTicketBytes / sizeof(int), s);
+    st = mirror_attn_launch(ctx, kv, tree, ti, q, k_new, v_new, attn_out, nullptr, (float*)(ws + L.attn_partial), s);
     if (st != MIRROR_OK) return st;
     if (ev) MIRROR_CUDA_OK(cudaEventRecord(ctx->stage_ev[1], s));
 
