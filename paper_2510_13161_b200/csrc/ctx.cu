@@ -149,7 +149,10 @@ void mirror_ws_layout(const mirror_ctx* ctx, size_t M, MirrorWsLayout* out, size
     at += L.attn_partial_bytes;
     L.end_attn = at;
     L.lm_partial = at;
-    L.lm_partial_bytes = align_up((size_t)ctx->num_sms * M * 12, 256);
+    // one partial per CTA (weight-stream kernel) or per 128-row vocabulary tile (pair kernel), whichever is more
+    const size_t n_part = (size_t)(ctx->num_sms > mirror_lmhead_pair_partials(ctx->desc.vocab) ? ctx->num_sms
+                                                                                                : mirror_lmhead_pair_partials(ctx->desc.vocab));
+    L.lm_partial_bytes = align_up(n_part * M * 12, 256);
     at += L.lm_partial_bytes;
     L.lse = at;
     at += align_up(M * sizeof(float), 256);

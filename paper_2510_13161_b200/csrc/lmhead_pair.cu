@@ -1,0 +1,442 @@
+// LM head for many hidden rows (Eq. 1 over the B * (1 + kappa*gamma) rows of a batched verify step): the same fused
+// GEMM + row reductions as lmhead_kernel, issued on CTA PAIRS (tcgen05 cta_group::2).
+//
+// Why a second kernel: with M >= ~200 rows the LM head stops being a weight stream and becomes a GEMM, and a
+// single-CTA 128 x N tile asks the L2 for more bytes per flop than it delivers.  A pair of CTAs (the two SMs of a
+// TPC) runs one UMMA of 256 vocabulary rows x N hidden rows per K step: each CTA stages its own 128 weight rows and
+// only HALF of the hidden rows, and the tensor cores of both SMs read both halves.  Per K block of 64 a CTA loads
+// 16 KB + N/2 * 128 B for 128 * N * 64 * 2 flop: 131 flop/B at N = 256 against 79 flop/B before.
+//
+// Work unit = (256-row vocabulary tile, row chunk of N <= 256 hidden rows).  Units are dealt to the pairs round-robin
+// in the order (tile major, chunk minor), so that at any time the pairs work on a handful of neighbouring tiles and
+// the chunks of one tile run on different pairs at the same moment: every weight tile leaves HBM once and the other
+// chunks hit it in L2.  Each unit leaves one partial (max, argmax, sum-exp) per hidden row and 128-row half tile;
+// lmhead_merge_kernel folds them in a fixed order, so the result does not depend on which pair ran which unit.
+//
+// Per CTA, 6 warps as in lmhead_kernel: warp 0 TMA producer (own W rows + own half of the hidden chunk), warp 1
+// TMEM owner; in the pair's leader (cluster rank 0) its elected lane issues the UMMAs for both CTAs; warps 2..5
+// epilogue over the CTA's own 128 accumulator lanes.
+// Barriers that the other CTA signals: the copies of BOTH CTAs complete their bytes on the leader's `full` barrier
+// (the peer's TMA names the leader's barrier; no thread sits in between), the UMMA completion is committed with a
+// multicast arrive to `empty` / `acc_full` of both CTAs, and the peer's epilogue warps arrive remotely on the leader's
+// `acc_empty`.  Every wait is bounded; both CTAs meet at a cluster barrier before the TMEM is released.
+#include <math.h>
+#include <stdlib.h>
+
+#include "mirror_internal.h"
+
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kBK = 64;
+constexpr int kTileV = 128;                 // vocabulary rows per CTA and unit
+constexpr int kPairV = 2 * kTileV;          // per pair
+constexpr int kATileBytes = kTileV * kBK * 2;
+constexpr int kMaxStages = 8;
+constexpr int kAcc = 2;
+constexpr int kMaxChunkRows = 256;
+constexpr int kSmemBudget = 232448;
+constexpr int kCtrlBytes = 1024 + 4 * kMaxChunkRows * 12;
+
+struct PairParams {
+    int M, V, H;
+    int n_chunks, chunk_rows, half_rows;
+    int acc_stride, tmem_cols;
+    int stages, stage_bytes;
+    int n_units;
+    int w_keep;                             // 1: weight tiles are re-read by other chunks, keep them in L2
+    float inv_T, inv_T_log2e;
+    float* logits_out;
+    float* part_max;                        // [partials][M]
+    int* part_idx;
+    float* part_sum;
+    int* status;
+};
+
+struct Ctrl {
+    uint64_t full[kMaxStages];              // leader only: the stage has landed in both CTAs (transaction bytes of both)
+    uint64_t empty[kMaxStages];             // UMMAs that read the stage have completed (multicast commit)
+    uint64_t acc_full[kAcc];                // accumulator complete (multicast commit)
+    uint64_t acc_empty[kAcc];               // leader only: 4 + 4 epilogue warps have drained the accumulator
+    uint32_t tmem_base;
+    volatile int abort;
+};
+
+__device__ __forceinline__ void fail(const PairParams& p, Ctrl* c, int where) {
+    c->abort = 1;
+    if (atomicCAS(p.status, 0, MIRROR_DEV_TIMEOUT) == 0) atomicExch(p.status + 1, where);
+}
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {      // every thread of both CTAs
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory object in the CTA of rank `rank`
+__device__ __forceinline__ uint32_t map_to_rank(const void* smem_ptr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(ptx::smem_u32(smem_ptr)), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// bounded wait on a barrier that the other CTA of the pair arrives on
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, long long limit_cycles = 4000000000ll) {
+    const uint32_t a = ptx::smem_u32(bar);
+    const long long t0 = clock64();
+    for (;;) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(a), "r"(parity), "r"(MIRROR_PARK_NS)
+            : "memory");
+        if (ok) return true;
+        if (clock64() - t0 > limit_cycles) return false;
+    }
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t* smem_result, uint32_t ncols) {    // one warp of EACH CTA
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(ptx::smem_u32(smem_result)), "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {         // one warp of EACH CTA
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// TMA load into this CTA's shared memory whose bytes are counted on a barrier of the pair's leader (cluster address)
+__device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const void* map, uint32_t bar_cluster_addr, int x, int y,
+                                                 uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(ptx::smem_u32(smem_dst)), "l"(map), "r"(bar_cluster_addr), "r"(x), "r"(y), "l"(policy)
+        : "memory");
+}
+// D[tmem of both CTAs] (+)= A (128 rows from each CTA's shared memory) * B (N/2 rows from each CTA's shared memory)
+__device__ __forceinline__ void umma_pair_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                              uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// arrive on the barrier at this shared-memory offset in BOTH CTAs once all UMMAs issued so far have completed
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(ptx::smem_u32(bar)), "h"((uint16_t)3)
+                 : "memory");
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+lmhead_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_h, const PairParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    // (the dynamic shared window starts at the same offset in both CTAs, so the aligned layout is the same too)
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t* stage_base = smem;
+    Ctrl* ctrl = (Ctrl*)(smem + (size_t)p.stages * p.stage_bytes);
+    float* st_max = (float*)((uint8_t*)ctrl + 1024);          // [4][kMaxChunkRows]
+    int* st_idx = (int*)(st_max + 4 * kMaxChunkRows);
+    float* st_sum = (float*)(st_idx + 4 * kMaxChunkRows);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = cluster_rank();
+    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    const int n_kb = p.H / kBK;
+
+    if (tid == 0) {
+        for (int s = 0; s < p.stages; ++s) {
+            ptx::mbar_init(&ctrl->full[s], 1);
+            ptx::mbar_init(&ctrl->empty[s], 1);
+        }
+        for (int a = 0; a < kAcc; ++a) { ptx::mbar_init(&ctrl->acc_full[a], 1); ptx::mbar_init(&ctrl->acc_empty[a], 8); }
+        ctrl->abort = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tmap(&tm_w);
+        ptx::prefetch_tmap(&tm_h);
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(&ctrl->tmem_base, (uint32_t)p.tmem_cols);
+        tmem_relinquish_pair();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                 // the other CTA's barriers exist before anything arrives on them
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = ctrl->tmem_base;
+    ptx::grid_dep_wait();
+    ptx::grid_dep_launch();
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (both CTAs)
+        if (lane == 0) {
+            const uint64_t pol_w = p.w_keep ? ptx::policy_evict_normal() : ptx::policy_evict_first();
+            const uint64_t pol_h = ptx::policy_evict_last();
+            int s = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int u = pair; u < p.n_units && ok; u += n_pairs) {
+                const int tile = u / p.n_chunks, chunk = u - tile * p.n_chunks;
+                const int w_row = tile * kPairV + (int)rank * kTileV;
+                const int h_row = chunk * p.chunk_rows + (int)rank * p.half_rows;
+                for (int kb = 0; kb < n_kb; ++kb) {
+                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->empty[s], ph ^ 1)) { fail(p, ctrl, 11); ok = false; break; }
+                    if (rank == 0) ptx::mbar_arrive_expect_tx(&ctrl->full[s], 2u * (uint32_t)p.stage_bytes);
+                    const uint32_t bar = map_to_rank(&ctrl->full[s], 0);
+                    uint8_t* dst = stage_base + s * p.stage_bytes;
+                    tma_load_2d_pair(dst, &tm_w, bar, kb * kBK, w_row, pol_w);
+                    tma_load_2d_pair(dst + kATileBytes, &tm_h, bar, kb * kBK, h_row, pol_h);
+                    if (++s == p.stages) { s = 0; ph ^= 1; }
+                }
+            }
+            // (copies still in flight after a failure: the leader's issuer or its 2 s limit outlasts them, and both CTAs
+            // meet at the cluster barrier below before either one's shared memory goes away)
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            // -------------------------------------------------------------- UMMA issuer (leader)
+            const uint32_t idesc = ptx::umma_idesc_bf16(kPairV, p.chunk_rows);
+            const uint32_t stage_u32 = ptx::smem_u32(stage_base);
+            int s = 0, ab = 0;
+            uint32_t ph = 0, aph = 0;
+            bool ok = true;
+            for (int u = pair; u < p.n_units && ok; u += n_pairs) {
+                if (ctrl->abort || !mbar_wait_cluster(&ctrl->acc_empty[ab], aph ^ 1)) { fail(p, ctrl, 12); ok = false; break; }
+                ptx::tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(ab * p.acc_stride);
+                for (int kb = 0; kb < n_kb; ++kb) {
+                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->full[s], ph)) { fail(p, ctrl, 13); ok = false; break; }
+                    ptx::tc_fence_after();
+                    const uint32_t sa = stage_u32 + (uint32_t)(s * p.stage_bytes);
+                    const uint32_t sb = sa + kATileBytes;
+#pragma unroll
+                    for (int k4 = 0; k4 < kBK / 16; ++k4)
+                        umma_pair_f16(d_tmem, ptx::umma_desc_k_sw128(sa + k4 * 32), ptx::umma_desc_k_sw128(sb + k4 * 32), idesc,
+                                      (kb | k4) != 0);
+                    umma_commit_pair(&ctrl->empty[s]);
+                    if (++s == p.stages) { s = 0; ph ^= 1; }
+                }
+                if (ok) umma_commit_pair(&ctrl->acc_full[ab]);
+                if (++ab == kAcc) { ab = 0; aph ^= 1; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (both CTAs, own 128 lanes)
+        const int q = warp & 3;
+        float* my_max = st_max + q * kMaxChunkRows;
+        int* my_idx = st_idx + q * kMaxChunkRows;
+        float* my_sum = st_sum + q * kMaxChunkRows;
+        const int n_cg = (p.chunk_rows + 31) / 32;
+        // the four warps hold disjoint vocabulary rows: one partial per hidden row out of their four states
+        auto flush = [&](size_t pbase, int rbase) {
+            for (int c = (warp - 2) * 32 + lane; c < p.chunk_rows; c += 128) {
+                const int row = rbase + c;
+                if (row >= p.M) continue;
+                float m = -INFINITY, s = 0.f;
+                int idx = 0x7fffffff;
+#pragma unroll
+                for (int w = 0; w < 4; ++w) {
+                    const float pm = st_max[w * kMaxChunkRows + c], ps = st_sum[w * kMaxChunkRows + c];
+                    const int pi = st_idx[w * kMaxChunkRows + c];
+                    if (pm == -INFINITY) continue;
+                    if (pm > m || (pm == m && pi < idx)) {
+                        s = ps + (m == -INFINITY ? 0.f : s * exp2f((m - pm) * p.inv_T_log2e));
+                        m = pm; idx = pi;
+                    } else {
+                        s += ps * exp2f((pm - m) * p.inv_T_log2e);
+                    }
+                }
+                p.part_max[pbase + row] = m;
+                p.part_idx[pbase + row] = idx;
+                p.part_sum[pbase + row] = s;
+            }
+        };
+        int ab = 0;
+        uint32_t aph = 0;
+        bool ok = true;
+        // One row chunk: a CTA meets the same hidden rows in every unit and keeps a running state per row, flushed once
+        // (one partial per CTA).  Several chunks: every unit flushes its own partial (one per 128-row vocabulary tile).
+        const bool running = p.n_chunks == 1;
+        if (running) {
+            for (int c = lane; c < kMaxChunkRows; c += 32) { my_max[c] = -INFINITY; my_idx[c] = 0x7fffffff; my_sum[c] = 0.f; }
+            __syncwarp();
+        }
+        for (int u = pair; u < p.n_units; u += n_pairs) {
+            const int tile = u / p.n_chunks, chunk = u - tile * p.n_chunks;
+            const int rbase = chunk * p.chunk_rows;
+            const int vt = tile * 2 + (int)rank;                 // 128-row vocabulary tile of this CTA
+            if (ok && (ctrl->abort || !ptx::mbar_wait(&ctrl->acc_full[ab], aph))) { fail(p, ctrl, 16); ok = false; }
+            if (ok) {
+                ptx::tc_fence_after();
+                const int vid = vt * kTileV + q * 32 + lane;
+                const bool valid = vid < p.V;
+                const bool any_valid = __ballot_sync(0xffffffffu, valid) != 0;          // warp-uniform
+                const int n_rows = min(p.chunk_rows, p.M - rbase);                       // hidden rows of this chunk
+                for (int cg = 0; cg < n_cg; ++cg) {
+                    uint32_t r[32];
+                    ptx::tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * p.acc_stride + cg * 32), r);
+                    ptx::tmem_ld_wait();
+                    float upd_m = -INFINITY, upd_s = 0.f;
+                    int upd_i = 0x7fffffff;
+                    const int ncol = n_rows - cg * 32;       // columns of this group that are hidden rows (the rest hold zeros)
+                    if (any_valid && ncol > 0) {
+                        // The 32 columns go through the reductions side by side (no branch inside, so the shuffle
+                        // chains of different columns overlap); lane j keeps the result of column j.
+                        float v[32], m[32];
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) m[j] = v[j] = valid ? __uint_as_float(r[j]) : -INFINITY;
+                        if (p.logits_out && valid) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (j < ncol) p.logits_out[(size_t)(rbase + cg * 32 + j) * p.V + vid] = v[j];
+                        }
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) m[j] = fmaxf(m[j], __shfl_xor_sync(0xffffffffu, m[j], o));
+                        }
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const unsigned eq = __ballot_sync(0xffffffffu, v[j] == m[j]);
+                            if (lane == j) { upd_m = m[j]; upd_i = vid - lane + (__ffs(eq) - 1); }
+                            v[j] = exp2f((v[j] - m[j]) * p.inv_T_log2e);
+                        }
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) v[j] += __shfl_xor_sync(0xffffffffu, v[j], o);
+                        }
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (lane == j) upd_s = v[j];
+                    }
+                    const int c = cg * 32 + lane;          // lane j holds column cg*32+j of this unit
+                    if (!running) {
+                        my_max[c] = upd_m; my_idx[c] = upd_i; my_sum[c] = upd_s;
+                    } else if (upd_m != -INFINITY) {
+                        const float om = my_max[c], os = my_sum[c];
+                        if (upd_m > om) {           // ids only grow along a CTA's units: equality keeps the older, lower id
+                            my_sum[c] = upd_s + (om == -INFINITY ? 0.f : os * exp2f((om - upd_m) * p.inv_T_log2e));
+                            my_max[c] = upd_m;
+                            my_idx[c] = upd_i;
+                        } else {
+                            my_sum[c] = os + upd_s * exp2f((upd_m - om) * p.inv_T_log2e);
+                        }
+                    }
+                }
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(map_to_rank(&ctrl->acc_empty[ab], 0));
+            }
+            if (++ab == kAcc) { ab = 0; aph ^= 1; }
+            if (!running) {
+                // fold the four warps' results (disjoint vocabulary rows) into one partial per hidden row
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (ok && !ctrl->abort) flush((size_t)vt * p.M, rbase);
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+            }
+        }
+        if (running) {
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (ok && !ctrl->abort) flush((size_t)blockIdx.x * p.M, 0);
+        }
+    }
+
+    ptx::tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                 // no remote arrive or multicast commit is in flight towards a CTA that has left
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        tmem_dealloc_pair(tmem_base, (uint32_t)p.tmem_cols);
+    }
+}
+
+int next_pow2(int x) {
+    int p = 1;
+    while (p < x) p <<= 1;
+    return p;
+}
+
+}  // namespace
+
+int mirror_lmhead_pair_partials(int V) { return 2 * ((V + kPairV - 1) / kPairV); }
+
+mirror_status mirror_lmhead_pair_launch(mirror_ctx* ctx, const void* hidden, int M, const void* W, float* logits_out,
+                                        void* partial_ws, size_t partial_bytes, cudaStream_t stream, int* n_partials) {
+    const int V = ctx->desc.vocab, H = ctx->desc.hidden;
+    const int n_tiles = (V + kPairV - 1) / kPairV;
+    PairParams p;
+    p.M = M; p.V = V; p.H = H;
+    p.n_chunks = (M + kMaxChunkRows - 1) / kMaxChunkRows;
+    p.chunk_rows = (int)align_up((size_t)((M + p.n_chunks - 1) / p.n_chunks), 16);
+    p.half_rows = p.chunk_rows / 2;
+    p.acc_stride = next_pow2(p.chunk_rows < 32 ? 32 : p.chunk_rows);
+    p.tmem_cols = kAcc * p.acc_stride;
+    p.stage_bytes = kATileBytes + p.half_rows * kBK * 2;
+    p.stages = (kSmemBudget - kCtrlBytes - 1024) / p.stage_bytes;
+    if (p.stages > kMaxStages) p.stages = kMaxStages;
+    if (const char* e = getenv("MIRROR_LM_STAGES")) { const int s = atoi(e); if (s >= 2 && s < p.stages) p.stages = s; }
+    if (p.stages < 2) return MIRROR_ERR_SHAPE;
+    p.n_units = n_tiles * p.n_chunks;
+    int n_pairs = ctx->num_sms / 2;
+    if (n_pairs > p.n_units) n_pairs = p.n_units;
+    if (n_pairs < 1) return MIRROR_ERR_UNSUPPORTED;
+    // partials: one per CTA (single row chunk: running state) or one per 128-row vocabulary tile
+    const size_t P = p.n_chunks == 1 ? (size_t)2 * n_pairs : (size_t)2 * n_tiles;
+    if (partial_bytes < P * M * 12) return MIRROR_ERR_WORKSPACE;
+    p.w_keep = p.n_chunks > 1;
+    p.inv_T = 1.0f / ctx->temperature;
+    p.inv_T_log2e = p.inv_T * 1.4426950408889634f;
+    p.logits_out = logits_out;
+    p.part_max = (float*)partial_ws;
+    p.part_idx = (int*)(p.part_max + P * M);
+    p.part_sum = (float*)(p.part_idx + P * M);
+    p.status = ctx->d_status;
+
+    CUtensorMap tm_w, tm_h;
+    {
+        const uint64_t dims[2] = {(uint64_t)H, (uint64_t)V};
+        const uint64_t strides[1] = {(uint64_t)H * 2};
+        const uint32_t box_w[2] = {kBK, kTileV};
+        mirror_status st = mirror_make_tmap(ctx, &tm_w, W, 2, dims, strides, box_w);
+        if (st != MIRROR_OK) return st;
+        const uint64_t hdims[2] = {(uint64_t)H, (uint64_t)M};
+        const uint32_t box_h[2] = {kBK, (uint32_t)p.half_rows};
+        st = mirror_make_tmap(ctx, &tm_h, hidden, 2, hdims, strides, box_h);
+        if (st != MIRROR_OK) return st;
+    }
+    const size_t smem = (size_t)p.stages * p.stage_bytes + kCtrlBytes + 1024;
+    if (!ctx->lm_pair_attr_set) {
+        MIRROR_CUDA_OK(cudaFuncSetAttribute(lmhead_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+        ctx->lm_pair_attr_set = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)n_pairs * 2);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    MIRROR_CUDA_OK(cudaLaunchKernelEx(&cfg, lmhead_pair_kernel, tm_w, tm_h, p));
+    ctx->launches += 1;
+    MIRROR_CUDA_OK(cudaGetLastError());
+    *n_partials = (int)P;
+    return MIRROR_OK;
+}

@@ -440,6 +440,37 @@ int next_pow2(int x) {
     return p;
 }
 
+// What follows the GEMM, whichever kernel ran it: merge of the row partials, Top-kappa, gathers.
+mirror_status lmhead_tail(mirror_ctx* ctx, const void* hidden, int M, const void* W, int topk, const int32_t* gather_row,
+                          const int32_t* gather_tok, int n_gather, int32_t* argmax, float* maxlogit, float* lse, int32_t* topk_id,
+                          float* topk_logprob, float* gather_logit, float* logits_out, float* lse_scratch, cudaStream_t stream,
+                          void* topk_logprob_bf16, int P, float inv_T, float inv_T_log2e, const float* part_max, const int* part_idx,
+                          const float* part_sum) {
+    const int V = ctx->desc.vocab, H = ctx->desc.hidden;
+    float* lse_dst = lse ? lse : (topk > 0 ? lse_scratch : nullptr);
+    if (argmax || maxlogit || lse_dst) {
+        MIRROR_CUDA_OK(mirror_launch_pdl(lmhead_merge_kernel, dim3(M), dim3(256), 0, stream, M, P, inv_T, inv_T_log2e,
+                                         part_max, part_idx, part_sum, argmax, maxlogit, lse_dst));
+        ctx->launches += 1;
+        MIRROR_CUDA_OK(cudaGetLastError());
+    }
+    if (topk > 0) {
+        MIRROR_CUDA_OK(mirror_launch_pdl(lmhead_topk_kernel, dim3(M), dim3(1024), 0, stream, V, topk, inv_T, logits_out, lse_dst,
+                                         topk_id, topk_logprob, (__nv_bfloat16*)topk_logprob_bf16));
+        ctx->launches += 1;
+        MIRROR_CUDA_OK(cudaGetLastError());
+    }
+    if (n_gather > 0) {
+        const int warps = 8;
+        lmhead_gather_kernel<<<(n_gather + warps - 1) / warps, warps * 32, 0, stream>>>(
+            n_gather, M, V, H, (const __nv_bfloat16*)hidden, (const __nv_bfloat16*)W, gather_row, gather_tok, gather_logit,
+            ctx->d_status);
+        ctx->launches += 1;
+        MIRROR_CUDA_OK(cudaGetLastError());
+    }
+    return MIRROR_OK;
+}
+
 }  // namespace
 
 mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, const void* W, int topk,
@@ -449,6 +480,25 @@ mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, c
                                    void* partial_ws, size_t partial_bytes, float* lse_scratch, cudaStream_t stream,
                                    cudaEvent_t after_gemm, void* topk_logprob_bf16) {
     const int V = ctx->desc.vocab, H = ctx->desc.hidden;
+    // The GEMM runs on CTA pairs (lmhead_pair.cu) whenever the partials it leaves fit the scratch it was given; the
+    // single-CTA weight-stream kernel below is the fallback (and what MIRROR_LM_PAIR_MIN_ROWS can force for comparison).
+    int pair_min_rows = 1;
+    if (const char* e = getenv("MIRROR_LM_PAIR_MIN_ROWS")) pair_min_rows = atoi(e);
+    if (M >= pair_min_rows && ctx->num_sms >= 2) {
+        int P = 0;
+        mirror_status st = mirror_lmhead_pair_launch(ctx, hidden, M, W, logits_out, partial_ws, partial_bytes, stream, &P);
+        if (st == MIRROR_OK) {
+            if (after_gemm) MIRROR_CUDA_OK(cudaEventRecord(after_gemm, stream));
+            const float inv_T = 1.0f / ctx->temperature, inv_T_log2e = inv_T * 1.4426950408889634f;
+            float* part_max = (float*)partial_ws;
+            int* part_idx = (int*)(part_max + (size_t)P * M);
+            float* part_sum = (float*)(part_idx + (size_t)P * M);
+            return lmhead_tail(ctx, hidden, M, W, topk, gather_row, gather_tok, n_gather, argmax, maxlogit, lse, topk_id, topk_logprob,
+                               gather_logit, logits_out, lse_scratch, stream, topk_logprob_bf16, P, inv_T, inv_T_log2e, part_max,
+                               part_idx, part_sum);
+        }
+        if (st != MIRROR_ERR_WORKSPACE) return st;
+    }
     LmParams p;
     p.M = M; p.V = V; p.H = H;
     p.n_chunks = (M + kMaxChunkRows - 1) / kMaxChunkRows;
@@ -508,28 +558,9 @@ mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, c
     MIRROR_CUDA_OK(cudaGetLastError());
     if (after_gemm) MIRROR_CUDA_OK(cudaEventRecord(after_gemm, stream));
 
-    float* lse_dst = lse ? lse : (topk > 0 ? lse_scratch : nullptr);
-    if (argmax || maxlogit || lse_dst) {
-        MIRROR_CUDA_OK(mirror_launch_pdl(lmhead_merge_kernel, dim3(M), dim3(256), 0, stream, M, (int)P, p.inv_T, p.inv_T_log2e,
-                                         p.part_max, p.part_idx, p.part_sum, argmax, maxlogit, lse_dst));
-        ctx->launches += 1;
-        MIRROR_CUDA_OK(cudaGetLastError());
-    }
-    if (topk > 0) {
-        MIRROR_CUDA_OK(mirror_launch_pdl(lmhead_topk_kernel, dim3(M), dim3(1024), 0, stream, V, topk, p.inv_T, logits_out, lse_dst,
-                                         topk_id, topk_logprob, (__nv_bfloat16*)topk_logprob_bf16));
-        ctx->launches += 1;
-        MIRROR_CUDA_OK(cudaGetLastError());
-    }
-    if (n_gather > 0) {
-        const int warps = 8;
-        lmhead_gather_kernel<<<(n_gather + warps - 1) / warps, warps * 32, 0, stream>>>(
-            n_gather, M, V, H, (const __nv_bfloat16*)hidden, (const __nv_bfloat16*)W, gather_row, gather_tok, gather_logit,
-            ctx->d_status);
-        ctx->launches += 1;
-        MIRROR_CUDA_OK(cudaGetLastError());
-    }
-    return MIRROR_OK;
+    return lmhead_tail(ctx, hidden, M, W, topk, gather_row, gather_tok, n_gather, argmax, maxlogit, lse, topk_id, topk_logprob,
+                       gather_logit, logits_out, lse_scratch, stream, topk_logprob_bf16, (int)P, p.inv_T, p.inv_T_log2e, p.part_max,
+                       p.part_idx, p.part_sum);
 }
 
 extern "C" mirror_status mirror_lmhead_reduce(mirror_ctx* ctx, const void* hidden, int M, const void* W, int topk,
@@ -583,7 +614,7 @@ struct NoAllocDevice {          // host-side, per device, filled by the first ca
     bool ready = false;
     unsigned char* scratch = nullptr;
     int num_sms = 0;
-    bool attr_set = false;
+    bool attr_set = false, pair_attr_set = false;
     PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
 };
 NoAllocDevice g_noalloc_dev[64];
@@ -632,6 +663,7 @@ extern "C" mirror_status mirror_lmhead_reduce_noalloc(int device, const void* hi
     tmp.d_status = (int*)d.scratch;
     tmp.encode = d.encode;
     tmp.lm_attr_set = d.attr_set;
+    tmp.lm_pair_attr_set = d.pair_attr_set;
     cudaStream_t s = (cudaStream_t)stream;
     // the status words must start at zero; the partials are fully rewritten by every launch before they are read
     MIRROR_CUDA_OK(cudaMemsetAsync(d.scratch, 0, kNoAllocHeader, s));
@@ -639,5 +671,6 @@ extern "C" mirror_status mirror_lmhead_reduce_noalloc(int device, const void* hi
                                             nullptr, nullptr, d.scratch + kNoAllocHeader, kNoAllocBytes - kNoAllocHeader,
                                             nullptr, s, nullptr);
     d.attr_set = tmp.lm_attr_set;
+    d.pair_attr_set = tmp.lm_pair_attr_set;
     return st;
 }

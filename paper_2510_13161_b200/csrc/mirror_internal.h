@@ -31,6 +31,7 @@ struct mirror_ctx {
     size_t ws_bytes = 0;
     long long launches = 0;
     bool lm_attr_set = false;
+    bool lm_pair_attr_set = false;
     cudaEvent_t stage_ev[4] = {nullptr, nullptr, nullptr, nullptr};
     bool stage_ev_on = false;
     PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
@@ -45,7 +46,7 @@ constexpr size_t kWsZeroedBytes = 4096;     // words at the front of the workspa
 struct MirrorWsLayout {
     size_t zeroed = 0;                                   // kWsZeroedBytes of zeroed words
     size_t attn_partial = 0, attn_partial_bytes = 0;     // split-KV partial accumulators
-    size_t lm_partial = 0, lm_partial_bytes = 0;         // per-(CTA, warp) row partials
+    size_t lm_partial = 0, lm_partial_bytes = 0;         // per-CTA (or per-unit) row partials
     size_t lse = 0, argmax = 0;                          // [M] scratch each
     size_t logits = 0, logits_bytes = 0;                 // fp32 [M, V]
     size_t accept_scratch = 0;                           // fp64 [B, 2, V]: running distribution of the tree acceptance
@@ -62,6 +63,11 @@ mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, c
                                    float* topk_logprob, float* gather_logit, float* logits_out,
                                    void* partial_ws, size_t partial_bytes, float* lse_scratch, cudaStream_t stream,
                                    cudaEvent_t after_gemm = nullptr, void* topk_logprob_bf16 = nullptr);
+// LM-head GEMM + per-unit row partials on CTA pairs (many hidden rows); *n_partials partials of [M] rows are left in
+// partial_ws for lmhead_merge_kernel.  mirror_lmhead_pair_partials(V) is that count.
+int mirror_lmhead_pair_partials(int V);
+mirror_status mirror_lmhead_pair_launch(mirror_ctx* ctx, const void* hidden, int M, const void* W, float* logits_out,
+                                        void* partial_ws, size_t partial_bytes, cudaStream_t stream, int* n_partials);
 mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const MirrorTreeInfo& ti,
                                  const void* q, const void* k_new, const void* v_new, void* out, float* lse_out,
                                  float* partial_ws, cudaStream_t stream);
@@ -180,6 +186,11 @@ __device__ __forceinline__ void tma_load_5d(void* smem_dst, const void* map, uin
 __device__ __forceinline__ uint64_t policy_evict_first() {
     uint64_t p;
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_normal() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
     return p;
 }
 __device__ __forceinline__ uint64_t policy_evict_last() {
