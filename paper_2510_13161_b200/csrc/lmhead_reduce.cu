@@ -1,8 +1,11 @@
-// LM head logits = W h (Eq. 1; early-exit proxy Eq. 5) as a tcgen05 / TMEM GEMM with the per-row
-// argmax / max / log-sum-exp reduction fused into the epilogue, so that the [M, V] logits never
-// travel through HBM unless the caller asks for them (speculative sampling, Top-kappa of Eq. 6).
+// LM head logits = W h (Eq. 1; early-exit proxy Eq. 5): what surrounds the GEMM (dispatch, merge of the row partials,
+// Top-kappa of Eq. 6, gathers, the public entry points) and the single-CTA GEMM kernel.  The GEMM normally runs on CTA
+// pairs (lmhead_pair.cu); lmhead_kernel below is the one-CTA-per-SM version that serves when the scratch a caller gave
+// cannot hold the pair kernel's partials.  Both fuse the per-row argmax / max / log-sum-exp reduction into the
+// epilogue, so that the [M, V] logits never travel through HBM unless the caller asks for them (speculative sampling,
+// Top-kappa).
 //
-// Orientation ("swap-AB"): the vocabulary is the UMMA M axis (128 weight rows per tile, one TMEM
+// lmhead_kernel, orientation ("swap-AB"): the vocabulary is the UMMA M axis (128 weight rows per tile, one TMEM
 // lane per vocabulary id), the hidden rows are the UMMA N axis (<= 256 per chunk, one TMEM column
 // per hidden row).  The verify step has few rows (B * (1 + kappa*gamma)), so the kernel is a weight
 // stream: W leaves HBM exactly once per row chunk and the per-SM TMA pipeline is what has to keep
@@ -15,7 +18,7 @@
 //               reductions, running (max, argmax, sum-exp) per hidden row, optional fp32 spill
 // The vocabulary is split over CTAs in 8-row groups (the swizzle atom), so every CTA streams the same
 // number of weight bytes (+-8 rows); the ragged last tile of a CTA is fetched as 8-row TMA boxes.
-// Each (CTA, epilogue warp) leaves one partial per hidden row; a second tiny kernel merges them in a
+// Each CTA leaves one partial per hidden row; lmhead_merge_kernel merges them in a
 // fixed order with the comparator (logit descending, id ascending).
 //
 // Every mbarrier wait is bounded; on expiry the kernel records MIRROR_DEV_TIMEOUT and unwinds.

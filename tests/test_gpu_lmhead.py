@@ -56,9 +56,9 @@ def test_logits_and_reductions_match_oracle(M, V, H):
     assert torch.equal(res["maxlogit"], res2["maxlogit"]) and torch.equal(res["lse"], res2["lse"])
 
 
-@pytest.mark.parametrize("M", [300, 392])
-def test_row_chunking(M):
-    V, H = 4096, 256
+@pytest.mark.parametrize("M,V,H", [(300, 4096, 256), (392, 4096, 256), (520, 5003, 320), (1040, 2600, 192)])
+def test_row_chunking(M, V, H):
+    """More than 256 rows: several row chunks per vocabulary tile, one partial per unit (ragged last tile included)."""
     W = rand_bf16((V, H), 0.05, 3); hid = rand_bf16((M, H), 1.0, 4)
     m = make_mirror(lm_cfg(V, H))
     res = m.mirror_lmhead_reduce(hid.cuda(), W.cuda(), want_logits=True)
@@ -66,6 +66,24 @@ def test_row_chunking(M):
     logits = O.lmhead_logits(I.bf16_bits(hid), I.bf16_bits(W))
     assert np.abs(res["logits"].cpu().numpy() - logits).max() < LOGIT_TOL_TIGHT
     check_reductions(res, logits)
+
+
+@pytest.mark.parametrize("M,V,H", [(17, 5000, 512), (130, 3000, 256), (300, 4096, 256)])
+def test_single_cta_fallback_kernel_matches_oracle_and_pair_kernel(M, V, H, monkeypatch):
+    """The one-CTA-per-SM kernel that serves when the scratch cannot hold the pair kernel's partials: forced here."""
+    W = rand_bf16((V, H), 0.05, 11); hid = rand_bf16((M, H), 1.0, 12)
+    m = make_mirror(lm_cfg(V, H))
+    res_pair = m.mirror_lmhead_reduce(hid.cuda(), W.cuda(), want_logits=True)
+    monkeypatch.setenv("MIRROR_LM_PAIR_MIN_ROWS", "1000000")
+    res = m.mirror_lmhead_reduce(hid.cuda(), W.cuda(), want_logits=True)
+    monkeypatch.delenv("MIRROR_LM_PAIR_MIN_ROWS")
+    assert m.device_status() == (0, 0)
+    logits = O.lmhead_logits(I.bf16_bits(hid), I.bf16_bits(W))
+    assert np.abs(res["logits"].cpu().numpy() - logits).max() < LOGIT_TOL_TIGHT
+    check_reductions(res, logits)
+    # same accumulation order per logit in both kernels (K ascending): the logits agree bit for bit
+    assert torch.equal(res["logits"], res_pair["logits"])
+    assert torch.equal(res["argmax"], res_pair["argmax"]) and torch.equal(res["maxlogit"], res_pair["maxlogit"])
 
 
 def test_ties_go_to_lowest_id_and_topk_gather_temperature():
