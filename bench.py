@@ -233,6 +233,50 @@ def job_throughput(steps_per_rank: int, world: int, ms_max: float) -> float:
 # ---------------------------------------------------------------------------------------------------
 # the CUDA arm
 # ---------------------------------------------------------------------------------------------------
+def attn_per_layer(m, x, tree, cfg, reps: int = 10):
+    """Attention launched layer by layer (one mirror_attn_verify call per layer): ms for all layers, as plain launches and
+    as a CUDA-graph replay.  The fused step passes all layers in one launch because its Q tensors are inputs."""
+    import torch
+    L = x.q.shape[0]
+    kvs = [m.kv(x.k_pool[l:l + 1], x.v_pool[l:l + 1], x.page_table, x.prefix_len) for l in range(L)]
+    out = torch.empty_like(x.q)
+    s = torch.cuda.Stream()
+
+    def run():
+        for l in range(L):
+            m.mirror_attn_verify(kvs[l], tree, x.q[l:l + 1], x.k_new[l:l + 1], x.v_new[l:l + 1], out=out[l:l + 1], stream=s)
+
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    res = {}
+    with torch.cuda.stream(s):
+        for _ in range(3):
+            run()
+        s.synchronize()
+        e0.record(s)
+        for _ in range(reps):
+            run()
+        e1.record(s)
+        s.synchronize()
+        res["launches"] = e0.elapsed_time(e1) / reps
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            run()
+        for _ in range(3):
+            g.replay()
+        s.synchronize()
+        e0.record(s)
+        for _ in range(reps):
+            g.replay()
+        e1.record(s)
+        s.synchronize()
+        res["graph"] = e0.elapsed_time(e1) / reps
+    code, detail = m.device_status()
+    if code != 0:
+        raise SystemExit(f"device status {code} (detail {detail}) in the per-layer attention variant")
+    res["kernel_launches"] = 2 * L
+    return res
+
+
 def run_mirror(args):
     import torch
     import torch.distributed as dist
@@ -356,6 +400,10 @@ def run_mirror(args):
               "attn_tflops": work["attn_flops"] / (attn_ms * 1e-3) / 1e12,
               "lmhead_tflops": work["lm_flops"] / (lm_ms * 1e-3) / 1e12,
               "step_hbm_frac": (work["attn_bytes"] + work["lm_bytes"]) / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+
+    # ---- attention with one launch pair per layer: the order a real target enforces (layer l+1's queries depend on
+    # layer l's output), as plain stream-ordered launches and replayed from a CUDA graph.  Outside the timed region.
+    stages["attn_per_layer_ms"] = attn_per_layer(m, x, tree, cfg)
 
     cpu = None
     if not args.no_cpu_baseline and world == 1:

@@ -897,10 +897,11 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     }
 }
 
-// Merge of the units that the partition cut across CTA groups.  One block per (inner boundary, row block): the
-// block whose boundary is the first one inside a unit combines all of that unit's parts, in group order, from the
-// (max, sum, accumulator) records the attention kernel left, exactly like split-KV partials.  Blocks whose boundary
-// coincides with a unit boundary, or is not the first inside its unit, have nothing to do.
+// Merge of the units that the partition cut across CTA groups.  One block per (inner boundary, row block).  A unit
+// cut by k boundaries left k + 1 (max, sum, accumulator) records, like split-KV partials; the k blocks of those
+// boundaries share its merge by output columns (8-column chunks dealt round-robin), each combining all parts of its
+// columns in group order, so a unit that many CTAs shared (few units per launch, long contexts) is not merged by one
+// block alone.  Blocks whose boundary coincides with a unit boundary have nothing to do.
 constexpr int kMergeThreads = 512;        // 128 rows x 4 column quarters
 template <int D>
 __global__ void __launch_bounds__(kMergeThreads) attn_merge_kernel(const AttnParams p) {
@@ -928,24 +929,37 @@ __global__ void __launch_bounds__(kMergeThreads) attn_merge_kernel(const AttnPar
     const long long x = group_begin(part, g, p, cumT);
     const UnitPos u = locate(x, p, cumT, part.tiles_per_layer);
     if (u.tile_in_unit == 0) return;                                            // the boundary is a unit boundary
-    if (group_begin(part, g - 1, p, cumT) > u.unit_first_tile) return;          // an earlier boundary cuts this unit too
-    const int ga = g - 1;
+    // the groups ga..gb hold this unit's parts; the blocks of the boundaries ga+1..gb share the merge by columns
+    int ga = g - 1;
+    while (ga > 0 && group_begin(part, ga, p, cumT) > u.unit_first_tile) --ga;
     int gb = g;
     const long long unit_last = u.unit_first_tile + u.tiles_in_unit - 1;
     while (gb + 1 < part.n_groups && group_begin(part, gb + 1, p, cumT) <= unit_last) ++gb;
     const int parts = gb - ga + 1;
+    const int n_blocks = parts - 1, j_blk = g - (ga + 1);
     // launched with programmatic stream serialization: everything above overlaps the attention kernel's tail;
     // its records (and the outputs this block overwrites) are only touched after it has completed
     ptx::grid_dep_wait();
     ptx::grid_dep_launch();
 
     constexpr int kRowW = D + 4;
-    constexpr int kQ = D / 4;                                                   // columns per thread
+    constexpr int kChunks = D / 8;                                              // 8 output columns = one 16-byte store
+    constexpr int kPer = (kChunks + 3) / 4;                                     // chunks per thread when one block has them all
     const int row = tid & (kRows - 1), cq = tid >> 7;
     const int rb_row0 = rb * p.rows_per_rb;
     const int rb_rows = min(p.rows_per_rb, p.rows - rb_row0);
     if (row >= rb_rows) return;
     const int r_abs = rb_row0 + row, node = r_abs / p.G, hl = r_abs % p.G;
+    // chunk c belongs to block c mod n_blocks; inside the block its chunks go round the four thread quarters
+    int chunk[kPer];
+    bool any = false;
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) {
+        chunk[i] = j_blk + (cq + 4 * i) * n_blocks;
+        any |= chunk[i] < kChunks;
+    }
+    const bool writes_lse = p.lse_out && j_blk == 0 && cq == 0;
+    if (!any && !writes_lse) return;
     // group ga holds the unit's first tile (its record is in slot 1), the later groups began inside the unit (slot 0)
     auto part_of = [&](int k) -> const float* {
         return p.partial + ((size_t)((ga + k) * p.n_rb + rb) * 2 + (k == 0 ? 1 : 0)) * kRowW * kRows + row;
@@ -954,9 +968,11 @@ __global__ void __launch_bounds__(kMergeThreads) attn_merge_kernel(const AttnPar
 #pragma unroll 4
     for (int k = 0; k < parts; ++k) Mm = fmaxf(Mm, __ldcg(part_of(k) + (size_t)D * kRows));
     float Lm = 0.f;
-    float acc[kQ];
+    float acc[kPer][8];
 #pragma unroll
-    for (int j = 0; j < kQ; ++j) acc[j] = 0.f;
+    for (int i = 0; i < kPer; ++i)
+#pragma unroll
+        for (int c = 0; c < 8; ++c) acc[i][c] = 0.f;
 #pragma unroll 2
     for (int k = 0; k < parts; ++k) {
         const float* src = part_of(k);
@@ -964,20 +980,25 @@ __global__ void __launch_bounds__(kMergeThreads) attn_merge_kernel(const AttnPar
         const float wgt = (pm == -INFINITY) ? 0.f : exp2f((pm - Mm) * p.scale_log2e);
         Lm = fmaf(wgt, __ldcg(src + (size_t)(D + 1) * kRows), Lm);
 #pragma unroll
-        for (int j = 0; j < kQ; ++j) acc[j] = fmaf(wgt, __ldcg(src + (size_t)(cq * kQ + j) * kRows), acc[j]);
+        for (int i = 0; i < kPer; ++i)
+            if (chunk[i] < kChunks) {
+#pragma unroll
+                for (int c = 0; c < 8; ++c) acc[i][c] = fmaf(wgt, __ldcg(src + (size_t)(chunk[i] * 8 + c) * kRows), acc[i][c]);
+            }
     }
     const float inv = 1.f / Lm;
-    __nv_bfloat16* orow = p.out + ((((size_t)u.layer * p.B + u.b) * p.n + node) * (size_t)p.Hq + u.g * p.G + hl) * D + cq * kQ;
+    __nv_bfloat16* orow = p.out + ((((size_t)u.layer * p.B + u.b) * p.n + node) * (size_t)p.Hq + u.g * p.G + hl) * D;
 #pragma unroll
-    for (int j = 0; j < kQ / 8; ++j) {
-        uint4 v;
-        v.x = pack_bf16(acc[j * 8 + 0] * inv, acc[j * 8 + 1] * inv);
-        v.y = pack_bf16(acc[j * 8 + 2] * inv, acc[j * 8 + 3] * inv);
-        v.z = pack_bf16(acc[j * 8 + 4] * inv, acc[j * 8 + 5] * inv);
-        v.w = pack_bf16(acc[j * 8 + 6] * inv, acc[j * 8 + 7] * inv);
-        *reinterpret_cast<uint4*>(orow + j * 8) = v;
-    }
-    if (p.lse_out && cq == 0)
+    for (int i = 0; i < kPer; ++i)
+        if (chunk[i] < kChunks) {
+            uint4 v;
+            v.x = pack_bf16(acc[i][0] * inv, acc[i][1] * inv);
+            v.y = pack_bf16(acc[i][2] * inv, acc[i][3] * inv);
+            v.z = pack_bf16(acc[i][4] * inv, acc[i][5] * inv);
+            v.w = pack_bf16(acc[i][6] * inv, acc[i][7] * inv);
+            *reinterpret_cast<uint4*>(orow + chunk[i] * 8) = v;
+        }
+    if (writes_lse)
         p.lse_out[(((size_t)u.layer * p.B + u.b) * p.Hq + u.g * p.G + hl) * p.n + node] = Mm * p.scale + logf(Lm);
 }
 
