@@ -43,10 +43,11 @@ struct PairParams {
     int n_chunks, chunk_rows, half_rows;
     int acc_stride, tmem_cols;
     int stages, stage_bytes;
+    int k_slices, kb_per_slice;             // split-K (plain GEMM mode only): K blocks of 64 per unit
     int n_units;
     int w_keep;                             // 1: weight tiles are re-read by other chunks, keep them in L2
     float inv_T, inv_T_log2e;
-    float* logits_out;
+    float* logits_out;                      // reduce mode: nullable [M, V]; plain GEMM mode: [k_slices][M, V] partial sums
     float* part_max;                        // [partials][M]
     int* part_idx;
     float* part_sum;
@@ -138,8 +139,10 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
                  : "memory");
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
-lmhead_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_h, const PairParams p) {
+// kReduce: LM head (row reductions in the epilogue, optional spill).  !kReduce: plain GEMM C = W h^T for the layer
+// projections, split along K when there are fewer tiles than CTA pairs; the epilogue only stores fp32 partial sums.
+template <bool kReduce>
+__device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CUtensorMap& tm_h, const PairParams& p) {
     extern __shared__ uint8_t smem_raw[];
     // (the dynamic shared window starts at the same offset in both CTAs, so the aligned layout is the same too)
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -153,6 +156,13 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
     const uint32_t rank = cluster_rank();
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     const int n_kb = p.H / kBK;
+    // unit -> (vocabulary tile, K slice, row chunk); chunk fastest, so the chunks of a tile run side by side
+    auto decode = [&](int u, int& tile, int& slice, int& chunk) {
+        chunk = u % p.n_chunks;
+        const int t2 = u / p.n_chunks;
+        slice = t2 % p.k_slices;
+        tile = t2 / p.k_slices;
+    };
 
     if (tid == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -186,10 +196,12 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
             uint32_t ph = 0;
             bool ok = true;
             for (int u = pair; u < p.n_units && ok; u += n_pairs) {
-                const int tile = u / p.n_chunks, chunk = u - tile * p.n_chunks;
+                int tile, slice, chunk;
+                decode(u, tile, slice, chunk);
                 const int w_row = tile * kPairV + (int)rank * kTileV;
                 const int h_row = chunk * p.chunk_rows + (int)rank * p.half_rows;
-                for (int kb = 0; kb < n_kb; ++kb) {
+                const int kb_end = min(n_kb, (slice + 1) * p.kb_per_slice);
+                for (int kb = slice * p.kb_per_slice; kb < kb_end; ++kb) {
                     if (ctrl->abort || !ptx::mbar_wait(&ctrl->empty[s], ph ^ 1)) { fail(p, ctrl, 11); ok = false; break; }
                     if (rank == 0) ptx::mbar_arrive_expect_tx(&ctrl->full[s], 2u * (uint32_t)p.stage_bytes);
                     const uint32_t bar = map_to_rank(&ctrl->full[s], 0);
@@ -214,7 +226,10 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
                 if (ctrl->abort || !mbar_wait_cluster(&ctrl->acc_empty[ab], aph ^ 1)) { fail(p, ctrl, 12); ok = false; break; }
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(ab * p.acc_stride);
-                for (int kb = 0; kb < n_kb; ++kb) {
+                int tile, slice, chunk;
+                decode(u, tile, slice, chunk);
+                const int nk = min(n_kb, (slice + 1) * p.kb_per_slice) - slice * p.kb_per_slice;
+                for (int kb = 0; kb < nk; ++kb) {
                     if (ctrl->abort || !ptx::mbar_wait(&ctrl->full[s], ph)) { fail(p, ctrl, 13); ok = false; break; }
                     ptx::tc_fence_after();
                     const uint32_t sa = stage_u32 + (uint32_t)(s * p.stage_bytes);
@@ -267,12 +282,13 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
         // One row chunk: a CTA meets the same hidden rows in every unit and keeps a running state per row, flushed once
         // (one partial per CTA).  Several chunks: every unit flushes its own partial (one per 128-row vocabulary tile).
         const bool running = p.n_chunks == 1;
-        if (running) {
+        if (kReduce && running) {
             for (int c = lane; c < kMaxChunkRows; c += 32) { my_max[c] = -INFINITY; my_idx[c] = 0x7fffffff; my_sum[c] = 0.f; }
             __syncwarp();
         }
         for (int u = pair; u < p.n_units; u += n_pairs) {
-            const int tile = u / p.n_chunks, chunk = u - tile * p.n_chunks;
+            int tile, slice, chunk;
+            decode(u, tile, slice, chunk);
             const int rbase = chunk * p.chunk_rows;
             const int vt = tile * 2 + (int)rank;                 // 128-row vocabulary tile of this CTA
             if (ok && (ctrl->abort || !ptx::mbar_wait(&ctrl->acc_full[ab], aph))) { fail(p, ctrl, 16); ok = false; }
@@ -296,10 +312,12 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
 #pragma unroll
                         for (int j = 0; j < 32; ++j) m[j] = v[j] = valid ? __uint_as_float(r[j]) : -INFINITY;
                         if (p.logits_out && valid) {
+                            float* dst = p.logits_out + ((size_t)slice * p.M + rbase + cg * 32) * p.V + vid;
 #pragma unroll
                             for (int j = 0; j < 32; ++j)
-                                if (j < ncol) p.logits_out[(size_t)(rbase + cg * 32 + j) * p.V + vid] = v[j];
+                                if (j < ncol) dst[(size_t)j * p.V] = v[j];
                         }
+                        if (kReduce) {
 #pragma unroll
                         for (int o = 16; o > 0; o >>= 1) {
 #pragma unroll
@@ -319,9 +337,11 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
                             if (lane == j) upd_s = v[j];
+                        }
                     }
                     const int c = cg * 32 + lane;          // lane j holds column cg*32+j of this unit
-                    if (!running) {
+                    if (!kReduce) {
+                    } else if (!running) {
                         my_max[c] = upd_m; my_idx[c] = upd_i; my_sum[c] = upd_s;
                     } else if (upd_m != -INFINITY) {
                         const float om = my_max[c], os = my_sum[c];
@@ -339,14 +359,14 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
                 if (lane == 0) mbar_arrive_cluster(map_to_rank(&ctrl->acc_empty[ab], 0));
             }
             if (++ab == kAcc) { ab = 0; aph ^= 1; }
-            if (!running) {
+            if (kReduce && !running) {
                 // fold the four warps' results (disjoint vocabulary rows) into one partial per hidden row
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 if (ok && !ctrl->abort) flush((size_t)vt * p.M, rbase);
                 asm volatile("bar.sync 1, 128;" ::: "memory");
             }
         }
-        if (running) {
+        if (kReduce && running) {
             asm volatile("bar.sync 1, 128;" ::: "memory");
             if (ok && !ctrl->abort) flush((size_t)blockIdx.x * p.M, 0);
         }
@@ -361,63 +381,60 @@ lmhead_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
     }
 }
 
+__global__ void __launch_bounds__(kThreads, 1)
+lmhead_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_h, const PairParams p) {
+    pair_gemm_body<true>(tm_w, tm_h, p);
+}
+__global__ void __launch_bounds__(kThreads, 1)
+linear_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_h, const PairParams p) {
+    pair_gemm_body<false>(tm_w, tm_h, p);
+}
+
 int next_pow2(int x) {
     int p = 1;
     while (p < x) p <<= 1;
     return p;
 }
 
-}  // namespace
+// shapes shared by both modes: row chunks, accumulator layout, pipeline depth
+mirror_status pair_shape(int M, int V, int H, PairParams* p) {
+    if (M <= 0 || V <= 0 || H <= 0 || H % kBK != 0) return MIRROR_ERR_SHAPE;
+    p->M = M; p->V = V; p->H = H;
+    p->n_chunks = (M + kMaxChunkRows - 1) / kMaxChunkRows;
+    p->chunk_rows = (int)align_up((size_t)((M + p->n_chunks - 1) / p->n_chunks), 16);
+    p->half_rows = p->chunk_rows / 2;
+    p->acc_stride = next_pow2(p->chunk_rows < 32 ? 32 : p->chunk_rows);
+    p->tmem_cols = kAcc * p->acc_stride;
+    p->stage_bytes = kATileBytes + p->half_rows * kBK * 2;
+    p->stages = (kSmemBudget - kCtrlBytes - 1024) / p->stage_bytes;
+    if (p->stages > kMaxStages) p->stages = kMaxStages;
+    if (const char* e = getenv("MIRROR_LM_STAGES")) { const int s = atoi(e); if (s >= 2 && s < p->stages) p->stages = s; }
+    if (p->stages < 2) return MIRROR_ERR_SHAPE;
+    p->k_slices = 1;
+    p->kb_per_slice = H / kBK;
+    p->inv_T = p->inv_T_log2e = 1.f;
+    p->logits_out = nullptr;
+    p->part_max = nullptr; p->part_idx = nullptr; p->part_sum = nullptr;
+    return MIRROR_OK;
+}
 
-int mirror_lmhead_pair_partials(int V) { return 2 * ((V + kPairV - 1) / kPairV); }
-
-mirror_status mirror_lmhead_pair_launch(mirror_ctx* ctx, const void* hidden, int M, const void* W, float* logits_out,
-                                        void* partial_ws, size_t partial_bytes, cudaStream_t stream, int* n_partials) {
-    const int V = ctx->desc.vocab, H = ctx->desc.hidden;
-    const int n_tiles = (V + kPairV - 1) / kPairV;
-    PairParams p;
-    p.M = M; p.V = V; p.H = H;
-    p.n_chunks = (M + kMaxChunkRows - 1) / kMaxChunkRows;
-    p.chunk_rows = (int)align_up((size_t)((M + p.n_chunks - 1) / p.n_chunks), 16);
-    p.half_rows = p.chunk_rows / 2;
-    p.acc_stride = next_pow2(p.chunk_rows < 32 ? 32 : p.chunk_rows);
-    p.tmem_cols = kAcc * p.acc_stride;
-    p.stage_bytes = kATileBytes + p.half_rows * kBK * 2;
-    p.stages = (kSmemBudget - kCtrlBytes - 1024) / p.stage_bytes;
-    if (p.stages > kMaxStages) p.stages = kMaxStages;
-    if (const char* e = getenv("MIRROR_LM_STAGES")) { const int s = atoi(e); if (s >= 2 && s < p.stages) p.stages = s; }
-    if (p.stages < 2) return MIRROR_ERR_SHAPE;
-    p.n_units = n_tiles * p.n_chunks;
-    int n_pairs = ctx->num_sms / 2;
-    if (n_pairs > p.n_units) n_pairs = p.n_units;
-    if (n_pairs < 1) return MIRROR_ERR_UNSUPPORTED;
-    // partials: one per CTA (single row chunk: running state) or one per 128-row vocabulary tile
-    const size_t P = p.n_chunks == 1 ? (size_t)2 * n_pairs : (size_t)2 * n_tiles;
-    if (partial_bytes < P * M * 12) return MIRROR_ERR_WORKSPACE;
-    p.w_keep = p.n_chunks > 1;
-    p.inv_T = 1.0f / ctx->temperature;
-    p.inv_T_log2e = p.inv_T * 1.4426950408889634f;
-    p.logits_out = logits_out;
-    p.part_max = (float*)partial_ws;
-    p.part_idx = (int*)(p.part_max + P * M);
-    p.part_sum = (float*)(p.part_idx + P * M);
-    p.status = ctx->d_status;
-
+mirror_status pair_launch(mirror_ctx* ctx, bool reduce, const void* x, const void* W, PairParams& p, int n_pairs, cudaStream_t stream) {
     CUtensorMap tm_w, tm_h;
     {
-        const uint64_t dims[2] = {(uint64_t)H, (uint64_t)V};
-        const uint64_t strides[1] = {(uint64_t)H * 2};
+        const uint64_t dims[2] = {(uint64_t)p.H, (uint64_t)p.V};
+        const uint64_t strides[1] = {(uint64_t)p.H * 2};
         const uint32_t box_w[2] = {kBK, kTileV};
         mirror_status st = mirror_make_tmap(ctx, &tm_w, W, 2, dims, strides, box_w);
         if (st != MIRROR_OK) return st;
-        const uint64_t hdims[2] = {(uint64_t)H, (uint64_t)M};
+        const uint64_t hdims[2] = {(uint64_t)p.H, (uint64_t)p.M};
         const uint32_t box_h[2] = {kBK, (uint32_t)p.half_rows};
-        st = mirror_make_tmap(ctx, &tm_h, hidden, 2, hdims, strides, box_h);
+        st = mirror_make_tmap(ctx, &tm_h, x, 2, hdims, strides, box_h);
         if (st != MIRROR_OK) return st;
     }
     const size_t smem = (size_t)p.stages * p.stage_bytes + kCtrlBytes + 1024;
     if (!ctx->lm_pair_attr_set) {
         MIRROR_CUDA_OK(cudaFuncSetAttribute(lmhead_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+        MIRROR_CUDA_OK(cudaFuncSetAttribute(linear_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
         ctx->lm_pair_attr_set = true;
     }
     cudaLaunchConfig_t cfg = {};
@@ -434,9 +451,83 @@ mirror_status mirror_lmhead_pair_launch(mirror_ctx* ctx, const void* hidden, int
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    MIRROR_CUDA_OK(cudaLaunchKernelEx(&cfg, lmhead_pair_kernel, tm_w, tm_h, p));
+    MIRROR_CUDA_OK(cudaLaunchKernelEx(&cfg, reduce ? lmhead_pair_kernel : linear_pair_kernel, tm_w, tm_h, p));
     ctx->launches += 1;
     MIRROR_CUDA_OK(cudaGetLastError());
+    return MIRROR_OK;
+}
+
+}  // namespace
+
+int mirror_lmhead_pair_partials(int V) { return 2 * ((V + kPairV - 1) / kPairV); }
+
+mirror_status mirror_lmhead_pair_launch(mirror_ctx* ctx, const void* hidden, int M, const void* W, float* logits_out,
+                                        void* partial_ws, size_t partial_bytes, cudaStream_t stream, int* n_partials) {
+    const int V = ctx->desc.vocab, H = ctx->desc.hidden;
+    const int n_tiles = (V + kPairV - 1) / kPairV;
+    PairParams p;
+    mirror_status st = pair_shape(M, V, H, &p);
+    if (st != MIRROR_OK) return st;
+    p.n_units = n_tiles * p.n_chunks;
+    int n_pairs = ctx->num_sms / 2;
+    if (n_pairs > p.n_units) n_pairs = p.n_units;
+    if (n_pairs < 1) return MIRROR_ERR_UNSUPPORTED;
+    // partials: one per CTA (single row chunk: running state) or one per 128-row vocabulary tile
+    const size_t P = p.n_chunks == 1 ? (size_t)2 * n_pairs : (size_t)2 * n_tiles;
+    if (partial_bytes < P * M * 12) return MIRROR_ERR_WORKSPACE;
+    p.w_keep = p.n_chunks > 1;
+    p.inv_T = 1.0f / ctx->temperature;
+    p.inv_T_log2e = p.inv_T * 1.4426950408889634f;
+    p.logits_out = logits_out;
+    p.part_max = (float*)partial_ws;
+    p.part_idx = (int*)(p.part_max + P * M);
+    p.part_sum = (float*)(p.part_idx + P * M);
+    p.status = ctx->d_status;
+    st = pair_launch(ctx, true, hidden, W, p, n_pairs, stream);
+    if (st != MIRROR_OK) return st;
     *n_partials = (int)P;
+    return MIRROR_OK;
+}
+
+// Split of the K axis for a plain GEMM with few output tiles: the slice count that fills the CTA pairs best (whole
+// waves of units), slices of at least 512 K elements.
+int mirror_linear_slices(const mirror_ctx* ctx, int M, int N, int K) {
+    const int n_tiles = (N + kPairV - 1) / kPairV, n_chunks = (M + kMaxChunkRows - 1) / kMaxChunkRows;
+    const int n_kb = K / kBK, n_pairs = ctx->num_sms / 2 > 0 ? ctx->num_sms / 2 : 1;
+    int best = 1;
+    double best_eff = 0.0;
+    for (int s = 1; s <= 16; ++s) {
+        const int per = (n_kb + s - 1) / s;
+        if (s > 1 && per < 8) break;
+        const int eff_s = (n_kb + per - 1) / per;
+        const long long units = (long long)n_tiles * n_chunks * eff_s;
+        const long long waves = (units + n_pairs - 1) / n_pairs;
+        const double eff = (double)units / (double)(waves * n_pairs);
+        if (eff > best_eff + 0.02) { best_eff = eff; best = eff_s; }
+    }
+    return best;
+}
+
+// partial[s][M][N] (fp32) = sum over K slice s of x[M, K] * W[N, K]^T; the caller sums the slices in order.
+mirror_status mirror_linear_partial_launch(mirror_ctx* ctx, const void* x, int M, const void* W, int N, int K, float* partial,
+                                           size_t partial_bytes, cudaStream_t stream, int* k_slices) {
+    PairParams p;
+    mirror_status st = pair_shape(M, N, K, &p);
+    if (st != MIRROR_OK) return st;
+    const int n_tiles = (N + kPairV - 1) / kPairV, n_kb = K / kBK;
+    const int s = mirror_linear_slices(ctx, M, N, K);
+    p.kb_per_slice = (n_kb + s - 1) / s;
+    p.k_slices = (n_kb + p.kb_per_slice - 1) / p.kb_per_slice;
+    if (partial_bytes < (size_t)p.k_slices * M * N * sizeof(float)) return MIRROR_ERR_WORKSPACE;
+    p.n_units = n_tiles * p.n_chunks * p.k_slices;
+    int n_pairs = ctx->num_sms / 2;
+    if (n_pairs > p.n_units) n_pairs = p.n_units;
+    if (n_pairs < 1) return MIRROR_ERR_UNSUPPORTED;
+    p.w_keep = p.n_chunks > 1;
+    p.logits_out = partial;
+    p.status = ctx->d_status;
+    st = pair_launch(ctx, false, x, W, p, n_pairs, stream);
+    if (st != MIRROR_OK) return st;
+    *k_slices = p.k_slices;
     return MIRROR_OK;
 }
