@@ -261,6 +261,63 @@ mirror_status mirror_verify_step(mirror_ctx* ctx, const mirror_kv* kv, const mir
                                  const mirror_accept_out* out, void* attn_out, int32_t* argmax_out,
                                  void* stream);
 
+/* ------------------------------------------------------------------------------------------------------------
+ * The target's layers around the verify attention (the "target forward" of Sec. 3.1 that runs between the early
+ * exit and the final verification; Sec. 4.1 names pre-norm decoder stacks as targets).  The paper fixes no layer
+ * structure; this is the common pre-norm decoder layer: RMSNorm -> Q/K/V projection -> rotary embedding
+ * (rotate-half pairs i, i + d/2; angle = position * rope_theta^(-2i/d)) -> mirror_attn_verify for that layer ->
+ * output projection + residual -> RMSNorm -> SiLU(gate) * up -> down projection + residual.  Activations are stored
+ * in bf16 between the steps; sums are fp32.  Row r = (request, node) sits at position prefix_len[request] + depth(node).
+ * ------------------------------------------------------------------------------------------------------------ */
+typedef struct {
+    const void* w_qkv;      /* bf16 [(Hq + 2*Hkv)*d, H]: query rows, then key rows, then value rows */
+    const void* w_o;        /* bf16 [H, Hq*d] */
+    const void* w_gate_up;  /* bf16 [2*I, H]: gate rows, then up rows */
+    const void* w_down;     /* bf16 [H, I] */
+    const void* norm_attn;  /* bf16 [H]: RMSNorm weight ahead of attention */
+    const void* norm_mlp;   /* bf16 [H]: RMSNorm weight ahead of the MLP */
+} mirror_layer_weights;
+
+typedef struct {
+    int n_layers;                        /* layers to run; layer l uses kv layer l and k_new / v_new slab l */
+    int intermediate;                    /* I, a multiple of 64 (H and Hq*d must be multiples of 64 too) */
+    float rope_theta;                    /* e.g. 1e6 */
+    float rms_eps;                       /* e.g. 1e-6 */
+    const mirror_layer_weights* layers;  /* HOST array [n_layers] of device pointers */
+    const void* norm_final;              /* bf16 [H]: RMSNorm weight ahead of the LM head */
+} mirror_target;
+
+/* out[M, N] (bf16) = x[M, K] (bf16) * W[N, K]^T (bf16) (+ residual[M, N], bf16, nullable), fp32 accumulation, one
+ * rounding.  K a multiple of 64; x, W, out 16-byte aligned.  scratch: device memory of at least
+ * mirror_linear_scratch_bytes() bytes (fp32 partial sums of the K slices the GEMM is split into when it has fewer
+ * output tiles than the GPU has CTA pairs; the slices are added in a fixed order). */
+mirror_status mirror_linear_scratch_bytes(const mirror_ctx* ctx, int M, int N, int K, size_t* bytes);
+mirror_status mirror_linear(mirror_ctx* ctx, const void* x, int M, const void* W, int N, int K, const void* residual,
+                            void* out, void* scratch, size_t scratch_bytes, void* stream);
+
+/* out[M, H] (bf16) = x / sqrt(mean(x^2) + eps) * gamma, row by row (x bf16 [M, H], gamma bf16 [H]; H even). */
+mirror_status mirror_rmsnorm(mirror_ctx* ctx, const void* x, const void* gamma, int M, int H, float eps, void* out,
+                             void* stream);
+
+/* All layers of `t` on the step's rows, one after the other on `stream`:
+ *   x        bf16 [B*n, H]: the residual stream entering layer 0 (the embeddings of the tree's tokens); not written
+ *   kv, tree as for mirror_attn_verify (kv->num_layers >= t->n_layers; cached keys are already rotated)
+ *   q_out    bf16 [n_layers, B, n, Hq, d], k_new_out / v_new_out bf16 [n_layers, B, n, Hkv, d]: the projected and
+ *            rotated queries and the tree's own K/V of every layer (k_new_out / v_new_out are what
+ *            mirror_kv_commit appends afterwards)
+ *   attn_out bf16 [n_layers, B, n, Hq, d]
+ *   x_out    bf16 [B*n, H]: the residual stream after the last layer
+ *   hidden_out bf16 [B*n, H]: RMSNorm(x_out) with norm_final -- the LM-head rows (`hidden` of mirror_verify_step /
+ *            mirror_lmhead_reduce)
+ *   scratch  device memory of at least mirror_target_scratch_bytes() bytes
+ * Needs the workspace of mirror_attn_verify.  Per layer it enqueues 4 GEMMs, 4 fused finishing kernels (split-K sum
+ * + rotary embedding / residual + RMSNorm / SiLU gate) and the two attention kernels. */
+mirror_status mirror_target_scratch_bytes(const mirror_ctx* ctx, const mirror_tree* tree, const mirror_target* t,
+                                          size_t* bytes);
+mirror_status mirror_target_forward(mirror_ctx* ctx, const mirror_target* t, const mirror_kv* kv, const mirror_tree* tree,
+                                    const void* x, void* q_out, void* k_new_out, void* v_new_out, void* attn_out,
+                                    void* x_out, void* hidden_out, void* scratch, size_t scratch_bytes, void* stream);
+
 /* Optional timing hooks for mirror_verify_step: four cudaEvent_t (passed as void*) that every later
  * mirror_verify_step on this ctx records on its stream -- before attention, after attention, after the
  * LM-head GEMM kernel, after acceptance -- until cleared with NULL.  The caller owns the events. */

@@ -25,6 +25,7 @@ EXPORTS = [
     "mirror_attn_verify", "mirror_lmhead_reduce", "mirror_accept_select", "mirror_verify_step",
     "mirror_device_status", "mirror_launch_count", "mirror_status_str", "mirror_set_stage_events",
     "mirror_lmhead_reduce_noalloc", "mirror_early_exit_tap", "mirror_overlap_mass", "mirror_kv_commit",
+    "mirror_linear_scratch_bytes", "mirror_linear", "mirror_rmsnorm", "mirror_target_scratch_bytes", "mirror_target_forward",
 ]
 
 
@@ -42,6 +43,16 @@ class ModelDesc(C.Structure):
 class Tree(C.Structure):
     _fields_ = [("batch", C.c_int), ("n_nodes", C.c_int), ("kappa", C.c_int), ("gamma", C.c_int),
                 ("tokens", C.c_void_p), ("parent", C.POINTER(C.c_int32))]
+
+
+class LayerWeights(C.Structure):
+    _fields_ = [("w_qkv", C.c_void_p), ("w_o", C.c_void_p), ("w_gate_up", C.c_void_p), ("w_down", C.c_void_p),
+                ("norm_attn", C.c_void_p), ("norm_mlp", C.c_void_p)]
+
+
+class Target(C.Structure):
+    _fields_ = [("n_layers", C.c_int), ("intermediate", C.c_int), ("rope_theta", C.c_float), ("rms_eps", C.c_float),
+                ("layers", C.POINTER(LayerWeights)), ("norm_final", C.c_void_p)]
 
 
 class KV(C.Structure):
@@ -284,6 +295,68 @@ class Mirror:
                                          _ptr(v_new, torch.bfloat16, "v_new"), _ptr(res.accepted_nodes, torch.int32, "accepted_nodes"),
                                          _ptr(res.n_accepted, torch.int32, "n_accepted"), _ptr(prefix_len, torch.int32, "prefix_len"),
                                          _stream(stream)), "mirror_kv_commit")
+
+    # ---- the target's layers around the attention ---------------------------------------------
+    def target(self, layers: Sequence[dict], norm_final: torch.Tensor, intermediate: int, rope_theta: float = 1e6,
+               rms_eps: float = 1e-6) -> Target:
+        """layers: one dict per layer with bf16 CUDA tensors w_qkv, w_o, w_gate_up, w_down, norm_attn, norm_mlp."""
+        arr = (LayerWeights * len(layers))()
+        refs = [norm_final]
+        for i, w in enumerate(layers):
+            for f, _ in LayerWeights._fields_:
+                setattr(arr[i], f, _ptr(w[f], torch.bfloat16, f).value)
+                refs.append(w[f])
+        t = Target(len(layers), intermediate, rope_theta, rms_eps, arr, _ptr(norm_final, torch.bfloat16, "norm_final"))
+        t._refs = (arr, refs)
+        return t
+
+    def mirror_linear(self, x: torch.Tensor, W: torch.Tensor, residual: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        """x [M, K] @ W [N, K]^T (+ residual [M, N]) -> bf16 [M, N]."""
+        M, K = x.shape
+        N = W.shape[0]
+        need = C.c_size_t()
+        _check(self.lib.mirror_linear_scratch_bytes(self._ctx, M, N, K, C.byref(need)), "mirror_linear_scratch_bytes")
+        scratch = getattr(self, "_linear_scratch", None)          # grown on demand; calls on one stream may share it
+        if scratch is None or scratch.numel() < need.value:
+            scratch = self._linear_scratch = torch.empty(max(need.value, 256), dtype=torch.uint8, device=self.device)
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=self.device)
+        _check(self.lib.mirror_linear(self._ctx, _ptr(x, torch.bfloat16, "x"), M, _ptr(W, torch.bfloat16, "W"), N, K,
+                                      _ptr(residual, torch.bfloat16, "residual"), _ptr(out), _ptr(scratch),
+                                      C.c_size_t(scratch.numel()), _stream(stream)), "mirror_linear")
+        return out
+
+    def mirror_rmsnorm(self, x: torch.Tensor, gamma: torch.Tensor, eps: float = 1e-6, stream=None) -> torch.Tensor:
+        M, H = x.shape
+        out = torch.empty_like(x)
+        _check(self.lib.mirror_rmsnorm(self._ctx, _ptr(x, torch.bfloat16, "x"), _ptr(gamma, torch.bfloat16, "gamma"), M, H,
+                                       C.c_float(eps), _ptr(out), _stream(stream)), "mirror_rmsnorm")
+        return out
+
+    def target_scratch(self, tree: Tree, target: Target) -> torch.Tensor:
+        need = C.c_size_t()
+        _check(self.lib.mirror_target_scratch_bytes(self._ctx, C.byref(tree), C.byref(target), C.byref(need)),
+               "mirror_target_scratch_bytes")
+        return torch.empty(need.value, dtype=torch.uint8, device=self.device)
+
+    def mirror_target_forward(self, target: Target, kv: KV, tree: Tree, x: torch.Tensor, scratch: Optional[torch.Tensor] = None,
+                              out: Optional[dict] = None, stream=None) -> dict:
+        """All layers of `target` on the residual rows x [B*n, H]; returns q, k_new, v_new, attn_out ([L, B, n, heads, d]),
+        x_out and hidden (the LM-head rows)."""
+        L, B, n = target.n_layers, tree.batch, tree.n_nodes
+        Hq, Hkv, d = self.desc.n_q_heads, self.desc.n_kv_heads, self.desc.head_dim
+        if scratch is None:
+            scratch = self.target_scratch(tree, target)
+        if out is None:
+            e = lambda *shape: torch.empty(shape, dtype=torch.bfloat16, device=self.device)
+            out = dict(q=e(L, B, n, Hq, d), k_new=e(L, B, n, Hkv, d), v_new=e(L, B, n, Hkv, d), attn_out=e(L, B, n, Hq, d),
+                       x_out=torch.empty_like(x), hidden=torch.empty_like(x))
+        self.ensure_workspace(tree, kv, WS_ATTN)
+        _check(self.lib.mirror_target_forward(self._ctx, C.byref(target), C.byref(kv), C.byref(tree), _ptr(x, torch.bfloat16, "x"),
+                                              _ptr(out["q"]), _ptr(out["k_new"]), _ptr(out["v_new"]), _ptr(out["attn_out"]),
+                                              _ptr(out["x_out"]), _ptr(out["hidden"]), _ptr(scratch), C.c_size_t(scratch.numel()),
+                                              _stream(stream)), "mirror_target_forward")
+        out["_scratch"] = scratch
+        return out
 
     def mirror_accept_select(self, tree: Tree, acc: AcceptIn, out: Optional[AcceptResult] = None, stream=None,
                              tree_scratch: bool = False) -> AcceptResult:

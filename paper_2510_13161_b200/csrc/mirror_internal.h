@@ -68,6 +68,11 @@ mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, c
 int mirror_lmhead_pair_partials(int V);
 mirror_status mirror_lmhead_pair_launch(mirror_ctx* ctx, const void* hidden, int M, const void* W, float* logits_out,
                                         void* partial_ws, size_t partial_bytes, cudaStream_t stream, int* n_partials);
+// Plain GEMM on CTA pairs: partial[s][M][N] (fp32) = x[M, K-slice s] * W[N, K-slice s]^T for the *k_slices slices that
+// mirror_linear_slices() picks (1 when the output tiles alone fill the GPU); the caller adds the slices in order.
+int mirror_linear_slices(const mirror_ctx* ctx, int M, int N, int K);
+mirror_status mirror_linear_partial_launch(mirror_ctx* ctx, const void* x, int M, const void* W, int N, int K, float* partial,
+                                           size_t partial_bytes, cudaStream_t stream, int* k_slices);
 mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const MirrorTreeInfo& ti,
                                  const void* q, const void* k_new, const void* v_new, void* out, float* lse_out,
                                  float* partial_ws, cudaStream_t stream);

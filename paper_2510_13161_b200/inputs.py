@@ -218,6 +218,29 @@ def gen_verify_inputs(cfg: VerifyConfig, seed: int = 0, device: str = "cpu", *,
     return out
 
 
+def gen_layer_weights(cfg: VerifyConfig, intermediate: int, layers: int, seed: int = 0, device: str = "cpu",
+                      w_std: Optional[float] = None):
+    """Seeded weights of `layers` pre-norm decoder layers for the shape of `cfg` (bf16): per layer a dict with w_qkv
+    [(Hq + 2 Hkv) d, H] (query, key, value rows), w_o [H, Hq d], w_gate_up [2 I, H] (gate, up rows), w_down [H, I] and
+    the two RMSNorm weights [H] (around 1); plus the final norm weight and the residual rows x [B n, H] that enter
+    layer 0 (stand-ins for the embeddings of the tree's tokens).  Returns (list of dicts, norm_final, x)."""
+    H, Hq, Hkv, d = cfg.hidden, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+    std = cfg.w_std if w_std is None else w_std
+    bf = torch.bfloat16
+    out = []
+    for l in range(layers):
+        g = lambda name: _gen(device, seed, f"layer{l}.{name}")
+        norm = lambda name: (1.0 + 0.1 * torch.empty(H, dtype=torch.float32, device=device).normal_(0.0, 1.0, generator=g(name))).to(bf)
+        out.append(dict(w_qkv=_normal(((Hq + 2 * Hkv) * d, H), std, bf, device, g("w_qkv")),
+                        w_o=_normal((H, Hq * d), std, bf, device, g("w_o")),
+                        w_gate_up=_normal((2 * intermediate, H), std, bf, device, g("w_gate_up")),
+                        w_down=_normal((H, intermediate), std, bf, device, g("w_down")),
+                        norm_attn=norm("norm_attn"), norm_mlp=norm("norm_mlp")))
+    norm_final = (1.0 + 0.1 * torch.empty(H, dtype=torch.float32, device=device).normal_(0.0, 1.0, generator=_gen(device, seed, "norm_final"))).to(bf)
+    x = _normal((cfg.rows, H), 1.0, bf, device, _gen(device, seed, "x_embed"))
+    return out, norm_final, x
+
+
 def bf16_bits(t: torch.Tensor):
     """numpy uint16 view of a bf16 tensor's bits (host copy)."""
     return t.detach().to("cpu").contiguous().view(torch.uint16).numpy()
