@@ -40,6 +40,11 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--accept-mode", default=None, choices=["greedy", "spec_sampling", "spec_tree"],
                     help="override the workload's acceptance rule")
+    ap.add_argument("--target-layers", type=int, default=0,
+                    help="also time mirror_target_forward (projections, rotary embedding, attention, MLP) over this many "
+                         "decoder layers of the workload's shape with seeded random weights (0.66 GB per layer for the default "
+                         "workload); reported under stages.target_forward, outside the timed region")
+    ap.add_argument("--intermediate", type=int, default=17408, help="MLP width for --target-layers")
     ap.add_argument("--layers", type=int, default=None,
                     help="profiling aid: run the workload with this many attention layers (config.layers reports it); "
                          "the default, the workload's own layer count, is the only valid bench configuration")
@@ -277,6 +282,39 @@ def attn_per_layer(m, x, tree, cfg, reps: int = 10):
     return res
 
 
+def target_forward_stage(m, x, tree, kv, cfg, n_layers: int, intermediate: int, hbm_gbs: float, reps: int = 5):
+    """mirror_target_forward over n_layers decoder layers of the workload's shape (random weights): ms, weight bytes per
+    second against the HBM peak.  The layers are weight streams at these row counts."""
+    import torch
+    from paper_2510_13161_b200 import inputs as I
+    dev = x.q.device
+    layers, norm_final, emb = I.gen_layer_weights(cfg, intermediate, n_layers, 0, dev)
+    tgt = m.target(layers, norm_final, intermediate, 1.0e6, 1e-6)
+    scratch = m.target_scratch(tree, tgt)
+    out = m.mirror_target_forward(tgt, kv, tree, emb, scratch=scratch)
+    for _ in range(2):
+        m.mirror_target_forward(tgt, kv, tree, emb, scratch=scratch, out=out)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    l0 = m.launch_count()
+    e0.record()
+    for _ in range(reps):
+        m.mirror_target_forward(tgt, kv, tree, emb, scratch=scratch, out=out)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    code, detail = m.device_status()
+    if code != 0:
+        raise SystemExit(f"device status {code} (detail {detail}) in mirror_target_forward")
+    H, Hq, Hkv, d = cfg.hidden, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+    w_bytes = 2 * ((Hq + 2 * Hkv) * d * H + H * Hq * d + 2 * intermediate * H + H * intermediate)
+    kv_bytes = 2 * 2 * sum(int(l) for l in x.prefix_len.cpu().tolist()) * Hkv * d
+    gbs = (w_bytes + kv_bytes) * n_layers / (ms * 1e-3) / 1e9
+    return {"layers": n_layers, "intermediate": intermediate, "ms": ms, "us_per_layer": ms / n_layers * 1e3,
+            "bytes_per_layer": w_bytes + kv_bytes, "gbs": gbs, "frac_hbm": gbs / hbm_gbs,
+            "kernel_launches": (m.launch_count() - l0) // reps}
+
+
 def run_mirror(args):
     import torch
     import torch.distributed as dist
@@ -404,6 +442,9 @@ def run_mirror(args):
     # ---- attention with one launch pair per layer: the order a real target enforces (layer l+1's queries depend on
     # layer l's output), as plain stream-ordered launches and replayed from a CUDA graph.  Outside the timed region.
     stages["attn_per_layer_ms"] = attn_per_layer(m, x, tree, cfg)
+    if args.target_layers > 0:
+        stages["target_forward"] = target_forward_stage(m, x, tree, kv, cfg, min(args.target_layers, cfg.layers), args.intermediate,
+                                                        peaks["hbm_gbs"])
 
     cpu = None
     if not args.no_cpu_baseline and world == 1:

@@ -903,6 +903,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 // columns in group order, so a unit that many CTAs shared (few units per launch, long contexts) is not merged by one
 // block alone.  Blocks whose boundary coincides with a unit boundary have nothing to do.
 constexpr int kMergeThreads = 512;        // 128 rows x 4 column quarters
+constexpr int kMergeMaxGroups = 512;      // groups whose first tiles fit the lookup table (more: computed on demand)
 template <int D>
 __global__ void __launch_bounds__(kMergeThreads) attn_merge_kernel(const AttnParams p) {
     __shared__ int cumT[kMaxBatch + 1];
@@ -926,15 +927,24 @@ __global__ void __launch_bounds__(kMergeThreads) attn_merge_kernel(const AttnPar
     const Partition part = make_partition(p, cumT);
     const int g = blockIdx.x + 1, rb = blockIdx.y;
     if (g >= part.n_groups || part.total_tiles >= (1ll << 31)) return;
-    const long long x = group_begin(part, g, p, cumT);
+    // every group's first tile, computed side by side (a unit shared by many groups is looked up from here instead of
+    // by a chain of dependent calls)
+    __shared__ long long s_begin[kMergeMaxGroups];
+    const bool tabled = part.n_groups <= kMergeMaxGroups;
+    if (tabled) {
+        for (int t = tid; t < part.n_groups; t += kMergeThreads) s_begin[t] = group_begin(part, t, p, cumT);
+        __syncthreads();
+    }
+    auto begin_of = [&](int t) -> long long { return tabled ? s_begin[t] : group_begin(part, t, p, cumT); };
+    const long long x = begin_of(g);
     const UnitPos u = locate(x, p, cumT, part.tiles_per_layer);
     if (u.tile_in_unit == 0) return;                                            // the boundary is a unit boundary
     // the groups ga..gb hold this unit's parts; the blocks of the boundaries ga+1..gb share the merge by columns
     int ga = g - 1;
-    while (ga > 0 && group_begin(part, ga, p, cumT) > u.unit_first_tile) --ga;
+    while (ga > 0 && begin_of(ga) > u.unit_first_tile) --ga;
     int gb = g;
     const long long unit_last = u.unit_first_tile + u.tiles_in_unit - 1;
-    while (gb + 1 < part.n_groups && group_begin(part, gb + 1, p, cumT) <= unit_last) ++gb;
+    while (gb + 1 < part.n_groups && begin_of(gb + 1) <= unit_last) ++gb;
     const int parts = gb - ga + 1;
     const int n_blocks = parts - 1, j_blk = g - (ga + 1);
     // launched with programmatic stream serialization: everything above overlaps the attention kernel's tail;

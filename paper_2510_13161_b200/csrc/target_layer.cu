@@ -47,51 +47,80 @@ __global__ void rope_table_kernel(const int32_t* prefix_len, const TreeDepths td
 }
 
 // Q/K/V projection finish: split-K sum, rotary embedding on the query and key heads, bf16 stores into the step's
-// [M, Hq, d] / [M, Hkv, d] tensors.  One block per row.
-__global__ void __launch_bounds__(kFinThreads)
-finish_qkv_kernel(const float* partial, int slices, int M, int Hq, int Hkv, int d, const float2* cs, __nv_bfloat16* q_out,
-                  __nv_bfloat16* k_out, __nv_bfloat16* v_out) {
+// [M, Hq, d] / [M, Hkv, d] tensors.  One block per (row, head), one thread per rotation pair (f, f + d/2); all
+// slices of a thread's two columns are loaded before they are added (the loads are independent, the order of the sum
+// is fixed).
+__global__ void finish_qkv_kernel(const float* partial, int slices, int M, int Hq, int Hkv, int d, const float2* cs,
+                                  __nv_bfloat16* q_out, __nv_bfloat16* k_out, __nv_bfloat16* v_out) {
     ptx::grid_dep_wait();
     ptx::grid_dep_launch();
-    const int row = blockIdx.x, half = d >> 1;
+    const int row = blockIdx.x, head = blockIdx.y, half = d >> 1, f = threadIdx.x;
+    if (f >= half) return;
     const int N = (Hq + 2 * Hkv) * d;
-    const size_t MN = (size_t)M * N, base = (size_t)row * N;
-    for (int idx = threadIdx.x; idx < (Hq + Hkv) * half; idx += kFinThreads) {
-        const int head = idx / half, f = idx - head * half;
-        const int col = head * d + f;
-        const float a = sum_slices(partial, slices, MN, base + col), b = sum_slices(partial, slices, MN, base + col + half);
+    const size_t MN = (size_t)M * N;
+    const float* p0 = partial + (size_t)row * N + (size_t)head * d + f;
+    float a = 0.f, b = 0.f;
+#pragma unroll 8
+    for (int s = 0; s < slices; ++s) {
+        a += p0[(size_t)s * MN];
+        b += p0[(size_t)s * MN + half];
+    }
+    if (head < Hq + Hkv) {
         const float2 t = cs[(size_t)row * half + f];
         const float ra = a * t.x - b * t.y, rb = b * t.x + a * t.y;
         __nv_bfloat16* dst = head < Hq ? q_out + ((size_t)row * Hq + head) * d : k_out + ((size_t)row * Hkv + (head - Hq)) * d;
         dst[f] = __float2bfloat16_rn(ra);
         dst[f + half] = __float2bfloat16_rn(rb);
+    } else {
+        __nv_bfloat16* dst = v_out + ((size_t)row * Hkv + (head - Hq - Hkv)) * d;
+        dst[f] = __float2bfloat16_rn(a);
+        dst[f + half] = __float2bfloat16_rn(b);
     }
-    const int v0 = (Hq + Hkv) * d;
-    for (int idx = threadIdx.x; idx < Hkv * d; idx += kFinThreads)
-        v_out[(size_t)row * Hkv * d + idx] = __float2bfloat16_rn(sum_slices(partial, slices, MN, base + v0 + idx));
 }
 
 // Residual add + RMSNorm: r = residual + split-K sum, x_out = bf16(r); normed = bf16(x_out / sqrt(mean(x_out^2) + eps)
-// * gamma) (from the ROUNDED x_out: what a later reader of x_out would compute).  One block per row, the row kept in
-// shared memory between the two passes.  partial == nullptr: plain RMSNorm of `residual`; gamma == nullptr: no norm.
-__global__ void __launch_bounds__(kFinThreads)
+// * gamma) (from the ROUNDED x_out: what a later reader of x_out would compute).  One block of 1024 threads per row;
+// a thread keeps its columns (every 1024th) in registers between the two passes and issues the loads of all slices
+// of all its columns before adding them (in slice order).  partial == nullptr: plain RMSNorm of `residual`;
+// gamma == nullptr: no norm.
+constexpr int kNormThreads = 1024;
+constexpr int kNormCols = 16;                 // columns per thread: rows of up to 16384 elements
+__global__ void __launch_bounds__(kNormThreads)
 finish_residual_norm_kernel(const float* partial, int slices, int M, int H, const __nv_bfloat16* residual,
                             const __nv_bfloat16* gamma, float eps, __nv_bfloat16* x_out, __nv_bfloat16* normed) {
-    extern __shared__ float s_row[];
-    __shared__ float s_red[kFinThreads / 32];
+    __shared__ float s_red[kNormThreads / 32];
     ptx::grid_dep_wait();
     ptx::grid_dep_launch();
     const int row = blockIdx.x;
     const size_t MN = (size_t)M * H, base = (size_t)row * H;
+    float r[kNormCols];
+#pragma unroll
+    for (int c = 0; c < kNormCols; ++c) {
+        const int col = threadIdx.x + c * kNormThreads;
+        r[c] = col < H ? __bfloat162float(residual[base + col]) : 0.f;
+    }
+    if (partial) {
+        for (int s = 0; s < slices; ++s) {
+            float v[kNormCols];
+#pragma unroll
+            for (int c = 0; c < kNormCols; ++c) {
+                const int col = threadIdx.x + c * kNormThreads;
+                v[c] = col < H ? partial[(size_t)s * MN + base + col] : 0.f;
+            }
+#pragma unroll
+            for (int c = 0; c < kNormCols; ++c) r[c] += v[c];
+        }
+    }
     float ss = 0.f;
-    for (int col = threadIdx.x; col < H; col += kFinThreads) {
-        float r = __bfloat162float(residual[base + col]);
-        if (partial) r += sum_slices(partial, slices, MN, base + col);
-        const __nv_bfloat16 xb = __float2bfloat16_rn(r);
-        if (x_out) x_out[base + col] = xb;
-        const float xf = __bfloat162float(xb);
-        s_row[col] = xf;
-        ss = fmaf(xf, xf, ss);
+#pragma unroll
+    for (int c = 0; c < kNormCols; ++c) {
+        const int col = threadIdx.x + c * kNormThreads;
+        if (col < H) {
+            const __nv_bfloat16 xb = __float2bfloat16_rn(r[c]);
+            if (x_out) x_out[base + col] = xb;
+            r[c] = __bfloat162float(xb);
+            ss = fmaf(r[c], r[c], ss);
+        }
     }
     if (!gamma || !normed) return;
 #pragma unroll
@@ -100,10 +129,13 @@ finish_residual_norm_kernel(const float* partial, int slices, int M, int H, cons
     __syncthreads();
     float tot = 0.f;
 #pragma unroll
-    for (int w = 0; w < kFinThreads / 32; ++w) tot += s_red[w];                // same order in every thread
+    for (int w = 0; w < kNormThreads / 32; ++w) tot += s_red[w];               // same order in every thread
     const float rinv = 1.0f / sqrtf(tot / (float)H + eps);
-    for (int col = threadIdx.x; col < H; col += kFinThreads)
-        normed[base + col] = __float2bfloat16_rn(s_row[col] * rinv * __bfloat162float(gamma[col]));
+#pragma unroll
+    for (int c = 0; c < kNormCols; ++c) {
+        const int col = threadIdx.x + c * kNormThreads;
+        if (col < H) normed[base + col] = __float2bfloat16_rn(r[c] * rinv * __bfloat162float(gamma[col]));
+    }
 }
 
 // Gated MLP finish: act[row, j] = bf16(silu(gate) * up), gate = sum of column j, up = sum of column I + j.
@@ -196,11 +228,9 @@ extern "C" mirror_status mirror_linear(mirror_ctx* ctx, const void* x, int M, co
 extern "C" mirror_status mirror_rmsnorm(mirror_ctx* ctx, const void* x, const void* gamma, int M, int H, float eps, void* out,
                                         void* stream) {
     if (!ctx || !x || !gamma || !out || M <= 0 || H <= 0) return MIRROR_ERR_ARG;
-    if ((size_t)H * sizeof(float) > 200 * 1024) return MIRROR_ERR_SHAPE;
+    if (H > kNormThreads * kNormCols) return MIRROR_ERR_SHAPE;
     MIRROR_CUDA_OK(cudaSetDevice(ctx->device));
-    if ((size_t)H * sizeof(float) > 48 * 1024)
-        MIRROR_CUDA_OK(cudaFuncSetAttribute(finish_residual_norm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-    MIRROR_CUDA_OK(mirror_launch_pdl(finish_residual_norm_kernel, dim3(M), dim3(kFinThreads), (size_t)H * sizeof(float),
+    MIRROR_CUDA_OK(mirror_launch_pdl(finish_residual_norm_kernel, dim3(M), dim3(kNormThreads), 0,
                                      (cudaStream_t)stream, (const float*)nullptr, 0, M, H, (const __nv_bfloat16*)x,
                                      (const __nv_bfloat16*)gamma, eps, (__nv_bfloat16*)nullptr, (__nv_bfloat16*)out));
     ctx->launches += 1;
@@ -224,7 +254,7 @@ extern "C" mirror_status mirror_target_forward(mirror_ctx* ctx, const mirror_tar
     if (!t->layers || !t->norm_final || t->n_layers <= 0 || t->n_layers > kv->num_layers) return MIRROR_ERR_ARG;
     const int H = ctx->desc.hidden, Hq = ctx->desc.n_q_heads, Hkv = ctx->desc.n_kv_heads, d = ctx->desc.head_dim, I = t->intermediate;
     if (I <= 0 || I % 64 != 0 || H % 64 != 0 || (Hq * d) % 64 != 0 || (d & 1)) return MIRROR_ERR_SHAPE;
-    if ((size_t)H * sizeof(float) > 200 * 1024) return MIRROR_ERR_SHAPE;
+    if (H > kNormThreads * kNormCols || d / 2 > 1024) return MIRROR_ERR_SHAPE;
     if (!kv->k_pool || !kv->v_pool || !kv->page_table || !kv->prefix_len) return MIRROR_ERR_ARG;
     if (((uintptr_t)x & 15) || ((uintptr_t)scratch & 255)) return MIRROR_ERR_ARG;
     for (int l = 0; l < t->n_layers; ++l) {
@@ -249,9 +279,6 @@ extern "C" mirror_status mirror_target_forward(mirror_ctx* ctx, const mirror_tar
     __nv_bfloat16* act = (__nv_bfloat16*)(base + sc.act);
     __nv_bfloat16* xa = (__nv_bfloat16*)(base + sc.xa);
     __nv_bfloat16* xb = (__nv_bfloat16*)(base + sc.xb);
-    const size_t row_smem = (size_t)H * sizeof(float);
-    if (row_smem > 48 * 1024)
-        MIRROR_CUDA_OK(cudaFuncSetAttribute(finish_residual_norm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
 
     TreeDepths td;
     for (int i = 0; i < MIRROR_MAX_NODES; ++i) td.depth[i] = i < n ? ti.depth[i] : 0;
@@ -260,7 +287,7 @@ extern "C" mirror_status mirror_target_forward(mirror_ctx* ctx, const mirror_tar
                                      (double)t->rope_theta, cs));
     ctx->launches += 1;
     // the first layer's input norm; every later one comes out of the finish kernel of the layer before
-    MIRROR_CUDA_OK(mirror_launch_pdl(finish_residual_norm_kernel, dim3(M), dim3(kFinThreads), row_smem, s, (const float*)nullptr, 0, M, H,
+    MIRROR_CUDA_OK(mirror_launch_pdl(finish_residual_norm_kernel, dim3(M), dim3(kNormThreads), 0, s, (const float*)nullptr, 0, M, H,
                                      (const __nv_bfloat16*)x, (const __nv_bfloat16*)t->layers[0].norm_attn, t->rms_eps,
                                      (__nv_bfloat16*)nullptr, h));
     ctx->launches += 1;
@@ -279,7 +306,7 @@ extern "C" mirror_status mirror_target_forward(mirror_ctx* ctx, const mirror_tar
         // Q/K/V projection + rotary embedding
         st = mirror_linear_partial_launch(ctx, h, M, w.w_qkv, Nqkv, H, partial, sc.partial_bytes, s, &slices);
         if (st != MIRROR_OK) return st;
-        MIRROR_CUDA_OK(mirror_launch_pdl(finish_qkv_kernel, dim3(M), dim3(kFinThreads), 0, s, (const float*)partial, slices, M, Hq, Hkv, d,
+        MIRROR_CUDA_OK(mirror_launch_pdl(finish_qkv_kernel, dim3(M, Hq + 2 * Hkv), dim3(half), 0, s, (const float*)partial, slices, M, Hq, Hkv, d,
                                          (const float2*)cs, q_l, k_l, v_l));
         ctx->launches += 1;
         // attention of this layer over its slab of the cache
@@ -292,7 +319,7 @@ extern "C" mirror_status mirror_target_forward(mirror_ctx* ctx, const mirror_tar
         // output projection + residual + the MLP's norm
         st = mirror_linear_partial_launch(ctx, a_l, M, w.w_o, H, Hq * d, partial, sc.partial_bytes, s, &slices);
         if (st != MIRROR_OK) return st;
-        MIRROR_CUDA_OK(mirror_launch_pdl(finish_residual_norm_kernel, dim3(M), dim3(kFinThreads), row_smem, s, (const float*)partial, slices,
+        MIRROR_CUDA_OK(mirror_launch_pdl(finish_residual_norm_kernel, dim3(M), dim3(kNormThreads), 0, s, (const float*)partial, slices,
                                          M, H, x_cur, (const __nv_bfloat16*)w.norm_mlp, t->rms_eps, xa, h));
         ctx->launches += 1;
         // gate / up projection + SiLU gate
@@ -306,7 +333,7 @@ extern "C" mirror_status mirror_target_forward(mirror_ctx* ctx, const mirror_tar
         if (st != MIRROR_OK) return st;
         const void* g_next = last ? t->norm_final : t->layers[l + 1].norm_attn;
         __nv_bfloat16* x_new = last ? (__nv_bfloat16*)x_out : xb;
-        MIRROR_CUDA_OK(mirror_launch_pdl(finish_residual_norm_kernel, dim3(M), dim3(kFinThreads), row_smem, s, (const float*)partial, slices,
+        MIRROR_CUDA_OK(mirror_launch_pdl(finish_residual_norm_kernel, dim3(M), dim3(kNormThreads), 0, s, (const float*)partial, slices,
                                          M, H, (const __nv_bfloat16*)xa, (const __nv_bfloat16*)g_next, t->rms_eps, x_new,
                                          last ? (__nv_bfloat16*)hidden_out : h));
         ctx->launches += 1;
