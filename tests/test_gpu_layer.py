@@ -138,3 +138,42 @@ def test_target_forward_feeds_the_verify_step():
     logits = O.lmhead_logits(I.bf16_bits(out["hidden"]), I.bf16_bits(W))
     ref = O.row_reduce(logits, 1.0, 0)
     np.testing.assert_allclose(res["lse"].cpu().numpy(), ref["lse"], atol=2e-3)
+
+
+def test_argument_and_shape_errors_are_reported_not_launched():
+    from paper_2510_13161_b200 import binding as Bn
+    import ctypes as C
+    cfg = I.VerifyConfig("t", 256, 4, 2, 64, 1, 1, 16, 16, 2, 4, 1024, "greedy")
+    m = make_mirror(cfg)
+    x, W = rand_bf16((4, 96), 1.0, 1).cuda(), rand_bf16((128, 96), 0.05, 2).cuda()
+    with pytest.raises(Bn.MirrorError) as e:                     # K = 96 is not a multiple of 64
+        m.mirror_linear(x, W)
+    assert e.value.code == 2
+    # scratch too small for the K slices
+    x, W = rand_bf16((4, 1024), 1.0, 1).cuda(), rand_bf16((256, 1024), 0.05, 2).cuda()
+    out = torch.empty((4, 256), dtype=torch.bfloat16, device="cuda")
+    tiny = torch.empty(256, dtype=torch.uint8, device="cuda")
+    rc = m.lib.mirror_linear(m._ctx, C.c_void_p(x.data_ptr()), 4, C.c_void_p(W.data_ptr()), 256, 1024, None, C.c_void_p(out.data_ptr()),
+                             C.c_void_p(tiny.data_ptr()), C.c_size_t(256), None)
+    assert rc != 0 and b"workspace" in m.lib.mirror_status_str(rc).lower()
+    # null output
+    rc = m.lib.mirror_linear(m._ctx, C.c_void_p(x.data_ptr()), 4, C.c_void_p(W.data_ptr()), 256, 1024, None, None,
+                             C.c_void_p(tiny.data_ptr()), C.c_size_t(256), None)
+    assert rc != 0
+    assert m.device_status() == (0, 0)
+
+
+def test_root_only_tree_and_single_token_prefix():
+    """n = 1 (no draft tokens: a plain decode step) and a one-token prefix."""
+    case = dict(H=256, Hq=4, Hkv=2, d=64, inter=256, L=1, B=2, lo=1, hi=1, kappa=1, gamma=1, seed=7, parent=[-1])
+    cfg, x, layers, norm_final, emb = layer_case(**case)
+    ref = run_oracle(cfg, x, layers, norm_final, emb, 1.0e4, 1e-6)
+    m = make_mirror(cfg)
+    dev = lambda t: t.cuda()
+    tgt = m.target([{k: dev(v) for k, v in w.items()} for w in layers], dev(norm_final), case["inter"], 1.0e4, 1e-6)
+    kv = m.kv(dev(x.k_pool), dev(x.v_pool), dev(x.page_table), dev(x.prefix_len))
+    tree = m.tree(dev(x.tokens), cfg.kappa, cfg.gamma, parent=[-1])
+    out = m.mirror_target_forward(tgt, kv, tree, dev(emb))
+    assert m.device_status() == (0, 0)
+    close(out["q"][0], ref[0]["q"], "q0", ulps=1.5, exact_frac=0.99)
+    close(out["x_out"], ref[-1]["x"], "x_out", ulps=3.0, exact_frac=0.4)
