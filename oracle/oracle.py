@@ -202,3 +202,25 @@ def overlap_mass(q_final, ids) -> float:
     """Eq. 7: Omega_kappa, the final distribution's mass on the early-exit Top-kappa ids."""
     q_final = _c(q_final, np.float64); ids = _c(ids, np.int32)
     return float(lib().oracle_overlap_mass(_p(q_final), _p(ids), ids.shape[0]))
+
+
+def trie_build(branch_tokens, root_token: int):
+    """Token tree without duplicated prefixes out of kappa branches of gamma tokens (the branch-complete proposal of
+    Sec. 3.1 as a tree, "tree drafts"): branches that agree on their first r tokens share their first r nodes.  Written
+    as the definition: a node per distinct non-empty prefix, numbered in order of first appearance (branch by branch,
+    left to right), parent = the node of the prefix one token shorter (the root for length 1).
+    Returns (parent [n], tokens [n], node_of [kappa, gamma])."""
+    bt = np.asarray(branch_tokens, np.int64)
+    kappa, gamma = bt.shape
+    ids = {(): 0}
+    parent, tokens = [-1], [int(root_token)]
+    node_of = np.zeros((kappa, gamma), np.int32)
+    for i in range(kappa):
+        for j in range(gamma):
+            pre = tuple(int(t) for t in bt[i, :j + 1])
+            if pre not in ids:
+                ids[pre] = len(parent)
+                parent.append(ids[pre[:-1]])
+                tokens.append(pre[-1])
+            node_of[i, j] = ids[pre]
+    return np.asarray(parent, np.int32), np.asarray(tokens, np.int32), node_of

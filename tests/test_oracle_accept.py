@@ -384,3 +384,34 @@ def test_tree_rule_walk_order_on_a_two_level_tree():
     item = tree_inputs(p_rows, q_rows, [1, 0, 2, 2, 1], [0.0, 0.9, 0.0, 0.5, 0.5, 0.0], [0.5] * 6)
     o = batch_tree([item], parent, 2, emit_bonus=False)
     assert o["n_emitted"][0] == 2 and o["emitted"][0].tolist() == [0, 1, -1]
+
+
+def test_trie_build_shares_exactly_the_common_prefixes():
+    """Pins of the de-duplicated tree: a hand-worked case, and on random branches the brute-force properties that
+    define it (one node per distinct prefix, every branch recovered by walking up from its leaf)."""
+    bt = [[5, 7, 9], [5, 7, 2], [5, 1, 9], [4, 7, 9]]
+    parent, tokens, node_of = O.trie_build(bt, 99)
+    # prefixes in order of appearance: (5) (5,7) (5,7,9) | (5,7,2) | (5,1) (5,1,9) | (4) (4,7) (4,7,9)
+    assert parent.tolist() == [-1, 0, 1, 2, 2, 1, 5, 0, 7, 8]
+    assert tokens.tolist() == [99, 5, 7, 9, 2, 1, 9, 4, 7, 9]
+    assert node_of.tolist() == [[1, 2, 3], [1, 2, 4], [1, 5, 6], [7, 8, 9]]
+    rng = np.random.default_rng(0)
+    for _ in range(50):
+        kappa, gamma = int(rng.integers(1, 7)), int(rng.integers(1, 6))
+        bt = rng.integers(0, 3, size=(kappa, gamma))                      # tiny alphabet: many shared prefixes
+        parent, tokens, node_of = O.trie_build(bt, 7)
+        prefixes = {tuple(bt[i, :j + 1]) for i in range(kappa) for j in range(gamma)}
+        assert len(parent) == 1 + len(prefixes)
+        assert all(parent[i] < i for i in range(1, len(parent))) and parent[0] == -1
+        for i in range(kappa):
+            node, seq = int(node_of[i, gamma - 1]), []
+            while node != 0:
+                seq.append(int(tokens[node])); node = int(parent[node])
+            assert seq[::-1] == bt[i].tolist()
+        # identical branches end in the same leaf; branches that differ somewhere do not
+        for a in range(kappa):
+            for b in range(kappa):
+                assert (node_of[a, gamma - 1] == node_of[b, gamma - 1]) == bool(np.array_equal(bt[a], bt[b]))
+    # no sharing at all reproduces the comb tree
+    parent, tokens, node_of = O.trie_build([[1, 2], [3, 4]], 0)
+    assert parent.tolist() == [-1, 0, 1, 0, 3] and node_of.tolist() == [[1, 2], [3, 4]]
