@@ -248,6 +248,17 @@ mirror_status mirror_kv_commit(mirror_ctx* ctx, const mirror_kv* kv, const mirro
                                const void* v_new, const int32_t* accepted_nodes, const int32_t* n_accepted,
                                int32_t* prefix_len, void* stream);
 
+/* HOST helper (no device work): merge kappa branches of gamma tokens -- the branch-complete proposal of Sec. 3.1 --
+ * into a token tree without duplicated prefixes ("tree drafts"): branches that agree on their first r tokens share
+ * their first r nodes, so shared tokens are scored once.  All pointers are HOST pointers.
+ *   branch_tokens int32 [kappa, gamma]; root_token: the last committed token (node 0)
+ *   parent, tokens int32 [1 + kappa*gamma] (capacity; *n_nodes entries are written): node ids in order of first
+ *                  appearance, parent[i] < i -- the arrays mirror_tree takes (tokens go to the device per request)
+ *   node_of        int32 [kappa, gamma]: the node that holds position j of branch i
+ * kappa <= MIRROR_MAX_BRANCHES, gamma <= MIRROR_MAX_DEPTH, at most MIRROR_MAX_NODES nodes (else MIRROR_ERR_SHAPE). */
+mirror_status mirror_trie_build(const int32_t* branch_tokens, int kappa, int gamma, int32_t root_token, int32_t* parent,
+                                int32_t* tokens, int32_t* node_of, int* n_nodes);
+
 /* One whole verify step on one stream: attention over all layers -> LM head rows -> reductions -> acceptance.
  *   hidden   bf16 [B*n, H], or NULL to feed the last layer's attention output (requires Hq*d == H)
  *   attn_out bf16 [L, B, n, Hq, d]  (required: it is also the chained LM-head input)

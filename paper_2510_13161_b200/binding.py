@@ -25,7 +25,7 @@ EXPORTS = [
     "mirror_attn_verify", "mirror_lmhead_reduce", "mirror_accept_select", "mirror_verify_step",
     "mirror_device_status", "mirror_launch_count", "mirror_status_str", "mirror_set_stage_events",
     "mirror_lmhead_reduce_noalloc", "mirror_early_exit_tap", "mirror_overlap_mass", "mirror_kv_commit",
-    "mirror_linear_scratch_bytes", "mirror_linear", "mirror_rmsnorm", "mirror_target_scratch_bytes", "mirror_target_forward",
+    "mirror_linear_scratch_bytes", "mirror_linear", "mirror_rmsnorm", "mirror_target_scratch_bytes", "mirror_target_forward", "mirror_trie_build",
 ]
 
 
@@ -113,6 +113,20 @@ def _ptr(t: Optional[torch.Tensor], dtype=None, name: str = "tensor"):
 def _stream(stream) -> C.c_void_p:
     s = torch.cuda.current_stream() if stream is None else stream
     return C.c_void_p(s.cuda_stream)
+
+
+def mirror_trie_build(branch_tokens, root_token: int):
+    """Host helper: kappa branches of gamma tokens -> (parent list, tokens list, node_of [kappa][gamma]) of the tree
+    that shares common prefixes."""
+    lib = load_library()
+    rows = [list(map(int, r)) for r in branch_tokens]
+    kappa, gamma = len(rows), len(rows[0])
+    flat = (C.c_int32 * (kappa * gamma))(*[t for r in rows for t in r])
+    cap = 1 + kappa * gamma
+    parent, tokens, node_of = (C.c_int32 * cap)(), (C.c_int32 * cap)(), (C.c_int32 * (kappa * gamma))()
+    n = C.c_int()
+    _check(lib.mirror_trie_build(flat, kappa, gamma, int(root_token), parent, tokens, node_of, C.byref(n)), "mirror_trie_build")
+    return list(parent[:n.value]), list(tokens[:n.value]), [list(node_of[i * gamma:(i + 1) * gamma]) for i in range(kappa)]
 
 
 def mirror_lmhead_reduce_noalloc(hidden: torch.Tensor, W: torch.Tensor, temperature: float = 1.0, argmax=None,

@@ -136,6 +136,38 @@ mirror_status mirror_build_tree(const mirror_tree* tree, MirrorTreeInfo* info) {
 }
 
 // ---------------------------------------------------------------------------------------------
+// de-duplicated tree out of kappa branches (host only)
+// ---------------------------------------------------------------------------------------------
+extern "C" mirror_status mirror_trie_build(const int32_t* branch_tokens, int kappa, int gamma, int32_t root_token,
+                                           int32_t* parent, int32_t* tokens, int32_t* node_of, int* n_nodes) {
+    if (!branch_tokens || !parent || !tokens || !node_of || !n_nodes) return MIRROR_ERR_ARG;
+    if (kappa <= 0 || gamma <= 0) return MIRROR_ERR_ARG;
+    if (gamma > MIRROR_MAX_DEPTH || kappa > MIRROR_MAX_BRANCHES) return MIRROR_ERR_SHAPE;
+    int n = 1;
+    parent[0] = -1;
+    tokens[0] = root_token;
+    for (int i = 0; i < kappa; ++i) {
+        int cur = 0;                                        // walk down from the root, growing the tree where needed
+        for (int j = 0; j < gamma; ++j) {
+            const int32_t t = branch_tokens[(size_t)i * gamma + j];
+            int child = -1;
+            for (int c = cur + 1; c < n; ++c)               // children always have larger ids than their parent
+                if (parent[c] == cur && tokens[c] == t) { child = c; break; }
+            if (child < 0) {
+                if (n >= MIRROR_MAX_NODES) return MIRROR_ERR_SHAPE;
+                child = n++;
+                parent[child] = cur;
+                tokens[child] = t;
+            }
+            node_of[(size_t)i * gamma + j] = child;
+            cur = child;
+        }
+    }
+    *n_nodes = n;
+    return MIRROR_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
 // workspace
 // ---------------------------------------------------------------------------------------------
 void mirror_ws_layout(const mirror_ctx* ctx, size_t M, MirrorWsLayout* out, size_t B) {

@@ -201,3 +201,44 @@ def test_bad_arguments_are_rejected_on_the_host():
     with pytest.raises(MirrorError) as e:
         m.mirror_accept_select(m.tree(tok, 0, 2, parent=[-1, 0, 2, 1, 0]), m.accept_in(0, True, target_argmax=tok))
     assert e.value.code == 2
+
+
+def test_deduplicated_tree_commits_the_same_tokens_as_the_comb_tree():
+    """kappa branches that share prefixes: verifying the tree of distinct prefixes (mirror_trie_build) commits exactly
+    what verifying the kappa separate chains commits, with fewer rows to score."""
+    V, kappa, gamma, B = 11, 6, 5, 1
+    m = make_mirror(cfg_for(V, kappa, gamma, B))
+    rng = np.random.default_rng(5)
+    fewer = 0
+    for trial in range(20):
+        bt = rng.integers(0, 3, size=(kappa, gamma)).astype(np.int32)           # tiny alphabet: many shared prefixes
+        root = int(rng.integers(0, V))
+        parent, tokens, node_of = binding.mirror_trie_build(bt, root)
+        n_t = len(parent)
+        fewer += (1 + kappa * gamma) - n_t
+        # the target's greedy token per tree node; a row of the comb tree that repeats a prefix sees the same one
+        am_t = rng.integers(0, 3, size=(B, n_t)).astype(np.int32)
+        am_c = np.zeros((B, 1 + kappa * gamma), np.int32)
+        am_c[:, 0] = am_t[:, 0]
+        for i in range(kappa):
+            for j in range(gamma):
+                am_c[:, 1 + i * gamma + j] = am_t[:, node_of[i][j]]
+        tok_c = np.concatenate([[root], bt.reshape(-1)]).astype(np.int32)[None, :]
+        tok_t = np.asarray(tokens, np.int32)[None, :]
+        tree_c = m.tree(torch.from_numpy(tok_c).cuda(), kappa, gamma)
+        tree_t = m.tree(torch.from_numpy(tok_t).cuda(), 0, gamma, parent=parent)
+        got_c = m.mirror_accept_select(tree_c, m.accept_in(0, True, target_argmax=torch.from_numpy(am_c).cuda())).cpu()
+        got_t = m.mirror_accept_select(tree_t, m.accept_in(0, True, target_argmax=torch.from_numpy(am_t).cuda())).cpu()
+        ref_t = O.accept_greedy(tok_t, am_t, parent, gamma)
+        for f in FIELDS:
+            np.testing.assert_array_equal(got_t[f], ref_t[f], err_msg=f)
+        np.testing.assert_array_equal(got_t["n_accepted"], got_c["n_accepted"])
+        np.testing.assert_array_equal(got_t["n_emitted"], got_c["n_emitted"])
+        np.testing.assert_array_equal(got_t["emitted"], got_c["emitted"])
+        # the accepted path is the same sequence of tokens, node ids differ
+        a = int(got_t["n_accepted"][0])
+        path_t = [int(tok_t[0, v]) for v in got_t["accepted_nodes"][0][:a]]
+        path_c = [int(tok_c[0, v]) for v in got_c["accepted_nodes"][0][:a]]
+        assert path_t == path_c
+    assert fewer > 0
+    assert m.device_status() == (0, 0)

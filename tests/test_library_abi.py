@@ -39,3 +39,22 @@ def test_status_strings_and_argument_errors_without_a_gpu():
     assert lib.mirror_create(ctypes.byref(ctx), ctypes.byref(bad), 0) == 2
     bad = binding.ModelDesc(256, 4, 2, 96, 1024, 16, 0.0, 1.0)       # head_dim 96 unsupported
     assert lib.mirror_create(ctypes.byref(ctx), ctypes.byref(bad), 0) == 3
+
+
+def test_trie_build_matches_the_oracle_on_the_host():
+    """mirror_trie_build is host-only: it runs without a GPU and must agree with the oracle's definition."""
+    import numpy as np
+    from oracle import oracle as O
+    from paper_2510_13161_b200 import binding
+    rng = np.random.default_rng(1)
+    for _ in range(100):
+        kappa, gamma = int(rng.integers(1, 9)), int(rng.integers(1, 9))
+        bt = rng.integers(0, 3, size=(kappa, gamma))
+        parent, tokens, node_of = binding.mirror_trie_build(bt, 11)
+        rp, rt, rn = O.trie_build(bt, 11)
+        assert parent == rp.tolist() and tokens == rt.tolist() and node_of == rn.tolist()
+    # limits: more distinct prefixes than a tree may hold
+    import pytest
+    big = np.arange(64 * 2).reshape(64, 2)                    # 64 branches x 2 = 129 nodes with the root
+    with pytest.raises(binding.MirrorError):
+        binding.mirror_trie_build(big, 0)
