@@ -983,6 +983,24 @@ __global__ void __launch_bounds__(kMergeThreads) attn_merge_kernel(const AttnPar
     for (int i = 0; i < kPer; ++i)
 #pragma unroll
         for (int c = 0; c < 8; ++c) acc[i][c] = 0.f;
+    if (n_blocks >= 4) {
+        // many parts, at most one chunk per thread: six parts' loads in flight at a time (same order of additions)
+        if (chunk[0] < kChunks || writes_lse) {
+            const bool has = chunk[0] < kChunks;
+            const int c0 = has ? chunk[0] * 8 : 0;
+#pragma unroll 6
+            for (int k = 0; k < parts; ++k) {
+                const float* src = part_of(k);
+                const float pm = __ldcg(src + (size_t)D * kRows);
+                const float wgt = (pm == -INFINITY) ? 0.f : exp2f((pm - Mm) * p.scale_log2e);
+                Lm = fmaf(wgt, __ldcg(src + (size_t)(D + 1) * kRows), Lm);
+                if (has) {
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) acc[0][c] = fmaf(wgt, __ldcg(src + (size_t)(c0 + c) * kRows), acc[0][c]);
+                }
+            }
+        }
+    } else
 #pragma unroll 2
     for (int k = 0; k < parts; ++k) {
         const float* src = part_of(k);

@@ -84,7 +84,8 @@ __global__ void finish_qkv_kernel(const float* partial, int slices, int M, int H
 // of all its columns before adding them (in slice order).  partial == nullptr: plain RMSNorm of `residual`;
 // gamma == nullptr: no norm.
 constexpr int kNormThreads = 1024;
-constexpr int kNormCols = 16;                 // columns per thread: rows of up to 16384 elements
+constexpr int kNormMaxCols = 16;              // columns per thread: rows of up to 16384 elements
+template <int kNormCols, int kUnroll>         // kNormCols * 1024 >= H; kUnroll slices' loads in flight at a time
 __global__ void __launch_bounds__(kNormThreads)
 finish_residual_norm_kernel(const float* partial, int slices, int M, int H, const __nv_bfloat16* residual,
                             const __nv_bfloat16* gamma, float eps, __nv_bfloat16* x_out, __nv_bfloat16* normed) {
@@ -100,15 +101,20 @@ finish_residual_norm_kernel(const float* partial, int slices, int M, int H, cons
         r[c] = col < H ? __bfloat162float(residual[base + col]) : 0.f;
     }
     if (partial) {
-        for (int s = 0; s < slices; ++s) {
-            float v[kNormCols];
+        // several slices' loads in flight at a time; the additions stay in slice order
+        for (int s0 = 0; s0 < slices; s0 += kUnroll) {
+            float v[kUnroll][kNormCols];
 #pragma unroll
-            for (int c = 0; c < kNormCols; ++c) {
-                const int col = threadIdx.x + c * kNormThreads;
-                v[c] = col < H ? partial[(size_t)s * MN + base + col] : 0.f;
-            }
+            for (int k = 0; k < kUnroll; ++k)
 #pragma unroll
-            for (int c = 0; c < kNormCols; ++c) r[c] += v[c];
+                for (int c = 0; c < kNormCols; ++c) {
+                    const int col = threadIdx.x + c * kNormThreads;
+                    v[k][c] = (col < H && s0 + k < slices) ? partial[(size_t)(s0 + k) * MN + base + col] : 0.f;
+                }
+#pragma unroll
+            for (int k = 0; k < kUnroll; ++k)
+#pragma unroll
+                for (int c = 0; c < kNormCols; ++c) r[c] += v[k][c];
         }
     }
     float ss = 0.f;
@@ -161,6 +167,18 @@ finish_store_kernel(const float* partial, int slices, size_t MN, const __nv_bflo
         if (residual) r += __bfloat162float(residual[idx]);
         out[idx] = __float2bfloat16_rn(r);
     }
+}
+
+cudaError_t launch_residual_norm(cudaStream_t s, const float* partial, int slices, int M, int H, const __nv_bfloat16* residual,
+                                 const __nv_bfloat16* gamma, float eps, __nv_bfloat16* x_out, __nv_bfloat16* normed) {
+    if (H <= 4 * kNormThreads)
+        return mirror_launch_pdl(finish_residual_norm_kernel<4, 6>, dim3(M), dim3(kNormThreads), 0, s, partial, slices, M, H, residual, gamma,
+                                 eps, x_out, normed);
+    if (H <= 8 * kNormThreads)
+        return mirror_launch_pdl(finish_residual_norm_kernel<8, 4>, dim3(M), dim3(kNormThreads), 0, s, partial, slices, M, H, residual, gamma,
+                                 eps, x_out, normed);
+    return mirror_launch_pdl(finish_residual_norm_kernel<16, 2>, dim3(M), dim3(kNormThreads), 0, s, partial, slices, M, H, residual, gamma,
+                             eps, x_out, normed);
 }
 
 size_t partial_bytes_for(const mirror_ctx* ctx, int M, int N, int K) {
@@ -228,11 +246,10 @@ extern "C" mirror_status mirror_linear(mirror_ctx* ctx, const void* x, int M, co
 extern "C" mirror_status mirror_rmsnorm(mirror_ctx* ctx, const void* x, const void* gamma, int M, int H, float eps, void* out,
                                         void* stream) {
     if (!ctx || !x || !gamma || !out || M <= 0 || H <= 0) return MIRROR_ERR_ARG;
-    if (H > kNormThreads * kNormCols) return MIRROR_ERR_SHAPE;
+    if (H > kNormThreads * kNormMaxCols) return MIRROR_ERR_SHAPE;
     MIRROR_CUDA_OK(cudaSetDevice(ctx->device));
-    MIRROR_CUDA_OK(mirror_launch_pdl(finish_residual_norm_kernel, dim3(M), dim3(kNormThreads), 0,
-                                     (cudaStream_t)stream, (const float*)nullptr, 0, M, H, (const __nv_bfloat16*)x,
-                                     (const __nv_bfloat16*)gamma, eps, (__nv_bfloat16*)nullptr, (__nv_bfloat16*)out));
+    MIRROR_CUDA_OK(launch_residual_norm((cudaStream_t)stream, nullptr, 0, M, H, (const __nv_bfloat16*)x, (const __nv_bfloat16*)gamma, eps,
+                                        nullptr, (__nv_bfloat16*)out));
     ctx->launches += 1;
     MIRROR_CUDA_OK(cudaGetLastError());
     return MIRROR_OK;
@@ -254,7 +271,7 @@ extern "C" mirror_status mirror_target_forward(mirror_ctx* ctx, const mirror_tar
     if (!t->layers || !t->norm_final || t->n_layers <= 0 || t->n_layers > kv->num_layers) return MIRROR_ERR_ARG;
     const int H = ctx->desc.hidden, Hq = ctx->desc.n_q_heads, Hkv = ctx->desc.n_kv_heads, d = ctx->desc.head_dim, I = t->intermediate;
     if (I <= 0 || I % 64 != 0 || H % 64 != 0 || (Hq * d) % 64 != 0 || (d & 1)) return MIRROR_ERR_SHAPE;
-    if (H > kNormThreads * kNormCols || d / 2 > 1024) return MIRROR_ERR_SHAPE;
+    if (H > kNormThreads * kNormMaxCols || d / 2 > 1024) return MIRROR_ERR_SHAPE;
     if (!kv->k_pool || !kv->v_pool || !kv->page_table || !kv->prefix_len) return MIRROR_ERR_ARG;
     if (((uintptr_t)x & 15) || ((uintptr_t)scratch & 255)) return MIRROR_ERR_ARG;
     for (int l = 0; l < t->n_layers; ++l) {
@@ -287,9 +304,8 @@ extern "C" mirror_status mirror_target_forward(mirror_ctx* ctx, const mirror_tar
                                      (double)t->rope_theta, cs));
     ctx->launches += 1;
     // the first layer's input norm; every later one comes out of the finish kernel of the layer before
-    MIRROR_CUDA_OK(mirror_launch_pdl(finish_residual_norm_kernel, dim3(M), dim3(kNormThreads), 0, s, (const float*)nullptr, 0, M, H,
-                                     (const __nv_bfloat16*)x, (const __nv_bfloat16*)t->layers[0].norm_attn, t->rms_eps,
-                                     (__nv_bfloat16*)nullptr, h));
+    MIRROR_CUDA_OK(launch_residual_norm(s, nullptr, 0, M, H, (const __nv_bfloat16*)x, (const __nv_bfloat16*)t->layers[0].norm_attn, t->rms_eps,
+                                        nullptr, h));
     ctx->launches += 1;
 
     const int Nqkv = (Hq + 2 * Hkv) * d;
@@ -319,8 +335,7 @@ extern "C" mirror_status mirror_target_forward(mirror_ctx* ctx, const mirror_tar
         // output projection + residual + the MLP's norm
         st = mirror_linear_partial_launch(ctx, a_l, M, w.w_o, H, Hq * d, partial, sc.partial_bytes, s, &slices);
         if (st != MIRROR_OK) return st;
-        MIRROR_CUDA_OK(mirror_launch_pdl(finish_residual_norm_kernel, dim3(M), dim3(kNormThreads), 0, s, (const float*)partial, slices,
-                                         M, H, x_cur, (const __nv_bfloat16*)w.norm_mlp, t->rms_eps, xa, h));
+        MIRROR_CUDA_OK(launch_residual_norm(s, partial, slices, M, H, x_cur, (const __nv_bfloat16*)w.norm_mlp, t->rms_eps, xa, h));
         ctx->launches += 1;
         // gate / up projection + SiLU gate
         st = mirror_linear_partial_launch(ctx, h, M, w.w_gate_up, 2 * I, H, partial, sc.partial_bytes, s, &slices);
@@ -333,9 +348,8 @@ extern "C" mirror_status mirror_target_forward(mirror_ctx* ctx, const mirror_tar
         if (st != MIRROR_OK) return st;
         const void* g_next = last ? t->norm_final : t->layers[l + 1].norm_attn;
         __nv_bfloat16* x_new = last ? (__nv_bfloat16*)x_out : xb;
-        MIRROR_CUDA_OK(mirror_launch_pdl(finish_residual_norm_kernel, dim3(M), dim3(kNormThreads), 0, s, (const float*)partial, slices,
-                                         M, H, (const __nv_bfloat16*)xa, (const __nv_bfloat16*)g_next, t->rms_eps, x_new,
-                                         last ? (__nv_bfloat16*)hidden_out : h));
+        MIRROR_CUDA_OK(launch_residual_norm(s, partial, slices, M, H, xa, (const __nv_bfloat16*)g_next, t->rms_eps, x_new,
+                                            last ? (__nv_bfloat16*)hidden_out : h));
         ctx->launches += 1;
         x_cur = xb;
     }
