@@ -181,9 +181,9 @@ void mirror_ws_layout(const mirror_ctx* ctx, size_t M, MirrorWsLayout* out, size
     at += L.attn_partial_bytes;
     L.end_attn = at;
     L.lm_partial = at;
-    // one partial per CTA (weight-stream kernel) or per 128-row vocabulary tile (pair kernel), whichever is more
-    const size_t n_part = (size_t)(ctx->num_sms > mirror_lmhead_pair_partials(ctx->desc.vocab) ? ctx->num_sms
-                                                                                                : mirror_lmhead_pair_partials(ctx->desc.vocab));
+    // one partial per CTA (up to two CTAs per SM) or per 128-row vocabulary tile (several row chunks), whichever is more
+    const size_t per_cta = (size_t)2 * ctx->num_sms, per_tile = (size_t)mirror_lmhead_pair_partials(ctx->desc.vocab);
+    const size_t n_part = per_cta > per_tile ? per_cta : per_tile;
     L.lm_partial_bytes = align_up(n_part * M * 12, 256);
     at += L.lm_partial_bytes;
     L.lse = at;

@@ -43,6 +43,7 @@ struct PairParams {
     int n_chunks, chunk_rows, half_rows;
     int acc_stride, tmem_cols;
     int stages, stage_bytes;
+    int ctas_per_sm;                        // 2 when few rows leave room for two CTAs' pipelines on an SM
     int k_slices, kb_per_slice;             // split-K (plain GEMM mode only): K blocks of 64 per unit
     int n_units;
     int w_keep;                             // 1: weight tiles are re-read by other chunks, keep them in L2
@@ -381,11 +382,11 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
     }
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 lmhead_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_h, const PairParams p) {
     pair_gemm_body<true>(tm_w, tm_h, p);
 }
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 linear_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_h, const PairParams p) {
     pair_gemm_body<false>(tm_w, tm_h, p);
 }
@@ -394,6 +395,12 @@ int next_pow2(int x) {
     int p = 1;
     while (p < x) p <<= 1;
     return p;
+}
+
+int ctas_per_sm_for(int M) {
+    int c = M <= 32 ? 2 : 1;
+    if (const char* e = getenv("MIRROR_LM_CTAS_PER_SM")) { const int v = atoi(e); if (v == 1 || (v == 2 && M <= 32)) c = v; }
+    return c;
 }
 
 // shapes shared by both modes: row chunks, accumulator layout, pipeline depth
@@ -406,7 +413,10 @@ mirror_status pair_shape(int M, int V, int H, PairParams* p) {
     p->acc_stride = next_pow2(p->chunk_rows < 32 ? 32 : p->chunk_rows);
     p->tmem_cols = kAcc * p->acc_stride;
     p->stage_bytes = kATileBytes + p->half_rows * kBK * 2;
-    p->stages = (kSmemBudget - kCtrlBytes - 1024) / p->stage_bytes;
+    // Few rows (a weight stream): two CTAs per SM with five stages each keep more bytes in flight than one CTA with
+    // eight, deal the units to twice as many pairs, and let the CTAs of the next kernel move in one by one.
+    p->ctas_per_sm = ctas_per_sm_for(M);
+    p->stages = (kSmemBudget / p->ctas_per_sm - kCtrlBytes - 2048) / p->stage_bytes;
     if (p->stages > kMaxStages) p->stages = kMaxStages;
     if (const char* e = getenv("MIRROR_LM_STAGES")) { const int s = atoi(e); if (s >= 2 && s < p->stages) p->stages = s; }
     if (p->stages < 2) return MIRROR_ERR_SHAPE;
@@ -469,7 +479,7 @@ mirror_status mirror_lmhead_pair_launch(mirror_ctx* ctx, const void* hidden, int
     mirror_status st = pair_shape(M, V, H, &p);
     if (st != MIRROR_OK) return st;
     p.n_units = n_tiles * p.n_chunks;
-    int n_pairs = ctx->num_sms / 2;
+    int n_pairs = ctx->num_sms / 2 * p.ctas_per_sm;
     if (n_pairs > p.n_units) n_pairs = p.n_units;
     if (n_pairs < 1) return MIRROR_ERR_UNSUPPORTED;
     // partials: one per CTA (single row chunk: running state) or one per 128-row vocabulary tile
@@ -493,7 +503,7 @@ mirror_status mirror_lmhead_pair_launch(mirror_ctx* ctx, const void* hidden, int
 // waves of units), slices of at least 512 K elements.
 int mirror_linear_slices(const mirror_ctx* ctx, int M, int N, int K) {
     const int n_tiles = (N + kPairV - 1) / kPairV, n_chunks = (M + kMaxChunkRows - 1) / kMaxChunkRows;
-    const int n_kb = K / kBK, n_pairs = ctx->num_sms / 2 > 0 ? ctx->num_sms / 2 : 1;
+    const int n_kb = K / kBK, n_pairs = ctx->num_sms / 2 > 0 ? ctx->num_sms / 2 * ctas_per_sm_for(M) : 1;
     int best = 1;
     double best_eff = 0.0;
     for (int s = 1; s <= 16; ++s) {
@@ -520,7 +530,7 @@ mirror_status mirror_linear_partial_launch(mirror_ctx* ctx, const void* x, int M
     p.k_slices = (n_kb + p.kb_per_slice - 1) / p.kb_per_slice;
     if (partial_bytes < (size_t)p.k_slices * M * N * sizeof(float)) return MIRROR_ERR_WORKSPACE;
     p.n_units = n_tiles * p.n_chunks * p.k_slices;
-    int n_pairs = ctx->num_sms / 2;
+    int n_pairs = ctx->num_sms / 2 * p.ctas_per_sm;
     if (n_pairs > p.n_units) n_pairs = p.n_units;
     if (n_pairs < 1) return MIRROR_ERR_UNSUPPORTED;
     p.w_keep = p.n_chunks > 1;
