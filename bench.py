@@ -40,6 +40,9 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--accept-mode", default=None, choices=["greedy", "spec_sampling", "spec_tree"],
                     help="override the workload's acceptance rule")
+    ap.add_argument("--attn-per-layer", action="store_true",
+                    help="also time attention launched layer by layer (plain launches and a CUDA-graph replay); reported under "
+                         "stages.attn_per_layer_ms, outside the timed region")
     ap.add_argument("--target-layers", type=int, default=0,
                     help="also time mirror_target_forward (projections, rotary embedding, attention, MLP) over this many "
                          "decoder layers of the workload's shape with seeded random weights (0.66 GB per layer for the default "
@@ -441,7 +444,8 @@ def run_mirror(args):
 
     # ---- attention with one launch pair per layer: the order a real target enforces (layer l+1's queries depend on
     # layer l's output), as plain stream-ordered launches and replayed from a CUDA graph.  Outside the timed region.
-    stages["attn_per_layer_ms"] = attn_per_layer(m, x, tree, cfg)
+    if args.attn_per_layer:
+        stages["attn_per_layer_ms"] = attn_per_layer(m, x, tree, cfg)
     if args.target_layers > 0:
         stages["target_forward"] = target_forward_stage(m, x, tree, kv, cfg, min(args.target_layers, cfg.layers), args.intermediate,
                                                         peaks["hbm_gbs"])
