@@ -177,3 +177,22 @@ def test_root_only_tree_and_single_token_prefix():
     assert m.device_status() == (0, 0)
     close(out["q"][0], ref[0]["q"], "q0", ulps=1.5, exact_frac=0.99)
     close(out["x_out"], ref[-1]["x"], "x_out", ulps=3.0, exact_frac=0.4)
+
+
+def test_target_forward_repeated_runs_are_bitwise_equal():
+    """Split-K slices are added in slice order and the attention parts in group order: eight runs, bit for bit."""
+    case = dict(H=512, Hq=8, Hkv=2, d=128, inter=1344, L=2, B=2, lo=100, hi=900, kappa=4, gamma=4, seed=4)
+    cfg, x, layers, norm_final, emb = layer_case(**case)
+    m = make_mirror(cfg)
+    dev = lambda t: t.cuda()
+    tgt = m.target([{k: dev(v) for k, v in w.items()} for w in layers], dev(norm_final), case["inter"], 1.0e4, 1e-6)
+    kv = m.kv(dev(x.k_pool), dev(x.v_pool), dev(x.page_table), dev(x.prefix_len))
+    tree = m.tree(dev(x.tokens), cfg.kappa, cfg.gamma)
+    emb_d = dev(emb)
+    first = m.mirror_target_forward(tgt, kv, tree, emb_d)
+    first = {k: v.clone() for k, v in first.items() if not k.startswith("_")}
+    for _ in range(7):
+        out = m.mirror_target_forward(tgt, kv, tree, emb_d)
+        for k, v in first.items():
+            assert torch.equal(out[k], v), k
+    assert m.device_status() == (0, 0)

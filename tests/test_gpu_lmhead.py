@@ -122,3 +122,17 @@ def test_full_vocab_sampled_rows():
     assert err < LOGIT_TOL_TIGHT, err
     _, flips = check_reductions(res, logits)
     print("argmax flips", flips, "max logit err", err)
+
+
+@pytest.mark.parametrize("M,V,H", [(17, 20000, 512), (392, 6000, 512), (1040, 3000, 256)])
+def test_repeated_runs_are_bitwise_equal(M, V, H):
+    """Partials are merged in a fixed order whichever CTA pair ran which unit: twelve runs, bit for bit."""
+    W = rand_bf16((V, H), 0.05, 21).cuda(); hid = rand_bf16((M, H), 1.0, 22).cuda()
+    m = make_mirror(lm_cfg(V, H))
+    first = m.mirror_lmhead_reduce(hid, W, want_logits=True)
+    first = {k: v.clone() for k, v in first.items() if isinstance(v, torch.Tensor)}
+    for _ in range(11):
+        res = m.mirror_lmhead_reduce(hid, W, want_logits=True)
+        for k, v in first.items():
+            assert torch.equal(res[k], v), k
+    assert m.device_status() == (0, 0)
