@@ -403,12 +403,9 @@ def run_mirror(args):
     d2h = sum(v.numel() * v.element_size() for v in h_out.values())
 
     def e2e_step():
-        for k, v in h_in.items():
-            d_in[k].copy_(v, non_blocking=True)
-        m.mirror_verify_step(kv, tree_e, d_in["q"], d_in["k_new"], d_in["v_new"], x.hidden, x.W, acc, attn_out, out=res,
-                             stream=stream)
-        for k, v in h_out.items():
-            v.copy_(getattr(res, k), non_blocking=True)
+        # one C-ABI call with host buffers: it copies this step's inputs in on its own stream, piece by piece, runs the
+        # step and copies the decision back
+        m.mirror_verify_step_host(kv, tree_e, h_in, d_in, x.hidden, x.W, acc, attn_out, res, h_out=h_out, stream=stream)
         stream.synchronize()      # the caller needs the decision before it can build the next step
 
     for _ in range(3):

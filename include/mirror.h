@@ -329,6 +329,28 @@ mirror_status mirror_target_forward(mirror_ctx* ctx, const mirror_target* t, con
                                     const void* x, void* q_out, void* k_new_out, void* v_new_out, void* attn_out,
                                     void* x_out, void* hidden_out, void* scratch, size_t scratch_bytes, void* stream);
 
+/* mirror_verify_step for callers whose step inputs live in HOST memory (pinned for the copies to be asynchronous):
+ *   h_q bf16 [L, B, n, Hq, d], h_k_new / h_v_new bf16 [L, B, n, Hkv, d], h_tokens int32 [B, n]: HOST inputs of this step
+ *   d_q, d_k_new, d_v_new: DEVICE staging buffers of the same shapes, and tree->tokens (device, written here);
+ *                   they must not be in use by work on other streams
+ *   h_out           HOST copies of the decision (any member may be NULL); valid once `stream` has been synchronised
+ * Copies run on an internal stream (created on first use) and begin after all work already queued on `stream`.  The
+ * layers' attention problems are independent and the LM head reads only the last layer's output, so the last layer is
+ * copied and attended to first, the LM head and the acceptance follow, and the other layers arrive in three pieces
+ * while the LM head runs; each is attended to once it has landed, after the decision has been sent back.
+ * Everything else as in mirror_verify_step (attn_out holds all layers when `stream` has drained).  Does not synchronise. */
+typedef struct {
+    int32_t* n_accepted;   /* [B] */
+    int32_t* best_branch;  /* [B] */
+    int32_t* n_emitted;    /* [B] */
+    int32_t* emitted;      /* [B, gamma + 1] */
+} mirror_accept_host_out;
+mirror_status mirror_verify_step_host(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const void* h_q,
+                                      const void* h_k_new, const void* h_v_new, const int32_t* h_tokens, void* d_q,
+                                      void* d_k_new, void* d_v_new, const void* hidden, const void* W,
+                                      const mirror_accept_in* acc, const mirror_accept_out* out,
+                                      const mirror_accept_host_out* h_out, void* attn_out, void* stream);
+
 /* Optional timing hooks for mirror_verify_step: four cudaEvent_t (passed as void*) that every later
  * mirror_verify_step on this ctx records on its stream -- before attention, after attention, after the
  * LM-head GEMM kernel, after acceptance -- until cleared with NULL.  The caller owns the events. */

@@ -25,7 +25,7 @@ EXPORTS = [
     "mirror_attn_verify", "mirror_lmhead_reduce", "mirror_accept_select", "mirror_verify_step",
     "mirror_device_status", "mirror_launch_count", "mirror_status_str", "mirror_set_stage_events",
     "mirror_lmhead_reduce_noalloc", "mirror_early_exit_tap", "mirror_overlap_mass", "mirror_kv_commit",
-    "mirror_linear_scratch_bytes", "mirror_linear", "mirror_rmsnorm", "mirror_target_scratch_bytes", "mirror_target_forward", "mirror_trie_build",
+    "mirror_linear_scratch_bytes", "mirror_linear", "mirror_rmsnorm", "mirror_target_scratch_bytes", "mirror_target_forward", "mirror_trie_build", "mirror_verify_step_host",
 ]
 
 
@@ -43,6 +43,10 @@ class ModelDesc(C.Structure):
 class Tree(C.Structure):
     _fields_ = [("batch", C.c_int), ("n_nodes", C.c_int), ("kappa", C.c_int), ("gamma", C.c_int),
                 ("tokens", C.c_void_p), ("parent", C.POINTER(C.c_int32))]
+
+
+class AcceptHostOut(C.Structure):
+    _fields_ = [("n_accepted", C.c_void_p), ("best_branch", C.c_void_p), ("n_emitted", C.c_void_p), ("emitted", C.c_void_p)]
 
 
 class LayerWeights(C.Structure):
@@ -382,6 +386,27 @@ class Mirror:
         o = out.struct()
         _check(self.lib.mirror_accept_select(self._ctx, C.byref(tree), C.byref(acc), C.byref(o), _stream(stream)),
                "mirror_accept_select")
+        return out
+
+    def mirror_verify_step_host(self, kv: KV, tree: Tree, h_in: dict, d_in: dict, hidden, W, acc: AcceptIn, attn_out,
+                                out: "AcceptResult", h_out: Optional[dict] = None, stream=None) -> "AcceptResult":
+        """mirror_verify_step with this step's inputs in (pinned) host tensors h_in = {q, k_new, v_new, tokens}; d_in holds
+        the device staging tensors of the same shapes (d_in["tokens"] must be the tensor `tree` was built on); h_out:
+        optional pinned host tensors n_accepted, best_branch, n_emitted, emitted that receive the decision."""
+        def hp(t, dtype, name):
+            if t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+                raise ValueError(f"{name} must be a contiguous host tensor of {dtype}")
+            return C.c_void_p(t.data_ptr())
+        ho = AcceptHostOut(*[(C.c_void_p(h_out[f].data_ptr()) if h_out and f in h_out else None) for f, _ in AcceptHostOut._fields_])
+        self.ensure_workspace(tree, kv, {ACCEPT_GREEDY: WS_STEP_GREEDY, ACCEPT_SPEC_TREE: WS_STEP_TREE}.get(acc.mode, WS_STEP_SPEC))
+        o = out.struct()
+        _check(self.lib.mirror_verify_step_host(self._ctx, C.byref(kv), C.byref(tree), hp(h_in["q"], torch.bfloat16, "q"),
+                                                hp(h_in["k_new"], torch.bfloat16, "k_new"), hp(h_in["v_new"], torch.bfloat16, "v_new"),
+                                                hp(h_in["tokens"], torch.int32, "tokens"), _ptr(d_in["q"], torch.bfloat16, "d_q"),
+                                                _ptr(d_in["k_new"], torch.bfloat16, "d_k_new"), _ptr(d_in["v_new"], torch.bfloat16, "d_v_new"),
+                                                _ptr(hidden, torch.bfloat16, "hidden"), _ptr(W, torch.bfloat16, "W"), C.byref(acc),
+                                                C.byref(o), C.byref(ho), _ptr(attn_out, torch.bfloat16, "attn_out"), _stream(stream)),
+               "mirror_verify_step_host")
         return out
 
     def mirror_verify_step(self, kv: KV, tree: Tree, q, k_new, v_new, hidden, W, acc: AcceptIn, attn_out,

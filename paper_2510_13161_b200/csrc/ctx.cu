@@ -62,6 +62,11 @@ extern "C" mirror_status mirror_destroy(mirror_ctx* ctx) {
     if (!ctx) return MIRROR_ERR_ARG;
     cudaSetDevice(ctx->device);
     if (ctx->d_status) cudaFree(ctx->d_status);
+    if (ctx->copy_stream) {
+        cudaStreamDestroy(ctx->copy_stream);
+        for (cudaEvent_t e : ctx->copy_ev)
+            if (e) cudaEventDestroy(e);
+    }
     delete ctx;
     return MIRROR_OK;
 }

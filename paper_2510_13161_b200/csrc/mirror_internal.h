@@ -34,6 +34,8 @@ struct mirror_ctx {
     bool lm_pair_attr_set = false;
     cudaEvent_t stage_ev[4] = {nullptr, nullptr, nullptr, nullptr};
     bool stage_ev_on = false;
+    cudaStream_t copy_stream = nullptr;                     // mirror_verify_step_host: created on first use
+    cudaEvent_t copy_ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
     PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
 };
 

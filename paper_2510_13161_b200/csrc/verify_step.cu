@@ -35,10 +35,28 @@ extern "C" mirror_status mirror_attn_verify(mirror_ctx* ctx, const mirror_kv* kv
     return mirror_attn_launch(ctx, kv, tree, ti, q, k_new, v_new, out, lse_out, (float*)(ws + L.attn_partial), (cudaStream_t)stream);
 }
 
-extern "C" mirror_status mirror_verify_step(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree,
-                                            const void* q, const void* k_new, const void* v_new, const void* hidden,
-                                            const void* W, const mirror_accept_in* acc, const mirror_accept_out* out,
-                                            void* attn_out, int32_t* argmax_out, void* stream) {
+namespace {
+
+struct HostIO {                       // host-buffer variant: pinned host inputs / outputs of one step
+    const void* h_q;
+    const void* h_k_new;
+    const void* h_v_new;
+    const int32_t* h_tokens;
+    const mirror_accept_host_out* h_out;
+};
+
+constexpr int kHostChunks = 4;        // the step's layers are copied and attended to in this many pieces
+
+mirror_status ensure_copy_stream(mirror_ctx* ctx) {
+    if (ctx->copy_stream) return MIRROR_OK;
+    MIRROR_CUDA_OK(cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+    for (int i = 0; i < kHostChunks + 1; ++i) MIRROR_CUDA_OK(cudaEventCreateWithFlags(&ctx->copy_ev[i], cudaEventDisableTiming));
+    return MIRROR_OK;
+}
+
+mirror_status verify_step_impl(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const void* q, const void* k_new,
+                               const void* v_new, const void* hidden, const void* W, const mirror_accept_in* acc,
+                               const mirror_accept_out* out, void* attn_out, int32_t* argmax_out, void* stream, const HostIO* io) {
     if (!ctx || !kv || !tree || !q || !k_new || !v_new || !W || !acc || !out || !attn_out || !tree->tokens) return MIRROR_ERR_ARG;
     if (!out->n_accepted || !out->best_branch || !out->n_emitted || !out->emitted || !out->accepted_nodes ||
         !out->decide_row || !out->reuse_slot)
@@ -60,10 +78,58 @@ extern "C" mirror_status mirror_verify_step(mirror_ctx* ctx, const mirror_kv* kv
     uint8_t* ws = (uint8_t*)ctx->ws;
     cudaStream_t s = (cudaStream_t)stream;
 
-    const bool ev = ctx->stage_ev_on;
+    // (host-buffer variant) pieces of layers, copied on the second stream and attended to in that order
+    int n_pieces = 0, piece_l0[kHostChunks], piece_l1[kHostChunks];
+    const size_t q_layer = M * (size_t)ctx->desc.n_q_heads * ctx->desc.head_dim * 2;        // bytes per layer
+    const size_t kv_layer = M * (size_t)ctx->desc.n_kv_heads * ctx->desc.head_dim * 2;
+    auto attend_piece = [&](int c) -> mirror_status {
+        MIRROR_CUDA_OK(cudaStreamWaitEvent(s, ctx->copy_ev[c], 0));
+        const int l0 = piece_l0[c], l1 = piece_l1[c];
+        mirror_kv kv_c = *kv;
+        kv_c.k_pool = (const __nv_bfloat16*)kv->k_pool + (size_t)l0 * kv->layer_stride;
+        kv_c.v_pool = (const __nv_bfloat16*)kv->v_pool + (size_t)l0 * kv->layer_stride;
+        kv_c.num_layers = l1 - l0;
+        return mirror_attn_launch(ctx, &kv_c, tree, ti, (const uint8_t*)q + l0 * q_layer, (const uint8_t*)k_new + l0 * kv_layer,
+                                  (const uint8_t*)v_new + l0 * kv_layer, (uint8_t*)attn_out + l0 * q_layer, nullptr,
+                                  (float*)(ws + L.attn_partial), s);
+    };
+    const bool ev = ctx->stage_ev_on && !io;
     if (ev) MIRROR_CUDA_OK(cudaEventRecord(ctx->stage_ev[0], s));
-    st = mirror_attn_launch(ctx, kv, tree, ti, q, k_new, v_new, attn_out, nullptr, (float*)(ws + L.attn_partial), s);
-    if (st != MIRROR_OK) return st;
+    if (!io) {
+        st = mirror_attn_launch(ctx, kv, tree, ti, q, k_new, v_new, attn_out, nullptr, (float*)(ws + L.attn_partial), s);
+        if (st != MIRROR_OK) return st;
+    } else {
+        // Host inputs.  The layers' attention problems are independent of one another and the LM head reads only the
+        // last layer's output, so the last layer is copied and attended to first, the LM head and the acceptance follow
+        // at once, and the other layers are copied in pieces on a second stream while the LM head streams its weights;
+        // each piece is attended to as soon as it has landed (after the decision has gone back to the host).  The
+        // copies start only after everything already queued on `stream` (the previous step may still read the staging
+        // buffers).
+        st = ensure_copy_stream(ctx);
+        if (st != MIRROR_OK) return st;
+        cudaStream_t cs = ctx->copy_stream;
+        MIRROR_CUDA_OK(cudaEventRecord(ctx->copy_ev[kHostChunks], s));
+        MIRROR_CUDA_OK(cudaStreamWaitEvent(cs, ctx->copy_ev[kHostChunks], 0));
+        MIRROR_CUDA_OK(cudaMemcpyAsync((void*)tree->tokens, io->h_tokens, M * sizeof(int32_t), cudaMemcpyHostToDevice, cs));
+        const int Lyr = kv->num_layers;
+        n_pieces = 1 + (Lyr - 1 < kHostChunks - 1 ? Lyr - 1 : kHostChunks - 1);
+        for (int c = 0; c < n_pieces; ++c) {
+            // piece 0: the last layer; pieces 1..: the layers before it, in order
+            const int l0 = c == 0 ? Lyr - 1 : (int)((long long)(Lyr - 1) * (c - 1) / (n_pieces - 1));
+            const int l1 = c == 0 ? Lyr : (int)((long long)(Lyr - 1) * c / (n_pieces - 1));
+            piece_l0[c] = l0; piece_l1[c] = l1;
+            const size_t nl = (size_t)(l1 - l0);
+            MIRROR_CUDA_OK(cudaMemcpyAsync((uint8_t*)q + l0 * q_layer, (const uint8_t*)io->h_q + l0 * q_layer, nl * q_layer,
+                                           cudaMemcpyHostToDevice, cs));
+            MIRROR_CUDA_OK(cudaMemcpyAsync((uint8_t*)k_new + l0 * kv_layer, (const uint8_t*)io->h_k_new + l0 * kv_layer, nl * kv_layer,
+                                           cudaMemcpyHostToDevice, cs));
+            MIRROR_CUDA_OK(cudaMemcpyAsync((uint8_t*)v_new + l0 * kv_layer, (const uint8_t*)io->h_v_new + l0 * kv_layer, nl * kv_layer,
+                                           cudaMemcpyHostToDevice, cs));
+            MIRROR_CUDA_OK(cudaEventRecord(ctx->copy_ev[c], cs));
+        }
+        st = attend_piece(0);
+        if (st != MIRROR_OK) return st;
+    }
     if (ev) MIRROR_CUDA_OK(cudaEventRecord(ctx->stage_ev[1], s));
 
     // LM-head rows: the given hidden states, else the last layer's attention output ([B*n, Hq*d] == [M, H])
@@ -89,7 +155,38 @@ extern "C" mirror_status mirror_verify_step(mirror_ctx* ctx, const mirror_kv* kv
     st = mirror_accept_launch(ctx, tree, ti, &in, out, s, tree_scratch);
     if (st != MIRROR_OK) return st;
     if (ev) MIRROR_CUDA_OK(cudaEventRecord(ctx->stage_ev[3], s));
+    if (io && io->h_out) {
+        const mirror_accept_host_out* h = io->h_out;
+        const size_t B = (size_t)tree->batch;
+        if (h->n_accepted) MIRROR_CUDA_OK(cudaMemcpyAsync(h->n_accepted, out->n_accepted, B * 4, cudaMemcpyDeviceToHost, s));
+        if (h->best_branch) MIRROR_CUDA_OK(cudaMemcpyAsync(h->best_branch, out->best_branch, B * 4, cudaMemcpyDeviceToHost, s));
+        if (h->n_emitted) MIRROR_CUDA_OK(cudaMemcpyAsync(h->n_emitted, out->n_emitted, B * 4, cudaMemcpyDeviceToHost, s));
+        if (h->emitted) MIRROR_CUDA_OK(cudaMemcpyAsync(h->emitted, out->emitted, B * (size_t)(tree->gamma + 1) * 4, cudaMemcpyDeviceToHost, s));
+    }
+    for (int c = 1; c < n_pieces; ++c) {
+        st = attend_piece(c);
+        if (st != MIRROR_OK) return st;
+    }
     return MIRROR_OK;
+}
+
+}  // namespace
+
+extern "C" mirror_status mirror_verify_step(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree,
+                                            const void* q, const void* k_new, const void* v_new, const void* hidden,
+                                            const void* W, const mirror_accept_in* acc, const mirror_accept_out* out,
+                                            void* attn_out, int32_t* argmax_out, void* stream) {
+    return verify_step_impl(ctx, kv, tree, q, k_new, v_new, hidden, W, acc, out, attn_out, argmax_out, stream, nullptr);
+}
+
+extern "C" mirror_status mirror_verify_step_host(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const void* h_q,
+                                                 const void* h_k_new, const void* h_v_new, const int32_t* h_tokens, void* d_q,
+                                                 void* d_k_new, void* d_v_new, const void* hidden, const void* W,
+                                                 const mirror_accept_in* acc, const mirror_accept_out* out,
+                                                 const mirror_accept_host_out* h_out, void* attn_out, void* stream) {
+    if (!h_q || !h_k_new || !h_v_new || !h_tokens) return MIRROR_ERR_ARG;
+    HostIO io{h_q, h_k_new, h_v_new, h_tokens, h_out};
+    return verify_step_impl(ctx, kv, tree, d_q, d_k_new, d_v_new, hidden, W, acc, out, attn_out, nullptr, stream, &io);
 }
 
 extern "C" mirror_status mirror_set_stage_events(mirror_ctx* ctx, void* const* events4) {

@@ -4,8 +4,8 @@ import pytest
 import torch
 
 from oracle import oracle as O
-from paper_2510_13161_b200 import inputs as I
-from tests.helpers import make_mirror, oracle_attention
+from paper_2510_13161_b200 import binding, inputs as I
+from tests.helpers import make_mirror, oracle_attention, to_device
 
 pytestmark = pytest.mark.gpu
 FIELDS = ["n_accepted", "best_branch", "decide_row", "n_emitted", "emitted", "accepted_nodes", "reuse_slot"]
@@ -107,3 +107,37 @@ def test_full_size_14b_step_flip_count():
     ref = O.accept_greedy(tok, am.reshape(tok.shape), x.parent, cfg.gamma)
     for f in FIELDS:
         np.testing.assert_array_equal(got[f], ref[f], err_msg=f)
+
+
+@pytest.mark.parametrize("layers", [1, 2, 6])
+def test_host_buffer_step_equals_the_device_buffer_step(layers):
+    """mirror_verify_step_host (inputs in pinned host memory, copied in pieces on its own stream) decides exactly what
+    mirror_verify_step decides on the same inputs, call after call with changing inputs."""
+    cfg = I.shrink(I.CONFIGS["tiny"], layers=layers, batch=3, prefix_lo=40, prefix_hi=300, kappa=3, gamma=4, vocab=3000)
+    m = make_mirror(cfg)
+    x0 = to_device(I.gen_verify_inputs(cfg, 0, "cpu"))
+    kv = m.kv(x0.k_pool, x0.v_pool, x0.page_table, x0.prefix_len)
+    d_in = {k: torch.empty_like(getattr(x0, k)) for k in ("q", "k_new", "v_new", "tokens")}
+    tree_h = m.tree(d_in["tokens"], cfg.kappa, cfg.gamma)
+    acc = m.accept_in(binding.ACCEPT_GREEDY, True)
+    attn_h, attn_d = torch.empty_like(x0.q), torch.empty_like(x0.q)
+    res_h, res_d = binding.AcceptResult(cfg.batch, cfg.gamma, "cuda"), binding.AcceptResult(cfg.batch, cfg.gamma, "cuda")
+    h_out = {"n_accepted": torch.empty(cfg.batch, dtype=torch.int32).pin_memory(), "emitted": torch.empty((cfg.batch, cfg.gamma + 1), dtype=torch.int32).pin_memory(),
+             "n_emitted": torch.empty(cfg.batch, dtype=torch.int32).pin_memory(), "best_branch": torch.empty(cfg.batch, dtype=torch.int32).pin_memory()}
+    for seed in range(4):
+        xs = I.gen_verify_inputs(cfg, seed, "cpu")            # same cache (same config and page draw), new step inputs
+        h_in = {k: getattr(xs, k).contiguous().pin_memory() for k in ("q", "k_new", "v_new", "tokens")}
+        m.mirror_verify_step_host(kv, tree_h, h_in, d_in, x0.hidden, x0.W, acc, attn_h, res_h, h_out=h_out)
+        torch.cuda.synchronize()
+        xd = {k: v.cuda() for k, v in h_in.items()}
+        tree_d = m.tree(xd["tokens"], cfg.kappa, cfg.gamma)
+        m.mirror_verify_step(kv, tree_d, xd["q"], xd["k_new"], xd["v_new"], x0.hidden, x0.W, acc, attn_d, out=res_d)
+        torch.cuda.synchronize()
+        assert torch.equal(attn_h, attn_d)
+        for f in ("n_accepted", "best_branch", "n_emitted", "emitted", "accepted_nodes"):
+            assert torch.equal(getattr(res_h, f), getattr(res_d, f)), f
+        for f, t in h_out.items():
+            assert torch.equal(t, getattr(res_d, f).cpu()), f
+        for k in d_in:
+            assert torch.equal(d_in[k], xd[k]), k
+    assert m.device_status() == (0, 0)
