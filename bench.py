@@ -43,6 +43,9 @@ def parse_args():
     ap.add_argument("--attn-per-layer", action="store_true",
                     help="also time attention launched layer by layer (plain launches and a CUDA-graph replay); reported under "
                          "stages.attn_per_layer_ms, outside the timed region")
+    ap.add_argument("--overlap-draft", action="store_true",
+                    help="also run the verify step next to a synthetic draft on a second stream (latency law of Sec. 3.2: the "
+                         "step should cost max{target, draft}, not their sum); reported under stages.overlap_draft")
     ap.add_argument("--target-layers", type=int, default=0,
                     help="also time mirror_target_forward (projections, rotary embedding, attention, MLP) over this many "
                          "decoder layers of the workload's shape with seeded random weights (0.66 GB per layer for the default "
@@ -285,6 +288,59 @@ def attn_per_layer(m, x, tree, cfg, reps: int = 10):
     return res
 
 
+def overlap_draft_stage(step, stream, reps: int = 20):
+    """The verify step next to a synthetic draft on a second stream of the same GPU.  Two stand-ins for the draft's
+    generation phase, sized to take about as long as the verify step alone: a weight stream (a small model's
+    matrix-vector products: memory-bound like the verify step) and a chain of square tensor-core GEMMs (compute-bound).
+    For each: time alone, time of both launched together, and how much of the shorter one was hidden
+    (1 = the step costs max{target, draft}, 0 = it costs their sum)."""
+    import torch
+    s2 = torch.cuda.Stream()
+    dev = torch.cuda.current_device()
+    w_stream = torch.empty((24, 8192, 4096), dtype=torch.bfloat16, device=dev).normal_(0, 0.02)      # 1.6 GB of weights
+    v = torch.empty((4096, 8), dtype=torch.bfloat16, device=dev).normal_()
+    a = torch.empty((2048, 2048), dtype=torch.bfloat16, device=dev).normal_(0, 0.02)
+    b = torch.empty((2048, 2048), dtype=torch.bfloat16, device=dev).normal_(0, 0.02)
+
+    def draft_stream():
+        for i in range(w_stream.shape[0]):
+            torch.matmul(w_stream[i], v)
+
+    def draft_gemm():
+        x = a
+        for _ in range(24):
+            x = torch.matmul(x, b)
+
+    def timed(fn_main, fn_side):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        done = torch.cuda.Event()
+        for it in range(3 + reps):
+            if it == 3:
+                torch.cuda.synchronize()
+                e0.record(stream)
+            if fn_side is not None:
+                s2.wait_stream(stream)
+                with torch.cuda.stream(s2):
+                    fn_side()
+                    done.record(s2)
+            if fn_main is not None:
+                fn_main()
+            if fn_side is not None:
+                stream.wait_event(done)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    t_verify = timed(step, None)
+    out = {"verify_ms": t_verify}
+    for name, fn in (("weight_stream", draft_stream), ("tensor_gemms", draft_gemm)):
+        t_draft = timed(None, fn)
+        t_both = timed(step, fn)
+        out[name] = {"draft_ms": t_draft, "both_ms": t_both, "max_ms": max(t_verify, t_draft), "sum_ms": t_verify + t_draft,
+                     "hidden_frac": (t_verify + t_draft - t_both) / min(t_verify, t_draft)}
+    return out
+
+
 def target_forward_stage(m, x, tree, kv, cfg, n_layers: int, intermediate: int, hbm_gbs: float, reps: int = 5):
     """mirror_target_forward over n_layers decoder layers of the workload's shape (random weights): ms, weight bytes per
     second against the HBM peak.  The layers are weight streams at these row counts."""
@@ -443,6 +499,8 @@ def run_mirror(args):
     # layer l's output), as plain stream-ordered launches and replayed from a CUDA graph.  Outside the timed region.
     if args.attn_per_layer:
         stages["attn_per_layer_ms"] = attn_per_layer(m, x, tree, cfg)
+    if args.overlap_draft:
+        stages["overlap_draft"] = overlap_draft_stage(step, stream)
     if args.target_layers > 0:
         stages["target_forward"] = target_forward_stage(m, x, tree, kv, cfg, min(args.target_layers, cfg.layers), args.intermediate,
                                                         peaks["hbm_gbs"])
