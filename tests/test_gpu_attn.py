@@ -64,6 +64,7 @@ def test_tiny_config():
     dict(head_dim=128, n_q_heads=16, n_kv_heads=2, hidden=2048, kappa=8, gamma=8, batch=2, prefix_hi=500),   # 520 rows: five row blocks, n = 65
     dict(kappa=8, gamma=15, batch=1, prefix_hi=100),                 # n = 121 tree tokens: two tree tiles
     dict(prefix_lo=3000, prefix_hi=5000, batch=2, layers=1),         # long prefixes: units cut across many CTAs
+    dict(kappa=1, gamma=12, batch=2, prefix_hi=300),                 # one chain: the multi-stream mask of the draft side (13 streams)
 ])
 def test_shapes_and_ragged_cases(kw):
     cfg = small(**kw)

@@ -211,6 +211,18 @@ def test_single_branch_reduces_to_plain_causal_decode():
         np.testing.assert_allclose(out[0, :, h], ref, atol=1e-12)
 
 
+def test_multi_stream_attention_mask_is_the_chain_tree():
+    """The draft-side multi-stream mask (Speculative Streaming, Sec. 3.1: the main stream attends to the prefix only,
+    stream j to the prefix and the streams up to j) is the tree mask of a single chain: node 0 = main stream."""
+    n = 9
+    want = np.zeros((n, n), np.uint8)
+    for j in range(n):
+        want[j, :j + 1] = 1                      # streams <= j (itself included), written from the sentence
+    anc, depth = O.tree(I.comb_parent(1, n - 1))
+    np.testing.assert_array_equal(anc, want)
+    assert depth.tolist() == list(range(n))
+
+
 def test_kv_commit_then_root_only_attention_equals_attention_over_the_accepted_path():
     """Roll-forward pin: after committing the root and an accepted path into the paged cache, a fresh query that sees
     only the (longer) prefix must get exactly what it would get from the old prefix plus those tree tokens as visible
