@@ -43,6 +43,7 @@ struct PairParams {
     int n_chunks, chunk_rows, half_rows;
     int acc_stride, tmem_cols;
     int stages, stage_bytes;
+    int rows_cta, a_bytes;                  // vocabulary rows a CTA loads per unit (<= 128, a multiple of 8) and their bytes per stage
     int ctas_per_sm;                        // 2 when few rows leave room for two CTAs' pipelines on an SM
     int k_slices, kb_per_slice;             // split-K (plain GEMM mode only): K blocks of 64 per unit
     int n_units;
@@ -199,7 +200,7 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
             for (int u = pair; u < p.n_units && ok; u += n_pairs) {
                 int tile, slice, chunk;
                 decode(u, tile, slice, chunk);
-                const int w_row = tile * kPairV + (int)rank * kTileV;
+                const int w_row = (tile * 2 + (int)rank) * p.rows_cta;
                 const int h_row = chunk * p.chunk_rows + (int)rank * p.half_rows;
                 const int kb_end = min(n_kb, (slice + 1) * p.kb_per_slice);
                 for (int kb = slice * p.kb_per_slice; kb < kb_end; ++kb) {
@@ -208,7 +209,7 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
                     const uint32_t bar = map_to_rank(&ctrl->full[s], 0);
                     uint8_t* dst = stage_base + s * p.stage_bytes;
                     tma_load_2d_pair(dst, &tm_w, bar, kb * kBK, w_row, pol_w);
-                    tma_load_2d_pair(dst + kATileBytes, &tm_h, bar, kb * kBK, h_row, pol_h);
+                    tma_load_2d_pair(dst + p.a_bytes, &tm_h, bar, kb * kBK, h_row, pol_h);
                     if (++s == p.stages) { s = 0; ph ^= 1; }
                 }
             }
@@ -234,7 +235,7 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
                     if (ctrl->abort || !ptx::mbar_wait(&ctrl->full[s], ph)) { fail(p, ctrl, 13); ok = false; break; }
                     ptx::tc_fence_after();
                     const uint32_t sa = stage_u32 + (uint32_t)(s * p.stage_bytes);
-                    const uint32_t sb = sa + kATileBytes;
+                    const uint32_t sb = sa + (uint32_t)p.a_bytes;
 #pragma unroll
                     for (int k4 = 0; k4 < kBK / 16; ++k4)
                         umma_pair_f16(d_tmem, ptx::umma_desc_k_sw128(sa + k4 * 32), ptx::umma_desc_k_sw128(sb + k4 * 32), idesc,
@@ -295,8 +296,9 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
             if (ok && (ctrl->abort || !ptx::mbar_wait(&ctrl->acc_full[ab], aph))) { fail(p, ctrl, 16); ok = false; }
             if (ok) {
                 ptx::tc_fence_after();
-                const int vid = vt * kTileV + q * 32 + lane;
-                const bool valid = vid < p.V;
+                // (a unit of fewer than 128 rows per CTA leaves stale shared memory in the accumulator lanes beyond them)
+                const int vid = vt * p.rows_cta + q * 32 + lane;
+                const bool valid = q * 32 + lane < p.rows_cta && vid < p.V;
                 const bool any_valid = __ballot_sync(0xffffffffu, valid) != 0;          // warp-uniform
                 const int n_rows = min(p.chunk_rows, p.M - rbase);                       // hidden rows of this chunk
                 for (int cg = 0; cg < n_cg; ++cg) {
@@ -404,7 +406,7 @@ int ctas_per_sm_for(int M) {
 }
 
 // shapes shared by both modes: row chunks, accumulator layout, pipeline depth
-mirror_status pair_shape(int M, int V, int H, PairParams* p) {
+mirror_status pair_shape(int M, int V, int H, PairParams* p, int rows_cta = kTileV) {
     if (M <= 0 || V <= 0 || H <= 0 || H % kBK != 0) return MIRROR_ERR_SHAPE;
     p->M = M; p->V = V; p->H = H;
     p->n_chunks = (M + kMaxChunkRows - 1) / kMaxChunkRows;
@@ -412,7 +414,9 @@ mirror_status pair_shape(int M, int V, int H, PairParams* p) {
     p->half_rows = p->chunk_rows / 2;
     p->acc_stride = next_pow2(p->chunk_rows < 32 ? 32 : p->chunk_rows);
     p->tmem_cols = kAcc * p->acc_stride;
-    p->stage_bytes = kATileBytes + p->half_rows * kBK * 2;
+    p->rows_cta = rows_cta;
+    p->a_bytes = rows_cta * kBK * 2;
+    p->stage_bytes = p->a_bytes + p->half_rows * kBK * 2;
     // Few rows (a weight stream): two CTAs per SM with five stages each keep more bytes in flight than one CTA with
     // eight, deal the units to twice as many pairs, and let the CTAs of the next kernel move in one by one.
     p->ctas_per_sm = ctas_per_sm_for(M);
@@ -433,7 +437,7 @@ mirror_status pair_launch(mirror_ctx* ctx, bool reduce, const void* x, const voi
     {
         const uint64_t dims[2] = {(uint64_t)p.H, (uint64_t)p.V};
         const uint64_t strides[1] = {(uint64_t)p.H * 2};
-        const uint32_t box_w[2] = {kBK, kTileV};
+        const uint32_t box_w[2] = {kBK, (uint32_t)p.rows_cta};
         mirror_status st = mirror_make_tmap(ctx, &tm_w, W, 2, dims, strides, box_w);
         if (st != MIRROR_OK) return st;
         const uint64_t hdims[2] = {(uint64_t)p.H, (uint64_t)p.M};
@@ -474,9 +478,22 @@ int mirror_lmhead_pair_partials(int V) { return 2 * ((V + kPairV - 1) / kPairV);
 mirror_status mirror_lmhead_pair_launch(mirror_ctx* ctx, const void* hidden, int M, const void* W, float* logits_out,
                                         void* partial_ws, size_t partial_bytes, cudaStream_t stream, int* n_partials) {
     const int V = ctx->desc.vocab, H = ctx->desc.hidden;
-    const int n_tiles = (V + kPairV - 1) / kPairV;
+    // A weight stream (two CTAs per SM) is as long as its busiest pair: the rows a CTA takes per unit are chosen so that
+    // the units come out in whole waves over the pairs (152064 rows over 148 pairs: five units of 2 x 104 rows each
+    // instead of four or five of 2 x 128).
+    int rows_cta = kTileV;
+    if (ctas_per_sm_for(M) == 2) {
+        const int pairs = ctx->num_sms;
+        long long best = -1;
+        for (int r = kTileV; r >= 64; r -= 8) {
+            const long long units = (V + 2 * r - 1) / (2 * r), waves = (units + pairs - 1) / pairs;
+            if (best < 0 || waves * r < best) { best = waves * r; rows_cta = r; }
+        }
+        if (const char* e = getenv("MIRROR_LM_ROWS")) { const int r = atoi(e); if (r >= 8 && r <= kTileV && r % 8 == 0) rows_cta = r; }
+    }
+    const int n_tiles = (V + 2 * rows_cta - 1) / (2 * rows_cta);
     PairParams p;
-    mirror_status st = pair_shape(M, V, H, &p);
+    mirror_status st = pair_shape(M, V, H, &p, rows_cta);
     if (st != MIRROR_OK) return st;
     p.n_units = n_tiles * p.n_chunks;
     int n_pairs = ctx->num_sms / 2 * p.ctas_per_sm;
