@@ -40,6 +40,9 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--accept-mode", default=None, choices=["greedy", "spec_sampling", "spec_tree"],
                     help="override the workload's acceptance rule")
+    ap.add_argument("--skip-e2e", action="store_true",
+                    help="profiling aid: leave the end-to-end loop out (e2e.value is null), so that a launch list holds the "
+                         "device-resident steps only")
     ap.add_argument("--attn-per-layer", action="store_true",
                     help="also time attention launched layer by layer (plain launches and a CUDA-graph replay); reported under "
                          "stages.attn_per_layer_ms, outside the timed region")
@@ -464,17 +467,19 @@ def run_mirror(args):
         m.mirror_verify_step_host(kv, tree_e, h_in, d_in, x.hidden, x.W, acc, attn_out, res, h_out=h_out, stream=stream)
         stream.synchronize()      # the caller needs the decision before it can build the next step
 
-    for _ in range(3):
-        e2e_step()
-    Ke = max(10, min(K, 200))
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(Ke):
-        e2e_step()
-    e1.record(stream)
-    barrier()
-    e2e_value = job_throughput(Ke, world, max_over_ranks(e0.elapsed_time(e1), dev))
+    e2e_value = None
+    if not args.skip_e2e:
+        for _ in range(3):
+            e2e_step()
+        Ke = max(10, min(K, 200))
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(Ke):
+            e2e_step()
+        e1.record(stream)
+        barrier()
+        e2e_value = job_throughput(Ke, world, max_over_ranks(e0.elapsed_time(e1), dev))
 
     if rank != 0:
         if world > 1:
