@@ -297,16 +297,9 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     if (p.timing_exit == 1) return;
 #endif
 
-    // (programmatic dependent launch: nothing of global memory is touched before the kernel ahead in the stream has
-    // completed; the merge kernel behind may be scheduled as soon as SMs free up)
-    ptx::grid_dep_wait();
-    ptx::grid_dep_launch();
     // ---- prologue ---------------------------------------------------------------------------------
-    for (int b = tid; b < p.B; b += kThreads) {
-        int len = p.prefix_len[b];
-        if (len < 0 || len > p.max_pages * kSlotTok) { dev_check(p, 300 + b); len = len < 0 ? 0 : p.max_pages * kSlotTok; }
-        s_len[b] = len;
-    }
+    // (programmatic dependent launch: barriers and tensor memory are set up while the kernel ahead in the stream is
+    // still running; nothing of global memory is touched before it has completed)
     if (tid == 0) {
         for (int s = 0; s < kMaxStages; ++s) {
             ptx::mbar_init(&ctrl->k_full[s], 1); ptx::mbar_init(&ctrl->k_empty[s], 1);
@@ -331,6 +324,14 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     ptx::tc_fence_before();
     __syncthreads();
     ptx::tc_fence_after();
+    ptx::grid_dep_wait();
+    ptx::grid_dep_launch();                 // the merge kernel behind may be scheduled as soon as SMs free up
+    for (int b = tid; b < p.B; b += kThreads) {
+        int len = p.prefix_len[b];
+        if (len < 0 || len > p.max_pages * kSlotTok) { dev_check(p, 300 + b); len = len < 0 ? 0 : p.max_pages * kSlotTok; }
+        s_len[b] = len;
+    }
+    __syncthreads();
     if (tid == 0) {
         int acc = 0;
         cumT[0] = 0;
