@@ -54,6 +54,7 @@ struct PairParams {
     int* part_idx;
     float* part_sum;
     int* status;
+    long long* timing;                      // developer aid (timing builds): per-CTA start / end stamps
 };
 
 struct Ctrl {
@@ -158,6 +159,9 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
     const uint32_t rank = cluster_rank();
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     const int n_kb = p.H / kBK;
+#ifdef MIRROR_ATTN_TIMING
+    if (p.timing && tid == 0) { unsigned long long g__; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g__) :: "memory"); p.timing[blockIdx.x * 2] = (long long)g__; }
+#endif
     // unit -> (vocabulary tile, K slice, row chunk); chunk fastest, so the chunks of a tile run side by side
     auto decode = [&](int u, int& tile, int& slice, int& chunk) {
         chunk = u % p.n_chunks;
@@ -375,6 +379,9 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
         }
     }
 
+#ifdef MIRROR_ATTN_TIMING
+    if (p.timing && tid == 64) { unsigned long long g__; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g__) :: "memory"); p.timing[blockIdx.x * 2 + 1] = (long long)g__; }
+#endif
     ptx::tc_fence_before();
     __syncthreads();
     cluster_sync_all();                 // no remote arrive or multicast commit is in flight towards a CTA that has left
@@ -429,6 +436,10 @@ mirror_status pair_shape(int M, int V, int H, PairParams* p, int rows_cta = kTil
     p->inv_T = p->inv_T_log2e = 1.f;
     p->logits_out = nullptr;
     p->part_max = nullptr; p->part_idx = nullptr; p->part_sum = nullptr;
+    p->timing = nullptr;
+#ifdef MIRROR_ATTN_TIMING
+    if (const char* e = getenv("MIRROR_LM_TIMING_PTR")) p->timing = (long long*)strtoull(e, nullptr, 0);
+#endif
     return MIRROR_OK;
 }
 
