@@ -306,6 +306,11 @@ mirror_status mirror_linear_scratch_bytes(const mirror_ctx* ctx, int M, int N, i
 mirror_status mirror_linear(mirror_ctx* ctx, const void* x, int M, const void* W, int N, int K, const void* residual,
                             void* out, void* scratch, size_t scratch_bytes, void* stream);
 
+/* out[r, :] = table[tokens[r], :] for the M rows of a step: the residual rows that enter layer 0.
+ *   table bf16 [V, H] (V, H of the ctx; H a multiple of 8), tokens int32 [M] (device), out bf16 [M, H]
+ * A token outside [0, V) zeroes its row and is reported through mirror_device_status. */
+mirror_status mirror_embed_rows(mirror_ctx* ctx, const void* table, const int32_t* tokens, int M, void* out, void* stream);
+
 /* out[M, H] (bf16) = x / sqrt(mean(x^2) + eps) * gamma, row by row (x bf16 [M, H], gamma bf16 [H]; H even). */
 mirror_status mirror_rmsnorm(mirror_ctx* ctx, const void* x, const void* gamma, int M, int H, float eps, void* out,
                              void* stream);

@@ -25,7 +25,7 @@ EXPORTS = [
     "mirror_attn_verify", "mirror_lmhead_reduce", "mirror_accept_select", "mirror_verify_step",
     "mirror_device_status", "mirror_launch_count", "mirror_status_str", "mirror_set_stage_events",
     "mirror_lmhead_reduce_noalloc", "mirror_early_exit_tap", "mirror_overlap_mass", "mirror_kv_commit",
-    "mirror_linear_scratch_bytes", "mirror_linear", "mirror_rmsnorm", "mirror_target_scratch_bytes", "mirror_target_forward", "mirror_trie_build", "mirror_verify_step_host",
+    "mirror_linear_scratch_bytes", "mirror_linear", "mirror_rmsnorm", "mirror_target_scratch_bytes", "mirror_target_forward", "mirror_trie_build", "mirror_verify_step_host", "mirror_embed_rows",
 ]
 
 
@@ -341,6 +341,15 @@ class Mirror:
         _check(self.lib.mirror_linear(self._ctx, _ptr(x, torch.bfloat16, "x"), M, _ptr(W, torch.bfloat16, "W"), N, K,
                                       _ptr(residual, torch.bfloat16, "residual"), _ptr(out), _ptr(scratch),
                                       C.c_size_t(scratch.numel()), _stream(stream)), "mirror_linear")
+        return out
+
+    def mirror_embed_rows(self, table: torch.Tensor, tokens: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        """out[r] = table[tokens[r]]: table bf16 [V, H], tokens int32 (any shape, M entries) -> bf16 [M, H]."""
+        M = tokens.numel()
+        if out is None:
+            out = torch.empty((M, table.shape[1]), dtype=torch.bfloat16, device=self.device)
+        _check(self.lib.mirror_embed_rows(self._ctx, _ptr(table, torch.bfloat16, "table"), _ptr(tokens, torch.int32, "tokens"), M,
+                                          _ptr(out, torch.bfloat16, "out"), _stream(stream)), "mirror_embed_rows")
         return out
 
     def mirror_rmsnorm(self, x: torch.Tensor, gamma: torch.Tensor, eps: float = 1e-6, stream=None) -> torch.Tensor:

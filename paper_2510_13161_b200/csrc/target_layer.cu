@@ -181,6 +181,19 @@ cudaError_t launch_residual_norm(cudaStream_t s, const float* partial, int slice
                              eps, x_out, normed);
 }
 
+// Rows of the embedding table for the step's tokens: out[r] = table[tokens[r]] (16-byte copies; a token outside the
+// vocabulary is reported and its row zeroed).
+__global__ void embed_rows_kernel(const uint4* table, const int32_t* tokens, int M, int V, int row_vec, uint4* out, int* status) {
+    ptx::grid_dep_wait();
+    ptx::grid_dep_launch();
+    const int r = blockIdx.x;
+    const int t = tokens[r];
+    const bool ok = t >= 0 && t < V;
+    if (!ok && threadIdx.x == 0 && atomicCAS(status, 0, MIRROR_DEV_CHECK) == 0) atomicExch(status + 1, 900);
+    for (int i = threadIdx.x; i < row_vec; i += blockDim.x)
+        out[(size_t)r * row_vec + i] = ok ? table[(size_t)t * row_vec + i] : make_uint4(0, 0, 0, 0);
+}
+
 size_t partial_bytes_for(const mirror_ctx* ctx, int M, int N, int K) {
     return (size_t)mirror_linear_slices(ctx, M, N, K) * M * N * sizeof(float);
 }
@@ -238,6 +251,19 @@ extern "C" mirror_status mirror_linear(mirror_ctx* ctx, const void* x, int M, co
     const size_t MN = (size_t)M * N;
     MIRROR_CUDA_OK(mirror_launch_pdl(finish_store_kernel, dim3(grid_for(MN, ctx->num_sms)), dim3(kFinThreads), 0, s,
                                      (const float*)scratch, slices, MN, (const __nv_bfloat16*)residual, (__nv_bfloat16*)out));
+    ctx->launches += 1;
+    MIRROR_CUDA_OK(cudaGetLastError());
+    return MIRROR_OK;
+}
+
+extern "C" mirror_status mirror_embed_rows(mirror_ctx* ctx, const void* table, const int32_t* tokens, int M, void* out, void* stream) {
+    if (!ctx || !table || !tokens || !out || M <= 0) return MIRROR_ERR_ARG;
+    const int H = ctx->desc.hidden, V = ctx->desc.vocab;
+    if (H % 8 != 0) return MIRROR_ERR_SHAPE;
+    if (((uintptr_t)table & 15) || ((uintptr_t)out & 15)) return MIRROR_ERR_ARG;
+    MIRROR_CUDA_OK(cudaSetDevice(ctx->device));
+    MIRROR_CUDA_OK(mirror_launch_pdl(embed_rows_kernel, dim3(M), dim3(128), 0, (cudaStream_t)stream, (const uint4*)table, tokens, M, V, H / 8,
+                                     (uint4*)out, ctx->d_status));
     ctx->launches += 1;
     MIRROR_CUDA_OK(cudaGetLastError());
     return MIRROR_OK;
