@@ -90,6 +90,7 @@ def close(got_t, ref_bits, what, ulps=4.0, exact_frac=0.9):
     dict(H=512, Hq=8, Hkv=2, d=128, inter=1344, L=3, B=1, lo=300, hi=300, kappa=4, gamma=4, seed=1),
     dict(H=256, Hq=4, Hkv=4, d=64, inter=256, L=1, B=3, lo=1, hi=40, kappa=1, gamma=5, seed=2, parent=[-1, 0, 1, 1, 0, 4, 5, 2]),
     dict(H=1024, Hq=8, Hkv=2, d=128, inter=2048, L=1, B=2, lo=500, hi=3000, kappa=4, gamma=4, seed=3),
+    dict(H=256, Hq=4, Hkv=2, d=64, inter=512, L=1, B=6, lo=30, hi=200, kappa=8, gamma=6, seed=6),      # 294 rows: two row chunks in every GEMM
 ])
 def test_target_forward_matches_layer_oracle(case):
     theta, eps = 1.0e4, 1e-6
