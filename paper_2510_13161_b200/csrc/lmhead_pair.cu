@@ -407,8 +407,10 @@ int next_pow2(int x) {
 }
 
 int ctas_per_sm_for(int M) {
-    int c = M <= 32 ? 2 : 1;
-    if (const char* e = getenv("MIRROR_LM_CTAS_PER_SM")) { const int v = atoi(e); if (v == 1 || (v == 2 && M <= 32)) c = v; }
+    int max_rows = 128;                     // up to this many rows two CTAs share an SM (<= 256 TMEM columns and >= 4 stages each)
+    if (const char* e = getenv("MIRROR_LM_PAIR2_MAX_ROWS")) { const int v = atoi(e); if (v >= 0 && v <= 128) max_rows = v; }
+    int c = M <= max_rows ? 2 : 1;
+    if (const char* e = getenv("MIRROR_LM_CTAS_PER_SM")) { const int v = atoi(e); if (v == 1 || (v == 2 && M <= max_rows)) c = v; }
     return c;
 }
 
@@ -424,7 +426,7 @@ mirror_status pair_shape(int M, int V, int H, PairParams* p, int rows_cta = kTil
     p->rows_cta = rows_cta;
     p->a_bytes = rows_cta * kBK * 2;
     p->stage_bytes = p->a_bytes + p->half_rows * kBK * 2;
-    // Few rows (a weight stream): two CTAs per SM with five stages each keep more bytes in flight than one CTA with
+    // Few rows (a weight stream): two CTAs per SM with five or six stages each keep more bytes in flight than one CTA with
     // eight, deal the units to twice as many pairs, and let the CTAs of the next kernel move in one by one.
     p->ctas_per_sm = ctas_per_sm_for(M);
     p->stages = (kSmemBudget / p->ctas_per_sm - kCtrlBytes - 2048) / p->stage_bytes;
