@@ -63,7 +63,8 @@ struct AttnParams {
     int L, B, n, Hq, Hkv, G;
     int rows, n_rb, rows_per_rb;          // rows per unit, row blocks, rows per block
     int n_groups;                         // CTA groups (grid = n_groups * n_rb)
-    int snap_cap;                         // boundaries move to a unit boundary that is at most this many tiles away
+    int snap_cap;
+    int whole_units;               // 1: prefer a group count that divides equal-length units (no cuts)                         // boundaries move to a unit boundary that is at most this many tiles away
     int max_pages, num_pages, layer_pages;
     int q_half_bytes;                     // one 64-column half of a Q buffer: rows rounded up to 8, 128 B each
     int tree_slots;
@@ -256,7 +257,7 @@ __device__ __forceinline__ Partition make_partition(const AttnParams& p, const i
     // (384 units on 148 SMs: 128 groups of 3 units, attention 111 -> 105 us).
     bool equal_units = true;
     for (int b = 1; b < p.B; ++b) equal_units &= (cumT[b + 1] - cumT[b]) == cumT[1];
-    if (equal_units && q.n_groups == p.n_groups) {
+    if (p.whole_units && equal_units && q.n_groups == p.n_groups) {
         const long long units = (long long)p.L * p.B * p.Hkv;
         for (int g = p.n_groups; g * 100 >= p.n_groups * 85; --g)
             if (units % g == 0) { q.n_groups = g; break; }
@@ -1057,6 +1058,8 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
     if (const char* e = getenv("MIRROR_ATTN_GROUPS")) { const int g = atoi(e); if (g >= 1 && g <= p.n_groups) p.n_groups = g; }
     if (p.n_groups < 1) return MIRROR_ERR_SHAPE;
     p.snap_cap = 4;
+    p.whole_units = 1;
+    if (const char* e = getenv("MIRROR_ATTN_WHOLE_UNITS")) p.whole_units = atoi(e) != 0;
     if (const char* e = getenv("MIRROR_ATTN_SNAP")) { p.snap_cap = atoi(e); if (p.snap_cap < 0) p.snap_cap = 0; }
     p.max_pages = kv->max_pages_per_req; p.num_pages = kv->num_pages;
     const int64_t page_elems = (int64_t)Hkv * kSlotTok * D;

@@ -125,6 +125,7 @@ def test_bench_size_repeated_runs_are_bitwise_equal_when_every_cta_range_cuts_a_
     unit that is cut must match the oracle.  (A softmax warp that falls two completions behind a barrier it waits
     on by parity reads its accumulator too early; that shows up here as run-to-run differences.)"""
     monkeypatch.setenv("MIRROR_ATTN_SNAP", "0")
+    monkeypatch.setenv("MIRROR_ATTN_WHOLE_UNITS", "0")      # one range per CTA group of every SM, not whole units per group
     cfg = I.CONFIGS["qwen14b"]
     x = I.gen_verify_inputs(cfg, 0, "cuda", with_lm_head=False)
     m = make_mirror(cfg)
