@@ -940,6 +940,9 @@ __global__ void __launch_bounds__(kMergeThreads) attn_merge_kernel(const AttnPar
     const Partition part = make_partition(p, cumT);
     const int g = blockIdx.x + 1, rb = blockIdx.y;
     if (g >= part.n_groups || part.total_tiles >= (1ll << 31)) return;
+    const long long x = group_begin(part, g, p, cumT);
+    const UnitPos u = locate(x, p, cumT, part.tiles_per_layer);
+    if (u.tile_in_unit == 0) return;                                            // the boundary is a unit boundary (block-uniform)
     // every group's first tile, computed side by side (a unit shared by many groups is looked up from here instead of
     // by a chain of dependent calls)
     __shared__ long long s_begin[kMergeMaxGroups];
@@ -949,9 +952,6 @@ __global__ void __launch_bounds__(kMergeThreads) attn_merge_kernel(const AttnPar
         __syncthreads();
     }
     auto begin_of = [&](int t) -> long long { return tabled ? s_begin[t] : group_begin(part, t, p, cumT); };
-    const long long x = begin_of(g);
-    const UnitPos u = locate(x, p, cumT, part.tiles_per_layer);
-    if (u.tile_in_unit == 0) return;                                            // the boundary is a unit boundary
     // the groups ga..gb hold this unit's parts; the blocks of the boundaries ga+1..gb share the merge by columns
     int ga = g - 1;
     while (ga > 0 && begin_of(ga) > u.unit_first_tile) --ga;
