@@ -240,6 +240,14 @@ __device__ __noinline__ Segment make_segment(long long x, long long x_end, const
 }
 
 // How the tile sequence is cut into one range per CTA group.
+// Group count that gives every group the same number of whole units, if one exists within 15% of n_groups; else 0.
+// (Host and device: the host uses it to tell whether a launch can cut a unit at all.)
+__host__ __device__ inline int whole_unit_groups(int n_groups, long long units) {
+    for (int g = n_groups; g >= 1 && g * 100 >= n_groups * 85; --g)
+        if (units % g == 0) return g;
+    return 0;
+}
+
 struct Partition {
     long long tiles_per_layer, total_tiles, total_pairs, snap_tol;
     int n_groups;
@@ -258,9 +266,8 @@ __device__ __forceinline__ Partition make_partition(const AttnParams& p, const i
     bool equal_units = true;
     for (int b = 1; b < p.B; ++b) equal_units &= (cumT[b + 1] - cumT[b]) == cumT[1];
     if (p.whole_units && equal_units && q.n_groups == p.n_groups) {
-        const long long units = (long long)p.L * p.B * p.Hkv;
-        for (int g = p.n_groups; g * 100 >= p.n_groups * 85; --g)
-            if (units % g == 0) { q.n_groups = g; break; }
+        const int g = whole_unit_groups(p.n_groups, (long long)p.L * p.B * p.Hkv);
+        if (g > 0) q.n_groups = g;
     }
     // A boundary that falls within snap_tol tiles (a cut costs about as much as a few tiles) of a unit boundary
     // moves there: both neighbours then hold whole units and no partial has to be left and merged.  snap_tol is
@@ -1126,7 +1133,12 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
     if (lst != MIRROR_OK) return lst;
     ctx->launches += 1;
     MIRROR_CUDA_OK(cudaGetLastError());
-    if (p.n_groups > 1) {
+    // One request: all units have the same length whatever it is, so the host can tell when the partition gives every
+    // group whole units (each unit holds at least one pair of tiles, so there are at least L * Hkv pairs): nothing is cut
+    // and the merge kernel has nothing to do.
+    const bool no_cuts = p.whole_units && p.B == 1 && (long long)p.L * p.Hkv >= p.n_groups &&
+                         whole_unit_groups(p.n_groups, (long long)p.L * p.B * p.Hkv) > 0;
+    if (p.n_groups > 1 && !no_cuts) {
         // which units the partition cut is only known on the device (it depends on the prefix lengths)
         const dim3 mgrid((unsigned)(p.n_groups - 1), (unsigned)p.n_rb);
         if (D == 128) MIRROR_CUDA_OK(mirror_launch_pdl(attn_merge_kernel<128>, mgrid, dim3(kMergeThreads), 0, stream, p));
