@@ -141,3 +141,36 @@ def test_host_buffer_step_equals_the_device_buffer_step(layers):
         for k in d_in:
             assert torch.equal(d_in[k], xd[k]), k
     assert m.device_status() == (0, 0)
+
+
+def test_verify_step_replays_from_a_cuda_graph():
+    """The step only enqueues kernels (no allocation, no synchronisation once the workspace is attached), so it can be
+    captured in a CUDA graph; replays with new inputs in the same buffers decide like direct calls."""
+    cfg = I.shrink(I.CONFIGS["tiny"], layers=3, batch=2, prefix_lo=40, prefix_hi=200, kappa=3, gamma=4, vocab=3000)
+    m = make_mirror(cfg)
+    x = to_device(I.gen_verify_inputs(cfg, 0, "cpu"))
+    kv = m.kv(x.k_pool, x.v_pool, x.page_table, x.prefix_len)
+    tree = m.tree(x.tokens, cfg.kappa, cfg.gamma)
+    acc = m.accept_in(binding.ACCEPT_GREEDY, True)
+    attn_g, attn_d = torch.empty_like(x.q), torch.empty_like(x.q)
+    res_g, res_d = binding.AcceptResult(cfg.batch, cfg.gamma, "cuda"), binding.AcceptResult(cfg.batch, cfg.gamma, "cuda")
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        m.mirror_verify_step(kv, tree, x.q, x.k_new, x.v_new, x.hidden, x.W, acc, attn_g, out=res_g, stream=s)    # attaches the workspace
+        s.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            m.mirror_verify_step(kv, tree, x.q, x.k_new, x.v_new, x.hidden, x.W, acc, attn_g, out=res_g, stream=s)
+    for seed in (1, 2, 3):
+        xs = I.gen_verify_inputs(cfg, seed, "cpu")
+        for k in ("q", "k_new", "v_new", "tokens"):
+            getattr(x, k).copy_(getattr(xs, k))                 # new step inputs in the captured buffers
+        torch.cuda.synchronize()
+        g.replay()
+        torch.cuda.synchronize()
+        m.mirror_verify_step(kv, tree, x.q, x.k_new, x.v_new, x.hidden, x.W, acc, attn_d, out=res_d)
+        torch.cuda.synchronize()
+        assert torch.equal(attn_g, attn_d)
+        for f in FIELDS:
+            assert torch.equal(getattr(res_g, f), getattr(res_d, f)), f
+    assert m.device_status() == (0, 0)
