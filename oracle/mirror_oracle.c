@@ -21,7 +21,10 @@
  * the worked example of Fig. 1, and the reuse probability of Proposition 1.
  * The independent per-branch speculative-sampling rule over kappa > 1 branches
  * (oracle_accept_spec) is this build's own reading (the paper verifies one path
- * per step): parity unpinned for kappa > 1.  The lossless rule over sibling sets
+ * per step); for kappa > 1 it is pinned against that reading by hand-worked cases
+ * with deterministic uniforms (ties and A = 0 go to the lowest branch, the longer
+ * branch wins at any index, the residual and its uniform belong to the chosen
+ * branch's deciding row and first rejected node).  The lossless rule over sibling sets
  * (oracle_accept_tree) is pinned by exact integration for two and three independent
  * siblings (the emitted token follows the target distribution), by its chain special
  * case (equal to the single-branch rule) and by fixed walk-order cases.

@@ -13,7 +13,11 @@ tensor is stored and computes in fp64 in between.
 Pins (tests/test_oracle_layer.py): rmsnorm of a constant row and its scale invariance; rotary embedding keeps pair
 norms, is the identity at position 0, turns (1, 0) into (0, 1) at angle pi/2, and makes q.k depend on the position
 difference only; silu(x) - silu(-x) = x; the linear map against a brute-force triple loop and the identity weight; a
-layer whose output and down projections are zero returns its input.
+layer whose output and down projections are zero returns its input; the wiring of target_layer() itself by sparse
+weights with closed-form effects: one gate row, one up row and one down column (gate before up, MLP input =
+RMSNorm of the post-attention stream with the MLP's own norm weight, second residual onto that stream), a layer
+without MLP (x + W_o attention), and w_qkv with only its query or only its key block (block boundaries, both rotated,
+values not).
 """
 from __future__ import annotations
 

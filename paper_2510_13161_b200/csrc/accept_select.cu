@@ -72,8 +72,7 @@ accept_select_kernel(const __grid_constant__ AcceptTreeParams tp, const AcceptAr
                 pass = (x == a.target_argmax[(size_t)b * n + r]);
             } else if (x < 0 || x >= V) {
                 pass = false;
-                atomicExch(a.status, MIRROR_DEV_CHECK);
-                atomicExch(a.status + 1, 100 + c);
+                if (atomicCAS(a.status, 0, MIRROR_DEV_CHECK) == 0) atomicExch(a.status + 1, 100 + c);   // first error wins
             } else {
                 const size_t row = (size_t)b * n + r;
                 const double p = exp((double)a.logits[row * V + x] * a.inv_T - (double)a.lse[row]);
@@ -316,8 +315,7 @@ accept_tree_kernel(const __grid_constant__ AcceptTreeParams tp, const AcceptArgs
                 const int x = tok[c];
                 int pass = 0;
                 if (x < 0 || x >= V) {
-                    atomicExch(a.status, MIRROR_DEV_CHECK);
-                    atomicExch(a.status + 1, 100 + c);
+                    if (atomicCAS(a.status, 0, MIRROR_DEV_CHECK) == 0) atomicExch(a.status + 1, 100 + c);   // first error wins
                 } else {
                     const double lhs = (double)a.u_accept[(size_t)b * n + c] * (double)qc[x];
                     pass = (lhs <= mass(lr, lse_r, x)) ? 1 : 0;

@@ -946,10 +946,13 @@ __global__ void __launch_bounds__(kMergeThreads) attn_merge_kernel(const AttnPar
     __syncthreads();
     const Partition part = make_partition(p, cumT);
     const int g = blockIdx.x + 1, rb = blockIdx.y;
-    if (g >= part.n_groups || part.total_tiles >= (1ll << 31)) return;
+    // A block with nothing to merge must still wait for the attention kernel: the kernel behind this one in the stream
+    // only waits for THIS grid to complete, so a grid whose blocks all left early would let it read attention outputs
+    // that are still being written.
+    if (g >= part.n_groups || part.total_tiles >= (1ll << 31)) { ptx::grid_dep_wait(); return; }
     const long long x = group_begin(part, g, p, cumT);
     const UnitPos u = locate(x, p, cumT, part.tiles_per_layer);
-    if (u.tile_in_unit == 0) return;                                            // the boundary is a unit boundary (block-uniform)
+    if (u.tile_in_unit == 0) { ptx::grid_dep_wait(); return; }                  // the boundary is a unit boundary (block-uniform)
     // every group's first tile, computed side by side (a unit shared by many groups is looked up from here instead of
     // by a chain of dependent calls)
     __shared__ long long s_begin[kMergeMaxGroups];

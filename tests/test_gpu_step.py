@@ -174,3 +174,23 @@ def test_verify_step_replays_from_a_cuda_graph():
         for f in FIELDS:
             assert torch.equal(getattr(res_g, f), getattr(res_d, f)), f
     assert m.device_status() == (0, 0)
+
+
+def test_step_when_no_unit_is_cut_by_the_partition():
+    """Equal prefixes in a batch whose unit count the CTA groups divide: every group holds whole units, the merge kernel has
+    nothing to merge, and the LM head behind it must still see the finished attention rows (the merge kernel's blocks wait
+    for the attention kernel before they leave).  Many repetitions: a missing wait shows up now and then only."""
+    cfg = I.VerifyConfig("nocut", 1024, 8, 8, 128, 16, 2, 600, 600, 2, 3, 4096, "greedy")     # 16 x 2 x 8 = 256 units
+    x = I.gen_verify_inputs(cfg, 5, "cuda")
+    m = make_mirror(cfg)
+    logits, red = oracle_step_greedy(x)
+    ref_attn = oracle_attention(x, [cfg.layers - 1])[cfg.layers - 1][0]
+    tok = x.tokens.cpu().numpy()
+    for rep in range(20):
+        got, am, attn_out = gpu_step(m, x)
+        err = np.abs(attn_out[-1].float().cpu().numpy() - ref_attn).max()
+        assert err <= 1e-2 * np.abs(ref_attn).max() + 1e-5, (rep, err)
+        count_flips(am, logits)
+        ref = O.accept_greedy(tok, am.reshape(tok.shape), x.parent, cfg.gamma)
+        for f in FIELDS:
+            np.testing.assert_array_equal(got[f], ref[f], err_msg=f)

@@ -217,6 +217,89 @@ def test_spec_rule_special_cases():
     assert o["n_accepted"][0] == 1
 
 
+def spec_inputs_tree(p_rows, q_rows, xs, u_acc, u_res):
+    """One request over an arbitrary tree: p_rows[r] is the target distribution of node r's row, q_rows[c] node c's
+    draft distribution (c >= 1), xs[c] its token, u_acc[c] the uniform of its accept test, u_res[r] the uniform of an
+    extra token drawn at row r."""
+    n = len(xs)
+    logits = np.log(np.maximum(np.array(p_rows, np.float64), 1e-300)).astype(np.float32)
+    return (np.array(xs, np.int32), logits, np.zeros(n, np.float32), np.array(q_rows[1:], np.float32),
+            np.array(u_acc, np.float32), np.array(u_res, np.float32))
+
+
+def test_spec_rule_over_several_branches_hand_worked_cases():
+    """The independent per-branch rule for kappa > 1 (each branch tested as a chain with its own uniforms, the longest
+    wins, ties and A = 0 go to the lowest branch, the extra token is drawn at the chosen branch's deciding row from the
+    residual against the draft distribution of THAT branch's first rejected node).  Expected values are worked by hand
+    with deterministic devices: u_accept = 0 always passes; a token the target gives no mass always fails.
+    Tree: kappa = 3, gamma = 2; nodes 0 | 1,2 | 3,4 | 5,6."""
+    parent = comb_parent(3, 2)
+    V = 4
+    P0 = [0.0, 0.5, 0.25, 0.25]            # a row that gives token 0 no mass
+    PA = [0.1, 0.2, 0.3, 0.4]
+    QA = [0.5, 0.5, 0.0, 0.0]              # residual of P0 against QA: [0, 0, .25, .25]
+    QB = [0.5, 0.0, 0.5, 0.0]              # residual of P0 against QB: [0, .5, 0, .25]
+    flat = [0.25] * 4
+
+    def run(p_rows, q_rows, xs, u_acc, u_res, **kw):
+        return batch_spec([spec_inputs_tree(p_rows, q_rows, xs, u_acc, u_res)], parent, 2, **kw)
+
+    def check(o, A, best, R, emitted, nodes):
+        assert o["n_accepted"][0] == A and o["best_branch"][0] == best and o["decide_row"][0] == R
+        assert o["n_emitted"][0] == len(emitted)
+        assert o["emitted"][0].tolist() == emitted + [-1] * (3 - len(emitted))
+        assert o["accepted_nodes"][0].tolist() == nodes + [-1] * (2 - len(nodes))
+
+    # 1. every branch accepts its first node and fails its second: tie at A = 1 -> branch 0.  Deciding row = node 1;
+    #    rejected node 2 proposed token 0 from QA; residual [0, 0, .25, .25], Z = .5, u_res[1] = .6 -> threshold .3 -> id 3.
+    #    (QB, the other branches' distribution, would give id 1; u_res of another row (.1) id 2.)
+    p_rows = [PA, P0, PA, P0, PA, P0, PA]
+    q_rows = [None, flat, QA, flat, QB, flat, QB]
+    xs = [0, 1, 0, 2, 0, 3, 0]
+    u_acc = [0, 0.0, 0.5, 0.0, 0.5, 0.0, 0.5]
+    u_res = [0.1, 0.6, 0.1, 0.1, 0.1, 0.1, 0.1]
+    check(run(p_rows, q_rows, xs, u_acc, u_res), 1, 0, 1, [1, 3], [1])
+
+    # 2. the longer branch sits at the highest index: branch 0 accepts one node, branch 1 none, branch 2 both.
+    #    Whole branch accepted -> bonus from the last node's own row PA with u_res[6] = .35: cdf .1 .3 .6 -> id 2.
+    p_rows = [PA, P0, PA, PA, PA, PA, PA]
+    q_rows = [None, flat, QA, [0, 0, 0, 1.0], flat, flat, flat]
+    xs = [0, 1, 0, 3, 1, 2, 3]
+    u_acc = [0, 0.0, 0.5, 0.99, 0.0, 0.0, 0.0]          # node 3: .99 * 1 > PA[3] = .4 fails
+    u_res = [0.9, 0.9, 0.9, 0.9, 0.9, 0.9, 0.35]
+    check(run(p_rows, q_rows, xs, u_acc, u_res), 2, 2, 6, [2, 3, 2], [5, 6])
+    #    the same with emit_bonus off: nothing beyond the accepted tokens
+    check(run(p_rows, q_rows, xs, u_acc, u_res, emit_bonus=False), 2, 2, 6, [2, 3], [5, 6])
+
+    # 3. every branch fails at depth 0: A = 0, branch 0, deciding row = root; the residual uses branch 0's first node's
+    #    distribution (QA -> [0, 0, .25, .25]) and u_res[root] = .6 -> id 3; QB of branches 1, 2 would give id 1.
+    p_rows = [P0, PA, PA, PA, PA, PA, PA]
+    q_rows = [None, QA, flat, QB, flat, QB, flat]
+    xs = [0, 0, 1, 0, 1, 0, 1]
+    u_acc = [0, 0.5, 0.0, 0.5, 0.0, 0.5, 0.0]
+    u_res = [0.6, 0.1, 0.1, 0.1, 0.1, 0.1, 0.1]
+    check(run(p_rows, q_rows, xs, u_acc, u_res), 0, 0, 0, [3], [])
+
+    # 4. the winner is branch 1, rejected at depth 1: deciding row = node 3, residual of its row P0 against node 4's QA
+    #    with u_res[3] = .6 -> id 3 (node 2's or node 6's QB would give id 1; u_res of rows 0, 1, 5 (.1) id 2).
+    p_rows = [P0, PA, PA, P0, PA, PA, PA]
+    q_rows = [None, QB, QB, flat, QA, QB, QB]
+    xs = [0, 0, 1, 2, 0, 0, 1]
+    u_acc = [0, 0.5, 0.0, 0.0, 0.5, 0.5, 0.0]           # nodes 1 and 5 propose token 0 (no mass at the root): fail
+    u_res = [0.1, 0.1, 0.1, 0.6, 0.1, 0.1, 0.1]
+    check(run(p_rows, q_rows, xs, u_acc, u_res), 1, 1, 3, [2, 3], [3])
+
+    # 5. the accept test of a node reads ITS OWN uniform and its PARENT's row: node 4 (branch 1, depth 1) proposes
+    #    token 3 from a one-hot q; the parent row PA gives it .4: u = .39 passes, u = .41 fails.
+    p_rows = [PA, PA, PA, PA, P0, PA, PA]               # node 4's own row gives token 3 mass .25: not the one tested
+    q_rows = [None, flat, flat, flat, [0, 0, 0, 1.0], flat, flat]
+    xs = [0, 0, 0, 1, 3, 0, 0]
+    for u4, A in ((0.39, 2), (0.41, 1)):
+        u_acc = [0, 0.99, 0.99, 0.0, u4, 0.99, 0.99]    # nodes 1, 5: .99 * .25 > PA[0] = .1 fail
+        o = run(p_rows, q_rows, xs, u_acc, [0.5] * 7)
+        assert o["n_accepted"][0] == A and o["best_branch"][0] == 1
+
+
 def test_spec_rule_generic_grid_is_close_to_p():
     # the same law on values that are not grid-aligned: midpoint integration, tolerance ~ 1/N
     rng = np.random.default_rng(3)

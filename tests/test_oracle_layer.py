@@ -109,3 +109,85 @@ def test_layer_with_zero_output_projections_returns_its_input_and_positions_foll
     x1 = T.bf16_round(T.bf16_to_f64(x) + T.bf16_to_f64(full["attn"]) @ T.bf16_to_f64(w["w_o"]).T)
     assert np.abs(T.bf16_to_f64(full["x"]) - x1).max() > 0          # the MLP added something on top
     assert full["normed"].shape == x.shape
+
+
+# ---------------------------------------------------------------------------------------------
+# Composition of the layer (the pre-norm decoder layer the oracle's header states): every wiring choice inside
+# target_layer() is pinned by a sparse weight whose effect has a closed form in terms of the pinned pieces.
+# ---------------------------------------------------------------------------------------------
+def _layer_case(seed=7):
+    rng = np.random.default_rng(seed)
+    H, Hq, Hkv, d, inter, B = 64, 4, 2, 16, 96, 2
+    parent = [-1, 0, 1, 0, 3]
+    w = _tiny_layer(rng, H, Hq, Hkv, d, inter)
+    prefix_len = np.array([20, 33], np.int32)
+    pages = 3
+    page_table = np.arange(B * pages, dtype=np.int32).reshape(B, pages)
+    k_pool = T.bf16_round_bits(rng.normal(size=(B * pages, Hkv, 16, d)))
+    v_pool = T.bf16_round_bits(rng.normal(size=(B * pages, Hkv, 16, d)))
+    x = T.bf16_round_bits(rng.normal(size=(B * len(parent), H)))
+    dims = dict(H=H, Hq=Hq, Hkv=Hkv, d=d, inter=inter, B=B, n=len(parent))
+    run = lambda ww: T.target_layer(x, ww, k_pool, v_pool, page_table, prefix_len, parent, Hq, Hkv, d, 10000.0, 1e-6)
+    return dims, w, x, prefix_len, parent, run
+
+
+def _unit_rows(shape, entries):
+    m = np.zeros(shape)
+    for (r, c), v in entries.items():
+        m[r, c] = v
+    return T.bf16_round_bits(m)
+
+
+def test_layer_mlp_half_gate_first_then_up_on_the_normed_post_attention_stream():
+    """One gate row reads column 0 of the MLP's input, one up row column 1, one down column writes column 2:
+    the layer must add silu(h_0) * h_1 to column 2 of the post-attention stream x1 and nothing anywhere else, with
+    h = RMSNorm(x1; norm_mlp).  Fails if gate and up rows are swapped, if the MLP reads norm(x) instead of norm(x1),
+    if the second residual is taken from x instead of x1, or if the wrong norm weight is used."""
+    dims, w, x, _, _, run = _layer_case()
+    H, inter = dims["H"], dims["inter"]
+    ww = dict(w, w_gate_up=_unit_rows((2 * inter, H), {(0, 0): 1.0, (inter, 1): 1.0}),      # gate row 0 <- col 0, up row 0 <- col 1
+              w_down=_unit_rows((H, inter), {(2, 0): 1.0}))
+    res = run(ww)
+    x1 = T.bf16_round(T.bf16_to_f64(x) + T.bf16_to_f64(res["attn"]) @ T.bf16_to_f64(w["w_o"]).T)
+    assert np.abs(x1 - T.bf16_to_f64(x)).max() > 1e-2                     # attention really moved the stream
+    h = T.bf16_round(T.rmsnorm(x1, T.bf16_to_f64(w["norm_mlp"]), 1e-6))
+    a, b = h[:, 0], h[:, 1]
+    act = T.bf16_round(a / (1.0 + np.exp(-a)) * b)                         # silu(gate) * up, stored in bf16
+    want = x1.copy()
+    want[:, 2] = x1[:, 2] + act
+    np.testing.assert_array_equal(res["x"], T.bf16_round_bits(want))
+    swapped = x1[:, 2] + T.bf16_round(b / (1.0 + np.exp(-b)) * a)
+    assert np.abs(T.bf16_round(swapped) - T.bf16_to_f64(res["x"])[:, 2]).max() > 1e-3   # the case tells the two orders apart
+
+
+def test_layer_without_mlp_is_x_plus_output_projection_of_attention():
+    dims, w, x, _, _, run = _layer_case()
+    res = run(dict(w, w_down=np.zeros_like(w["w_down"])))
+    x1 = T.bf16_round_bits(T.bf16_to_f64(x) + T.bf16_to_f64(res["attn"]) @ T.bf16_to_f64(w["w_o"]).T)
+    np.testing.assert_array_equal(res["x"], x1)
+
+
+def test_layer_qkv_split_and_rotation_of_queries_and_keys():
+    """w_qkv rows are (query rows, key rows, value rows).  With only the key block non-zero the queries and values
+    come out zero and the keys are the ROTATED projection; with only the query block non-zero the queries are the
+    rotated projection and keys / values are zero.  Fails on a wrong Q/K/V boundary and on a missing rotation."""
+    dims, w, x, prefix_len, parent, run = _layer_case()
+    H, Hq, Hkv, d, B, n = (dims[k] for k in ("H", "Hq", "Hkv", "d", "B", "n"))
+    from oracle import oracle as O
+    _, depth = O.tree(parent)
+    pos = T.positions(prefix_len, depth)
+    h1 = T.bf16_round(T.rmsnorm(T.bf16_to_f64(x), T.bf16_to_f64(w["norm_attn"]), 1e-6))
+    Wf = T.bf16_to_f64(w["w_qkv"])
+    blocks = {"q": (0, Hq * d, Hq), "k": (Hq * d, (Hq + Hkv) * d, Hkv)}
+    for name, (lo, hi, heads) in blocks.items():
+        only = np.zeros_like(w["w_qkv"])
+        only[lo:hi] = w["w_qkv"][lo:hi]
+        res = run(dict(w, w_qkv=only))
+        proj = (h1 @ Wf[lo:hi].T).reshape(B * n, heads, d)
+        rotated = T.bf16_round_bits(T.rope(proj, pos, 10000.0)).reshape(B, n, heads, d)
+        got = res["q"] if name == "q" else res["k_new"]
+        np.testing.assert_array_equal(got, rotated)
+        assert not np.array_equal(got, T.bf16_round_bits(proj).reshape(B, n, heads, d))     # positions > 0: rotation matters
+        for other in ("q", "k_new", "v_new"):
+            if other != ("q" if name == "q" else "k_new"):
+                assert (T.bf16_to_f64(res[other]) == 0).all(), (name, other)        # (+0 or -0)
