@@ -19,16 +19,17 @@
 //   warp 0, 11  stage K and V into two rings of 4-slot stages (4 or 6 deep: whatever the Q buffers leave): one TMA box
 //               per page and tensor, 128-byte swizzle; ragged page and tree tokens by 16-byte asynchronous copies
 //               with zero fill
-//   warp 1      owns TMEM and issues S = Q K^T for a pair of tiles at a time (tcgen05.mma, M=128 rows, N up to 128
-//               tokens, d/16 instructions) into two adjacent of four S buffers, as far ahead as rings and buffers allow;
-//               Q is double-buffered, so it runs on into the next unit while the softmax warps finish this one
+//   warp 1      owns TMEM and issues S = Q K^T tile by tile (tcgen05.mma, M=128 rows, N up to 64 tokens, d/16
+//               instructions) into one of four S buffers, as far ahead as rings and buffers allow; Q is
+//               double-buffered, so it runs on into the next unit while the softmax warps finish this one
 //   warp 2      issues O += P V (P as the A operand from tensor memory, V as an MN-major operand from shared memory)
-//   warps 3..10 softmax, two groups of four warps on alternate tiles, one thread per row (TMEM lane): a first pass
-//               over the row's scores for the maximum, a second for P = exp2(s*c - offset), written as bf16 over the
-//               first half of the same S buffer (the buffer is released by the P V that reads it); no shuffles, no
-//               shared memory; each group keeps its own accumulator O in TMEM (rescaled only when a row's maximum
-//               grew by more than 2^8: the stale offset is carried exactly through the sum and the division) and the
-//               two are merged like split-KV partials; they also stage the next unit's Q a unit ahead
+//   warps 3..10 softmax, two groups of four warps on alternate tiles, one thread per row (TMEM lane): ONE pass over the
+//               row's 64 scores: P = exp2(s*c - offset) against the offset in use, written as bf16 over the first half
+//               of the same S buffer (the buffer is released by the P V that reads it); no shuffles, no shared memory,
+//               and no row maximum on the way: the offset is set by the row's first tile and moves only when a tile's
+//               SUM of P outgrows 2^14 (that tile is then redone; the stale offset is carried exactly through the sum
+//               and the division); each group keeps its own accumulator O in TMEM and the two are merged like
+//               split-KV partials; they also stage the next unit's Q a unit ahead
 // Every ring index and mbarrier parity is a function of one per-CTA tile counter, identical in all roles.
 // Every mbarrier wait is bounded; on expiry the kernel records MIRROR_DEV_TIMEOUT and unwinds.
 #include <math.h>
@@ -51,7 +52,9 @@ constexpr int kRows = 128;                          // UMMA M: rows per row bloc
 constexpr int kMaxBatch = 1024;
 constexpr int kMaxStages = 8;                       // ring depths are template parameters (even: tiles are staged in pairs)
 constexpr int kSBufs = 4;                           // S buffers in TMEM (power of two)
-constexpr float kRescaleLog2 = 8.0f;
+constexpr float kOffsetBias = 0.0f;                 // a row's offset puts the maximum of the tile that set it at 2^0 ...
+constexpr float kSumLimit = 16384.0f;               // ... and moves when a tile's sum of P passes 2^14 (no single P is beyond 2^14 then)
+constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kTmemCols = 512;                      // S0..S3 (64 columns each; P overwrites the first 32 of its S) | O of group 0 | O of group 1
 constexpr int kTmemO = kSBufs * kTileTok;
 
@@ -63,8 +66,8 @@ struct AttnParams {
     int L, B, n, Hq, Hkv, G;
     int rows, n_rb, rows_per_rb;          // rows per unit, row blocks, rows per block
     int n_groups;                         // CTA groups (grid = n_groups * n_rb)
-    int snap_cap;
-    int whole_units;               // 1: prefer a group count that divides equal-length units (no cuts)                         // boundaries move to a unit boundary that is at most this many tiles away
+    int snap_cap;                         // boundaries move to a unit boundary that is at most this many tiles away
+    int whole_units;                      // 1: prefer a group count that divides equal-length units (no cuts)
     int max_pages, num_pages, layer_pages;
     int q_half_bytes;                     // one 64-column half of a Q buffer: rows rounded up to 8, 128 B each
     int tree_slots;
@@ -80,8 +83,6 @@ struct AttnParams {
     float* lse_out;
     float* partial;                       // [grid][2][D+4][128]
     int* status;
-    int timing_exit;                      // developer aid: leave the kernel early (1: at entry, 2: after the prologue)
-    long long* timing;                    // developer aid (MIRROR_ATTN_TIMING builds): per-role cycle counters of one CTA
 };
 
 struct UnitPos {                          // where a global tile index falls
@@ -127,6 +128,21 @@ __device__ __noinline__ UnitPos locate(long long x, const AttnParams& p, const i
     return u;
 }
 
+// P = exp2(x) for two fp32 arguments: the pair rounded to bf16 (element `lo` in the low half, as the tensor core reads P);
+// the fp32 values are added to two running sums.
+__device__ __forceinline__ uint32_t exp2_pair(float lo, float hi, float& sum_lo, float& sum_hi) {
+    const float e0 = ptx::ex2_approx(lo), e1 = ptx::ex2_approx(hi);
+    sum_lo += e0;
+    sum_hi += e1;
+    uint32_t pk;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(e1), "f"(e0));
+    return pk;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float m;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(m) : "f"(a), "f"(b), "f"(c));
+    return m;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -157,30 +173,8 @@ __device__ __forceinline__ void tmem_st_32x32b_x32(uint32_t taddr, const uint32_
           "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
         : "memory");
 }
-__device__ __forceinline__ void tmem_st_32x32b_x16(uint32_t taddr, const uint32_t (&r)[16]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-        : "memory");
-}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// Developer timing aid: with -DMIRROR_ATTN_TIMING each role of CTA 5 accumulates the cycles it spends in its waits
-// and writes them to p.timing; otherwise these macros vanish.
-#ifdef MIRROR_ATTN_TIMING
-#define T_DECL(...) long long __VA_ARGS__
-#define T_WAIT(acc, expr) ({ long long t__ = clock64(); bool r__ = (expr); acc += clock64() - t__; r__; })
-#define T_NOW() clock64()
-#define T_MARK(acc) do { long long n__ = clock64(); acc += n__ - tm__; tm__ = n__; } while (0)
-#define T_STORE(base, ...) do { if (p.timing && blockIdx.x == 5) { long long v__[] = {__VA_ARGS__}; for (int i__ = 0; i__ < (int)(sizeof v__ / sizeof v__[0]); ++i__) p.timing[(base) + i__] = v__[i__]; } } while (0)
-#else
-#define T_DECL(...)
-#define T_WAIT(acc, expr) (expr)
-#define T_NOW() 0ll
-#define T_MARK(acc) do { } while (0)
-#define T_STORE(base, ...) do { } while (0)
-#endif
 
 template <int D>
 struct Cfg {
@@ -306,15 +300,6 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int group = blockIdx.x / p.n_rb, rb = blockIdx.x % p.n_rb;
-#ifdef MIRROR_ATTN_TIMING
-#define T_STAMP(i) do { if (p.timing && tid == 0) { unsigned long long g__; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g__) :: "memory"); p.timing[64 + blockIdx.x * 4 + (i)] = (long long)g__; } } while (0)
-#else
-#define T_STAMP(i) do { } while (0)
-#endif
-    T_STAMP(0);
-#ifdef MIRROR_ATTN_TIMING
-    if (p.timing_exit == 1) return;
-#endif
 
     // ---- prologue ---------------------------------------------------------------------------------
     // (programmatic dependent launch: barriers and tensor memory are set up while the kernel ahead in the stream is
@@ -369,15 +354,6 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     if (!fits && tid == 0) dev_check(p, 600);
     const long long x_begin = (fits && group < n_groups) ? group_begin(part, group, p, cumT) : 0;
     const long long x_end = (fits && group < n_groups) ? group_begin(part, group + 1, p, cumT) : 0;
-
-    T_STAMP(1);
-#ifdef MIRROR_ATTN_TIMING
-    if (p.timing_exit == 2) {
-        __syncthreads();
-        if (warp == 1) ptx::tmem_dealloc(tmem_base, kTmemCols);
-        return;
-    }
-#endif
     if (warp == 0 || warp == kVProducerWarp) {
         // =========================================================================== producers
         // warp 0 stages K, the last warp stages V: a warp issues its TMA boxes one after the other, so two
@@ -388,7 +364,6 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         uint32_t it = 0;                   // tiles issued by this CTA so far (ring index and parity source)
         bool ok = true;
         long long x = x_begin;
-        T_DECL(w_empty = 0, t0 = T_NOW(), tm__ = 0, p_pre = 0, p_issue = 0, p_fill = 0);
         // one TMA box (a whole page of this tensor) per lane
         const bool has_box = lane < kStageSlots;
         const int my_slot = lane;
@@ -417,14 +392,11 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 }
             }
             for (int t = sg.t_first; t < sg.t_last && ok; ++t, ++x, ++it) {
-#ifdef MIRROR_ATTN_TIMING
-                tm__ = T_NOW();
-#endif
                 const int st = vrole ? (int)(it % VS) : (int)(it % KR);
                 const uint32_t ph = (vrole ? it / VS : it / KR) & 1;
                 const int next_page = (t + 1 < sg.t_last) ? fetch_page(t + 1) : 0;
                 bool w = true;
-                if (lane == 0) w = !ctrl->abort && T_WAIT(w_empty, ptx::mbar_wait(&empty[st], ph ^ 1));
+                if (lane == 0) w = !ctrl->abort && ptx::mbar_wait(&empty[st], ph ^ 1);
                 w = __shfl_sync(0xffffffffu, w, 0);
                 if (!w) { if (lane == 0) timeout(p, ctrl, 10); ok = false; break; }
                 uint8_t* dst = (vrole ? sV : sK) + (size_t)st * C::kStageBytes;
@@ -432,7 +404,6 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 const int n_slots = max(0, min(kStageSlots, sg.slots_all - sl0));      // slots that exist in this stage
                 const int n_tma = max(0, min(kStageSlots, sg.pages_full - sl0));       // leading slots that are whole pages
                 const int n_fill = n_slots;
-                T_MARK(p_pre);
                 if (n_tma < n_fill) {
                     // ragged page and tree tokens by asynchronous 16-byte copies (rows beyond the valid count are
                     // zero-filled), all in flight together; the loops are kept rolled: this path runs once per unit, and
@@ -471,7 +442,6 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     ptx::fence_proxy_async();
                     __syncwarp();
                 }
-                T_MARK(p_fill);
                 // (the barrier's one arrival is this arming, so copies that land before it cannot complete the phase)
                 if (lane == 0) ptx::mbar_arrive_expect_tx(&full[st], (uint32_t)(n_tma * C::kSlotBytes));
                 if (has_box && my_slot < n_tma) {
@@ -484,10 +454,8 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                         ptx::tma_load_5d(dst + my_slot * C::kSlotBytes, &tm_k, &full[st], 0, 0, 0, 0, pg * p.Hkv + u.g);
                 }
                 my_page = next_page;
-                T_MARK(p_issue);
             }
         }
-        if (lane == 0) T_STORE(vrole ? 32 : 16, T_NOW() - t0, w_empty, (long long)it, p_pre, p_fill, p_issue);
         if (!ok && lane == 0) {
             // let copies already in flight land before the CTA's shared memory goes away
             const uint32_t ns = vrole ? VS : KR;
@@ -506,46 +474,33 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             uint32_t it = 0, seg = 0;
             bool ok = true;
             long long x = x_begin;
-            T_DECL(w_q = 0, w_k = 0, w_s = 0, t0 = T_NOW());
-#ifdef MIRROR_ATTN_TIMING
-            unsigned long long g0; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g0) :: "memory");
-#endif
             while (x < x_end && ok) {
                 const Segment sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
-                if (ctrl->abort || !T_WAIT(w_q, ptx::mbar_wait(&ctrl->q_full[seg & 1], (seg >> 1) & 1))) { timeout(p, ctrl, 20); ok = false; break; }
+                if (ctrl->abort || !ptx::mbar_wait(&ctrl->q_full[seg & 1], (seg >> 1) & 1)) { timeout(p, ctrl, 20); ok = false; break; }
                 const uint32_t q_seg = q_lo + (uint32_t)(((seg & 1) * q_buf_bytes) >> 4);
                 ++seg;
-                // parts begin and end on pairs of tiles: a pair is the eight slots of two consecutive ring stages
-                for (int t = sg.t_first; t < sg.t_last; t += 2, x += 2, it += 2) {
-                    bool ready = !ctrl->abort;
-                    for (int j = 0; j < 2 && ready; ++j) {
-                        const uint32_t i2 = it + j;
-                        ready = T_WAIT(w_k, ptx::mbar_wait(&ctrl->k_full[i2 % KR], (i2 / KR) & 1)) &&
-                                T_WAIT(w_s, ptx::mbar_wait(&ctrl->s_free[i2 & (kSBufs - 1)], ((i2 / kSBufs) & 1) ^ 1));
-                    }
-                    if (!ready) { timeout(p, ctrl, 21); ok = false; break; }
-                    ptx::tc_fence_after();
+                // one tile (a ring stage of four slots) per issue: each S buffer is scored as soon as the P V that read
+                // it has completed, so the two softmax groups run half a period apart instead of in step
+                for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
                     const int st = it % KR, sb = it & (kSBufs - 1);
-                    // one instruction per 16 columns of d scores both tiles: up to 128 tokens in token order
-                    const int n_sl = min(2 * kStageSlots, sg.slots_all - t * kStageSlots);
-                    const uint32_t idesc = ptx::umma_idesc_bf16(kRows, n_sl * kSlotTok);
-                    const uint32_t kb = k_lo + (uint32_t)((st * C::kStageBytes) >> 4);
-                    const uint32_t d = tmem_base + (uint32_t)(sb * kTileTok);
+                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->k_full[st], (it / KR) & 1) ||
+                        !ptx::mbar_wait(&ctrl->s_free[sb], ((it / kSBufs) & 1) ^ 1)) { timeout(p, ctrl, 21); ok = false; break; }
+                    ptx::tc_fence_after();
+                    const int n_sl = min(kStageSlots, sg.slots_all - t * kStageSlots);       // (a pair's second tile may be empty)
+                    if (n_sl > 0) {
+                        const uint32_t idesc = ptx::umma_idesc_bf16(kRows, n_sl * kSlotTok);
+                        const uint32_t kb = k_lo + (uint32_t)((st * C::kStageBytes) >> 4);
+                        const uint32_t d = tmem_base + (uint32_t)(sb * kTileTok);
 #pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk)
-                        ptx::umma_f16_lohi(d, q_seg + (uint32_t)(((kk >> 2) * p.q_half_bytes + (kk & 3) * 32) >> 4), hi_q,
-                                           kb + (uint32_t)(((kk >> 2) * 1024 + (kk & 3) * 32) >> 4), hi_k, idesc, kk != 0);
+                        for (int kk = 0; kk < D / 16; ++kk)
+                            ptx::umma_f16_lohi(d, q_seg + (uint32_t)(((kk >> 2) * p.q_half_bytes + (kk & 3) * 32) >> 4), hi_q,
+                                               kb + (uint32_t)(((kk >> 2) * 1024 + (kk & 3) * 32) >> 4), hi_k, idesc, kk != 0);
+                    }
                     ptx::umma_commit(&ctrl->s_full[sb]);
-                    ptx::umma_commit(&ctrl->s_full[sb + 1]);
                     ptx::umma_commit(&ctrl->k_empty[st]);
-                    ptx::umma_commit(&ctrl->k_empty[st + 1]);
                 }
                 if (!ok) break;
             }
-            T_STORE(0, T_NOW() - t0, w_q, w_k, w_s, (long long)it);
-#ifdef MIRROR_ATTN_TIMING
-            { unsigned long long g1; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g1) :: "memory"); T_STORE(48, (long long)(g1 - g0)); }
-#endif
         }
     } else if (warp == 2) {
         // =========================================================================== P V issuer
@@ -556,7 +511,6 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             uint32_t it = 0;
             bool ok = true;
             long long x = x_begin;
-            T_DECL(w_p = 0, w_v = 0, t0 = T_NOW());
             uint32_t seg = 0;
             while (x < x_end && ok) {
                 const Segment sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
@@ -565,8 +519,8 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 ++seg;
                 for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
                     const int st = it % VS, pb = it & 1, sb = it & (kSBufs - 1);
-                    if (ctrl->abort || !T_WAIT(w_p, ptx::mbar_wait(&ctrl->p_full[sb], (it / kSBufs) & 1)) ||
-                        !T_WAIT(w_v, ptx::mbar_wait(&ctrl->v_full[st], (it / VS) & 1))) {
+                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->p_full[sb], (it / kSBufs) & 1) ||
+                        !ptx::mbar_wait(&ctrl->v_full[st], (it / VS) & 1)) {
                         timeout(p, ctrl, 23); ok = false; break;
                     }
                     ptx::tc_fence_after();
@@ -583,7 +537,6 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     ptx::umma_commit(&ctrl->pv_done[pb]);
                 }
             }
-            T_STORE(24, T_NOW() - t0, w_p, w_v);
         }
     } else {
         // =========================================================================== softmax / epilogue
@@ -638,57 +591,23 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         uint32_t it = 0;
         bool ok = true;
         long long x = x_begin;
-        T_DECL(w_sf = 0, w_pv = 0, w_end = 0, t_epi = 0, t_q = 0, t0 = T_NOW(), te = 0, tm__ = 0, s_ld = 0, s_free = 0, s_max = 0, s_xch = 0, s_exp = 0, s_fin = 0, t_init = 0, t_loop = 0, tl = 0, t_max = 0, t_ld1 = 0);
         Segment sg;
-        // one 32-column chunk of this row's scores: tcgen05.ld, then the visibility mask (bit j: column j) where the
-        // tile needs one
-        auto load_scores = [&](int sb, int c4, uint32_t cm, float (&v)[32]) {
-            uint32_t r[32];
-            ptx::tmem_ld_32x32b_x32(lane_base + (uint32_t)(sb * kTileTok + c4 * 32), r);
-            ptx::tmem_ld_wait();
+        // P of one tile from the row's 64 scores v[]: p = exp2(s*c - offset) as bf16 pairs, and the row sum in fp32
+        auto tile_p = [&](const float (&v)[kTileTok], float off_log2, uint32_t (&pk)[kTileTok / 2]) -> float {
+            const float o = (off_log2 == -INFINITY) ? 0.f : off_log2;       // nothing visible yet: every score is -inf
+            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-            if (cm != 0xffffffffu) {
-#pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    if (!((cm >> j) & 1u)) v[j] = -INFINITY;
+            for (int j = 0; j < kTileTok / 2; j += 2) {
+                pk[j] = exp2_pair(fmaf(v[2 * j], p.scale_log2e, -o), fmaf(v[2 * j + 1], p.scale_log2e, -o), s0, s1);
+                pk[j + 1] = exp2_pair(fmaf(v[2 * j + 2], p.scale_log2e, -o), fmaf(v[2 * j + 3], p.scale_log2e, -o), s2, s3);
             }
+            return (s0 + s1) + (s2 + s3);
         };
-        // pass 1: the row maximum of a tile
-        auto tile_max = [&](int sb, uint32_t cm0, uint32_t cm1) -> float {
-            float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        auto tile_max = [&](const float (&v)[kTileTok]) -> float {
+            float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
-            for (int c4 = 0; c4 < kTileTok / 32; ++c4) {
-                float v[32];
-                load_scores(sb, c4, c4 == 0 ? cm0 : cm1, v);
-                if (c4 == 0) T_MARK(t_ld1);
-#pragma unroll
-                for (int j = 0; j < 32; ++j) m4[j & 3] = fmaxf(m4[j & 3], v[j]);
-            }
-            return fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
-        };
-        // pass 2: P = exp2(s*c - offset) as bf16 pairs over the first 32 columns of the same S buffer (a thread
-        // only ever touches its own lane, and a 32-column chunk of S is in registers before its P is written
-        // over columns that were read earlier); returns the row sum
-        auto tile_p = [&](int sb, uint32_t cm0, uint32_t cm1, float m_off) -> float {
-            const float off = (m_off == -INFINITY) ? 0.f : m_off * p.scale_log2e;
-            float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int c4 = 0; c4 < kTileTok / 32; ++c4) {
-                float v[32];
-                load_scores(sb, c4, c4 == 0 ? cm0 : cm1, v);
-                uint32_t pk[16];
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const float e0 = ptx::ex2_approx(fmaf(v[2 * j], p.scale_log2e, -off));
-                    const float e1 = ptx::ex2_approx(fmaf(v[2 * j + 1], p.scale_log2e, -off));
-                    sum4[j & 3] += e0 + e1;
-                    pk[j] = pack_bf16(e0, e1);
-                }
-                tmem_st_32x32b_x16(lane_base + (uint32_t)(sb * kTileTok + c4 * 16), pk);
-            }
-            tmem_st_wait();
-            return (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+            for (int j = 0; j < kTileTok; j += 4) { m0 = max3(m0, v[j], v[j + 1]); m1 = max3(m1, v[j + 2], v[j + 3]); }
+            return fmaxf(m0, m1);
         };
 
         uint32_t seg = 0;                                          // parts walked so far: Q buffer = seg & 1
@@ -697,94 +616,101 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             stage_q(sg.u, 0);
             q_ready(0);
         }
-#ifdef MIRROR_ATTN_TIMING
-        t_init = T_NOW() - t0;
-#endif
         while (x < x_end && ok) {
             const UnitPos u = sg.u;
             const bool whole_unit = (sg.t_first == 0 && sg.t_last == u.tiles_in_unit);
-            float m_used = -INFINITY, l_run = 0.f;                 // this group's offset and running sum
-            bool first = true;                                     // no tile of this unit's part seen by this group yet
+            float off_used = -INFINITY, l_run = 0.f;               // this group's offset (log2 units) and running sum
             // the part after this one: its Q goes into the other Q buffer now (every Q K^T that read that buffer
             // belongs to the part before this one and has completed), so the issuer can run on into the next unit
             Segment sg_next;
             const long long x_next = x + (sg.t_last - sg.t_first);
             const bool has_next = x_next < x_end;
-#ifdef MIRROR_ATTN_TIMING
-            te = T_NOW();
-#endif
             if (has_next) {
                 sg_next = make_segment(x_next, x_end, p, cumT, s_len, tiles_per_layer);
                 stage_q(sg_next.u, (seg + 1) & 1);
             }
             bool q_pending = has_next;
-#ifdef MIRROR_ATTN_TIMING
-            s_xch += T_NOW() - te;
-#endif
 
-#ifdef MIRROR_ATTN_TIMING
-            tl = T_NOW();
-#endif
             for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
                 if ((int)(it & 1) != grp) continue;
                 const int sb = it & (kSBufs - 1);
-                if (ctrl->abort || !T_WAIT(w_sf, ptx::mbar_wait(&ctrl->s_full[sb], (it / kSBufs) & 1))) { timeout(p, ctrl, 30); ok = false; break; }
+                if (ctrl->abort || !ptx::mbar_wait(&ctrl->s_full[sb], (it / kSBufs) & 1)) { timeout(p, ctrl, 30); ok = false; break; }
                 ptx::tc_fence_after();
-#ifdef MIRROR_ATTN_TIMING
-                tm__ = T_NOW();
-#endif
-                float mx = -INFINITY, sum = 0.f;
+                float sum = 0.f;
                 // visibility of this tile's columns for this row: all ones except in a unit's last pairs
                 uint32_t cm0 = 0xffffffffu, cm1 = 0xffffffffu;
                 if (t * kStageSlots + kStageSlots > sg.pages_full) {
                     cm0 = chunk_mask(t * kStageSlots, sg.pages_full, sg.pages_all, sg.slots_all, sg.len, anc0, anc1);
                     cm1 = chunk_mask(t * kStageSlots + 2, sg.pages_full, sg.pages_all, sg.slots_all, sg.len, anc0, anc1);
                 }
-                if (warp_has_rows) mx = tile_max(sb, cm0, cm1);
-                T_MARK(t_max);
-                if (first) m_used = mx;
-                // offset in use: set by the group's first tile, moved only when the row maximum outgrew it by more than 2^8
-                const bool move = warp_has_rows && !first &&
-                                  (((mx - m_used) * p.scale_log2e > kRescaleLog2) || (m_used == -INFINITY && mx > -INFINITY));
-                if (__any_sync(0xffffffffu, move)) {
-                    // rare: rescale this group's accumulator and running sum once its last P V (two tiles ago) is complete
-                    if (ctrl->abort || !T_WAIT(w_pv, ptx::mbar_wait(&ctrl->pv_done[grp], ((it - 2) >> 1) & 1))) { timeout(p, ctrl, 33); ok = false; break; }
-                    ptx::tc_fence_after();
-                    const float m_next = move ? fmaxf(mx, m_used) : m_used;
-                    const float alpha = (m_used == -INFINITY) ? ((m_next == -INFINITY) ? 1.f : 0.f)
-                                                              : exp2f((m_used - m_next) * p.scale_log2e);
-#pragma unroll 1
-                    for (int c4 = 0; c4 < D / 32; ++c4) {
-                        uint32_t r[32];
-                        ptx::tmem_ld_32x32b_x32(o_mine + (uint32_t)(c4 * 32), r);
+                if (warp_has_rows) {
+                    // one pass: the row's 64 scores are read once and P is computed against the offset in use, with no
+                    // row maximum in the way; only the tile's SUM is watched
+                    float v[kTileTok];
+                    {
+                        uint32_t r0[32], r1[32];
+                        ptx::tmem_ld_32x32b_x32(lane_base + (uint32_t)(sb * kTileTok), r0);
+                        ptx::tmem_ld_32x32b_x32(lane_base + (uint32_t)(sb * kTileTok + 32), r1);
                         ptx::tmem_ld_wait();
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * alpha);
-                        tmem_st_32x32b_x32(o_mine + (uint32_t)(c4 * 32), r);
+                        for (int j = 0; j < 32; ++j) { v[j] = __uint_as_float(r0[j]); v[32 + j] = __uint_as_float(r1[j]); }
                     }
+                    if ((cm0 & cm1) != 0xffffffffu) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            if (!((cm0 >> j) & 1u)) v[j] = -INFINITY;
+                            if (!((cm1 >> j) & 1u)) v[32 + j] = -INFINITY;
+                        }
+                    }
+                    // The offset (in log2 units) is set by the first tile in which the row sees anything: that tile's
+                    // maximum.  (Before that every P was 0: nothing to rescale.)
+                    if (__any_sync(0xffffffffu, off_used == -INFINITY)) {
+                        const float mx = tile_max(v);
+                        if (off_used == -INFINITY && mx > -INFINITY) off_used = mx * p.scale_log2e - kOffsetBias;
+                    }
+                    uint32_t pk[kTileTok / 2];
+                    sum = tile_p(v, off_used, pk);
+                    // The offset moves only when a tile's sum outgrows kSumLimit (an overflow makes the sum infinite, which
+                    // counts): rare, and then this tile is redone against its own maximum after the accumulator and the
+                    // running sum have been rescaled.  Whatever the offset, it is carried exactly through the sum and the
+                    // final division.
+                    const bool grow = !(sum <= kSumLimit);
+                    if (__any_sync(0xffffffffu, grow)) {
+                        // this group's last P V (two tiles ago) must be complete before its accumulator is touched
+                        if (it >= 2 && (ctrl->abort || !ptx::mbar_wait(&ctrl->pv_done[grp], ((it - 2) >> 1) & 1))) { timeout(p, ctrl, 33); ok = false; break; }
+                        ptx::tc_fence_after();
+                        const float off_next = grow ? tile_max(v) * p.scale_log2e - kOffsetBias : off_used;
+                        const float alpha = grow ? exp2f(off_used - off_next) : 1.f;
+#pragma unroll 1
+                        for (int c4 = 0; c4 < D / 32; ++c4) {
+                            uint32_t r[32];
+                            ptx::tmem_ld_32x32b_x32(o_mine + (uint32_t)(c4 * 32), r);
+                            ptx::tmem_ld_wait();
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * alpha);
+                            tmem_st_32x32b_x32(o_mine + (uint32_t)(c4 * 32), r);
+                        }
+                        l_run *= alpha;
+                        off_used = off_next;
+                        sum = tile_p(v, off_used, pk);
+                    }
+                    // P over the first 32 columns of the same S buffer (a thread only touches its own lane, and all of
+                    // its scores are in registers)
+                    tmem_st_32x32b_x32(lane_base + (uint32_t)(sb * kTileTok), pk);
                     tmem_st_wait();
-                    l_run *= alpha;
-                    m_used = m_next;
                 }
-                if (warp_has_rows) sum = tile_p(sb, cm0, cm1, m_used);
-                T_MARK(s_exp);
                 l_run += sum;
-                first = false;
                 // Keep in step with this group's P V barrier: a parity wait can only tell apart two consecutive
                 // phases, so a warp must never fall two completions behind it.  The P V of two tiles ago has
                 // normally long completed here.
-                if (it >= 2 && (ctrl->abort || !T_WAIT(w_pv, ptx::mbar_wait(&ctrl->pv_done[grp], ((it - 2) >> 1) & 1)))) { timeout(p, ctrl, 34); ok = false; break; }
+                if (it >= 2 && (ctrl->abort || !ptx::mbar_wait(&ctrl->pv_done[grp], ((it - 2) >> 1) & 1))) { timeout(p, ctrl, 34); ok = false; break; }
                 // P is in tensor memory (and any O rescale too): the P V of this tile may go
                 ptx::tc_fence_before();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&ctrl->p_full[sb]);
                 if (q_pending) { q_ready((seg + 1) & 1); q_pending = false; }
-                T_MARK(s_fin);
             }
             if (!ok) break;
-#ifdef MIRROR_ATTN_TIMING
-            t_loop += T_NOW() - tl;
-#endif
 
             // (This part's Q buffer is overwritten at the start of the next part.  Every Q K^T that reads it has
             // completed by then: below, each group waits for the P V of its own last tile and then meets the other;
@@ -798,28 +724,25 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             // ---- end of this CTA's part of the unit: the two groups exchange (offset, sum), then each warp
             //      combines its half of the columns of both accumulators once the last P V is complete
             float* xc = xch + (size_t)row_in_blk * 4;              // [row][group][max, sum]
-            xc[grp * 2] = m_used;
+            xc[grp * 2] = off_used;
             xc[grp * 2 + 1] = l_run;
             // each group waits for the P V of its own last tile (the barrier it has kept in step with), then the
             // groups meet: past the meeting both accumulators are complete
             {
                 const uint32_t j_last = (((it - 1) & 1) == (uint32_t)grp) ? it - 1 : it - 2;
-                if (ctrl->abort || !T_WAIT(w_end, ptx::mbar_wait(&ctrl->pv_done[grp], (j_last >> 1) & 1))) { timeout(p, ctrl, 32); ok = false; break; }
+                if (ctrl->abort || !ptx::mbar_wait(&ctrl->pv_done[grp], (j_last >> 1) & 1)) { timeout(p, ctrl, 32); ok = false; break; }
             }
             ptx::tc_fence_before();
-            if (!T_WAIT(s_ld, pair_sync())) { timeout(p, ctrl, 35); ok = false; break; }
+            if (!pair_sync()) { timeout(p, ctrl, 35); ok = false; break; }
             ptx::tc_fence_after();
             const float m_a = xc[0], l_a = xc[1], m_b = xc[2], l_b = xc[3];
-#ifdef MIRROR_ATTN_TIMING
-            te = T_NOW();
-#endif
             const bool has_b = (sg.t_last - sg.t_first) >= 2;      // did the later-starting group see any tile?
             // group of the first tile of this part: the tile counter's parity when the part began
             const int g_first = (int)((it - (uint32_t)(sg.t_last - sg.t_first)) & 1);
             const bool has0 = has_b || g_first == 0, has1 = has_b || g_first == 1;
             const float M = fmaxf(has0 ? m_a : -INFINITY, has1 ? m_b : -INFINITY);
-            const float w0 = (has0 && m_a != -INFINITY) ? exp2f((m_a - M) * p.scale_log2e) : 0.f;
-            const float w1 = (has1 && m_b != -INFINITY) ? exp2f((m_b - M) * p.scale_log2e) : 0.f;
+            const float w0 = (has0 && m_a != -INFINITY) ? exp2f(m_a - M) : 0.f;          // (offsets are in log2 units)
+            const float w1 = (has1 && m_b != -INFINITY) ? exp2f(m_b - M) : 0.f;
             const float Lsum = w0 * (has0 ? l_a : 0.f) + w1 * (has1 ? l_b : 0.f);
 
             if (warp_has_rows) {
@@ -871,7 +794,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&ctrl->o_free);
                 if (whole_unit) {
-                    if (lse_ptr && row_ok) *lse_ptr = M * p.scale + logf(Lsum);
+                    if (lse_ptr && row_ok) *lse_ptr = M * kLn2 + logf(Lsum);
                 } else {
                     // ---- the unit is cut across CTA groups: this part's (max, sum, accumulator) is left for the merge
                     //      kernel that follows; nothing here waits for another CTA
@@ -883,37 +806,18 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&ctrl->o_free);
             }
-#ifdef MIRROR_ATTN_TIMING
-            t_epi += T_NOW() - te;
-#endif
             // the exchange words are rewritten at the end of the next part: the partner must have read them
-            if (!T_WAIT(s_free, pair_sync())) { timeout(p, ctrl, 36); ok = false; break; }
+            if (!pair_sync()) { timeout(p, ctrl, 36); ok = false; break; }
             if (has_next) sg = sg_next;
         }
         asm volatile("cp.async.wait_all;" ::: "memory");      // (only an aborted run can still have copies in flight here)
-        if (warp == 4 && lane == 0) { T_STORE(8, T_NOW() - t0, w_sf, w_pv, w_end, t_epi, t_q, (long long)it); T_STORE(40, s_ld, s_free, s_max, s_xch, s_exp, s_fin); T_STORE(52, t_init, t_loop, t_max, t_ld1); }
     }
 
-#ifdef MIRROR_ATTN_TIMING
-#define T_G(i) do { if (p.timing && blockIdx.x == 5) { unsigned long long g__; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g__) :: "memory"); p.timing[680 + (i)] = (long long)g__; } } while (0)
-#else
-#define T_G(i) do { } while (0)
-#endif
-    if (lane == 0) T_G(warp);
-    if (warp == 1 && lane == 1) T_G(12);
     ptx::tc_fence_before();
     __syncthreads();
-    T_STAMP(2);
-    if (lane == 0) T_G(16 + warp);
-    if (lane == 0 && warp == 1) T_G(13);
     if (warp == 1) {
         ptx::tc_fence_after();
-        if (lane == 0) T_G(14);
         ptx::tmem_dealloc(tmem_base, kTmemCols);
-        if (lane == 0) T_G(15);
-#ifdef MIRROR_ATTN_TIMING
-        if (p.timing && lane == 0) { unsigned long long g__; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g__) :: "memory"); p.timing[64 + blockIdx.x * 4 + 3] = (long long)g__; }
-#endif
     }
 }
 
@@ -1015,7 +919,7 @@ __global__ void __launch_bounds__(kMergeThreads) attn_merge_kernel(const AttnPar
             for (int k = 0; k < parts; ++k) {
                 const float* src = part_of(k);
                 const float pm = __ldcg(src + (size_t)D * kRows);
-                const float wgt = (pm == -INFINITY) ? 0.f : exp2f((pm - Mm) * p.scale_log2e);
+                const float wgt = (pm == -INFINITY) ? 0.f : exp2f(pm - Mm);
                 Lm = fmaf(wgt, __ldcg(src + (size_t)(D + 1) * kRows), Lm);
                 if (has) {
 #pragma unroll
@@ -1028,7 +932,7 @@ __global__ void __launch_bounds__(kMergeThreads) attn_merge_kernel(const AttnPar
     for (int k = 0; k < parts; ++k) {
         const float* src = part_of(k);
         const float pm = __ldcg(src + (size_t)D * kRows);
-        const float wgt = (pm == -INFINITY) ? 0.f : exp2f((pm - Mm) * p.scale_log2e);
+        const float wgt = (pm == -INFINITY) ? 0.f : exp2f(pm - Mm);
         Lm = fmaf(wgt, __ldcg(src + (size_t)(D + 1) * kRows), Lm);
 #pragma unroll
         for (int i = 0; i < kPer; ++i)
@@ -1050,7 +954,7 @@ __global__ void __launch_bounds__(kMergeThreads) attn_merge_kernel(const AttnPar
             *reinterpret_cast<uint4*>(orow + chunk[i] * 8) = v;
         }
     if (writes_lse)
-        p.lse_out[(((size_t)u.layer * p.B + u.b) * p.Hq + u.g * p.G + hl) * p.n + node] = Mm * p.scale + logf(Lm);
+        p.lse_out[(((size_t)u.layer * p.B + u.b) * p.Hq + u.g * p.G + hl) * p.n + node] = Mm * kLn2 + logf(Lm);
 }
 
 }  // namespace
@@ -1086,12 +990,6 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
     p.k_new = (const __nv_bfloat16*)k_new; p.v_new = (const __nv_bfloat16*)v_new;
     p.out = (__nv_bfloat16*)out; p.lse_out = lse_out;
     p.partial = partial_ws; p.status = ctx->d_status;
-    p.timing = nullptr;
-    p.timing_exit = 0;
-#ifdef MIRROR_ATTN_TIMING
-    if (const char* e = getenv("MIRROR_ATTN_TIMING_PTR")) p.timing = (long long*)strtoull(e, nullptr, 0);
-    if (const char* e = getenv("MIRROR_ATTN_EXIT")) p.timing_exit = atoi(e);
-#endif
     if (p.B > kMaxBatch) return MIRROR_ERR_SHAPE;
 
     AttnTree at;
