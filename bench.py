@@ -3,14 +3,17 @@
 
 One "step" is one whole pass of the hot path over one batch of synthetic input: branch-tree attention
 for all layers -> LM head with fused reductions -> acceptance / branch selection, through the C-ABI
-call mirror_verify_step.  The workload is the 14B-shaped configuration (48 layers, prefix 2048 in
-16-token pages, kappa 4 x gamma 4, vocab 152064, greedy), which fits one GPU.
+call mirror_verify_step.  The headline workload is the largest configuration that fits one GPU, the
+66B-class one (80 layers, 16 requests with prefixes of 1024..8192 tokens in 16-token pages, kappa 8 x
+gamma 8, vocab 128256, speculative-sampling acceptance; about 31 GB on the device).  The other
+configurations are timed in the same run and reported under "workloads" (shorter loops).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload NAME]
 
 Prints ONE JSON line.  With --impl reference the CPU oracle is timed instead (a deliberately plain
 program: the ratio to it says nothing about kernel quality; parity and the roofline fraction do).
-N > 1 runs independent replicas (the path does not shard): launch under torch.distributed.run.
+N > 1 runs independent replicas (the path does not shard): bench.py starts the N ranks itself (it re-runs
+itself under torch.distributed.run on 127.0.0.1) unless it is already running under a launcher.
 """
 from __future__ import annotations
 
@@ -27,15 +30,24 @@ sys.path.insert(0, ROOT)
 
 METRIC = "verify_steps_per_sec"
 UNIT = "steps/s"
+HEADLINE = "opt66b_b16"                       # the largest single-GPU configuration
+OTHERS = ["qwen14b", "qwen14b_b8", "qwen32b_long", "paper_native"]
 
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="mirror", choices=["mirror", "reference"])
-    ap.add_argument("--workload", default="qwen14b")
+    ap.add_argument("--workload", default=HEADLINE)
+    ap.add_argument("--others", default=",".join(OTHERS),
+                    help="comma-separated workloads also timed (short loops) and reported under 'workloads'; '' for none")
+    ap.add_argument("--min-seconds", type=float, default=1.0,
+                    help="the K-step block is repeated until this much device time has been timed; the median block is reported")
+    ap.add_argument("--rendezvous-only", action="store_true",
+                    help="start the ranks, run the barrier and the max-over-ranks reduction on a dummy timing and print a "
+                         "skeleton line (gloo when there is no CUDA device): checks the launch path without a GPU")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--accept-mode", default=None, choices=["greedy", "spec_sampling", "spec_tree"],
@@ -84,13 +96,19 @@ def measured_peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1400.0, source="fallback")
 
 
-def profiled_traffic(kernel_md: str):
-    """DRAM bytes per launch of the dominant kernel from the committed ncu summary (None if absent)."""
+def profiled_traffic(kernel_md: str, scale: float = 1.0):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary (None if absent).  A summary that was
+    captured on a cut-down case says so with a line `dram_bytes_per_layer:`; it is scaled by `scale` (the layers of a
+    full launch: traffic grows in proportion to the layers, each layer has its own cache)."""
     path = os.path.join(ROOT, "profiles", kernel_md)
     if not os.path.exists(path):
         return None
-    m = re.search(r"dram_bytes_per_launch:\s*([0-9.eE+]+)", open(path).read())
-    return float(m.group(1)) if m else None
+    text = open(path).read()
+    m = re.search(r"dram_bytes_per_launch:\s*([0-9.eE+]+)", text)
+    if m:
+        return float(m.group(1))
+    m = re.search(r"dram_bytes_per_layer:\s*([0-9.eE+]+)", text)
+    return float(m.group(1)) * scale if m else None
 
 
 # ---------------------------------------------------------------------------------------------------
@@ -218,8 +236,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
             "warmup": warm, "ms_per_step": full * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f64", "data": "synthetic", "draft_tokens_per_sec": value * cfg.draft_tokens,
-            "config": {"workload": cfg.name, "kappa": cfg.kappa, "gamma": cfg.gamma, "batch": cfg.batch,
-                       "layers": cfg.layers, "prefix": [cfg.prefix_lo, cfg.prefix_hi], "vocab": cfg.vocab},
+            "config": config_dict(cfg, int(os.environ.get("WORLD_SIZE", "1"))),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle", "sample": desc,
                              "sample_seconds": sum(samples) / len(samples)},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -377,10 +394,123 @@ def target_forward_stage(m, x, tree, kv, cfg, n_layers: int, intermediate: int, 
             "kernel_launches": (m.launch_count() - l0) // reps}
 
 
+def config_dict(cfg, world: int):
+    """The `config` object of the JSON line: the same keys and values in both arms."""
+    return {"workload": cfg.name, "kappa": cfg.kappa, "gamma": cfg.gamma, "batch": cfg.batch, "layers": cfg.layers,
+            "prefix": [cfg.prefix_lo, cfg.prefix_hi], "vocab": cfg.vocab, "hidden": cfg.hidden, "accept": cfg.mode,
+            "l2": "inputs (KV cache + LM-head weights, gigabytes) are far larger than L2; no flush",
+            "parallelism": "replicas only" if world > 1 else "single GPU"}
+
+
+def stage_rooflines(work, peaks):
+    """Binding roofline of each stage (the slower of its HBM and tensor time) and of the step, in ms."""
+    attn = max(work["attn_bytes"] / peaks["hbm_gbs"] / 1e6, work["attn_flops"] / peaks["bf16_tflops"] / 1e9)
+    lm = max(work["lm_bytes"] / peaks["hbm_gbs"] / 1e6, work["lm_flops"] / peaks["bf16_tflops"] / 1e9)
+    return {"attn_ms": attn, "lmhead_ms": lm, "step_ms": attn + lm,
+            "attn_bound": "hbm" if work["attn_bytes"] / peaks["hbm_gbs"] / 1e6 >= attn else "tensor",
+            "lmhead_bound": "hbm" if work["lm_bytes"] / peaks["hbm_gbs"] / 1e6 >= lm else "tensor"}
+
+
+class Workload:
+    """One configuration resident on the device with everything a step needs."""
+
+    def __init__(self, name, args, rank, local, dev):
+        import torch
+        from paper_2510_13161_b200 import binding, inputs as I
+        cfg = I.CONFIGS[name]
+        if args.accept_mode:
+            cfg = I.shrink(cfg, mode=args.accept_mode)
+        if args.layers is not None:
+            cfg = I.shrink(cfg, layers=args.layers)
+        self.cfg = cfg
+        self.x = x = I.gen_verify_inputs(cfg, args.seed + rank, dev)          # replicas: each rank draws its own problem
+        self.m = m = binding.Mirror(cfg.hidden, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.vocab,
+                                    temperature=cfg.temperature, device=local)
+        self.kv = m.kv(x.k_pool, x.v_pool, x.page_table, x.prefix_len)
+        self.tree = m.tree(x.tokens, cfg.kappa, cfg.gamma)
+        mode = {"spec_sampling": binding.ACCEPT_SPEC_SAMPLING, "spec_tree": binding.ACCEPT_SPEC_TREE}.get(cfg.mode, binding.ACCEPT_GREEDY)
+        self.acc = m.accept_in(mode, True, q_probs=x.q_probs, u_accept=x.u_accept, u_resample=x.u_resample)
+        self.attn_out = torch.empty_like(x.q)
+        self.res = binding.AcceptResult(cfg.batch, cfg.gamma, dev)
+        self.stream = torch.cuda.current_stream()
+        self.work = algorithmic_work(cfg, x.prefix_len.cpu().tolist())
+        self.resident_gb = sum(t.numel() * t.element_size() for t in (x.k_pool, x.v_pool, x.W)) / 1e9
+
+    def step(self):
+        x = self.x
+        self.m.mirror_verify_step(self.kv, self.tree, x.q, x.k_new, x.v_new, x.hidden, x.W, self.acc, self.attn_out,
+                                  out=self.res, stream=self.stream)
+
+    def check(self, where):
+        code, detail = self.m.device_status()
+        if code != 0:
+            raise SystemExit(f"device status {code} (detail {detail}) {where} ({self.cfg.name})")
+
+
+def time_blocks(w: Workload, K: int, warmup: int, min_seconds: float, barrier, world, dev, max_blocks: int = 50):
+    """Warm-up, then blocks of exactly K steps, each bracketed by CUDA events on the launching stream (resident inputs),
+    repeated until `min_seconds` of device time has been timed.  Per-stage events ride on every step of a long step (an
+    event record between two kernels keeps the second from being scheduled early, which matters for sub-millisecond
+    steps only: there they ride on every fourth step).  Returns the median block and the stage means."""
+    import torch
+    for _ in range(max(warmup, 3)):
+        w.step()
+    barrier()
+    w.check("during warm-up")
+    # one probe block sizes the stage-event stride and the number of blocks
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(w.stream)
+    for _ in range(3):
+        w.step()
+    e1.record(w.stream)
+    torch.cuda.synchronize()
+    est_ms = e0.elapsed_time(e1) / 3
+    every = 1 if est_ms >= 1.0 else 4
+    n_blocks = int(min(max_blocks, max(1, -(-min_seconds * 1e3 // (est_ms * K)), -(-20 * every // K))))
+    stage_ev, blocks = [], []
+    launches0 = w.m.launch_count()
+    barrier()
+    for b in range(n_blocks):
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(w.stream)
+        for k in range(K):
+            if (b * K + k) % every == 0:
+                stage_ev.append([torch.cuda.Event(enable_timing=True) for _ in range(4)])
+                w.m.set_stage_events(stage_ev[-1])
+            else:
+                w.m.set_stage_events(None)
+            w.step()
+        ev1.record(w.stream)
+        blocks.append((ev0, ev1))
+    w.m.set_stage_events(None)
+    barrier()
+    launches = w.m.launch_count() - launches0
+    w.check("during the timed region")
+    block_ms = sorted(max_over_ranks(a.elapsed_time(b), dev) for a, b in blocks)
+    med = block_ms[len(block_ms) // 2]
+    mean = lambda i: sum(e[i].elapsed_time(e[i + 1]) for e in stage_ev) / len(stage_ev)
+    return {"block_ms": med, "ms_per_step": med / K, "blocks": len(block_ms), "block_ms_min": block_ms[0], "block_ms_max": block_ms[-1],
+            "attn_ms": mean(0), "lmhead_ms": mean(1), "tail_ms": mean(2), "stage_samples": len(stage_ev),
+            "launches_per_block": launches // len(block_ms)}
+
+
+def stages_of(t, work, peaks):
+    ms_step = t["ms_per_step"]
+    return {"attn_ms": t["attn_ms"], "lmhead_ms": t["lmhead_ms"], "merge_accept_ms": t["tail_ms"], "stage_samples": t["stage_samples"],
+            "attn_gbs": work["attn_bytes"] / (t["attn_ms"] * 1e-3) / 1e9,
+            "attn_frac_hbm": work["attn_bytes"] / (t["attn_ms"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+            "attn_tflops": work["attn_flops"] / (t["attn_ms"] * 1e-3) / 1e12,
+            "attn_frac_tensor": work["attn_flops"] / (t["attn_ms"] * 1e-3) / 1e12 / peaks["bf16_tflops"],
+            "lmhead_gbs": work["lm_bytes"] / (t["lmhead_ms"] * 1e-3) / 1e9,
+            "lmhead_tflops": work["lm_flops"] / (t["lmhead_ms"] * 1e-3) / 1e12,
+            "lmhead_frac_tensor": work["lm_flops"] / (t["lmhead_ms"] * 1e-3) / 1e12 / peaks["bf16_tflops"],
+            "step_hbm_frac": (work["attn_bytes"] + work["lm_bytes"]) / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+
+
 def run_mirror(args):
     import torch
     import torch.distributed as dist
-    from paper_2510_13161_b200 import binding, inputs as I
+    from paper_2510_13161_b200 import inputs as I
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -392,150 +522,182 @@ def run_mirror(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dev = torch.device("cuda", local)
 
-    cfg = I.CONFIGS[args.workload]
-    if args.accept_mode:
-        cfg = I.shrink(cfg, mode=args.accept_mode)
-    if args.layers is not None:
-        cfg = I.shrink(cfg, layers=args.layers)
-    x = I.gen_verify_inputs(cfg, args.seed + rank, dev)          # replicas: each rank draws its own problem
-    m = binding.Mirror(cfg.hidden, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.vocab, temperature=cfg.temperature,
-                       device=local)
-    kv = m.kv(x.k_pool, x.v_pool, x.page_table, x.prefix_len)
-    tree = m.tree(x.tokens, cfg.kappa, cfg.gamma)
-    mode = {"spec_sampling": binding.ACCEPT_SPEC_SAMPLING, "spec_tree": binding.ACCEPT_SPEC_TREE}.get(cfg.mode, binding.ACCEPT_GREEDY)
-    acc = m.accept_in(mode, True, q_probs=x.q_probs, u_accept=x.u_accept, u_resample=x.u_resample)
-    attn_out = torch.empty_like(x.q)
-    res = binding.AcceptResult(cfg.batch, cfg.gamma, dev)
-    stream = torch.cuda.current_stream()
-
-    def step():
-        m.mirror_verify_step(kv, tree, x.q, x.k_new, x.v_new, x.hidden, x.W, acc, attn_out, out=res, stream=stream)
-
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
-        step()
-    barrier()
-    code, detail = m.device_status()
-    if code != 0:
-        raise SystemExit(f"device status {code} (detail {detail}) during warm-up")
-
-    # ---- timed region: K steps, resident inputs, CUDA events on the launching stream; per-stage events ride along
+    peaks = measured_peaks()
+    w = Workload(args.workload, args, rank, local, dev)
+    cfg, x, m = w.cfg, w.x, w.m
     K = args.steps
-    # (an event record between two kernels also keeps the second from being scheduled early, so the per-stage events
-    # ride on every eighth step only; ev0 / ev1 bracket all K steps)
-    EVERY = 8
-    stage_ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range((K + EVERY - 1) // EVERY)]
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    # ---- timed region: blocks of K steps, resident inputs, CUDA events on the launching stream, clocks sampled throughout
     sampler = ClockSampler(local)
-    launches0 = m.launch_count()
-    barrier()
     sampler.start()
-    ev0.record(stream)
-    for k in range(K):
-        m.set_stage_events(stage_ev[k // EVERY] if k % EVERY == 0 else None)
-        step()
-    ev1.record(stream)
-    m.set_stage_events(None)
-    barrier()
+    t = time_blocks(w, K, args.warmup, args.min_seconds, barrier, world, dev)
     clocks = sampler.stop()
-    launches = m.launch_count() - launches0
-    ms_total = max_over_ranks(ev0.elapsed_time(ev1), dev)
-    ms_step = ms_total / K
-    value = job_throughput(K, world, ms_total)
-    attn_ms = sum(e[0].elapsed_time(e[1]) for e in stage_ev) / len(stage_ev)
-    lm_ms = sum(e[1].elapsed_time(e[2]) for e in stage_ev) / len(stage_ev)
-    tail_ms = sum(e[2].elapsed_time(e[3]) for e in stage_ev) / len(stage_ev)
-    code, detail = m.device_status()
-    if code != 0:
-        raise SystemExit(f"device status {code} (detail {detail}) during the timed region")
+    ms_step = t["ms_per_step"]
+    value = job_throughput(K, world, t["block_ms"])
 
     # ---- end to end: per step, this step's inputs come from pinned host memory and the decision goes back
+    from paper_2510_13161_b200 import binding
     h_in = {k: getattr(x, k).cpu().pin_memory() for k in ("q", "k_new", "v_new", "tokens")}
     d_in = {k: torch.empty_like(getattr(x, k)) for k in h_in}
     tree_e = m.tree(d_in["tokens"], cfg.kappa, cfg.gamma)
-    h_out = {k: torch.empty_like(getattr(res, k), device="cpu").pin_memory() for k in ("n_accepted", "n_emitted", "emitted", "best_branch")}
+    h_out = {k: torch.empty_like(getattr(w.res, k), device="cpu").pin_memory() for k in ("n_accepted", "n_emitted", "emitted", "best_branch")}
     h2d = sum(v.numel() * v.element_size() for v in h_in.values())
     d2h = sum(v.numel() * v.element_size() for v in h_out.values())
 
     def e2e_step():
         # one C-ABI call with host buffers: it copies this step's inputs in on its own stream, piece by piece, runs the
         # step and copies the decision back
-        m.mirror_verify_step_host(kv, tree_e, h_in, d_in, x.hidden, x.W, acc, attn_out, res, h_out=h_out, stream=stream)
-        stream.synchronize()      # the caller needs the decision before it can build the next step
+        m.mirror_verify_step_host(w.kv, tree_e, h_in, d_in, x.hidden, x.W, w.acc, w.attn_out, w.res, h_out=h_out, stream=w.stream)
+        w.stream.synchronize()      # the caller needs the decision before it can build the next step
 
     e2e_value = None
     if not args.skip_e2e:
         for _ in range(3):
             e2e_step()
-        Ke = max(10, min(K, 200))
+        Ke = max(5, min(K, 200))
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
+        e0.record(w.stream)
         for _ in range(Ke):
             e2e_step()
-        e1.record(stream)
+        e1.record(w.stream)
         barrier()
         e2e_value = job_throughput(Ke, world, max_over_ranks(e0.elapsed_time(e1), dev))
+        w.check("in the end-to-end loop")
+    del h_in, d_in, tree_e
+
+    work = w.work
+    stages = stages_of(t, work, peaks)
+    rl = stage_rooflines(work, peaks)
+    stages["roofline_ms"] = rl
+    stages["step_frac_of_binding_roofline"] = rl["step_ms"] / ms_step
+    # the dominant kernel of the step and the roofline that binds it
+    if t["attn_ms"] >= t["lmhead_ms"]:
+        tensor = rl["attn_bound"] == "tensor"
+        ach = stages["attn_tflops"] if tensor else stages["attn_gbs"]
+        roofline = {"kernel": "attn_verify_kernel", "bound": "tensor" if tensor else "hbm", "achieved": ach,
+                    "peak": peaks["bf16_tflops"] if tensor else peaks["hbm_gbs"], "unit": "TFLOP/s" if tensor else "GB/s",
+                    "frac": ach / (peaks["bf16_tflops"] if tensor else peaks["hbm_gbs"]), "peak_source": peaks["source"] + (" (sustained bf16)" if tensor else " (copy)"),
+                    "traffic": profiled_traffic(f"attn_verify_kernel_{cfg.name}.md", scale=cfg.layers),
+                    "algorithmic_flops_per_launch": work["attn_flops"], "algorithmic_bytes_per_launch": work["attn_bytes"],
+                    "ms_per_launch": t["attn_ms"], "note": "ms_per_launch covers the attention stage (the main kernel and the small merge kernel behind it)"}
+    else:
+        tensor = rl["lmhead_bound"] == "tensor"
+        ach = stages["lmhead_tflops"] if tensor else stages["lmhead_gbs"]
+        roofline = {"kernel": "lmhead_pair_kernel", "bound": "tensor" if tensor else "hbm", "achieved": ach,
+                    "peak": peaks["bf16_tflops"] if tensor else peaks["hbm_gbs"], "unit": "TFLOP/s" if tensor else "GB/s",
+                    "frac": ach / (peaks["bf16_tflops"] if tensor else peaks["hbm_gbs"]), "peak_source": peaks["source"] + (" (sustained bf16)" if tensor else " (copy: a read + write stream; a read-only weight stream can read slightly above it)"),
+                    "traffic": profiled_traffic(f"lmhead_pair_kernel_{cfg.name}.md"),
+                    "algorithmic_flops_per_launch": work["lm_flops"], "algorithmic_bytes_per_launch": work["lm_bytes"],
+                    "ms_per_launch": t["lmhead_ms"]}
+
+    # ---- optional extra stages (outside the timed region)
+    if args.attn_per_layer:
+        stages["attn_per_layer_ms"] = attn_per_layer(m, x, w.tree, cfg)
+    if args.overlap_draft:
+        stages["overlap_draft"] = overlap_draft_stage(w.step, w.stream)
+    if args.target_layers > 0:
+        stages["target_forward"] = target_forward_stage(m, x, w.tree, w.kv, cfg, min(args.target_layers, cfg.layers), args.intermediate,
+                                                        peaks["hbm_gbs"])
+
+    headline = {"ms_per_step": ms_step, "steps_per_sec": value, "draft_tokens_per_sec": value * cfg.draft_tokens,
+                "attn_ms": t["attn_ms"], "lmhead_ms": t["lmhead_ms"], "merge_accept_ms": t["tail_ms"],
+                "roofline_step_ms": rl["step_ms"], "frac_of_binding_roofline": rl["step_ms"] / ms_step,
+                "attn_bound": rl["attn_bound"], "lmhead_bound": rl["lmhead_bound"], "step_hbm_frac": stages["step_hbm_frac"],
+                "attn_frac": rl["attn_ms"] / t["attn_ms"], "lmhead_frac": rl["lmhead_ms"] / t["lmhead_ms"]}
+    resident_gb = w.resident_gb
+    del w, x, m
+    torch.cuda.empty_cache()
+
+    # ---- the other configurations, one after the other (shorter loops; same step, same events)
+    workloads = {cfg.name: headline}
+    for name in [n for n in args.others.split(",") if n and n != cfg.name]:
+        wo = Workload(name, args, rank, local, dev)
+        to = time_blocks(wo, K, 3, min(args.min_seconds, 0.3), barrier, world, dev, max_blocks=20)
+        ro = stage_rooflines(wo.work, peaks)
+        so = stages_of(to, wo.work, peaks)
+        vo = job_throughput(K, world, to["block_ms"])
+        workloads[name] = {"ms_per_step": to["ms_per_step"], "steps_per_sec": vo, "draft_tokens_per_sec": vo * wo.cfg.draft_tokens,
+                           "attn_ms": to["attn_ms"], "lmhead_ms": to["lmhead_ms"], "merge_accept_ms": to["tail_ms"],
+                           "roofline_step_ms": ro["step_ms"], "frac_of_binding_roofline": ro["step_ms"] / to["ms_per_step"],
+                           "attn_bound": ro["attn_bound"], "lmhead_bound": ro["lmhead_bound"], "step_hbm_frac": so["step_hbm_frac"],
+                           "attn_frac": ro["attn_ms"] / to["attn_ms"], "lmhead_frac": ro["lmhead_ms"] / to["lmhead_ms"],
+                           "blocks": to["blocks"]}
+        del wo
+        torch.cuda.empty_cache()
 
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    work = algorithmic_work(cfg, x.prefix_len.cpu().tolist())
-    peaks = measured_peaks()
-    lm_gbs = work["lm_bytes"] / (lm_ms * 1e-3) / 1e9
-    attn_gbs = work["attn_bytes"] / (attn_ms * 1e-3) / 1e9
-    roofline = {"kernel": "lmhead_pair_kernel", "bound": "hbm", "achieved": lm_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": lm_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                "traffic": profiled_traffic("lmhead_pair_kernel_qwen14b.md"),
-                "algorithmic_bytes_per_launch": work["lm_bytes"], "ms_per_launch": lm_ms}
-    stages = {"attn_ms": attn_ms, "lmhead_ms": lm_ms, "merge_accept_ms": tail_ms,
-              "attn_gbs": attn_gbs, "attn_frac_hbm": attn_gbs / peaks["hbm_gbs"],
-              "attn_tflops": work["attn_flops"] / (attn_ms * 1e-3) / 1e12,
-              "lmhead_tflops": work["lm_flops"] / (lm_ms * 1e-3) / 1e12,
-              "step_hbm_frac": (work["attn_bytes"] + work["lm_bytes"]) / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"]}
-
-    # ---- attention with one launch pair per layer: the order a real target enforces (layer l+1's queries depend on
-    # layer l's output), as plain stream-ordered launches and replayed from a CUDA graph.  Outside the timed region.
-    if args.attn_per_layer:
-        stages["attn_per_layer_ms"] = attn_per_layer(m, x, tree, cfg)
-    if args.overlap_draft:
-        stages["overlap_draft"] = overlap_draft_stage(step, stream)
-    if args.target_layers > 0:
-        stages["target_forward"] = target_forward_stage(m, x, tree, kv, cfg, min(args.target_layers, cfg.layers), args.intermediate,
-                                                        peaks["hbm_gbs"])
-
     cpu = None
     if not args.no_cpu_baseline and world == 1:
         from oracle import oracle as O
         xs = I.gen_verify_inputs(cfg, args.seed, "cpu", layers=1, force_hidden=cfg.explicit_hidden)
-        s, full, desc = oracle_sample_seconds(xs, cfg)
+        sec, full, desc = oracle_sample_seconds(xs, cfg)
         cpu = {"value": 1.0 / full, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle", "sample": desc,
-               "sample_seconds": s}
+               "sample_seconds": sec}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic", "draft_tokens_per_sec": value * cfg.draft_tokens,
-            "config": {"workload": cfg.name, "kappa": cfg.kappa, "gamma": cfg.gamma, "batch": cfg.batch, "layers": cfg.layers,
-                       "prefix": [cfg.prefix_lo, cfg.prefix_hi], "vocab": cfg.vocab, "hidden": cfg.hidden, "accept": cfg.mode,
-                       "l2": "inputs (KV cache + LM-head weights, about 2 GB) are larger than L2; no flush",
-                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "timing": {"blocks": t["blocks"], "steps_per_block": K, "block_ms_median": t["block_ms"], "block_ms_min": t["block_ms_min"],
+                       "block_ms_max": t["block_ms_max"], "value_from": "median block"},
+            "config": config_dict(cfg, world), "resident_gb": resident_gb,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "resident": "KV cache and LM-head weights stay on the device; Q, tree K/V and tokens are copied every step"},
-            "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "stages": stages, "cpu_baseline": cpu}
+                    "resident": "KV cache and LM-head weights (and, for stochastic acceptance, the draft distributions) stay on the "
+                                "device; Q of every layer, the tree's K/V and the tokens are inputs of the synthetic step and are "
+                                "copied every step: Q dominates the copies"},
+            "gpu_launches": t["launches_per_block"], "clocks": clocks, "roofline": roofline, "stages": stages, "workloads": workloads,
+            "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
 
 
+def rendezvous_only(args):
+    """The launch path without the GPU work: process group (nccl with a CUDA device, gloo without), barrier, max-over-ranks of a
+    dummy per-rank time, and a skeleton line from rank 0."""
+    import torch
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("nccl" if torch.cuda.is_available() else "gloo")
+        dist.barrier()
+    ms = max_over_ranks(10.0 + 5.0 * rank, torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0"))) if torch.cuda.is_available() else None)
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "rendezvous_only": True, "n_gpus": world, "requested_gpus": args.gpus, "ms_max": ms,
+                          "value": job_throughput(args.steps, world, ms), "unit": UNIT}), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def spawn_ranks(args) -> int:
+    """--gpus N without a launcher: run this script again under torch.distributed.run with N ranks on this node."""
+    import socket
+    import subprocess
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     args = parse_args()
-    if args.impl == "reference":
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args))
+    if args.rendezvous_only:
+        rendezvous_only(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_mirror(args)

@@ -50,3 +50,20 @@ def test_single_process_is_identity():
     import bench
     assert bench.max_over_ranks(3.5) == 3.5
     assert bench.job_throughput(10, 1, 5.0) == 2000.0
+
+
+def test_bench_starts_its_own_ranks_when_no_launcher_did():
+    """`python bench.py --gpus 2` with no WORLD_SIZE in the environment re-runs itself under torch.distributed.run on
+    127.0.0.1; the launch path (process group, barrier, max over ranks, one line from rank 0) is checked without a GPU."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "20", "--rendezvous-only"],
+                       capture_output=True, text=True, env=env, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                         # rank 0 alone prints
+    line = lines[0]
+    assert line["n_gpus"] == 2 and line["requested_gpus"] == 2
+    assert line["ms_max"] == 15.0                                   # the slower rank's time
+    assert abs(line["value"] - 2 * 20 * 1e3 / 15.0) < 1e-9
