@@ -178,8 +178,8 @@ mirror_status mirror_lmhead_reduce(mirror_ctx* ctx, const void* hidden, int M, c
  * (the paper has no counterpart: this is a deployment variant of mirror_lmhead_reduce, same kernels).
  * Who needs it: a host that has given all device memory to its own pool, a plugin called inside an
  * allocator-guarded region, or any code path where cudaMalloc is forbidden.  No context and no workspace:
- * the kernel's scratch (one partial per CTA and row) is a fixed array inside the library image, 393,472
- * bytes on every GPU that loads the library, held until the process exits.
+ * the kernel's scratch (one partial per CTA and row, two CTAs per SM) is a fixed array inside the library image,
+ * 491,776 bytes on every GPU that loads the library, held until the process exits.
  *   device       CUDA device ordinal (made current for the call)
  *   hidden, W    bf16 [M, H] and [V, H] as in mirror_lmhead_reduce; H a multiple of 64
  *   M            at most 128 rows; more returns MIRROR_ERR_SHAPE (use mirror_lmhead_reduce with a workspace)
@@ -189,10 +189,18 @@ mirror_status mirror_lmhead_reduce(mirror_ctx* ctx, const void* hidden, int M, c
  * scratch array's device address (cudaGetSymbolAddress) and the tensor-map encoder; make that first call
  * before any stream capture begins.  Every call on a device shares the one scratch array: calls that
  * overlap on the GPU (different streams, no ordering) race on it and give wrong results -- order them.
- * The call clears the status words it needs on `stream`; the rest of the array is rewritten before it is read. */
+ * The partials are rewritten by every call before they are read.  A device-side problem (a bounded wait that ran
+ * out) is recorded in the array's first words and kept until mirror_lmhead_noalloc_status asks for it; the
+ * outputs of such a call are not valid.  The one-time set-up is guarded, so first calls may come from any thread. */
 mirror_status mirror_lmhead_reduce_noalloc(int device, const void* hidden, int M, const void* W, int V, int H,
                                            float temperature, int32_t* argmax, float* maxlogit, float* lse,
                                            void* stream);
+
+/* Device-side status of the mirror_lmhead_reduce_noalloc calls made on `device` (they have no context to ask;
+ * the paper has no counterpart): synchronises the device, returns in *code the first problem since the last query
+ * (MIRROR_OK, MIRROR_ERR_TIMEOUT or MIRROR_ERR_DEVICE_CHECK) with a detail word in *detail (nullable), and clears it.
+ * Allocates nothing. */
+mirror_status mirror_lmhead_noalloc_status(int device, int* code, int* detail);
 
 /* Acceptance, branch selection, emitted tokens and reuse lookup (a5 + a6).
  * Greedy (Eq. 3 / Eq. 10): branch length a = number of leading nodes c with tokens[c] == target_argmax[parent(c)].

@@ -24,7 +24,7 @@ EXPORTS = [
     "mirror_create", "mirror_destroy", "mirror_workspace_bytes", "mirror_set_workspace",
     "mirror_attn_verify", "mirror_lmhead_reduce", "mirror_accept_select", "mirror_verify_step",
     "mirror_device_status", "mirror_launch_count", "mirror_status_str", "mirror_set_stage_events",
-    "mirror_lmhead_reduce_noalloc", "mirror_early_exit_tap", "mirror_overlap_mass", "mirror_kv_commit",
+    "mirror_lmhead_reduce_noalloc", "mirror_lmhead_noalloc_status", "mirror_early_exit_tap", "mirror_overlap_mass", "mirror_kv_commit",
     "mirror_linear_scratch_bytes", "mirror_linear", "mirror_rmsnorm", "mirror_target_scratch_bytes", "mirror_target_forward", "mirror_trie_build", "mirror_verify_step_host", "mirror_embed_rows",
 ]
 
@@ -155,6 +155,14 @@ def mirror_lmhead_reduce_noalloc(hidden: torch.Tensor, W: torch.Tensor, temperat
                                             _ptr(maxlogit, torch.float32, "maxlogit"), _ptr(lse, torch.float32, "lse"),
                                             _stream(stream)), "mirror_lmhead_reduce_noalloc")
     return dict(argmax=argmax, maxlogit=maxlogit, lse=lse)
+
+
+def mirror_lmhead_noalloc_status(device: int = 0):
+    """(code, detail) of the first device-side problem of the no-allocation LM-head calls on `device` since the last
+    query (synchronises the device; (0, 0) when there was none)."""
+    code, detail = C.c_int(), C.c_int()
+    _check(load_library().mirror_lmhead_noalloc_status(int(device), C.byref(code), C.byref(detail)), "mirror_lmhead_noalloc_status")
+    return code.value, detail.value
 
 
 class AcceptResult:

@@ -83,6 +83,8 @@ struct AttnParams {
     float* lse_out;
     float* partial;                       // [grid][2][D+4][128]
     int* status;
+    long long wait_limit;                 // SM cycles after which a wait gives up
+    int stall_after;                      // test aid: the K producer stops after this many stages (-1: never)
 };
 
 struct UnitPos {                          // where a global tile index falls
@@ -392,11 +394,12 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 }
             }
             for (int t = sg.t_first; t < sg.t_last && ok; ++t, ++x, ++it) {
+                if (!vrole && p.stall_after >= 0 && (int)it >= p.stall_after) { x = x_end; break; }      // (test aid: see AttnParams)
                 const int st = vrole ? (int)(it % VS) : (int)(it % KR);
                 const uint32_t ph = (vrole ? it / VS : it / KR) & 1;
                 const int next_page = (t + 1 < sg.t_last) ? fetch_page(t + 1) : 0;
                 bool w = true;
-                if (lane == 0) w = !ctrl->abort && ptx::mbar_wait(&empty[st], ph ^ 1);
+                if (lane == 0) w = !ctrl->abort && ptx::mbar_wait(&empty[st], ph ^ 1, p.wait_limit);
                 w = __shfl_sync(0xffffffffu, w, 0);
                 if (!w) { if (lane == 0) timeout(p, ctrl, 10); ok = false; break; }
                 uint8_t* dst = (vrole ? sV : sK) + (size_t)st * C::kStageBytes;
@@ -476,15 +479,15 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             long long x = x_begin;
             while (x < x_end && ok) {
                 const Segment sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
-                if (ctrl->abort || !ptx::mbar_wait(&ctrl->q_full[seg & 1], (seg >> 1) & 1)) { timeout(p, ctrl, 20); ok = false; break; }
+                if (ctrl->abort || !ptx::mbar_wait(&ctrl->q_full[seg & 1], (seg >> 1) & 1, p.wait_limit)) { timeout(p, ctrl, 20); ok = false; break; }
                 const uint32_t q_seg = q_lo + (uint32_t)(((seg & 1) * q_buf_bytes) >> 4);
                 ++seg;
                 // one tile (a ring stage of four slots) per issue: each S buffer is scored as soon as the P V that read
                 // it has completed, so the two softmax groups run half a period apart instead of in step
                 for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
                     const int st = it % KR, sb = it & (kSBufs - 1);
-                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->k_full[st], (it / KR) & 1) ||
-                        !ptx::mbar_wait(&ctrl->s_free[sb], ((it / kSBufs) & 1) ^ 1)) { timeout(p, ctrl, 21); ok = false; break; }
+                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->k_full[st], (it / KR) & 1, p.wait_limit) ||
+                        !ptx::mbar_wait(&ctrl->s_free[sb], ((it / kSBufs) & 1) ^ 1, p.wait_limit)) { timeout(p, ctrl, 21); ok = false; break; }
                     ptx::tc_fence_after();
                     const int n_sl = min(kStageSlots, sg.slots_all - t * kStageSlots);       // (a pair's second tile may be empty)
                     if (n_sl > 0) {
@@ -515,12 +518,12 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             while (x < x_end && ok) {
                 const Segment sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
                 // the accumulators of the previous part must have been read out by every softmax warp
-                if (seg > 0 && (ctrl->abort || !ptx::mbar_wait(&ctrl->o_free, (seg - 1) & 1))) { timeout(p, ctrl, 24); ok = false; break; }
+                if (seg > 0 && (ctrl->abort || !ptx::mbar_wait(&ctrl->o_free, (seg - 1) & 1, p.wait_limit))) { timeout(p, ctrl, 24); ok = false; break; }
                 ++seg;
                 for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
                     const int st = it % VS, pb = it & 1, sb = it & (kSBufs - 1);
-                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->p_full[sb], (it / kSBufs) & 1) ||
-                        !ptx::mbar_wait(&ctrl->v_full[st], (it / VS) & 1)) {
+                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->p_full[sb], (it / kSBufs) & 1, p.wait_limit) ||
+                        !ptx::mbar_wait(&ctrl->v_full[st], (it / VS) & 1, p.wait_limit)) {
                         timeout(p, ctrl, 23); ok = false; break;
                     }
                     ptx::tc_fence_after();
@@ -562,7 +565,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         auto pair_sync = [&]() -> bool {
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&ctrl->pair[w4]);
-            const bool r = !ctrl->abort && ptx::mbar_wait(&ctrl->pair[w4], xph);
+            const bool r = !ctrl->abort && ptx::mbar_wait(&ctrl->pair[w4], xph, p.wait_limit);
             xph ^= 1;
             return r;
         };
@@ -634,7 +637,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
                 if ((int)(it & 1) != grp) continue;
                 const int sb = it & (kSBufs - 1);
-                if (ctrl->abort || !ptx::mbar_wait(&ctrl->s_full[sb], (it / kSBufs) & 1)) { timeout(p, ctrl, 30); ok = false; break; }
+                if (ctrl->abort || !ptx::mbar_wait(&ctrl->s_full[sb], (it / kSBufs) & 1, p.wait_limit)) { timeout(p, ctrl, 30); ok = false; break; }
                 ptx::tc_fence_after();
                 float sum = 0.f;
                 // visibility of this tile's columns for this row: all ones except in a unit's last pairs
@@ -677,7 +680,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     const bool grow = !(sum <= kSumLimit);
                     if (__any_sync(0xffffffffu, grow)) {
                         // this group's last P V (two tiles ago) must be complete before its accumulator is touched
-                        if (it >= 2 && (ctrl->abort || !ptx::mbar_wait(&ctrl->pv_done[grp], ((it - 2) >> 1) & 1))) { timeout(p, ctrl, 33); ok = false; break; }
+                        if (it >= 2 && (ctrl->abort || !ptx::mbar_wait(&ctrl->pv_done[grp], ((it - 2) >> 1) & 1, p.wait_limit))) { timeout(p, ctrl, 33); ok = false; break; }
                         ptx::tc_fence_after();
                         const float off_next = grow ? tile_max(v) * p.scale_log2e - kOffsetBias : off_used;
                         const float alpha = grow ? exp2f(off_used - off_next) : 1.f;
@@ -703,7 +706,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 // Keep in step with this group's P V barrier: a parity wait can only tell apart two consecutive
                 // phases, so a warp must never fall two completions behind it.  The P V of two tiles ago has
                 // normally long completed here.
-                if (it >= 2 && (ctrl->abort || !ptx::mbar_wait(&ctrl->pv_done[grp], ((it - 2) >> 1) & 1))) { timeout(p, ctrl, 34); ok = false; break; }
+                if (it >= 2 && (ctrl->abort || !ptx::mbar_wait(&ctrl->pv_done[grp], ((it - 2) >> 1) & 1, p.wait_limit))) { timeout(p, ctrl, 34); ok = false; break; }
                 // P is in tensor memory (and any O rescale too): the P V of this tile may go
                 ptx::tc_fence_before();
                 __syncwarp();
@@ -730,7 +733,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             // groups meet: past the meeting both accumulators are complete
             {
                 const uint32_t j_last = (((it - 1) & 1) == (uint32_t)grp) ? it - 1 : it - 2;
-                if (ctrl->abort || !ptx::mbar_wait(&ctrl->pv_done[grp], (j_last >> 1) & 1)) { timeout(p, ctrl, 32); ok = false; break; }
+                if (ctrl->abort || !ptx::mbar_wait(&ctrl->pv_done[grp], (j_last >> 1) & 1, p.wait_limit)) { timeout(p, ctrl, 32); ok = false; break; }
             }
             ptx::tc_fence_before();
             if (!pair_sync()) { timeout(p, ctrl, 35); ok = false; break; }
@@ -969,19 +972,18 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
     p.n_rb = (p.rows + kRows - 1) / kRows;
     p.rows_per_rb = (p.rows + p.n_rb - 1) / p.n_rb;
     p.n_groups = ctx->num_sms / p.n_rb;
-    if (const char* e = getenv("MIRROR_ATTN_GROUPS")) { const int g = atoi(e); if (g >= 1 && g <= p.n_groups) p.n_groups = g; }
+    if (ctx->tune.attn_groups >= 1 && ctx->tune.attn_groups <= p.n_groups) p.n_groups = ctx->tune.attn_groups;
     if (p.n_groups < 1) return MIRROR_ERR_SHAPE;
-    p.snap_cap = 4;
-    p.whole_units = 1;
-    if (const char* e = getenv("MIRROR_ATTN_WHOLE_UNITS")) p.whole_units = atoi(e) != 0;
-    if (const char* e = getenv("MIRROR_ATTN_SNAP")) { p.snap_cap = atoi(e); if (p.snap_cap < 0) p.snap_cap = 0; }
+    p.snap_cap = ctx->tune.attn_snap;
+    p.whole_units = ctx->tune.attn_whole_units;
+    p.wait_limit = ctx->tune.wait_limit_cycles;
+    p.stall_after = (ctx->tune.test_stall_after >= 0 && ctx->tune.test_stall_attn_left-- > 0) ? ctx->tune.test_stall_after : -1;
     p.max_pages = kv->max_pages_per_req; p.num_pages = kv->num_pages;
     const int64_t page_elems = (int64_t)Hkv * kSlotTok * D;
     if (kv->layer_stride % page_elems != 0) return MIRROR_ERR_UNSUPPORTED;
     p.layer_pages = (int)(kv->layer_stride / page_elems);
     p.tree_slots = (p.n + kSlotTok - 1) / kSlotTok;
     p.q_half_bytes = ((p.rows_per_rb + 7) / 8) * 8 * 128;
-    if (getenv("MIRROR_ATTN_QFULL")) p.q_half_bytes = kRows * 128;
     p.scale = ctx->scale;
     p.scale_log2e = ctx->scale * 1.4426950408889634f;
     p.page_table = kv->page_table; p.prefix_len = kv->prefix_len;
@@ -1017,7 +1019,7 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
         int ks = 4, vs = 4;
         if (C::smem_bytes(p.q_half_bytes, 6, 4) <= kSmemLimit) ks = 6;
         if (C::smem_bytes(p.q_half_bytes, 6, 6) <= kSmemLimit) vs = 6;
-        if (const char* e = getenv("MIRROR_ATTN_RING")) { const int r = atoi(e); ks = r / 10; vs = r % 10; }
+        if (ctx->tune.attn_ring) { ks = ctx->tune.attn_ring / 10; vs = ctx->tune.attn_ring % 10; }
         if (!((ks == 4 || ks == 6) && (vs == 4 || (vs == 6 && ks == 6)))) return MIRROR_ERR_ARG;
         const size_t smem = C::smem_bytes(p.q_half_bytes, ks, vs);
         if (smem > kSmemLimit) return MIRROR_ERR_UNSUPPORTED;

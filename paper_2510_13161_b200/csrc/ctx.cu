@@ -1,4 +1,5 @@
 // Context, argument digests (token tree), workspace carving, tensor maps, status plumbing.
+#include <stdlib.h>
 #include <string.h>
 
 #include <new>
@@ -38,6 +39,7 @@ extern "C" mirror_status mirror_create(mirror_ctx** out, const mirror_model_desc
     mirror_ctx* ctx = new (std::nothrow) mirror_ctx();
     if (!ctx) return MIRROR_ERR_ARG;
     ctx->desc = *desc;
+    mirror_tuning_from_env(&ctx->tune);
     ctx->device = device;
     ctx->num_sms = prop.multiProcessorCount;
     ctx->scale = desc->softmax_scale > 0.f ? desc->softmax_scale : 1.0f / sqrtf((float)desc->head_dim);
@@ -56,6 +58,24 @@ extern "C" mirror_status mirror_create(mirror_ctx** out, const mirror_model_desc
     }
     *out = ctx;
     return MIRROR_OK;
+}
+
+void mirror_tuning_from_env(MirrorTuning* t) {
+    auto geti = [](const char* name, int* v, int lo, int hi) {
+        if (const char* e = getenv(name)) { const long x = strtol(e, nullptr, 10); if (x >= lo && x <= hi) *v = (int)x; }
+    };
+    geti("MIRROR_ATTN_GROUPS", &t->attn_groups, 1, 1 << 20);
+    geti("MIRROR_ATTN_WHOLE_UNITS", &t->attn_whole_units, 0, 1);
+    geti("MIRROR_ATTN_SNAP", &t->attn_snap, 0, 1 << 20);
+    geti("MIRROR_ATTN_RING", &t->attn_ring, 44, 66);
+    geti("MIRROR_LM_PAIR2_MAX_ROWS", &t->lm_pair2_max_rows, 0, 128);
+    geti("MIRROR_LM_CTAS_PER_SM", &t->lm_ctas_per_sm, 1, 2);
+    geti("MIRROR_LM_STAGES", &t->lm_stages, 2, 64);
+    geti("MIRROR_LM_ROWS", &t->lm_rows, 8, 128);
+    geti("MIRROR_LM_PAIR_MIN_ROWS", &t->lm_pair_min_rows, 0, 1 << 30);
+    geti("MIRROR_LM_KGROUP", &t->lm_kgroup, 1, 64);
+    geti("MIRROR_TEST_STALL_AFTER_STAGES", &t->test_stall_after, 0, 1 << 30);
+    if (const char* e = getenv("MIRROR_WAIT_LIMIT_CYCLES")) { const long long x = strtoll(e, nullptr, 10); if (x >= 1000) t->wait_limit_cycles = x; }
 }
 
 extern "C" mirror_status mirror_destroy(mirror_ctx* ctx) {

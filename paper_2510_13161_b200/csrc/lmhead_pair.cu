@@ -54,7 +54,8 @@ struct PairParams {
     int* part_idx;
     float* part_sum;
     int* status;
-    long long* timing;                      // developer aid (timing builds): per-CTA start / end stamps
+    long long wait_limit;                   // SM cycles after which a wait gives up
+    int stall_after;                        // test aid: the producers stop after this many stages (-1: never)
 };
 
 struct Ctrl {
@@ -159,9 +160,6 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
     const uint32_t rank = cluster_rank();
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     const int n_kb = p.H / kBK;
-#ifdef MIRROR_ATTN_TIMING
-    if (p.timing && tid == 0) { unsigned long long g__; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g__) :: "memory"); p.timing[blockIdx.x * 2] = (long long)g__; }
-#endif
     // unit -> (vocabulary tile, K slice, row chunk); chunk fastest, so the chunks of a tile run side by side
     auto decode = [&](int u, int& tile, int& slice, int& chunk) {
         chunk = u % p.n_chunks;
@@ -198,7 +196,7 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
         if (lane == 0) {
             const uint64_t pol_w = p.w_keep ? ptx::policy_evict_normal() : ptx::policy_evict_first();
             const uint64_t pol_h = ptx::policy_evict_last();
-            int s = 0;
+            int s = 0, n_issued = 0;
             uint32_t ph = 0;
             bool ok = true;
             for (int u = pair; u < p.n_units && ok; u += n_pairs) {
@@ -208,12 +206,14 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
                 const int h_row = chunk * p.chunk_rows + (int)rank * p.half_rows;
                 const int kb_end = min(n_kb, (slice + 1) * p.kb_per_slice);
                 for (int kb = slice * p.kb_per_slice; kb < kb_end; ++kb) {
-                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->empty[s], ph ^ 1)) { fail(p, ctrl, 11); ok = false; break; }
+                    if (p.stall_after >= 0 && n_issued >= p.stall_after) { ok = false; break; }       // (test aid: neither arms nor copies)
+                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->empty[s], ph ^ 1, p.wait_limit)) { fail(p, ctrl, 11); ok = false; break; }
                     if (rank == 0) ptx::mbar_arrive_expect_tx(&ctrl->full[s], 2u * (uint32_t)p.stage_bytes);
                     const uint32_t bar = map_to_rank(&ctrl->full[s], 0);
                     uint8_t* dst = stage_base + s * p.stage_bytes;
                     tma_load_2d_pair(dst, &tm_w, bar, kb * kBK, w_row, pol_w);
                     tma_load_2d_pair(dst + p.a_bytes, &tm_h, bar, kb * kBK, h_row, pol_h);
+                    ++n_issued;
                     if (++s == p.stages) { s = 0; ph ^= 1; }
                 }
             }
@@ -229,14 +229,14 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
             uint32_t ph = 0, aph = 0;
             bool ok = true;
             for (int u = pair; u < p.n_units && ok; u += n_pairs) {
-                if (ctrl->abort || !mbar_wait_cluster(&ctrl->acc_empty[ab], aph ^ 1)) { fail(p, ctrl, 12); ok = false; break; }
+                if (ctrl->abort || !mbar_wait_cluster(&ctrl->acc_empty[ab], aph ^ 1, p.wait_limit)) { fail(p, ctrl, 12); ok = false; break; }
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(ab * p.acc_stride);
                 int tile, slice, chunk;
                 decode(u, tile, slice, chunk);
                 const int nk = min(n_kb, (slice + 1) * p.kb_per_slice) - slice * p.kb_per_slice;
                 for (int kb = 0; kb < nk; ++kb) {
-                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->full[s], ph)) { fail(p, ctrl, 13); ok = false; break; }
+                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->full[s], ph, p.wait_limit)) { fail(p, ctrl, 13); ok = false; break; }
                     ptx::tc_fence_after();
                     const uint32_t sa = stage_u32 + (uint32_t)(s * p.stage_bytes);
                     const uint32_t sb = sa + (uint32_t)p.a_bytes;
@@ -297,7 +297,7 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
             decode(u, tile, slice, chunk);
             const int rbase = chunk * p.chunk_rows;
             const int vt = tile * 2 + (int)rank;                 // 128-row vocabulary tile of this CTA
-            if (ok && (ctrl->abort || !ptx::mbar_wait(&ctrl->acc_full[ab], aph))) { fail(p, ctrl, 16); ok = false; }
+            if (ok && (ctrl->abort || !ptx::mbar_wait(&ctrl->acc_full[ab], aph, p.wait_limit))) { fail(p, ctrl, 16); ok = false; }
             if (ok) {
                 ptx::tc_fence_after();
                 // (a unit of fewer than 128 rows per CTA leaves stale shared memory in the accumulator lanes beyond them)
@@ -379,9 +379,6 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
         }
     }
 
-#ifdef MIRROR_ATTN_TIMING
-    if (p.timing && tid == 64) { unsigned long long g__; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g__) :: "memory"); p.timing[blockIdx.x * 2 + 1] = (long long)g__; }
-#endif
     ptx::tc_fence_before();
     __syncthreads();
     cluster_sync_all();                 // no remote arrive or multicast commit is in flight towards a CTA that has left
@@ -406,16 +403,15 @@ int next_pow2(int x) {
     return p;
 }
 
-int ctas_per_sm_for(int M) {
-    int max_rows = 128;                     // up to this many rows two CTAs share an SM (<= 256 TMEM columns and >= 4 stages each)
-    if (const char* e = getenv("MIRROR_LM_PAIR2_MAX_ROWS")) { const int v = atoi(e); if (v >= 0 && v <= 128) max_rows = v; }
+int ctas_per_sm_for(const MirrorTuning& tune, int M) {
+    const int max_rows = tune.lm_pair2_max_rows;      // up to this many rows two CTAs share an SM (<= 256 TMEM columns and >= 4 stages each)
     int c = M <= max_rows ? 2 : 1;
-    if (const char* e = getenv("MIRROR_LM_CTAS_PER_SM")) { const int v = atoi(e); if (v == 1 || (v == 2 && M <= max_rows)) c = v; }
+    if (tune.lm_ctas_per_sm == 1 || (tune.lm_ctas_per_sm == 2 && M <= max_rows)) c = tune.lm_ctas_per_sm;
     return c;
 }
 
 // shapes shared by both modes: row chunks, accumulator layout, pipeline depth
-mirror_status pair_shape(int M, int V, int H, PairParams* p, int rows_cta = kTileV) {
+mirror_status pair_shape(const MirrorTuning& tune, int M, int V, int H, PairParams* p, int rows_cta = kTileV) {
     if (M <= 0 || V <= 0 || H <= 0 || H % kBK != 0) return MIRROR_ERR_SHAPE;
     p->M = M; p->V = V; p->H = H;
     p->n_chunks = (M + kMaxChunkRows - 1) / kMaxChunkRows;
@@ -428,20 +424,18 @@ mirror_status pair_shape(int M, int V, int H, PairParams* p, int rows_cta = kTil
     p->stage_bytes = p->a_bytes + p->half_rows * kBK * 2;
     // Few rows (a weight stream): two CTAs per SM with five or six stages each keep more bytes in flight than one CTA with
     // eight, deal the units to twice as many pairs, and let the CTAs of the next kernel move in one by one.
-    p->ctas_per_sm = ctas_per_sm_for(M);
+    p->ctas_per_sm = ctas_per_sm_for(tune, M);
     p->stages = (kSmemBudget / p->ctas_per_sm - kCtrlBytes - 2048) / p->stage_bytes;
     if (p->stages > kMaxStages) p->stages = kMaxStages;
-    if (const char* e = getenv("MIRROR_LM_STAGES")) { const int s = atoi(e); if (s >= 2 && s < p->stages) p->stages = s; }
+    if (tune.lm_stages >= 2 && tune.lm_stages < p->stages) p->stages = tune.lm_stages;
+    p->wait_limit = tune.wait_limit_cycles;
+    p->stall_after = -1;
     if (p->stages < 2) return MIRROR_ERR_SHAPE;
     p->k_slices = 1;
     p->kb_per_slice = H / kBK;
     p->inv_T = p->inv_T_log2e = 1.f;
     p->logits_out = nullptr;
     p->part_max = nullptr; p->part_idx = nullptr; p->part_sum = nullptr;
-    p->timing = nullptr;
-#ifdef MIRROR_ATTN_TIMING
-    if (const char* e = getenv("MIRROR_LM_TIMING_PTR")) p->timing = (long long*)strtoull(e, nullptr, 0);
-#endif
     return MIRROR_OK;
 }
 
@@ -495,18 +489,18 @@ mirror_status mirror_lmhead_pair_launch(mirror_ctx* ctx, const void* hidden, int
     // the units come out in whole waves over the pairs (152064 rows over 148 pairs: five units of 2 x 104 rows each
     // instead of four or five of 2 x 128).
     int rows_cta = kTileV;
-    if (ctas_per_sm_for(M) == 2) {
+    if (ctas_per_sm_for(ctx->tune, M) == 2) {
         const int pairs = ctx->num_sms;
         long long best = -1;
         for (int r = kTileV; r >= 64; r -= 8) {
             const long long units = (V + 2 * r - 1) / (2 * r), waves = (units + pairs - 1) / pairs;
             if (best < 0 || waves * r < best) { best = waves * r; rows_cta = r; }
         }
-        if (const char* e = getenv("MIRROR_LM_ROWS")) { const int r = atoi(e); if (r >= 8 && r <= kTileV && r % 8 == 0) rows_cta = r; }
+        if (ctx->tune.lm_rows >= 8 && ctx->tune.lm_rows <= kTileV && ctx->tune.lm_rows % 8 == 0) rows_cta = ctx->tune.lm_rows;
     }
     const int n_tiles = (V + 2 * rows_cta - 1) / (2 * rows_cta);
     PairParams p;
-    mirror_status st = pair_shape(M, V, H, &p, rows_cta);
+    mirror_status st = pair_shape(ctx->tune, M, V, H, &p, rows_cta);
     if (st != MIRROR_OK) return st;
     p.n_units = n_tiles * p.n_chunks;
     int n_pairs = ctx->num_sms / 2 * p.ctas_per_sm;
@@ -516,6 +510,7 @@ mirror_status mirror_lmhead_pair_launch(mirror_ctx* ctx, const void* hidden, int
     const size_t P = p.n_chunks == 1 ? (size_t)2 * n_pairs : (size_t)2 * n_tiles;
     if (partial_bytes < P * M * 12) return MIRROR_ERR_WORKSPACE;
     p.w_keep = p.n_chunks > 1;
+    if (ctx->tune.test_stall_after >= 0 && ctx->tune.test_stall_lm_left-- > 0) p.stall_after = ctx->tune.test_stall_after;
     p.inv_T = 1.0f / ctx->temperature;
     p.inv_T_log2e = p.inv_T * 1.4426950408889634f;
     p.logits_out = logits_out;
@@ -533,7 +528,7 @@ mirror_status mirror_lmhead_pair_launch(mirror_ctx* ctx, const void* hidden, int
 // waves of units), slices of at least 512 K elements.
 int mirror_linear_slices(const mirror_ctx* ctx, int M, int N, int K) {
     const int n_tiles = (N + kPairV - 1) / kPairV, n_chunks = (M + kMaxChunkRows - 1) / kMaxChunkRows;
-    const int n_kb = K / kBK, n_pairs = ctx->num_sms / 2 > 0 ? ctx->num_sms / 2 * ctas_per_sm_for(M) : 1;
+    const int n_kb = K / kBK, n_pairs = ctx->num_sms / 2 > 0 ? ctx->num_sms / 2 * ctas_per_sm_for(ctx->tune, M) : 1;
     int best = 1;
     double best_eff = 0.0;
     for (int s = 1; s <= 16; ++s) {
@@ -552,7 +547,7 @@ int mirror_linear_slices(const mirror_ctx* ctx, int M, int N, int K) {
 mirror_status mirror_linear_partial_launch(mirror_ctx* ctx, const void* x, int M, const void* W, int N, int K, float* partial,
                                            size_t partial_bytes, cudaStream_t stream, int* k_slices) {
     PairParams p;
-    mirror_status st = pair_shape(M, N, K, &p);
+    mirror_status st = pair_shape(ctx->tune, M, N, K, &p);
     if (st != MIRROR_OK) return st;
     const int n_tiles = (N + kPairV - 1) / kPairV, n_kb = K / kBK;
     const int s = mirror_linear_slices(ctx, M, N, K);

@@ -25,6 +25,8 @@
 #include <math.h>
 #include <stdlib.h>
 
+#include <mutex>
+
 #include "mirror_internal.h"
 
 namespace {
@@ -52,7 +54,7 @@ struct LmParams {
     int* part_idx;
     float* part_sum;
     int* status;
-    long long* timing;                  // developer aid (timing builds): per-CTA start / end stamps
+    long long wait_limit;               // SM cycles after which a wait gives up
 };
 
 struct Ctrl {
@@ -81,9 +83,6 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tm_w_full, const __grid_consta
     float* st_sum = (float*)(st_idx + 4 * kMaxChunkRows);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-#ifdef MIRROR_ATTN_TIMING
-    if (p.timing && tid == 0) { unsigned long long g__; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g__) :: "memory"); p.timing[blockIdx.x * 2] = (long long)g__; }
-#endif
 
     // this CTA's slice of the vocabulary, in 8-row groups
     const int g0 = (int)(((long long)p.groups_total * blockIdx.x) / gridDim.x);
@@ -141,7 +140,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tm_w_full, const __grid_consta
                             int s = s0;
                             uint32_t ph = ph0;
                             for (int j = 0; j < nk; ++j) {
-                                if (ctrl->abort || !ptx::mbar_wait(&ctrl->empty[s], ph ^ 1)) { fail(p, ctrl, 1); ok = false; break; }
+                                if (ctrl->abort || !ptx::mbar_wait(&ctrl->empty[s], ph ^ 1, p.wait_limit)) { fail(p, ctrl, 1); ok = false; break; }
                                 ptx::mbar_arrive_expect_tx(&ctrl->full[s], tx_bytes);
                                 if (++s == p.stages) { s = 0; ph ^= 1; }
                             }
@@ -195,11 +194,11 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tm_w_full, const __grid_consta
             bool ok = true;
             for (int chunk = 0; chunk < p.n_chunks && ok; ++chunk)
                 for (int t = 0; t < n_tiles && ok; ++t) {
-                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->acc_empty[ab], aph ^ 1)) { fail(p, ctrl, 2); ok = false; break; }
+                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->acc_empty[ab], aph ^ 1, p.wait_limit)) { fail(p, ctrl, 2); ok = false; break; }
                     ptx::tc_fence_after();
                     const uint32_t d_tmem = tmem_base + (uint32_t)(ab * p.acc_stride);
                     for (int kb = 0; kb < n_kb; ++kb) {
-                        if (ctrl->abort || !ptx::mbar_wait(&ctrl->full[s], ph)) { fail(p, ctrl, 3); ok = false; break; }
+                        if (ctrl->abort || !ptx::mbar_wait(&ctrl->full[s], ph, p.wait_limit)) { fail(p, ctrl, 3); ok = false; break; }
                         ptx::tc_fence_after();
                         const uint32_t sa = stage_u32 + (uint32_t)(s * p.stage_bytes);
                         const uint32_t sb = sa + kATileBytes;
@@ -229,7 +228,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tm_w_full, const __grid_consta
             for (int c = lane; c < kMaxChunkRows; c += 32) { my_max[c] = -INFINITY; my_idx[c] = 0x7fffffff; my_sum[c] = 0.f; }
             __syncwarp();
             for (int t = 0; t < n_tiles && ok; ++t) {
-                if (ctrl->abort || !ptx::mbar_wait(&ctrl->acc_full[ab], aph)) { fail(p, ctrl, 4); ok = false; break; }
+                if (ctrl->abort || !ptx::mbar_wait(&ctrl->acc_full[ab], aph, p.wait_limit)) { fail(p, ctrl, 4); ok = false; break; }
                 ptx::tc_fence_after();
                 const int vid = row_begin + t * kTileV + q * 32 + lane;      // this thread's vocabulary id
                 const bool valid = vid < row_end;
@@ -303,9 +302,6 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tm_w_full, const __grid_consta
         }
     }
 
-#ifdef MIRROR_ATTN_TIMING
-    if (p.timing && tid == 64) { unsigned long long g__; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g__) :: "memory"); p.timing[blockIdx.x * 2 + 1] = (long long)g__; }
-#endif
     ptx::tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -485,8 +481,7 @@ mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, c
     const int V = ctx->desc.vocab, H = ctx->desc.hidden;
     // The GEMM runs on CTA pairs (lmhead_pair.cu) whenever the partials it leaves fit the scratch it was given; the
     // single-CTA weight-stream kernel below is the fallback (and what MIRROR_LM_PAIR_MIN_ROWS can force for comparison).
-    int pair_min_rows = 1;
-    if (const char* e = getenv("MIRROR_LM_PAIR_MIN_ROWS")) pair_min_rows = atoi(e);
+    const int pair_min_rows = ctx->tune.lm_pair_min_rows;
     if (M >= pair_min_rows && ctx->num_sms >= 2) {
         int P = 0;
         mirror_status st = mirror_lmhead_pair_launch(ctx, hidden, M, W, logits_out, partial_ws, partial_bytes, stream, &P);
@@ -515,8 +510,8 @@ mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, c
     if (p.stages < 2) return MIRROR_ERR_SHAPE;
     // producer batching (tuning knobs; the defaults were picked by measurement on B200)
     p.k_group = p.stages / 2 < 5 ? (p.stages / 2 > 0 ? p.stages / 2 : 1) : 5;
-    if (const char* e = getenv("MIRROR_LM_KGROUP")) p.k_group = atoi(e);
-    if (const char* e = getenv("MIRROR_LM_STAGES")) { const int s = atoi(e); if (s >= 2 && s < p.stages) p.stages = s; }
+    if (ctx->tune.lm_kgroup > 0) p.k_group = ctx->tune.lm_kgroup;
+    if (ctx->tune.lm_stages >= 2 && ctx->tune.lm_stages < p.stages) p.stages = ctx->tune.lm_stages;
     if (p.k_group < 1) p.k_group = 1;
     if (p.k_group > p.stages) p.k_group = p.stages;
     p.groups_total = (V + 7) / 8;
@@ -524,10 +519,7 @@ mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, c
     p.inv_T_log2e = p.inv_T * 1.4426950408889634f;
     p.logits_out = logits_out;
     p.status = ctx->d_status;
-    p.timing = nullptr;
-#ifdef MIRROR_ATTN_TIMING
-    if (const char* e = getenv("MIRROR_LM_TIMING_PTR")) p.timing = (long long*)strtoull(e, nullptr, 0);
-#endif
+    p.wait_limit = ctx->tune.wait_limit_cycles;
 
     int grid = ctx->num_sms;
     if (grid > p.groups_total) grid = p.groups_total;
@@ -605,11 +597,11 @@ extern "C" mirror_status mirror_lmhead_reduce(mirror_ctx* ctx, const void* hidde
 namespace {
 
 constexpr int kNoAllocMaxRows = 128;      // M limit of the no-allocation entry point
-constexpr int kNoAllocMaxCtas = 256;      // >= SM count of any device this library supports
+constexpr int kNoAllocMaxCtas = 320;      // partials of one launch: up to two CTAs on each of 160 SMs (a B200 has 148)
 constexpr size_t kNoAllocHeader = 256;    // {status code, detail} words in front of the partials
 constexpr size_t kNoAllocBytes = kNoAllocHeader + (size_t)kNoAllocMaxCtas * kNoAllocMaxRows * 12;
 
-// Lives in every GPU's copy of the library image from load until exit (393,472 bytes per device).
+// Lives in every GPU's copy of the library image from load until exit (491,776 bytes per device).
 // In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
 
@@ -621,6 +613,7 @@ struct NoAllocDevice {          // host-side, per device, filled by the first ca
     PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
 };
 NoAllocDevice g_noalloc_dev[64];
+std::mutex g_noalloc_mutex;      // the one-time set-up of a device, and its `ready` flag, from any host thread
 
 }  // namespace
 
@@ -633,12 +626,13 @@ extern "C" mirror_status mirror_lmhead_reduce_noalloc(int device, const void* hi
     if (((uintptr_t)hidden & 15) || ((uintptr_t)W & 15)) return MIRROR_ERR_ARG;
     MIRROR_CUDA_OK(cudaSetDevice(device));
     NoAllocDevice& d = g_noalloc_dev[device];
+    std::unique_lock<std::mutex> lock(g_noalloc_mutex);
     if (!d.ready) {
         // one-time set-up on this device (no allocation): resolve the device address of the scratch array
         cudaDeviceProp prop;
         MIRROR_CUDA_OK(cudaGetDeviceProperties(&prop, device));
         if (prop.major != 10) return MIRROR_ERR_UNSUPPORTED;
-        if (prop.multiProcessorCount > kNoAllocMaxCtas) return MIRROR_ERR_UNSUPPORTED;
+        if (2 * prop.multiProcessorCount > kNoAllocMaxCtas) return MIRROR_ERR_UNSUPPORTED;
         void* ptr = nullptr;
         if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) return MIRROR_ERR_CUDA;
         void* fn = nullptr;
@@ -651,6 +645,7 @@ extern "C" mirror_status mirror_lmhead_reduce_noalloc(int device, const void* hi
         d.encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
         d.ready = true;
     }
+    lock.unlock();
     // A context on the stack stands in for mirror_create's: same launch path, nothing allocated.
     mirror_ctx tmp;
     tmp.desc.hidden = H;
@@ -668,12 +663,36 @@ extern "C" mirror_status mirror_lmhead_reduce_noalloc(int device, const void* hi
     tmp.lm_attr_set = d.attr_set;
     tmp.lm_pair_attr_set = d.pair_attr_set;
     cudaStream_t s = (cudaStream_t)stream;
-    // the status words must start at zero; the partials are fully rewritten by every launch before they are read
-    MIRROR_CUDA_OK(cudaMemsetAsync(d.scratch, 0, kNoAllocHeader, s));
+    // (the status words in the header start at zero with the library image and keep the first problem until
+    // mirror_lmhead_noalloc_status reads and clears them; the partials are fully rewritten by every launch before
+    // they are read)
     mirror_status st = mirror_lmhead_launch(&tmp, hidden, M, W, 0, nullptr, nullptr, 0, argmax, maxlogit, lse, nullptr, nullptr,
                                             nullptr, nullptr, d.scratch + kNoAllocHeader, kNoAllocBytes - kNoAllocHeader,
                                             nullptr, s, nullptr);
     d.attr_set = tmp.lm_attr_set;
     d.pair_attr_set = tmp.lm_pair_attr_set;
     return st;
+}
+
+// Device-side problems of mirror_lmhead_reduce_noalloc calls (a bounded wait that ran out, a failed bounds check) are
+// recorded in the first words of the scratch array, since there is no context to ask.  Synchronises the device, returns
+// the first problem since the last query (0: none) and clears it.  Allocates nothing.
+extern "C" mirror_status mirror_lmhead_noalloc_status(int device, int* code, int* detail) {
+    if (!code || device < 0 || device >= 64) return MIRROR_ERR_ARG;
+    unsigned char* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        if (g_noalloc_dev[device].ready) scratch = g_noalloc_dev[device].scratch;
+    }
+    *code = 0;
+    if (detail) *detail = 0;
+    if (!scratch) return MIRROR_OK;                      // no call was ever made on this device
+    MIRROR_CUDA_OK(cudaSetDevice(device));
+    MIRROR_CUDA_OK(cudaDeviceSynchronize());
+    int words[2] = {0, 0};
+    MIRROR_CUDA_OK(cudaMemcpy(words, scratch, sizeof words, cudaMemcpyDeviceToHost));
+    if (words[0] != 0) MIRROR_CUDA_OK(cudaMemset(scratch, 0, sizeof words));
+    *code = words[0] == MIRROR_DEV_TIMEOUT ? MIRROR_ERR_TIMEOUT : (words[0] != 0 ? MIRROR_ERR_DEVICE_CHECK : MIRROR_OK);
+    if (detail) *detail = words[1];
+    return MIRROR_OK;
 }

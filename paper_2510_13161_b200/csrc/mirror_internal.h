@@ -20,8 +20,31 @@ struct MirrorTreeInfo {            // host-side digest of one token tree, rebuil
     unsigned char path_len[MIRROR_MAX_BRANCHES];
 };
 
+// Tuning values, read ONCE from the environment when a context is created (defaults measured on B200); a context made
+// on the stack by the no-allocation entry point keeps the defaults.  The last two exist for the tests of the bounded
+// waits: a short limit, and a producer that stops issuing copies after a number of stages, so that a consumer's wait
+// runs out and the kernel has to unwind (nothing traps, nothing spins without limit, no memory fault is provoked).
+struct MirrorTuning {
+    int attn_groups = 0;             // MIRROR_ATTN_GROUPS: upper limit of CTA groups (0: all)
+    int attn_whole_units = 1;        // MIRROR_ATTN_WHOLE_UNITS: 0 = never trade CTA groups for whole units
+    int attn_snap = 4;               // MIRROR_ATTN_SNAP: boundary snapping distance in tiles
+    int attn_ring = 0;               // MIRROR_ATTN_RING: K/V ring depths as two digits, e.g. 64 (0: deepest that fits)
+    int lm_pair2_max_rows = 128;     // MIRROR_LM_PAIR2_MAX_ROWS: two CTAs per SM up to this many rows
+    int lm_ctas_per_sm = 0;          // MIRROR_LM_CTAS_PER_SM: 1 or 2 (0: by rows)
+    int lm_stages = 0;               // MIRROR_LM_STAGES: fewer pipeline stages than fit (0: all)
+    int lm_rows = 0;                 // MIRROR_LM_ROWS: rows per CTA and unit of the LM head as a weight stream (0: balanced choice)
+    int lm_pair_min_rows = 1;        // MIRROR_LM_PAIR_MIN_ROWS: rows from which the pair kernel is used
+    int lm_kgroup = 0;               // MIRROR_LM_KGROUP: K blocks requested at a time by the single-CTA kernel (0: default)
+    long long wait_limit_cycles = 4000000000ll;   // MIRROR_WAIT_LIMIT_CYCLES: SM cycles after which a device-side wait gives up
+    int test_stall_after = -1;       // MIRROR_TEST_STALL_AFTER_STAGES: a producer issues this many stages, then stops (-1: off);
+                                     // applies to the FIRST attention launch and the first LM-head launch of a context only
+    int test_stall_attn_left = 1, test_stall_lm_left = 1;
+};
+void mirror_tuning_from_env(MirrorTuning* t);
+
 struct mirror_ctx {
     mirror_model_desc desc;
+    MirrorTuning tune;
     int device = 0;
     int num_sms = 0;
     float scale = 0.f;

@@ -74,10 +74,11 @@ def test_single_cta_fallback_kernel_matches_oracle_and_pair_kernel(M, V, H, monk
     W = rand_bf16((V, H), 0.05, 11); hid = rand_bf16((M, H), 1.0, 12)
     m = make_mirror(lm_cfg(V, H))
     res_pair = m.mirror_lmhead_reduce(hid.cuda(), W.cuda(), want_logits=True)
-    monkeypatch.setenv("MIRROR_LM_PAIR_MIN_ROWS", "1000000")
-    res = m.mirror_lmhead_reduce(hid.cuda(), W.cuda(), want_logits=True)
+    monkeypatch.setenv("MIRROR_LM_PAIR_MIN_ROWS", "1000000")      # (tuning values are read when a context is created)
+    m1 = make_mirror(lm_cfg(V, H))
     monkeypatch.delenv("MIRROR_LM_PAIR_MIN_ROWS")
-    assert m.device_status() == (0, 0)
+    res = m1.mirror_lmhead_reduce(hid.cuda(), W.cuda(), want_logits=True)
+    assert m.device_status() == (0, 0) and m1.device_status() == (0, 0)
     logits = O.lmhead_logits(I.bf16_bits(hid), I.bf16_bits(W))
     assert np.abs(res["logits"].cpu().numpy() - logits).max() < LOGIT_TOL_TIGHT
     check_reductions(res, logits)

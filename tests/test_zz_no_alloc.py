@@ -2,12 +2,14 @@
 (all memory owned by the host's own pool, allocator-guarded plugin regions).  Its scratch is a fixed
 array inside the library, so it needs neither a context nor a workspace.  The test calls it through the
 C ABI twice in a row and checks each result against the regular entry point, which uses a caller
-workspace.  Collected last on purpose: a failure here cannot hide any other test."""
+workspace, and against the CPU oracle.  Collected last on purpose: a failure here cannot hide any other test."""
 import ctypes as C
 
+import numpy as np
 import pytest
 import torch
 
+from oracle import oracle as O
 from paper_2510_13161_b200 import binding, inputs as I
 from tests.helpers import make_mirror
 
@@ -61,3 +63,28 @@ def test_noalloc_rejects_sizes_beyond_its_scratch():
     res = binding.mirror_lmhead_reduce_noalloc(hid[:128], W)              # the limit itself is accepted
     ref = make_mirror(I.VerifyConfig("t", H, 4, 2, 64, 1, 1, 16, 16, 2, 4, V, "greedy")).mirror_lmhead_reduce(hid[:128], W)
     assert torch.equal(res["argmax"], ref["argmax"])
+
+
+@pytest.mark.parametrize("rows", [(111, 128), (128, 17)])
+def test_noalloc_against_the_oracle_at_row_counts_where_every_sm_holds_two_ctas(rows):
+    """Up to 128 rows two CTAs share an SM, so a launch leaves twice as many partials as the GPU has SMs: the fixed
+    array holds them (111 rows was the first count that did not fit an array sized by the SM count).  Two calls in a
+    row, the second on fewer or more rows than the first, each compared with the fp64 oracle."""
+    lib = binding.load_library()
+    V, H, T = 40960, 512, 1.0
+    W = rand_bf16((V, H), 0.05, 21)
+    Wb = I.bf16_bits(W)
+    for seed, M in enumerate(rows):
+        hid = rand_bf16((M, H), 1.0, 30 + seed)
+        am = torch.empty(M, dtype=torch.int32, device="cuda")
+        mx = torch.empty(M, dtype=torch.float32, device="cuda")
+        ls = torch.empty(M, dtype=torch.float32, device="cuda")
+        assert call_noalloc(lib, hid, W, T, am, mx, ls) == 0
+        assert binding.mirror_lmhead_noalloc_status(0) == (0, 0)
+        logits = O.lmhead_logits(I.bf16_bits(hid), Wb)
+        red = O.row_reduce(logits)
+        got = am.cpu().numpy()
+        for r in np.nonzero(got != red["argmax"])[0]:          # a flip only inside the logit error bound
+            assert logits[r, red["argmax"][r]] - logits[r, got[r]] < 2e-3, r
+        assert np.abs(mx.cpu().numpy() - red["maxlogit"]).max() <= 2e-3
+        assert np.abs(ls.cpu().numpy() - red["lse"]).max() <= 2e-3
