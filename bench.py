@@ -66,6 +66,9 @@ def parse_args():
                          "decoder layers of the workload's shape with seeded random weights (0.66 GB per layer for the default "
                          "workload); reported under stages.target_forward, outside the timed region")
     ap.add_argument("--intermediate", type=int, default=17408, help="MLP width for --target-layers")
+    ap.add_argument("--lmhead-fp8", action="store_true",
+                    help="also time the low-precision LM head (e4m3 weights and hidden rows, one scale per row) next to the bf16 "
+                         "head on the workload's rows; reported under stages.lmhead_fp8, outside the timed region")
     ap.add_argument("--layers", type=int, default=None,
                     help="profiling aid: run the workload with this many attention layers (config.layers reports it); "
                          "the default, the workload's own layer count, is the only valid bench configuration")
@@ -361,6 +364,41 @@ def overlap_draft_stage(step, stream, reps: int = 20):
     return out
 
 
+def lmhead_fp8_stage(m, x, cfg, hbm_gbs: float, reps: int = 20):
+    """bf16 LM head against the e4m3 one on the same rows (random rows of the workload's shape): ms and weight GB/s each.
+    The weights are quantised once, outside the timing; the per-step quantisation of the hidden rows is timed with it."""
+    import torch
+    dev = x.W.device
+    hid = torch.empty((cfg.rows, cfg.hidden), dtype=torch.bfloat16, device=dev).normal_(0, 1.0)
+    W8, ws = m.mirror_quantize_rows_fp8(x.W)
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    def fp8():
+        h8, hs = m.mirror_quantize_rows_fp8(hid)
+        m.mirror_lmhead_reduce_fp8(h8, hs, W8, ws)
+
+    t16 = timed(lambda: m.mirror_lmhead_reduce(hid, x.W))
+    t8 = timed(fp8)
+    code, detail = m.device_status()
+    if code != 0:
+        raise SystemExit(f"device status {code} (detail {detail}) in the fp8 LM head")
+    wb = cfg.vocab * cfg.hidden
+    return {"rows": cfg.rows, "bf16_ms": t16, "fp8_ms": t8, "bf16_weight_gbs": 2 * wb / t16 / 1e6, "fp8_weight_gbs": wb / t8 / 1e6,
+            "fp8_frac_hbm": wb / t8 / 1e6 / hbm_gbs, "speedup": t16 / t8,
+            "note": "both include the merge kernel; fp8 also includes quantising the hidden rows"}
+
+
 def target_forward_stage(m, x, tree, kv, cfg, n_layers: int, intermediate: int, hbm_gbs: float, reps: int = 5):
     """mirror_target_forward over n_layers decoder layers of the workload's shape (random weights): ms, weight bytes per
     second against the HBM peak.  The layers are weight streams at these row counts."""
@@ -601,6 +639,8 @@ def run_mirror(args):
         stages["attn_per_layer_ms"] = attn_per_layer(m, x, w.tree, cfg)
     if args.overlap_draft:
         stages["overlap_draft"] = overlap_draft_stage(w.step, w.stream)
+    if args.lmhead_fp8:
+        stages["lmhead_fp8"] = lmhead_fp8_stage(m, x, cfg, peaks["hbm_gbs"])
     if args.target_layers > 0:
         stages["target_forward"] = target_forward_stage(m, x, w.tree, w.kv, cfg, min(args.target_layers, cfg.layers), args.intermediate,
                                                         peaks["hbm_gbs"])

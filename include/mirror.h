@@ -174,6 +174,21 @@ mirror_status mirror_lmhead_reduce(mirror_ctx* ctx, const void* hidden, int M, c
                                    int32_t* topk_id, float* topk_logprob, float* gather_logit,
                                    float* logits_out, void* stream);
 
+/* Low-precision LM head (Eq. 1 / Eq. 5 with quantised operands; the paper states no precision for the LM head:
+ * an opt-in mode for the weight stream, the bf16 head stays the default).
+ * mirror_quantize_rows_fp8: x bf16 [rows, cols] (device) -> out_fp8 [rows, cols] e4m3 bytes and out_scale [rows] fp32 with
+ *   scale = max|x_row| / 448 (1 for an all-zero row) and code = e4m3(x / scale), round to nearest even (fp32 division).
+ *   Use it once for W [V, H] (one scale per vocabulary row) and per step for the hidden rows.
+ * mirror_lmhead_reduce_fp8: logits[r, v] = w_scale[v] * h_scale[r] * sum_k W8[v, k] * h8[r, k] (exact e4m3 products,
+ *   fp32 accumulation on the tensor cores), then argmax (ties -> lowest id), max and lse = log sum exp(logits / T) as in
+ *   mirror_lmhead_reduce; logits_out nullable fp32 [M, V].  hidden must be a multiple of 128; 16-byte aligned pointers.
+ *   Needs a workspace sized for MIRROR_WS_LMHEAD.  Outputs nullable. */
+mirror_status mirror_quantize_rows_fp8(mirror_ctx* ctx, const void* x, int rows, int cols, void* out_fp8, float* out_scale,
+                                       void* stream);
+mirror_status mirror_lmhead_reduce_fp8(mirror_ctx* ctx, const void* hidden_fp8, const float* h_scale, int M, const void* W_fp8,
+                                       const float* w_scale, int32_t* argmax, float* maxlogit, float* lse, float* logits_out,
+                                       void* stream);
+
 /* LM head with fused argmax / max / log-sum-exp for callers that must not allocate device memory
  * (the paper has no counterpart: this is a deployment variant of mirror_lmhead_reduce, same kernels).
  * Who needs it: a host that has given all device memory to its own pool, a plugin called inside an

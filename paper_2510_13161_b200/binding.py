@@ -24,7 +24,7 @@ EXPORTS = [
     "mirror_create", "mirror_destroy", "mirror_workspace_bytes", "mirror_set_workspace",
     "mirror_attn_verify", "mirror_lmhead_reduce", "mirror_accept_select", "mirror_verify_step",
     "mirror_device_status", "mirror_launch_count", "mirror_status_str", "mirror_set_stage_events",
-    "mirror_lmhead_reduce_noalloc", "mirror_lmhead_noalloc_status", "mirror_early_exit_tap", "mirror_overlap_mass", "mirror_kv_commit",
+    "mirror_lmhead_reduce_noalloc", "mirror_lmhead_noalloc_status", "mirror_quantize_rows_fp8", "mirror_lmhead_reduce_fp8", "mirror_early_exit_tap", "mirror_overlap_mass", "mirror_kv_commit",
     "mirror_linear_scratch_bytes", "mirror_linear", "mirror_rmsnorm", "mirror_target_scratch_bytes", "mirror_target_forward", "mirror_trie_build", "mirror_verify_step_host", "mirror_embed_rows",
 ]
 
@@ -281,6 +281,30 @@ class Mirror:
                                              _ptr(res["argmax"]), _ptr(res["maxlogit"]), _ptr(res["lse"]),
                                              _ptr(res["topk_id"]), _ptr(res["topk_logprob"]), _ptr(res["gather_logit"]),
                                              _ptr(res["logits"]), _stream(stream)), "mirror_lmhead_reduce")
+        return res
+
+    def mirror_quantize_rows_fp8(self, x: torch.Tensor, stream=None):
+        """x bf16 [rows, cols] -> (e4m3 codes uint8 [rows, cols], scales fp32 [rows])."""
+        rows, cols = x.shape
+        out = torch.empty((rows, cols), dtype=torch.uint8, device=x.device)
+        scale = torch.empty(rows, dtype=torch.float32, device=x.device)
+        _check(self.lib.mirror_quantize_rows_fp8(self._ctx, _ptr(x, torch.bfloat16, "x"), rows, cols, _ptr(out, torch.uint8, "out"),
+                                                 _ptr(scale, torch.float32, "scale"), _stream(stream)), "mirror_quantize_rows_fp8")
+        return out, scale
+
+    def mirror_lmhead_reduce_fp8(self, hidden8, h_scale, W8, w_scale, want_logits: bool = False, stream=None) -> dict:
+        M = hidden8.shape[0]
+        dev = hidden8.device
+        res = dict(argmax=torch.empty(M, dtype=torch.int32, device=dev), maxlogit=torch.empty(M, dtype=torch.float32, device=dev),
+                   lse=torch.empty(M, dtype=torch.float32, device=dev),
+                   logits=torch.empty((M, self.desc.vocab), dtype=torch.float32, device=dev) if want_logits else None)
+        t = Tree(1, M if M <= 128 else 128, 0, 0, None, None)
+        t.batch, t.n_nodes = (M + 127) // 128, min(M, 128)      # sizes only: batch * n_nodes >= M
+        self.ensure_workspace(t, None, WS_LMHEAD)
+        _check(self.lib.mirror_lmhead_reduce_fp8(self._ctx, _ptr(hidden8, torch.uint8, "hidden8"), _ptr(h_scale, torch.float32, "h_scale"),
+                                                 M, _ptr(W8, torch.uint8, "W8"), _ptr(w_scale, torch.float32, "w_scale"),
+                                                 _ptr(res["argmax"]), _ptr(res["maxlogit"]), _ptr(res["lse"]), _ptr(res["logits"]),
+                                                 _stream(stream)), "mirror_lmhead_reduce_fp8")
         return res
 
     def accept_in(self, mode: int, emit_bonus: bool = True, target_argmax=None, logits=None, lse=None, q_probs=None,

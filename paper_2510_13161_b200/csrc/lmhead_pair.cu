@@ -54,6 +54,9 @@ struct PairParams {
     int* part_idx;
     float* part_sum;
     int* status;
+    int fp8;                                // 1: W and the hidden rows are e4m3 bytes (K counted in 128-byte blocks all the same)
+    const float* w_scale;                   // fp8: [V] scale of each weight row
+    const float* h_scale;                   // fp8: [M] scale of each hidden row
     long long wait_limit;                   // SM cycles after which a wait gives up
     int stall_after;                        // test aid: the producers stop after this many stages (-1: never)
 };
@@ -135,6 +138,20 @@ __device__ __forceinline__ void umma_pair_f16(uint32_t d_tmem, uint64_t a_desc, 
         "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
+}
+// the same for e4m3 operands (32 elements of K per instruction: the same 32 bytes of a 128-byte swizzled row)
+__device__ __forceinline__ void umma_pair_f8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// instruction descriptor for e4m3 x e4m3 -> fp32, both operands K-major
+__host__ __device__ __forceinline__ uint32_t umma_idesc_e4m3(int M, int N) {
+    return (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 // arrive on the barrier at this shared-memory offset in BOTH CTAs once all UMMAs issued so far have completed
 __device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
@@ -223,7 +240,7 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
     } else if (warp == 1) {
         if (lane == 0 && rank == 0) {
             // -------------------------------------------------------------- UMMA issuer (leader)
-            const uint32_t idesc = ptx::umma_idesc_bf16(kPairV, p.chunk_rows);
+            const uint32_t idesc = p.fp8 ? umma_idesc_e4m3(kPairV, p.chunk_rows) : ptx::umma_idesc_bf16(kPairV, p.chunk_rows);
             const uint32_t stage_u32 = ptx::smem_u32(stage_base);
             int s = 0, ab = 0;
             uint32_t ph = 0, aph = 0;
@@ -240,10 +257,17 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
                     ptx::tc_fence_after();
                     const uint32_t sa = stage_u32 + (uint32_t)(s * p.stage_bytes);
                     const uint32_t sb = sa + (uint32_t)p.a_bytes;
+                    if (p.fp8) {
 #pragma unroll
-                    for (int k4 = 0; k4 < kBK / 16; ++k4)
-                        umma_pair_f16(d_tmem, ptx::umma_desc_k_sw128(sa + k4 * 32), ptx::umma_desc_k_sw128(sb + k4 * 32), idesc,
-                                      (kb | k4) != 0);
+                        for (int k4 = 0; k4 < kBK / 16; ++k4)
+                            umma_pair_f8(d_tmem, ptx::umma_desc_k_sw128(sa + k4 * 32), ptx::umma_desc_k_sw128(sb + k4 * 32), idesc,
+                                         (kb | k4) != 0);
+                    } else {
+#pragma unroll
+                        for (int k4 = 0; k4 < kBK / 16; ++k4)
+                            umma_pair_f16(d_tmem, ptx::umma_desc_k_sw128(sa + k4 * 32), ptx::umma_desc_k_sw128(sb + k4 * 32), idesc,
+                                          (kb | k4) != 0);
+                    }
                     umma_commit_pair(&ctrl->empty[s]);
                     if (++s == p.stages) { s = 0; ph ^= 1; }
                 }
@@ -305,6 +329,7 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
                 const bool valid = q * 32 + lane < p.rows_cta && vid < p.V;
                 const bool any_valid = __ballot_sync(0xffffffffu, valid) != 0;          // warp-uniform
                 const int n_rows = min(p.chunk_rows, p.M - rbase);                       // hidden rows of this chunk
+                const float sw = (p.fp8 && valid) ? p.w_scale[vid] : 1.f;                 // fp8: this lane's weight-row scale
                 for (int cg = 0; cg < n_cg; ++cg) {
                     uint32_t r[32];
                     ptx::tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * p.acc_stride + cg * 32), r);
@@ -316,6 +341,13 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
                         // The 32 columns go through the reductions side by side (no branch inside, so the shuffle
                         // chains of different columns overlap); lane j keeps the result of column j.
                         float v[32], m[32];
+                        if (p.fp8) {
+                            // logit = (sum of e4m3 products) * weight-row scale * hidden-row scale; lane j fetches column j's scale
+                            const int cr = rbase + cg * 32 + lane;
+                            const float sh = cr < p.M ? p.h_scale[cr] : 0.f;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * (sw * __shfl_sync(0xffffffffu, sh, j)));
+                        }
 #pragma unroll
                         for (int j = 0; j < 32; ++j) m[j] = v[j] = valid ? __uint_as_float(r[j]) : -INFINITY;
                         if (p.logits_out && valid) {
@@ -435,6 +467,7 @@ mirror_status pair_shape(const MirrorTuning& tune, int M, int V, int H, PairPara
     p->kb_per_slice = H / kBK;
     p->inv_T = p->inv_T_log2e = 1.f;
     p->logits_out = nullptr;
+    p->fp8 = 0; p->w_scale = nullptr; p->h_scale = nullptr;
     p->part_max = nullptr; p->part_idx = nullptr; p->part_sum = nullptr;
     return MIRROR_OK;
 }
@@ -483,8 +516,12 @@ mirror_status pair_launch(mirror_ctx* ctx, bool reduce, const void* x, const voi
 int mirror_lmhead_pair_partials(int V) { return 2 * ((V + kPairV - 1) / kPairV); }
 
 mirror_status mirror_lmhead_pair_launch(mirror_ctx* ctx, const void* hidden, int M, const void* W, float* logits_out,
-                                        void* partial_ws, size_t partial_bytes, cudaStream_t stream, int* n_partials) {
-    const int V = ctx->desc.vocab, H = ctx->desc.hidden;
+                                        void* partial_ws, size_t partial_bytes, cudaStream_t stream, int* n_partials,
+                                        const float* w_scale, const float* h_scale) {
+    const bool fp8 = w_scale != nullptr;
+    if (fp8 && (!h_scale || ctx->desc.hidden % 128 != 0)) return MIRROR_ERR_SHAPE;
+    // (e4m3 rows are staged exactly like bf16 rows of half as many elements: the same bytes, boxes and swizzle)
+    const int V = ctx->desc.vocab, H = fp8 ? ctx->desc.hidden / 2 : ctx->desc.hidden;
     // A weight stream (two CTAs per SM) is as long as its busiest pair: the rows a CTA takes per unit are chosen so that
     // the units come out in whole waves over the pairs (152064 rows over 148 pairs: five units of 2 x 104 rows each
     // instead of four or five of 2 x 128).
@@ -518,6 +555,9 @@ mirror_status mirror_lmhead_pair_launch(mirror_ctx* ctx, const void* hidden, int
     p.part_idx = (int*)(p.part_max + P * M);
     p.part_sum = (float*)(p.part_idx + P * M);
     p.status = ctx->d_status;
+    p.fp8 = fp8 ? 1 : 0;
+    p.w_scale = w_scale;
+    p.h_scale = h_scale;
     st = pair_launch(ctx, true, hidden, W, p, n_pairs, stream);
     if (st != MIRROR_OK) return st;
     *n_partials = (int)P;

@@ -27,6 +27,8 @@
 
 #include <mutex>
 
+#include <cuda_fp8.h>
+
 #include "mirror_internal.h"
 
 namespace {
@@ -582,6 +584,77 @@ extern "C" mirror_status mirror_lmhead_reduce(mirror_ctx* ctx, const void* hidde
     return mirror_lmhead_launch(ctx, hidden, M, W, topk, gather_row, gather_tok, n_gather, argmax, maxlogit, lse, topk_id,
                                 topk_logprob, gather_logit, logits_out, (uint8_t*)ctx->ws + L.lm_partial, L.lm_partial_bytes, lse_scratch,
                                 (cudaStream_t)stream);
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Low-precision LM head: W and the hidden rows as e4m3 bytes with one fp32 scale per row (W ~ w_scale[v] * W8[v, :],
+// h ~ h_scale[r] * h8[r, :]); the GEMM runs on kind::f8f6f4 tensor-core instructions (fp32 accumulation of exact e4m3
+// products) and the epilogue multiplies each accumulator by the two scales before the row reductions.  Half the weight
+// bytes of the bf16 head: the weight stream of a verify step with few rows takes half the time.
+// ---------------------------------------------------------------------------------------------------
+namespace {
+
+// one block per row: scale = max|x| / 448 (1 for an all-zero row), code = e4m3(x / scale), round to nearest even
+__global__ void __launch_bounds__(256) quantize_rows_e4m3_kernel(const __nv_bfloat16* x, int cols, uint8_t* out, float* scale) {
+    __shared__ float s_part[8];
+    __shared__ float s_scale;
+    const __nv_bfloat16* row = x + (size_t)blockIdx.x * cols;
+    ptx::grid_dep_wait();
+    ptx::grid_dep_launch();
+    float amax = 0.f;
+    for (int c = threadIdx.x; c < cols; c += 256) amax = fmaxf(amax, fabsf(__bfloat162float(row[c])));
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = amax;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float a = 0.f;
+        for (int w = 0; w < 8; ++w) a = fmaxf(a, s_part[w]);
+        const float sc = a > 0.f ? __fdiv_rn(a, 448.f) : 1.f;
+        s_scale = sc;
+        scale[blockIdx.x] = sc;
+    }
+    __syncthreads();
+    const float sc = s_scale;
+    uint8_t* dst = out + (size_t)blockIdx.x * cols;
+    for (int c = threadIdx.x; c < cols; c += 256)
+        dst[c] = (uint8_t)__nv_cvt_float_to_fp8(__fdiv_rn(__bfloat162float(row[c]), sc), __NV_SATFINITE, __NV_E4M3);
+}
+
+}  // namespace
+
+extern "C" mirror_status mirror_quantize_rows_fp8(mirror_ctx* ctx, const void* x, int rows, int cols, void* out_fp8,
+                                                  float* out_scale, void* stream) {
+    if (!ctx || !x || !out_fp8 || !out_scale || rows <= 0 || cols <= 0) return MIRROR_ERR_ARG;
+    MIRROR_CUDA_OK(cudaSetDevice(ctx->device));
+    MIRROR_CUDA_OK(mirror_launch_pdl(quantize_rows_e4m3_kernel, dim3((unsigned)rows), dim3(256), 0, (cudaStream_t)stream,
+                                     (const __nv_bfloat16*)x, cols, (uint8_t*)out_fp8, out_scale));
+    ctx->launches += 1;
+    MIRROR_CUDA_OK(cudaGetLastError());
+    return MIRROR_OK;
+}
+
+extern "C" mirror_status mirror_lmhead_reduce_fp8(mirror_ctx* ctx, const void* hidden_fp8, const float* h_scale, int M,
+                                                  const void* W_fp8, const float* w_scale, int32_t* argmax, float* maxlogit,
+                                                  float* lse, float* logits_out, void* stream) {
+    if (!ctx || !hidden_fp8 || !h_scale || !W_fp8 || !w_scale || M <= 0) return MIRROR_ERR_ARG;
+    if (((uintptr_t)hidden_fp8 & 15) || ((uintptr_t)W_fp8 & 15)) return MIRROR_ERR_ARG;
+    if (ctx->desc.hidden % 128 != 0) return MIRROR_ERR_SHAPE;          // K in 128-byte blocks
+    if (!ctx->ws) return MIRROR_ERR_WORKSPACE;
+    MIRROR_CUDA_OK(cudaSetDevice(ctx->device));
+    MirrorWsLayout L;
+    mirror_ws_layout(ctx, (size_t)M, &L);
+    if (ctx->ws_bytes < L.end_lmhead) return MIRROR_ERR_WORKSPACE;
+    void* partial_ws = (uint8_t*)ctx->ws + L.lm_partial;
+    int P = 0;
+    mirror_status st = mirror_lmhead_pair_launch(ctx, hidden_fp8, M, W_fp8, logits_out, partial_ws, L.lm_partial_bytes,
+                                                 (cudaStream_t)stream, &P, w_scale, h_scale);
+    if (st != MIRROR_OK) return st;
+    const float inv_T = 1.0f / ctx->temperature, inv_T_log2e = inv_T * 1.4426950408889634f;
+    float* part_max = (float*)partial_ws;
+    int* part_idx = (int*)(part_max + (size_t)P * M);
+    float* part_sum = (float*)(part_idx + (size_t)P * M);
+    return lmhead_tail(ctx, nullptr, M, nullptr, 0, nullptr, nullptr, 0, argmax, maxlogit, lse, nullptr, nullptr, nullptr, logits_out,
+                       nullptr, (cudaStream_t)stream, nullptr, P, inv_T, inv_T_log2e, part_max, part_idx, part_sum);
 }
 
 // ---------------------------------------------------------------------------------------------------

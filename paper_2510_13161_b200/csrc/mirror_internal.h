@@ -91,8 +91,10 @@ mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, c
 // LM-head GEMM + per-unit row partials on CTA pairs (many hidden rows); *n_partials partials of [M] rows are left in
 // partial_ws for lmhead_merge_kernel.  mirror_lmhead_pair_partials(V) is that count.
 int mirror_lmhead_pair_partials(int V);
+// w_scale / h_scale non-null: W and hidden are e4m3 bytes with one scale per row (the GEMM runs on kind::f8f6f4).
 mirror_status mirror_lmhead_pair_launch(mirror_ctx* ctx, const void* hidden, int M, const void* W, float* logits_out,
-                                        void* partial_ws, size_t partial_bytes, cudaStream_t stream, int* n_partials);
+                                        void* partial_ws, size_t partial_bytes, cudaStream_t stream, int* n_partials,
+                                        const float* w_scale = nullptr, const float* h_scale = nullptr);
 // Plain GEMM on CTA pairs: partial[s][M][N] (fp32) = x[M, K-slice s] * W[N, K-slice s]^T for the *k_slices slices that
 // mirror_linear_slices() picks (1 when the output tiles alone fill the GPU); the caller adds the slices in order.
 int mirror_linear_slices(const mirror_ctx* ctx, int M, int N, int K);
