@@ -127,7 +127,10 @@ typedef struct {
 /* What mirror_workspace_bytes should size for. */
 #define MIRROR_WS_ATTN 1u           /* mirror_attn_verify */
 #define MIRROR_WS_LMHEAD 2u         /* mirror_lmhead_reduce (M = batch * n_nodes rows) */
-#define MIRROR_WS_LMHEAD_LOGITS 10u /* mirror_lmhead_reduce with topk > 0 and logits_out == NULL */
+#define MIRROR_WS_LMHEAD_LOGITS 10u /* mirror_lmhead_reduce with a workspace that can hold the fp32 logits [M, V] */
+#define MIRROR_WS_LMHEAD_TOPK 34u   /* mirror_lmhead_reduce with topk > 0, mirror_early_exit_tap.  Up to 256 rows the Top-kappa is
+                                       selected inside the GEMM's epilogue: candidate lists instead of an [M, V] buffer; with more
+                                       rows this sizes like MIRROR_WS_LMHEAD_LOGITS (the selection reads spilled logits) */
 #define MIRROR_WS_STEP_GREEDY 7u    /* mirror_verify_step, greedy */
 #define MIRROR_WS_STEP_SPEC 15u     /* mirror_verify_step, speculative sampling (holds the fp32 logits) */
 #define MIRROR_WS_ACCEPT_TREE 16u   /* adds the fp64 scratch of MIRROR_ACCEPT_SPEC_TREE (optional: without it the rule
@@ -165,9 +168,10 @@ mirror_status mirror_attn_verify(mirror_ctx* ctx, const mirror_kv* kv, const mir
  *   topk > 0: topk_id int32 [M, topk], topk_logprob fp32 [M, topk] = logits/T - lse, ordered by
  *             (logit descending, id ascending): the Top-kappa message of Eq. 6.  topk <= MIRROR_MAX_TOPK.
  *   gather_row/gather_tok int32 [n_gather] -> gather_logit fp32 [n_gather] = logits[row][tok]  (nullable)
- *   logits_out fp32 [M, V], nullable: the full logits (needed by speculative sampling; Top-kappa uses the
- *             workspace when this is NULL)
- * Needs a workspace sized for MIRROR_WS_LMHEAD. */
+ *   logits_out fp32 [M, V], nullable: the full logits (needed by speculative sampling)
+ * Needs a workspace sized for MIRROR_WS_LMHEAD; with topk > 0 one sized for MIRROR_WS_LMHEAD_TOPK: with up to 256 rows the
+ * Top-kappa is then selected inside the GEMM's epilogue (sorted lists per epilogue warp and row that live as long as the
+ * CTA, merged afterwards) and the logits never reach memory; with more rows the selection runs over spilled fp32 logits. */
 mirror_status mirror_lmhead_reduce(mirror_ctx* ctx, const void* hidden, int M, const void* W, int topk,
                                    const int32_t* gather_row, const int32_t* gather_tok, int n_gather,
                                    int32_t* argmax, float* maxlogit, float* lse,
@@ -242,8 +246,8 @@ mirror_status mirror_accept_select(mirror_ctx* ctx, const mirror_tree* tree, con
  *   msg_ids          int32 [M, kappa]: candidate ids ordered by (logit descending, id ascending)
  *   msg_logprob_bf16 bf16 [M, kappa]: their log-probabilities logit/T - lse under the early-exit proxy (the token
  *                    channel's payload type)
- * kappa <= MIRROR_MAX_TOPK.  Needs a workspace sized for MIRROR_WS_LMHEAD_LOGITS with M rows (the selection runs over
- * the spilled fp32 logits).  msg_ids is what mirror_accept_select / mirror_verify_step take as cand_ids (n_cand =
+ * kappa <= MIRROR_MAX_TOPK.  Needs a workspace sized for MIRROR_WS_LMHEAD_TOPK with M rows (up to 256 rows the selection
+ * happens in the GEMM's epilogue and there is no [M, V] buffer).  msg_ids is what mirror_accept_select / mirror_verify_step take as cand_ids (n_cand =
  * kappa) for the reuse decision of the same rows. */
 mirror_status mirror_early_exit_tap(mirror_ctx* ctx, const void* hidden_le, int M, const void* W, int kappa,
                                     int32_t* msg_ids, void* msg_logprob_bf16, void* stream);

@@ -19,6 +19,7 @@ ACCEPT_GREEDY = 0
 ACCEPT_SPEC_SAMPLING = 1
 ACCEPT_SPEC_TREE = 2
 WS_ATTN, WS_LMHEAD, WS_LMHEAD_LOGITS, WS_STEP_GREEDY, WS_STEP_SPEC, WS_ACCEPT_TREE, WS_STEP_TREE = 1, 2, 10, 7, 15, 16, 31
+WS_LMHEAD_TOPK = 34
 
 EXPORTS = [
     "mirror_create", "mirror_destroy", "mirror_workspace_bytes", "mirror_set_workspace",
@@ -273,7 +274,7 @@ class Mirror:
             res["logits"] = torch.empty((M, self.desc.vocab), dtype=torch.float32, device=dev)
         t = Tree(1, M if M <= 128 else 128, 0, 0, None, None)
         t.batch, t.n_nodes = (M + 127) // 128, min(M, 128)      # sizes only: batch * n_nodes >= M
-        self.ensure_workspace(t, None, WS_LMHEAD_LOGITS if (topk and not want_logits) else WS_LMHEAD)
+        self.ensure_workspace(t, None, WS_LMHEAD_TOPK if topk else WS_LMHEAD)
         _check(self.lib.mirror_lmhead_reduce(self._ctx, _ptr(hidden, torch.bfloat16, "hidden"), M,
                                              _ptr(W, torch.bfloat16, "W"), topk,
                                              _ptr(gather_row, torch.int32, "gather_row"),
@@ -324,7 +325,7 @@ class Mirror:
         lp = torch.empty((M, kappa), dtype=torch.bfloat16, device=hidden_le.device)
         t = Tree(1, M if M <= 128 else 128, 0, 0, None, None)
         t.batch, t.n_nodes = (M + 127) // 128, min(M, 128)      # sizes only: batch * n_nodes >= M
-        self.ensure_workspace(t, None, WS_LMHEAD_LOGITS)
+        self.ensure_workspace(t, None, WS_LMHEAD_TOPK)
         _check(self.lib.mirror_early_exit_tap(self._ctx, _ptr(hidden_le, torch.bfloat16, "hidden_le"), M,
                                               _ptr(W, torch.bfloat16, "W"), kappa, _ptr(ids, torch.int32, "msg_ids"),
                                               _ptr(lp, torch.bfloat16, "msg_logprob"), _stream(stream)), "mirror_early_exit_tap")

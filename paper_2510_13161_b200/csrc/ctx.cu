@@ -223,6 +223,11 @@ void mirror_ws_layout(const mirror_ctx* ctx, size_t M, MirrorWsLayout* out, size
     L.accept_scratch = at;
     at += align_up(B * 2 * (size_t)ctx->desc.vocab * sizeof(double), 256);
     L.end_accept = at;
+    // the candidate lists of the fused Top-kappa share the front of the logits region (a call either spills or selects)
+    L.lm_topk = L.logits;
+    // (four lists per CTA and row, two CTAs per SM; only up to 256 rows, one row chunk: beyond, Top-kappa selects from spilled logits)
+    L.lm_topk_bytes = M <= 256 ? align_up((size_t)8 * ctx->num_sms * M * (size_t)MIRROR_MAX_TOPK * 8, 256) : 0;
+    L.end_topk = L.lm_topk + L.lm_topk_bytes;
     *out = L;
 }
 
@@ -235,7 +240,12 @@ extern "C" mirror_status mirror_workspace_bytes(const mirror_ctx* ctx, const mir
     mirror_ws_layout(ctx, (size_t)tree->batch * tree->n_nodes, &L, (size_t)tree->batch);
     size_t need = L.end_attn;
     if (what & (MIRROR_WS_LMHEAD | 4u)) need = L.end_lmhead;
-    if (what & 8u) need = L.end_logits;
+    if (what & 32u) {
+        // room for the candidate lists; and for the logits where the largest kappa could not be selected in the epilogue
+        if (L.lm_topk_bytes && L.end_topk > need) need = L.end_topk;
+        if (!mirror_lmhead_topk_fusable(ctx, (int)((size_t)tree->batch * tree->n_nodes), MIRROR_MAX_TOPK) && L.end_logits > need) need = L.end_logits;
+    }
+    if (what & 8u) need = L.end_logits > need ? L.end_logits : need;
     if (what & 16u) need = L.end_accept;
     *bytes = need;
     return MIRROR_OK;

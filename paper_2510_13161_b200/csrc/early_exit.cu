@@ -38,9 +38,15 @@ extern "C" mirror_status mirror_early_exit_tap(mirror_ctx* ctx, const void* hidd
     MIRROR_CUDA_OK(cudaSetDevice(ctx->device));
     MirrorWsLayout L;
     mirror_ws_layout(ctx, (size_t)M, &L);
-    if (ctx->ws_bytes < L.end_logits) return MIRROR_ERR_WORKSPACE;
     uint8_t* ws = (uint8_t*)ctx->ws;
-    // the Top-kappa selection runs over the spilled fp32 logits of the early-exit rows
+    if (L.lm_topk_bytes && ctx->ws_bytes >= L.end_topk && mirror_lmhead_topk_fusable(ctx, M, kappa)) {
+        // the Top-kappa is selected inside the GEMM's epilogue: the proxy's logits never reach memory
+        return mirror_lmhead_launch(ctx, hidden_le, M, W, kappa, nullptr, nullptr, 0, nullptr, nullptr, nullptr, msg_ids, nullptr,
+                                    nullptr, nullptr, ws + L.lm_partial, L.lm_partial_bytes, (float*)(ws + L.lse),
+                                    (cudaStream_t)stream, nullptr, msg_logprob_bf16, ws + L.lm_topk, L.lm_topk_bytes);
+    }
+    if (ctx->ws_bytes < L.end_logits) return MIRROR_ERR_WORKSPACE;
+    // a workspace without room for the candidate lists but with room for the logits: the selection runs over spilled logits
     return mirror_lmhead_launch(ctx, hidden_le, M, W, kappa, nullptr, nullptr, 0, nullptr, nullptr, nullptr, msg_ids, nullptr,
                                 nullptr, (float*)(ws + L.logits), ws + L.lm_partial, L.lm_partial_bytes, (float*)(ws + L.lse),
                                 (cudaStream_t)stream, nullptr, msg_logprob_bf16);

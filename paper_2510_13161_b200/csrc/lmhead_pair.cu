@@ -54,6 +54,10 @@ struct PairParams {
     int* part_idx;
     float* part_sum;
     int* status;
+    int topk;                               // > 0: the epilogue keeps each row's topk best (logit, id) pairs per CTA or unit
+    int topk_bytes;                         // shared memory of those lists
+    float* part_topv;                       // [partials][M][topk]
+    int* part_topi;
     int fp8;                                // 1: W and the hidden rows are e4m3 bytes (K counted in 128-byte blocks all the same)
     const float* w_scale;                   // fp8: [V] scale of each weight row
     const float* h_scale;                   // fp8: [M] scale of each hidden row
@@ -160,6 +164,18 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
                  : "memory");
 }
 
+// Fused Top-kappa (Eq. 6).  Every epilogue warp keeps, for every hidden row, its own sorted list of K (logit, id) pairs in
+// shared memory (order: logit descending, id ascending); lane j owns the lists of the rows in column j of each 32-column
+// group, so 32 rows are updated side by side and nothing is locked.  A list lives as long as the CTA (one row chunk: the CTA
+// meets the same rows in every unit), so after the first tiles only a few logits pass its last entry.
+__device__ __forceinline__ void topk_list_insert(float* lv, int* li, int K, float x, int xi) {
+    int i = K - 1;
+    if (!(x > lv[i] || (x == lv[i] && xi < li[i]))) return;
+    while (i > 0 && (x > lv[i - 1] || (x == lv[i - 1] && xi < li[i - 1]))) { lv[i] = lv[i - 1]; li[i] = li[i - 1]; --i; }
+    lv[i] = x;
+    li[i] = xi;
+}
+
 // kReduce: LM head (row reductions in the epilogue, optional spill).  !kReduce: plain GEMM C = W h^T for the layer
 // projections, split along K when there are fewer tiles than CTA pairs; the epilogue only stores fp32 partial sums.
 template <bool kReduce>
@@ -172,6 +188,8 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
     float* st_max = (float*)((uint8_t*)ctrl + 1024);          // [4][kMaxChunkRows]
     int* st_idx = (int*)(st_max + 4 * kMaxChunkRows);
     float* st_sum = (float*)(st_idx + 4 * kMaxChunkRows);
+    float* tk_val = (float*)((uint8_t*)ctrl + kCtrlBytes);    // [4 warps][chunk_rows][topk]  (only when p.topk > 0)
+    int* tk_idx = (int*)(tk_val + (size_t)4 * p.chunk_rows * p.topk);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t rank = cluster_rank();
@@ -304,8 +322,18 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
                 p.part_max[pbase + row] = m;
                 p.part_idx[pbase + row] = idx;
                 p.part_sum[pbase + row] = s;
+                // each warp's list is a partial list of its own: [4 * CTA + warp][row][topk]
+                for (int w = 0; w < 4 && p.topk > 0; ++w)
+                    for (int i = 0; i < p.topk; ++i) {
+                        const size_t at = (((size_t)blockIdx.x * 4 + w) * p.M + row) * p.topk + i;
+                        p.part_topv[at] = tk_val[((size_t)w * p.chunk_rows + c) * p.topk + i];
+                        p.part_topi[at] = tk_idx[((size_t)w * p.chunk_rows + c) * p.topk + i];
+                    }
             }
         };
+        // this warp's Top-kappa lists start empty: (-inf, no id)
+        float* const my_tv = tk_val + (size_t)q * p.chunk_rows * p.topk;
+        int* const my_ti = tk_idx + (size_t)q * p.chunk_rows * p.topk;
         int ab = 0;
         uint32_t aph = 0;
         bool ok = true;
@@ -314,6 +342,10 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
         const bool running = p.n_chunks == 1;
         if (kReduce && running) {
             for (int c = lane; c < kMaxChunkRows; c += 32) { my_max[c] = -INFINITY; my_idx[c] = 0x7fffffff; my_sum[c] = 0.f; }
+            __syncwarp();
+        }
+        if (kReduce && p.topk > 0) {
+            for (int i = lane; i < p.chunk_rows * p.topk; i += 32) { my_tv[i] = -INFINITY; my_ti[i] = 0x7fffffff; }
             __syncwarp();
         }
         for (int u = pair; u < p.n_units; u += n_pairs) {
@@ -355,6 +387,35 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
 #pragma unroll
                             for (int j = 0; j < 32; ++j)
                                 if (j < ncol) dst[(size_t)j * p.V] = v[j];
+                        }
+                        if (kReduce && p.topk > 0) {
+                            // lane j owns column j's list.  Its last entry is the bar: which lanes hold a logit of column j that
+                            // passes it?  (Nothing to do but for a few tiles.)
+                            const int K = p.topk;
+                            float* const lv = my_tv + (size_t)(cg * 32 + lane) * K;
+                            int* const li = my_ti + (size_t)(cg * 32 + lane) * K;
+                            const float bar_mine = lane < ncol ? lv[K - 1] : INFINITY;
+                            unsigned myhit = 0;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                const float bar_j = __shfl_sync(0xffffffffu, bar_mine, j);
+                                const unsigned hit = __ballot_sync(0xffffffffu, v[j] >= bar_j && v[j] > -INFINITY);
+                                if (lane == j) myhit = hit;
+                            }
+                            // rounds: every owner takes the next lane of its mask; one shuffle per column fetches that logit
+                            while (__any_sync(0xffffffffu, myhit != 0)) {
+                                const int src = myhit ? __ffs(myhit) - 1 : 0;
+                                const bool have = myhit != 0;
+                                myhit &= myhit - 1;
+                                float x = -INFINITY;
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) {
+                                    const float t = __shfl_sync(0xffffffffu, v[j], src);
+                                    if (lane == j) x = t;
+                                }
+                                if (have) topk_list_insert(lv, li, K, x, vid - lane + src);
+                            }
+                            __syncwarp();
                         }
                         if (kReduce) {
 #pragma unroll
@@ -443,7 +504,7 @@ int ctas_per_sm_for(const MirrorTuning& tune, int M) {
 }
 
 // shapes shared by both modes: row chunks, accumulator layout, pipeline depth
-mirror_status pair_shape(const MirrorTuning& tune, int M, int V, int H, PairParams* p, int rows_cta = kTileV) {
+mirror_status pair_shape(const MirrorTuning& tune, int M, int V, int H, PairParams* p, int rows_cta = kTileV, int topk = 0) {
     if (M <= 0 || V <= 0 || H <= 0 || H % kBK != 0) return MIRROR_ERR_SHAPE;
     p->M = M; p->V = V; p->H = H;
     p->n_chunks = (M + kMaxChunkRows - 1) / kMaxChunkRows;
@@ -457,7 +518,11 @@ mirror_status pair_shape(const MirrorTuning& tune, int M, int V, int H, PairPara
     // Few rows (a weight stream): two CTAs per SM with five or six stages each keep more bytes in flight than one CTA with
     // eight, deal the units to twice as many pairs, and let the CTAs of the next kernel move in one by one.
     p->ctas_per_sm = ctas_per_sm_for(tune, M);
-    p->stages = (kSmemBudget / p->ctas_per_sm - kCtrlBytes - 2048) / p->stage_bytes;
+    p->topk = topk;
+    p->topk_bytes = topk > 0 ? (int)align_up((size_t)4 * p->chunk_rows * (size_t)topk * 8, 256) : 0;
+    p->part_topv = nullptr; p->part_topi = nullptr;
+    if (p->topk_bytes > (32 << 10)) p->ctas_per_sm = 1;
+    p->stages = (kSmemBudget / p->ctas_per_sm - kCtrlBytes - 2048 - p->topk_bytes) / p->stage_bytes;
     if (p->stages > kMaxStages) p->stages = kMaxStages;
     if (tune.lm_stages >= 2 && tune.lm_stages < p->stages) p->stages = tune.lm_stages;
     p->wait_limit = tune.wait_limit_cycles;
@@ -485,7 +550,7 @@ mirror_status pair_launch(mirror_ctx* ctx, bool reduce, const void* x, const voi
         st = mirror_make_tmap(ctx, &tm_h, x, 2, hdims, strides, box_h);
         if (st != MIRROR_OK) return st;
     }
-    const size_t smem = (size_t)p.stages * p.stage_bytes + kCtrlBytes + 1024;
+    const size_t smem = (size_t)p.stages * p.stage_bytes + kCtrlBytes + p.topk_bytes + 1024;
     if (!ctx->lm_pair_attr_set) {
         MIRROR_CUDA_OK(cudaFuncSetAttribute(lmhead_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
         MIRROR_CUDA_OK(cudaFuncSetAttribute(linear_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
@@ -515,9 +580,15 @@ mirror_status pair_launch(mirror_ctx* ctx, bool reduce, const void* x, const voi
 
 int mirror_lmhead_pair_partials(int V) { return 2 * ((V + kPairV - 1) / kPairV); }
 
+bool mirror_lmhead_topk_fusable(const mirror_ctx* ctx, int M, int topk) {
+    if (topk <= 0 || M > kMaxChunkRows || M < ctx->tune.lm_pair_min_rows) return false;
+    const size_t bytes = (size_t)4 * align_up((size_t)M, 16) * (size_t)topk * 8;
+    return bytes <= ((size_t)96 << 10);           // (beyond 32 KB the kernel runs one CTA per SM)
+}
+
 mirror_status mirror_lmhead_pair_launch(mirror_ctx* ctx, const void* hidden, int M, const void* W, float* logits_out,
                                         void* partial_ws, size_t partial_bytes, cudaStream_t stream, int* n_partials,
-                                        const float* w_scale, const float* h_scale) {
+                                        const float* w_scale, const float* h_scale, int topk, void* topk_ws, size_t topk_ws_bytes) {
     const bool fp8 = w_scale != nullptr;
     if (fp8 && (!h_scale || ctx->desc.hidden % 128 != 0)) return MIRROR_ERR_SHAPE;
     // (e4m3 rows are staged exactly like bf16 rows of half as many elements: the same bytes, boxes and swizzle)
@@ -537,7 +608,7 @@ mirror_status mirror_lmhead_pair_launch(mirror_ctx* ctx, const void* hidden, int
     }
     const int n_tiles = (V + 2 * rows_cta - 1) / (2 * rows_cta);
     PairParams p;
-    mirror_status st = pair_shape(ctx->tune, M, V, H, &p, rows_cta);
+    mirror_status st = pair_shape(ctx->tune, M, V, H, &p, rows_cta, topk);
     if (st != MIRROR_OK) return st;
     p.n_units = n_tiles * p.n_chunks;
     int n_pairs = ctx->num_sms / 2 * p.ctas_per_sm;
@@ -555,6 +626,13 @@ mirror_status mirror_lmhead_pair_launch(mirror_ctx* ctx, const void* hidden, int
     p.part_idx = (int*)(p.part_max + P * M);
     p.part_sum = (float*)(p.part_idx + P * M);
     p.status = ctx->d_status;
+    if (topk > 0) {
+        // the lists live as long as the CTA: one row chunk only (and four lists per CTA and row have to fit beside the stages)
+        if (p.n_chunks != 1 || p.stages < 3) return MIRROR_ERR_UNSUPPORTED;
+        if (!topk_ws || topk_ws_bytes < 4 * P * M * (size_t)topk * 8) return MIRROR_ERR_WORKSPACE;
+        p.part_topv = (float*)topk_ws;
+        p.part_topi = (int*)(p.part_topv + 4 * P * M * (size_t)topk);
+    }
     p.fp8 = fp8 ? 1 : 0;
     p.w_scale = w_scale;
     p.h_scale = h_scale;

@@ -352,11 +352,13 @@ lmhead_merge_kernel(int M, int P, float inv_T, float inv_T_log2e, const float* p
     }
 }
 
-// Top-kappa of each row from the fp32 logits (Eq. 6): k rounds of "best element strictly after the
-// previous pick" in the order (logit descending, id ascending).  One block per row.
+// Top-kappa of each row (Eq. 6): k rounds of "best element strictly after the previous pick" in the order (logit
+// descending, id ascending).  One block per row.  Either over the row's fp32 logits (cand_id == nullptr: V values, the
+// id is the position), or over the candidate lists that the GEMM's epilogue left: n_part lists of list_k (logit, id)
+// pairs per row, laid out [partial][row][list_k] (empty places hold -inf).
 __global__ void __launch_bounds__(1024, 1)
 lmhead_topk_kernel(int V, int topk, float inv_T, const float* logits, const float* lse, int32_t* topk_id,
-                   float* topk_logprob, __nv_bfloat16* topk_logprob_bf16) {
+                   float* topk_logprob, __nv_bfloat16* topk_logprob_bf16, const int* cand_id, int M, int list_k) {
     ptx::grid_dep_wait();
     ptx::grid_dep_launch();
     __shared__ float s_v[32];
@@ -364,7 +366,9 @@ lmhead_topk_kernel(int V, int topk, float inv_T, const float* logits, const floa
     __shared__ float s_prev_v;
     __shared__ int s_prev_i;
     const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const float* l = logits + (size_t)row * V;
+    const float* l = logits + (size_t)row * (cand_id ? list_k : V);
+    const int* li = cand_id ? cand_id + (size_t)row * list_k : nullptr;
+    const size_t part_stride = (size_t)M * list_k;                 // candidates: from one partial's list to the next
     if (tid == 0) { s_prev_v = INFINITY; s_prev_i = -1; }
     __syncthreads();
     for (int k = 0; k < topk; ++k) {
@@ -372,8 +376,16 @@ lmhead_topk_kernel(int V, int topk, float inv_T, const float* logits, const floa
         const int pi = s_prev_i;
         float bv = -INFINITY;
         int bi = 0x7fffffff;
-        for (int v = tid; v < V; v += blockDim.x) {
-            const float x = l[v];
+        for (int n = tid; n < V; n += blockDim.x) {
+            float x;
+            int v = n;
+            if (li) {
+                const size_t at = (size_t)(n / list_k) * part_stride + (size_t)(n % list_k);
+                x = l[at];
+                v = li[at];
+            } else {
+                x = l[n];
+            }
             const bool after = (x < pv) || (x == pv && v > pi);
             if (after && (x > bv || (x == bv && v < bi))) { bv = x; bi = v; }
         }
@@ -446,7 +458,7 @@ mirror_status lmhead_tail(mirror_ctx* ctx, const void* hidden, int M, const void
                           const int32_t* gather_tok, int n_gather, int32_t* argmax, float* maxlogit, float* lse, int32_t* topk_id,
                           float* topk_logprob, float* gather_logit, float* logits_out, float* lse_scratch, cudaStream_t stream,
                           void* topk_logprob_bf16, int P, float inv_T, float inv_T_log2e, const float* part_max, const int* part_idx,
-                          const float* part_sum) {
+                          const float* part_sum, const float* cand_v = nullptr, const int* cand_i = nullptr) {
     const int V = ctx->desc.vocab, H = ctx->desc.hidden;
     float* lse_dst = lse ? lse : (topk > 0 ? lse_scratch : nullptr);
     if (argmax || maxlogit || lse_dst) {
@@ -456,8 +468,12 @@ mirror_status lmhead_tail(mirror_ctx* ctx, const void* hidden, int M, const void
         MIRROR_CUDA_OK(cudaGetLastError());
     }
     if (topk > 0) {
-        MIRROR_CUDA_OK(mirror_launch_pdl(lmhead_topk_kernel, dim3(M), dim3(1024), 0, stream, V, topk, inv_T, logits_out, lse_dst,
-                                         topk_id, topk_logprob, (__nv_bfloat16*)topk_logprob_bf16));
+        if (cand_v)      // (four lists per partial: one per epilogue warp)
+            MIRROR_CUDA_OK(mirror_launch_pdl(lmhead_topk_kernel, dim3(M), dim3(1024), 0, stream, 4 * P * topk, topk, inv_T, cand_v, lse_dst,
+                                             topk_id, topk_logprob, (__nv_bfloat16*)topk_logprob_bf16, cand_i, M, topk));
+        else
+            MIRROR_CUDA_OK(mirror_launch_pdl(lmhead_topk_kernel, dim3(M), dim3(1024), 0, stream, V, topk, inv_T, (const float*)logits_out,
+                                             lse_dst, topk_id, topk_logprob, (__nv_bfloat16*)topk_logprob_bf16, (const int*)nullptr, M, 0));
         ctx->launches += 1;
         MIRROR_CUDA_OK(cudaGetLastError());
     }
@@ -479,14 +495,19 @@ mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, c
                                    int32_t* argmax, float* maxlogit, float* lse, int32_t* topk_id,
                                    float* topk_logprob, float* gather_logit, float* logits_out,
                                    void* partial_ws, size_t partial_bytes, float* lse_scratch, cudaStream_t stream,
-                                   cudaEvent_t after_gemm, void* topk_logprob_bf16) {
+                                   cudaEvent_t after_gemm, void* topk_logprob_bf16, void* topk_ws, size_t topk_ws_bytes) {
     const int V = ctx->desc.vocab, H = ctx->desc.hidden;
+    // Top-kappa inside the GEMM's epilogue whenever the caller's scratch holds the candidate lists; otherwise (or on the
+    // single-CTA fallback kernel) the selection runs over spilled logits, which then have to be there.
+    const bool fused_topk = topk > 0 && topk_ws != nullptr;
+    if (topk > 0 && !fused_topk && !logits_out) return MIRROR_ERR_WORKSPACE;
     // The GEMM runs on CTA pairs (lmhead_pair.cu) whenever the partials it leaves fit the scratch it was given; the
     // single-CTA weight-stream kernel below is the fallback (and what MIRROR_LM_PAIR_MIN_ROWS can force for comparison).
     const int pair_min_rows = ctx->tune.lm_pair_min_rows;
     if (M >= pair_min_rows && ctx->num_sms >= 2) {
         int P = 0;
-        mirror_status st = mirror_lmhead_pair_launch(ctx, hidden, M, W, logits_out, partial_ws, partial_bytes, stream, &P);
+        mirror_status st = mirror_lmhead_pair_launch(ctx, hidden, M, W, logits_out, partial_ws, partial_bytes, stream, &P, nullptr,
+                                                     nullptr, fused_topk ? topk : 0, topk_ws, topk_ws_bytes);
         if (st == MIRROR_OK) {
             if (after_gemm) MIRROR_CUDA_OK(cudaEventRecord(after_gemm, stream));
             const float inv_T = 1.0f / ctx->temperature, inv_T_log2e = inv_T * 1.4426950408889634f;
@@ -495,10 +516,12 @@ mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, c
             float* part_sum = (float*)(part_idx + (size_t)P * M);
             return lmhead_tail(ctx, hidden, M, W, topk, gather_row, gather_tok, n_gather, argmax, maxlogit, lse, topk_id, topk_logprob,
                                gather_logit, logits_out, lse_scratch, stream, topk_logprob_bf16, P, inv_T, inv_T_log2e, part_max,
-                               part_idx, part_sum);
+                               part_idx, part_sum, fused_topk ? (const float*)topk_ws : nullptr,
+                               fused_topk ? (const int*)((const float*)topk_ws + (size_t)4 * P * M * topk) : nullptr);
         }
         if (st != MIRROR_ERR_WORKSPACE) return st;
     }
+    if (topk > 0 && !logits_out) return MIRROR_ERR_WORKSPACE;       // the single-CTA kernel selects from spilled logits only
     LmParams p;
     p.M = M; p.V = V; p.H = H;
     p.n_chunks = (M + kMaxChunkRows - 1) / kMaxChunkRows;
@@ -576,14 +599,20 @@ extern "C" mirror_status mirror_lmhead_reduce(mirror_ctx* ctx, const void* hidde
     mirror_ws_layout(ctx, (size_t)M, &L);
     size_t need = L.end_lmhead;
     float* lse_scratch = (float*)((uint8_t*)ctx->ws + L.lse);
-    if (topk > 0 && !logits_out) {
-        logits_out = (float*)((uint8_t*)ctx->ws + L.logits);
-        need = L.end_logits;
+    void* topk_ws = nullptr;
+    if (topk > 0) {
+        if (L.lm_topk_bytes && ctx->ws_bytes >= L.end_topk && mirror_lmhead_topk_fusable(ctx, M, topk)) {
+            topk_ws = (uint8_t*)ctx->ws + L.lm_topk;       // Top-kappa inside the GEMM's epilogue: no [M, V] buffer
+            need = L.end_topk;
+        } else if (!logits_out) {
+            logits_out = (float*)((uint8_t*)ctx->ws + L.logits);
+            need = L.end_logits;
+        }
     }
     if (ctx->ws_bytes < need) return MIRROR_ERR_WORKSPACE;
     return mirror_lmhead_launch(ctx, hidden, M, W, topk, gather_row, gather_tok, n_gather, argmax, maxlogit, lse, topk_id,
                                 topk_logprob, gather_logit, logits_out, (uint8_t*)ctx->ws + L.lm_partial, L.lm_partial_bytes, lse_scratch,
-                                (cudaStream_t)stream);
+                                (cudaStream_t)stream, nullptr, nullptr, topk_ws, L.lm_topk_bytes);
 }
 
 // ---------------------------------------------------------------------------------------------------

@@ -75,7 +75,8 @@ struct MirrorWsLayout {
     size_t lse = 0, argmax = 0;                          // [M] scratch each
     size_t logits = 0, logits_bytes = 0;                 // fp32 [M, V]
     size_t accept_scratch = 0;                           // fp64 [B, 2, V]: running distribution of the tree acceptance
-    size_t end_attn = 0, end_lmhead = 0, end_logits = 0, end_accept = 0;   // bytes needed up to each region
+    size_t lm_topk = 0, lm_topk_bytes = 0;               // per partial and row: the MIRROR_MAX_TOPK best (logit, id) pairs of the fused Top-kappa
+    size_t end_attn = 0, end_lmhead = 0, end_logits = 0, end_accept = 0, end_topk = 0;   // bytes needed up to each region
 };
 void mirror_ws_layout(const mirror_ctx* ctx, size_t M, MirrorWsLayout* out, size_t B = 0);
 
@@ -87,14 +88,19 @@ mirror_status mirror_lmhead_launch(mirror_ctx* ctx, const void* hidden, int M, c
                                    int32_t* argmax, float* maxlogit, float* lse, int32_t* topk_id,
                                    float* topk_logprob, float* gather_logit, float* logits_out,
                                    void* partial_ws, size_t partial_bytes, float* lse_scratch, cudaStream_t stream,
-                                   cudaEvent_t after_gemm = nullptr, void* topk_logprob_bf16 = nullptr);
+                                   cudaEvent_t after_gemm = nullptr, void* topk_logprob_bf16 = nullptr,
+                                   void* topk_ws = nullptr, size_t topk_ws_bytes = 0);
 // LM-head GEMM + per-unit row partials on CTA pairs (many hidden rows); *n_partials partials of [M] rows are left in
 // partial_ws for lmhead_merge_kernel.  mirror_lmhead_pair_partials(V) is that count.
 int mirror_lmhead_pair_partials(int V);
+// Can the Top-kappa of M rows be selected inside the GEMM's epilogue?  (One row chunk, and four lists per CTA and row in
+// shared memory beside a pipeline that is still deep enough.)
+bool mirror_lmhead_topk_fusable(const mirror_ctx* ctx, int M, int topk);
 // w_scale / h_scale non-null: W and hidden are e4m3 bytes with one scale per row (the GEMM runs on kind::f8f6f4).
 mirror_status mirror_lmhead_pair_launch(mirror_ctx* ctx, const void* hidden, int M, const void* W, float* logits_out,
                                         void* partial_ws, size_t partial_bytes, cudaStream_t stream, int* n_partials,
-                                        const float* w_scale = nullptr, const float* h_scale = nullptr);
+                                        const float* w_scale = nullptr, const float* h_scale = nullptr,
+                                        int topk = 0, void* topk_ws = nullptr, size_t topk_ws_bytes = 0);
 // Plain GEMM on CTA pairs: partial[s][M][N] (fp32) = x[M, K-slice s] * W[N, K-slice s]^T for the *k_slices slices that
 // mirror_linear_slices() picks (1 when the output tiles alone fill the GPU); the caller adds the slices in order.
 int mirror_linear_slices(const mirror_ctx* ctx, int M, int N, int K);
