@@ -160,6 +160,33 @@ mirror_status mirror_attn_verify(mirror_ctx* ctx, const mirror_kv* kv, const mir
                                  const void* q, const void* k_new, const void* v_new,
                                  void* out, float* lse_out, void* stream);
 
+/* The same attention over an 8-bit cache.  The paper states no storage precision for the target's cache (Sec. 3,
+ * Eq. 1); this mode is the library's own option and halves the bytes the step reads.  Its definition:
+ *   kv->k_pool, kv->v_pool, k_new, v_new hold e4m3 codes (one byte per element; same shapes, kv->layer_stride counts
+ *   elements), value = code * scale[layer, KV head] with k_scale, v_scale: device fp32 [L, Hkv];
+ *   the queries enter as q8 = q_scale * e4m3(q / q_scale) (q stays bf16 in memory; q_scale: host fp32 > 0, one for
+ *   the call, e.g. max|q| / 448; fp32 division, round to nearest even, saturating);
+ *   out = softmax(scale * q8 (k_scale K)^T) (v_scale V) over the same visible set.
+ * Inside, the unnormalised softmax weights are rounded to e4m3 too (both operands of an 8-bit tensor-core product are
+ * 8-bit), relative to a running offset per row: weights below 2^-12 of it round to zero; the row sum, and so lse_out,
+ * is taken before that rounding.  Head dimension 128 only (MIRROR_ERR_UNSUPPORTED otherwise); q, out, lse_out and
+ * the workspace as for mirror_attn_verify. */
+mirror_status mirror_attn_verify_fp8(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const void* q,
+                                     const void* k_new_fp8, const void* v_new_fp8, const float* k_scale,
+                                     const float* v_scale, float q_scale, void* out, float* lse_out, void* stream);
+
+/* Scales and codes of a bf16 K or V tensor for that cache.  The tensor is addressed as [layer][...][head][inner]:
+ * `inner` consecutive elements (a multiple of 8) belong to one KV head -- page_size * d for a pool, d for the tree's
+ * own k_new / v_new -- and heads cycle above that; `layer_elems` elements of each layer are in use, layers are
+ * `layer_stride` elements apart (codes are written at the same element offsets).
+ *   mirror_kv_scales_fp8:   scale[layer, head] = max|x| / 448 over the layer's and head's elements (1 if all zero)
+ *   mirror_kv_quantize_fp8: code = e4m3(x / scale[layer, head]), fp32 division, round to nearest even, saturating
+ * x: device bf16, 16-byte aligned; scale: device fp32 [n_layers, Hkv]; out_fp8: device bytes, 8-byte aligned. */
+mirror_status mirror_kv_scales_fp8(mirror_ctx* ctx, const void* x, int n_layers, int64_t layer_stride, int64_t layer_elems,
+                                   int inner, float* scale, void* stream);
+mirror_status mirror_kv_quantize_fp8(mirror_ctx* ctx, const void* x, int n_layers, int64_t layer_stride,
+                                     int64_t layer_elems, int inner, const float* scale, void* out_fp8, void* stream);
+
 /* LM head with fused row reductions: logits[r][v] = sum_k hidden[r][k] * W[v][k]  (Eq. 1, Eq. 5).
  *   hidden bf16 [M, H] (row stride H);  W bf16 [V, H]
  *   argmax   int32 [M]  lowest id attaining the maximum          (nullable)

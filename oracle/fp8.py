@@ -1,4 +1,4 @@
-"""CPU oracle of the low-precision LM head: the e4m3 rounding model of its operands.
+"""CPU oracle of the low-precision modes: the e4m3 rounding model of the LM head's operands and of the KV cache.
 
 TEST INFRASTRUCTURE ONLY: imported by tests/ (and nothing in the CUDA package).  Plain numpy.
 
@@ -9,6 +9,13 @@ format with 4 exponent bits (bias 7), 3 mantissa bits, subnormals, no infinities
 rounding to nearest with ties to the even mantissa, values beyond 448 saturating.  The scale and the quotient are
 computed in fp32 (that decides the 8-bit code, so both sides take that decision in the same precision); everything
 after the rounding is fp64: logits = (scale_w * scale_h) * sum_k code_w[k] * code_h[k].
+
+The 8-bit KV cache (also this build's own option: Section 3 and Eq. 1 state no storage precision) keeps one scale per
+(layer, KV head): scale = max|x| / 448 over that layer's and head's K (or V) elements, codes as above.  Attention over
+such a cache is the plain branch-tree attention of the decoded values, K = scale_k * code, V = scale_v * code, with the
+queries rounded the same way under one scale for the call (q8 = q_scale * e4m3(q / q_scale)) and fp64 arithmetic after
+the rounding: attention_layer_fp8 feeds the decoded codes (exact in bf16) to the C oracle head by head, folding
+scale_k * q_scale into the score scale and multiplying the output by scale_v.
 
 Pins (tests/test_oracle_fp8.py): all 256 code points decode to the values of the format's definition and encode back to
 themselves; hand-picked ties; saturation; subnormals; monotonicity; values exactly representable are recovered, so the
@@ -66,3 +73,55 @@ def lmhead_logits_fp8(h_codes, h_scale, w_codes, w_scale) -> np.ndarray:
     w = e4m3_decode(w_codes)
     acc = h @ w.T
     return acc * (np.asarray(h_scale, np.float64)[:, None] * np.asarray(w_scale, np.float64)[None, :])
+
+
+def kv_scales(x: np.ndarray, head_axis: int) -> np.ndarray:
+    """x [L, ..., Hkv, ...] (values exact in fp32) -> fp32 scales [L, Hkv]: max|x| / 448 per layer and head (1 if zero)."""
+    x32 = np.abs(np.asarray(x, np.float32))
+    axes = tuple(a for a in range(x32.ndim) if a not in (0, head_axis))
+    amax = x32.max(axis=axes)
+    return np.where(amax > 0, amax / np.float32(448.0), np.float32(1.0)).astype(np.float32)
+
+
+def kv_quantize(x: np.ndarray, scale: np.ndarray, head_axis: int) -> np.ndarray:
+    """e4m3 codes of x under scale [L, Hkv] (fp32 division, round to nearest even, saturating)."""
+    x32 = np.asarray(x, np.float32)
+    shape = [1] * x32.ndim
+    shape[0], shape[head_axis] = scale.shape
+    ratio = (x32 / np.asarray(scale, np.float32).reshape(shape)).astype(np.float32)
+    return e4m3_encode(ratio.astype(np.float64))
+
+
+def _codes_as_bf16_bits(codes: np.ndarray) -> np.ndarray:
+    """e4m3 values have 4 significant bits: exact in bf16."""
+    v = e4m3_decode(codes).astype(np.float32)
+    return (v.view(np.uint32) >> 16).astype(np.uint16)
+
+
+def quantize_tensor(x: np.ndarray, scale: float) -> np.ndarray:
+    """e4m3 codes of x under one scale (fp32 division, round to nearest even, saturating)."""
+    ratio = (np.asarray(x, np.float32) / np.float32(scale)).astype(np.float32)
+    return e4m3_encode(ratio.astype(np.float64))
+
+
+def attention_layer_fp8(q_codes, q_scale: float, k_codes, v_codes, k_scale, v_scale, page_table, prefix_len, k_new_codes,
+                        v_new_codes, anc, scale: float):
+    """Branch-tree attention of one layer over an e4m3 cache.  q_codes uint8 [B,n,Hq,d]; k_codes / v_codes uint8
+    [pages,Hkv,P,d]; k_new_codes / v_new_codes uint8 [B,n,Hkv,d]; k_scale / v_scale fp32 [Hkv].
+    Returns (out [B,n,Hq,d], lse [B,Hq,n]) in fp64."""
+    from oracle import oracle as O
+    q_bits = _codes_as_bf16_bits(q_codes)
+    B, n, Hq, d = q_bits.shape
+    Hkv = k_codes.shape[1]
+    G = Hq // Hkv
+    out = np.zeros((B, n, Hq, d), np.float64)
+    lse = np.zeros((B, Hq, n), np.float64)
+    for g in range(Hkv):
+        o_g, lse_g, _ = O.attention_layer(
+            np.ascontiguousarray(q_bits[:, :, g * G:(g + 1) * G]),
+            _codes_as_bf16_bits(k_codes[:, g:g + 1]), _codes_as_bf16_bits(v_codes[:, g:g + 1]), page_table, prefix_len,
+            _codes_as_bf16_bits(k_new_codes[:, :, g:g + 1]), _codes_as_bf16_bits(v_new_codes[:, :, g:g + 1]), anc,
+            scale * float(k_scale[g]) * float(np.float32(q_scale)))
+        out[:, :, g * G:(g + 1) * G] = o_g * float(v_scale[g])
+        lse[:, g * G:(g + 1) * G] = lse_g
+    return out, lse

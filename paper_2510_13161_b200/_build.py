@@ -12,7 +12,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 OBJ_DIR = os.path.join(ROOT, "build", "obj")
 LIB = os.path.join(HERE, "libmirror.so")
-SOURCES = ["ctx.cu", "accept_select.cu", "lmhead_reduce.cu", "attn_verify.cu", "verify_step.cu", "early_exit.cu", "kv_commit.cu", "lmhead_pair.cu", "target_layer.cu"]
+SOURCES = ["ctx.cu", "accept_select.cu", "lmhead_reduce.cu", "attn_verify.cu", "verify_step.cu", "early_exit.cu", "kv_commit.cu", "lmhead_pair.cu", "target_layer.cu", "kv_fp8.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC]
 

@@ -27,6 +27,7 @@ EXPORTS = [
     "mirror_device_status", "mirror_launch_count", "mirror_status_str", "mirror_set_stage_events",
     "mirror_lmhead_reduce_noalloc", "mirror_lmhead_noalloc_status", "mirror_quantize_rows_fp8", "mirror_lmhead_reduce_fp8", "mirror_early_exit_tap", "mirror_overlap_mass", "mirror_kv_commit",
     "mirror_linear_scratch_bytes", "mirror_linear", "mirror_rmsnorm", "mirror_target_scratch_bytes", "mirror_target_forward", "mirror_trie_build", "mirror_verify_step_host", "mirror_embed_rows",
+    "mirror_attn_verify_fp8", "mirror_kv_scales_fp8", "mirror_kv_quantize_fp8",
 ]
 
 
@@ -254,6 +255,51 @@ class Mirror:
                                            _ptr(k_new, torch.bfloat16, "k_new"), _ptr(v_new, torch.bfloat16, "v_new"),
                                            _ptr(out, torch.bfloat16, "out"), _ptr(lse_out, torch.float32, "lse_out"),
                                            _stream(stream)), "mirror_attn_verify")
+        return out
+
+    # ---- e4m3 cache ----------------------------------------------------------------------------
+    def kv_fp8(self, k_codes: torch.Tensor, v_codes: torch.Tensor, page_table: torch.Tensor, prefix_len: torch.Tensor) -> KV:
+        """k_codes / v_codes: uint8 e4m3 codes [L, num_pages, Hkv, page, d] (one allocation, layers consecutive)."""
+        L, num_pages = k_codes.shape[0], k_codes.shape[1]
+        stride = k_codes.stride(0) if L > 1 else k_codes[0].numel()
+        kv = KV(_ptr(k_codes, torch.uint8, "k_codes"), _ptr(v_codes, torch.uint8, "v_codes"), stride, L, num_pages,
+                page_table.shape[1], _ptr(page_table, torch.int32, "page_table"), _ptr(prefix_len, torch.int32, "prefix_len"))
+        kv._refs = (k_codes, v_codes, page_table, prefix_len)
+        return kv
+
+    def _kv_fp8_dims(self, x: torch.Tensor, inner: int):
+        L = x.shape[0]
+        layer_elems = x[0].numel()
+        stride = x.stride(0) if L > 1 else layer_elems
+        return L, stride, layer_elems, inner
+
+    def mirror_kv_scales_fp8(self, x: torch.Tensor, inner: int, stream=None) -> torch.Tensor:
+        """x bf16 [L, ..., Hkv, <inner elements>] -> fp32 scales [L, Hkv] (max|x| / 448 per layer and KV head)."""
+        L, stride, layer_elems, inner = self._kv_fp8_dims(x, inner)
+        scale = torch.empty((L, self.desc.n_kv_heads), dtype=torch.float32, device=x.device)
+        _check(self.lib.mirror_kv_scales_fp8(self._ctx, _ptr(x, torch.bfloat16, "x"), L, C.c_int64(stride), C.c_int64(layer_elems),
+                                             inner, _ptr(scale, torch.float32, "scale"), _stream(stream)), "mirror_kv_scales_fp8")
+        return scale
+
+    def mirror_kv_quantize_fp8(self, x: torch.Tensor, inner: int, scale: torch.Tensor, stream=None) -> torch.Tensor:
+        """x bf16 -> e4m3 codes (uint8, same shape) under the given [L, Hkv] scales."""
+        L, stride, layer_elems, inner = self._kv_fp8_dims(x, inner)
+        out = torch.empty(x.shape, dtype=torch.uint8, device=x.device)
+        _check(self.lib.mirror_kv_quantize_fp8(self._ctx, _ptr(x, torch.bfloat16, "x"), L, C.c_int64(stride), C.c_int64(layer_elems),
+                                               inner, _ptr(scale, torch.float32, "scale"), _ptr(out, torch.uint8, "out"),
+                                               _stream(stream)), "mirror_kv_quantize_fp8")
+        return out
+
+    def mirror_attn_verify_fp8(self, kv: KV, tree: Tree, q, k_new8, v_new8, k_scale, v_scale, q_scale: float, out=None,
+                               lse_out=None, stream=None):
+        if out is None:
+            out = torch.empty_like(q)
+        self.ensure_workspace(tree, kv, WS_ATTN)
+        _check(self.lib.mirror_attn_verify_fp8(self._ctx, C.byref(kv), C.byref(tree), _ptr(q, torch.bfloat16, "q"),
+                                               _ptr(k_new8, torch.uint8, "k_new8"), _ptr(v_new8, torch.uint8, "v_new8"),
+                                               _ptr(k_scale, torch.float32, "k_scale"), _ptr(v_scale, torch.float32, "v_scale"),
+                                               C.c_float(q_scale), _ptr(out, torch.bfloat16, "out"),
+                                               _ptr(lse_out, torch.float32, "lse_out"), _stream(stream)), "mirror_attn_verify_fp8")
         return out
 
     def mirror_lmhead_reduce(self, hidden, W, topk: int = 0, gather_row=None, gather_tok=None, want_lse: bool = True,

@@ -52,8 +52,13 @@ constexpr int kRows = 128;                          // UMMA M: rows per row bloc
 constexpr int kMaxBatch = 1024;
 constexpr int kMaxStages = 8;                       // ring depths are template parameters (even: tiles are staged in pairs)
 constexpr int kSBufs = 4;                           // S buffers in TMEM (power of two)
-constexpr float kOffsetBias = 0.0f;                 // a row's offset puts the maximum of the tile that set it at 2^0 ...
-constexpr float kSumLimit = 16384.0f;               // ... and moves when a tile's sum of P passes 2^14 (no single P is beyond 2^14 then)
+// A row's offset puts the maximum of the tile that set it at 2^bias and moves when a tile's sum of P passes the limit
+// (no single P is beyond the limit then).  bf16 P: 2^0 and 2^14.  e4m3 P: 2^2 and 448, the largest e4m3 value (a tile
+// of 64 equal scores sums to 256); weights below 2^-12 of the maximum that set the offset round to zero.
+template <bool F8> struct POffset {
+    static constexpr float kBias = F8 ? 2.0f : 0.0f;
+    static constexpr float kSumLimit = F8 ? 448.0f : 16384.0f;
+};
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kTmemCols = 512;                      // S0..S3 (64 columns each; P overwrites the first 32 of its S) | O of group 0 | O of group 1
 constexpr int kTmemO = kSBufs * kTileTok;
@@ -83,6 +88,11 @@ struct AttnParams {
     float* lse_out;
     float* partial;                       // [grid][2][D+4][128]
     int* status;
+    // e4m3 cache: pools, k_new and v_new hold e4m3 codes (one byte per element); a code times its (layer, KV head)
+    // scale is the value.  Q stays bf16 in memory; its operand is e4m3(q / q_scale), rounded when it is staged.
+    const float* k_scale;                 // [L, Hkv]
+    const float* v_scale;                 // [L, Hkv]
+    float q_scale;
     long long wait_limit;                 // SM cycles after which a wait gives up
     int stall_after;                      // test aid: the K producer stops after this many stages (-1: never)
 };
@@ -150,15 +160,64 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// Four fp32 values as e4m3 codes in one word (element 0 in the lowest byte, as the tensor core reads an 8-bit operand);
+// values beyond +-448 saturate.
+__device__ __forceinline__ uint32_t pack_e4m3x4(float a, float b, float c, float d) {
+    uint32_t r;
+    asm("{\n\t.reg .b16 lo, hi;\n\t"
+        "cvt.rn.satfinite.e4m3x2.f32 lo, %2, %1;\n\t"
+        "cvt.rn.satfinite.e4m3x2.f32 hi, %4, %3;\n\t"
+        "mov.b32 %0, {lo, hi};\n\t}"
+        : "=r"(r) : "f"(a), "f"(b), "f"(c), "f"(d));
+    return r;
+}
+// tcgen05.mma with both operands in shared memory (descriptor halves) or A in tensor memory; F8 selects e4m3 inputs.
+template <bool F8>
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                        uint32_t idesc, uint32_t accumulate) {
+    if constexpr (F8) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+            "mov.b64 da, {%1, %2};\n\t"
+            "mov.b64 db, {%3, %4};\n\t"
+            "setp.ne.b32 p, %6, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], da, db, %5, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+            : "memory");
+    } else {
+        ptx::umma_f16_lohi(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
+    }
+}
+template <bool F8>
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                        uint32_t accumulate) {
+    if constexpr (F8) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+            "mov.b64 db, {%2, %3};\n\t"
+            "setp.ne.b32 p, %5, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], [%1], db, %4, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+            : "memory");
+    } else {
+        ptx::umma_f16_tmem_a(d_tmem, a_tmem, b_lo, b_hi, idesc, accumulate);
+    }
+}
+// Instruction descriptor: e4m3 x e4m3 -> fp32 (format codes 0), tile M x N.
+__device__ __forceinline__ uint32_t umma_idesc_e4m3(int M, int N) {
+    return (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
 // Shared-memory operand tiles are [64-column half][row][128 B] with the 128-byte swizzle: the 16-byte chunk
 // index is XORed with (row % 8).  A half of Q or P holds 128 rows (16 KB), a half of a K/V stage 64 tokens (8 KB).
 constexpr int kStageSlots = 4;                      // slots per ring stage
 // A K/V slot (16 tokens of one head) is [token / 8][64-column half][token % 8][128 B]: the 8-token groups of one half
 // are 1024 * (d / 64) bytes apart, uniformly across the slots of a ring, which is the 8-row-group stride (SBO) of the
 // K-major Q K^T operand over up to 128 tokens and, with the halves 1024 B apart (LBO), the MN-major P V operand.
-template <int D>
+// (An e4m3 row of 128 elements is a single 128-byte half.)
+template <int HALVES>
 __device__ __forceinline__ uint32_t kv_slot_off(int tok, int chunk) {                 // chunk: 16-byte column chunk
-    return (uint32_t)((tok >> 3) * (D / 64) * 1024 + (chunk >> 3) * 1024 + (tok & 7) * 128 + (((chunk & 7) ^ (tok & 7)) << 4));
+    return (uint32_t)((tok >> 3) * HALVES * 1024 + (chunk >> 3) * 1024 + (tok & 7) * 128 + (((chunk & 7) ^ (tok & 7)) << 4));
 }
 __device__ __forceinline__ uint32_t tile_off(int row, int chunk, int half_bytes) {   // chunk: 16-byte column chunk
     return (uint32_t)((chunk >> 3) * half_bytes + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
@@ -175,12 +234,23 @@ __device__ __forceinline__ void tmem_st_32x32b_x32(uint32_t taddr, const uint32_
           "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
         : "memory");
 }
+__device__ __forceinline__ void tmem_st_32x32b_x16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 
-template <int D>
+template <int D, bool F8>
 struct Cfg {
-    static constexpr int kHalves = D / 64;
+    static_assert(!F8 || D == 128, "an e4m3 row must fill a 128-byte swizzle row");
+    static constexpr int kElemBytes = F8 ? 1 : 2;
+    static constexpr int kRowBytes = D * kElemBytes;               // one token's K (or V) row of one head
+    static constexpr int kHalves = kRowBytes / 128;
     static constexpr int kSlotBytes = kHalves * kSlotTok * 128;    // one slot of K or V (see kv_slot_off) = one TMA box
     static constexpr int kGroupStride = kHalves * 1024;            // between the 8-token groups of one half
     static constexpr int kStageBytes = kStageSlots * kSlotBytes;   // one K (or V) stage: 4 slots; stages are contiguous
@@ -283,11 +353,12 @@ __device__ __noinline__ long long group_begin(const Partition& q, int g, const A
     return dist <= q.snap_tol ? best : e;
 }
 
-template <int D, int KS, int VS>
+template <int D, int KS, int VS, bool F8>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                    const __grid_constant__ AttnTree tree, const AttnParams p) {
-    using C = Cfg<D>;
+    using C = Cfg<D, F8>;
+    using PO = POffset<F8>;
     constexpr int KR = KS;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -383,14 +454,14 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 // the unit's last slots (a ragged page, the tree's own tokens) are staged by plain loads many tiles
                 // from now: pull them into L2 so that those loads do not hold up the ring for an HBM round trip
                 for (int j = lane; j < p.n; j += 32) {
-                    const __nv_bfloat16* row = (vrole ? p.v_new : p.k_new) + ((((size_t)u.layer * p.B + u.b) * p.n + j) * p.Hkv + u.g) * (size_t)D;
+                    const uint8_t* row = (const uint8_t*)(vrole ? p.v_new : p.k_new) + ((((size_t)u.layer * p.B + u.b) * p.n + j) * p.Hkv + u.g) * (size_t)C::kRowBytes;
                     ptx::prefetch_l2(row);
-                    if (D == 128) ptx::prefetch_l2(row + 64);
+                    if (C::kRowBytes == 256) ptx::prefetch_l2(row + 128);
                 }
                 if (sg.pages_all > sg.pages_full) {
                     const int page = pt[sg.pages_full];
-                    if (page >= 0 && page < p.num_pages && lane < kSlotTok * D * 2 / 128)
-                        ptx::prefetch_l2((vrole ? p.v_pool : p.k_pool) + (((size_t)u.layer * p.layer_pages + page) * p.Hkv + u.g) * (size_t)(kSlotTok * D) + lane * 64);
+                    if (page >= 0 && page < p.num_pages && lane < kSlotTok * C::kRowBytes / 128)
+                        ptx::prefetch_l2((const uint8_t*)(vrole ? p.v_pool : p.k_pool) + (((size_t)u.layer * p.layer_pages + page) * p.Hkv + u.g) * (size_t)(kSlotTok * C::kRowBytes) + lane * 128);
                 }
             }
             for (int t = sg.t_first; t < sg.t_last && ok; ++t, ++x, ++it) {
@@ -406,38 +477,40 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 const int sl0 = t * kStageSlots;
                 const int n_slots = max(0, min(kStageSlots, sg.slots_all - sl0));      // slots that exist in this stage
                 const int n_tma = max(0, min(kStageSlots, sg.pages_full - sl0));       // leading slots that are whole pages
-                const int n_fill = n_slots;
+                // (e4m3: a P V step spans two slots, so an odd last slot gets a partner of zeros: stale bytes could be NaN codes)
+                const int n_fill = F8 ? min(kStageSlots, (n_slots + 1) & ~1) : n_slots;
                 if (n_tma < n_fill) {
                     // ragged page and tree tokens by asynchronous 16-byte copies (rows beyond the valid count are
                     // zero-filled), all in flight together; the loops are kept rolled: this path runs once per unit, and
                     // what it costs is mostly the instruction fetch
-                    constexpr int kChunks = kSlotTok * D / 8;          // 16-byte chunks per slot
+                    constexpr int kRowChunks = C::kRowBytes / 16;      // 16-byte chunks per token row
+                    constexpr int kChunks = kSlotTok * kRowChunks;     // ... and per slot
                     constexpr int kPer = kChunks / 32;
 #pragma unroll 1
                     for (int j = n_tma; j < n_fill; ++j) {
                         const int sl = sl0 + j;
-                        const __nv_bfloat16* src = p.k_pool;
+                        const uint8_t* src = (const uint8_t*)p.k_pool;             // (bytes)
                         size_t row_stride = 0;
                         int valid = 0;
                         if (sl < sg.pages_all) {
                             int page = pt[sl];
                             if (page < 0 || page >= p.num_pages) { if (lane == 0) dev_check(p, 401); page = 0; }
-                            src = (vrole ? p.v_pool : p.k_pool) + (((size_t)u.layer * p.layer_pages + page) * p.Hkv + u.g) * (size_t)(kSlotTok * D);
-                            row_stride = D;
+                            src = (const uint8_t*)(vrole ? p.v_pool : p.k_pool) + (((size_t)u.layer * p.layer_pages + page) * p.Hkv + u.g) * (size_t)(kSlotTok * C::kRowBytes);
+                            row_stride = C::kRowBytes;
                             valid = sg.len - sg.pages_full * kSlotTok;
-                        } else {
+                        } else if (sl < sg.slots_all) {
                             const int j0 = (sl - sg.pages_all) * kSlotTok;
-                            src = (vrole ? p.v_new : p.k_new) + ((((size_t)u.layer * p.B + u.b) * p.n + j0) * p.Hkv + u.g) * (size_t)D;
-                            row_stride = (size_t)p.Hkv * D;
+                            src = (const uint8_t*)(vrole ? p.v_new : p.k_new) + ((((size_t)u.layer * p.B + u.b) * p.n + j0) * p.Hkv + u.g) * (size_t)C::kRowBytes;
+                            row_stride = (size_t)p.Hkv * C::kRowBytes;
                             valid = min(kSlotTok, p.n - j0);
                         }
 #pragma unroll 1
                         for (int i = 0; i < kPer; ++i) {
-                            const int c = lane + i * 32, tr = c / (D / 8), cc = c % (D / 8);
+                            const int c = lane + i * 32, tr = c / kRowChunks, cc = c % kRowChunks;
                             const bool in = tr < valid;
                             asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
-                                         ::"r"(ptx::smem_u32(dst + j * C::kSlotBytes + kv_slot_off<D>(tr, cc))),
-                                           "l"(in ? src + tr * row_stride + cc * 8 : p.k_pool), "r"(in ? 16u : 0u) : "memory");
+                                         ::"r"(ptx::smem_u32(dst + j * C::kSlotBytes + kv_slot_off<C::kHalves>(tr, cc))),
+                                           "l"(in ? src + tr * row_stride + cc * 16 : (const uint8_t*)p.k_pool), "r"(in ? 16u : 0u) : "memory");
                         }
                     }
                     asm volatile("cp.async.wait_all;" ::: "memory");
@@ -491,12 +564,12 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     ptx::tc_fence_after();
                     const int n_sl = min(kStageSlots, sg.slots_all - t * kStageSlots);       // (a pair's second tile may be empty)
                     if (n_sl > 0) {
-                        const uint32_t idesc = ptx::umma_idesc_bf16(kRows, n_sl * kSlotTok);
+                        const uint32_t idesc = F8 ? umma_idesc_e4m3(kRows, n_sl * kSlotTok) : ptx::umma_idesc_bf16(kRows, n_sl * kSlotTok);
                         const uint32_t kb = k_lo + (uint32_t)((st * C::kStageBytes) >> 4);
                         const uint32_t d = tmem_base + (uint32_t)(sb * kTileTok);
 #pragma unroll
-                        for (int kk = 0; kk < D / 16; ++kk)
-                            ptx::umma_f16_lohi(d, q_seg + (uint32_t)(((kk >> 2) * p.q_half_bytes + (kk & 3) * 32) >> 4), hi_q,
+                        for (int kk = 0; kk < C::kRowBytes / 32; ++kk)          // 32 bytes of every row per instruction
+                            umma_ss<F8>(d, q_seg + (uint32_t)(((kk >> 2) * p.q_half_bytes + (kk & 3) * 32) >> 4), hi_q,
                                                kb + (uint32_t)(((kk >> 2) * 1024 + (kk & 3) * 32) >> 4), hi_k, idesc, kk != 0);
                     }
                     ptx::umma_commit(&ctrl->s_full[sb]);
@@ -510,7 +583,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         if (lane == 0) {
             const uint32_t hi_v = ptx::umma_desc_hi_sw128(C::kGroupStride);                // the two 8-token groups of a slot
             const uint32_t v_lo = ptx::umma_desc_lo(ptx::smem_u32(sV), 1024);             // MN-major: LBO = next 64-column atom
-            const uint32_t idesc_pv = ptx::umma_idesc_bf16(kRows, D) | (1u << 16);          // B operand MN-major
+            const uint32_t idesc_pv = (F8 ? umma_idesc_e4m3(kRows, D) : ptx::umma_idesc_bf16(kRows, D)) | (1u << 16);   // B operand MN-major
             uint32_t it = 0;
             bool ok = true;
             long long x = x_begin;
@@ -530,11 +603,13 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     const int n_sl = max(0, min(kStageSlots, sg.slots_all - t * kStageSlots));    // one 16-token step per slot
                     const uint32_t vb = v_lo + (uint32_t)((st * C::kStageBytes) >> 4);
                     const uint32_t pa = tmem_base + (uint32_t)(sb * kTileTok);       // P: 8 columns per 16-token step
+                    // (e4m3: 32 tokens, two slots, per step; P is four codes per column, so a step is 8 columns either way)
+                    constexpr int kStepSlots = F8 ? 2 : 1;
 #pragma unroll
-                    for (int k = 0; k < kStageSlots; ++k)
-                        if (k < n_sl)
-                            ptx::umma_f16_tmem_a(tmem_base + kTmemO + (uint32_t)(pb * D), pa + (uint32_t)(k * 8),
-                                                 vb + (uint32_t)(k * (C::kSlotBytes / 16)), hi_v, idesc_pv, (t >= sg.t_first + 2) || (k != 0));
+                    for (int k = 0; k < kStageSlots / kStepSlots; ++k)
+                        if (k * kStepSlots < n_sl)
+                            umma_ts<F8>(tmem_base + kTmemO + (uint32_t)(pb * D), pa + (uint32_t)(k * 8),
+                                        vb + (uint32_t)(k * (kStepSlots * C::kSlotBytes / 16)), hi_v, idesc_pv, (t >= sg.t_first + 2) || (k != 0));
                     ptx::umma_commit(&ctrl->v_empty[st]);
                     ptx::umma_commit(&ctrl->s_free[sb]);
                     ptx::umma_commit(&ctrl->pv_done[pb]);
@@ -577,6 +652,25 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             uint8_t* q = sQ + buf * q_buf_bytes;
             const uint32_t src_bytes = row_ok ? 16u : 0u;
             if (row_in_blk * 128 >= p.q_half_bytes) return;        // the buffer holds no such row
+            if constexpr (F8) {
+                // this thread's 64 elements, divided by the Q scale and rounded to e4m3: four 16-byte chunks of the row
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    uint4 o = make_uint4(0, 0, 0, 0);
+                    if (row_ok) {
+                        const uint4 a = *reinterpret_cast<const uint4*>(qrow + grp * 64 + i * 16);
+                        const uint4 b = *reinterpret_cast<const uint4*>(qrow + grp * 64 + i * 16 + 8);
+                        auto cv = [&](uint32_t w0, uint32_t w1) -> uint32_t {      // two bf16 pairs -> four codes
+                            // (a true fp32 division: the quotient decides the code)
+                            return pack_e4m3x4(__fdiv_rn(__uint_as_float(w0 << 16), p.q_scale), __fdiv_rn(__uint_as_float(w0 & 0xffff0000u), p.q_scale),
+                                               __fdiv_rn(__uint_as_float(w1 << 16), p.q_scale), __fdiv_rn(__uint_as_float(w1 & 0xffff0000u), p.q_scale));
+                        };
+                        o = make_uint4(cv(a.x, a.y), cv(a.z, a.w), cv(b.x, b.y), cv(b.z, b.w));
+                    }
+                    *reinterpret_cast<uint4*>(q + tile_off(row_in_blk, grp * 4 + i, p.q_half_bytes)) = o;
+                }
+                return;
+            }
 #pragma unroll
             for (int i = 0; i < D / 16; ++i) {
                 const int chunk = grp * (D / 16) + i;
@@ -596,13 +690,26 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         long long x = x_begin;
         Segment sg;
         // P of one tile from the row's 64 scores v[]: p = exp2(s*c - offset) as bf16 pairs, and the row sum in fp32
-        auto tile_p = [&](const float (&v)[kTileTok], float off_log2, uint32_t (&pk)[kTileTok / 2]) -> float {
+        float sc = p.scale_log2e;                                  // scores -> log2 units (e4m3: times the unit's Q and K scales)
+        float vsc = 1.f;                                           // e4m3: the unit's V scale
+        constexpr int kPW = F8 ? kTileTok / 4 : kTileTok / 2;      // 32-bit words of P per row and tile
+        auto tile_p = [&](const float (&v)[kTileTok], float off_log2, uint32_t (&pk)[kPW]) -> float {
             const float o = (off_log2 == -INFINITY) ? 0.f : off_log2;       // nothing visible yet: every score is -inf
             float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+            if constexpr (F8) {
+#pragma unroll
+                for (int j = 0; j < kPW; ++j) {
+                    const float e0 = ptx::ex2_approx(fmaf(v[4 * j], sc, -o)), e1 = ptx::ex2_approx(fmaf(v[4 * j + 1], sc, -o));
+                    const float e2 = ptx::ex2_approx(fmaf(v[4 * j + 2], sc, -o)), e3 = ptx::ex2_approx(fmaf(v[4 * j + 3], sc, -o));
+                    s0 += e0; s1 += e1; s2 += e2; s3 += e3;
+                    pk[j] = pack_e4m3x4(e0, e1, e2, e3);
+                }
+                return (s0 + s1) + (s2 + s3);
+            } else
 #pragma unroll
             for (int j = 0; j < kTileTok / 2; j += 2) {
-                pk[j] = exp2_pair(fmaf(v[2 * j], p.scale_log2e, -o), fmaf(v[2 * j + 1], p.scale_log2e, -o), s0, s1);
-                pk[j + 1] = exp2_pair(fmaf(v[2 * j + 2], p.scale_log2e, -o), fmaf(v[2 * j + 3], p.scale_log2e, -o), s2, s3);
+                pk[j] = exp2_pair(fmaf(v[2 * j], sc, -o), fmaf(v[2 * j + 1], sc, -o), s0, s1);
+                pk[j + 1] = exp2_pair(fmaf(v[2 * j + 2], sc, -o), fmaf(v[2 * j + 3], sc, -o), s2, s3);
             }
             return (s0 + s1) + (s2 + s3);
         };
@@ -623,6 +730,10 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             const UnitPos u = sg.u;
             const bool whole_unit = (sg.t_first == 0 && sg.t_last == u.tiles_in_unit);
             float off_used = -INFINITY, l_run = 0.f;               // this group's offset (log2 units) and running sum
+            if constexpr (F8) {
+                sc = p.scale_log2e * p.q_scale * __ldg(p.k_scale + u.layer * p.Hkv + u.g);
+                vsc = __ldg(p.v_scale + u.layer * p.Hkv + u.g);
+            }
             // the part after this one: its Q goes into the other Q buffer now (every Q K^T that read that buffer
             // belongs to the part before this one and has completed), so the issuer can run on into the next unit
             Segment sg_next;
@@ -669,20 +780,20 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     // maximum.  (Before that every P was 0: nothing to rescale.)
                     if (__any_sync(0xffffffffu, off_used == -INFINITY)) {
                         const float mx = tile_max(v);
-                        if (off_used == -INFINITY && mx > -INFINITY) off_used = mx * p.scale_log2e - kOffsetBias;
+                        if (off_used == -INFINITY && mx > -INFINITY) off_used = mx * sc - PO::kBias;
                     }
-                    uint32_t pk[kTileTok / 2];
+                    uint32_t pk[kPW];
                     sum = tile_p(v, off_used, pk);
                     // The offset moves only when a tile's sum outgrows kSumLimit (an overflow makes the sum infinite, which
                     // counts): rare, and then this tile is redone against its own maximum after the accumulator and the
                     // running sum have been rescaled.  Whatever the offset, it is carried exactly through the sum and the
                     // final division.
-                    const bool grow = !(sum <= kSumLimit);
+                    const bool grow = !(sum <= PO::kSumLimit);
                     if (__any_sync(0xffffffffu, grow)) {
                         // this group's last P V (two tiles ago) must be complete before its accumulator is touched
                         if (it >= 2 && (ctrl->abort || !ptx::mbar_wait(&ctrl->pv_done[grp], ((it - 2) >> 1) & 1, p.wait_limit))) { timeout(p, ctrl, 33); ok = false; break; }
                         ptx::tc_fence_after();
-                        const float off_next = grow ? tile_max(v) * p.scale_log2e - kOffsetBias : off_used;
+                        const float off_next = grow ? tile_max(v) * sc - PO::kBias : off_used;
                         const float alpha = grow ? exp2f(off_used - off_next) : 1.f;
 #pragma unroll 1
                         for (int c4 = 0; c4 < D / 32; ++c4) {
@@ -699,7 +810,8 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     }
                     // P over the first 32 columns of the same S buffer (a thread only touches its own lane, and all of
                     // its scores are in registers)
-                    tmem_st_32x32b_x32(lane_base + (uint32_t)(sb * kTileTok), pk);
+                    if constexpr (F8) tmem_st_32x32b_x16(lane_base + (uint32_t)(sb * kTileTok), pk);
+                    else tmem_st_32x32b_x32(lane_base + (uint32_t)(sb * kTileTok), pk);
                     tmem_st_wait();
                 }
                 l_run += sum;
@@ -755,7 +867,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 // partial layout [column][row]: a warp's store of one column is one contiguous 128-byte line;
                 // each warp of a pair leaves its own copy of (max, sum) so that its columns stand alone
                 float* my = p.partial + ((size_t)blockIdx.x * 2 + slot) * kRowW * kRows + row_in_blk;
-                const float inv = 1.f / Lsum;
+                const float inv = vsc / Lsum;                      // (e4m3: V codes times the unit's V scale)
                 // combined accumulator columns [grp*kDH, (grp+1)*kDH) of both groups' O, 32 at a time
 #pragma unroll 1
                 for (int c4 = 0; c4 < kDH / 32; ++c4) {
@@ -789,7 +901,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                         }
                     } else {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) my[(size_t)(grp * kDH + c4 * 32 + j) * kRows] = acc[j];
+                        for (int j = 0; j < 32; ++j) my[(size_t)(grp * kDH + c4 * 32 + j) * kRows] = acc[j] * vsc;
                     }
                 }
                 // both accumulators have been read by this warp: the next unit's P V may overwrite them once all have
@@ -964,7 +1076,7 @@ __global__ void __launch_bounds__(kMergeThreads) attn_merge_kernel(const AttnPar
 
 mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const MirrorTreeInfo& ti,
                                  const void* q, const void* k_new, const void* v_new, void* out, float* lse_out,
-                                 float* partial_ws, cudaStream_t stream) {
+                                 float* partial_ws, cudaStream_t stream, const MirrorAttnFp8* f8) {
     const int D = ctx->desc.head_dim, Hkv = ctx->desc.n_kv_heads, Hq = ctx->desc.n_q_heads;
     AttnParams p;
     p.L = kv->num_layers; p.B = tree->batch; p.n = ti.n; p.Hq = Hq; p.Hkv = Hkv; p.G = Hq / Hkv;
@@ -981,6 +1093,10 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
     p.max_pages = kv->max_pages_per_req; p.num_pages = kv->num_pages;
     const int64_t page_elems = (int64_t)Hkv * kSlotTok * D;
     if (kv->layer_stride % page_elems != 0) return MIRROR_ERR_UNSUPPORTED;
+    if (f8 && (D != 128 || !f8->k_scale || !f8->v_scale || !(f8->q_scale > 0.f))) return f8 && D != 128 ? MIRROR_ERR_UNSUPPORTED : MIRROR_ERR_ARG;
+    p.k_scale = f8 ? f8->k_scale : nullptr;
+    p.v_scale = f8 ? f8->v_scale : nullptr;
+    p.q_scale = f8 ? f8->q_scale : 1.f;
     p.layer_pages = (int)(kv->layer_stride / page_elems);
     p.tree_slots = (p.n + kSlotTok - 1) / kSlotTok;
     p.q_half_bytes = ((p.rows_per_rb + 7) / 8) * 8 * 128;
@@ -1001,10 +1117,12 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
     {
         // pool viewed as (64 columns, 8 tokens, D/64 halves, 2 token groups, (layer*page)*head): one box is one page of
         // one head, landing as [token / 8][half][token % 8][128 B] (see kv_slot_off)
+        // (an e4m3 pool is described through the same 16-bit map: 64 "columns" are the 128 bytes of a row's only half)
         const uint64_t total_pages = (uint64_t)(p.L - 1) * p.layer_pages + p.num_pages;
-        const uint64_t dims[5] = {64, 8, (uint64_t)(D / 64), 2, total_pages * (uint64_t)Hkv};
-        const uint64_t strides[4] = {(uint64_t)D * 2, 128, (uint64_t)8 * D * 2, (uint64_t)kSlotTok * D * 2};
-        const uint32_t box[5] = {64, 8, (uint32_t)(D / 64), 2, 1};
+        const uint64_t row_bytes = (uint64_t)D * (f8 ? 1 : 2);
+        const uint64_t dims[5] = {64, 8, row_bytes / 128, 2, total_pages * (uint64_t)Hkv};
+        const uint64_t strides[4] = {row_bytes, 128, 8 * row_bytes, kSlotTok * row_bytes};
+        const uint32_t box[5] = {64, 8, (uint32_t)(row_bytes / 128), 2, 1};
         mirror_status st = mirror_make_tmap(ctx, &tm_k, kv->k_pool, 5, dims, strides, box);
         if (st != MIRROR_OK) return st;
         st = mirror_make_tmap(ctx, &tm_v, kv->v_pool, 5, dims, strides, box);
@@ -1013,9 +1131,10 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
     const int grid = p.n_groups * p.n_rb;
     // ring depths: the deepest pair (K, V) that fits beside the Q buffers
     constexpr size_t kSmemLimit = 232448;       // 227 KB
-    auto launch = [&](auto d_tag) -> mirror_status {
+    auto launch = [&](auto d_tag, auto f8_tag) -> mirror_status {
         constexpr int DD = decltype(d_tag)::value;
-        using C = Cfg<DD>;
+        constexpr bool FF = decltype(f8_tag)::value;
+        using C = Cfg<DD, FF>;
         int ks = 4, vs = 4;
         if (C::smem_bytes(p.q_half_bytes, 6, 4) <= kSmemLimit) ks = 6;
         if (C::smem_bytes(p.q_half_bytes, 6, 6) <= kSmemLimit) vs = 6;
@@ -1028,11 +1147,16 @@ mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mir
             MIRROR_CUDA_OK(mirror_launch_pdl(kern, dim3(grid), dim3(kThreads), smem, stream, tm_k, tm_v, at, p));
             return MIRROR_OK;
         };
-        if (ks == 6 && vs == 6) return go(attn_verify_kernel<DD, 6, 6>);
-        if (ks == 6) return go(attn_verify_kernel<DD, 6, 4>);
-        return go(attn_verify_kernel<DD, 4, 4>);
+        if (ks == 6 && vs == 6) return go(attn_verify_kernel<DD, 6, 6, FF>);
+        if constexpr (!FF) {
+            if (ks == 6) return go(attn_verify_kernel<DD, 6, 4, false>);
+            return go(attn_verify_kernel<DD, 4, 4, false>);
+        }
+        return MIRROR_ERR_ARG;
     };
-    mirror_status lst = (D == 128) ? launch(std::integral_constant<int, 128>{}) : launch(std::integral_constant<int, 64>{});
+    mirror_status lst = f8 ? launch(std::integral_constant<int, 128>{}, std::true_type{})
+                      : (D == 128) ? launch(std::integral_constant<int, 128>{}, std::false_type{})
+                                   : launch(std::integral_constant<int, 64>{}, std::false_type{});
     if (lst != MIRROR_OK) return lst;
     ctx->launches += 1;
     MIRROR_CUDA_OK(cudaGetLastError());

@@ -106,9 +106,15 @@ mirror_status mirror_lmhead_pair_launch(mirror_ctx* ctx, const void* hidden, int
 int mirror_linear_slices(const mirror_ctx* ctx, int M, int N, int K);
 mirror_status mirror_linear_partial_launch(mirror_ctx* ctx, const void* x, int M, const void* W, int N, int K, float* partial,
                                            size_t partial_bytes, cudaStream_t stream, int* k_slices);
+// e4m3 cache for mirror_attn_launch: pools, k_new and v_new hold codes; device scales per (layer, KV head), host Q scale.
+struct MirrorAttnFp8 {
+    const float* k_scale;
+    const float* v_scale;
+    float q_scale;
+};
 mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const MirrorTreeInfo& ti,
                                  const void* q, const void* k_new, const void* v_new, void* out, float* lse_out,
-                                 float* partial_ws, cudaStream_t stream);
+                                 float* partial_ws, cudaStream_t stream, const MirrorAttnFp8* f8 = nullptr);
 
 // bf16 tensor map with 128-byte swizzle.  dims/box are innermost-first; strides_bytes[i] is the byte
 // stride of dimension i+1 (rank-1 entries).

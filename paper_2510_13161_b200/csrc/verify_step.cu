@@ -35,6 +35,27 @@ extern "C" mirror_status mirror_attn_verify(mirror_ctx* ctx, const mirror_kv* kv
     return mirror_attn_launch(ctx, kv, tree, ti, q, k_new, v_new, out, lse_out, (float*)(ws + L.attn_partial), (cudaStream_t)stream);
 }
 
+extern "C" mirror_status mirror_attn_verify_fp8(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const void* q,
+                                                const void* k_new_fp8, const void* v_new_fp8, const float* k_scale,
+                                                const float* v_scale, float q_scale, void* out, float* lse_out, void* stream) {
+    if (!ctx || !kv || !tree || !q || !k_new_fp8 || !v_new_fp8 || !k_scale || !v_scale || !out || !(q_scale > 0.f)) return MIRROR_ERR_ARG;
+    if (ctx->desc.head_dim != 128) return MIRROR_ERR_UNSUPPORTED;
+    mirror_status st = check_kv(ctx, kv, tree);
+    if (st != MIRROR_OK) return st;
+    if (((uintptr_t)q & 15) || ((uintptr_t)k_new_fp8 & 15) || ((uintptr_t)v_new_fp8 & 15) || ((uintptr_t)out & 15)) return MIRROR_ERR_ARG;
+    MirrorTreeInfo ti;
+    st = mirror_build_tree(tree, &ti);
+    if (st != MIRROR_OK) return st;
+    MirrorWsLayout L;
+    mirror_ws_layout(ctx, (size_t)tree->batch * tree->n_nodes, &L);
+    if (!ctx->ws || ctx->ws_bytes < L.end_attn) return MIRROR_ERR_WORKSPACE;
+    MIRROR_CUDA_OK(cudaSetDevice(ctx->device));
+    uint8_t* ws = (uint8_t*)ctx->ws;
+    const MirrorAttnFp8 f8 = {k_scale, v_scale, q_scale};
+    return mirror_attn_launch(ctx, kv, tree, ti, q, k_new_fp8, v_new_fp8, out, lse_out, (float*)(ws + L.attn_partial),
+                              (cudaStream_t)stream, &f8);
+}
+
 namespace {
 
 struct HostIO {                       // host-buffer variant: pinned host inputs / outputs of one step

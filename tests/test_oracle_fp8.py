@@ -82,3 +82,70 @@ def test_quantised_lmhead_equals_the_plain_one_on_exactly_representable_operands
     Wq = F.e4m3_decode(wc) * ws[:, None]; hq = F.e4m3_decode(hc) * hs[:, None]
     assert (np.abs(Wq - W) <= np.maximum(np.abs(W) * 2.0 ** -4, ws[:, None] * 2.0 ** -10) * 1.0001).all()
     assert (np.abs(hq - h) <= np.maximum(np.abs(h) * 2.0 ** -4, hs[:, None] * 2.0 ** -10) * 1.0001).all()
+
+
+# ---- the 8-bit KV cache -------------------------------------------------------------------------
+
+def _bf16_bits(v: np.ndarray) -> np.ndarray:
+    return (np.asarray(v, np.float32).view(np.uint32) >> 16).astype(np.uint16)
+
+
+def test_kv_scales_and_codes_per_layer_and_head():
+    rng = np.random.default_rng(5)
+    L, pages, Hkv, P, d = 2, 3, 2, 16, 8
+    x = rng.standard_normal((L, pages, Hkv, P, d)).astype(np.float32)
+    x[1, 2, 1, 7, 3] = -9.5                                       # the known extreme of (layer 1, head 1)
+    x[0, :, 1] = 0.0                                              # an all-zero head keeps scale 1
+    sc = F.kv_scales(x, head_axis=2)
+    assert sc.shape == (L, Hkv) and sc.dtype == np.float32
+    assert sc[1, 1] == np.float32(9.5) / np.float32(448.0) and sc[0, 1] == 1.0
+    for l in range(L):
+        for h in range(Hkv):
+            if (l, h) != (0, 1):
+                assert sc[l, h] == np.abs(x[l, :, h]).max() / np.float32(448.0)
+    codes = F.kv_quantize(x, sc, head_axis=2)
+    assert codes[1, 2, 1, 7, 3] == 0xFE                           # -448: sign bit, exponent 1111, mantissa 110
+    dec = F.e4m3_decode(codes) * sc.astype(np.float64)[:, None, :, None, None]
+    # every element within half a step of the format at its magnitude (step <= 2^-3 relative above the subnormals)
+    err = np.abs(dec - x)
+    bound = np.maximum(np.abs(x) * 2.0 ** -4, sc.astype(np.float64)[:, None, :, None, None] * 2.0 ** -10) * (1 + 1e-6)
+    assert (err <= bound).all()
+    # the tree's rows [L, B, n, Hkv, d] use axis 3
+    y = rng.standard_normal((L, 2, 5, Hkv, d)).astype(np.float32)
+    sy = F.kv_scales(y, head_axis=3)
+    assert sy[1, 0] == np.abs(y[1, :, :, 0]).max() / np.float32(448.0)
+
+
+def test_fp8_attention_equals_plain_attention_of_the_decoded_cache():
+    """Power-of-two scales keep scale * code exact in bf16, so the same cache can be handed to the plain oracle; the
+    scales differ per head, so a swapped head, a scale applied to the wrong operand or a missing one shows."""
+    from oracle import oracle as O
+    rng = np.random.default_rng(11)
+    B, n, Hq, Hkv, d, P = 2, 5, 4, 2, 16, 16
+    pages = 6
+    parent = [-1, 0, 1, 0, 3]
+    anc, _ = O.tree(parent)
+    page_table = np.array([[4, 1, 0], [2, 5, 3]], np.int32)
+    prefix_len = np.array([37, 16], np.int32)
+    q_codes = rng.integers(0, 256, (B, n, Hq, d)).astype(np.uint8)
+    k_codes = rng.integers(0, 256, (pages, Hkv, P, d)).astype(np.uint8)
+    v_codes = rng.integers(0, 256, (pages, Hkv, P, d)).astype(np.uint8)
+    kn_codes = rng.integers(0, 256, (B, n, Hkv, d)).astype(np.uint8)
+    vn_codes = rng.integers(0, 256, (B, n, Hkv, d)).astype(np.uint8)
+    for c in (q_codes, k_codes, v_codes, kn_codes, vn_codes):
+        c[(c & 0x7F) == 0x7F] = 0x30                              # no NaN codes
+        c[(c & 0x78) > 0x48] &= 0xC7                              # keep magnitudes small: scores stay moderate
+    k_scale = np.array([0.25, 2.0], np.float32)
+    v_scale = np.array([4.0, 0.5], np.float32)
+    q = F.e4m3_decode(q_codes) * 0.125                            # q_scale = 2^-3: exact in bf16 as well
+    out8, lse8 = F.attention_layer_fp8(q_codes, 0.125, k_codes, v_codes, k_scale, v_scale, page_table, prefix_len, kn_codes,
+                                       vn_codes, anc, 0.3)
+    def dec(c, s, axis):
+        shape = [1] * c.ndim
+        shape[axis] = Hkv
+        return _bf16_bits(F.e4m3_decode(c) * s.astype(np.float64).reshape(shape))
+    out, lse, _ = O.attention_layer(_bf16_bits(q), dec(k_codes, k_scale, 1), dec(v_codes, v_scale, 1), page_table, prefix_len,
+                                    dec(kn_codes, k_scale, 2), dec(vn_codes, v_scale, 2), anc, 0.3)
+    np.testing.assert_allclose(out8, out, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(lse8, lse, rtol=1e-12, atol=1e-12)
+    assert np.abs(out).max() > 0.1
