@@ -69,6 +69,9 @@ def parse_args():
     ap.add_argument("--lmhead-fp8", action="store_true",
                     help="also time the low-precision LM head (e4m3 weights and hidden rows, one scale per row) next to the bf16 "
                          "head on the workload's rows; reported under stages.lmhead_fp8, outside the timed region")
+    ap.add_argument("--attn-fp8", action="store_true",
+                    help="also time the attention over an e4m3 KV cache next to the bf16 one on the workload (head dimension 128); "
+                         "reported under stages.attn_fp8, outside the timed region")
     ap.add_argument("--layers", type=int, default=None,
                     help="profiling aid: run the workload with this many attention layers (config.layers reports it); "
                          "the default, the workload's own layer count, is the only valid bench configuration")
@@ -399,6 +402,43 @@ def lmhead_fp8_stage(m, x, cfg, hbm_gbs: float, reps: int = 20):
             "note": "both include the merge kernel; fp8 also includes quantising the hidden rows"}
 
 
+def attn_fp8_stage(m, x, tree, kv, cfg, peaks: dict, algo: dict, reps: int = 5):
+    """bf16 attention against the e4m3-cache one over the workload's layers: ms, flop/s and cache bytes per second each.
+    The cache is quantised once, outside the timing (as a serving engine would when it writes the cache)."""
+    import torch
+    P, d = x.k_pool.shape[3], x.k_pool.shape[4]
+    ks, vs = m.mirror_kv_scales_fp8(x.k_pool, P * d), m.mirror_kv_scales_fp8(x.v_pool, P * d)
+    k8, v8 = m.mirror_kv_quantize_fp8(x.k_pool, P * d, ks), m.mirror_kv_quantize_fp8(x.v_pool, P * d, vs)
+    kn8, vn8 = m.mirror_kv_quantize_fp8(x.k_new, d, ks), m.mirror_kv_quantize_fp8(x.v_new, d, vs)
+    kv8 = m.kv_fp8(k8, v8, x.page_table, x.prefix_len)
+    q_scale = float(x.q[0].float().abs().max()) / 448.0
+    out = torch.empty_like(x.q)
+
+    def timed(fn):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    t16 = timed(lambda: m.mirror_attn_verify(kv, tree, x.q, x.k_new, x.v_new, out=out))
+    t8 = timed(lambda: m.mirror_attn_verify_fp8(kv8, tree, x.q, kn8, vn8, ks, vs, q_scale, out=out))
+    code, detail = m.device_status()
+    if code != 0:
+        raise SystemExit(f"device status {code} (detail {detail}) in the fp8 attention")
+    kv_bytes = algo["attn_bytes"]          # (cache, tree rows, Q and O: the cache is nearly all of it)
+    return {"bf16_ms": t16, "fp8_ms": t8, "speedup": t16 / t8,
+            "bf16_tflops": algo["attn_flops"] / t16 / 1e9, "fp8_tflops": algo["attn_flops"] / t8 / 1e9,
+            "bf16_gbs": kv_bytes / t16 / 1e6, "fp8_gbs": kv_bytes / 2 / t8 / 1e6,
+            "fp8_frac_hbm": kv_bytes / 2 / t8 / 1e6 / peaks["hbm_gbs"],
+            "note": "all layers, inputs larger than L2; merge kernel included in both"}
+
+
 def target_forward_stage(m, x, tree, kv, cfg, n_layers: int, intermediate: int, hbm_gbs: float, reps: int = 5):
     """mirror_target_forward over n_layers decoder layers of the workload's shape (random weights): ms, weight bytes per
     second against the HBM peak.  The layers are weight streams at these row counts."""
@@ -641,6 +681,8 @@ def run_mirror(args):
         stages["overlap_draft"] = overlap_draft_stage(w.step, w.stream)
     if args.lmhead_fp8:
         stages["lmhead_fp8"] = lmhead_fp8_stage(m, x, cfg, peaks["hbm_gbs"])
+    if args.attn_fp8:
+        stages["attn_fp8"] = attn_fp8_stage(m, x, w.tree, w.kv, cfg, peaks, work)
     if args.target_layers > 0:
         stages["target_forward"] = target_forward_stage(m, x, w.tree, w.kv, cfg, min(args.target_layers, cfg.layers), args.intermediate,
                                                         peaks["hbm_gbs"])
