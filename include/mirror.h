@@ -301,6 +301,11 @@ mirror_status mirror_overlap_mass(mirror_ctx* ctx, const float* logits_final, co
 mirror_status mirror_kv_commit(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const void* k_new,
                                const void* v_new, const int32_t* accepted_nodes, const int32_t* n_accepted,
                                int32_t* prefix_len, void* stream);
+/* The same roll-forward of an e4m3 cache (see mirror_attn_verify_fp8): pools, k_new_fp8 and v_new_fp8 hold codes, one
+ * byte per element, already under the cache's scales (mirror_kv_quantize_fp8); d must be a multiple of 16. */
+mirror_status mirror_kv_commit_fp8(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const void* k_new_fp8,
+                                   const void* v_new_fp8, const int32_t* accepted_nodes, const int32_t* n_accepted,
+                                   int32_t* prefix_len, void* stream);
 
 /* HOST helper (no device work): merge kappa branches of gamma tokens -- the branch-complete proposal of Sec. 3.1 --
  * into a token tree without duplicated prefixes ("tree drafts"): branches that agree on their first r tokens share

@@ -27,7 +27,7 @@ EXPORTS = [
     "mirror_device_status", "mirror_launch_count", "mirror_status_str", "mirror_set_stage_events",
     "mirror_lmhead_reduce_noalloc", "mirror_lmhead_noalloc_status", "mirror_quantize_rows_fp8", "mirror_lmhead_reduce_fp8", "mirror_early_exit_tap", "mirror_overlap_mass", "mirror_kv_commit",
     "mirror_linear_scratch_bytes", "mirror_linear", "mirror_rmsnorm", "mirror_target_scratch_bytes", "mirror_target_forward", "mirror_trie_build", "mirror_verify_step_host", "mirror_embed_rows",
-    "mirror_attn_verify_fp8", "mirror_kv_scales_fp8", "mirror_kv_quantize_fp8",
+    "mirror_attn_verify_fp8", "mirror_kv_scales_fp8", "mirror_kv_quantize_fp8", "mirror_kv_commit_fp8",
 ]
 
 
@@ -392,6 +392,13 @@ class Mirror:
                                          _ptr(v_new, torch.bfloat16, "v_new"), _ptr(res.accepted_nodes, torch.int32, "accepted_nodes"),
                                          _ptr(res.n_accepted, torch.int32, "n_accepted"), _ptr(prefix_len, torch.int32, "prefix_len"),
                                          _stream(stream)), "mirror_kv_commit")
+
+    def mirror_kv_commit_fp8(self, kv: KV, tree: Tree, k_new8, v_new8, res: "AcceptResult", prefix_len: torch.Tensor, stream=None):
+        """mirror_kv_commit for an e4m3 cache (kv from kv_fp8, k_new8 / v_new8 uint8 codes under the cache's scales)."""
+        _check(self.lib.mirror_kv_commit_fp8(self._ctx, C.byref(kv), C.byref(tree), _ptr(k_new8, torch.uint8, "k_new8"),
+                                             _ptr(v_new8, torch.uint8, "v_new8"), _ptr(res.accepted_nodes, torch.int32, "accepted_nodes"),
+                                             _ptr(res.n_accepted, torch.int32, "n_accepted"), _ptr(prefix_len, torch.int32, "prefix_len"),
+                                             _stream(stream)), "mirror_kv_commit_fp8")
 
     # ---- the target's layers around the attention ---------------------------------------------
     def target(self, layers: Sequence[dict], norm_final: torch.Tensor, intermediate: int, rope_theta: float = 1e6,

@@ -60,9 +60,10 @@ __global__ void kv_advance_kernel(int B, int gamma, const int32_t* n_accepted, i
 
 }  // namespace
 
-extern "C" mirror_status mirror_kv_commit(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const void* k_new,
-                                          const void* v_new, const int32_t* accepted_nodes, const int32_t* n_accepted,
-                                          int32_t* prefix_len, void* stream) {
+// elem_bytes 2: bf16 cache.  1: e4m3 codes; a row of d codes is moved as d / 2 16-bit units, the layout is the same.
+static mirror_status kv_commit_impl(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const void* k_new,
+                                    const void* v_new, const int32_t* accepted_nodes, const int32_t* n_accepted,
+                                    int32_t* prefix_len, void* stream, int elem_bytes) {
     if (!ctx || !kv || !tree || !k_new || !v_new || !accepted_nodes || !n_accepted || !prefix_len) return MIRROR_ERR_ARG;
     if (!kv->k_pool || !kv->v_pool || !kv->page_table) return MIRROR_ERR_ARG;
     if (tree->batch <= 0 || tree->n_nodes <= 0 || tree->n_nodes > MIRROR_MAX_NODES || tree->gamma < 0 || tree->gamma > MIRROR_MAX_DEPTH)
@@ -71,9 +72,11 @@ extern "C" mirror_status mirror_kv_commit(mirror_ctx* ctx, const mirror_kv* kv, 
     if (((uintptr_t)k_new & 15) || ((uintptr_t)v_new & 15) || ((uintptr_t)kv->k_pool & 15) || ((uintptr_t)kv->v_pool & 15)) return MIRROR_ERR_ARG;
     MIRROR_CUDA_OK(cudaSetDevice(ctx->device));
     CommitParams p;
-    p.L = kv->num_layers; p.B = tree->batch; p.n = tree->n_nodes; p.Hkv = ctx->desc.n_kv_heads; p.d = ctx->desc.head_dim;
+    p.L = kv->num_layers; p.B = tree->batch; p.n = tree->n_nodes; p.Hkv = ctx->desc.n_kv_heads;
+    p.d = ctx->desc.head_dim * elem_bytes / 2;
+    if (kv->layer_stride * elem_bytes % 2 != 0) return MIRROR_ERR_SHAPE;
     p.gamma = tree->gamma; p.max_pages = kv->max_pages_per_req; p.num_pages = kv->num_pages;
-    p.layer_stride = kv->layer_stride;
+    p.layer_stride = kv->layer_stride * elem_bytes / 2;
     p.k_pool = (__nv_bfloat16*)const_cast<void*>(kv->k_pool);
     p.v_pool = (__nv_bfloat16*)const_cast<void*>(kv->v_pool);
     p.k_new = (const __nv_bfloat16*)k_new; p.v_new = (const __nv_bfloat16*)v_new;
@@ -86,4 +89,16 @@ extern "C" mirror_status mirror_kv_commit(mirror_ctx* ctx, const mirror_kv* kv, 
     ctx->launches += 2;
     MIRROR_CUDA_OK(cudaGetLastError());
     return MIRROR_OK;
+}
+
+extern "C" mirror_status mirror_kv_commit(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const void* k_new,
+                                          const void* v_new, const int32_t* accepted_nodes, const int32_t* n_accepted,
+                                          int32_t* prefix_len, void* stream) {
+    return kv_commit_impl(ctx, kv, tree, k_new, v_new, accepted_nodes, n_accepted, prefix_len, stream, 2);
+}
+
+extern "C" mirror_status mirror_kv_commit_fp8(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const void* k_new_fp8,
+                                              const void* v_new_fp8, const int32_t* accepted_nodes, const int32_t* n_accepted,
+                                              int32_t* prefix_len, void* stream) {
+    return kv_commit_impl(ctx, kv, tree, k_new_fp8, v_new_fp8, accepted_nodes, n_accepted, prefix_len, stream, 1);
 }

@@ -154,3 +154,44 @@ def test_head_dim_64_is_refused():
         m.mirror_attn_verify_fp8(m.kv_fp8(z8, z8, x.page_table, x.prefix_len), m.tree(x.tokens, cfg.kappa, cfg.gamma, parent=x.parent),
                                  x.q, n8, n8, s, s, 1.0)
     assert e.value.code == 3
+
+
+def test_commit_of_codes_then_attention_on_the_committed_cache():
+    """The accepted path's codes are appended to the 8-bit cache byte for byte (oracle: kv_commit on the code arrays), and
+    the next step's attention over that cache matches the oracle over the oracle's committed cache."""
+    from paper_2510_13161_b200 import binding
+    cfg = small(batch=3, prefix_lo=20, prefix_hi=120, kappa=2, gamma=3)
+    x = I.gen_verify_inputs(cfg, 9, "cuda", with_lm_head=False, headroom=cfg.gamma + 1)
+    m = make_mirror(cfg)
+    ks, vs, k8, v8, kn8, vn8 = quantise(m, x)
+    paths = [[1, 2], [], [4, 5, 6]]
+    res = binding.AcceptResult(cfg.batch, cfg.gamma, "cuda")
+    acc = np.full((cfg.batch, cfg.gamma), -1, np.int32)
+    n_acc = np.array([len(p) for p in paths], np.int32)
+    for b, p in enumerate(paths):
+        acc[b, :len(p)] = p
+    res.accepted_nodes.copy_(torch.from_numpy(acc))
+    res.n_accepted.copy_(torch.from_numpy(n_acc))
+    k_ref, v_ref, pl_ref = O.kv_commit(k8.cpu().numpy(), v8.cpu().numpy(), x.page_table.cpu().numpy(), x.prefix_len.cpu().numpy(),
+                                       kn8.cpu().numpy(), vn8.cpu().numpy(), acc, n_acc)
+    pl = x.prefix_len.clone()
+    kv = m.kv_fp8(k8, v8, x.page_table, pl)
+    tree = m.tree(x.tokens, cfg.kappa, cfg.gamma, parent=x.parent)
+    m.mirror_kv_commit_fp8(kv, tree, kn8, vn8, res, pl)
+    torch.cuda.synchronize()
+    assert m.device_status() == (0, 0)
+    assert np.array_equal(k8.cpu().numpy(), k_ref) and np.array_equal(v8.cpu().numpy(), v_ref)
+    assert np.array_equal(pl.cpu().numpy(), pl_ref)
+    # next step: same tree rows on the longer prefixes
+    L, B, n, Hq, d = x.q.shape
+    q_scale = float(np.float32(float(x.q.float().abs().max())) / np.float32(448.0))
+    out = m.mirror_attn_verify_fp8(kv, tree, x.q, kn8, vn8, ks, vs, q_scale)
+    torch.cuda.synchronize()
+    assert m.device_status() == (0, 0)
+    anc, _ = O.tree(x.parent)
+    for l in range(L):
+        ref, _ = F.attention_layer_fp8(F.quantize_tensor(f32(x.q[l]), q_scale), q_scale, k_ref[l], v_ref[l], ks[l].cpu().numpy(),
+                                       vs[l].cpu().numpy(), x.page_table.cpu().numpy(), pl_ref, kn8[l].cpu().numpy(), vn8[l].cpu().numpy(),
+                                       anc, 1.0 / np.sqrt(d))
+        got = f32(out[l]).astype(np.float64)
+        assert np.abs(got - ref).max() <= FP8_REL * np.abs(ref).max(), l
