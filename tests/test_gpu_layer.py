@@ -122,6 +122,35 @@ def test_target_forward_matches_layer_oracle(case):
     close(out["hidden"], ref[-1]["normed"], "hidden", ulps=3.0 if tight else 8.0, exact_frac=0.4 if tight else 0.15)
 
 
+@pytest.mark.parametrize("case", [
+    dict(H=256, Hq=4, Hkv=2, d=64, inter=512, L=2, B=2, lo=70, hi=200, kappa=2, gamma=3, seed=0),
+    dict(H=512, Hq=8, Hkv=2, d=128, inter=1344, L=3, B=1, lo=300, hi=300, kappa=4, gamma=4, seed=1),
+])
+def test_every_layer_alone_from_the_oracles_input_meets_the_first_layers_gates(case):
+    """The gates of the layers after the first in the test above allow for drift inherited from the layers before.  Here
+    every layer runs alone from the ORACLE's input to that layer (its stored bf16 stream), so both sides read identical
+    inputs again and each layer has to meet the gates of layer 0: what a layer adds on its own is bounded layer by layer."""
+    theta, eps = 1.0e4, 1e-6
+    cfg, x, layers, norm_final, emb = layer_case(**case)
+    ref = run_oracle(cfg, x, layers, norm_final, emb, theta, eps)
+    m = make_mirror(cfg)
+    dev = lambda t: t.cuda()
+    tree = m.tree(dev(x.tokens), cfg.kappa, cfg.gamma)
+    for l in range(1, len(layers)):
+        x_in = torch.from_numpy(np.ascontiguousarray(ref[l - 1]["x"]).view(np.int16)).view(torch.bfloat16)
+        nxt = layers[l + 1]["norm_attn"] if l + 1 < len(layers) else norm_final
+        tgt = m.target([{k: dev(v) for k, v in layers[l].items()}], dev(nxt), case["inter"], theta, eps)
+        kv = m.kv(dev(x.k_pool[l:l + 1].contiguous()), dev(x.v_pool[l:l + 1].contiguous()), dev(x.page_table), dev(x.prefix_len))
+        out = m.mirror_target_forward(tgt, kv, tree, dev(x_in))
+        assert m.device_status() == (0, 0)
+        close(out["q"][0], ref[l]["q"], f"q{l}", ulps=1.5, exact_frac=0.99)
+        close(out["k_new"][0], ref[l]["k_new"], f"k{l}", ulps=1.5, exact_frac=0.99)
+        close(out["v_new"][0], ref[l]["v_new"], f"v{l}", ulps=1.5, exact_frac=0.99)
+        close(out["attn_out"][0], ref[l]["attn"], f"attn{l}", ulps=3.0, exact_frac=0.4)
+        close(out["x_out"], ref[l]["x"], f"x{l}", ulps=3.0, exact_frac=0.4)
+        close(out["hidden"], ref[l]["normed"], f"hidden{l}", ulps=3.0, exact_frac=0.4)
+
+
 def test_target_forward_feeds_the_verify_step():
     """hidden rows out of the layers go straight into the LM head + acceptance of the fused step."""
     from oracle import oracle as O
