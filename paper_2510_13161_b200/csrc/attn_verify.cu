@@ -123,6 +123,18 @@ __device__ __forceinline__ void timeout(const AttnParams& p, Ctrl* c, int where)
     if (atomicCAS(p.status, 0, MIRROR_DEV_TIMEOUT) == 0) atomicExch(p.status + 1, where);
 }
 
+// A bounded wait that looks at the CTA's abort flag only when the barrier is not complete yet (the common case is one
+// try_wait), and between parks while it waits.
+__device__ __forceinline__ bool wait_bar(Ctrl* c, uint64_t* bar, uint32_t parity, long long limit_cycles) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        if (c->abort) return false;
+        if (ptx::mbar_try_wait_park(bar, parity, MIRROR_PARK_NS)) return true;
+        if (clock64() - t0 > limit_cycles) return false;
+    }
+}
+
 __device__ __noinline__ UnitPos locate(long long x, const AttnParams& p, const int* cumT, long long tiles_per_layer) {
     UnitPos u;
     // (the tile count fits 31 bits: checked in the prologue; 32-bit divisions are several times cheaper)
@@ -470,7 +482,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 const uint32_t ph = (vrole ? it / VS : it / KR) & 1;
                 const int next_page = (t + 1 < sg.t_last) ? fetch_page(t + 1) : 0;
                 bool w = true;
-                if (lane == 0) w = !ctrl->abort && ptx::mbar_wait(&empty[st], ph ^ 1, p.wait_limit);
+                if (lane == 0) w = wait_bar(ctrl, &empty[st], ph ^ 1, p.wait_limit);
                 w = __shfl_sync(0xffffffffu, w, 0);
                 if (!w) { if (lane == 0) timeout(p, ctrl, 10); ok = false; break; }
                 uint8_t* dst = (vrole ? sV : sK) + (size_t)st * C::kStageBytes;
@@ -547,26 +559,33 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             const uint32_t hi_k = ptx::umma_desc_hi_sw128(C::kGroupStride);   // 8-token groups of a half: uniform over the pair's slots
             const uint32_t q_lo = ptx::umma_desc_lo(ptx::smem_u32(sQ), 16);
             const uint32_t k_lo = ptx::umma_desc_lo(ptx::smem_u32(sK), 16);
-            uint32_t it = 0, seg = 0;
+            // This one thread is busy for the whole tile period (its tcgen05.mma chain into one S buffer advances at
+            // one instruction per ~100 cycles and holds it up meanwhile), so what it does between two chains is kept
+            // short: ring stage, buffer and their parities are running counters, and the descriptor of a full tile is
+            // made once.
+            const uint32_t idesc_full = F8 ? umma_idesc_e4m3(kRows, kTileTok) : ptx::umma_idesc_bf16(kRows, kTileTok);
+            uint32_t seg = 0;
+            uint32_t st = 0, k_par = 0;            // K ring stage of the next tile and the parity its data completes
+            uint32_t sb = 0, s_par = 1;            // S buffer of the next tile and the parity that says it is free
             bool ok = true;
             long long x = x_begin;
             while (x < x_end && ok) {
                 const Segment sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
-                if (ctrl->abort || !ptx::mbar_wait(&ctrl->q_full[seg & 1], (seg >> 1) & 1, p.wait_limit)) { timeout(p, ctrl, 20); ok = false; break; }
+                if (!wait_bar(ctrl, &ctrl->q_full[seg & 1], (seg >> 1) & 1, p.wait_limit)) { timeout(p, ctrl, 20); ok = false; break; }
                 const uint32_t q_seg = q_lo + (uint32_t)(((seg & 1) * q_buf_bytes) >> 4);
                 ++seg;
                 // one tile (a ring stage of four slots) per issue: each S buffer is scored as soon as the P V that read
                 // it has completed, so the two softmax groups run half a period apart instead of in step
-                for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
-                    const int st = it % KR, sb = it & (kSBufs - 1);
-                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->k_full[st], (it / KR) & 1, p.wait_limit) ||
-                        !ptx::mbar_wait(&ctrl->s_free[sb], ((it / kSBufs) & 1) ^ 1, p.wait_limit)) { timeout(p, ctrl, 21); ok = false; break; }
+                int rem = sg.slots_all - sg.t_first * kStageSlots;               // slots left in the unit from this tile on
+                for (int t = sg.t_first; t < sg.t_last; ++t, rem -= kStageSlots) {
+                    if (!wait_bar(ctrl, &ctrl->k_full[st], k_par, p.wait_limit) ||
+                        !wait_bar(ctrl, &ctrl->s_free[sb], s_par, p.wait_limit)) { timeout(p, ctrl, 21); ok = false; break; }
                     ptx::tc_fence_after();
-                    const int n_sl = min(kStageSlots, sg.slots_all - t * kStageSlots);       // (a pair's second tile may be empty)
-                    if (n_sl > 0) {
-                        const uint32_t idesc = F8 ? umma_idesc_e4m3(kRows, n_sl * kSlotTok) : ptx::umma_idesc_bf16(kRows, n_sl * kSlotTok);
-                        const uint32_t kb = k_lo + (uint32_t)((st * C::kStageBytes) >> 4);
-                        const uint32_t d = tmem_base + (uint32_t)(sb * kTileTok);
+                    if (rem > 0) {                                                     // (a pair's second tile may be empty)
+                        const uint32_t idesc = rem >= kStageSlots ? idesc_full
+                                             : (F8 ? umma_idesc_e4m3(kRows, rem * kSlotTok) : ptx::umma_idesc_bf16(kRows, rem * kSlotTok));
+                        const uint32_t kb = k_lo + st * (uint32_t)(C::kStageBytes >> 4);
+                        const uint32_t d = tmem_base + sb * (uint32_t)kTileTok;
 #pragma unroll
                         for (int kk = 0; kk < C::kRowBytes / 32; ++kk)          // 32 bytes of every row per instruction
                             umma_ss<F8>(d, q_seg + (uint32_t)(((kk >> 2) * p.q_half_bytes + (kk & 3) * 32) >> 4), hi_q,
@@ -574,7 +593,11 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     }
                     ptx::umma_commit(&ctrl->s_full[sb]);
                     ptx::umma_commit(&ctrl->k_empty[st]);
+                    if (++st == (uint32_t)KR) { st = 0; k_par ^= 1; }
+                    sb = (sb + 1) & (kSBufs - 1);
+                    if (sb == 0) s_par ^= 1;
                 }
+                x += sg.t_last - sg.t_first;
                 if (!ok) break;
             }
         }
@@ -591,12 +614,12 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             while (x < x_end && ok) {
                 const Segment sg = make_segment(x, x_end, p, cumT, s_len, tiles_per_layer);
                 // the accumulators of the previous part must have been read out by every softmax warp
-                if (seg > 0 && (ctrl->abort || !ptx::mbar_wait(&ctrl->o_free, (seg - 1) & 1, p.wait_limit))) { timeout(p, ctrl, 24); ok = false; break; }
+                if (seg > 0 && (!wait_bar(ctrl, &ctrl->o_free, (seg - 1) & 1, p.wait_limit))) { timeout(p, ctrl, 24); ok = false; break; }
                 ++seg;
                 for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
                     const int st = it % VS, pb = it & 1, sb = it & (kSBufs - 1);
-                    if (ctrl->abort || !ptx::mbar_wait(&ctrl->p_full[sb], (it / kSBufs) & 1, p.wait_limit) ||
-                        !ptx::mbar_wait(&ctrl->v_full[st], (it / VS) & 1, p.wait_limit)) {
+                    if (!wait_bar(ctrl, &ctrl->p_full[sb], (it / kSBufs) & 1, p.wait_limit) ||
+                        !wait_bar(ctrl, &ctrl->v_full[st], (it / VS) & 1, p.wait_limit)) {
                         timeout(p, ctrl, 23); ok = false; break;
                     }
                     ptx::tc_fence_after();
@@ -640,7 +663,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         auto pair_sync = [&]() -> bool {
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&ctrl->pair[w4]);
-            const bool r = !ctrl->abort && ptx::mbar_wait(&ctrl->pair[w4], xph, p.wait_limit);
+            const bool r = wait_bar(ctrl, &ctrl->pair[w4], xph, p.wait_limit);
             xph ^= 1;
             return r;
         };
@@ -748,7 +771,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
                 if ((int)(it & 1) != grp) continue;
                 const int sb = it & (kSBufs - 1);
-                if (ctrl->abort || !ptx::mbar_wait(&ctrl->s_full[sb], (it / kSBufs) & 1, p.wait_limit)) { timeout(p, ctrl, 30); ok = false; break; }
+                if (!wait_bar(ctrl, &ctrl->s_full[sb], (it / kSBufs) & 1, p.wait_limit)) { timeout(p, ctrl, 30); ok = false; break; }
                 ptx::tc_fence_after();
                 float sum = 0.f;
                 // visibility of this tile's columns for this row: all ones except in a unit's last pairs
@@ -791,7 +814,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     const bool grow = !(sum <= PO::kSumLimit);
                     if (__any_sync(0xffffffffu, grow)) {
                         // this group's last P V (two tiles ago) must be complete before its accumulator is touched
-                        if (it >= 2 && (ctrl->abort || !ptx::mbar_wait(&ctrl->pv_done[grp], ((it - 2) >> 1) & 1, p.wait_limit))) { timeout(p, ctrl, 33); ok = false; break; }
+                        if (it >= 2 && (!wait_bar(ctrl, &ctrl->pv_done[grp], ((it - 2) >> 1) & 1, p.wait_limit))) { timeout(p, ctrl, 33); ok = false; break; }
                         ptx::tc_fence_after();
                         const float off_next = grow ? tile_max(v) * sc - PO::kBias : off_used;
                         const float alpha = grow ? exp2f(off_used - off_next) : 1.f;
@@ -818,7 +841,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 // Keep in step with this group's P V barrier: a parity wait can only tell apart two consecutive
                 // phases, so a warp must never fall two completions behind it.  The P V of two tiles ago has
                 // normally long completed here.
-                if (it >= 2 && (ctrl->abort || !ptx::mbar_wait(&ctrl->pv_done[grp], ((it - 2) >> 1) & 1, p.wait_limit))) { timeout(p, ctrl, 34); ok = false; break; }
+                if (it >= 2 && (!wait_bar(ctrl, &ctrl->pv_done[grp], ((it - 2) >> 1) & 1, p.wait_limit))) { timeout(p, ctrl, 34); ok = false; break; }
                 // P is in tensor memory (and any O rescale too): the P V of this tile may go
                 ptx::tc_fence_before();
                 __syncwarp();
@@ -845,7 +868,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             // groups meet: past the meeting both accumulators are complete
             {
                 const uint32_t j_last = (((it - 1) & 1) == (uint32_t)grp) ? it - 1 : it - 2;
-                if (ctrl->abort || !ptx::mbar_wait(&ctrl->pv_done[grp], (j_last >> 1) & 1, p.wait_limit)) { timeout(p, ctrl, 32); ok = false; break; }
+                if (!wait_bar(ctrl, &ctrl->pv_done[grp], (j_last >> 1) & 1, p.wait_limit)) { timeout(p, ctrl, 32); ok = false; break; }
             }
             ptx::tc_fence_before();
             if (!pair_sync()) { timeout(p, ctrl, 35); ok = false; break; }
