@@ -768,8 +768,10 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             }
             bool q_pending = has_next;
 
-            for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
-                if ((int)(it & 1) != grp) continue;
+            // this group's tiles of the part: those whose counter has the group's parity
+            const uint32_t it0 = it;
+            for (int t = sg.t_first + (int)((it0 ^ (uint32_t)grp) & 1u); t < sg.t_last; t += 2) {
+                it = it0 + (uint32_t)(t - sg.t_first);
                 const int sb = it & (kSBufs - 1);
                 if (!wait_bar(ctrl, &ctrl->s_full[sb], (it / kSBufs) & 1, p.wait_limit)) { timeout(p, ctrl, 30); ok = false; break; }
                 ptx::tc_fence_after();
@@ -849,6 +851,8 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 if (q_pending) { q_ready((seg + 1) & 1); q_pending = false; }
             }
             if (!ok) break;
+            it = it0 + (uint32_t)(sg.t_last - sg.t_first);
+            x = x_next;
 
             // (This part's Q buffer is overwritten at the start of the next part.  Every Q K^T that reads it has
             // completed by then: below, each group waits for the P V of its own last tile and then meets the other;
