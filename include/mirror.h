@@ -400,7 +400,7 @@ mirror_status mirror_target_forward(mirror_ctx* ctx, const mirror_target* t, con
  *   h_out           HOST copies of the decision (any member may be NULL); valid once `stream` has been synchronised
  * Copies run on an internal stream (created on first use) and begin after all work already queued on `stream`.  The
  * layers' attention problems are independent and the LM head reads only the last layer's output, so the last layer is
- * copied and attended to first, the LM head and the acceptance follow, and the other layers arrive in three pieces
+ * copied and attended to first, the LM head and the acceptance follow, and the other layers arrive in up to eleven pieces
  * while the LM head runs; each is attended to once it has landed, after the decision has been sent back.
  * Everything else as in mirror_verify_step (attn_out holds all layers when `stream` has drained).  Does not synchronise. */
 typedef struct {

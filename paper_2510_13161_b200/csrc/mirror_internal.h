@@ -42,6 +42,10 @@ struct MirrorTuning {
 };
 void mirror_tuning_from_env(MirrorTuning* t);
 
+// mirror_verify_step_host copies and attends to a step's layers in this many pieces (the last layer first, alone).  The
+// pieces' copies are what bounds the host-buffer step on a large model (1.7 GB of Q per step on the 66B-class workload),
+// and the last piece's attention is what is left exposed behind them, so the pieces are kept small.
+constexpr int kMirrorHostChunks = 12;
 struct mirror_ctx {
     mirror_model_desc desc;
     MirrorTuning tune;
@@ -58,7 +62,7 @@ struct mirror_ctx {
     cudaEvent_t stage_ev[4] = {nullptr, nullptr, nullptr, nullptr};
     bool stage_ev_on = false;
     cudaStream_t copy_stream = nullptr;                     // mirror_verify_step_host: created on first use
-    cudaEvent_t copy_ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+    cudaEvent_t copy_ev[kMirrorHostChunks + 1] = {};
     PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
 };
 

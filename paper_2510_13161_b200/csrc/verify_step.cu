@@ -66,7 +66,7 @@ struct HostIO {                       // host-buffer variant: pinned host inputs
     const mirror_accept_host_out* h_out;
 };
 
-constexpr int kHostChunks = 4;        // the step's layers are copied and attended to in this many pieces
+constexpr int kHostChunks = kMirrorHostChunks;
 
 mirror_status ensure_copy_stream(mirror_ctx* ctx) {
     if (ctx->copy_stream) return MIRROR_OK;
@@ -100,7 +100,7 @@ mirror_status verify_step_impl(mirror_ctx* ctx, const mirror_kv* kv, const mirro
     cudaStream_t s = (cudaStream_t)stream;
 
     // (host-buffer variant) pieces of layers, copied on the second stream and attended to in that order
-    int n_pieces = 0, piece_l0[kHostChunks] = {0, 0, 0, 0}, piece_l1[kHostChunks] = {0, 0, 0, 0};
+    int n_pieces = 0, piece_l0[kHostChunks] = {}, piece_l1[kHostChunks] = {};
     const size_t q_layer = M * (size_t)ctx->desc.n_q_heads * ctx->desc.head_dim * 2;        // bytes per layer
     const size_t kv_layer = M * (size_t)ctx->desc.n_kv_heads * ctx->desc.head_dim * 2;
     auto attend_piece = [&](int c) -> mirror_status {
