@@ -135,6 +135,13 @@ __device__ __forceinline__ bool wait_bar(Ctrl* c, uint64_t* bar, uint32_t parity
     }
 }
 
+// Two barriers at once: both polls are issued before either result is looked at.
+__device__ __forceinline__ bool wait_bar2(Ctrl* c, uint64_t* bar_a, uint32_t par_a, uint64_t* bar_b, uint32_t par_b, long long limit_cycles) {
+    const bool a = ptx::mbar_try_wait(bar_a, par_a), b = ptx::mbar_try_wait(bar_b, par_b);
+    if (a && b) return true;
+    return (a || wait_bar(c, bar_a, par_a, limit_cycles)) && (b || wait_bar(c, bar_b, par_b, limit_cycles));
+}
+
 __device__ __noinline__ UnitPos locate(long long x, const AttnParams& p, const int* cumT, long long tiles_per_layer) {
     UnitPos u;
     // (the tile count fits 31 bits: checked in the prologue; 32-bit divisions are several times cheaper)
@@ -567,6 +574,7 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             uint32_t seg = 0;
             uint32_t st = 0, k_par = 0;            // K ring stage of the next tile and the parity its data completes
             uint32_t sb = 0, s_par = 1;            // S buffer of the next tile and the parity that says it is free
+            bool ready = false;                    // both barriers of the next tile were seen complete already
             bool ok = true;
             long long x = x_begin;
             while (x < x_end && ok) {
@@ -578,9 +586,14 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 // it has completed, so the two softmax groups run half a period apart instead of in step
                 int rem = sg.slots_all - sg.t_first * kStageSlots;               // slots left in the unit from this tile on
                 for (int t = sg.t_first; t < sg.t_last; ++t, rem -= kStageSlots) {
-                    if (!wait_bar(ctrl, &ctrl->k_full[st], k_par, p.wait_limit) ||
-                        !wait_bar(ctrl, &ctrl->s_free[sb], s_par, p.wait_limit)) { timeout(p, ctrl, 21); ok = false; break; }
+                    if (!ready && !wait_bar2(ctrl, &ctrl->k_full[st], k_par, &ctrl->s_free[sb], s_par, p.wait_limit)) { timeout(p, ctrl, 21); ok = false; break; }
                     ptx::tc_fence_after();
+                    // the barriers of the tile after this one are polled now: the answers come back while this tile's
+                    // chain holds the thread up (in the steady state both are complete long before)
+                    const uint32_t st_n = (st + 1 == (uint32_t)KR) ? 0u : st + 1, k_par_n = k_par ^ (st_n == 0 ? 1u : 0u);
+                    const uint32_t sb_n = (sb + 1) & (kSBufs - 1), s_par_n = s_par ^ (sb_n == 0 ? 1u : 0u);
+                    const bool k_next = ptx::mbar_try_wait(&ctrl->k_full[st_n], k_par_n);
+                    const bool s_next = ptx::mbar_try_wait(&ctrl->s_free[sb_n], s_par_n);
                     if (rem > 0) {                                                     // (a pair's second tile may be empty)
                         const uint32_t idesc = rem >= kStageSlots ? idesc_full
                                              : (F8 ? umma_idesc_e4m3(kRows, rem * kSlotTok) : ptx::umma_idesc_bf16(kRows, rem * kSlotTok));
@@ -593,9 +606,9 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     }
                     ptx::umma_commit(&ctrl->s_full[sb]);
                     ptx::umma_commit(&ctrl->k_empty[st]);
-                    if (++st == (uint32_t)KR) { st = 0; k_par ^= 1; }
-                    sb = (sb + 1) & (kSBufs - 1);
-                    if (sb == 0) s_par ^= 1;
+                    st = st_n; k_par = k_par_n;
+                    sb = sb_n; s_par = s_par_n;
+                    ready = k_next && s_next;
                 }
                 x += sg.t_last - sg.t_first;
                 if (!ok) break;
@@ -608,6 +621,8 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             const uint32_t v_lo = ptx::umma_desc_lo(ptx::smem_u32(sV), 1024);             // MN-major: LBO = next 64-column atom
             const uint32_t idesc_pv = (F8 ? umma_idesc_e4m3(kRows, D) : ptx::umma_idesc_bf16(kRows, D)) | (1u << 16);   // B operand MN-major
             uint32_t it = 0;
+            int st = 0, sb = 0;                     // V ring stage and S / P buffer of the next tile, with their parities
+            uint32_t v_par = 0, p_par = 0;
             bool ok = true;
             long long x = x_begin;
             uint32_t seg = 0;
@@ -617,9 +632,8 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 if (seg > 0 && (!wait_bar(ctrl, &ctrl->o_free, (seg - 1) & 1, p.wait_limit))) { timeout(p, ctrl, 24); ok = false; break; }
                 ++seg;
                 for (int t = sg.t_first; t < sg.t_last; ++t, ++x, ++it) {
-                    const int st = it % VS, pb = it & 1, sb = it & (kSBufs - 1);
-                    if (!wait_bar(ctrl, &ctrl->p_full[sb], (it / kSBufs) & 1, p.wait_limit) ||
-                        !wait_bar(ctrl, &ctrl->v_full[st], (it / VS) & 1, p.wait_limit)) {
+                    const int pb = sb & 1;
+                    if (!wait_bar2(ctrl, &ctrl->p_full[sb], p_par, &ctrl->v_full[st], v_par, p.wait_limit)) {
                         timeout(p, ctrl, 23); ok = false; break;
                     }
                     ptx::tc_fence_after();
@@ -636,6 +650,9 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     ptx::umma_commit(&ctrl->v_empty[st]);
                     ptx::umma_commit(&ctrl->s_free[sb]);
                     ptx::umma_commit(&ctrl->pv_done[pb]);
+                    if (++st == VS) { st = 0; v_par ^= 1; }
+                    sb = (sb + 1) & (kSBufs - 1);
+                    if (sb == 0) p_par ^= 1;
                 }
             }
         }
