@@ -178,7 +178,9 @@ __device__ __forceinline__ void topk_list_insert(float* lv, int* li, int K, floa
 
 // kReduce: LM head (row reductions in the epilogue, optional spill).  !kReduce: plain GEMM C = W h^T for the layer
 // projections, split along K when there are fewer tiles than CTA pairs; the epilogue only stores fp32 partial sums.
-template <bool kReduce>
+// kFp8 / kTopk: e4m3 operands with per-row scales / Top-kappa lists in the epilogue, as separate instantiations so that
+// the plain bf16 head carries none of their registers and branches.
+template <bool kReduce, bool kFp8, bool kTopk>
 __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CUtensorMap& tm_h, const PairParams& p) {
     extern __shared__ uint8_t smem_raw[];
     // (the dynamic shared window starts at the same offset in both CTAs, so the aligned layout is the same too)
@@ -258,7 +260,7 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
     } else if (warp == 1) {
         if (lane == 0 && rank == 0) {
             // -------------------------------------------------------------- UMMA issuer (leader)
-            const uint32_t idesc = p.fp8 ? umma_idesc_e4m3(kPairV, p.chunk_rows) : ptx::umma_idesc_bf16(kPairV, p.chunk_rows);
+            const uint32_t idesc = kFp8 ? umma_idesc_e4m3(kPairV, p.chunk_rows) : ptx::umma_idesc_bf16(kPairV, p.chunk_rows);
             const uint32_t stage_u32 = ptx::smem_u32(stage_base);
             int s = 0, ab = 0;
             uint32_t ph = 0, aph = 0;
@@ -275,7 +277,7 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
                     ptx::tc_fence_after();
                     const uint32_t sa = stage_u32 + (uint32_t)(s * p.stage_bytes);
                     const uint32_t sb = sa + (uint32_t)p.a_bytes;
-                    if (p.fp8) {
+                    if constexpr (kFp8) {
 #pragma unroll
                         for (int k4 = 0; k4 < kBK / 16; ++k4)
                             umma_pair_f8(d_tmem, ptx::umma_desc_k_sw128(sa + k4 * 32), ptx::umma_desc_k_sw128(sb + k4 * 32), idesc,
@@ -323,7 +325,7 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
                 p.part_idx[pbase + row] = idx;
                 p.part_sum[pbase + row] = s;
                 // each warp's list is a partial list of its own: [4 * CTA + warp][row][topk]
-                for (int w = 0; w < 4 && p.topk > 0; ++w)
+                for (int w = 0; w < 4 && kTopk; ++w)
                     for (int i = 0; i < p.topk; ++i) {
                         const size_t at = (((size_t)blockIdx.x * 4 + w) * p.M + row) * p.topk + i;
                         p.part_topv[at] = tk_val[((size_t)w * p.chunk_rows + c) * p.topk + i];
@@ -344,7 +346,7 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
             for (int c = lane; c < kMaxChunkRows; c += 32) { my_max[c] = -INFINITY; my_idx[c] = 0x7fffffff; my_sum[c] = 0.f; }
             __syncwarp();
         }
-        if (kReduce && p.topk > 0) {
+        if constexpr (kReduce && kTopk) {
             for (int i = lane; i < p.chunk_rows * p.topk; i += 32) { my_tv[i] = -INFINITY; my_ti[i] = 0x7fffffff; }
             __syncwarp();
         }
@@ -361,7 +363,7 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
                 const bool valid = q * 32 + lane < p.rows_cta && vid < p.V;
                 const bool any_valid = __ballot_sync(0xffffffffu, valid) != 0;          // warp-uniform
                 const int n_rows = min(p.chunk_rows, p.M - rbase);                       // hidden rows of this chunk
-                const float sw = (p.fp8 && valid) ? p.w_scale[vid] : 1.f;                 // fp8: this lane's weight-row scale
+                const float sw = (kFp8 && valid) ? p.w_scale[vid] : 1.f;                 // fp8: this lane's weight-row scale
                 for (int cg = 0; cg < n_cg; ++cg) {
                     uint32_t r[32];
                     ptx::tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * p.acc_stride + cg * 32), r);
@@ -373,7 +375,7 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
                         // The 32 columns go through the reductions side by side (no branch inside, so the shuffle
                         // chains of different columns overlap); lane j keeps the result of column j.
                         float v[32], m[32];
-                        if (p.fp8) {
+                        if constexpr (kFp8) {
                             // logit = (sum of e4m3 products) * weight-row scale * hidden-row scale; lane j fetches column j's scale
                             const int cr = rbase + cg * 32 + lane;
                             const float sh = cr < p.M ? p.h_scale[cr] : 0.f;
@@ -388,7 +390,7 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
                             for (int j = 0; j < 32; ++j)
                                 if (j < ncol) dst[(size_t)j * p.V] = v[j];
                         }
-                        if (kReduce && p.topk > 0) {
+                        if constexpr (kReduce && kTopk) {
                             // lane j owns column j's list.  Its last entry is the bar: which lanes hold a logit of column j that
                             // passes it?  (Nothing to do but for a few tiles.)
                             const int K = p.topk;
@@ -483,11 +485,19 @@ __device__ __forceinline__ void pair_gemm_body(const CUtensorMap& tm_w, const CU
 
 __global__ void __launch_bounds__(kThreads, 2)
 lmhead_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_h, const PairParams p) {
-    pair_gemm_body<true>(tm_w, tm_h, p);
+    pair_gemm_body<true, false, false>(tm_w, tm_h, p);
+}
+__global__ void __launch_bounds__(kThreads, 2)
+lmhead_pair_topk_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_h, const PairParams p) {
+    pair_gemm_body<true, false, true>(tm_w, tm_h, p);
+}
+__global__ void __launch_bounds__(kThreads, 2)
+lmhead_pair_fp8_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_h, const PairParams p) {
+    pair_gemm_body<true, true, false>(tm_w, tm_h, p);
 }
 __global__ void __launch_bounds__(kThreads, 2)
 linear_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_h, const PairParams p) {
-    pair_gemm_body<false>(tm_w, tm_h, p);
+    pair_gemm_body<false, false, false>(tm_w, tm_h, p);
 }
 
 int next_pow2(int x) {
@@ -553,6 +563,8 @@ mirror_status pair_launch(mirror_ctx* ctx, bool reduce, const void* x, const voi
     const size_t smem = (size_t)p.stages * p.stage_bytes + kCtrlBytes + p.topk_bytes + 1024;
     if (!ctx->lm_pair_attr_set) {
         MIRROR_CUDA_OK(cudaFuncSetAttribute(lmhead_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+        MIRROR_CUDA_OK(cudaFuncSetAttribute(lmhead_pair_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+        MIRROR_CUDA_OK(cudaFuncSetAttribute(lmhead_pair_fp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
         MIRROR_CUDA_OK(cudaFuncSetAttribute(linear_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
         ctx->lm_pair_attr_set = true;
     }
@@ -570,7 +582,9 @@ mirror_status pair_launch(mirror_ctx* ctx, bool reduce, const void* x, const voi
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    MIRROR_CUDA_OK(cudaLaunchKernelEx(&cfg, reduce ? lmhead_pair_kernel : linear_pair_kernel, tm_w, tm_h, p));
+    if (p.fp8 && (p.topk > 0 || !reduce)) return MIRROR_ERR_UNSUPPORTED;
+    auto kern = !reduce ? linear_pair_kernel : p.fp8 ? lmhead_pair_fp8_kernel : p.topk > 0 ? lmhead_pair_topk_kernel : lmhead_pair_kernel;
+    MIRROR_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, tm_w, tm_h, p));
     ctx->launches += 1;
     MIRROR_CUDA_OK(cudaGetLastError());
     return MIRROR_OK;
