@@ -393,6 +393,15 @@ mirror_status mirror_target_forward(mirror_ctx* ctx, const mirror_target* t, con
                                     const void* x, void* q_out, void* k_new_out, void* v_new_out, void* attn_out,
                                     void* x_out, void* hidden_out, void* scratch, size_t scratch_bytes, void* stream);
 
+/* mirror_verify_step over an e4m3 KV cache: the attention is mirror_attn_verify_fp8's (kv, k_new_fp8, v_new_fp8, the
+ * scales and q_scale as there; head dimension 128), everything behind it (attn_out in bf16, LM head, acceptance) is
+ * unchanged. */
+mirror_status mirror_verify_step_fp8(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const void* q,
+                                     const void* k_new_fp8, const void* v_new_fp8, const float* k_scale,
+                                     const float* v_scale, float q_scale, const void* hidden, const void* W,
+                                     const mirror_accept_in* acc, const mirror_accept_out* out, void* attn_out,
+                                     int32_t* argmax_out, void* stream);
+
 /* mirror_verify_step for callers whose step inputs live in HOST memory (pinned for the copies to be asynchronous):
  *   h_q bf16 [L, B, n, Hq, d], h_k_new / h_v_new bf16 [L, B, n, Hkv, d], h_tokens int32 [B, n]: HOST inputs of this step
  *   d_q, d_k_new, d_v_new: DEVICE staging buffers of the same shapes, and tree->tokens (device, written here);

@@ -27,7 +27,7 @@ EXPORTS = [
     "mirror_device_status", "mirror_launch_count", "mirror_status_str", "mirror_set_stage_events",
     "mirror_lmhead_reduce_noalloc", "mirror_lmhead_noalloc_status", "mirror_quantize_rows_fp8", "mirror_lmhead_reduce_fp8", "mirror_early_exit_tap", "mirror_overlap_mass", "mirror_kv_commit",
     "mirror_linear_scratch_bytes", "mirror_linear", "mirror_rmsnorm", "mirror_target_scratch_bytes", "mirror_target_forward", "mirror_trie_build", "mirror_verify_step_host", "mirror_embed_rows",
-    "mirror_attn_verify_fp8", "mirror_kv_scales_fp8", "mirror_kv_quantize_fp8", "mirror_kv_commit_fp8",
+    "mirror_attn_verify_fp8", "mirror_kv_scales_fp8", "mirror_kv_quantize_fp8", "mirror_kv_commit_fp8", "mirror_verify_step_fp8",
 ]
 
 
@@ -516,6 +516,22 @@ class Mirror:
                                            C.byref(acc), C.byref(o), _ptr(attn_out, torch.bfloat16, "attn_out"),
                                            _ptr(argmax_out, torch.int32, "argmax_out"), _stream(stream)),
                "mirror_verify_step")
+        return out
+
+    def mirror_verify_step_fp8(self, kv: KV, tree: Tree, q, k_new8, v_new8, k_scale, v_scale, q_scale: float, hidden, W,
+                               acc: AcceptIn, attn_out, out: Optional[AcceptResult] = None, argmax_out=None, stream=None) -> AcceptResult:
+        """mirror_verify_step over an e4m3 cache (kv from kv_fp8; k_new8 / v_new8 uint8 codes under the cache's scales)."""
+        if out is None:
+            out = AcceptResult(tree.batch, tree.gamma, self.device)
+        self.ensure_workspace(tree, kv, {ACCEPT_GREEDY: WS_STEP_GREEDY, ACCEPT_SPEC_TREE: WS_STEP_TREE}.get(acc.mode, WS_STEP_SPEC))
+        o = out.struct()
+        _check(self.lib.mirror_verify_step_fp8(self._ctx, C.byref(kv), C.byref(tree), _ptr(q, torch.bfloat16, "q"),
+                                               _ptr(k_new8, torch.uint8, "k_new8"), _ptr(v_new8, torch.uint8, "v_new8"),
+                                               _ptr(k_scale, torch.float32, "k_scale"), _ptr(v_scale, torch.float32, "v_scale"),
+                                               C.c_float(q_scale), _ptr(hidden, torch.bfloat16, "hidden"), _ptr(W, torch.bfloat16, "W"),
+                                               C.byref(acc), C.byref(o), _ptr(attn_out, torch.bfloat16, "attn_out"),
+                                               _ptr(argmax_out, torch.int32, "argmax_out"), _stream(stream)),
+               "mirror_verify_step_fp8")
         return out
 
     def set_stage_events(self, events):

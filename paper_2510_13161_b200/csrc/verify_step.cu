@@ -77,7 +77,9 @@ mirror_status ensure_copy_stream(mirror_ctx* ctx) {
 
 mirror_status verify_step_impl(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const void* q, const void* k_new,
                                const void* v_new, const void* hidden, const void* W, const mirror_accept_in* acc,
-                               const mirror_accept_out* out, void* attn_out, int32_t* argmax_out, void* stream, const HostIO* io) {
+                               const mirror_accept_out* out, void* attn_out, int32_t* argmax_out, void* stream, const HostIO* io,
+                               const MirrorAttnFp8* f8 = nullptr) {
+    if (f8 && io) return MIRROR_ERR_UNSUPPORTED;          // (the host-buffer step takes the bf16 cache)
     if (!ctx || !kv || !tree || !q || !k_new || !v_new || !W || !acc || !out || !attn_out || !tree->tokens) return MIRROR_ERR_ARG;
     if (!out->n_accepted || !out->best_branch || !out->n_emitted || !out->emitted || !out->accepted_nodes ||
         !out->decide_row || !out->reuse_slot)
@@ -117,7 +119,7 @@ mirror_status verify_step_impl(mirror_ctx* ctx, const mirror_kv* kv, const mirro
     const bool ev = ctx->stage_ev_on && !io;
     if (ev) MIRROR_CUDA_OK(cudaEventRecord(ctx->stage_ev[0], s));
     if (!io) {
-        st = mirror_attn_launch(ctx, kv, tree, ti, q, k_new, v_new, attn_out, nullptr, (float*)(ws + L.attn_partial), s);
+        st = mirror_attn_launch(ctx, kv, tree, ti, q, k_new, v_new, attn_out, nullptr, (float*)(ws + L.attn_partial), s, f8);
         if (st != MIRROR_OK) return st;
     } else {
         // Host inputs.  The layers' attention problems are independent of one another and the LM head reads only the
@@ -198,6 +200,17 @@ extern "C" mirror_status mirror_verify_step(mirror_ctx* ctx, const mirror_kv* kv
                                             const void* W, const mirror_accept_in* acc, const mirror_accept_out* out,
                                             void* attn_out, int32_t* argmax_out, void* stream) {
     return verify_step_impl(ctx, kv, tree, q, k_new, v_new, hidden, W, acc, out, attn_out, argmax_out, stream, nullptr);
+}
+
+extern "C" mirror_status mirror_verify_step_fp8(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const void* q,
+                                                const void* k_new_fp8, const void* v_new_fp8, const float* k_scale,
+                                                const float* v_scale, float q_scale, const void* hidden, const void* W,
+                                                const mirror_accept_in* acc, const mirror_accept_out* out, void* attn_out,
+                                                int32_t* argmax_out, void* stream) {
+    if (!k_scale || !v_scale || !(q_scale > 0.f)) return MIRROR_ERR_ARG;
+    if (ctx && ctx->desc.head_dim != 128) return MIRROR_ERR_UNSUPPORTED;
+    const MirrorAttnFp8 f8 = {k_scale, v_scale, q_scale};
+    return verify_step_impl(ctx, kv, tree, q, k_new_fp8, v_new_fp8, hidden, W, acc, out, attn_out, argmax_out, stream, nullptr, &f8);
 }
 
 extern "C" mirror_status mirror_verify_step_host(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const void* h_q,

@@ -195,3 +195,34 @@ def test_commit_of_codes_then_attention_on_the_committed_cache():
                                        anc, 1.0 / np.sqrt(d))
         got = f32(out[l]).astype(np.float64)
         assert np.abs(got - ref).max() <= FP8_REL * np.abs(ref).max(), l
+
+
+def test_fused_step_over_the_8_bit_cache_equals_its_parts():
+    """mirror_verify_step_fp8 = mirror_attn_verify_fp8 -> LM head -> acceptance: the same attention bits and the same
+    decision as the three calls made one after the other (each part has its own parity test against the oracle)."""
+    from paper_2510_13161_b200 import binding
+    cfg = small(batch=3, layers=2, prefix_lo=40, prefix_hi=400, kappa=3, gamma=3, vocab=1500)
+    x = I.gen_verify_inputs(cfg, 12, "cuda")
+    m = make_mirror(cfg)
+    ks, vs, k8, v8, kn8, vn8 = quantise(m, x)
+    kv = m.kv_fp8(k8, v8, x.page_table, x.prefix_len)
+    tree = m.tree(x.tokens, cfg.kappa, cfg.gamma, parent=x.parent)
+    q_scale = float(np.float32(float(x.q.float().abs().max())) / np.float32(448.0))
+    acc = m.accept_in(binding.ACCEPT_GREEDY, True)
+    attn_fused = torch.empty_like(x.q)
+    argmax_fused = torch.empty(cfg.batch * cfg.n_nodes, dtype=torch.int32, device="cuda")
+    res = m.mirror_verify_step_fp8(kv, tree, x.q, kn8, vn8, ks, vs, q_scale, None, x.W, acc, attn_fused, argmax_out=argmax_fused)
+    torch.cuda.synchronize()
+    assert m.device_status() == (0, 0)
+    attn = m.mirror_attn_verify_fp8(kv, tree, x.q, kn8, vn8, ks, vs, q_scale)
+    rows = attn[-1].reshape(cfg.batch * cfg.n_nodes, cfg.hidden)
+    lm = m.mirror_lmhead_reduce(rows, x.W)
+    acc2 = m.accept_in(binding.ACCEPT_GREEDY, True, target_argmax=lm["argmax"])
+    res2 = m.mirror_accept_select(tree, acc2)
+    torch.cuda.synchronize()
+    assert m.device_status() == (0, 0)
+    assert torch.equal(attn_fused, attn)
+    assert torch.equal(argmax_fused, lm["argmax"])
+    a, b = res.cpu(), res2.cpu()
+    for f in ("n_accepted", "best_branch", "n_emitted", "emitted", "accepted_nodes", "decide_row"):
+        assert np.array_equal(a[f], b[f]), f
