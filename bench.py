@@ -50,6 +50,9 @@ def parse_args():
                          "skeleton line (gloo when there is no CUDA device): checks the launch path without a GPU")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-low-precision", action="store_true",
+                    help="leave out stages.lmhead_fp8 and stages.attn_fp8 (the opt-in e4m3 modes timed beside the bf16 path, "
+                         "outside the timed region; on by default when the head dimension is 128)")
     ap.add_argument("--accept-mode", default=None, choices=["greedy", "spec_sampling", "spec_tree"],
                     help="override the workload's acceptance rule")
     ap.add_argument("--skip-e2e", action="store_true",
@@ -679,9 +682,10 @@ def run_mirror(args):
         stages["attn_per_layer_ms"] = attn_per_layer(m, x, w.tree, cfg)
     if args.overlap_draft:
         stages["overlap_draft"] = overlap_draft_stage(w.step, w.stream)
-    if args.lmhead_fp8:
+    low_precision = not args.no_low_precision and cfg.head_dim == 128 and cfg.hidden % 128 == 0 and args.layers is None
+    if args.lmhead_fp8 or low_precision:
         stages["lmhead_fp8"] = lmhead_fp8_stage(m, x, cfg, peaks["hbm_gbs"])
-    if args.attn_fp8:
+    if args.attn_fp8 or low_precision:
         stages["attn_fp8"] = attn_fp8_stage(m, x, w.tree, w.kv, cfg, peaks, work)
     if args.target_layers > 0:
         stages["target_forward"] = target_forward_stage(m, x, w.tree, w.kv, cfg, min(args.target_layers, cfg.layers), args.intermediate,
