@@ -392,6 +392,17 @@ mirror_status mirror_target_scratch_bytes(const mirror_ctx* ctx, const mirror_tr
 mirror_status mirror_target_forward(mirror_ctx* ctx, const mirror_target* t, const mirror_kv* kv, const mirror_tree* tree,
                                     const void* x, void* q_out, void* k_new_out, void* v_new_out, void* attn_out,
                                     void* x_out, void* hidden_out, void* scratch, size_t scratch_bytes, void* stream);
+/* The same layers over an e4m3 KV cache (see mirror_attn_verify_fp8; head dimension 128).  kv holds codes; k_scale and
+ * v_scale are the cache's scales (device fp32 [n_layers, Hkv]); h_q_scale is a HOST array [n_layers] with one Q scale
+ * per layer (e.g. from a calibration pass: max|q| / 448 with some head room; larger values saturate).  Every layer's new
+ * K/V rows are written as bf16 (k_new_out, v_new_out, as before) and as codes under the cache's scales (k_new8_out,
+ * v_new8_out: bytes [n_layers, B, n, Hkv, d], what mirror_kv_commit_fp8 appends); the layer's attention reads the codes.
+ * Two more small kernels per layer. */
+mirror_status mirror_target_forward_fp8(mirror_ctx* ctx, const mirror_target* t, const mirror_kv* kv, const mirror_tree* tree,
+                                        const void* x, const float* k_scale, const float* v_scale, const float* h_q_scale,
+                                        void* q_out, void* k_new_out, void* v_new_out, void* k_new8_out, void* v_new8_out,
+                                        void* attn_out, void* x_out, void* hidden_out, void* scratch, size_t scratch_bytes,
+                                        void* stream);
 
 /* mirror_verify_step over an e4m3 KV cache: the attention is mirror_attn_verify_fp8's (kv, k_new_fp8, v_new_fp8, the
  * scales and q_scale as there; head dimension 128), everything behind it (attn_out in bf16, LM head, acceptance) is

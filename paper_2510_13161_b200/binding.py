@@ -27,7 +27,7 @@ EXPORTS = [
     "mirror_device_status", "mirror_launch_count", "mirror_status_str", "mirror_set_stage_events",
     "mirror_lmhead_reduce_noalloc", "mirror_lmhead_noalloc_status", "mirror_quantize_rows_fp8", "mirror_lmhead_reduce_fp8", "mirror_early_exit_tap", "mirror_overlap_mass", "mirror_kv_commit",
     "mirror_linear_scratch_bytes", "mirror_linear", "mirror_rmsnorm", "mirror_target_scratch_bytes", "mirror_target_forward", "mirror_trie_build", "mirror_verify_step_host", "mirror_embed_rows",
-    "mirror_attn_verify_fp8", "mirror_kv_scales_fp8", "mirror_kv_quantize_fp8", "mirror_kv_commit_fp8", "mirror_verify_step_fp8",
+    "mirror_attn_verify_fp8", "mirror_kv_scales_fp8", "mirror_kv_quantize_fp8", "mirror_kv_commit_fp8", "mirror_verify_step_fp8", "mirror_target_forward_fp8",
 ]
 
 
@@ -468,6 +468,29 @@ class Mirror:
                                               _ptr(out["q"]), _ptr(out["k_new"]), _ptr(out["v_new"]), _ptr(out["attn_out"]),
                                               _ptr(out["x_out"]), _ptr(out["hidden"]), _ptr(scratch), C.c_size_t(scratch.numel()),
                                               _stream(stream)), "mirror_target_forward")
+        out["_scratch"] = scratch
+        return out
+
+    def mirror_target_forward_fp8(self, target: Target, kv: KV, tree: Tree, x: torch.Tensor, k_scale, v_scale, q_scales,
+                                  scratch: Optional[torch.Tensor] = None, stream=None) -> dict:
+        """mirror_target_forward over an e4m3 cache (kv from kv_fp8); q_scales: one host float per layer.  Also returns
+        k_new8 / v_new8: the new rows' codes under the cache's scales."""
+        L, B, n = target.n_layers, tree.batch, tree.n_nodes
+        Hq, Hkv, d = self.desc.n_q_heads, self.desc.n_kv_heads, self.desc.head_dim
+        if scratch is None:
+            scratch = self.target_scratch(tree, target)
+        e = lambda *shape: torch.empty(shape, dtype=torch.bfloat16, device=self.device)
+        e8 = lambda *shape: torch.empty(shape, dtype=torch.uint8, device=self.device)
+        out = dict(q=e(L, B, n, Hq, d), k_new=e(L, B, n, Hkv, d), v_new=e(L, B, n, Hkv, d), k_new8=e8(L, B, n, Hkv, d),
+                   v_new8=e8(L, B, n, Hkv, d), attn_out=e(L, B, n, Hq, d), x_out=torch.empty_like(x), hidden=torch.empty_like(x))
+        qs = (C.c_float * L)(*[float(v) for v in q_scales])
+        self.ensure_workspace(tree, kv, WS_ATTN)
+        _check(self.lib.mirror_target_forward_fp8(self._ctx, C.byref(target), C.byref(kv), C.byref(tree), _ptr(x, torch.bfloat16, "x"),
+                                                  _ptr(k_scale, torch.float32, "k_scale"), _ptr(v_scale, torch.float32, "v_scale"), qs,
+                                                  _ptr(out["q"]), _ptr(out["k_new"]), _ptr(out["v_new"]), _ptr(out["k_new8"]),
+                                                  _ptr(out["v_new8"]), _ptr(out["attn_out"]), _ptr(out["x_out"]), _ptr(out["hidden"]),
+                                                  _ptr(scratch), C.c_size_t(scratch.numel()), _stream(stream)),
+               "mirror_target_forward_fp8")
         out["_scratch"] = scratch
         return out
 

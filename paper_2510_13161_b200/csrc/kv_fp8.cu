@@ -126,6 +126,19 @@ extern "C" mirror_status mirror_kv_scales_fp8(mirror_ctx* ctx, const void* x, in
     return MIRROR_OK;
 }
 
+mirror_status mirror_kv_quantize_launch(mirror_ctx* ctx, const void* x, int n_layers, int64_t layer_stride, int64_t layer_elems,
+                                       int inner, const float* scale, void* out_fp8, cudaStream_t stream) {
+    KvQuantParams p;
+    mirror_status st = fill(ctx, &p, x, n_layers, layer_stride, layer_elems, inner, const_cast<float*>(scale));
+    if (st != MIRROR_OK) return st;
+    if (!out_fp8 || ((uintptr_t)out_fp8 & 7)) return MIRROR_ERR_ARG;
+    p.out = (uint8_t*)out_fp8;
+    MIRROR_CUDA_OK(mirror_launch_pdl(kv_quantize_kernel, dim3(grid_for(ctx, p)), dim3(256), 0, stream, p));
+    MIRROR_CUDA_OK(cudaGetLastError());
+    ctx->launches += 1;
+    return MIRROR_OK;
+}
+
 extern "C" mirror_status mirror_kv_quantize_fp8(mirror_ctx* ctx, const void* x, int n_layers, int64_t layer_stride,
                                                 int64_t layer_elems, int inner, const float* scale, void* out_fp8, void* stream) {
     KvQuantParams p;

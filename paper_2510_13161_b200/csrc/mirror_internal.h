@@ -116,6 +116,10 @@ struct MirrorAttnFp8 {
     const float* v_scale;
     float q_scale;
 };
+// e4m3 codes of a bf16 K or V tensor under given scales (see mirror_kv_quantize_fp8), launched with programmatic stream
+// serialization.
+mirror_status mirror_kv_quantize_launch(mirror_ctx* ctx, const void* x, int n_layers, int64_t layer_stride, int64_t layer_elems,
+                                       int inner, const float* scale, void* out_fp8, cudaStream_t stream);
 mirror_status mirror_attn_launch(mirror_ctx* ctx, const mirror_kv* kv, const mirror_tree* tree, const MirrorTreeInfo& ti,
                                  const void* q, const void* k_new, const void* v_new, void* out, float* lse_out,
                                  float* partial_ws, cudaStream_t stream, const MirrorAttnFp8* f8 = nullptr);

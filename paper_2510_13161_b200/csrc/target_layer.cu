@@ -289,9 +289,19 @@ extern "C" mirror_status mirror_target_scratch_bytes(const mirror_ctx* ctx, cons
     return MIRROR_OK;
 }
 
-extern "C" mirror_status mirror_target_forward(mirror_ctx* ctx, const mirror_target* t, const mirror_kv* kv, const mirror_tree* tree,
-                                               const void* x, void* q_out, void* k_new_out, void* v_new_out, void* attn_out,
-                                               void* x_out, void* hidden_out, void* scratch, size_t scratch_bytes, void* stream) {
+namespace {
+// e4m3 cache: the cache's scales, one Q scale per layer (host), and where the codes of the new K/V rows go
+struct TargetFp8 {
+    const float* k_scale;      // device [L, Hkv]
+    const float* v_scale;
+    const float* q_scale;      // HOST [L]
+    void* k_new8_out;          // device [L, B, n, Hkv, d] bytes
+    void* v_new8_out;
+};
+
+mirror_status target_forward_impl(mirror_ctx* ctx, const mirror_target* t, const mirror_kv* kv, const mirror_tree* tree,
+                                  const void* x, void* q_out, void* k_new_out, void* v_new_out, void* attn_out,
+                                  void* x_out, void* hidden_out, void* scratch, size_t scratch_bytes, void* stream, const TargetFp8* f8) {
     if (!ctx || !t || !kv || !tree || !x || !q_out || !k_new_out || !v_new_out || !attn_out || !x_out || !hidden_out || !scratch)
         return MIRROR_ERR_ARG;
     if (!t->layers || !t->norm_final || t->n_layers <= 0 || t->n_layers > kv->num_layers) return MIRROR_ERR_ARG;
@@ -353,10 +363,24 @@ extern "C" mirror_status mirror_target_forward(mirror_ctx* ctx, const mirror_tar
         ctx->launches += 1;
         // attention of this layer over its slab of the cache
         mirror_kv kv_l = *kv;
-        kv_l.k_pool = (const __nv_bfloat16*)kv->k_pool + (size_t)l * kv->layer_stride;
-        kv_l.v_pool = (const __nv_bfloat16*)kv->v_pool + (size_t)l * kv->layer_stride;
         kv_l.num_layers = 1;
-        st = mirror_attn_launch(ctx, &kv_l, tree, ti, q_l, k_l, v_l, a_l, nullptr, (float*)((uint8_t*)ctx->ws + L.attn_partial), s);
+        if (!f8) {
+            kv_l.k_pool = (const __nv_bfloat16*)kv->k_pool + (size_t)l * kv->layer_stride;
+            kv_l.v_pool = (const __nv_bfloat16*)kv->v_pool + (size_t)l * kv->layer_stride;
+            st = mirror_attn_launch(ctx, &kv_l, tree, ti, q_l, k_l, v_l, a_l, nullptr, (float*)((uint8_t*)ctx->ws + L.attn_partial), s);
+        } else {
+            // the layer's new K/V rows as codes under the cache's scales (the caller commits them), then the 8-bit attention
+            uint8_t* k8_l = (uint8_t*)f8->k_new8_out + (size_t)l * kv_elems;
+            uint8_t* v8_l = (uint8_t*)f8->v_new8_out + (size_t)l * kv_elems;
+            st = mirror_kv_quantize_launch(ctx, k_l, 1, (int64_t)kv_elems, (int64_t)kv_elems, d, f8->k_scale + (size_t)l * Hkv, k8_l, s);
+            if (st != MIRROR_OK) return st;
+            st = mirror_kv_quantize_launch(ctx, v_l, 1, (int64_t)kv_elems, (int64_t)kv_elems, d, f8->v_scale + (size_t)l * Hkv, v8_l, s);
+            if (st != MIRROR_OK) return st;
+            kv_l.k_pool = (const uint8_t*)kv->k_pool + (size_t)l * kv->layer_stride;
+            kv_l.v_pool = (const uint8_t*)kv->v_pool + (size_t)l * kv->layer_stride;
+            const MirrorAttnFp8 a8 = {f8->k_scale + (size_t)l * Hkv, f8->v_scale + (size_t)l * Hkv, f8->q_scale[l]};
+            st = mirror_attn_launch(ctx, &kv_l, tree, ti, q_l, k8_l, v8_l, a_l, nullptr, (float*)((uint8_t*)ctx->ws + L.attn_partial), s, &a8);
+        }
         if (st != MIRROR_OK) return st;
         // output projection + residual + the MLP's norm
         st = mirror_linear_partial_launch(ctx, a_l, M, w.w_o, H, Hq * d, partial, sc.partial_bytes, s, &slices);
@@ -381,4 +405,26 @@ extern "C" mirror_status mirror_target_forward(mirror_ctx* ctx, const mirror_tar
     }
     MIRROR_CUDA_OK(cudaGetLastError());
     return MIRROR_OK;
+}
+
+}  // namespace
+
+extern "C" mirror_status mirror_target_forward(mirror_ctx* ctx, const mirror_target* t, const mirror_kv* kv, const mirror_tree* tree,
+                                               const void* x, void* q_out, void* k_new_out, void* v_new_out, void* attn_out,
+                                               void* x_out, void* hidden_out, void* scratch, size_t scratch_bytes, void* stream) {
+    return target_forward_impl(ctx, t, kv, tree, x, q_out, k_new_out, v_new_out, attn_out, x_out, hidden_out, scratch, scratch_bytes,
+                               stream, nullptr);
+}
+
+extern "C" mirror_status mirror_target_forward_fp8(mirror_ctx* ctx, const mirror_target* t, const mirror_kv* kv, const mirror_tree* tree,
+                                                   const void* x, const float* k_scale, const float* v_scale, const float* h_q_scale,
+                                                   void* q_out, void* k_new_out, void* v_new_out, void* k_new8_out, void* v_new8_out,
+                                                   void* attn_out, void* x_out, void* hidden_out, void* scratch, size_t scratch_bytes,
+                                                   void* stream) {
+    if (!k_scale || !v_scale || !h_q_scale || !k_new8_out || !v_new8_out) return MIRROR_ERR_ARG;
+    if (ctx && ctx->desc.head_dim != 128) return MIRROR_ERR_UNSUPPORTED;
+    if (t) for (int l = 0; l < t->n_layers; ++l) if (!(h_q_scale[l] > 0.f)) return MIRROR_ERR_ARG;
+    const TargetFp8 f8 = {k_scale, v_scale, h_q_scale, k_new8_out, v_new8_out};
+    return target_forward_impl(ctx, t, kv, tree, x, q_out, k_new_out, v_new_out, attn_out, x_out, hidden_out, scratch, scratch_bytes,
+                               stream, &f8);
 }
