@@ -585,8 +585,9 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 // one tile (a ring stage of four slots) per issue: each S buffer is scored as soon as the P V that read
                 // it has completed, so the two softmax groups run half a period apart instead of in step
                 int rem = sg.slots_all - sg.t_first * kStageSlots;               // slots left in the unit from this tile on
-                for (int t = sg.t_first; t < sg.t_last; ++t, rem -= kStageSlots) {
-                    if (!ready && !wait_bar2(ctrl, &ctrl->k_full[st], k_par, &ctrl->s_free[sb], s_par, p.wait_limit)) { timeout(p, ctrl, 21); ok = false; break; }
+                // (parts hold whole pairs of tiles: two tiles per loop iteration halve what the loop itself costs this thread)
+                auto issue_tile = [&](int rem_t) -> bool {
+                    if (!ready && !wait_bar2(ctrl, &ctrl->k_full[st], k_par, &ctrl->s_free[sb], s_par, p.wait_limit)) return false;
                     ptx::tc_fence_after();
                     // the barriers of the tile after this one are polled now: the answers come back while this tile's
                     // chain holds the thread up (in the steady state both are complete long before)
@@ -594,9 +595,9 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     const uint32_t sb_n = (sb + 1) & (kSBufs - 1), s_par_n = s_par ^ (sb_n == 0 ? 1u : 0u);
                     const bool k_next = ptx::mbar_try_wait(&ctrl->k_full[st_n], k_par_n);
                     const bool s_next = ptx::mbar_try_wait(&ctrl->s_free[sb_n], s_par_n);
-                    if (rem > 0) {                                                     // (a pair's second tile may be empty)
-                        const uint32_t idesc = rem >= kStageSlots ? idesc_full
-                                             : (F8 ? umma_idesc_e4m3(kRows, rem * kSlotTok) : ptx::umma_idesc_bf16(kRows, rem * kSlotTok));
+                    if (rem_t > 0) {                                                   // (a pair's second tile may be empty)
+                        const uint32_t idesc = rem_t >= kStageSlots ? idesc_full
+                                             : (F8 ? umma_idesc_e4m3(kRows, rem_t * kSlotTok) : ptx::umma_idesc_bf16(kRows, rem_t * kSlotTok));
                         const uint32_t kb = k_lo + st * (uint32_t)(C::kStageBytes >> 4);
                         const uint32_t d = tmem_base + sb * (uint32_t)kTileTok;
 #pragma unroll
@@ -609,6 +610,10 @@ attn_verify_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     st = st_n; k_par = k_par_n;
                     sb = sb_n; s_par = s_par_n;
                     ready = k_next && s_next;
+                    return true;
+                };
+                for (int t = sg.t_first; t < sg.t_last; t += 2, rem -= 2 * kStageSlots) {
+                    if (!issue_tile(rem) || !issue_tile(rem - kStageSlots)) { timeout(p, ctrl, 21); ok = false; break; }
                 }
                 x += sg.t_last - sg.t_first;
                 if (!ok) break;
